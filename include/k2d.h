@@ -1,0 +1,190 @@
+/*
+ * k2d.h -- C ABI of the batched 2D rigid-body environment step (sm_100a CUDA library).
+ *
+ * The library advances thousands of independent fixed-size scenes of the Kinetix / Jax2D
+ * kind (arxiv 2410.23208): circles, convex polygons of 3 or 4 vertices, revolute joints with
+ * motors, thrusters.  One call of k2d_step runs, for every scene and for n_steps steps, the
+ * paper's Algorithm 1 (gravity, collision manifolds, motors, thrusters, warm start, a fixed
+ * number of sequential-impulse solver iterations over joints then contacts, Euler step),
+ * followed by Kinetix's touch reward / termination ("Reward" paragraph: green touches blue
+ * = +1 and done, green touches red = -1 and done) and the auto-reset.
+ *
+ * Conventions
+ *  - C99 types only; every function returns int: 0 = K2D_OK, negative = error, and on error
+ *    no device work has been enqueued.
+ *  - The CALLER owns every device buffer and the CUDA stream.  The library owns only the host
+ *    handle; it never allocates or frees device memory.  k2d_step and k2d_obs are asynchronous
+ *    on the stream given in the config; k2d_create, k2d_reset, k2d_get_state, k2d_set_state
+ *    and k2d_status synchronise that stream.
+ *  - "dev_" pointers are device memory, 16-byte aligned; "host_" pointers are host memory.
+ *  - Shape index inside a scene: polygons 0 .. n_polygons-1, then circles.  Pair order (used by
+ *    the solver and by the accumulated-impulse slots): polygon-polygon pairs (i<j,
+ *    lexicographic), polygon-circle pairs (polygon major), circle-circle pairs (i<j);
+ *    polygon-polygon pairs own two manifold slots, the others one.
+ *  - All floating point is IEEE binary32.  Results are bit-reproducible from run to run and
+ *    do not depend on n_envs, on lanes_per_scene or on how many steps are fused per call.
+ */
+#ifndef K2D_H_
+#define K2D_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define K2D_OK 0
+#define K2D_ERR_NULL (-1)          /* a required pointer is null                         */
+#define K2D_ERR_CONFIG (-2)        /* a config field is out of range                     */
+#define K2D_ERR_ALIGN (-3)         /* a device pointer is not 16-byte aligned            */
+#define K2D_ERR_LEVEL (-4)         /* level data invalid (non-finite, bad index, ...)    */
+#define K2D_ERR_STEPS (-5)         /* n_steps < 1 or > max_fused_steps                   */
+#define K2D_ERR_CUDA (-6)          /* a CUDA runtime call failed                         */
+#define K2D_ERR_ARG (-7)           /* another argument is invalid                        */
+
+#define K2D_MAX_POLYGONS 12
+#define K2D_MAX_CIRCLES 4
+#define K2D_MAX_SHAPES 16
+#define K2D_MAX_JOINTS 6
+#define K2D_MAX_THRUSTERS 2
+
+#define K2D_RESET_NONE 0           /* keep stepping; flags are reported every step they hold */
+#define K2D_RESET_SAME_LEVEL 1     /* on done, the env restarts on its own level              */
+#define K2D_RESET_POOL 2           /* on done, level = hash(seed, env, episode) mod n_levels  */
+
+#define K2D_ROLE_NONE 0
+#define K2D_ROLE_GREEN 1
+#define K2D_ROLE_BLUE 2
+#define K2D_ROLE_RED 3
+
+#define K2D_STATUS_NONFINITE 1     /* per-env status bit: the state became non-finite         */
+
+/* Engine and environment parameters.  The paper leaves dt, the iteration count and the
+ * correction coefficients open; the defaults written by k2d_default_config are dt = 1/60,
+ * gravity_y = -9.81, 8 solver iterations, contact_alpha = joint_alpha = 6 /s,
+ * contact_beta = joint_beta = 0.1, slop = 0.005 m, restitution_threshold = 1 m/s,
+ * face_tol = 1e-3 m, motor_rho = 1, aabb_margin = 0.01 m, warm starting on. */
+typedef struct k2d_config {
+    int32_t n_envs;                /* >= 1                                                      */
+    int32_t n_polygons;            /* 1 .. K2D_MAX_POLYGONS                                     */
+    int32_t n_circles;             /* 0 .. K2D_MAX_CIRCLES                                      */
+    int32_t n_joints;              /* 0 .. K2D_MAX_JOINTS                                       */
+    int32_t n_thrusters;           /* 0 .. K2D_MAX_THRUSTERS                                    */
+    int32_t n_actions;             /* >= 1; bindings index into the action row                  */
+    int32_t n_levels;              /* >= 1, size of the level pool                              */
+    int32_t solver_iters;          /* >= 0                                                      */
+    int32_t warm_start;            /* 0 / 1 (paper: "Impulse Accumulation and Warm Starting")   */
+    int32_t auto_reset;            /* K2D_RESET_*                                               */
+    int32_t max_episode_steps;     /* 0 = no horizon; else done when step_count reaches it      */
+    int32_t max_fused_steps;       /* largest n_steps k2d_step accepts                          */
+    float dt, gravity_y;
+    float contact_alpha;           /* velocity correction: bias = alpha * max(pen - slop, 0)    */
+    float contact_beta;            /* positional correction: beta * max(pen - slop, 0)          */
+    float slop;
+    float restitution_threshold;   /* approach speed below which a contact does not bounce      */
+    float face_tol;                /* polygon-polygon reference face hysteresis                 */
+    float joint_alpha, joint_beta; /* the same two corrections for the joint's point constraint */
+    float motor_rho;               /* rho of the motor law j = p tanh((wa - wb - s A) rho)      */
+    float aabb_margin;             /* bounding boxes further apart than this skip narrowphase   */
+    uint64_t seed;                 /* seed of the K2D_RESET_POOL hash                           */
+    int64_t env_offset;            /* global index of env 0 (sharding over several GPUs)        */
+    int32_t device;                /* CUDA device ordinal                                       */
+    int32_t lanes_per_scene;       /* 0 = library default; else 8, 16 or 32                     */
+    void *cuda_stream;             /* cudaStream_t of the caller (NULL = default stream)        */
+} k2d_config;
+
+/* One scene as the caller describes it.  Entities beyond the config's counts are ignored.
+ * Polygon vertices are in the body frame, counter-clockwise, with the centroid at the origin
+ * (|centroid| <= 1e-3 x extent is enforced).  Mass and inertia follow from density (uniform
+ * lamina); is_static shapes have infinite mass (paper: fixated shapes). */
+typedef struct k2d_level {
+    float poly_verts[K2D_MAX_POLYGONS][4][2];
+    int32_t poly_nverts[K2D_MAX_POLYGONS];           /* 3 or 4                                  */
+    float circle_radius[K2D_MAX_CIRCLES];
+    float pos[K2D_MAX_SHAPES][2], angle[K2D_MAX_SHAPES];      /* initial pose                   */
+    float vel[K2D_MAX_SHAPES][2], angvel[K2D_MAX_SHAPES];     /* initial velocity               */
+    float density[K2D_MAX_SHAPES], friction[K2D_MAX_SHAPES], restitution[K2D_MAX_SHAPES];
+    int32_t is_static[K2D_MAX_SHAPES], role[K2D_MAX_SHAPES], active[K2D_MAX_SHAPES];
+    int32_t joint_a[K2D_MAX_JOINTS], joint_b[K2D_MAX_JOINTS]; /* shape indices                  */
+    float joint_anchor_a[K2D_MAX_JOINTS][2], joint_anchor_b[K2D_MAX_JOINTS][2]; /* body frame   */
+    float motor_speed[K2D_MAX_JOINTS], motor_power[K2D_MAX_JOINTS];
+    int32_t motor_binding[K2D_MAX_JOINTS], joint_active[K2D_MAX_JOINTS];
+    int32_t thr_shape[K2D_MAX_THRUSTERS];
+    float thr_pos[K2D_MAX_THRUSTERS][2], thr_rot[K2D_MAX_THRUSTERS], thr_power[K2D_MAX_THRUSTERS];
+    int32_t thr_binding[K2D_MAX_THRUSTERS], thr_active[K2D_MAX_THRUSTERS];
+} k2d_level;
+
+typedef struct k2d_state k2d_state;   /* opaque host handle */
+
+/* Fills *cfg with the defaults listed above for the given scene dimensions (n_actions =
+ * n_joints + n_thrusters, n_levels = n_envs, auto_reset = NONE, max_fused_steps = 64). */
+int k2d_default_config(k2d_config *cfg, int32_t n_envs, int32_t n_polygons, int32_t n_circles,
+                       int32_t n_joints, int32_t n_thrusters);
+
+/* Bytes of device memory the caller must provide for the state buffer (scene state of all
+ * envs, a small control block, and the solver's overflow scratch) and for the level pool.
+ * Host-only; 0 on an invalid config. */
+size_t k2d_state_bytes(const k2d_config *cfg);
+size_t k2d_level_pool_bytes(const k2d_config *cfg);
+
+/* Validates the config and the n_levels host levels, derives mass properties and the pair
+ * collision mask (joined shapes do not collide: paper, "Joints"), uploads the level pool to
+ * dev_level_pool_buf, resets every env (env i on level i mod n_levels) and returns a handle.
+ * Both buffers stay owned by the caller and must outlive the handle. */
+int k2d_create(const k2d_config *cfg, void *dev_state_buf, void *dev_level_pool_buf,
+               const k2d_level *host_levels, k2d_state **out);
+
+/* Restarts every env: env i on level host_level_ids[i] (NULL: i mod n_levels), episode 0,
+ * zero accumulated impulses, zero counters. */
+int k2d_reset(k2d_state *s, const int32_t *host_level_ids);
+
+/* Advances every env by n_steps steps (paper, Algorithm 1 + "Reward").  dev_actions is
+ * [n_steps][n_envs][n_actions] floats, one row consumed per step (motor actions are clipped
+ * to [-1, 1], thruster actions to [0, 1]: paper, "Action Space"); dev_reward [n_steps][n_envs]
+ * floats in {-1, 0, +1}; dev_done [n_steps][n_envs] bytes.  1 <= n_steps <= max_fused_steps.
+ * The whole call is one kernel launch; scene state stays on chip between the fused steps. */
+int k2d_step(k2d_state *s, const float *dev_actions, int32_t n_steps, float *dev_reward, uint8_t *dev_done);
+
+/* Symbolic per-entity observation (paper, tables "Information provided for shapes / joints /
+ * thrusters"): dev_obs is [n_envs][k2d_obs_floats] floats; per env the shape rows (29 floats
+ * each), two rows per joint (11 + n_actions floats each), one row per thruster (6 floats). */
+int k2d_obs(k2d_state *s, float *dev_obs);
+int k2d_obs_floats(const k2d_config *cfg);
+
+/* Canonical host copy of the dynamic state, for checkpoints and comparisons: per env
+ * k2d_canonical_words 4-byte words: pos[N][2], angle[N], vel[N][2], angvel[N] (floats),
+ * acc[n_slots][2] (accumulated normal, tangent impulse per manifold slot), jacc[n_joints][2],
+ * then int32 step_count, episode_count, level_id, status.  set_state followed by k2d_step
+ * continues bit-identically. */
+int k2d_canonical_words(const k2d_config *cfg);
+int k2d_get_state(k2d_state *s, void *host_canonical);
+int k2d_set_state(k2d_state *s, const void *host_canonical);
+
+/* host_counts[4] (int64): non-finite events, auto-resets, active manifolds summed over
+ * env-steps, env-steps, all since the last k2d_reset. */
+int k2d_status(k2d_state *s, int64_t *host_counts);
+
+/* Host only, no device needed: validates one level against the config and returns the constants
+ * the library derives from it: inv_mass[N], inv_inertia[N] (floats; 0 for fixated or absent shapes)
+ * and collide[n_pairs] (bytes; pair order as above).  Any output pointer may be NULL. */
+int k2d_level_info(const k2d_config *cfg, const k2d_level *host_level, float *host_inv_mass, float *host_inv_inertia,
+                   uint8_t *host_collide);
+
+/* Debug aid: when dev_trace is non-null every later step also writes the manifolds of each
+ * env's latest step to dev_trace[n_envs][n_slots][6] = px, py, nx, ny, penetration, active
+ * (slots indexed in the library's internal size class, see k2d_trace_slots). */
+int k2d_set_trace(k2d_state *s, float *dev_trace);
+int k2d_trace_slots(const k2d_state *s);
+
+/* Evaluates the library's own sine/cosine and tanh routines on n device floats (the step
+ * uses these instead of libm so that results are reproducible bit for bit). */
+int k2d_eval_sincos_tanh(const float *dev_x, int32_t n, float *dev_cos, float *dev_sin, float *dev_tanh, void *cuda_stream);
+
+const char *k2d_error_string(int code);
+void k2d_destroy(k2d_state *s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* K2D_H_ */

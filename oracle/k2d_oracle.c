@@ -674,8 +674,8 @@ static void step_env(ref_sim *S, int e, const real *act, real *out_reward, uint8
      * applied once; a loses j_r / I_a and b gains j_r / I_b so that wa - wb is
      * driven towards s A.  A = action clipped to [-1, 1]. */
     for (int j = 0; j < J; ++j) {
-        if (!S->lv_joint_active[l * J + j]) continue;
         int a = S->lv_joint_a[l * J + j], b = S->lv_joint_b[l * J + j];
+        if (!(S->lv_joint_active[l * J + j] && active[a] && active[b] && (inv_mass[a] + inv_mass[b] > RC(0)))) continue;
         real A = rmax(rmin(act[S->lv_motor_binding[l * J + j]], RC(1)), RC(-1));
         real d = angvel[a] - angvel[b];
         real arg = R_FMA(-S->lv_motor_speed[l * J + j], A, d) * cf->motor_rho;

@@ -1,0 +1,211 @@
+"""GPU parity: the CUDA library (through its C ABI) against the CPU oracle on the same seeded inputs."""
+import numpy as np
+import pytest
+
+from oracle import k2d_ref
+from paper_2410_23208_b200 import k2d, scenes
+from tests import parity
+from tests.parity import POS_TOL_1, TOL_16, VEL_TOL_1
+
+pytestmark = pytest.mark.gpu
+
+
+def _check_tolerances(err, after_steps):
+    if after_steps <= 1:
+        assert max(err["pos"], err["angle"]) <= POS_TOL_1 and max(err["vel"], err["angvel"]) <= VEL_TOL_1, err
+    else:
+        assert max(err["pos"], err["angle"], err["vel"], err["angvel"]) <= TOL_16, err
+    for k in parity.META_KEYS:
+        assert err[k] == 0.0, err
+
+
+def test_sincos_tanh_bit_equal_to_the_oracle():
+    import torch
+    rng = np.random.default_rng(0)
+    x = np.concatenate([rng.uniform(-50, 50, 100000), rng.uniform(-0.01, 0.01, 5000), rng.uniform(-2000, 2000, 20000),
+                        [0.0, -0.0, 10.0, -10.0, 1e5, np.inf, -np.inf, 3e7]]).astype(np.float32)
+    c, s, t = k2d.eval_sincos_tanh(torch.from_numpy(x).cuda())
+    rc, rs = k2d_ref.sincos(x)
+    rt = k2d_ref.tanh(x)
+    for got, want in ((c, rc), (s, rs), (t, rt)):
+        assert np.array_equal(got.cpu().numpy().view(np.uint32), want.view(np.uint32))
+
+
+@pytest.mark.parametrize("size,n_envs,seed", [("S", 16, 1000), ("M", 48, 1002), ("L", 80, 1003)])
+def test_step_parity_1_16_and_100_steps(size, n_envs, seed):
+    lv = scenes.make_levels(size, n_envs, seed, static_prob=0.1)
+    env, ref = parity.make_pair(lv, n_envs, max_fused_steps=128)
+    act = scenes.make_actions(100, n_envs, env.n_actions, seed)
+    (r, d), (rr, dr) = parity.step_both(env, ref, act[:1])
+    err, exact = parity.errors(env, ref)
+    _check_tolerances(err, 1)
+    assert np.array_equal(r, rr) and np.array_equal(d, dr)
+    (r, d), (rr, dr) = parity.step_both(env, ref, act[1:16])
+    err, exact16 = parity.errors(env, ref)
+    _check_tolerances(err, 16)
+    assert np.array_equal(r, rr) and np.array_equal(d, dr)          # reward / done bit-exact over 16 steps
+    (r, d), (rr, dr) = parity.step_both(env, ref, act[16:])
+    err, exact100 = parity.errors(env, ref)
+    _check_tolerances(err, 100)
+    assert np.array_equal(r, rr) and np.array_equal(d, dr)
+    # the arithmetic contract makes the two bit-identical, which is what keeps the flags exact
+    assert exact and exact16 and exact100
+    assert np.array_equal(env.status(), ref.counters)
+
+
+@pytest.mark.parametrize("lanes", [8, 16, 32])
+def test_lanes_per_scene_does_not_change_results(lanes):
+    lv = scenes.make_levels("L", 40, 7, static_prob=0.1, triangle_prob=0.2)
+    env, ref = parity.make_pair(lv, 40, lanes_per_scene=lanes)
+    act = scenes.make_actions(48, 40, env.n_actions, 7)
+    (r, d), (rr, dr) = parity.step_both(env, ref, act, chunk=16)
+    err, exact = parity.errors(env, ref)
+    assert exact, err
+    assert np.array_equal(r, rr) and np.array_equal(d, dr)
+
+
+def test_fusing_steps_does_not_change_results():
+    import torch
+    lv = scenes.make_levels("M", 32, 3, static_prob=0.1)
+    a = k2d.Env(lv, 32)
+    b = k2d.Env(lv, 32)
+    act = torch.from_numpy(scenes.make_actions(32, 32, a.n_actions, 3)).cuda()
+    ra, da = a.step(act)
+    rb, db = zip(*[b.step(act[s:s + 1]) for s in range(32)])
+    sa, sb = a.get_state(), b.get_state()
+    for k in sa:
+        assert np.array_equal(sa[k].view(np.uint32) if sa[k].dtype == np.float32 else sa[k],
+                              sb[k].view(np.uint32) if sb[k].dtype == np.float32 else sb[k]), k
+    assert torch.equal(ra, torch.cat(rb)) and torch.equal(da, torch.cat(db))
+
+
+def test_checkpoint_resume_is_bit_identical():
+    import torch
+    lv = scenes.make_levels("L", 24, 5, static_prob=0.1)
+    act = torch.from_numpy(scenes.make_actions(32, 24, 8, 5)).cuda()
+    a = k2d.Env(lv, 24, auto_reset=1, max_episode_steps=20)
+    a.step(act[:16])
+    saved = a.get_state()
+    a.step(act[16:])
+    b = k2d.Env(lv, 24, auto_reset=1, max_episode_steps=20)
+    b.set_state(saved)
+    again = b.get_state()
+    for k in saved:
+        assert np.array_equal(saved[k], again[k], equal_nan=True), k
+    b.step(act[16:])
+    sa, sb = a.get_state(), b.get_state()
+    for k in sa:
+        assert np.array_equal(sa[k], sb[k], equal_nan=True), k
+
+
+@pytest.mark.parametrize("mode,horizon", [(1, 12), (2, 9)])
+def test_auto_reset_modes_match_the_oracle(mode, horizon):
+    lv = scenes.make_levels("S", 32, 21, static_prob=0.1)
+    env, ref = parity.make_pair(lv, 64, auto_reset=mode, max_episode_steps=horizon, seed=99, env_offset=1000)
+    act = scenes.make_actions(60, 64, env.n_actions, 21)
+    (r, d), (rr, dr) = parity.step_both(env, ref, act, chunk=20)
+    err, exact = parity.errors(env, ref)
+    assert exact, err
+    assert np.array_equal(r, rr) and np.array_equal(d, dr) and d.sum() >= 64 * (60 // horizon)
+    assert np.array_equal(env.status(), ref.counters)
+    if mode == 2:
+        assert len(set(ref.level_id.tolist())) > 8
+
+
+def test_touch_rewards_match_on_crowded_scenes():
+    # no horizon: every done comes from a green-blue or green-red touch
+    lv = scenes.make_levels("L", 64, 33, static_prob=0.1)
+    env, ref = parity.make_pair(lv, 256, auto_reset=2, seed=5)
+    act = scenes.make_actions(64, 256, env.n_actions, 33)
+    (r, d), (rr, dr) = parity.step_both(env, ref, act, chunk=32)
+    assert np.array_equal(r, rr) and np.array_equal(d, dr)
+    assert (r > 0).sum() > 0 and (r < 0).sum() > 0
+    err, exact = parity.errors(env, ref)
+    assert exact, err
+
+
+def test_custom_dimensions_and_inactive_entities():
+    dims = scenes.SceneDims(3, 3, 1, 1)
+    lv = scenes.make_levels(dims, 16, 41, static_prob=0.2, triangle_prob=0.4)
+    lv["active"][2, 2] = 0
+    lv["joint_active"][3, 0] = 0
+    lv["thr_active"][4, 0] = 0
+    env, ref = parity.make_pair(lv, 16)
+    act = scenes.make_actions(40, 16, env.n_actions, 41)
+    (r, d), (rr, dr) = parity.step_both(env, ref, act, chunk=8)
+    err, exact = parity.errors(env, ref)
+    assert exact, err
+    assert np.array_equal(r, rr) and np.array_equal(d, dr)
+
+
+def test_more_active_pairs_than_lanes_and_than_shared_memory_records():
+    # every shape of an L scene dropped on the same spot: far more than 32 touching pairs, so the
+    # records beyond the shared-memory capacity go through the global-memory scratch
+    lv = scenes.make_levels("L", 6, 51)
+    rng = np.random.default_rng(51)
+    lv["pos"][:, 1:, 0] = rng.uniform(-0.3, 0.3, (6, 15)).astype(np.float32)
+    lv["pos"][:, 1:, 1] = rng.uniform(0.8, 1.4, (6, 15)).astype(np.float32)
+    lv["joint_active"][:] = 0
+    env, ref = parity.make_pair(lv, 6)
+    trace = env.enable_trace()
+    act = scenes.make_actions(12, 6, env.n_actions, 51)
+    (r, d), (rr, dr) = parity.step_both(env, ref, act[:1])
+    active_pairs = (ref.manifold[:, :, 5] > 0).sum(1)
+    assert active_pairs.max() > 48
+    assert np.array_equal(trace.cpu().numpy()[:, :, 5], ref.manifold[:, :, 5])
+    err, exact = parity.errors(env, ref)
+    assert exact, err
+    (r, d), (rr, dr) = parity.step_both(env, ref, act[1:], chunk=4)
+    err, exact = parity.errors(env, ref)
+    assert exact, err
+    assert np.array_equal(r, rr) and np.array_equal(d, dr)
+
+
+def test_manifold_trace_matches_the_oracle():
+    lv = scenes.make_levels("L", 32, 61, static_prob=0.1, triangle_prob=0.3)
+    env, ref = parity.make_pair(lv, 32)
+    trace = env.enable_trace()
+    act = scenes.make_actions(30, 32, env.n_actions, 61)
+    parity.step_both(env, ref, act)
+    t = trace.cpu().numpy()
+    m = ref.manifold
+    assert np.array_equal(t[:, :, 5], m[:, :, 5]) and m[:, :, 5].sum() > 100
+    on = m[:, :, 5] > 0
+    assert np.array_equal(t[on].view(np.uint32), m[on].view(np.uint32))
+
+
+@pytest.mark.parametrize("size", ["S", "M", "L"])
+def test_observation_parity(size):
+    lv = scenes.make_levels(size, 32, 71, static_prob=0.1, triangle_prob=0.3)
+    lv["thr_active"][1, 0] = 0
+    lv["joint_active"][2, 0] = 0
+    env, ref = parity.make_pair(lv, 32)
+    act = scenes.make_actions(10, 32, env.n_actions, 71)
+    parity.step_both(env, ref, act)
+    got = env.obs().cpu().numpy()
+    want = ref.obs()
+    assert got.shape == want.shape == (32, {"S": 235, "M": 333, "L": 704}[size])
+    assert np.max(np.abs(got - want)) <= 1e-5
+    assert np.array_equal(got.view(np.uint32), want.view(np.uint32))
+
+
+def test_non_finite_state_is_flagged_not_propagated():
+    lv = scenes.make_levels("S", 8, 81)
+    env, ref = parity.make_pair(lv, 8)
+    st = env.get_state()
+    st["vel"][3, 2, 0] = np.inf
+    env.set_state(st)
+    ref.vel[3, 2, 0] = np.inf
+    act = scenes.make_actions(3, 8, env.n_actions, 81)
+    (r, d), (rr, dr) = parity.step_both(env, ref, act)
+    assert np.array_equal(r, rr) and np.array_equal(d, dr) and d[:, 3].all()
+    assert env.get_state()["status"][3] == 1 and np.array_equal(env.status(), ref.counters)
+
+
+def test_step_rejects_too_many_fused_steps():
+    import torch
+    lv = scenes.make_levels("S", 4, 1)
+    env = k2d.Env(lv, 4, max_fused_steps=4)
+    act = torch.zeros((5, 4, env.n_actions), device="cuda")
+    with pytest.raises(k2d.K2DError):
+        env.step(act)
