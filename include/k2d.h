@@ -161,8 +161,9 @@ int k2d_canonical_words(const k2d_config *cfg);
 int k2d_get_state(k2d_state *s, void *host_canonical);
 int k2d_set_state(k2d_state *s, const void *host_canonical);
 
-/* host_counts[4] (int64): non-finite events, auto-resets, active manifolds summed over
- * env-steps, env-steps, all since the last k2d_reset. */
+/* host_counts[8] (int64), all since the last k2d_reset: non-finite events, auto-resets, active
+ * manifolds summed over env-steps, env-steps, pairs that passed the bounding-box test (polygon-
+ * polygon, polygon-circle, circle-circle), pairs with at least one active manifold. */
 int k2d_status(k2d_state *s, int64_t *host_counts);
 
 /* Host only, no device needed: validates one level against the config and returns the constants

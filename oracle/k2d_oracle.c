@@ -104,7 +104,8 @@ typedef struct {
     int32_t *step_count, *episode_count, *level_id, *status;
     /* per env trace of the last step's manifolds: [E][n_slots][6] = px,py,nx,ny,pen,active */
     real *manifold;
-    int64_t *counters; /* [4]: nonfinite events, resets, active manifolds (sum), env-steps */
+    int64_t *counters; /* [8]: nonfinite events, resets, active manifolds (sum), env-steps,
+                          pairs past the box test: polygon-polygon, polygon-circle, circle-circle, pairs with an active manifold */
 } ref_sim;
 
 typedef struct {
@@ -513,7 +514,7 @@ ref_sim *k2d_ref_create(const ref_config *cfg, const ref_levels *L) {
     NEW_ARR(S->step_count, E, int32_t); NEW_ARR(S->episode_count, E, int32_t);
     NEW_ARR(S->level_id, E, int32_t); NEW_ARR(S->status, E, int32_t);
     NEW_ARR(S->manifold, (size_t)E * S->n_slots * 6, real);
-    NEW_ARR(S->counters, 4, int64_t);
+    NEW_ARR(S->counters, 8, int64_t);
     for (int e = 0; e < E; ++e) { reset_env(S, e, e % nl); S->episode_count[e] = 0; }
     return S;
 }
@@ -537,7 +538,7 @@ void k2d_ref_reset(ref_sim *S, const int32_t *ids) {
         reset_env(S, e, ids ? ids[e] : e % S->cfg.n_levels);
         S->episode_count[e] = 0;
     }
-    memset(S->counters, 0, sizeof(int64_t) * 4);
+    memset(S->counters, 0, sizeof(int64_t) * 8);
 }
 
 void k2d_ref_views(ref_sim *S, ref_views *V) {
@@ -655,11 +656,13 @@ static void step_env(ref_sim *S, int e, const real *act, real *out_reward, uint8
         }
         vec2 pa = { pos[2 * a], pos[2 * a + 1] }, pb = { pos[2 * b], pos[2 * b + 1] };
         int any;
+        cnt[4 + (b < P ? 0 : (a < P ? 1 : 2))] += 1;
         if (b < P) { manifold_pp(&W[a], &W[b], cf->face_tol, &man[s]); any = man[s].active || man[s + 1].active; }
         else if (a < P) { manifold_pc(&W[a], pb, S->lv_radius[l * C + (b - P)], &man[s]); any = man[s].active; }
         else { manifold_cc(pa, S->lv_radius[l * C + (a - P)], pb, S->lv_radius[l * C + (b - P)], &man[s]); any = man[s].active; }
         /* touch flags of this step: an active manifold between green and blue / green and red */
         if (any) {
+            cnt[7] += 1;
             int r1 = role[a], r2 = role[b];
             if ((r1 == ROLE_GREEN && r2 == ROLE_BLUE) || (r1 == ROLE_BLUE && r2 == ROLE_GREEN)) touch_gb = 1;
             if ((r1 == ROLE_GREEN && r2 == ROLE_RED) || (r1 == ROLE_RED && r2 == ROLE_GREEN)) touch_gr = 1;
@@ -877,7 +880,7 @@ static void step_range(ref_sim *S, int e0, int e1, const real *actions, int n_st
             step_env(S, e, actions + ((size_t)s * E + e) * A, reward + (size_t)s * E + e, done + (size_t)s * E + e, cnt);
 }
 
-typedef struct { ref_sim *S; int e0, e1, n_steps; const real *actions; real *reward; uint8_t *done; int64_t cnt[4]; } job;
+typedef struct { ref_sim *S; int e0, e1, n_steps; const real *actions; real *reward; uint8_t *done; int64_t cnt[8]; } job;
 static void *job_main(void *arg) {
     job *j = (job *)arg;
     step_range(j->S, j->e0, j->e1, j->actions, j->n_steps, j->reward, j->done, j->cnt);
@@ -897,7 +900,7 @@ void k2d_ref_step(ref_sim *S, const real *actions, int n_steps, real *reward, ui
     }
     for (int t = 0; t < n_threads; ++t) {
         if (n_threads > 1) pthread_join(th[t], NULL);
-        for (int k = 0; k < 4; ++k) S->counters[k] += jobs[t].cnt[k];
+        for (int k = 0; k < 8; ++k) S->counters[k] += jobs[t].cnt[k];
     }
     free(jobs); free(th);
 }

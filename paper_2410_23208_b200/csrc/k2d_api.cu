@@ -16,7 +16,7 @@ using ClassM = SizeClass<6, 3, 2, 2, 36>;
 using ClassL = SizeClass<12, 4, 6, 2, 32>;
 
 constexpr int kMaxSlots = 8192;      // resident scene groups a launch may use (bounds the overflow scratch)
-constexpr size_t kCtrlBytes = 256;   // control block at the start of the state buffer: 4 x uint64 counters
+constexpr size_t kCtrlBytes = 256;   // control block at the start of the state buffer: 8 x uint64 counters
 
 // run-time view of a size class
 struct ClassInfo {
@@ -495,7 +495,7 @@ int k2d_status(k2d_state *s, int64_t *host_counts) {
     if (!s || !host_counts) return K2D_ERR_NULL;
     CUDA_OK(cudaSetDevice(s->cfg.device));
     CUDA_OK(cudaStreamSynchronize(s->stream));
-    CUDA_OK(cudaMemcpy(host_counts, s->dev_counters, 4 * sizeof(int64_t), cudaMemcpyDeviceToHost));
+    CUDA_OK(cudaMemcpy(host_counts, s->dev_counters, 8 * sizeof(int64_t), cudaMemcpyDeviceToHost));
     return K2D_OK;
 }
 

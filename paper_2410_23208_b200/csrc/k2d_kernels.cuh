@@ -544,7 +544,7 @@ struct Scene {
     }
 
     // ---- one environment step.  Returns through meta[]: step_count, episode_count, level_id, status, nwarm
-    __device__ void step(int e, int s, int (&meta)[5], unsigned long long (&cnt)[4]) {
+    __device__ void step(int e, int s, int (&meta)[5], unsigned (&cnt)[8]) {
         const uint32_t *lv = prm.levels + (size_t)meta[2] * SC::LV_WORDS;
         // frozen env: reports done, nothing else
         if (meta[3] & 1) {
@@ -682,6 +682,7 @@ struct Scene {
             }
         }
         g.sync();
+        if (lane == 0) { cnt[4] += ns_pp; cnt[5] += ns_pc - ns_pp; cnt[6] += nsurv - ns_pc; }
 
         // narrowphase + contact pre-step: survivors of one kind at a time, records in pair order
         int nrec = 0;
@@ -828,6 +829,7 @@ struct Scene {
             nman += __popc(am);
         }
         meta[4] = nrec;
+        if (lane == 0) cnt[7] += nrec;
 
         // reward, termination, counters, auto-reset
         meta[0] += 1;
@@ -879,7 +881,7 @@ struct Scene {
             widx()[p] = (uint8_t)k;
         }
         g.sync();
-        unsigned long long cnt[4] = { 0ULL, 0ULL, 0ULL, 0ULL };
+        unsigned cnt[8] = { 0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u };
         for (int s = 0; s < prm.n_steps; ++s) { step(e, s, meta, cnt); g.sync(); }
         // write back
         for (int i = lane; i < 6 * SC::N; i += G) st[SC::ST_BODY + i] = smu[SC::BX + i];
@@ -892,14 +894,13 @@ struct Scene {
 #pragma unroll
             for (int q = 0; q < 5; ++q) st[SC::ST_WARM + kWarmWords * k + q] = warm_ld(q, k);
         }
-        // counters: lane 0 holds event counts, every lane holds its share of the manifold count
-        unsigned long long nm = cnt[2];
+        // counters: lane 0 holds the event counts, every lane holds its share of the manifold count
+        unsigned nm = cnt[2];
         for (int off = G / 2; off > 0; off >>= 1) nm += __shfl_down_sync(g.mask, nm, off, G);
         if (lane == 0) {
-            if (cnt[0]) atomicAdd(prm.counters + 0, cnt[0]);
-            if (cnt[1]) atomicAdd(prm.counters + 1, cnt[1]);
-            if (nm) atomicAdd(prm.counters + 2, nm);
-            if (cnt[3]) atomicAdd(prm.counters + 3, cnt[3]);
+            cnt[2] = nm;
+#pragma unroll
+            for (int q = 0; q < 8; ++q) if (cnt[q]) atomicAdd(prm.counters + q, (unsigned long long)cnt[q]);
         }
     }
 };

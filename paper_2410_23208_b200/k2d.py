@@ -215,7 +215,7 @@ class Env:
         _check(self.lib.k2d_set_state(self._h, raw.ctypes.data), "k2d_set_state")
 
     def status(self) -> np.ndarray:
-        out = np.zeros(4, np.int64)
+        out = np.zeros(8, np.int64)
         _check(self.lib.k2d_status(self._h, out.ctypes.data), "k2d_status")
         return out
 
