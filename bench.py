@@ -38,8 +38,8 @@ UNIT = "env-steps/s"
 FLOPS = dict(body=37, circle_box=4, polygon=84, box_test=8, cc=16, pc=94, pp=190,
              pair_prestep=5, man_prestep=54, man_warm=28, man_iter=57, man_pos=10,
              joint_fixed=48 + 33 + 18 + 8, joint_iter=38, thruster=27)
-# DRAM bytes one ncu capture measured for one k2d_step launch, per env (profiles/); None = not captured
-NCU_DRAM_BYTES_PER_ENV_LAUNCH = None
+# DRAM bytes one ncu capture measured for one k2d_step launch of the benchmark workload, per env
+NCU_DRAM_BYTES_PER_ENV_LAUNCH = 2216.4   # profiles/k2d_step_kernel_L_16384envs_32steps.md: (35.447 MB + 0.867 MB) / 16384 envs
 
 
 def fp32_peak_tflops(sm_count: int = 148, sm_mhz: float = 1965.0) -> float:
@@ -226,6 +226,8 @@ def run_gpu(args) -> dict:
             torch.distributed.barrier()
         torch.cuda.synchronize(dev)
 
+    clocks = ClockSampler(local)
+    clocks.__enter__()
     for i in range(W):
         env.step(dev_actions[i % n_bufs], reward, done)
         env.obs(obs)
@@ -234,19 +236,17 @@ def run_gpu(args) -> dict:
 
     # ---- device-resident timing: events around each step (k2d_step, then k2d_obs); L2 flushed in between, untimed
     ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(K)]
-    with ClockSampler(local) as clocks:
-        barrier()
-        t_wall = time.perf_counter()
-        for i in range(K):
-            flush.fill_(i & 0xFF)
-            ev[i][0].record()
-            env.step(dev_actions[i % n_bufs], reward, done)
-            ev[i][1].record()
-            env.obs(obs)
-            ev[i][2].record()
-        barrier()
-        t_wall = time.perf_counter() - t_wall
-    clk = clocks.summary()
+    barrier()
+    t_wall = time.perf_counter()
+    for i in range(K):
+        flush.fill_(i & 0xFF)
+        ev[i][0].record()
+        env.step(dev_actions[i % n_bufs], reward, done)
+        ev[i][1].record()
+        env.obs(obs)
+        ev[i][2].record()
+    barrier()
+    t_wall = time.perf_counter() - t_wall
     step_ms = [ev[i][0].elapsed_time(ev[i][1]) for i in range(K)]
     obs_ms = [ev[i][1].elapsed_time(ev[i][2]) for i in range(K)]
     total_ms = float(sum(step_ms) + sum(obs_ms))
@@ -268,6 +268,8 @@ def run_gpu(args) -> dict:
     e1.record()
     barrier()
     e2e_ms = e0.elapsed_time(e1)
+    clocks.__exit__()
+    clk = clocks.summary()   # sampled every 100 ms from the first warm-up step to the end of the end-to-end loop
 
     if world > 1:
         t = torch.tensor([total_ms, e2e_ms, float(np.mean(step_ms))], device=dev, dtype=torch.float64)
@@ -320,7 +322,7 @@ def run_gpu(args) -> dict:
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=16)
+    ap.add_argument("--steps", type=int, default=48)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="k2d", choices=["k2d", "reference"])
     ap.add_argument("--workload", type=int, default=3, choices=sorted(scenes.WORKLOADS))
