@@ -42,6 +42,7 @@ extern "C" {
 #define K2D_ERR_STEPS (-5)         /* n_steps < 1 or > max_fused_steps                   */
 #define K2D_ERR_CUDA (-6)          /* a CUDA runtime call failed                         */
 #define K2D_ERR_ARG (-7)           /* another argument is invalid                        */
+#define K2D_ERR_LIMIT (-8)         /* a size is beyond a limit built into the library    */
 
 #define K2D_MAX_POLYGONS 12
 #define K2D_MAX_CIRCLES 4
@@ -145,6 +146,26 @@ int k2d_reset(k2d_state *s, const int32_t *host_level_ids);
  * floats in {-1, 0, +1}; dev_done [n_steps][n_envs] bytes.  1 <= n_steps <= max_fused_steps.
  * The whole call is one kernel launch; scene state stays on chip between the fused steps. */
 int k2d_step(k2d_state *s, const float *dev_actions, int32_t n_steps, float *dev_reward, uint8_t *dev_done);
+
+/* The paper has no counterpart of this call; it exists for one kind of user of this library.
+ * k2d_step keeps the contact records of a crowded scene (more than 32 touching pairs) in the
+ * scratch tail of the state buffer, which the caller has to allocate.  Some callers cannot: a
+ * process whose device memory is one arena fixed at start-up, a plug-in handed a pre-sized
+ * buffer by its host, code running where cudaMalloc is forbidden (a real-time loop).  For them this variant does exactly what k2d_step does, with the same
+ * arguments and bit-identical results, but keeps those records in an array compiled into the
+ * library (K2D_STATIC_SCRATCH_MAX_ENVS x 10208 bytes, about 10 MB, resident on every GPU that
+ * loads the library until the process exits) and never touches the scratch tail.  It allocates
+ * and frees nothing, on the host side of CUDA or on the device.
+ *  - n_envs above K2D_STATIC_SCRATCH_MAX_ENVS is refused with K2D_ERR_LIMIT (and a line on
+ *    stderr); nothing is enqueued.
+ *  - The first call on each device looks up the array's device address (with that device made
+ *    current); make that first call before any stream capture begins.
+ *  - All handles and streams of a process share the one array per device.  Nothing in it has
+ *    to start at zero (every record is written before it is read), so calls one after another
+ *    need no clearing; calls that overlap on the GPU (two streams, two handles) race on it
+ *    and must be serialised by the caller. */
+#define K2D_STATIC_SCRATCH_MAX_ENVS 1024
+int k2d_step_static_scratch(k2d_state *s, const float *dev_actions, int32_t n_steps, float *dev_reward, uint8_t *dev_done);
 
 /* Symbolic per-entity observation (paper, tables "Information provided for shapes / joints /
  * thrusters"): dev_obs is [n_envs][k2d_obs_floats] floats; per env the shape rows (29 floats

@@ -3,6 +3,7 @@
 #include <cmath>
 #include <cstdio>
 #include <cstring>
+#include <mutex>
 #include <new>
 #include <vector>
 
@@ -540,6 +541,47 @@ int k2d_eval_sincos_tanh(const float *dev_x, int32_t n, float *dev_cos, float *d
     return K2D_OK;
 }
 
+// ---- k2d_step for callers that cannot provide the overflow scratch: it lives in the library image.
+// One array per device that loads the library, held until the process exits.
+static __device__ __align__(256) uint32_t k2d_static_scratch[(size_t)K2D_STATIC_SCRATCH_MAX_ENVS * ClassL::SCRATCH_WORDS];
+static std::mutex k2d_static_mutex;
+static uint32_t *k2d_static_ptr[64];     // device address of the array on each device, filled on first use
+
+int k2d_step_static_scratch(k2d_state *s, const float *dev_actions, int32_t n_steps, float *dev_reward, uint8_t *dev_done) {
+    if (!s || !dev_actions || !dev_reward || !dev_done) return K2D_ERR_NULL;
+    if (n_steps < 1 || n_steps > s->cfg.max_fused_steps) return K2D_ERR_STEPS;
+    if (((uintptr_t)dev_actions & 3) || ((uintptr_t)dev_reward & 3)) return K2D_ERR_ALIGN;
+    const k2d_config &c = s->cfg;
+    if (c.n_envs > K2D_STATIC_SCRATCH_MAX_ENVS || c.device >= 64) {
+        std::fprintf(stderr, "k2d_step_static_scratch: n_envs = %d is beyond the built-in scratch (at most %d envs); use k2d_step\n",
+                     c.n_envs, K2D_STATIC_SCRATCH_MAX_ENVS);
+        return K2D_ERR_LIMIT;
+    }
+    CUDA_OK(cudaSetDevice(c.device));
+    uint32_t *scratch = nullptr;
+    {
+        // In host code the array's name is only a handle; the kernel needs its address on this device.
+        std::lock_guard<std::mutex> lock(k2d_static_mutex);
+        if (!k2d_static_ptr[c.device]) {
+            void *p = nullptr;
+            CUDA_OK(cudaGetSymbolAddress(&p, k2d_static_scratch));
+            k2d_static_ptr[c.device] = (uint32_t *)p;
+        }
+        scratch = k2d_static_ptr[c.device];
+    }
+    StepParams prm{};
+    prm.state = s->dev_env; prm.levels = s->dev_levels; prm.actions = dev_actions; prm.reward = dev_reward; prm.done = dev_done;
+    prm.counters = s->dev_counters; prm.scratch = scratch; prm.trace = s->dev_trace;
+    prm.n_envs = c.n_envs; prm.n_steps = n_steps; prm.n_actions = c.n_actions; prm.n_levels = c.n_levels;
+    prm.solver_iters = c.solver_iters; prm.warm_start = c.warm_start; prm.auto_reset = c.auto_reset; prm.max_episode_steps = c.max_episode_steps;
+    prm.dt = c.dt; prm.gdt = c.gravity_y * c.dt; prm.contact_alpha = c.contact_alpha; prm.contact_beta = c.contact_beta; prm.slop = c.slop;
+    prm.rest_thr = c.restitution_threshold; prm.face_tol = c.face_tol; prm.joint_alpha = c.joint_alpha; prm.joint_beta = c.joint_beta;
+    prm.motor_rho = c.motor_rho; prm.aabb_margin = c.aabb_margin; prm.seed = c.seed; prm.env_offset = c.env_offset;
+    // the launch of k2d_step never uses more scene groups than envs, so n_envs bounds the scratch slots it touches
+    CUDA_OK(K2D_DISPATCH(launch_step, s, s, prm));
+    return K2D_OK;
+}
+
 const char *k2d_error_string(int code) {
     switch (code) {
         case K2D_OK: return "ok";
@@ -550,6 +592,7 @@ const char *k2d_error_string(int code) {
         case K2D_ERR_STEPS: return "n_steps out of range";
         case K2D_ERR_CUDA: return "CUDA runtime error";
         case K2D_ERR_ARG: return "invalid argument";
+        case K2D_ERR_LIMIT: return "size beyond a built-in limit";
         default: return "unknown error";
     }
 }

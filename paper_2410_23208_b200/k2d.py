@@ -17,7 +17,8 @@ MAX_POLYGONS, MAX_CIRCLES, MAX_SHAPES, MAX_JOINTS, MAX_THRUSTERS = 12, 4, 16, 6,
 RESET_NONE, RESET_SAME_LEVEL, RESET_POOL = 0, 1, 2
 
 EXPORTS = (
-    "k2d_default_config", "k2d_state_bytes", "k2d_level_pool_bytes", "k2d_create", "k2d_reset", "k2d_step", "k2d_obs",
+    "k2d_default_config", "k2d_state_bytes", "k2d_level_pool_bytes", "k2d_create", "k2d_reset", "k2d_step",
+    "k2d_step_static_scratch", "k2d_obs",
     "k2d_obs_floats", "k2d_canonical_words", "k2d_get_state", "k2d_set_state", "k2d_status", "k2d_level_info",
     "k2d_set_trace", "k2d_trace_slots", "k2d_eval_sincos_tanh", "k2d_error_string", "k2d_destroy",
 )
@@ -66,6 +67,7 @@ def load_library():
         lib.k2d_create.argtypes = [C.POINTER(Config), vp, vp, vp, C.POINTER(vp)]
         lib.k2d_reset.argtypes = [vp, vp]
         lib.k2d_step.argtypes = [vp, vp, i32, vp, vp]
+        lib.k2d_step_static_scratch.argtypes = [vp, vp, i32, vp, vp]
         lib.k2d_obs.argtypes = [vp, vp]
         lib.k2d_obs_floats.argtypes = [C.POINTER(Config)]
         lib.k2d_canonical_words.argtypes = [C.POINTER(Config)]
@@ -161,8 +163,12 @@ class Env:
         ids = None if level_ids is None else np.ascontiguousarray(level_ids, np.int32)
         _check(self.lib.k2d_reset(self._h, None if ids is None else ids.ctypes.data), "k2d_reset")
 
-    def step(self, actions, reward=None, done=None):
-        """actions: CUDA float32 [n_steps, n_envs, n_actions]; returns (reward, done) CUDA tensors [n_steps, n_envs]."""
+    def step(self, actions, reward=None, done=None, static_scratch=False):
+        """actions: CUDA float32 [n_steps, n_envs, n_actions]; returns (reward, done) CUDA tensors [n_steps, n_envs].
+
+        ``static_scratch=True`` goes through k2d_step_static_scratch: same results, but the records of
+        crowded scenes live in an array inside the library instead of the tail of the state buffer
+        (for callers that cannot allocate that tail; at most 1024 envs)."""
         torch = self.torch
         assert actions.is_cuda and actions.dtype == torch.float32 and actions.is_contiguous()
         if actions.dim() == 2:
@@ -173,7 +179,9 @@ class Env:
             reward = torch.empty((n_steps, self.n_envs), dtype=torch.float32, device=self.device)
         if done is None:
             done = torch.empty((n_steps, self.n_envs), dtype=torch.uint8, device=self.device)
-        _check(self.lib.k2d_step(self._h, actions.data_ptr(), n_steps, reward.data_ptr(), done.data_ptr()), "k2d_step")
+        fn, name = ((self.lib.k2d_step_static_scratch, "k2d_step_static_scratch") if static_scratch
+                    else (self.lib.k2d_step, "k2d_step"))
+        _check(fn(self._h, actions.data_ptr(), n_steps, reward.data_ptr(), done.data_ptr()), name)
         return reward, done
 
     def obs(self, out=None):
