@@ -12,17 +12,17 @@
 
 namespace k2d {
 
-using ClassS = SizeClass<5, 2, 1, 1, 21>;
-using ClassM = SizeClass<6, 3, 2, 2, 36>;
-using ClassL = SizeClass<12, 4, 6, 2, 32>;
+using ClassS = SizeClass<5, 2, 1, 1>;
+using ClassM = SizeClass<6, 3, 2, 2>;
+using ClassL = SizeClass<12, 4, 6, 2>;
 
 constexpr int kMaxSlots = 8192;      // resident scene groups a launch may use (bounds the overflow scratch)
 constexpr size_t kCtrlBytes = 256;   // control block at the start of the state buffer: 8 x uint64 counters
 
 // run-time view of a size class
 struct ClassInfo {
-    int id, P, C, N, J, T, NPP, NPC, NCC, NPAIRS, NSLOTS, CAP, MASKW;
-    int LV_WORDS, ST_WORDS, SCRATCH_WORDS, PTAB_WORDS, REGION_RAW;
+    int id, P, C, N, J, T, NPP, NPC, NCC, NPAIRS, NSLOTS, MASKW;
+    int LV_WORDS, ST_WORDS, SCRATCH_WORDS, PTAB_WORDS;
     int LV_X, LV_IM, LV_II, LV_FR, LV_RE, LV_FLAGS, LV_DENS, LV_RAD, LV_PVX, LV_PVY, LV_PNX, LV_PNY, LV_ELEN, LV_JOINT, LV_THR, LV_MASK;
     int ST_JACC, ST_META, ST_WARM;
 };
@@ -30,9 +30,8 @@ template <class SC>
 static ClassInfo make_info(int id) {
     ClassInfo c{};
     c.id = id; c.P = SC::P; c.C = SC::C; c.N = SC::N; c.J = SC::J; c.T = SC::T;
-    c.NPP = SC::NPP; c.NPC = SC::NPC; c.NCC = SC::NCC; c.NPAIRS = SC::NPAIRS; c.NSLOTS = SC::NSLOTS; c.CAP = SC::CAP; c.MASKW = SC::MASKW;
+    c.NPP = SC::NPP; c.NPC = SC::NPC; c.NCC = SC::NCC; c.NPAIRS = SC::NPAIRS; c.NSLOTS = SC::NSLOTS; c.MASKW = SC::MASKW;
     c.LV_WORDS = SC::LV_WORDS; c.ST_WORDS = SC::ST_WORDS; c.SCRATCH_WORDS = SC::SCRATCH_WORDS; c.PTAB_WORDS = SC::PTAB_WORDS;
-    c.REGION_RAW = SC::REGION_RAW;
     c.LV_X = SC::LV_X; c.LV_IM = SC::LV_IM; c.LV_II = SC::LV_II; c.LV_FR = SC::LV_FR; c.LV_RE = SC::LV_RE; c.LV_FLAGS = SC::LV_FLAGS;
     c.LV_DENS = SC::LV_DENS; c.LV_RAD = SC::LV_RAD; c.LV_PVX = SC::LV_PVX; c.LV_PVY = SC::LV_PVY; c.LV_PNX = SC::LV_PNX; c.LV_PNY = SC::LV_PNY;
     c.LV_ELEN = SC::LV_ELEN; c.LV_JOINT = SC::LV_JOINT; c.LV_THR = SC::LV_THR; c.LV_MASK = SC::LV_MASK;

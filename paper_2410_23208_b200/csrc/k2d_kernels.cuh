@@ -24,15 +24,14 @@ constexpr int kBlockThreads = 128;
 constexpr int kMaxActions = 16;
 constexpr int kRecWords = 24;   // contact pair record
 constexpr int kWarmWords = 5;   // pair index + 4 accumulated impulses
+constexpr int kStageWords = 9;  // packed pair word, normal, two contact points with penetration
 
 // ---------------------------------------------------------------- size classes and layouts
-template <int P_, int C_, int J_, int T_, int CAP_>
+template <int P_, int C_, int J_, int T_>
 struct SizeClass {
     static constexpr int P = P_, C = C_, N = P_ + C_, J = J_, T = T_;
     static constexpr int NPP = P * (P - 1) / 2, NPC = P * C, NCC = C * (C - 1) / 2;
     static constexpr int NPAIRS = NPP + NPC + NCC, NSLOTS = 2 * NPP + NPC + NCC;
-    static constexpr int CAP = CAP_ < NPAIRS ? CAP_ : NPAIRS;   // pair records kept in shared memory
-    static constexpr int OVF = NPAIRS - CAP;                     // the rest live in global scratch
     static constexpr int MASKW = (NPAIRS + 31) / 32;
     static constexpr int P4 = 4 * P;
     // level record (32-bit words)
@@ -47,33 +46,34 @@ struct SizeClass {
     // state record: bodies (same order as shared memory), joint impulses, meta, warm list
     static constexpr int ST_BODY = 0, ST_JACC = 6 * N, ST_META = ST_JACC + 2 * J, ST_WARM = ST_META + 8;
     static constexpr int ST_WORDS = (ST_WARM + kWarmWords * NPAIRS + 3) / 4 * 4;
-    static constexpr int SCRATCH_WORDS = OVF * (kRecWords + kWarmWords);
+    // Contact pair records beyond the first G of a scene (one per lane, in registers) live in global
+    // scratch; sized for the narrowest group (8 lanes).
+    static constexpr int OVF_MAX = NPAIRS > 8 ? NPAIRS - 8 : 0;
+    static constexpr int SCRATCH_WORDS = OVF_MAX * (kRecWords + kWarmWords);
     // shared memory region of one scene (words)
     static constexpr int BX = 0, BY = N, BTH = 2 * N, BVX = 3 * N, BVY = 4 * N, BW = 5 * N;
     static constexpr int BIM = 6 * N, BII = 7 * N, BFR = 8 * N, BRE = 9 * N, BC = 10 * N, BS = 11 * N, BFL = 12 * N;
     static constexpr int RAD = 13 * N;
-    static constexpr int WVX = RAD + C, WVY = WVX + P4, WNX = WVY + P4, WNY = WNX + P4, WOFF = WNY + P4, ELEN = WOFF + P4;
-    static constexpr int AMINX = ELEN + P4, AMINY = AMINX + N, AMAXX = AMINY + N, AMAXY = AMAXX + N;
-    static constexpr int JNT = AMAXY + N;                // 14 arrays of J
-    static constexpr int MASK = JNT + 14 * J;
+    static constexpr int WVX = RAD + C, WVY = WVX + P4, WNX = WVY + P4, WNY = WNX + P4, WOFF = WNY + P4;
+    static constexpr int BOX = (WOFF + P4 + 3) / 4 * 4;  // N x (min x, min y, max x, max y), 16-byte aligned
+    static constexpr int MASK = BOX + 4 * N;
     static constexpr int ACT = MASK + MASKW;
-    static constexpr int SURV = ACT + kMaxActions;       // bytes
-    static constexpr int WIDX = SURV + (NPAIRS + 3) / 4; // bytes
-    static constexpr int REC = WIDX + (NPAIRS + 3) / 4;
-    static constexpr int WARM = REC + kRecWords * CAP;
-    static constexpr int REGION_RAW = WARM + kWarmWords * CAP;
-    static constexpr int PTAB_WORDS = (NPAIRS + 1) / 2;  // block-shared pair table, 16 bits per pair
+    static constexpr int SURV = ACT + kMaxActions;       // bytes: pairs that passed the box test
+    static constexpr int WIDX = SURV + (NPAIRS + 3) / 4; // bytes: pair -> record index of the previous step
+    static constexpr int STG = WIDX + (NPAIRS + 3) / 4;  // kStageWords x G: manifolds on their way to the owning lane
+    static constexpr int PTAB_WORDS = ((NPAIRS + 1) / 2 + 3) / 4 * 4;  // block-shared pair table, 16 bits per pair
 };
-// joint arrays inside JNT
-enum { JA_AB = 0, JA_RAX, JA_RAY, JA_RBX, JA_RBY, JA_I11, JA_I12, JA_I22, JA_BX, JA_BY, JA_CX, JA_CY, JA_ACCX, JA_ACCY };
-// record fields
+// record fields (memory form of a contact pair record, used for records beyond the first G)
 enum { R_AB = 0, R_NX, R_NY, R_MU, R_M0 = 4 };
 enum { M_RNA = 0, M_RNB, M_RTA, M_RTB, M_MASSN, M_MASST, M_TARGET, M_CORR, M_ACCN, M_ACCT, M_WORDS };
 static_assert(R_M0 + 2 * M_WORDS == kRecWords, "record size");
+// staged manifold fields
+enum { S_AB = 0, S_NX, S_NY, S_PX0, S_PY0, S_PEN0, S_PX1, S_PY1, S_PEN1 };
+static_assert(S_PEN1 + 1 == kStageWords, "stage size");
 
 // shared-memory words per scene: padded so that the groups of one warp start in different banks
 template <class SC, int G>
-__host__ __device__ constexpr int region_words() { return (SC::REGION_RAW + 31) / 32 * 32 + (G < 32 ? G : 0); }
+__host__ __device__ constexpr int region_words() { return (SC::STG + kStageWords * G + 31) / 32 * 32 + (G < 32 ? G : 0); }
 
 // body flag word
 constexpr uint32_t F_ACTIVE = 1u, F_DYNAMIC = 2u;
@@ -183,7 +183,9 @@ struct Group {
     }
     __device__ __forceinline__ int shfl(int v, int src) const { return __shfl_sync(mask, v, src, G); }
     __device__ __forceinline__ unsigned shflu(unsigned v, int src) const { return __shfl_sync(mask, v, src, G); }
+    __device__ __forceinline__ float shflf(float v, int src) const { return __shfl_sync(mask, v, src, G); }
     __device__ __forceinline__ int max_int(int v) const { return __reduce_max_sync(mask, v); }
+    __device__ __forceinline__ int sum_int(int v) const { return (int)__reduce_add_sync(mask, (unsigned)v); }
     __device__ __forceinline__ bool any(bool p) const { return __ballot_sync(mask, p) != 0; }
     __device__ __forceinline__ unsigned lanes_below() const { return (1u << lane) - 1u; }
 };
@@ -191,43 +193,335 @@ struct Group {
 // one manifold as the narrowphase leaves it
 struct Manifold { float px, py, nx, ny, pen; };
 
+// A contact pair record as the lane that owns it keeps it in registers for the whole step:
+// the pair (packed word), the shared normal, the friction coefficient, the inverse masses and
+// inertias of its two bodies, and per manifold the lever-arm cross products, effective masses,
+// target normal velocity, positional correction and the accumulated normal / tangent impulse.
+struct Rec {
+    uint32_t ab;
+    float nx, ny, mu, ma, mb, ia, ib;
+    float rna[2], rnb[2], rta[2], rtb[2], massn[2], masst[2], target[2], corr[2], accn[2], acct[2];
+};
+// The point constraint of a revolute joint as the lane that owns it keeps it: lever arms, inverse
+// effective mass (symmetric 2x2), velocity bias, positional correction, accumulated impulse.
+struct JointRow { float rax, ray, rbx, rby, i11, i12, i22, bx, by, cx, cy, accx, accy; };
+
+struct ContactConsts { float slop, rest_thr, alpha, beta; };
+
+// ---- contact pre-step for manifold mi of pair (a, b)
+template <class SC>
+__device__ __forceinline__ void prestep_manifold(Rec &c, int mi, int a, int b, float px, float py, float pen, float acc_n, float acc_t,
+                                                 float er, const float *sm, const ContactConsts &cc) {
+    const float nx = c.nx, ny = c.ny;
+    const float rax = px - sm[SC::BX + a], ray = py - sm[SC::BY + a];
+    const float rbx = px - sm[SC::BX + b], rby = py - sm[SC::BY + b];
+    const float ma = c.ma, mb = c.mb, ia = c.ia, ib = c.ib;
+    const float tx = -ny, ty = nx;
+    const float rna = cross2(rax, ray, nx, ny), rnb = cross2(rbx, rby, nx, ny);
+    const float rta = cross2(rax, ray, tx, ty), rtb = cross2(rbx, rby, tx, ty);
+    float kn = ma + mb; kn = __fmaf_rn(ia * rna, rna, kn); kn = __fmaf_rn(ib * rnb, rnb, kn);
+    float kt = ma + mb; kt = __fmaf_rn(ia * rta, rta, kt); kt = __fmaf_rn(ib * rtb, rtb, kt);
+    // normal approach speed before warm starting
+    float vn0 = dot2(nx, ny, sm[SC::BVX + b] - sm[SC::BVX + a], sm[SC::BVY + b] - sm[SC::BVY + a]);
+    vn0 = __fmaf_rn(sm[SC::BW + b], rnb, vn0);
+    vn0 = __fmaf_rn(-sm[SC::BW + a], rna, vn0);
+    const float depth = fmax_cmp(pen - cc.slop, 0.0f);
+    const float bounce = (vn0 < -cc.rest_thr) ? (-er * vn0) : 0.0f;
+    c.rna[mi] = rna; c.rnb[mi] = rnb; c.rta[mi] = rta; c.rtb[mi] = rtb;
+    c.massn[mi] = 1.0f / kn; c.masst[mi] = 1.0f / kt;
+    c.target[mi] = bounce + cc.alpha * depth;
+    c.corr[mi] = (cc.beta * depth) / (ma + mb);
+    c.accn[mi] = acc_n; c.acct[mi] = acc_t;
+}
+
+// Builds the record of a staged pair: stage word ab, normal, and per manifold contact point and
+// penetration; w[] are the accumulated impulses the pair's slots carried out of the previous step.
+template <class SC>
+__device__ __forceinline__ void build_record(Rec &c, uint32_t ab, float nx, float ny, const float (&pt)[6], const float (&w)[4],
+                                             const float *sm, const ContactConsts &cc) {
+    const int a = ab & 31, b = (ab >> 5) & 31;
+    c.ab = ab; c.nx = nx; c.ny = ny;
+    c.ma = sm[SC::BIM + a]; c.mb = sm[SC::BIM + b]; c.ia = sm[SC::BII + a]; c.ib = sm[SC::BII + b];
+    const float fra = sm[SC::BFR + a], frb = sm[SC::BFR + b];
+    const float er = fmin_cmp(sm[SC::BRE + a], sm[SC::BRE + b]);
+    c.mu = sqrtf(__fmaf_rn(fra, fra, frb * frb));
+#pragma unroll
+    for (int mi = 0; mi < 2; ++mi) {
+        if ((ab >> 10) & (1u << mi)) prestep_manifold<SC>(c, mi, a, b, pt[3 * mi], pt[3 * mi + 1], pt[3 * mi + 2], w[2 * mi], w[2 * mi + 1], er, sm, cc);
+        else {
+            c.rna[mi] = 0.0f; c.rnb[mi] = 0.0f; c.rta[mi] = 0.0f; c.rtb[mi] = 0.0f; c.massn[mi] = 0.0f; c.masst[mi] = 0.0f;
+            c.target[mi] = 0.0f; c.corr[mi] = 0.0f; c.accn[mi] = 0.0f; c.acct[mi] = 0.0f;
+        }
+    }
+}
+
+// ---- one visit of a contact pair record.  MODE 0: warm start, 1: solver iteration, 2: positional correction
+template <class SC, int MODE>
+__device__ __forceinline__ void visit_pair(Rec &c, float *sm) {
+    const uint32_t ab = c.ab;
+    const int a = ab & 31, b = (ab >> 5) & 31;
+    const unsigned amask = (ab >> 10) & 3u;
+    const bool dyn_a = (ab >> 26) & 1u, dyn_b = (ab >> 27) & 1u;
+    const float nx = c.nx, ny = c.ny;
+    const float ma = c.ma, mb = c.mb;
+    if (MODE == 2) {
+        float xa = sm[SC::BX + a], ya = sm[SC::BY + a], xb = sm[SC::BX + b], yb = sm[SC::BY + b];
+#pragma unroll
+        for (int mi = 0; mi < 2; ++mi) {
+            if (amask & (1u << mi)) {
+                const float corr = c.corr[mi];
+                const float ca = ma * corr, cb = mb * corr;
+                xa = __fmaf_rn(-ca, nx, xa); ya = __fmaf_rn(-ca, ny, ya);
+                xb = __fmaf_rn(cb, nx, xb); yb = __fmaf_rn(cb, ny, yb);
+            }
+        }
+        if (dyn_a) { sm[SC::BX + a] = xa; sm[SC::BY + a] = ya; }
+        if (dyn_b) { sm[SC::BX + b] = xb; sm[SC::BY + b] = yb; }
+        return;
+    }
+    const float ia = c.ia, ib = c.ib;
+    const float tx = -ny, ty = nx;
+    const float mu = c.mu;
+    float vax = sm[SC::BVX + a], vay = sm[SC::BVY + a], wa = sm[SC::BW + a];
+    float vbx = sm[SC::BVX + b], vby = sm[SC::BVY + b], wb = sm[SC::BW + b];
+#pragma unroll
+    for (int mi = 0; mi < 2; ++mi) {
+        if (amask & (1u << mi)) {
+            const float rna = c.rna[mi], rnb = c.rnb[mi], rta = c.rta[mi], rtb = c.rtb[mi];
+            const float wna = ia * rna, wnb = ib * rnb, wta = ia * rta, wtb = ib * rtb;
+            float accn = c.accn[mi], acct = c.acct[mi];
+            float dn, dt_;
+            if (MODE == 0) { dn = accn; }
+            else {
+                float vn = dot2(nx, ny, vbx - vax, vby - vay);
+                vn = __fmaf_rn(wb, rnb, vn);
+                vn = __fmaf_rn(-wa, rna, vn);
+                const float lam = (c.target[mi] - vn) * c.massn[mi];
+                const float nw = fmax_cmp(accn + lam, 0.0f);
+                dn = nw - accn; accn = nw;
+            }
+            {
+                const float px = dn * nx, py = dn * ny;
+                vax = __fmaf_rn(-ma, px, vax); vay = __fmaf_rn(-ma, py, vay); wa = __fmaf_rn(-wna, dn, wa);
+                vbx = __fmaf_rn(mb, px, vbx); vby = __fmaf_rn(mb, py, vby); wb = __fmaf_rn(wnb, dn, wb);
+            }
+            if (MODE == 0) { dt_ = acct; }
+            else {
+                float vt = dot2(tx, ty, vbx - vax, vby - vay);
+                vt = __fmaf_rn(wb, rtb, vt);
+                vt = __fmaf_rn(-wa, rta, vt);
+                const float lam = (-vt) * c.masst[mi];
+                const float lim = mu * accn;
+                const float nw = fmax_cmp(fmin_cmp(acct + lam, lim), -lim);
+                dt_ = nw - acct; acct = nw;
+            }
+            {
+                const float px = dt_ * tx, py = dt_ * ty;
+                vax = __fmaf_rn(-ma, px, vax); vay = __fmaf_rn(-ma, py, vay); wa = __fmaf_rn(-wta, dt_, wa);
+                vbx = __fmaf_rn(mb, px, vbx); vby = __fmaf_rn(mb, py, vby); wb = __fmaf_rn(wtb, dt_, wb);
+            }
+            if (MODE == 1) { c.accn[mi] = accn; c.acct[mi] = acct; }
+        }
+    }
+    if (dyn_a) { sm[SC::BVX + a] = vax; sm[SC::BVY + a] = vay; sm[SC::BW + a] = wa; }
+    if (dyn_b) { sm[SC::BVX + b] = vbx; sm[SC::BVY + b] = vby; sm[SC::BW + b] = wb; }
+}
+
+// ---- records beyond the first G of a scene: memory form in global scratch, cold code
+__device__ __forceinline__ void rec_load(const uint32_t *r, Rec &c, const float *sm_im, const float *sm_ii) {
+    c.ab = r[R_AB]; c.nx = __uint_as_float(r[R_NX]); c.ny = __uint_as_float(r[R_NY]); c.mu = __uint_as_float(r[R_MU]);
+    const int a = c.ab & 31, b = (c.ab >> 5) & 31;
+    c.ma = sm_im[a]; c.mb = sm_im[b]; c.ia = sm_ii[a]; c.ib = sm_ii[b];
+#pragma unroll
+    for (int mi = 0; mi < 2; ++mi) {
+        const uint32_t *m = r + R_M0 + mi * M_WORDS;
+        c.rna[mi] = __uint_as_float(m[M_RNA]); c.rnb[mi] = __uint_as_float(m[M_RNB]);
+        c.rta[mi] = __uint_as_float(m[M_RTA]); c.rtb[mi] = __uint_as_float(m[M_RTB]);
+        c.massn[mi] = __uint_as_float(m[M_MASSN]); c.masst[mi] = __uint_as_float(m[M_MASST]);
+        c.target[mi] = __uint_as_float(m[M_TARGET]); c.corr[mi] = __uint_as_float(m[M_CORR]);
+        c.accn[mi] = __uint_as_float(m[M_ACCN]); c.acct[mi] = __uint_as_float(m[M_ACCT]);
+    }
+}
+__device__ __forceinline__ void rec_store(uint32_t *r, const Rec &c) {
+    r[R_AB] = c.ab; r[R_NX] = __float_as_uint(c.nx); r[R_NY] = __float_as_uint(c.ny); r[R_MU] = __float_as_uint(c.mu);
+#pragma unroll
+    for (int mi = 0; mi < 2; ++mi) {
+        uint32_t *m = r + R_M0 + mi * M_WORDS;
+        m[M_RNA] = __float_as_uint(c.rna[mi]); m[M_RNB] = __float_as_uint(c.rnb[mi]);
+        m[M_RTA] = __float_as_uint(c.rta[mi]); m[M_RTB] = __float_as_uint(c.rtb[mi]);
+        m[M_MASSN] = __float_as_uint(c.massn[mi]); m[M_MASST] = __float_as_uint(c.masst[mi]);
+        m[M_TARGET] = __float_as_uint(c.target[mi]); m[M_CORR] = __float_as_uint(c.corr[mi]);
+        m[M_ACCN] = __float_as_uint(c.accn[mi]); m[M_ACCT] = __float_as_uint(c.acct[mi]);
+    }
+}
+
+// Levels of all nrec records by one lane (per-body table), then the pre-step of records G..nrec-1.
+// old[] are this lane's accumulated impulses of the previous step.  Returns the highest level.
+template <class SC, int G>
+__device__ __noinline__ int ovf_prepare(float *sm, uint32_t *ovf, int nrec, float old0, float old1, float old2, float old3,
+                                        int warm_start, ContactConsts cc) {
+    Group<G> g;
+    const int lane = g.lane;
+    uint32_t *smu = reinterpret_cast<uint32_t *>(sm);
+    uint8_t *bl = reinterpret_cast<uint8_t *>(smu + SC::SURV);   // the survivor list is no longer needed
+    const uint8_t *widx = reinterpret_cast<const uint8_t *>(smu + SC::WIDX);
+    int max_level = 0;
+    if (lane == 0) {
+        for (int i = 0; i < SC::N; ++i) bl[i] = 0;
+        for (int k = 0; k < nrec; ++k) {
+            uint32_t *w = (k < G) ? (smu + SC::STG + S_AB * G + k) : (ovf + (size_t)(k - G) * kRecWords + S_AB);
+            const uint32_t ab = *w;
+            const int a = ab & 31, b = (ab >> 5) & 31;
+            int lvl = 1;
+            if ((ab >> 26) & 1u) lvl = max(lvl, bl[a] + 1);
+            if ((ab >> 27) & 1u) lvl = max(lvl, bl[b] + 1);
+            if ((ab >> 26) & 1u) bl[a] = (uint8_t)lvl;
+            if ((ab >> 27) & 1u) bl[b] = (uint8_t)lvl;
+            *w = ab | ((uint32_t)lvl << 19);
+            max_level = max(max_level, lvl);
+        }
+    }
+    __threadfence_block();
+    g.sync();
+    max_level = g.shfl(max_level, 0);
+    for (int base = G; base < nrec; base += G) {
+        const int k = base + lane;
+        const bool valid = k < nrec;
+        uint32_t *r = ovf + (size_t)(valid ? k - G : 0) * kRecWords;
+        uint32_t ab = 0u;
+        int wi = 255;
+        if (valid) { ab = r[S_AB]; wi = widx[(ab >> 12) & 127]; }
+        const int src = (wi < G) ? wi : 0;
+        float w[4] = { g.shflf(old0, src), g.shflf(old1, src), g.shflf(old2, src), g.shflf(old3, src) };
+        if (wi >= G && wi != 255) {
+            const uint32_t *wr = ovf + (size_t)SC::OVF_MAX * kRecWords + (size_t)(wi - G) * kWarmWords;
+#pragma unroll
+            for (int q = 0; q < 4; ++q) w[q] = __uint_as_float(wr[1 + q]);
+        }
+        if (wi == 255 || !warm_start) { w[0] = 0.0f; w[1] = 0.0f; w[2] = 0.0f; w[3] = 0.0f; }
+        if (valid) {
+            const float nx = __uint_as_float(r[S_NX]), ny = __uint_as_float(r[S_NY]);
+            const float pt[6] = { __uint_as_float(r[S_PX0]), __uint_as_float(r[S_PY0]), __uint_as_float(r[S_PEN0]),
+                                  __uint_as_float(r[S_PX1]), __uint_as_float(r[S_PY1]), __uint_as_float(r[S_PEN1]) };
+            Rec c;
+            build_record<SC>(c, ab, nx, ny, pt, w, sm, cc);
+            rec_store(r, c);
+        }
+    }
+    g.sync();
+    return max_level;
+}
+
+// One level of one sweep over records G..nrec-1.
+template <class SC, int G>
+__device__ __noinline__ void ovf_visit(float *sm, uint32_t *ovf, int nrec, int lvl, int mode) {
+    Group<G> g;
+    for (int k = G + g.lane; k < nrec; k += G) {
+        uint32_t *r = ovf + (size_t)(k - G) * kRecWords;
+        if (((r[R_AB] >> 19) & 127u) != (unsigned)lvl) continue;
+        Rec c;
+        rec_load(r, c, sm + SC::BIM, sm + SC::BII);
+        if (mode == 0) visit_pair<SC, 0>(c, sm);
+        else if (mode == 1) {
+            visit_pair<SC, 1>(c, sm);
+#pragma unroll
+            for (int mi = 0; mi < 2; ++mi) {
+                r[R_M0 + mi * M_WORDS + M_ACCN] = __float_as_uint(c.accn[mi]);
+                r[R_M0 + mi * M_WORDS + M_ACCT] = __float_as_uint(c.acct[mi]);
+            }
+        } else visit_pair<SC, 2>(c, sm);
+    }
+}
+
+// End of a step: the accumulated impulses of records G..nrec-1 become warm entries, the pair index
+// table learns where they are; returns this group's number of active manifolds among them.
+template <class SC, int G>
+__device__ __noinline__ int ovf_finish(float *sm, uint32_t *ovf, int nrec) {
+    Group<G> g;
+    uint8_t *widx = reinterpret_cast<uint8_t *>(reinterpret_cast<uint32_t *>(sm) + SC::WIDX);
+    int nman = 0;
+    for (int k = G + g.lane; k < nrec; k += G) {
+        const uint32_t *r = ovf + (size_t)(k - G) * kRecWords;
+        uint32_t *wr = ovf + (size_t)SC::OVF_MAX * kRecWords + (size_t)(k - G) * kWarmWords;
+        const uint32_t ab = r[R_AB];
+        const int p = (ab >> 12) & 127;
+        const unsigned am = (ab >> 10) & 3u;
+        wr[0] = (uint32_t)p;
+        wr[1] = (am & 1u) ? r[R_M0 + M_ACCN] : 0u;
+        wr[2] = (am & 1u) ? r[R_M0 + M_ACCT] : 0u;
+        wr[3] = (am & 2u) ? r[R_M0 + M_WORDS + M_ACCN] : 0u;
+        wr[4] = (am & 2u) ? r[R_M0 + M_WORDS + M_ACCT] : 0u;
+        widx[p] = (uint8_t)k;
+        nman += __popc(am);
+    }
+    return g.sum_int(nman);
+}
+
+// Launch boundaries: warm entries G.. between the state record and the scratch.
+template <class SC, int G>
+__device__ __noinline__ void ovf_warm_in(float *sm, uint32_t *ovf, const uint32_t *st_warm, int nwarm) {
+    Group<G> g;
+    uint8_t *widx = reinterpret_cast<uint8_t *>(reinterpret_cast<uint32_t *>(sm) + SC::WIDX);
+    for (int k = G + g.lane; k < nwarm; k += G) {
+        uint32_t *wr = ovf + (size_t)SC::OVF_MAX * kRecWords + (size_t)(k - G) * kWarmWords;
+#pragma unroll
+        for (int q = 0; q < kWarmWords; ++q) wr[q] = st_warm[kWarmWords * k + q];
+        widx[wr[0]] = (uint8_t)k;
+    }
+}
+template <class SC, int G>
+__device__ __noinline__ void ovf_warm_out(const uint32_t *ovf, uint32_t *st_warm, int nwarm) {
+    Group<G> g;
+    for (int k = G + g.lane; k < nwarm; k += G) {
+        const uint32_t *wr = ovf + (size_t)SC::OVF_MAX * kRecWords + (size_t)(k - G) * kWarmWords;
+#pragma unroll
+        for (int q = 0; q < kWarmWords; ++q) st_warm[kWarmWords * k + q] = wr[q];
+    }
+}
+
 // ---------------------------------------------------------------- scene processing
 template <class SC, int G>
 struct Scene {
+    static_assert(SC::J <= G && SC::T <= G && kMaxActions <= 32, "one lane per joint / thruster");
     float *sm;            // this scene's shared-memory region
     uint32_t *smu;
     const uint16_t *ptab; // block-shared pair table
-    uint32_t *ovf;        // this group's overflow scratch in global memory (SC::OVF > 0 only)
+    uint32_t *ovf;        // this group's overflow scratch in global memory
     const StepParams &prm;
     Group<G> g;
     int lane;
+    // state a lane keeps in registers from step to step
+    Rec rec;              // contact pair record number `lane` of the latest step (its accumulated impulses warm-start the next)
+    JointRow jr;          // joint number `lane`
+    uint32_t jab;         // packed word of joint number `lane` (0 beyond the last joint)
+    unsigned c_surv, c_rec, c_man;   // packed work counters: pp | pc << 16, cc | active pairs << 16, manifolds | env-steps << 16
 
     __device__ __forceinline__ Scene(uint32_t *region, const uint16_t *pt, uint32_t *scratch, const StepParams &p)
-        : sm(reinterpret_cast<float *>(region)), smu(region), ptab(pt), ovf(scratch), prm(p), g() { lane = g.lane; }
+        : sm(reinterpret_cast<float *>(region)), smu(region), ptab(pt), ovf(scratch), prm(p), g() {
+        lane = g.lane; jab = 0u; c_surv = 0u; c_rec = 0u; c_man = 0u;
+    }
 
     __device__ __forceinline__ uint8_t *surv() { return reinterpret_cast<uint8_t *>(smu + SC::SURV); }
     __device__ __forceinline__ uint8_t *widx() { return reinterpret_cast<uint8_t *>(smu + SC::WIDX); }
-
-    // record / warm accessors; k >= CAP lives in global scratch
-    __device__ __forceinline__ float rec_ld(int f, int k) const {
-        if (SC::OVF == 0 || k < SC::CAP) return sm[SC::REC + f * SC::CAP + k];
-        return __uint_as_float(ovf[(k - SC::CAP) * kRecWords + f]);
+    __device__ __forceinline__ float4 &box4(int i) { return *reinterpret_cast<float4 *>(sm + SC::BOX + 4 * i); }
+    __device__ __forceinline__ ContactConsts contact_consts() const {
+        ContactConsts cc; cc.slop = prm.slop; cc.rest_thr = prm.rest_thr; cc.alpha = prm.contact_alpha; cc.beta = prm.contact_beta; return cc;
     }
-    __device__ __forceinline__ void rec_st(int f, int k, float v) {
-        if (SC::OVF == 0 || k < SC::CAP) sm[SC::REC + f * SC::CAP + k] = v;
-        else ovf[(k - SC::CAP) * kRecWords + f] = __float_as_uint(v);
-    }
-    __device__ __forceinline__ uint32_t warm_ld(int f, int k) const {
-        if (SC::OVF == 0 || k < SC::CAP) return smu[SC::WARM + f * SC::CAP + k];
-        return ovf[SC::OVF * kRecWords + (k - SC::CAP) * kWarmWords + f];
-    }
-    __device__ __forceinline__ void warm_st(int f, int k, uint32_t v) {
-        if (SC::OVF == 0 || k < SC::CAP) smu[SC::WARM + f * SC::CAP + k] = v;
-        else ovf[SC::OVF * kRecWords + (k - SC::CAP) * kWarmWords + f] = v;
+    __device__ __forceinline__ void flush_counters() {
+        if (lane == 0) {
+            const unsigned v[5] = { c_man & 0xffffu, c_man >> 16, c_surv & 0xffffu, c_surv >> 16, c_rec & 0xffffu };
+            if (v[0]) atomicAdd(prm.counters + 2, (unsigned long long)v[0]);
+            if (v[1]) atomicAdd(prm.counters + 3, (unsigned long long)v[1]);
+            if (v[2]) atomicAdd(prm.counters + 4, (unsigned long long)v[2]);
+            if (v[3]) atomicAdd(prm.counters + 5, (unsigned long long)v[3]);
+            if (v[4]) atomicAdd(prm.counters + 6, (unsigned long long)v[4]);
+            if (c_rec >> 16) atomicAdd(prm.counters + 7, (unsigned long long)(c_rec >> 16));
+        }
+        c_surv = 0u; c_rec = 0u; c_man = 0u;
     }
 
-    // ---- level constants into shared memory
-    __device__ void load_level_consts(const uint32_t *lv) {
+    // ---- level constants into shared memory / registers
+    __device__ __forceinline__ void load_level_consts(const uint32_t *lv) {
         for (int i = lane; i < SC::N; i += G) {
             smu[SC::BIM + i] = lv[SC::LV_IM + i];
             smu[SC::BII + i] = lv[SC::LV_II + i];
@@ -236,12 +530,12 @@ struct Scene {
             smu[SC::BFL + i] = lv[SC::LV_FLAGS + i];
         }
         for (int i = lane; i < SC::C; i += G) smu[SC::RAD + i] = lv[SC::LV_RAD + i];
-        for (int i = lane; i < SC::P4; i += G) smu[SC::ELEN + i] = lv[SC::LV_ELEN + i];
         for (int i = lane; i < SC::MASKW; i += G) smu[SC::MASK + i] = lv[SC::LV_MASK + i];
+        jab = (SC::J > 0 && lane < SC::J) ? lv[SC::LV_JOINT + 8 * lane] : 0u;
     }
-    __device__ void load_level_pose(const uint32_t *lv) {
+    __device__ __forceinline__ void load_level_pose(const uint32_t *lv) {
         for (int i = lane; i < 6 * SC::N; i += G) smu[SC::BX + i] = lv[SC::LV_X + i];
-        for (int i = lane; i < SC::J; i += G) { sm[SC::JNT + JA_ACCX * SC::J + i] = 0.0f; sm[SC::JNT + JA_ACCY * SC::J + i] = 0.0f; }
+        jr.accx = 0.0f; jr.accy = 0.0f;
         for (int i = lane; i < (SC::NPAIRS + 3) / 4; i += G) smu[SC::WIDX + i] = 0xffffffffu;
     }
 
@@ -325,7 +619,7 @@ struct Scene {
     }
 
     // polygon a against circle b
-    __device__ unsigned manifold_pc(int a, int b, Manifold &m) const {
+    __device__ unsigned manifold_pc(int a, int b, Manifold &m, const uint32_t *lv) const {
         const int cnt = flag_nverts(smu[SC::BFL + a]);
         const float cx = sm[SC::BX + b], cy = sm[SC::BY + b], r = sm[SC::RAD + (b - SC::P)];
         float maxsep = 0.0f, mind2 = 0.0f, qx = 0.0f, qy = 0.0f, dqx = 0.0f, dqy = 0.0f;
@@ -338,7 +632,7 @@ struct Scene {
                 const float sep = dot2(nx, ny, cx, cy) - sm[SC::WOFF + 4 * a + k];
                 const float tx = -ny, ty = nx;
                 float s = dot2(tx, ty, cx - wx, cy - wy);
-                s = fmax_cmp(fmin_cmp(s, sm[SC::ELEN + 4 * a + k]), 0.0f);
+                s = fmax_cmp(fmin_cmp(s, __uint_as_float(lv[SC::LV_ELEN + 4 * a + k])), 0.0f);
                 const float px = __fmaf_rn(s, tx, wx), py = __fmaf_rn(s, ty, wy);
                 const float ex = cx - px, ey = cy - py;
                 const float d2 = dot2(ex, ey, ex, ey);
@@ -370,156 +664,42 @@ struct Scene {
         return m.pen > 0.0f ? 1u : 0u;
     }
 
-    // ---- contact pre-step for one manifold of pair (a, b): writes the manifold part of record k
-    __device__ __forceinline__ void prestep_manifold(int k, int mi, int a, int b, const Manifold &m, float acc_n, float acc_t, float er) {
-        const float rax = m.px - sm[SC::BX + a], ray = m.py - sm[SC::BY + a];
-        const float rbx = m.px - sm[SC::BX + b], rby = m.py - sm[SC::BY + b];
-        const float ma = sm[SC::BIM + a], mb = sm[SC::BIM + b], ia = sm[SC::BII + a], ib = sm[SC::BII + b];
-        const float tx = -m.ny, ty = m.nx;
-        const float rna = cross2(rax, ray, m.nx, m.ny), rnb = cross2(rbx, rby, m.nx, m.ny);
-        const float rta = cross2(rax, ray, tx, ty), rtb = cross2(rbx, rby, tx, ty);
-        float kn = ma + mb; kn = __fmaf_rn(ia * rna, rna, kn); kn = __fmaf_rn(ib * rnb, rnb, kn);
-        float kt = ma + mb; kt = __fmaf_rn(ia * rta, rta, kt); kt = __fmaf_rn(ib * rtb, rtb, kt);
-        // normal approach speed before warm starting
-        float vn0 = dot2(m.nx, m.ny, sm[SC::BVX + b] - sm[SC::BVX + a], sm[SC::BVY + b] - sm[SC::BVY + a]);
-        vn0 = __fmaf_rn(sm[SC::BW + b], rnb, vn0);
-        vn0 = __fmaf_rn(-sm[SC::BW + a], rna, vn0);
-        const float depth = fmax_cmp(m.pen - prm.slop, 0.0f);
-        const float bounce = (vn0 < -prm.rest_thr) ? (-er * vn0) : 0.0f;
-        const int f = R_M0 + mi * M_WORDS;
-        rec_st(f + M_RNA, k, rna); rec_st(f + M_RNB, k, rnb); rec_st(f + M_RTA, k, rta); rec_st(f + M_RTB, k, rtb);
-        rec_st(f + M_MASSN, k, 1.0f / kn); rec_st(f + M_MASST, k, 1.0f / kt);
-        rec_st(f + M_TARGET, k, bounce + prm.contact_alpha * depth);
-        rec_st(f + M_CORR, k, (prm.contact_beta * depth) / (ma + mb));
-        rec_st(f + M_ACCN, k, acc_n); rec_st(f + M_ACCT, k, acc_t);
-    }
-
-    // ---- one visit of contact pair record k.  MODE 0: warm start, 1: solver iteration, 2: positional correction
-    template <int MODE>
-    __device__ __forceinline__ void visit_pair(int k, uint32_t ab) {
-        const int a = ab & 31, b = (ab >> 5) & 31;
-        const unsigned amask = (ab >> 10) & 3u;
-        const bool dyn_a = (ab >> 26) & 1u, dyn_b = (ab >> 27) & 1u;
-        const float nx = rec_ld(R_NX, k), ny = rec_ld(R_NY, k);
-        const float ma = sm[SC::BIM + a], mb = sm[SC::BIM + b];
-        if (MODE == 2) {
-            float xa = sm[SC::BX + a], ya = sm[SC::BY + a], xb = sm[SC::BX + b], yb = sm[SC::BY + b];
-#pragma unroll
-            for (int mi = 0; mi < 2; ++mi) {
-                if (amask & (1u << mi)) {
-                    const float corr = rec_ld(R_M0 + mi * M_WORDS + M_CORR, k);
-                    const float ca = ma * corr, cb = mb * corr;
-                    xa = __fmaf_rn(-ca, nx, xa); ya = __fmaf_rn(-ca, ny, ya);
-                    xb = __fmaf_rn(cb, nx, xb); yb = __fmaf_rn(cb, ny, yb);
-                }
-            }
-            if (dyn_a) { sm[SC::BX + a] = xa; sm[SC::BY + a] = ya; }
-            if (dyn_b) { sm[SC::BX + b] = xb; sm[SC::BY + b] = yb; }
-            return;
-        }
-        const float ia = sm[SC::BII + a], ib = sm[SC::BII + b];
-        const float tx = -ny, ty = nx;
-        const float mu = rec_ld(R_MU, k);
-        float vax = sm[SC::BVX + a], vay = sm[SC::BVY + a], wa = sm[SC::BW + a];
-        float vbx = sm[SC::BVX + b], vby = sm[SC::BVY + b], wb = sm[SC::BW + b];
-#pragma unroll
-        for (int mi = 0; mi < 2; ++mi) {
-            if (amask & (1u << mi)) {
-                const int f = R_M0 + mi * M_WORDS;
-                const float rna = rec_ld(f + M_RNA, k), rnb = rec_ld(f + M_RNB, k);
-                const float rta = rec_ld(f + M_RTA, k), rtb = rec_ld(f + M_RTB, k);
-                const float wna = ia * rna, wnb = ib * rnb, wta = ia * rta, wtb = ib * rtb;
-                float accn = rec_ld(f + M_ACCN, k), acct = rec_ld(f + M_ACCT, k);
-                float dn, dt_;
-                if (MODE == 0) { dn = accn; }
-                else {
-                    float vn = dot2(nx, ny, vbx - vax, vby - vay);
-                    vn = __fmaf_rn(wb, rnb, vn);
-                    vn = __fmaf_rn(-wa, rna, vn);
-                    const float lam = (rec_ld(f + M_TARGET, k) - vn) * rec_ld(f + M_MASSN, k);
-                    const float nw = fmax_cmp(accn + lam, 0.0f);
-                    dn = nw - accn; accn = nw;
-                }
-                {
-                    const float px = dn * nx, py = dn * ny;
-                    vax = __fmaf_rn(-ma, px, vax); vay = __fmaf_rn(-ma, py, vay); wa = __fmaf_rn(-wna, dn, wa);
-                    vbx = __fmaf_rn(mb, px, vbx); vby = __fmaf_rn(mb, py, vby); wb = __fmaf_rn(wnb, dn, wb);
-                }
-                if (MODE == 0) { dt_ = acct; }
-                else {
-                    float vt = dot2(tx, ty, vbx - vax, vby - vay);
-                    vt = __fmaf_rn(wb, rtb, vt);
-                    vt = __fmaf_rn(-wa, rta, vt);
-                    const float lam = (-vt) * rec_ld(f + M_MASST, k);
-                    const float lim = mu * accn;
-                    const float nw = fmax_cmp(fmin_cmp(acct + lam, lim), -lim);
-                    dt_ = nw - acct; acct = nw;
-                }
-                {
-                    const float px = dt_ * tx, py = dt_ * ty;
-                    vax = __fmaf_rn(-ma, px, vax); vay = __fmaf_rn(-ma, py, vay); wa = __fmaf_rn(-wta, dt_, wa);
-                    vbx = __fmaf_rn(mb, px, vbx); vby = __fmaf_rn(mb, py, vby); wb = __fmaf_rn(wtb, dt_, wb);
-                }
-                if (MODE == 1) { rec_st(f + M_ACCN, k, accn); rec_st(f + M_ACCT, k, acct); }
-            }
-        }
-        if (dyn_a) { sm[SC::BVX + a] = vax; sm[SC::BVY + a] = vay; sm[SC::BW + a] = wa; }
-        if (dyn_b) { sm[SC::BVX + b] = vbx; sm[SC::BVY + b] = vby; sm[SC::BW + b] = wb; }
-    }
-
-    template <int MODE>
-    __device__ __forceinline__ void sweep_pairs(int nrec, int max_level, uint32_t my_ab) {
-        for (int lvl = 1; lvl <= max_level; ++lvl) {
-            if (lane < nrec && ((my_ab >> 19) & 127u) == (unsigned)lvl) visit_pair<MODE>(lane, my_ab);
-            if (nrec > G) {
-                for (int k = lane + G; k < nrec; k += G) {
-                    const uint32_t ab = __float_as_uint(rec_ld(R_AB, k));
-                    if (((ab >> 19) & 127u) == (unsigned)lvl) visit_pair<MODE>(k, ab);
-                }
-            }
-            g.sync();
-        }
-    }
-
     // ---- joints.  MODE 0: warm start, 1: solver iteration, 2: positional correction, 3: motor
     template <int MODE>
-    __device__ __forceinline__ void visit_joint(int j, uint32_t jab, const uint32_t *lv) {
+    __device__ __forceinline__ void visit_joint(const uint32_t *lv) {
         const int a = jab & 255, b = (jab >> 8) & 255;
         const bool dyn_a = smu[SC::BFL + a] & F_DYNAMIC, dyn_b = smu[SC::BFL + b] & F_DYNAMIC;
-        float *jn = sm + SC::JNT;
         if (MODE == 3) {
             const float A = fmax_cmp(fmin_cmp(sm[SC::ACT + ((jab >> 16) & 255)], 1.0f), -1.0f);
-            const float speed = __uint_as_float(lv[SC::LV_JOINT + 8 * j + 5]), power = __uint_as_float(lv[SC::LV_JOINT + 8 * j + 6]);
+            const float speed = __uint_as_float(lv[SC::LV_JOINT + 8 * lane + 5]), power = __uint_as_float(lv[SC::LV_JOINT + 8 * lane + 6]);
             const float wa = sm[SC::BW + a], wb = sm[SC::BW + b];
             const float arg = __fmaf_rn(-speed, A, wa - wb) * prm.motor_rho;
-            const float jr = power * tanh_spec(arg);
-            if (dyn_a) sm[SC::BW + a] = __fmaf_rn(-jr, sm[SC::BII + a], wa);
-            if (dyn_b) sm[SC::BW + b] = __fmaf_rn(jr, sm[SC::BII + b], wb);
+            const float jr_ = power * tanh_spec(arg);
+            if (dyn_a) sm[SC::BW + a] = __fmaf_rn(-jr_, sm[SC::BII + a], wa);
+            if (dyn_b) sm[SC::BW + b] = __fmaf_rn(jr_, sm[SC::BII + b], wb);
             return;
         }
         const float ma = sm[SC::BIM + a], mb = sm[SC::BIM + b];
         if (MODE == 2) {
-            const float cx = jn[JA_CX * SC::J + j], cy = jn[JA_CY * SC::J + j];
+            const float cx = jr.cx, cy = jr.cy;
             if (dyn_a) { sm[SC::BX + a] = __fmaf_rn(ma, cx, sm[SC::BX + a]); sm[SC::BY + a] = __fmaf_rn(ma, cy, sm[SC::BY + a]); }
             if (dyn_b) { sm[SC::BX + b] = __fmaf_rn(-mb, cx, sm[SC::BX + b]); sm[SC::BY + b] = __fmaf_rn(-mb, cy, sm[SC::BY + b]); }
             return;
         }
         const float ia = sm[SC::BII + a], ib = sm[SC::BII + b];
-        const float rax = jn[JA_RAX * SC::J + j], ray = jn[JA_RAY * SC::J + j];
-        const float rbx = jn[JA_RBX * SC::J + j], rby = jn[JA_RBY * SC::J + j];
+        const float rax = jr.rax, ray = jr.ray, rbx = jr.rbx, rby = jr.rby;
         float vax = sm[SC::BVX + a], vay = sm[SC::BVY + a], wa = sm[SC::BW + a];
         float vbx = sm[SC::BVX + b], vby = sm[SC::BVY + b], wb = sm[SC::BW + b];
         float lx, ly;
-        if (MODE == 0) { lx = jn[JA_ACCX * SC::J + j]; ly = jn[JA_ACCY * SC::J + j]; }
+        if (MODE == 0) { lx = jr.accx; ly = jr.accy; }
         else {
             const float cx = __fmaf_rn(-wb, rby, vbx) - __fmaf_rn(-wa, ray, vax);
             const float cy = __fmaf_rn(wb, rbx, vby) - __fmaf_rn(wa, rax, vay);
-            const float rx = -(cx + jn[JA_BX * SC::J + j]), ry = -(cy + jn[JA_BY * SC::J + j]);
-            const float i11 = jn[JA_I11 * SC::J + j], i12 = jn[JA_I12 * SC::J + j], i22 = jn[JA_I22 * SC::J + j];
-            lx = __fmaf_rn(i11, rx, i12 * ry);
-            ly = __fmaf_rn(i12, rx, i22 * ry);
-            jn[JA_ACCX * SC::J + j] = jn[JA_ACCX * SC::J + j] + lx;
-            jn[JA_ACCY * SC::J + j] = jn[JA_ACCY * SC::J + j] + ly;
+            const float rx = -(cx + jr.bx), ry = -(cy + jr.by);
+            lx = __fmaf_rn(jr.i11, rx, jr.i12 * ry);
+            ly = __fmaf_rn(jr.i12, rx, jr.i22 * ry);
+            jr.accx = jr.accx + lx;
+            jr.accy = jr.accy + ly;
         }
         if (dyn_a) {
             sm[SC::BVX + a] = __fmaf_rn(-ma, lx, vax); sm[SC::BVY + a] = __fmaf_rn(-ma, ly, vay);
@@ -531,20 +711,28 @@ struct Scene {
         }
     }
 
+    // joints of one level touch disjoint movable bodies; levels in order keep the joint order
     template <int MODE>
-    __device__ __forceinline__ void sweep_joints(int max_level, uint32_t my_jab, const uint32_t *lv) {
+    __device__ __forceinline__ void sweep_joints(int jmax, int jlevel, const uint32_t *lv) {
         if (SC::J == 0) return;
-        for (int lvl = 1; lvl <= max_level; ++lvl) {
-            for (int j = lane, r = 0; j < SC::J; j += G, ++r) {
-                const uint32_t jab = (r == 0) ? my_jab : smu[SC::JNT + JA_AB * SC::J + j];
-                if (((jab >> 24) & 1u) && ((jab >> 25) & 7u) == (unsigned)lvl) visit_joint<MODE>(j, jab, lv);
-            }
+#pragma unroll 1
+        for (int lvl = 1; lvl <= jmax; ++lvl) {
+            if (jlevel == lvl) visit_joint<MODE>(lv);
+            g.sync();
+        }
+    }
+    template <int MODE>
+    __device__ __forceinline__ void sweep_pairs(int nrec, int cmax, int clevel) {
+#pragma unroll 1
+        for (int lvl = 1; lvl <= cmax; ++lvl) {
+            if (clevel == lvl) visit_pair<SC, MODE>(rec, sm);
+            if (nrec > G) ovf_visit<SC, G>(sm, ovf, nrec, lvl, MODE);
             g.sync();
         }
     }
 
-    // ---- one environment step.  Returns through meta[]: step_count, episode_count, level_id, status, nwarm
-    __device__ void step(int e, int s, int (&meta)[5], unsigned (&cnt)[8]) {
+    // ---- one environment step.  meta[]: step_count, episode_count, level_id, status, number of warm entries
+    __device__ __forceinline__ void step(int e, int s, int (&meta)[5]) {
         const uint32_t *lv = prm.levels + (size_t)meta[2] * SC::LV_WORDS;
         // frozen env: reports done, nothing else
         if (meta[3] & 1) {
@@ -552,7 +740,8 @@ struct Scene {
             return;
         }
         // actions of this step
-        for (int i = lane; i < prm.n_actions; i += G) sm[SC::ACT + i] = prm.actions[((size_t)s * prm.n_envs + e) * prm.n_actions + i];
+        if (lane < prm.n_actions) sm[SC::ACT + lane] = prm.actions[((size_t)s * prm.n_envs + e) * prm.n_actions + lane];
+        if (G < kMaxActions && lane + G < prm.n_actions) sm[SC::ACT + lane + G] = prm.actions[((size_t)s * prm.n_envs + e) * prm.n_actions + lane + G];
         // gravity, rotation, circle boxes
         for (int i = lane; i < SC::N; i += G) {
             const uint32_t fl = smu[SC::BFL + i];
@@ -562,7 +751,7 @@ struct Scene {
             sm[SC::BC + i] = c; sm[SC::BS + i] = sn;
             if (i >= SC::P) {
                 const float r = sm[SC::RAD + (i - SC::P)], x = sm[SC::BX + i], y = sm[SC::BY + i];
-                sm[SC::AMINX + i] = x - r; sm[SC::AMINY + i] = y - r; sm[SC::AMAXX + i] = x + r; sm[SC::AMAXY + i] = y + r;
+                box4(i) = make_float4(x - r, y - r, x + r, y + r);
             }
         }
         g.sync();
@@ -579,19 +768,9 @@ struct Scene {
                 sm[SC::WOFF + v] = dot2(nx, ny, wx, wy);
             }
         }
-        // joints: read the packed word once per step
-        uint32_t my_jab = 0u;
-        if (SC::J > 0 && lane < SC::J) my_jab = lv[SC::LV_JOINT + 8 * lane];
-        int jmax = 0;
-        if (SC::J > 0) {
-            int jl = 0;
-            for (int j = lane, r = 0; j < SC::J; j += G, ++r) {
-                const uint32_t jab = (r == 0) ? my_jab : lv[SC::LV_JOINT + 8 * j];
-                smu[SC::JNT + JA_AB * SC::J + j] = jab;
-                if ((jab >> 24) & 1u) jl = max(jl, (int)((jab >> 25) & 7u));
-            }
-            jmax = g.max_int(jl);
-        }
+        // this lane's joint: "on" bit and level come with the level record
+        const int jlevel = ((jab >> 24) & 1u) ? (int)((jab >> 25) & 7u) : 0;
+        const int jmax = (SC::J > 0) ? g.max_int(jlevel) : 0;
         g.sync();
         // polygon boxes
         for (int i = lane; i < SC::P; i += G) {
@@ -604,16 +783,17 @@ struct Scene {
                     x0 = fmin_cmp(x0, x); y0 = fmin_cmp(y0, y); x1 = fmax_cmp(x1, x); y1 = fmax_cmp(y1, y);
                 }
             }
-            sm[SC::AMINX + i] = x0; sm[SC::AMINY + i] = y0; sm[SC::AMAXX + i] = x1; sm[SC::AMAXY + i] = y1;
+            box4(i) = make_float4(x0, y0, x1, y1);
         }
         // motors (joint order), thrusters (thruster order)
-        sweep_joints<3>(jmax, my_jab, lv);
+        sweep_joints<3>(jmax, jlevel, lv);
         if (SC::T > 0) {
             int tl = 0; uint32_t tp = 0u;
             if (lane < SC::T) { tp = lv[SC::LV_THR + 8 * lane]; if ((tp >> 16) & 1u) tl = (tp >> 17) & 7u; }
             const int tmax = g.max_int(tl);
+#pragma unroll 1
             for (int lvl = 1; lvl <= tmax; ++lvl) {
-                if (lane < SC::T && tl == lvl) {
+                if (tl == lvl) {
                     const int i = tp & 255;
                     const uint32_t *th = lv + SC::LV_THR + 8 * lane;
                     const float A = fmax_cmp(fmin_cmp(sm[SC::ACT + ((tp >> 8) & 255)], 1.0f), 0.0f);
@@ -631,77 +811,82 @@ struct Scene {
                 g.sync();
             }
         }
-        // joint pre-step
-        for (int j = lane, r = 0; j < SC::J; j += G, ++r) {
-            const uint32_t jab = (r == 0) ? my_jab : smu[SC::JNT + JA_AB * SC::J + j];
-            float *jn = sm + SC::JNT;
-            if (!((jab >> 24) & 1u)) { jn[JA_ACCX * SC::J + j] = 0.0f; jn[JA_ACCY * SC::J + j] = 0.0f; continue; }
-            if (!prm.warm_start) { jn[JA_ACCX * SC::J + j] = 0.0f; jn[JA_ACCY * SC::J + j] = 0.0f; }
-            const int a = jab & 255, b = (jab >> 8) & 255;
-            const uint32_t *jl = lv + SC::LV_JOINT + 8 * j;
-            float rax, ray, rbx, rby;
-            rot2(sm[SC::BC + a], sm[SC::BS + a], __uint_as_float(jl[1]), __uint_as_float(jl[2]), rax, ray);
-            rot2(sm[SC::BC + b], sm[SC::BS + b], __uint_as_float(jl[3]), __uint_as_float(jl[4]), rbx, rby);
-            const float ma = sm[SC::BIM + a], mb = sm[SC::BIM + b], ia = sm[SC::BII + a], ib = sm[SC::BII + b];
-            const float gx = (sm[SC::BX + b] + rbx) - (sm[SC::BX + a] + rax), gy = (sm[SC::BY + b] + rby) - (sm[SC::BY + a] + ray);
-            const float msum = ma + mb;
-            float k11 = msum; k11 = __fmaf_rn(ia * ray, ray, k11); k11 = __fmaf_rn(ib * rby, rby, k11);
-            float k22 = msum; k22 = __fmaf_rn(ia * rax, rax, k22); k22 = __fmaf_rn(ib * rbx, rbx, k22);
-            float k12 = -((ia * rax) * ray); k12 = __fmaf_rn(-(ib * rbx), rby, k12);
-            const float det = __fmaf_rn(k11, k22, -(k12 * k12));
-            const float inv_det = 1.0f / det;
-            jn[JA_RAX * SC::J + j] = rax; jn[JA_RAY * SC::J + j] = ray; jn[JA_RBX * SC::J + j] = rbx; jn[JA_RBY * SC::J + j] = rby;
-            jn[JA_I11 * SC::J + j] = k22 * inv_det; jn[JA_I22 * SC::J + j] = k11 * inv_det; jn[JA_I12 * SC::J + j] = -(k12 * inv_det);
-            jn[JA_BX * SC::J + j] = prm.joint_alpha * gx; jn[JA_BY * SC::J + j] = prm.joint_alpha * gy;
-            const float share = prm.joint_beta / msum;
-            jn[JA_CX * SC::J + j] = share * gx; jn[JA_CY * SC::J + j] = share * gy;
+        // joint pre-step (poses only; velocities are not read)
+        if (SC::J > 0 && lane < SC::J) {
+            if (!((jab >> 24) & 1u) || !prm.warm_start) { jr.accx = 0.0f; jr.accy = 0.0f; }
+            if ((jab >> 24) & 1u) {
+                const int a = jab & 255, b = (jab >> 8) & 255;
+                const uint32_t *jl = lv + SC::LV_JOINT + 8 * lane;
+                float rax, ray, rbx, rby;
+                rot2(sm[SC::BC + a], sm[SC::BS + a], __uint_as_float(jl[1]), __uint_as_float(jl[2]), rax, ray);
+                rot2(sm[SC::BC + b], sm[SC::BS + b], __uint_as_float(jl[3]), __uint_as_float(jl[4]), rbx, rby);
+                const float ma = sm[SC::BIM + a], mb = sm[SC::BIM + b], ia = sm[SC::BII + a], ib = sm[SC::BII + b];
+                const float gx = (sm[SC::BX + b] + rbx) - (sm[SC::BX + a] + rax), gy = (sm[SC::BY + b] + rby) - (sm[SC::BY + a] + ray);
+                const float msum = ma + mb;
+                float k11 = msum; k11 = __fmaf_rn(ia * ray, ray, k11); k11 = __fmaf_rn(ib * rby, rby, k11);
+                float k22 = msum; k22 = __fmaf_rn(ia * rax, rax, k22); k22 = __fmaf_rn(ib * rbx, rbx, k22);
+                float k12 = -((ia * rax) * ray); k12 = __fmaf_rn(-(ib * rbx), rby, k12);
+                const float det = __fmaf_rn(k11, k22, -(k12 * k12));
+                const float inv_det = 1.0f / det;
+                jr.rax = rax; jr.ray = ray; jr.rbx = rbx; jr.rby = rby;
+                jr.i11 = k22 * inv_det; jr.i22 = k11 * inv_det; jr.i12 = -(k12 * inv_det);
+                jr.bx = prm.joint_alpha * gx; jr.by = prm.joint_alpha * gy;
+                const float share = prm.joint_beta / msum;
+                jr.cx = share * gx; jr.cy = share * gy;
+            }
         }
         g.sync();
 
         // bounding-box test over all pairs -> compact list of surviving pairs, in pair order
-        int nsurv = 0, ns_pp = 0, ns_pc = 0;
-        for (int base = 0; base < SC::NPAIRS; base += G) {
-            const int p = base + lane;
-            bool keep = false;
-            if (p < SC::NPAIRS && ((smu[SC::MASK + (p >> 5)] >> (p & 31)) & 1u)) {
-                const int a = ptab[p] & 255, b = ptab[p] >> 8;
-                const float mg = prm.aabb_margin;
-                keep = !(sm[SC::AMAXX + a] + mg < sm[SC::AMINX + b] || sm[SC::AMAXX + b] + mg < sm[SC::AMINX + a] ||
-                         sm[SC::AMAXY + a] + mg < sm[SC::AMINY + b] || sm[SC::AMAXY + b] + mg < sm[SC::AMINY + a]);
+        int nsurv = 0, ns_pp, ns_pc;
+        {
+            int mine_pp = 0, mine_pc = 0;     // this lane's survivors below the polygon-circle / circle-circle boundary
+            const float mg = prm.aabb_margin;
+#pragma unroll 1
+            for (int base = 0; base < SC::NPAIRS; base += G) {
+                const int p = base + lane;
+                bool keep = false;
+                if (p < SC::NPAIRS && ((smu[SC::MASK + (p >> 5)] >> (p & 31)) & 1u)) {
+                    const uint32_t code = ptab[p];
+                    const float4 ba = box4(code & 255), bb = box4(code >> 8);
+                    keep = !(ba.z + mg < bb.x || bb.z + mg < ba.x || ba.w + mg < bb.y || bb.w + mg < ba.y);
+                }
+                const unsigned bal = g.ballot(keep);
+                if (keep) surv()[nsurv + __popc(bal & g.lanes_below())] = (uint8_t)p;
+                nsurv += __popc(bal);
+                mine_pp += (keep && p < SC::NPP) ? 1 : 0;
+                mine_pc += (keep && p < SC::NPP + SC::NPC) ? 1 : 0;
             }
-            const unsigned bal = g.ballot(keep);
-            if (keep) surv()[nsurv + __popc(bal & g.lanes_below())] = (uint8_t)p;
-            nsurv += __popc(bal);
-            // segment boundaries: survivors below NPP are polygon-polygon, below NPP+NPC polygon-circle
-            if (base + G <= SC::NPP) ns_pp = nsurv;
-            else if (base < SC::NPP) ns_pp += __popc(bal & ((SC::NPP - base >= 32) ? 0xffffffffu : ((1u << (SC::NPP - base)) - 1u)));
-            if (base + G <= SC::NPP + SC::NPC) ns_pc = nsurv;
-            else if (base < SC::NPP + SC::NPC) {
-                const int lim = SC::NPP + SC::NPC - base;
-                ns_pc += __popc(bal & ((lim >= 32) ? 0xffffffffu : ((1u << lim) - 1u)));
-            }
+            ns_pp = g.sum_int(mine_pp);
+            ns_pc = g.sum_int(mine_pc);
         }
         g.sync();
-        if (lane == 0) { cnt[4] += ns_pp; cnt[5] += ns_pc - ns_pp; cnt[6] += nsurv - ns_pc; }
+        c_surv += (unsigned)ns_pp | ((unsigned)(ns_pc - ns_pp) << 16);
+        c_rec += (unsigned)(nsurv - ns_pc);
 
-        // narrowphase + contact pre-step: survivors of one kind at a time, records in pair order
+        // narrowphase: survivors of one kind at a time; active pairs are staged in pair order
         int nrec = 0;
         bool t_gb = false, t_gr = false;
         float *trace = prm.trace ? prm.trace + (size_t)e * SC::NSLOTS * 6 : nullptr;
-        if (trace) for (int i = lane; i < SC::NSLOTS * 6; i += G) trace[i] = ((i % 6) == 3) ? 1.0f : ((i % 6) == 4 ? -1.0f : 0.0f);
-        if (trace) g.sync();
+        if (trace) {
+            for (int i = lane; i < SC::NSLOTS * 6; i += G) trace[i] = ((i % 6) == 3) ? 1.0f : ((i % 6) == 4 ? -1.0f : 0.0f);
+            g.sync();
+        }
+#pragma unroll 1
         for (int kind = 0; kind < 3; ++kind) {
             const int lo = kind == 0 ? 0 : (kind == 1 ? ns_pp : ns_pc);
             const int hi = kind == 0 ? ns_pp : (kind == 1 ? ns_pc : nsurv);
+#pragma unroll 1
             for (int base = lo; base < hi; base += G) {
                 const int idx = base + lane;
                 unsigned act = 0u;
                 Manifold m[2];
+                m[1].px = 0.0f; m[1].py = 0.0f; m[1].pen = 0.0f;
                 int p = 0, a = 0, b = 0;
                 if (idx < hi) {
                     p = surv()[idx]; a = ptab[p] & 255; b = ptab[p] >> 8;
                     if (kind == 0) act = manifold_pp(a, b, m);
-                    else if (kind == 1) act = manifold_pc(a, b, m[0]);
+                    else if (kind == 1) act = manifold_pc(a, b, m[0], lv);
                     else act = manifold_cc(a, b, m[0]);
                     // a polygon pair rejected before its manifolds exist leaves its slots at the default
                     if (trace && !(kind == 0 && act == 0u)) {
@@ -721,23 +906,20 @@ struct Scene {
                     const uint32_t ra = flag_role(fa), rb = flag_role(fb);
                     t_gb |= (ra == 1u && rb == 2u) || (ra == 2u && rb == 1u);
                     t_gr |= (ra == 1u && rb == 3u) || (ra == 3u && rb == 1u);
-                    // accumulated impulses of the previous step, kept per slot while the slot stays active
-                    float wacc[4] = { 0.0f, 0.0f, 0.0f, 0.0f };
-                    const int wi = widx()[p];
-                    if (prm.warm_start && wi != 255) {
-#pragma unroll
-                        for (int q = 0; q < 4; ++q) wacc[q] = __uint_as_float(warm_ld(1 + q, wi));
-                    }
-                    const float fra = sm[SC::BFR + a], frb = sm[SC::BFR + b];
-                    const float er = fmin_cmp(sm[SC::BRE + a], sm[SC::BRE + b]);
                     const uint32_t ab = (uint32_t)a | ((uint32_t)b << 5) | (act << 10) | ((uint32_t)p << 12) |
                                         (((fa & F_DYNAMIC) ? 1u : 0u) << 26) | (((fb & F_DYNAMIC) ? 1u : 0u) << 27);
-                    rec_st(R_AB, k, __uint_as_float(ab));
-                    rec_st(R_NX, k, (act & 1u) ? m[0].nx : m[1].nx);
-                    rec_st(R_NY, k, (act & 1u) ? m[0].ny : m[1].ny);
-                    rec_st(R_MU, k, sqrtf(__fmaf_rn(fra, fra, frb * frb)));
-                    if (act & 1u) prestep_manifold(k, 0, a, b, m[0], wacc[0], wacc[1], er);
-                    if (act & 2u) prestep_manifold(k, 1, a, b, m[1], wacc[2], wacc[3], er);
+                    const float nx = (act & 1u) ? m[0].nx : m[1].nx, ny = (act & 1u) ? m[0].ny : m[1].ny;
+                    if (k < G) {
+                        float *st = sm + SC::STG + k;
+                        st[S_AB * G] = __uint_as_float(ab); st[S_NX * G] = nx; st[S_NY * G] = ny;
+                        st[S_PX0 * G] = m[0].px; st[S_PY0 * G] = m[0].py; st[S_PEN0 * G] = m[0].pen;
+                        st[S_PX1 * G] = m[1].px; st[S_PY1 * G] = m[1].py; st[S_PEN1 * G] = m[1].pen;
+                    } else {
+                        uint32_t *st = ovf + (size_t)(k - G) * kRecWords;
+                        st[S_AB] = ab; st[S_NX] = __float_as_uint(nx); st[S_NY] = __float_as_uint(ny);
+                        st[S_PX0] = __float_as_uint(m[0].px); st[S_PY0] = __float_as_uint(m[0].py); st[S_PEN0] = __float_as_uint(m[0].pen);
+                        st[S_PX1] = __float_as_uint(m[1].px); st[S_PY1] = __float_as_uint(m[1].py); st[S_PEN1] = __float_as_uint(m[1].pen);
+                    }
                 }
                 nrec += __popc(bal);
             }
@@ -745,58 +927,64 @@ struct Scene {
         const bool touch_gb = g.any(t_gb), touch_gr = g.any(t_gr);
         g.sync();
 
-        // levels of the contact pair records (canonical order = record order)
-        uint32_t my_ab = 0u;
-        int max_level = 0;
+        // every staged pair becomes a record in its own lane: accumulated impulses of the same pair in the
+        // previous step come from the lane that owned it then
+        const ContactConsts cc = contact_consts();
+        const float old0 = rec.accn[0], old1 = rec.acct[0], old2 = rec.accn[1], old3 = rec.acct[1];
+        int cmax = 0;
+        if (nrec > G) cmax = ovf_prepare<SC, G>(sm, ovf, nrec, old0, old1, old2, old3, prm.warm_start, cc);
+        {
+            const bool mine = lane < nrec;
+            uint32_t ab = 0u;
+            int wi = 255;
+            if (mine) { ab = smu[SC::STG + S_AB * G + lane]; wi = widx()[(ab >> 12) & 127]; }
+            const int src = (wi < G) ? wi : 0;
+            float w[4] = { g.shflf(old0, src), g.shflf(old1, src), g.shflf(old2, src), g.shflf(old3, src) };
+            if (wi >= G && wi != 255) {
+                const uint32_t *wr = ovf + (size_t)SC::OVF_MAX * kRecWords + (size_t)(wi - G) * kWarmWords;
+#pragma unroll
+                for (int q = 0; q < 4; ++q) w[q] = __uint_as_float(wr[1 + q]);
+            }
+            if (wi == 255 || !prm.warm_start) { w[0] = 0.0f; w[1] = 0.0f; w[2] = 0.0f; w[3] = 0.0f; }
+            if (mine) {
+                const float *st = sm + SC::STG + lane;
+                const float pt[6] = { st[S_PX0 * G], st[S_PY0 * G], st[S_PEN0 * G], st[S_PX1 * G], st[S_PY1 * G], st[S_PEN1 * G] };
+                build_record<SC>(rec, ab, st[S_NX * G], st[S_NY * G], pt, w, sm, cc);
+            } else rec.ab = 0u;
+        }
+        // levels of the records (canonical order = record order): one more than the highest level of an
+        // earlier record that shares a movable body
         if (nrec <= G) {
-            int lvl = 0;
-            if (lane < nrec) { my_ab = __float_as_uint(rec_ld(R_AB, lane)); lvl = 1; }
+            const uint32_t my_ab = rec.ab;
+            int lvl = (lane < nrec) ? 1 : 0;
             const int a = my_ab & 31, b = (my_ab >> 5) & 31;
             const bool da = (my_ab >> 26) & 1u, db = (my_ab >> 27) & 1u;
-            for (int q = 0; q < nrec; ++q) {
+#pragma unroll 1
+            for (int q = 0; q + 1 < nrec; ++q) {
                 const uint32_t abq = g.shflu(my_ab, q);
                 const int lq = g.shfl(lvl, q);
                 const int aq = abq & 31, bq = (abq >> 5) & 31;
                 const bool hit = (da && (a == aq || a == bq)) || (db && (b == aq || b == bq));
                 if (q < lane && lane < nrec && hit) lvl = max(lvl, lq + 1);
             }
-            my_ab |= (uint32_t)lvl << 19;
-            if (lane < nrec) rec_st(R_AB, lane, __uint_as_float(my_ab));
-            max_level = g.max_int(lvl);
-        } else {
-            // rare: more active pairs than lanes; one lane assigns levels with a per-body table
-            if (lane == 0) {
-                uint8_t *bl = surv();   // the survivor list is no longer needed
-                for (int i = 0; i < SC::N; ++i) bl[i] = 0;
-                for (int k = 0; k < nrec; ++k) {
-                    uint32_t ab = __float_as_uint(rec_ld(R_AB, k));
-                    const int a = ab & 31, b = (ab >> 5) & 31;
-                    int lvl = 1;
-                    if ((ab >> 26) & 1u) lvl = max(lvl, bl[a] + 1);
-                    if ((ab >> 27) & 1u) lvl = max(lvl, bl[b] + 1);
-                    if ((ab >> 26) & 1u) bl[a] = (uint8_t)lvl;
-                    if ((ab >> 27) & 1u) bl[b] = (uint8_t)lvl;
-                    rec_st(R_AB, k, __uint_as_float(ab | ((uint32_t)lvl << 19)));
-                    max_level = max(max_level, lvl);
-                }
-            }
-            __threadfence_block();
-            g.sync();
-            max_level = g.shfl(max_level, 0);
-            if (lane < nrec) my_ab = __float_as_uint(rec_ld(R_AB, lane));
+            rec.ab = my_ab | ((uint32_t)lvl << 19);
+            cmax = g.max_int(lvl);
         }
-        g.sync();
+        const int clevel = (int)((rec.ab >> 19) & 127u);
+        const unsigned am_mine = (rec.ab >> 10) & 3u;
+        c_man += (unsigned)(__popc(g.ballot(am_mine & 1u)) + __popc(g.ballot(am_mine & 2u)));
+        c_rec += (unsigned)nrec << 16;
 
         // warm start: contacts, then joints
-        sweep_pairs<0>(nrec, max_level, my_ab);
-        if (SC::J > 0) sweep_joints<0>(jmax, my_jab, lv);
+        sweep_pairs<0>(nrec, cmax, clevel);
+        sweep_joints<0>(jmax, jlevel, lv);
         // solver iterations: joints, then contacts
+#pragma unroll 1
         for (int it = 0; it < prm.solver_iters; ++it) {
-            sweep_joints<1>(jmax, my_jab, lv);
-            sweep_pairs<1>(nrec, max_level, my_ab);
+            sweep_joints<1>(jmax, jlevel, lv);
+            sweep_pairs<1>(nrec, cmax, clevel);
         }
         // Euler step with the solved velocities
-        bool finite = true;
         for (int i = lane; i < SC::N; i += G) {
             if (smu[SC::BFL + i] & F_ACTIVE) {
                 sm[SC::BX + i] = __fmaf_rn(prm.dt, sm[SC::BVX + i], sm[SC::BX + i]);
@@ -805,44 +993,32 @@ struct Scene {
             }
         }
         g.sync();
-        sweep_pairs<2>(nrec, max_level, my_ab);
-        sweep_joints<2>(jmax, my_jab, lv);
+        sweep_pairs<2>(nrec, cmax, clevel);
+        sweep_joints<2>(jmax, jlevel, lv);
+        bool finite = true;
         for (int i = lane; i < SC::N; i += G)
             finite = finite && finite_bits(sm[SC::BX + i]) && finite_bits(sm[SC::BY + i]) && finite_bits(sm[SC::BTH + i]) &&
                      finite_bits(sm[SC::BVX + i]) && finite_bits(sm[SC::BVY + i]) && finite_bits(sm[SC::BW + i]);
         finite = !g.any(!finite);
 
-        // accumulated impulses of this step become the warm list of the next one
+        // where the pairs of this step keep their accumulated impulses for the next one
         for (int i = lane; i < (SC::NPAIRS + 3) / 4; i += G) smu[SC::WIDX + i] = 0xffffffffu;
         g.sync();
-        int nman = 0;
-        for (int k = lane; k < nrec; k += G) {
-            const uint32_t ab = (k == lane) ? my_ab : __float_as_uint(rec_ld(R_AB, k));
-            const int p = (ab >> 12) & 127;
-            const unsigned am = (ab >> 10) & 3u;
-            warm_st(0, k, (uint32_t)p);
-            warm_st(1, k, (am & 1u) ? __float_as_uint(rec_ld(R_M0 + M_ACCN, k)) : 0u);
-            warm_st(2, k, (am & 1u) ? __float_as_uint(rec_ld(R_M0 + M_ACCT, k)) : 0u);
-            warm_st(3, k, (am & 2u) ? __float_as_uint(rec_ld(R_M0 + M_WORDS + M_ACCN, k)) : 0u);
-            warm_st(4, k, (am & 2u) ? __float_as_uint(rec_ld(R_M0 + M_WORDS + M_ACCT, k)) : 0u);
-            widx()[p] = (uint8_t)k;
-            nman += __popc(am);
-        }
+        if (lane < nrec) widx()[(rec.ab >> 12) & 127] = (uint8_t)lane;
+        if (nrec > G) c_man += (unsigned)ovf_finish<SC, G>(sm, ovf, nrec);
         meta[4] = nrec;
-        if (lane == 0) cnt[7] += nrec;
 
         // reward, termination, counters, auto-reset
         meta[0] += 1;
         const bool timeout = prm.max_episode_steps > 0 && meta[0] >= prm.max_episode_steps;
         float reward = (float)((int)touch_gb - (int)touch_gr);
         bool done = touch_gb || touch_gr || timeout;
-        if (!finite) { reward = 0.0f; done = true; meta[3] |= 1; if (lane == 0) cnt[0] += 1; }
+        if (!finite) { reward = 0.0f; done = true; meta[3] |= 1; if (lane == 0) atomicAdd(prm.counters + 0, 1ULL); }
         if (lane == 0) {
             prm.reward[(size_t)s * prm.n_envs + e] = reward;
             prm.done[(size_t)s * prm.n_envs + e] = done ? 1 : 0;
-            cnt[3] += 1;
         }
-        cnt[2] += nman;
+        c_man += 1u << 16;
         g.sync();
         if (done && prm.auto_reset != 0) {
             meta[1] += 1;
@@ -854,54 +1030,55 @@ struct Scene {
             }
             load_level_pose(prm.levels + (size_t)meta[2] * SC::LV_WORDS);
             meta[0] = 0; meta[3] = 0; meta[4] = 0;
-            if (lane == 0) cnt[1] += 1;
+            if (lane == 0) atomicAdd(prm.counters + 1, 1ULL);
             g.sync();
         }
     }
 
     // ---- whole launch for one scene
-    __device__ void run(int e) {
+    __device__ __forceinline__ void run(int e) {
         uint32_t *st = prm.state + (size_t)e * SC::ST_WORDS;
         int meta[5];
 #pragma unroll
         for (int i = 0; i < 5; ++i) meta[i] = (int)st[SC::ST_META + i];
         for (int i = lane; i < 6 * SC::N; i += G) smu[SC::BX + i] = st[SC::ST_BODY + i];
-        for (int i = lane; i < SC::J; i += G) {
-            smu[SC::JNT + JA_ACCX * SC::J + i] = st[SC::ST_JACC + 2 * i];
-            smu[SC::JNT + JA_ACCY * SC::J + i] = st[SC::ST_JACC + 2 * i + 1];
-        }
+        jr.accx = 0.0f; jr.accy = 0.0f;
+        if (SC::J > 0 && lane < SC::J) { jr.accx = __uint_as_float(st[SC::ST_JACC + 2 * lane]); jr.accy = __uint_as_float(st[SC::ST_JACC + 2 * lane + 1]); }
         for (int i = lane; i < (SC::NPAIRS + 3) / 4; i += G) smu[SC::WIDX + i] = 0xffffffffu;
         load_level_consts(prm.levels + (size_t)meta[2] * SC::LV_WORDS);
         g.sync();
-        for (int k = lane; k < meta[4]; k += G) {
-            const uint32_t p = st[SC::ST_WARM + kWarmWords * k];
-            warm_st(0, k, p);
-#pragma unroll
-            for (int q = 1; q < 5; ++q) warm_st(q, k, st[SC::ST_WARM + kWarmWords * k + q]);
-            widx()[p] = (uint8_t)k;
+        // accumulated impulses of the previous launch: entry k goes to lane k
+        rec.ab = 0u;
+        rec.accn[0] = 0.0f; rec.acct[0] = 0.0f; rec.accn[1] = 0.0f; rec.acct[1] = 0.0f;
+        if (lane < meta[4]) {
+            const uint32_t *wr = st + SC::ST_WARM + kWarmWords * lane;
+            rec.accn[0] = __uint_as_float(wr[1]); rec.acct[0] = __uint_as_float(wr[2]);
+            rec.accn[1] = __uint_as_float(wr[3]); rec.acct[1] = __uint_as_float(wr[4]);
+            widx()[wr[0]] = (uint8_t)lane;
         }
+        if (meta[4] > G) ovf_warm_in<SC, G>(sm, ovf, st + SC::ST_WARM, meta[4]);
         g.sync();
-        unsigned cnt[8] = { 0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u };
-        for (int s = 0; s < prm.n_steps; ++s) { step(e, s, meta, cnt); g.sync(); }
+#pragma unroll 1
+        for (int s = 0; s < prm.n_steps; ++s) {
+            step(e, s, meta);
+            g.sync();
+            if ((s & 255) == 255) flush_counters();
+        }
         // write back
         for (int i = lane; i < 6 * SC::N; i += G) st[SC::ST_BODY + i] = smu[SC::BX + i];
-        for (int i = lane; i < SC::J; i += G) {
-            st[SC::ST_JACC + 2 * i] = smu[SC::JNT + JA_ACCX * SC::J + i];
-            st[SC::ST_JACC + 2 * i + 1] = smu[SC::JNT + JA_ACCY * SC::J + i];
-        }
-        if (lane < 5) st[SC::ST_META + lane] = (uint32_t)meta[lane];
-        for (int k = lane; k < meta[4]; k += G) {
-#pragma unroll
-            for (int q = 0; q < 5; ++q) st[SC::ST_WARM + kWarmWords * k + q] = warm_ld(q, k);
-        }
-        // counters: lane 0 holds the event counts, every lane holds its share of the manifold count
-        unsigned nm = cnt[2];
-        for (int off = G / 2; off > 0; off >>= 1) nm += __shfl_down_sync(g.mask, nm, off, G);
+        if (SC::J > 0 && lane < SC::J) { st[SC::ST_JACC + 2 * lane] = __float_as_uint(jr.accx); st[SC::ST_JACC + 2 * lane + 1] = __float_as_uint(jr.accy); }
         if (lane == 0) {
-            cnt[2] = nm;
 #pragma unroll
-            for (int q = 0; q < 8; ++q) if (cnt[q]) atomicAdd(prm.counters + q, (unsigned long long)cnt[q]);
+            for (int i = 0; i < 5; ++i) st[SC::ST_META + i] = (uint32_t)meta[i];
         }
+        if (lane < meta[4]) {
+            uint32_t *wr = st + SC::ST_WARM + kWarmWords * lane;
+            wr[0] = (rec.ab >> 12) & 127u;
+            wr[1] = __float_as_uint(rec.accn[0]); wr[2] = __float_as_uint(rec.acct[0]);
+            wr[3] = __float_as_uint(rec.accn[1]); wr[4] = __float_as_uint(rec.acct[1]);
+        }
+        if (meta[4] > G) ovf_warm_out<SC, G>(ovf, st + SC::ST_WARM, meta[4]);
+        flush_counters();
     }
 };
 
@@ -924,8 +1101,9 @@ __global__ void __launch_bounds__(kBlockThreads) k2d_step_kernel(const StepParam
     const int gib = threadIdx.x / G;
     const int slot = blockIdx.x * GPB + gib, nslots = gridDim.x * GPB;
     uint32_t *region = smem_raw + SC::PTAB_WORDS + gib * region_words<SC, G>();
-    uint32_t *scratch = SC::OVF > 0 ? prm.scratch + (size_t)slot * SC::SCRATCH_WORDS : nullptr;
+    uint32_t *scratch = prm.scratch + (size_t)slot * SC::SCRATCH_WORDS;
     Scene<SC, G> scene(region, ptab, scratch, prm);
+#pragma unroll 1
     for (int e = slot; e < prm.n_envs; e += nslots) { scene.run(e); scene.g.sync(); }
 }
 
