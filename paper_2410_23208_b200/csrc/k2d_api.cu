@@ -201,7 +201,8 @@ static int pack_level(const k2d_config *cfg, const ClassInfo &ci, const k2d_leve
             if (!is_static[a]) body_level[a] = lvl;
             if (!is_static[b]) body_level[b] = lvl;
         }
-        jw[0] = (uint32_t)a | ((uint32_t)b << 8) | ((uint32_t)L->motor_binding[j] << 16) | ((on ? 1u : 0u) << 24) | ((uint32_t)lvl << 25) | (1u << 28);
+        jw[0] = (uint32_t)a | ((uint32_t)b << 8) | ((uint32_t)L->motor_binding[j] << 16) | ((on ? 1u : 0u) << 24) | ((uint32_t)lvl << 25) | (1u << 28) |
+                ((is_static[a] ? 0u : 1u) << 29) | ((is_static[b] ? 0u : 1u) << 30);
         for (int k = 0; k < 6; ++k) jw[1 + k] = f2u(v[k]);
         joined.emplace_back(a, b);
     }

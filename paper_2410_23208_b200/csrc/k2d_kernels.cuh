@@ -25,6 +25,7 @@ constexpr int kMaxActions = 16;
 constexpr int kRecWords = 24;   // contact pair record
 constexpr int kWarmWords = 5;   // pair index + 4 accumulated impulses
 constexpr int kStageWords = 9;  // packed pair word, normal, two contact points with penetration
+constexpr int kJointWords = 13; // joint row kept in shared memory
 
 // ---------------------------------------------------------------- size classes and layouts
 template <int P_, int C_, int J_, int T_>
@@ -46,10 +47,10 @@ struct SizeClass {
     // state record: bodies (same order as shared memory), joint impulses, meta, warm list
     static constexpr int ST_BODY = 0, ST_JACC = 6 * N, ST_META = ST_JACC + 2 * J, ST_WARM = ST_META + 8;
     static constexpr int ST_WORDS = (ST_WARM + kWarmWords * NPAIRS + 3) / 4 * 4;
-    // Contact pair records beyond the first G of a scene (one per lane, in registers) live in global
-    // scratch; sized for the narrowest group (8 lanes).
-    static constexpr int OVF_MAX = NPAIRS > 8 ? NPAIRS - 8 : 0;
-    static constexpr int SCRATCH_WORDS = OVF_MAX * (kRecWords + kWarmWords);
+    // A scene with more touching pairs than lanes takes the step's contact solve through global
+    // scratch: one memory record and one warm entry per pair.
+    static constexpr int SCRATCH_WORDS = NPAIRS * (kRecWords + kWarmWords);
+    static constexpr int SCRATCH_WARM = NPAIRS * kRecWords;
     // shared memory region of one scene (words)
     static constexpr int BX = 0, BY = N, BTH = 2 * N, BVX = 3 * N, BVY = 4 * N, BW = 5 * N;
     static constexpr int BIM = 6 * N, BII = 7 * N, BFR = 8 * N, BRE = 9 * N, BC = 10 * N, BS = 11 * N, BFL = 12 * N;
@@ -58,28 +59,40 @@ struct SizeClass {
     static constexpr int BOX = (WOFF + P4 + 3) / 4 * 4;  // N x (min x, min y, max x, max y), 16-byte aligned
     static constexpr int MASK = BOX + 4 * N;
     static constexpr int ACT = MASK + MASKW;
-    static constexpr int SURV = ACT + kMaxActions;       // bytes: pairs that passed the box test
+    static constexpr int META = ACT + kMaxActions;       // step_count, episode_count, level_id, status, warm entries
+    static constexpr int JROW = META + 8;                // kJointWords x J, field-major
+    static constexpr int SURV = JROW + kJointWords * J;  // bytes: pairs that passed the box test
     static constexpr int WIDX = SURV + (NPAIRS + 3) / 4; // bytes: pair -> record index of the previous step
-    static constexpr int STG = WIDX + (NPAIRS + 3) / 4;  // kStageWords x G: manifolds on their way to the owning lane
+    // then, per lane of the group (field-major, G words per field):
+    //   STG  kStageWords fields: manifolds on their way to the owning lane; afterwards the second manifold's constants
+    //   ACC2 2 fields: accumulated impulses of the second manifold;  CORR 2 fields: positional corrections
+    static constexpr int STG = WIDX + (NPAIRS + 3) / 4;
+    static constexpr int LANE_FIELDS = kStageWords + 4;
     static constexpr int PTAB_WORDS = ((NPAIRS + 1) / 2 + 3) / 4 * 4;  // block-shared pair table, 16 bits per pair
 };
-// record fields (memory form of a contact pair record, used for records beyond the first G)
+// memory form of a contact pair record (the overflow path keeps records in global scratch)
 enum { R_AB = 0, R_NX, R_NY, R_MU, R_M0 = 4 };
 enum { M_RNA = 0, M_RNB, M_RTA, M_RTB, M_MASSN, M_MASST, M_TARGET, M_CORR, M_ACCN, M_ACCT, M_WORDS };
 static_assert(R_M0 + 2 * M_WORDS == kRecWords, "record size");
 // staged manifold fields
 enum { S_AB = 0, S_NX, S_NY, S_PX0, S_PY0, S_PEN0, S_PX1, S_PY1, S_PEN1 };
 static_assert(S_PEN1 + 1 == kStageWords, "stage size");
+// second-manifold constants reuse the stage fields of the same lane
+enum { M2_RNA = 0, M2_RNB, M2_RTA, M2_RTB, M2_MASSN, M2_MASST, M2_TARGET };
+// joint row fields
+enum { JR_RAX = 0, JR_RAY, JR_RBX, JR_RBY, JR_I11, JR_I12, JR_I22, JR_BX, JR_BY, JR_CX, JR_CY, JR_ACCX, JR_ACCY };
+static_assert(JR_ACCY + 1 == kJointWords, "joint row size");
+enum { META_STEP = 0, META_EPISODE, META_LEVEL, META_STATUS, META_NWARM };
 
 // shared-memory words per scene: padded so that the groups of one warp start in different banks
 template <class SC, int G>
-__host__ __device__ constexpr int region_words() { return (SC::STG + kStageWords * G + 31) / 32 * 32 + (G < 32 ? G : 0); }
+__host__ __device__ constexpr int region_words() { return (SC::STG + SC::LANE_FIELDS * G + 31) / 32 * 32 + (G < 32 ? G : 0); }
 
 // body flag word
 constexpr uint32_t F_ACTIVE = 1u, F_DYNAMIC = 2u;
 __host__ __device__ inline uint32_t flag_role(uint32_t f) { return (f >> 2) & 3u; }
 __host__ __device__ inline uint32_t flag_nverts(uint32_t f) { return (f >> 4) & 7u; }
-// joint packed word: a | b<<8 | binding<<16 | on<<24 | level<<25 | active<<28
+// joint packed word: a | b<<8 | binding<<16 | on<<24 | level<<25 | active<<28 | a movable<<29 | b movable<<30
 // thruster packed word: shape | binding<<8 | on<<16 | level<<17 | active<<20
 // record AB word: a | b<<5 | amask<<10 | pair<<12 | level<<19 | dynA<<26 | dynB<<27
 
@@ -193,32 +206,36 @@ struct Group {
 // one manifold as the narrowphase leaves it
 struct Manifold { float px, py, nx, ny, pen; };
 
-// A contact pair record as the lane that owns it keeps it in registers for the whole step:
-// the pair (packed word), the shared normal, the friction coefficient, the inverse masses and
-// inertias of its two bodies, and per manifold the lever-arm cross products, effective masses,
-// target normal velocity, positional correction and the accumulated normal / tangent impulse.
+// What the lane that owns a contact pair record keeps in registers for the whole step: the pair
+// (packed word), the shared normal, the friction coefficient, the inverse masses and inertias of
+// the two bodies, and the first manifold's lever-arm cross products, effective masses, target
+// normal velocity and accumulated impulses.  The second manifold (polygon-polygon pairs only) is
+// in the lane's shared-memory fields.
 struct Rec {
     uint32_t ab;
     float nx, ny, mu, ma, mb, ia, ib;
+    float rna, rnb, rta, rtb, massn, masst, target, accn, acct;
+};
+// memory form (overflow path)
+struct RecM {
+    uint32_t ab;
+    float nx, ny, mu;
     float rna[2], rnb[2], rta[2], rtb[2], massn[2], masst[2], target[2], corr[2], accn[2], acct[2];
 };
-// The point constraint of a revolute joint as the lane that owns it keeps it: lever arms, inverse
-// effective mass (symmetric 2x2), velocity bias, positional correction, accumulated impulse.
-struct JointRow { float rax, ray, rbx, rby, i11, i12, i22, bx, by, cx, cy, accx, accy; };
 
 struct ContactConsts { float slop, rest_thr, alpha, beta; };
 
-// ---- contact pre-step for manifold mi of pair (a, b)
+// ---- contact pre-step for one manifold of pair (a, b) with normal (nx, ny)
 template <class SC>
-__device__ __forceinline__ void prestep_manifold(Rec &c, int mi, int a, int b, float px, float py, float pen, float acc_n, float acc_t,
-                                                 float er, const float *sm, const ContactConsts &cc) {
-    const float nx = c.nx, ny = c.ny;
+__device__ __forceinline__ void prestep_manifold(int a, int b, float nx, float ny, float ma, float mb, float ia, float ib,
+                                                 float px, float py, float pen, float er, const float *sm, const ContactConsts &cc,
+                                                 float &rna, float &rnb, float &rta, float &rtb, float &massn, float &masst,
+                                                 float &target, float &corr) {
     const float rax = px - sm[SC::BX + a], ray = py - sm[SC::BY + a];
     const float rbx = px - sm[SC::BX + b], rby = py - sm[SC::BY + b];
-    const float ma = c.ma, mb = c.mb, ia = c.ia, ib = c.ib;
     const float tx = -ny, ty = nx;
-    const float rna = cross2(rax, ray, nx, ny), rnb = cross2(rbx, rby, nx, ny);
-    const float rta = cross2(rax, ray, tx, ty), rtb = cross2(rbx, rby, tx, ty);
+    rna = cross2(rax, ray, nx, ny); rnb = cross2(rbx, rby, nx, ny);
+    rta = cross2(rax, ray, tx, ty); rtb = cross2(rbx, rby, tx, ty);
     float kn = ma + mb; kn = __fmaf_rn(ia * rna, rna, kn); kn = __fmaf_rn(ib * rnb, rnb, kn);
     float kt = ma + mb; kt = __fmaf_rn(ia * rta, rta, kt); kt = __fmaf_rn(ib * rtb, rtb, kt);
     // normal approach speed before warm starting
@@ -227,111 +244,136 @@ __device__ __forceinline__ void prestep_manifold(Rec &c, int mi, int a, int b, f
     vn0 = __fmaf_rn(-sm[SC::BW + a], rna, vn0);
     const float depth = fmax_cmp(pen - cc.slop, 0.0f);
     const float bounce = (vn0 < -cc.rest_thr) ? (-er * vn0) : 0.0f;
-    c.rna[mi] = rna; c.rnb[mi] = rnb; c.rta[mi] = rta; c.rtb[mi] = rtb;
-    c.massn[mi] = 1.0f / kn; c.masst[mi] = 1.0f / kt;
-    c.target[mi] = bounce + cc.alpha * depth;
-    c.corr[mi] = (cc.beta * depth) / (ma + mb);
-    c.accn[mi] = acc_n; c.acct[mi] = acc_t;
+    massn = 1.0f / kn; masst = 1.0f / kt;
+    target = bounce + cc.alpha * depth;
+    corr = (cc.beta * depth) / (ma + mb);
 }
 
-// Builds the record of a staged pair: stage word ab, normal, and per manifold contact point and
-// penetration; w[] are the accumulated impulses the pair's slots carried out of the previous step.
-template <class SC>
-__device__ __forceinline__ void build_record(Rec &c, uint32_t ab, float nx, float ny, const float (&pt)[6], const float (&w)[4],
-                                             const float *sm, const ContactConsts &cc) {
-    const int a = ab & 31, b = (ab >> 5) & 31;
-    c.ab = ab; c.nx = nx; c.ny = ny;
-    c.ma = sm[SC::BIM + a]; c.mb = sm[SC::BIM + b]; c.ia = sm[SC::BII + a]; c.ib = sm[SC::BII + b];
-    const float fra = sm[SC::BFR + a], frb = sm[SC::BFR + b];
-    const float er = fmin_cmp(sm[SC::BRE + a], sm[SC::BRE + b]);
-    c.mu = sqrtf(__fmaf_rn(fra, fra, frb * frb));
-#pragma unroll
-    for (int mi = 0; mi < 2; ++mi) {
-        if ((ab >> 10) & (1u << mi)) prestep_manifold<SC>(c, mi, a, b, pt[3 * mi], pt[3 * mi + 1], pt[3 * mi + 2], w[2 * mi], w[2 * mi + 1], er, sm, cc);
-        else {
-            c.rna[mi] = 0.0f; c.rnb[mi] = 0.0f; c.rta[mi] = 0.0f; c.rtb[mi] = 0.0f; c.massn[mi] = 0.0f; c.masst[mi] = 0.0f;
-            c.target[mi] = 0.0f; c.corr[mi] = 0.0f; c.accn[mi] = 0.0f; c.acct[mi] = 0.0f;
-        }
+// ---- one manifold's normal row then friction row on the velocities of its two bodies.
+// MODE 0: apply the accumulated impulses (warm start); MODE 1: one solver iteration.
+template <int MODE>
+__device__ __forceinline__ void manifold_rows(float nx, float ny, float mu, float ma, float mb, float ia, float ib,
+                                              float rna, float rnb, float rta, float rtb, float massn, float masst, float target,
+                                              float &accn, float &acct,
+                                              float &vax, float &vay, float &wa, float &vbx, float &vby, float &wb) {
+    const float tx = -ny, ty = nx;
+    const float wna = ia * rna, wnb = ib * rnb, wta = ia * rta, wtb = ib * rtb;
+    float dn, dt_;
+    if (MODE == 0) { dn = accn; }
+    else {
+        float vn = dot2(nx, ny, vbx - vax, vby - vay);
+        vn = __fmaf_rn(wb, rnb, vn);
+        vn = __fmaf_rn(-wa, rna, vn);
+        const float lam = (target - vn) * massn;
+        const float nw = fmax_cmp(accn + lam, 0.0f);
+        dn = nw - accn; accn = nw;
+    }
+    {
+        const float px = dn * nx, py = dn * ny;
+        vax = __fmaf_rn(-ma, px, vax); vay = __fmaf_rn(-ma, py, vay); wa = __fmaf_rn(-wna, dn, wa);
+        vbx = __fmaf_rn(mb, px, vbx); vby = __fmaf_rn(mb, py, vby); wb = __fmaf_rn(wnb, dn, wb);
+    }
+    if (MODE == 0) { dt_ = acct; }
+    else {
+        float vt = dot2(tx, ty, vbx - vax, vby - vay);
+        vt = __fmaf_rn(wb, rtb, vt);
+        vt = __fmaf_rn(-wa, rta, vt);
+        const float lam = (-vt) * masst;
+        const float lim = mu * accn;
+        const float nw = fmax_cmp(fmin_cmp(acct + lam, lim), -lim);
+        dt_ = nw - acct; acct = nw;
+    }
+    {
+        const float px = dt_ * tx, py = dt_ * ty;
+        vax = __fmaf_rn(-ma, px, vax); vay = __fmaf_rn(-ma, py, vay); wa = __fmaf_rn(-wta, dt_, wa);
+        vbx = __fmaf_rn(mb, px, vbx); vby = __fmaf_rn(mb, py, vby); wb = __fmaf_rn(wtb, dt_, wb);
     }
 }
 
-// ---- one visit of a contact pair record.  MODE 0: warm start, 1: solver iteration, 2: positional correction
+// positional correction of one pair: each active manifold moves the two bodies apart along the normal
+__device__ __forceinline__ void correct_pair(float *bx, float *by, int a, int b, unsigned amask, bool dyn_a, bool dyn_b,
+                                             float nx, float ny, float ma, float mb, float corr0, float corr1) {
+    float xa = bx[a], ya = by[a], xb = bx[b], yb = by[b];
+    if (amask & 1u) {
+        const float ca = ma * corr0, cb = mb * corr0;
+        xa = __fmaf_rn(-ca, nx, xa); ya = __fmaf_rn(-ca, ny, ya);
+        xb = __fmaf_rn(cb, nx, xb); yb = __fmaf_rn(cb, ny, yb);
+    }
+    if (amask & 2u) {
+        const float ca = ma * corr1, cb = mb * corr1;
+        xa = __fmaf_rn(-ca, nx, xa); ya = __fmaf_rn(-ca, ny, ya);
+        xb = __fmaf_rn(cb, nx, xb); yb = __fmaf_rn(cb, ny, yb);
+    }
+    if (dyn_a) { bx[a] = xa; by[a] = ya; }
+    if (dyn_b) { bx[b] = xb; by[b] = yb; }
+}
+
+// ---- joints; the row of joint j is in shared memory.  MODE 0: warm start, 1: solver iteration,
+// 2: positional correction, 3: motor
 template <class SC, int MODE>
-__device__ __forceinline__ void visit_pair(Rec &c, float *sm) {
-    const uint32_t ab = c.ab;
-    const int a = ab & 31, b = (ab >> 5) & 31;
-    const unsigned amask = (ab >> 10) & 3u;
-    const bool dyn_a = (ab >> 26) & 1u, dyn_b = (ab >> 27) & 1u;
-    const float nx = c.nx, ny = c.ny;
-    const float ma = c.ma, mb = c.mb;
-    if (MODE == 2) {
-        float xa = sm[SC::BX + a], ya = sm[SC::BY + a], xb = sm[SC::BX + b], yb = sm[SC::BY + b];
-#pragma unroll
-        for (int mi = 0; mi < 2; ++mi) {
-            if (amask & (1u << mi)) {
-                const float corr = c.corr[mi];
-                const float ca = ma * corr, cb = mb * corr;
-                xa = __fmaf_rn(-ca, nx, xa); ya = __fmaf_rn(-ca, ny, ya);
-                xb = __fmaf_rn(cb, nx, xb); yb = __fmaf_rn(cb, ny, yb);
-            }
-        }
-        if (dyn_a) { sm[SC::BX + a] = xa; sm[SC::BY + a] = ya; }
-        if (dyn_b) { sm[SC::BX + b] = xb; sm[SC::BY + b] = yb; }
+__device__ __forceinline__ void visit_joint(float *sm, uint32_t jab, int j, const uint32_t *lv, float motor_rho) {
+    const int a = jab & 255, b = (jab >> 8) & 255;
+    const bool dyn_a = (jab >> 29) & 1u, dyn_b = (jab >> 30) & 1u;
+    float *jr = sm + SC::JROW + j;
+    if (MODE == 3) {
+        const float A = fmax_cmp(fmin_cmp(sm[SC::ACT + ((jab >> 16) & 255)], 1.0f), -1.0f);
+        const float speed = __uint_as_float(lv[SC::LV_JOINT + 8 * j + 5]), power = __uint_as_float(lv[SC::LV_JOINT + 8 * j + 6]);
+        const float wa = sm[SC::BW + a], wb = sm[SC::BW + b];
+        const float arg = __fmaf_rn(-speed, A, wa - wb) * motor_rho;
+        const float jr_ = power * tanh_spec(arg);
+        if (dyn_a) sm[SC::BW + a] = __fmaf_rn(-jr_, sm[SC::BII + a], wa);
+        if (dyn_b) sm[SC::BW + b] = __fmaf_rn(jr_, sm[SC::BII + b], wb);
         return;
     }
-    const float ia = c.ia, ib = c.ib;
-    const float tx = -ny, ty = nx;
-    const float mu = c.mu;
+    const float ma = sm[SC::BIM + a], mb = sm[SC::BIM + b];
+    if (MODE == 2) {
+        const float cx = jr[JR_CX * SC::J], cy = jr[JR_CY * SC::J];
+        if (dyn_a) { sm[SC::BX + a] = __fmaf_rn(ma, cx, sm[SC::BX + a]); sm[SC::BY + a] = __fmaf_rn(ma, cy, sm[SC::BY + a]); }
+        if (dyn_b) { sm[SC::BX + b] = __fmaf_rn(-mb, cx, sm[SC::BX + b]); sm[SC::BY + b] = __fmaf_rn(-mb, cy, sm[SC::BY + b]); }
+        return;
+    }
+    const float ia = sm[SC::BII + a], ib = sm[SC::BII + b];
+    const float rax = jr[JR_RAX * SC::J], ray = jr[JR_RAY * SC::J], rbx = jr[JR_RBX * SC::J], rby = jr[JR_RBY * SC::J];
     float vax = sm[SC::BVX + a], vay = sm[SC::BVY + a], wa = sm[SC::BW + a];
     float vbx = sm[SC::BVX + b], vby = sm[SC::BVY + b], wb = sm[SC::BW + b];
-#pragma unroll
-    for (int mi = 0; mi < 2; ++mi) {
-        if (amask & (1u << mi)) {
-            const float rna = c.rna[mi], rnb = c.rnb[mi], rta = c.rta[mi], rtb = c.rtb[mi];
-            const float wna = ia * rna, wnb = ib * rnb, wta = ia * rta, wtb = ib * rtb;
-            float accn = c.accn[mi], acct = c.acct[mi];
-            float dn, dt_;
-            if (MODE == 0) { dn = accn; }
-            else {
-                float vn = dot2(nx, ny, vbx - vax, vby - vay);
-                vn = __fmaf_rn(wb, rnb, vn);
-                vn = __fmaf_rn(-wa, rna, vn);
-                const float lam = (c.target[mi] - vn) * c.massn[mi];
-                const float nw = fmax_cmp(accn + lam, 0.0f);
-                dn = nw - accn; accn = nw;
-            }
-            {
-                const float px = dn * nx, py = dn * ny;
-                vax = __fmaf_rn(-ma, px, vax); vay = __fmaf_rn(-ma, py, vay); wa = __fmaf_rn(-wna, dn, wa);
-                vbx = __fmaf_rn(mb, px, vbx); vby = __fmaf_rn(mb, py, vby); wb = __fmaf_rn(wnb, dn, wb);
-            }
-            if (MODE == 0) { dt_ = acct; }
-            else {
-                float vt = dot2(tx, ty, vbx - vax, vby - vay);
-                vt = __fmaf_rn(wb, rtb, vt);
-                vt = __fmaf_rn(-wa, rta, vt);
-                const float lam = (-vt) * c.masst[mi];
-                const float lim = mu * accn;
-                const float nw = fmax_cmp(fmin_cmp(acct + lam, lim), -lim);
-                dt_ = nw - acct; acct = nw;
-            }
-            {
-                const float px = dt_ * tx, py = dt_ * ty;
-                vax = __fmaf_rn(-ma, px, vax); vay = __fmaf_rn(-ma, py, vay); wa = __fmaf_rn(-wta, dt_, wa);
-                vbx = __fmaf_rn(mb, px, vbx); vby = __fmaf_rn(mb, py, vby); wb = __fmaf_rn(wtb, dt_, wb);
-            }
-            if (MODE == 1) { c.accn[mi] = accn; c.acct[mi] = acct; }
-        }
+    float lx, ly;
+    if (MODE == 0) { lx = jr[JR_ACCX * SC::J]; ly = jr[JR_ACCY * SC::J]; }
+    else {
+        const float cx = __fmaf_rn(-wb, rby, vbx) - __fmaf_rn(-wa, ray, vax);
+        const float cy = __fmaf_rn(wb, rbx, vby) - __fmaf_rn(wa, rax, vay);
+        const float rx = -(cx + jr[JR_BX * SC::J]), ry = -(cy + jr[JR_BY * SC::J]);
+        const float i11 = jr[JR_I11 * SC::J], i12 = jr[JR_I12 * SC::J], i22 = jr[JR_I22 * SC::J];
+        lx = __fmaf_rn(i11, rx, i12 * ry);
+        ly = __fmaf_rn(i12, rx, i22 * ry);
+        jr[JR_ACCX * SC::J] = jr[JR_ACCX * SC::J] + lx;
+        jr[JR_ACCY * SC::J] = jr[JR_ACCY * SC::J] + ly;
     }
-    if (dyn_a) { sm[SC::BVX + a] = vax; sm[SC::BVY + a] = vay; sm[SC::BW + a] = wa; }
-    if (dyn_b) { sm[SC::BVX + b] = vbx; sm[SC::BVY + b] = vby; sm[SC::BW + b] = wb; }
+    if (dyn_a) {
+        sm[SC::BVX + a] = __fmaf_rn(-ma, lx, vax); sm[SC::BVY + a] = __fmaf_rn(-ma, ly, vay);
+        sm[SC::BW + a] = __fmaf_rn(-ia, cross2(rax, ray, lx, ly), wa);
+    }
+    if (dyn_b) {
+        sm[SC::BVX + b] = __fmaf_rn(mb, lx, vbx); sm[SC::BVY + b] = __fmaf_rn(mb, ly, vby);
+        sm[SC::BW + b] = __fmaf_rn(ib, cross2(rbx, rby, lx, ly), wb);
+    }
+}
+// joints of one level touch disjoint movable bodies; levels in order keep the joint order
+template <class SC, int G, int MODE>
+__device__ __forceinline__ void sweep_joints(float *sm, uint32_t jab, int lane, int jlevel, int jmax, const uint32_t *lv, float motor_rho) {
+    const unsigned mask = Group<G>().mask;
+    if (SC::J == 0) return;
+#pragma unroll 1
+    for (int lvl = 1; lvl <= jmax; ++lvl) {
+        if (jlevel == lvl) visit_joint<SC, MODE>(sm, jab, lane, lv, motor_rho);
+        __syncwarp(mask);
+    }
 }
 
-// ---- records beyond the first G of a scene: memory form in global scratch, cold code
-__device__ __forceinline__ void rec_load(const uint32_t *r, Rec &c, const float *sm_im, const float *sm_ii) {
+// ================================================================ overflow path (cold code)
+// A scene with more touching pairs than lanes (nrec > G) solves this step's contacts from memory
+// records in global scratch, one loop over records per level, with the same row arithmetic.
+__device__ __forceinline__ void recm_load(const uint32_t *r, RecM &c) {
     c.ab = r[R_AB]; c.nx = __uint_as_float(r[R_NX]); c.ny = __uint_as_float(r[R_NY]); c.mu = __uint_as_float(r[R_MU]);
-    const int a = c.ab & 31, b = (c.ab >> 5) & 31;
-    c.ma = sm_im[a]; c.mb = sm_im[b]; c.ia = sm_ii[a]; c.ib = sm_ii[b];
 #pragma unroll
     for (int mi = 0; mi < 2; ++mi) {
         const uint32_t *m = r + R_M0 + mi * M_WORDS;
@@ -342,7 +384,7 @@ __device__ __forceinline__ void rec_load(const uint32_t *r, Rec &c, const float 
         c.accn[mi] = __uint_as_float(m[M_ACCN]); c.acct[mi] = __uint_as_float(m[M_ACCT]);
     }
 }
-__device__ __forceinline__ void rec_store(uint32_t *r, const Rec &c) {
+__device__ __forceinline__ void recm_store(uint32_t *r, const RecM &c) {
     r[R_AB] = c.ab; r[R_NX] = __float_as_uint(c.nx); r[R_NY] = __float_as_uint(c.ny); r[R_MU] = __float_as_uint(c.mu);
 #pragma unroll
     for (int mi = 0; mi < 2; ++mi) {
@@ -355,21 +397,65 @@ __device__ __forceinline__ void rec_store(uint32_t *r, const Rec &c) {
     }
 }
 
-// Levels of all nrec records by one lane (per-body table), then the pre-step of records G..nrec-1.
-// old[] are this lane's accumulated impulses of the previous step.  Returns the highest level.
+template <class SC, int G, int MODE>
+__device__ __forceinline__ void slow_sweep_pairs(float *sm, uint32_t *ovf, int nrec, int cmax) {
+    Group<G> g;
+    for (int lvl = 1; lvl <= cmax; ++lvl) {
+        for (int k = g.lane; k < nrec; k += G) {
+            uint32_t *r = ovf + (size_t)k * kRecWords;
+            if (((r[R_AB] >> 19) & 127u) != (unsigned)lvl) continue;
+            RecM c;
+            recm_load(r, c);
+            const int a = c.ab & 31, b = (c.ab >> 5) & 31;
+            const unsigned amask = (c.ab >> 10) & 3u;
+            const bool dyn_a = (c.ab >> 26) & 1u, dyn_b = (c.ab >> 27) & 1u;
+            const float ma = sm[SC::BIM + a], mb = sm[SC::BIM + b];
+            if (MODE == 2) { correct_pair(sm + SC::BX, sm + SC::BY, a, b, amask, dyn_a, dyn_b, c.nx, c.ny, ma, mb, c.corr[0], c.corr[1]); continue; }
+            const float ia = sm[SC::BII + a], ib = sm[SC::BII + b];
+            float vax = sm[SC::BVX + a], vay = sm[SC::BVY + a], wa = sm[SC::BW + a];
+            float vbx = sm[SC::BVX + b], vby = sm[SC::BVY + b], wb = sm[SC::BW + b];
+#pragma unroll
+            for (int mi = 0; mi < 2; ++mi) {
+                if (amask & (1u << mi)) {
+                    manifold_rows<MODE>(c.nx, c.ny, c.mu, ma, mb, ia, ib, c.rna[mi], c.rnb[mi], c.rta[mi], c.rtb[mi], c.massn[mi], c.masst[mi],
+                                        c.target[mi], c.accn[mi], c.acct[mi], vax, vay, wa, vbx, vby, wb);
+                    if (MODE == 1) {
+                        r[R_M0 + mi * M_WORDS + M_ACCN] = __float_as_uint(c.accn[mi]);
+                        r[R_M0 + mi * M_WORDS + M_ACCT] = __float_as_uint(c.acct[mi]);
+                    }
+                }
+            }
+            if (dyn_a) { sm[SC::BVX + a] = vax; sm[SC::BVY + a] = vay; sm[SC::BW + a] = wa; }
+            if (dyn_b) { sm[SC::BVX + b] = vbx; sm[SC::BVY + b] = vby; sm[SC::BW + b] = wb; }
+        }
+        g.sync();
+    }
+}
+
+// Records from the staged manifolds (the first G in shared memory, the rest already in scratch),
+// their levels, warm start and all solver iterations, joints included.  old_n / old_t: this lane's
+// first-manifold accumulated impulses of the previous step.  Returns the highest contact level.
 template <class SC, int G>
-__device__ __noinline__ int ovf_prepare(float *sm, uint32_t *ovf, int nrec, float old0, float old1, float old2, float old3,
-                                        int warm_start, ContactConsts cc) {
+__device__ __noinline__ int slow_solve(float *sm, uint32_t *ovf, const uint32_t *lv, int nrec, uint32_t jab, int jlevel, int jmax,
+                                       int solver_iters, int warm_start, float motor_rho, float old_n, float old_t, ContactConsts cc) {
     Group<G> g;
     const int lane = g.lane;
     uint32_t *smu = reinterpret_cast<uint32_t *>(sm);
     uint8_t *bl = reinterpret_cast<uint8_t *>(smu + SC::SURV);   // the survivor list is no longer needed
     const uint8_t *widx = reinterpret_cast<const uint8_t *>(smu + SC::WIDX);
-    int max_level = 0;
+    const float *lanef = sm + SC::STG;
+    // the staged manifolds of the first G pairs join the others in scratch
+    {
+        uint32_t *r = ovf + (size_t)lane * kRecWords;
+#pragma unroll
+        for (int f = 0; f < kStageWords; ++f) r[f] = smu[SC::STG + f * G + lane];
+    }
+    g.sync();
+    int cmax = 0;
     if (lane == 0) {
         for (int i = 0; i < SC::N; ++i) bl[i] = 0;
         for (int k = 0; k < nrec; ++k) {
-            uint32_t *w = (k < G) ? (smu + SC::STG + S_AB * G + k) : (ovf + (size_t)(k - G) * kRecWords + S_AB);
+            uint32_t *w = ovf + (size_t)k * kRecWords + S_AB;
             const uint32_t ab = *w;
             const int a = ab & 31, b = (ab >> 5) & 31;
             int lvl = 1;
@@ -378,71 +464,79 @@ __device__ __noinline__ int ovf_prepare(float *sm, uint32_t *ovf, int nrec, floa
             if ((ab >> 26) & 1u) bl[a] = (uint8_t)lvl;
             if ((ab >> 27) & 1u) bl[b] = (uint8_t)lvl;
             *w = ab | ((uint32_t)lvl << 19);
-            max_level = max(max_level, lvl);
+            cmax = max(cmax, lvl);
         }
     }
     __threadfence_block();
     g.sync();
-    max_level = g.shfl(max_level, 0);
-    for (int base = G; base < nrec; base += G) {
+    cmax = g.shfl(cmax, 0);
+    // pre-step of every pair; accumulated impulses of the previous step come from the lane that
+    // owned the pair then (first manifold in its registers, second in its shared-memory fields)
+    // or from the warm entries in scratch
+    for (int base = 0; base < nrec; base += G) {
         const int k = base + lane;
         const bool valid = k < nrec;
-        uint32_t *r = ovf + (size_t)(valid ? k - G : 0) * kRecWords;
+        uint32_t *r = ovf + (size_t)(valid ? k : 0) * kRecWords;
         uint32_t ab = 0u;
         int wi = 255;
         if (valid) { ab = r[S_AB]; wi = widx[(ab >> 12) & 127]; }
         const int src = (wi < G) ? wi : 0;
-        float w[4] = { g.shflf(old0, src), g.shflf(old1, src), g.shflf(old2, src), g.shflf(old3, src) };
+        float w[4] = { g.shflf(old_n, src), g.shflf(old_t, src), lanef[kStageWords * G + src], lanef[(kStageWords + 1) * G + src] };
         if (wi >= G && wi != 255) {
-            const uint32_t *wr = ovf + (size_t)SC::OVF_MAX * kRecWords + (size_t)(wi - G) * kWarmWords;
+            const uint32_t *wr = ovf + SC::SCRATCH_WARM + (size_t)wi * kWarmWords;
 #pragma unroll
             for (int q = 0; q < 4; ++q) w[q] = __uint_as_float(wr[1 + q]);
         }
         if (wi == 255 || !warm_start) { w[0] = 0.0f; w[1] = 0.0f; w[2] = 0.0f; w[3] = 0.0f; }
         if (valid) {
-            const float nx = __uint_as_float(r[S_NX]), ny = __uint_as_float(r[S_NY]);
+            RecM c;
+            c.ab = ab; c.nx = __uint_as_float(r[S_NX]); c.ny = __uint_as_float(r[S_NY]);
             const float pt[6] = { __uint_as_float(r[S_PX0]), __uint_as_float(r[S_PY0]), __uint_as_float(r[S_PEN0]),
                                   __uint_as_float(r[S_PX1]), __uint_as_float(r[S_PY1]), __uint_as_float(r[S_PEN1]) };
-            Rec c;
-            build_record<SC>(c, ab, nx, ny, pt, w, sm, cc);
-            rec_store(r, c);
+            const int a = ab & 31, b = (ab >> 5) & 31;
+            const float ma = sm[SC::BIM + a], mb = sm[SC::BIM + b], ia = sm[SC::BII + a], ib = sm[SC::BII + b];
+            const float fra = sm[SC::BFR + a], frb = sm[SC::BFR + b];
+            const float er = fmin_cmp(sm[SC::BRE + a], sm[SC::BRE + b]);
+            c.mu = sqrtf(__fmaf_rn(fra, fra, frb * frb));
+#pragma unroll
+            for (int mi = 0; mi < 2; ++mi) {
+                if ((ab >> 10) & (1u << mi)) {
+                    prestep_manifold<SC>(a, b, c.nx, c.ny, ma, mb, ia, ib, pt[3 * mi], pt[3 * mi + 1], pt[3 * mi + 2], er, sm, cc,
+                                         c.rna[mi], c.rnb[mi], c.rta[mi], c.rtb[mi], c.massn[mi], c.masst[mi], c.target[mi], c.corr[mi]);
+                    c.accn[mi] = w[2 * mi]; c.acct[mi] = w[2 * mi + 1];
+                } else {
+                    c.rna[mi] = 0.0f; c.rnb[mi] = 0.0f; c.rta[mi] = 0.0f; c.rtb[mi] = 0.0f; c.massn[mi] = 0.0f; c.masst[mi] = 0.0f;
+                    c.target[mi] = 0.0f; c.corr[mi] = 0.0f; c.accn[mi] = 0.0f; c.acct[mi] = 0.0f;
+                }
+            }
+            recm_store(r, c);
         }
     }
     g.sync();
-    return max_level;
-}
-
-// One level of one sweep over records G..nrec-1.
-template <class SC, int G>
-__device__ __noinline__ void ovf_visit(float *sm, uint32_t *ovf, int nrec, int lvl, int mode) {
-    Group<G> g;
-    for (int k = G + g.lane; k < nrec; k += G) {
-        uint32_t *r = ovf + (size_t)(k - G) * kRecWords;
-        if (((r[R_AB] >> 19) & 127u) != (unsigned)lvl) continue;
-        Rec c;
-        rec_load(r, c, sm + SC::BIM, sm + SC::BII);
-        if (mode == 0) visit_pair<SC, 0>(c, sm);
-        else if (mode == 1) {
-            visit_pair<SC, 1>(c, sm);
-#pragma unroll
-            for (int mi = 0; mi < 2; ++mi) {
-                r[R_M0 + mi * M_WORDS + M_ACCN] = __float_as_uint(c.accn[mi]);
-                r[R_M0 + mi * M_WORDS + M_ACCT] = __float_as_uint(c.acct[mi]);
-            }
-        } else visit_pair<SC, 2>(c, sm);
+    slow_sweep_pairs<SC, G, 0>(sm, ovf, nrec, cmax);
+    sweep_joints<SC, G, 0>(sm, jab, lane, jlevel, jmax, lv, motor_rho);
+    for (int it = 0; it < solver_iters; ++it) {
+        sweep_joints<SC, G, 1>(sm, jab, lane, jlevel, jmax, lv, motor_rho);
+        slow_sweep_pairs<SC, G, 1>(sm, ovf, nrec, cmax);
     }
+    return cmax;
 }
 
-// End of a step: the accumulated impulses of records G..nrec-1 become warm entries, the pair index
-// table learns where they are; returns this group's number of active manifolds among them.
 template <class SC, int G>
-__device__ __noinline__ int ovf_finish(float *sm, uint32_t *ovf, int nrec) {
+__device__ __noinline__ void slow_correct(float *sm, uint32_t *ovf, int nrec, int cmax) {
+    slow_sweep_pairs<SC, G, 2>(sm, ovf, nrec, cmax);
+}
+
+// End of an overflow step: every pair's accumulated impulses become warm entries in scratch and the
+// pair index table learns where they are; returns the number of active manifolds.
+template <class SC, int G>
+__device__ __noinline__ int slow_finish(float *sm, uint32_t *ovf, int nrec) {
     Group<G> g;
     uint8_t *widx = reinterpret_cast<uint8_t *>(reinterpret_cast<uint32_t *>(sm) + SC::WIDX);
     int nman = 0;
-    for (int k = G + g.lane; k < nrec; k += G) {
-        const uint32_t *r = ovf + (size_t)(k - G) * kRecWords;
-        uint32_t *wr = ovf + (size_t)SC::OVF_MAX * kRecWords + (size_t)(k - G) * kWarmWords;
+    for (int k = g.lane; k < nrec; k += G) {
+        const uint32_t *r = ovf + (size_t)k * kRecWords;
+        uint32_t *wr = ovf + SC::SCRATCH_WARM + (size_t)k * kWarmWords;
         const uint32_t ab = r[R_AB];
         const int p = (ab >> 12) & 127;
         const unsigned am = (ab >> 10) & 3u;
@@ -454,26 +548,28 @@ __device__ __noinline__ int ovf_finish(float *sm, uint32_t *ovf, int nrec) {
         widx[p] = (uint8_t)k;
         nman += __popc(am);
     }
-    return g.sum_int(nman);
+    nman = g.sum_int(nman);
+    g.sync();
+    return nman;
 }
 
 // Launch boundaries: warm entries G.. between the state record and the scratch.
 template <class SC, int G>
-__device__ __noinline__ void ovf_warm_in(float *sm, uint32_t *ovf, const uint32_t *st_warm, int nwarm) {
+__device__ __noinline__ void warm_in(float *sm, uint32_t *ovf, const uint32_t *st_warm, int nwarm) {
     Group<G> g;
     uint8_t *widx = reinterpret_cast<uint8_t *>(reinterpret_cast<uint32_t *>(sm) + SC::WIDX);
     for (int k = G + g.lane; k < nwarm; k += G) {
-        uint32_t *wr = ovf + (size_t)SC::OVF_MAX * kRecWords + (size_t)(k - G) * kWarmWords;
+        uint32_t *wr = ovf + SC::SCRATCH_WARM + (size_t)k * kWarmWords;
 #pragma unroll
         for (int q = 0; q < kWarmWords; ++q) wr[q] = st_warm[kWarmWords * k + q];
         widx[wr[0]] = (uint8_t)k;
     }
 }
 template <class SC, int G>
-__device__ __noinline__ void ovf_warm_out(const uint32_t *ovf, uint32_t *st_warm, int nwarm) {
+__device__ __noinline__ void warm_out(const uint32_t *ovf, uint32_t *st_warm, int nwarm) {
     Group<G> g;
     for (int k = G + g.lane; k < nwarm; k += G) {
-        const uint32_t *wr = ovf + (size_t)SC::OVF_MAX * kRecWords + (size_t)(k - G) * kWarmWords;
+        const uint32_t *wr = ovf + SC::SCRATCH_WARM + (size_t)k * kWarmWords;
 #pragma unroll
         for (int q = 0; q < kWarmWords; ++q) st_warm[kWarmWords * k + q] = wr[q];
     }
@@ -482,7 +578,7 @@ __device__ __noinline__ void ovf_warm_out(const uint32_t *ovf, uint32_t *st_warm
 // ---------------------------------------------------------------- scene processing
 template <class SC, int G>
 struct Scene {
-    static_assert(SC::J <= G && SC::T <= G && kMaxActions <= 32, "one lane per joint / thruster");
+    static_assert(SC::J <= G && SC::T <= G && kMaxActions <= 2 * G, "one lane per joint / thruster");
     float *sm;            // this scene's shared-memory region
     uint32_t *smu;
     const uint16_t *ptab; // block-shared pair table
@@ -492,7 +588,6 @@ struct Scene {
     int lane;
     // state a lane keeps in registers from step to step
     Rec rec;              // contact pair record number `lane` of the latest step (its accumulated impulses warm-start the next)
-    JointRow jr;          // joint number `lane`
     uint32_t jab;         // packed word of joint number `lane` (0 beyond the last joint)
     unsigned c_surv, c_rec, c_man;   // packed work counters: pp | pc << 16, cc | active pairs << 16, manifolds | env-steps << 16
 
@@ -504,6 +599,8 @@ struct Scene {
     __device__ __forceinline__ uint8_t *surv() { return reinterpret_cast<uint8_t *>(smu + SC::SURV); }
     __device__ __forceinline__ uint8_t *widx() { return reinterpret_cast<uint8_t *>(smu + SC::WIDX); }
     __device__ __forceinline__ float4 &box4(int i) { return *reinterpret_cast<float4 *>(sm + SC::BOX + 4 * i); }
+    // this lane's word of per-lane field f
+    __device__ __forceinline__ float &lanef(int f) { return sm[SC::STG + f * G + lane]; }
     __device__ __forceinline__ ContactConsts contact_consts() const {
         ContactConsts cc; cc.slop = prm.slop; cc.rest_thr = prm.rest_thr; cc.alpha = prm.contact_alpha; cc.beta = prm.contact_beta; return cc;
     }
@@ -535,7 +632,7 @@ struct Scene {
     }
     __device__ __forceinline__ void load_level_pose(const uint32_t *lv) {
         for (int i = lane; i < 6 * SC::N; i += G) smu[SC::BX + i] = lv[SC::LV_X + i];
-        jr.accx = 0.0f; jr.accy = 0.0f;
+        if (SC::J > 0 && lane < SC::J) { sm[SC::JROW + JR_ACCX * SC::J + lane] = 0.0f; sm[SC::JROW + JR_ACCY * SC::J + lane] = 0.0f; }
         for (int i = lane; i < (SC::NPAIRS + 3) / 4; i += G) smu[SC::WIDX + i] = 0xffffffffu;
     }
 
@@ -664,81 +761,50 @@ struct Scene {
         return m.pen > 0.0f ? 1u : 0u;
     }
 
-    // ---- joints.  MODE 0: warm start, 1: solver iteration, 2: positional correction, 3: motor
+    // ---- one visit of this lane's contact pair record.  MODE 0: warm start, 1: solver iteration, 2: positional correction
     template <int MODE>
-    __device__ __forceinline__ void visit_joint(const uint32_t *lv) {
-        const int a = jab & 255, b = (jab >> 8) & 255;
-        const bool dyn_a = smu[SC::BFL + a] & F_DYNAMIC, dyn_b = smu[SC::BFL + b] & F_DYNAMIC;
-        if (MODE == 3) {
-            const float A = fmax_cmp(fmin_cmp(sm[SC::ACT + ((jab >> 16) & 255)], 1.0f), -1.0f);
-            const float speed = __uint_as_float(lv[SC::LV_JOINT + 8 * lane + 5]), power = __uint_as_float(lv[SC::LV_JOINT + 8 * lane + 6]);
-            const float wa = sm[SC::BW + a], wb = sm[SC::BW + b];
-            const float arg = __fmaf_rn(-speed, A, wa - wb) * prm.motor_rho;
-            const float jr_ = power * tanh_spec(arg);
-            if (dyn_a) sm[SC::BW + a] = __fmaf_rn(-jr_, sm[SC::BII + a], wa);
-            if (dyn_b) sm[SC::BW + b] = __fmaf_rn(jr_, sm[SC::BII + b], wb);
-            return;
-        }
-        const float ma = sm[SC::BIM + a], mb = sm[SC::BIM + b];
+    __device__ __forceinline__ void visit_pair() {
+        const uint32_t ab = rec.ab;
+        const int a = ab & 31, b = (ab >> 5) & 31;
+        const unsigned amask = (ab >> 10) & 3u;
+        const bool dyn_a = (ab >> 26) & 1u, dyn_b = (ab >> 27) & 1u;
         if (MODE == 2) {
-            const float cx = jr.cx, cy = jr.cy;
-            if (dyn_a) { sm[SC::BX + a] = __fmaf_rn(ma, cx, sm[SC::BX + a]); sm[SC::BY + a] = __fmaf_rn(ma, cy, sm[SC::BY + a]); }
-            if (dyn_b) { sm[SC::BX + b] = __fmaf_rn(-mb, cx, sm[SC::BX + b]); sm[SC::BY + b] = __fmaf_rn(-mb, cy, sm[SC::BY + b]); }
+            correct_pair(sm + SC::BX, sm + SC::BY, a, b, amask, dyn_a, dyn_b, rec.nx, rec.ny, rec.ma, rec.mb,
+                         lanef(kStageWords + 2), lanef(kStageWords + 3));
             return;
         }
-        const float ia = sm[SC::BII + a], ib = sm[SC::BII + b];
-        const float rax = jr.rax, ray = jr.ray, rbx = jr.rbx, rby = jr.rby;
         float vax = sm[SC::BVX + a], vay = sm[SC::BVY + a], wa = sm[SC::BW + a];
         float vbx = sm[SC::BVX + b], vby = sm[SC::BVY + b], wb = sm[SC::BW + b];
-        float lx, ly;
-        if (MODE == 0) { lx = jr.accx; ly = jr.accy; }
-        else {
-            const float cx = __fmaf_rn(-wb, rby, vbx) - __fmaf_rn(-wa, ray, vax);
-            const float cy = __fmaf_rn(wb, rbx, vby) - __fmaf_rn(wa, rax, vay);
-            const float rx = -(cx + jr.bx), ry = -(cy + jr.by);
-            lx = __fmaf_rn(jr.i11, rx, jr.i12 * ry);
-            ly = __fmaf_rn(jr.i12, rx, jr.i22 * ry);
-            jr.accx = jr.accx + lx;
-            jr.accy = jr.accy + ly;
+        if (amask & 1u)
+            manifold_rows<MODE>(rec.nx, rec.ny, rec.mu, rec.ma, rec.mb, rec.ia, rec.ib, rec.rna, rec.rnb, rec.rta, rec.rtb,
+                                rec.massn, rec.masst, rec.target, rec.accn, rec.acct, vax, vay, wa, vbx, vby, wb);
+        if (amask & 2u) {
+            float accn = lanef(kStageWords), acct = lanef(kStageWords + 1);
+            manifold_rows<MODE>(rec.nx, rec.ny, rec.mu, rec.ma, rec.mb, rec.ia, rec.ib, lanef(M2_RNA), lanef(M2_RNB), lanef(M2_RTA),
+                                lanef(M2_RTB), lanef(M2_MASSN), lanef(M2_MASST), lanef(M2_TARGET), accn, acct, vax, vay, wa, vbx, vby, wb);
+            if (MODE == 1) { lanef(kStageWords) = accn; lanef(kStageWords + 1) = acct; }
         }
-        if (dyn_a) {
-            sm[SC::BVX + a] = __fmaf_rn(-ma, lx, vax); sm[SC::BVY + a] = __fmaf_rn(-ma, ly, vay);
-            sm[SC::BW + a] = __fmaf_rn(-ia, cross2(rax, ray, lx, ly), wa);
-        }
-        if (dyn_b) {
-            sm[SC::BVX + b] = __fmaf_rn(mb, lx, vbx); sm[SC::BVY + b] = __fmaf_rn(mb, ly, vby);
-            sm[SC::BW + b] = __fmaf_rn(ib, cross2(rbx, rby, lx, ly), wb);
-        }
+        if (dyn_a) { sm[SC::BVX + a] = vax; sm[SC::BVY + a] = vay; sm[SC::BW + a] = wa; }
+        if (dyn_b) { sm[SC::BVX + b] = vbx; sm[SC::BVY + b] = vby; sm[SC::BW + b] = wb; }
     }
-
-    // joints of one level touch disjoint movable bodies; levels in order keep the joint order
+    // records of one level touch disjoint movable bodies; levels in order keep the record order
     template <int MODE>
-    __device__ __forceinline__ void sweep_joints(int jmax, int jlevel, const uint32_t *lv) {
-        if (SC::J == 0) return;
-#pragma unroll 1
-        for (int lvl = 1; lvl <= jmax; ++lvl) {
-            if (jlevel == lvl) visit_joint<MODE>(lv);
-            g.sync();
-        }
-    }
-    template <int MODE>
-    __device__ __forceinline__ void sweep_pairs(int nrec, int cmax, int clevel) {
+    __device__ __forceinline__ void sweep_pairs(int cmax, int clevel) {
 #pragma unroll 1
         for (int lvl = 1; lvl <= cmax; ++lvl) {
-            if (clevel == lvl) visit_pair<SC, MODE>(rec, sm);
-            if (nrec > G) ovf_visit<SC, G>(sm, ovf, nrec, lvl, MODE);
+            if (clevel == lvl) visit_pair<MODE>();
             g.sync();
         }
     }
 
-    // ---- one environment step.  meta[]: step_count, episode_count, level_id, status, number of warm entries
-    __device__ __forceinline__ void step(int e, int s, int (&meta)[5]) {
-        const uint32_t *lv = prm.levels + (size_t)meta[2] * SC::LV_WORDS;
+    // ---- one environment step
+    __device__ __forceinline__ void step(int e, int s) {
         // frozen env: reports done, nothing else
-        if (meta[3] & 1) {
+        if (smu[SC::META + META_STATUS] & 1u) {
             if (lane == 0) { prm.reward[(size_t)s * prm.n_envs + e] = 0.0f; prm.done[(size_t)s * prm.n_envs + e] = 1; }
             return;
         }
+        const uint32_t *lv = prm.levels + (size_t)smu[SC::META + META_LEVEL] * SC::LV_WORDS;
         // actions of this step
         if (lane < prm.n_actions) sm[SC::ACT + lane] = prm.actions[((size_t)s * prm.n_envs + e) * prm.n_actions + lane];
         if (G < kMaxActions && lane + G < prm.n_actions) sm[SC::ACT + lane + G] = prm.actions[((size_t)s * prm.n_envs + e) * prm.n_actions + lane + G];
@@ -786,7 +852,7 @@ struct Scene {
             box4(i) = make_float4(x0, y0, x1, y1);
         }
         // motors (joint order), thrusters (thruster order)
-        sweep_joints<3>(jmax, jlevel, lv);
+        sweep_joints<SC, G, 3>(sm, jab, lane, jlevel, jmax, lv, prm.motor_rho);
         if (SC::T > 0) {
             int tl = 0; uint32_t tp = 0u;
             if (lane < SC::T) { tp = lv[SC::LV_THR + 8 * lane]; if ((tp >> 16) & 1u) tl = (tp >> 17) & 7u; }
@@ -811,9 +877,10 @@ struct Scene {
                 g.sync();
             }
         }
-        // joint pre-step (poses only; velocities are not read)
+        // joint pre-step (poses only; velocities are not read): the row goes to shared memory
         if (SC::J > 0 && lane < SC::J) {
-            if (!((jab >> 24) & 1u) || !prm.warm_start) { jr.accx = 0.0f; jr.accy = 0.0f; }
+            float *jr = sm + SC::JROW + lane;
+            if (!((jab >> 24) & 1u) || !prm.warm_start) { jr[JR_ACCX * SC::J] = 0.0f; jr[JR_ACCY * SC::J] = 0.0f; }
             if ((jab >> 24) & 1u) {
                 const int a = jab & 255, b = (jab >> 8) & 255;
                 const uint32_t *jl = lv + SC::LV_JOINT + 8 * lane;
@@ -828,11 +895,11 @@ struct Scene {
                 float k12 = -((ia * rax) * ray); k12 = __fmaf_rn(-(ib * rbx), rby, k12);
                 const float det = __fmaf_rn(k11, k22, -(k12 * k12));
                 const float inv_det = 1.0f / det;
-                jr.rax = rax; jr.ray = ray; jr.rbx = rbx; jr.rby = rby;
-                jr.i11 = k22 * inv_det; jr.i22 = k11 * inv_det; jr.i12 = -(k12 * inv_det);
-                jr.bx = prm.joint_alpha * gx; jr.by = prm.joint_alpha * gy;
+                jr[JR_RAX * SC::J] = rax; jr[JR_RAY * SC::J] = ray; jr[JR_RBX * SC::J] = rbx; jr[JR_RBY * SC::J] = rby;
+                jr[JR_I11 * SC::J] = k22 * inv_det; jr[JR_I22 * SC::J] = k11 * inv_det; jr[JR_I12 * SC::J] = -(k12 * inv_det);
+                jr[JR_BX * SC::J] = prm.joint_alpha * gx; jr[JR_BY * SC::J] = prm.joint_alpha * gy;
                 const float share = prm.joint_beta / msum;
-                jr.cx = share * gx; jr.cy = share * gy;
+                jr[JR_CX * SC::J] = share * gx; jr[JR_CY * SC::J] = share * gy;
             }
         }
         g.sync();
@@ -842,7 +909,7 @@ struct Scene {
         {
             int mine_pp = 0, mine_pc = 0;     // this lane's survivors below the polygon-circle / circle-circle boundary
             const float mg = prm.aabb_margin;
-#pragma unroll 1
+#pragma unroll 2
             for (int base = 0; base < SC::NPAIRS; base += G) {
                 const int p = base + lane;
                 bool keep = false;
@@ -915,7 +982,7 @@ struct Scene {
                         st[S_PX0 * G] = m[0].px; st[S_PY0 * G] = m[0].py; st[S_PEN0 * G] = m[0].pen;
                         st[S_PX1 * G] = m[1].px; st[S_PY1 * G] = m[1].py; st[S_PEN1 * G] = m[1].pen;
                     } else {
-                        uint32_t *st = ovf + (size_t)(k - G) * kRecWords;
+                        uint32_t *st = ovf + (size_t)k * kRecWords;
                         st[S_AB] = ab; st[S_NX] = __float_as_uint(nx); st[S_NY] = __float_as_uint(ny);
                         st[S_PX0] = __float_as_uint(m[0].px); st[S_PY0] = __float_as_uint(m[0].py); st[S_PEN0] = __float_as_uint(m[0].pen);
                         st[S_PX1] = __float_as_uint(m[1].px); st[S_PY1] = __float_as_uint(m[1].py); st[S_PEN1] = __float_as_uint(m[1].pen);
@@ -926,63 +993,87 @@ struct Scene {
         }
         const bool touch_gb = g.any(t_gb), touch_gr = g.any(t_gr);
         g.sync();
+        c_rec += (unsigned)nrec << 16;
 
-        // every staged pair becomes a record in its own lane: accumulated impulses of the same pair in the
-        // previous step come from the lane that owned it then
-        const ContactConsts cc = contact_consts();
-        const float old0 = rec.accn[0], old1 = rec.acct[0], old2 = rec.accn[1], old3 = rec.acct[1];
-        int cmax = 0;
-        if (nrec > G) cmax = ovf_prepare<SC, G>(sm, ovf, nrec, old0, old1, old2, old3, prm.warm_start, cc);
-        {
+        const bool overflow = nrec > G;
+        int cmax = 0, clevel = 0;
+        if (overflow) {
+            cmax = slow_solve<SC, G>(sm, ovf, lv, nrec, jab, jlevel, jmax, prm.solver_iters, prm.warm_start, prm.motor_rho,
+                                     rec.accn, rec.acct, contact_consts());
+        } else {
+            // every staged pair becomes a record in its own lane: accumulated impulses of the same pair in the
+            // previous step come from the lane that owned it then
+            const ContactConsts cc = contact_consts();
             const bool mine = lane < nrec;
             uint32_t ab = 0u;
             int wi = 255;
-            if (mine) { ab = smu[SC::STG + S_AB * G + lane]; wi = widx()[(ab >> 12) & 127]; }
+            float nx = 0.0f, ny = 0.0f, pt[6] = { 0.0f, 0.0f, 0.0f, 0.0f, 0.0f, 0.0f };
+            if (mine) {
+                ab = __float_as_uint(lanef(S_AB)); wi = widx()[(ab >> 12) & 127];
+                nx = lanef(S_NX); ny = lanef(S_NY);
+                pt[0] = lanef(S_PX0); pt[1] = lanef(S_PY0); pt[2] = lanef(S_PEN0); pt[3] = lanef(S_PX1); pt[4] = lanef(S_PY1); pt[5] = lanef(S_PEN1);
+            }
             const int src = (wi < G) ? wi : 0;
-            float w[4] = { g.shflf(old0, src), g.shflf(old1, src), g.shflf(old2, src), g.shflf(old3, src) };
+            float w[4] = { g.shflf(rec.accn, src), g.shflf(rec.acct, src), sm[SC::STG + kStageWords * G + src], sm[SC::STG + (kStageWords + 1) * G + src] };
             if (wi >= G && wi != 255) {
-                const uint32_t *wr = ovf + (size_t)SC::OVF_MAX * kRecWords + (size_t)(wi - G) * kWarmWords;
+                const uint32_t *wr = ovf + SC::SCRATCH_WARM + (size_t)wi * kWarmWords;
 #pragma unroll
                 for (int q = 0; q < 4; ++q) w[q] = __uint_as_float(wr[1 + q]);
             }
             if (wi == 255 || !prm.warm_start) { w[0] = 0.0f; w[1] = 0.0f; w[2] = 0.0f; w[3] = 0.0f; }
-            if (mine) {
-                const float *st = sm + SC::STG + lane;
-                const float pt[6] = { st[S_PX0 * G], st[S_PY0 * G], st[S_PEN0 * G], st[S_PX1 * G], st[S_PY1 * G], st[S_PEN1 * G] };
-                build_record<SC>(rec, ab, st[S_NX * G], st[S_NY * G], pt, w, sm, cc);
-            } else rec.ab = 0u;
-        }
-        // levels of the records (canonical order = record order): one more than the highest level of an
-        // earlier record that shares a movable body
-        if (nrec <= G) {
-            const uint32_t my_ab = rec.ab;
-            int lvl = (lane < nrec) ? 1 : 0;
-            const int a = my_ab & 31, b = (my_ab >> 5) & 31;
-            const bool da = (my_ab >> 26) & 1u, db = (my_ab >> 27) & 1u;
-#pragma unroll 1
-            for (int q = 0; q + 1 < nrec; ++q) {
-                const uint32_t abq = g.shflu(my_ab, q);
-                const int lq = g.shfl(lvl, q);
-                const int aq = abq & 31, bq = (abq >> 5) & 31;
-                const bool hit = (da && (a == aq || a == bq)) || (db && (b == aq || b == bq));
-                if (q < lane && lane < nrec && hit) lvl = max(lvl, lq + 1);
+            g.sync();     // every lane has read the fields it needs from other lanes before they are rewritten
+            const int a = ab & 31, b = (ab >> 5) & 31;
+            const unsigned amask = (ab >> 10) & 3u;
+            rec.ab = ab; rec.nx = nx; rec.ny = ny;
+            rec.ma = sm[SC::BIM + a]; rec.mb = sm[SC::BIM + b]; rec.ia = sm[SC::BII + a]; rec.ib = sm[SC::BII + b];
+            const float fra = sm[SC::BFR + a], frb = sm[SC::BFR + b];
+            const float er = fmin_cmp(sm[SC::BRE + a], sm[SC::BRE + b]);
+            rec.mu = sqrtf(__fmaf_rn(fra, fra, frb * frb));
+            float corr0 = 0.0f, corr1 = 0.0f;
+            rec.rna = 0.0f; rec.rnb = 0.0f; rec.rta = 0.0f; rec.rtb = 0.0f; rec.massn = 0.0f; rec.masst = 0.0f; rec.target = 0.0f;
+            rec.accn = 0.0f; rec.acct = 0.0f;
+            if (amask & 1u) {
+                prestep_manifold<SC>(a, b, nx, ny, rec.ma, rec.mb, rec.ia, rec.ib, pt[0], pt[1], pt[2], er, sm, cc,
+                                     rec.rna, rec.rnb, rec.rta, rec.rtb, rec.massn, rec.masst, rec.target, corr0);
+                rec.accn = w[0]; rec.acct = w[1];
             }
-            rec.ab = my_ab | ((uint32_t)lvl << 19);
-            cmax = g.max_int(lvl);
-        }
-        const int clevel = (int)((rec.ab >> 19) & 127u);
-        const unsigned am_mine = (rec.ab >> 10) & 3u;
-        c_man += (unsigned)(__popc(g.ballot(am_mine & 1u)) + __popc(g.ballot(am_mine & 2u)));
-        c_rec += (unsigned)nrec << 16;
-
-        // warm start: contacts, then joints
-        sweep_pairs<0>(nrec, cmax, clevel);
-        sweep_joints<0>(jmax, jlevel, lv);
-        // solver iterations: joints, then contacts
+            float acc2n = 0.0f, acc2t = 0.0f;
+            if (amask & 2u) {
+                float rna, rnb, rta, rtb, massn, masst, target;
+                prestep_manifold<SC>(a, b, nx, ny, rec.ma, rec.mb, rec.ia, rec.ib, pt[3], pt[4], pt[5], er, sm, cc,
+                                     rna, rnb, rta, rtb, massn, masst, target, corr1);
+                lanef(M2_RNA) = rna; lanef(M2_RNB) = rnb; lanef(M2_RTA) = rta; lanef(M2_RTB) = rtb;
+                lanef(M2_MASSN) = massn; lanef(M2_MASST) = masst; lanef(M2_TARGET) = target;
+                acc2n = w[2]; acc2t = w[3];
+            }
+            lanef(kStageWords) = acc2n; lanef(kStageWords + 1) = acc2t;
+            lanef(kStageWords + 2) = corr0; lanef(kStageWords + 3) = corr1;
+            // levels of the records (canonical order = record order): one more than the highest level of an
+            // earlier record that shares a movable body
+            {
+                int lvl = mine ? 1 : 0;
+                const bool da = (ab >> 26) & 1u, db = (ab >> 27) & 1u;
 #pragma unroll 1
-        for (int it = 0; it < prm.solver_iters; ++it) {
-            sweep_joints<1>(jmax, jlevel, lv);
-            sweep_pairs<1>(nrec, cmax, clevel);
+                for (int q = 0; q + 1 < nrec; ++q) {
+                    const uint32_t abq = g.shflu(ab, q);
+                    const int lq = g.shfl(lvl, q);
+                    const int aq = abq & 31, bq = (abq >> 5) & 31;
+                    const bool hit = (da && (a == aq || a == bq)) || (db && (b == aq || b == bq));
+                    if (q < lane && mine && hit) lvl = max(lvl, lq + 1);
+                }
+                clevel = lvl;
+                cmax = g.max_int(lvl);
+            }
+            c_man += (unsigned)(__popc(g.ballot(amask & 1u)) + __popc(g.ballot(amask & 2u)));
+            // warm start: contacts, then joints
+            sweep_pairs<0>(cmax, clevel);
+            sweep_joints<SC, G, 0>(sm, jab, lane, jlevel, jmax, lv, prm.motor_rho);
+            // solver iterations: joints, then contacts
+#pragma unroll 1
+            for (int it = 0; it < prm.solver_iters; ++it) {
+                sweep_joints<SC, G, 1>(sm, jab, lane, jlevel, jmax, lv, prm.motor_rho);
+                sweep_pairs<1>(cmax, clevel);
+            }
         }
         // Euler step with the solved velocities
         for (int i = lane; i < SC::N; i += G) {
@@ -993,8 +1084,9 @@ struct Scene {
             }
         }
         g.sync();
-        sweep_pairs<2>(nrec, cmax, clevel);
-        sweep_joints<2>(jmax, jlevel, lv);
+        if (overflow) slow_correct<SC, G>(sm, ovf, nrec, cmax);
+        else sweep_pairs<2>(cmax, clevel);
+        sweep_joints<SC, G, 2>(sm, jab, lane, jlevel, jmax, lv, prm.motor_rho);
         bool finite = true;
         for (int i = lane; i < SC::N; i += G)
             finite = finite && finite_bits(sm[SC::BX + i]) && finite_bits(sm[SC::BY + i]) && finite_bits(sm[SC::BTH + i]) &&
@@ -1003,34 +1095,47 @@ struct Scene {
 
         // where the pairs of this step keep their accumulated impulses for the next one
         for (int i = lane; i < (SC::NPAIRS + 3) / 4; i += G) smu[SC::WIDX + i] = 0xffffffffu;
+        const int step_count = (int)smu[SC::META + META_STEP] + 1;
         g.sync();
-        if (lane < nrec) widx()[(rec.ab >> 12) & 127] = (uint8_t)lane;
-        if (nrec > G) c_man += (unsigned)ovf_finish<SC, G>(sm, ovf, nrec);
-        meta[4] = nrec;
+        if (overflow) {
+            c_man += (unsigned)slow_finish<SC, G>(sm, ovf, nrec);
+            // the first G pairs go back to their lanes
+            const uint32_t *wr = ovf + SC::SCRATCH_WARM + (size_t)lane * kWarmWords;
+            rec.ab = wr[0] << 12;
+            rec.accn = __uint_as_float(wr[1]); rec.acct = __uint_as_float(wr[2]);
+            lanef(kStageWords) = __uint_as_float(wr[3]); lanef(kStageWords + 1) = __uint_as_float(wr[4]);
+        } else if (lane < nrec) widx()[(rec.ab >> 12) & 127] = (uint8_t)lane;
 
         // reward, termination, counters, auto-reset
-        meta[0] += 1;
-        const bool timeout = prm.max_episode_steps > 0 && meta[0] >= prm.max_episode_steps;
+        const bool timeout = prm.max_episode_steps > 0 && step_count >= prm.max_episode_steps;
         float reward = (float)((int)touch_gb - (int)touch_gr);
         bool done = touch_gb || touch_gr || timeout;
-        if (!finite) { reward = 0.0f; done = true; meta[3] |= 1; if (lane == 0) atomicAdd(prm.counters + 0, 1ULL); }
+        if (!finite) { reward = 0.0f; done = true; }
         if (lane == 0) {
             prm.reward[(size_t)s * prm.n_envs + e] = reward;
             prm.done[(size_t)s * prm.n_envs + e] = done ? 1 : 0;
+            smu[SC::META + META_STEP] = (uint32_t)step_count;
+            smu[SC::META + META_NWARM] = (uint32_t)nrec;
+            if (!finite) { smu[SC::META + META_STATUS] |= 1u; atomicAdd(prm.counters + 0, 1ULL); }
         }
         c_man += 1u << 16;
         g.sync();
         if (done && prm.auto_reset != 0) {
-            meta[1] += 1;
+            const int episode = (int)smu[SC::META + META_EPISODE] + 1;
+            int level = (int)smu[SC::META + META_LEVEL];
+            g.sync();
             if (prm.auto_reset == 2) {
                 const unsigned long long h = mix64(prm.seed + ((unsigned long long)(prm.env_offset + e) + 1ULL) * 0x9E3779B97F4A7C15ULL +
-                                                   (unsigned long long)meta[1] * 0xD1B54A32D192ED03ULL);
+                                                   (unsigned long long)episode * 0xD1B54A32D192ED03ULL);
                 const int nl = (int)(h % (unsigned long long)prm.n_levels);
-                if (nl != meta[2]) { meta[2] = nl; load_level_consts(prm.levels + (size_t)nl * SC::LV_WORDS); }
+                if (nl != level) { level = nl; load_level_consts(prm.levels + (size_t)nl * SC::LV_WORDS); }
             }
-            load_level_pose(prm.levels + (size_t)meta[2] * SC::LV_WORDS);
-            meta[0] = 0; meta[3] = 0; meta[4] = 0;
-            if (lane == 0) atomicAdd(prm.counters + 1, 1ULL);
+            load_level_pose(prm.levels + (size_t)level * SC::LV_WORDS);
+            if (lane == 0) {
+                smu[SC::META + META_STEP] = 0u; smu[SC::META + META_EPISODE] = (uint32_t)episode; smu[SC::META + META_LEVEL] = (uint32_t)level;
+                smu[SC::META + META_STATUS] = 0u; smu[SC::META + META_NWARM] = 0u;
+                atomicAdd(prm.counters + 1, 1ULL);
+            }
             g.sync();
         }
     }
@@ -1038,47 +1143,52 @@ struct Scene {
     // ---- whole launch for one scene
     __device__ __forceinline__ void run(int e) {
         uint32_t *st = prm.state + (size_t)e * SC::ST_WORDS;
-        int meta[5];
-#pragma unroll
-        for (int i = 0; i < 5; ++i) meta[i] = (int)st[SC::ST_META + i];
         for (int i = lane; i < 6 * SC::N; i += G) smu[SC::BX + i] = st[SC::ST_BODY + i];
-        jr.accx = 0.0f; jr.accy = 0.0f;
-        if (SC::J > 0 && lane < SC::J) { jr.accx = __uint_as_float(st[SC::ST_JACC + 2 * lane]); jr.accy = __uint_as_float(st[SC::ST_JACC + 2 * lane + 1]); }
+        if (lane < 5) smu[SC::META + lane] = st[SC::ST_META + lane];
+        if (SC::J > 0 && lane < SC::J) {
+            smu[SC::JROW + JR_ACCX * SC::J + lane] = st[SC::ST_JACC + 2 * lane];
+            smu[SC::JROW + JR_ACCY * SC::J + lane] = st[SC::ST_JACC + 2 * lane + 1];
+        }
         for (int i = lane; i < (SC::NPAIRS + 3) / 4; i += G) smu[SC::WIDX + i] = 0xffffffffu;
-        load_level_consts(prm.levels + (size_t)meta[2] * SC::LV_WORDS);
+        const int level = (int)st[SC::ST_META + META_LEVEL];
+        const int nwarm = (int)st[SC::ST_META + META_NWARM];
+        load_level_consts(prm.levels + (size_t)level * SC::LV_WORDS);
         g.sync();
         // accumulated impulses of the previous launch: entry k goes to lane k
-        rec.ab = 0u;
-        rec.accn[0] = 0.0f; rec.acct[0] = 0.0f; rec.accn[1] = 0.0f; rec.acct[1] = 0.0f;
-        if (lane < meta[4]) {
+        rec.ab = 0u; rec.accn = 0.0f; rec.acct = 0.0f;
+        lanef(kStageWords) = 0.0f; lanef(kStageWords + 1) = 0.0f;
+        if (lane < nwarm) {
             const uint32_t *wr = st + SC::ST_WARM + kWarmWords * lane;
-            rec.accn[0] = __uint_as_float(wr[1]); rec.acct[0] = __uint_as_float(wr[2]);
-            rec.accn[1] = __uint_as_float(wr[3]); rec.acct[1] = __uint_as_float(wr[4]);
+            rec.ab = wr[0] << 12;
+            rec.accn = __uint_as_float(wr[1]); rec.acct = __uint_as_float(wr[2]);
+            lanef(kStageWords) = __uint_as_float(wr[3]); lanef(kStageWords + 1) = __uint_as_float(wr[4]);
             widx()[wr[0]] = (uint8_t)lane;
         }
-        if (meta[4] > G) ovf_warm_in<SC, G>(sm, ovf, st + SC::ST_WARM, meta[4]);
+        if (nwarm > G) warm_in<SC, G>(sm, ovf, st + SC::ST_WARM, nwarm);
         g.sync();
 #pragma unroll 1
         for (int s = 0; s < prm.n_steps; ++s) {
-            step(e, s, meta);
+            step(e, s);
             g.sync();
             if ((s & 255) == 255) flush_counters();
         }
         // write back
         for (int i = lane; i < 6 * SC::N; i += G) st[SC::ST_BODY + i] = smu[SC::BX + i];
-        if (SC::J > 0 && lane < SC::J) { st[SC::ST_JACC + 2 * lane] = __float_as_uint(jr.accx); st[SC::ST_JACC + 2 * lane + 1] = __float_as_uint(jr.accy); }
-        if (lane == 0) {
-#pragma unroll
-            for (int i = 0; i < 5; ++i) st[SC::ST_META + i] = (uint32_t)meta[i];
+        if (SC::J > 0 && lane < SC::J) {
+            st[SC::ST_JACC + 2 * lane] = smu[SC::JROW + JR_ACCX * SC::J + lane];
+            st[SC::ST_JACC + 2 * lane + 1] = smu[SC::JROW + JR_ACCY * SC::J + lane];
         }
-        if (lane < meta[4]) {
+        if (lane < 5) st[SC::ST_META + lane] = smu[SC::META + lane];
+        const int nw = (int)smu[SC::META + META_NWARM];
+        if (lane < nw) {
             uint32_t *wr = st + SC::ST_WARM + kWarmWords * lane;
             wr[0] = (rec.ab >> 12) & 127u;
-            wr[1] = __float_as_uint(rec.accn[0]); wr[2] = __float_as_uint(rec.acct[0]);
-            wr[3] = __float_as_uint(rec.accn[1]); wr[4] = __float_as_uint(rec.acct[1]);
+            wr[1] = __float_as_uint(rec.accn); wr[2] = __float_as_uint(rec.acct);
+            wr[3] = __float_as_uint(lanef(kStageWords)); wr[4] = __float_as_uint(lanef(kStageWords + 1));
         }
-        if (meta[4] > G) ovf_warm_out<SC, G>(ovf, st + SC::ST_WARM, meta[4]);
+        if (nw > G) warm_out<SC, G>(ovf, st + SC::ST_WARM, nw);
         flush_counters();
+        g.sync();
     }
 };
 
@@ -1104,7 +1214,7 @@ __global__ void __launch_bounds__(kBlockThreads) k2d_step_kernel(const StepParam
     uint32_t *scratch = prm.scratch + (size_t)slot * SC::SCRATCH_WORDS;
     Scene<SC, G> scene(region, ptab, scratch, prm);
 #pragma unroll 1
-    for (int e = slot; e < prm.n_envs; e += nslots) { scene.run(e); scene.g.sync(); }
+    for (int e = slot; e < prm.n_envs; e += nslots) scene.run(e);
 }
 
 // ---------------------------------------------------------------- reset kernel: one thread per (env, word)
