@@ -66,8 +66,9 @@ struct SizeClass {
     // then, per lane of the group (field-major, G words per field):
     //   STG  kStageWords fields: manifolds on their way to the owning lane; afterwards the second manifold's constants
     //   ACC2 2 fields: accumulated impulses of the second manifold;  CORR 2 fields: positional corrections
+    //   OV   kRecWords fields: the lane's second record (pair number G + lane of a crowded scene) in memory form
     static constexpr int STG = WIDX + (NPAIRS + 3) / 4;
-    static constexpr int LANE_FIELDS = kStageWords + 4;
+    static constexpr int LANE_FIELDS = kStageWords + 4 + kRecWords;
     static constexpr int PTAB_WORDS = ((NPAIRS + 1) / 2 + 3) / 4 * 4;  // block-shared pair table, 16 bits per pair
 };
 // memory form of a contact pair record (the overflow path keeps records in global scratch)
@@ -79,6 +80,12 @@ enum { S_AB = 0, S_NX, S_NY, S_PX0, S_PY0, S_PEN0, S_PX1, S_PY1, S_PEN1 };
 static_assert(S_PEN1 + 1 == kStageWords, "stage size");
 // second-manifold constants reuse the stage fields of the same lane
 enum { M2_RNA = 0, M2_RNB, M2_RTA, M2_RTB, M2_MASSN, M2_MASST, M2_TARGET };
+// per-lane fields after the stage fields
+enum { LF_ACC2N = kStageWords, LF_ACC2T, LF_CORR0, LF_CORR1, LF_OV };
+// where stage field f of a lane's second record waits inside its memory-form fields (clear of the accumulated impulses)
+__host__ __device__ constexpr int ov_stage(int f) { return LF_OV + (f < 3 ? f : f + 1); }
+constexpr int LF_OV_ACC0N = LF_OV + R_M0 + M_ACCN, LF_OV_ACC0T = LF_OV + R_M0 + M_ACCT;
+constexpr int LF_OV_ACC1N = LF_OV + R_M0 + M_WORDS + M_ACCN, LF_OV_ACC1T = LF_OV + R_M0 + M_WORDS + M_ACCT;
 // joint row fields
 enum { JR_RAX = 0, JR_RAY, JR_RBX, JR_RBY, JR_I11, JR_I12, JR_I22, JR_BX, JR_BY, JR_CX, JR_CY, JR_ACCX, JR_ACCY };
 static_assert(JR_ACCY + 1 == kJointWords, "joint row size");
@@ -369,6 +376,56 @@ __device__ __forceinline__ void sweep_joints(float *sm, uint32_t jab, int lane, 
     }
 }
 
+// Accumulated impulses that pair record `wi` of the previous step left behind (255: the pair was not
+// touching).  Records 0..G-1 live with lane wi (first manifold in its registers: old_n / old_t are the
+// calling lane's own, fetched across lanes here, so every lane of the group must call; second manifold
+// in its shared-memory fields), records G..2G-1 in the second-record fields of lane wi - G, later ones
+// in the warm entries of the global scratch.
+template <class SC, int G>
+__device__ __forceinline__ void warm_lookup(const Group<G> &g, const float *sm, const uint32_t *ovf, int wi, float old_n, float old_t,
+                                            int warm_start, float (&w)[4]) {
+    const int src = (wi < G) ? wi : 0;
+    const float *lf = sm + SC::STG;
+    w[0] = g.shflf(old_n, src); w[1] = g.shflf(old_t, src);
+    w[2] = lf[LF_ACC2N * G + src]; w[3] = lf[LF_ACC2T * G + src];
+    if (wi >= G && wi != 255) {
+        if (wi < 2 * G) {
+            const float *o = lf + (wi - G);
+            w[0] = o[LF_OV_ACC0N * G]; w[1] = o[LF_OV_ACC0T * G]; w[2] = o[LF_OV_ACC1N * G]; w[3] = o[LF_OV_ACC1T * G];
+        } else {
+            const uint32_t *wr = ovf + SC::SCRATCH_WARM + (size_t)wi * kWarmWords;
+#pragma unroll
+            for (int q = 0; q < 4; ++q) w[q] = __uint_as_float(wr[1 + q]);
+        }
+    }
+    if (wi == 255 || !warm_start) { w[0] = 0.0f; w[1] = 0.0f; w[2] = 0.0f; w[3] = 0.0f; }
+}
+
+// Levels of nrec staged pairs by one lane with a per-body table (used when there are more pairs than
+// lanes): a pair's level is one more than the highest level of an earlier pair sharing a movable body.
+// The packed pair words of pairs 0..G-1 are in the stage fields, of G..2G-1 in the second-record
+// fields, of later ones in global scratch; the level goes into bits 19.. of each word.
+template <class SC, int G>
+__device__ __forceinline__ int levels_by_one_lane(uint32_t *smu, uint32_t *ovf, int nrec) {
+    uint8_t *bl = reinterpret_cast<uint8_t *>(smu + SC::SURV);   // the survivor list is no longer needed
+    int cmax = 0;
+    for (int i = 0; i < SC::N; ++i) bl[i] = 0;
+    for (int k = 0; k < nrec; ++k) {
+        uint32_t *w = (k < G) ? (smu + SC::STG + S_AB * G + k)
+                    : (k < 2 * G) ? (smu + SC::STG + ov_stage(S_AB) * G + (k - G)) : (ovf + (size_t)k * kRecWords + S_AB);
+        const uint32_t ab = *w;
+        const int a = ab & 31, b = (ab >> 5) & 31;
+        int lvl = 1;
+        if ((ab >> 26) & 1u) lvl = max(lvl, bl[a] + 1);
+        if ((ab >> 27) & 1u) lvl = max(lvl, bl[b] + 1);
+        if ((ab >> 26) & 1u) bl[a] = (uint8_t)lvl;
+        if ((ab >> 27) & 1u) bl[b] = (uint8_t)lvl;
+        *w = ab | ((uint32_t)lvl << 19);
+        cmax = max(cmax, lvl);
+    }
+    return cmax;
+}
+
 // ================================================================ overflow path (cold code)
 // A scene with more touching pairs than lanes (nrec > G) solves this step's contacts from memory
 // records in global scratch, one loop over records per level, with the same row arithmetic.
@@ -441,35 +498,19 @@ __device__ __noinline__ int slow_solve(float *sm, uint32_t *ovf, const uint32_t 
     Group<G> g;
     const int lane = g.lane;
     uint32_t *smu = reinterpret_cast<uint32_t *>(sm);
-    uint8_t *bl = reinterpret_cast<uint8_t *>(smu + SC::SURV);   // the survivor list is no longer needed
     const uint8_t *widx = reinterpret_cast<const uint8_t *>(smu + SC::WIDX);
-    const float *lanef = sm + SC::STG;
-    // the staged manifolds of the first G pairs join the others in scratch
-    {
-        uint32_t *r = ovf + (size_t)lane * kRecWords;
-#pragma unroll
-        for (int f = 0; f < kStageWords; ++f) r[f] = smu[SC::STG + f * G + lane];
-    }
-    g.sync();
     int cmax = 0;
-    if (lane == 0) {
-        for (int i = 0; i < SC::N; ++i) bl[i] = 0;
-        for (int k = 0; k < nrec; ++k) {
-            uint32_t *w = ovf + (size_t)k * kRecWords + S_AB;
-            const uint32_t ab = *w;
-            const int a = ab & 31, b = (ab >> 5) & 31;
-            int lvl = 1;
-            if ((ab >> 26) & 1u) lvl = max(lvl, bl[a] + 1);
-            if ((ab >> 27) & 1u) lvl = max(lvl, bl[b] + 1);
-            if ((ab >> 26) & 1u) bl[a] = (uint8_t)lvl;
-            if ((ab >> 27) & 1u) bl[b] = (uint8_t)lvl;
-            *w = ab | ((uint32_t)lvl << 19);
-            cmax = max(cmax, lvl);
-        }
-    }
+    if (lane == 0) cmax = levels_by_one_lane<SC, G>(smu, ovf, nrec);
     __threadfence_block();
     g.sync();
     cmax = g.shfl(cmax, 0);
+    // the staged manifolds of the first 2 G pairs join the others in scratch
+    {
+        uint32_t *r = ovf + (size_t)lane * kRecWords, *r2 = ovf + (size_t)(G + lane) * kRecWords;
+#pragma unroll
+        for (int f = 0; f < kStageWords; ++f) { r[f] = smu[SC::STG + f * G + lane]; r2[f] = smu[SC::STG + ov_stage(f) * G + lane]; }
+    }
+    g.sync();
     // pre-step of every pair; accumulated impulses of the previous step come from the lane that
     // owned the pair then (first manifold in its registers, second in its shared-memory fields)
     // or from the warm entries in scratch
@@ -480,14 +521,8 @@ __device__ __noinline__ int slow_solve(float *sm, uint32_t *ovf, const uint32_t 
         uint32_t ab = 0u;
         int wi = 255;
         if (valid) { ab = r[S_AB]; wi = widx[(ab >> 12) & 127]; }
-        const int src = (wi < G) ? wi : 0;
-        float w[4] = { g.shflf(old_n, src), g.shflf(old_t, src), lanef[kStageWords * G + src], lanef[(kStageWords + 1) * G + src] };
-        if (wi >= G && wi != 255) {
-            const uint32_t *wr = ovf + SC::SCRATCH_WARM + (size_t)wi * kWarmWords;
-#pragma unroll
-            for (int q = 0; q < 4; ++q) w[q] = __uint_as_float(wr[1 + q]);
-        }
-        if (wi == 255 || !warm_start) { w[0] = 0.0f; w[1] = 0.0f; w[2] = 0.0f; w[3] = 0.0f; }
+        float w[4];
+        warm_lookup<SC, G>(g, sm, ovf, wi, old_n, old_t, warm_start, w);
         if (valid) {
             RecM c;
             c.ab = ab; c.nx = __uint_as_float(r[S_NX]); c.ny = __uint_as_float(r[S_NY]);
@@ -553,12 +588,12 @@ __device__ __noinline__ int slow_finish(float *sm, uint32_t *ovf, int nrec) {
     return nman;
 }
 
-// Launch boundaries: warm entries G.. between the state record and the scratch.
+// Launch boundaries: warm entries 2 G.. between the state record and the scratch.
 template <class SC, int G>
 __device__ __noinline__ void warm_in(float *sm, uint32_t *ovf, const uint32_t *st_warm, int nwarm) {
     Group<G> g;
     uint8_t *widx = reinterpret_cast<uint8_t *>(reinterpret_cast<uint32_t *>(sm) + SC::WIDX);
-    for (int k = G + g.lane; k < nwarm; k += G) {
+    for (int k = 2 * G + g.lane; k < nwarm; k += G) {
         uint32_t *wr = ovf + SC::SCRATCH_WARM + (size_t)k * kWarmWords;
 #pragma unroll
         for (int q = 0; q < kWarmWords; ++q) wr[q] = st_warm[kWarmWords * k + q];
@@ -568,7 +603,7 @@ __device__ __noinline__ void warm_in(float *sm, uint32_t *ovf, const uint32_t *s
 template <class SC, int G>
 __device__ __noinline__ void warm_out(const uint32_t *ovf, uint32_t *st_warm, int nwarm) {
     Group<G> g;
-    for (int k = G + g.lane; k < nwarm; k += G) {
+    for (int k = 2 * G + g.lane; k < nwarm; k += G) {
         const uint32_t *wr = ovf + SC::SCRATCH_WARM + (size_t)k * kWarmWords;
 #pragma unroll
         for (int q = 0; q < kWarmWords; ++q) st_warm[kWarmWords * k + q] = wr[q];
@@ -770,7 +805,7 @@ struct Scene {
         const bool dyn_a = (ab >> 26) & 1u, dyn_b = (ab >> 27) & 1u;
         if (MODE == 2) {
             correct_pair(sm + SC::BX, sm + SC::BY, a, b, amask, dyn_a, dyn_b, rec.nx, rec.ny, rec.ma, rec.mb,
-                         lanef(kStageWords + 2), lanef(kStageWords + 3));
+                         lanef(LF_CORR0), lanef(LF_CORR1));
             return;
         }
         float vax = sm[SC::BVX + a], vay = sm[SC::BVY + a], wa = sm[SC::BW + a];
@@ -779,20 +814,52 @@ struct Scene {
             manifold_rows<MODE>(rec.nx, rec.ny, rec.mu, rec.ma, rec.mb, rec.ia, rec.ib, rec.rna, rec.rnb, rec.rta, rec.rtb,
                                 rec.massn, rec.masst, rec.target, rec.accn, rec.acct, vax, vay, wa, vbx, vby, wb);
         if (amask & 2u) {
-            float accn = lanef(kStageWords), acct = lanef(kStageWords + 1);
+            float accn = lanef(LF_ACC2N), acct = lanef(LF_ACC2T);
             manifold_rows<MODE>(rec.nx, rec.ny, rec.mu, rec.ma, rec.mb, rec.ia, rec.ib, lanef(M2_RNA), lanef(M2_RNB), lanef(M2_RTA),
                                 lanef(M2_RTB), lanef(M2_MASSN), lanef(M2_MASST), lanef(M2_TARGET), accn, acct, vax, vay, wa, vbx, vby, wb);
-            if (MODE == 1) { lanef(kStageWords) = accn; lanef(kStageWords + 1) = acct; }
+            if (MODE == 1) { lanef(LF_ACC2N) = accn; lanef(LF_ACC2T) = acct; }
+        }
+        if (dyn_a) { sm[SC::BVX + a] = vax; sm[SC::BVY + a] = vay; sm[SC::BW + a] = wa; }
+        if (dyn_b) { sm[SC::BVX + b] = vbx; sm[SC::BVY + b] = vby; sm[SC::BW + b] = wb; }
+    }
+    // ---- the same for the lane's second record (pair number G + lane of a scene with more than G touching
+    // pairs), which is in memory form in the lane's shared-memory fields
+    template <int MODE>
+    __device__ __forceinline__ void visit_pair2() {
+        const uint32_t ab = __float_as_uint(lanef(LF_OV + R_AB));
+        const int a = ab & 31, b = (ab >> 5) & 31;
+        const unsigned amask = (ab >> 10) & 3u;
+        const bool dyn_a = (ab >> 26) & 1u, dyn_b = (ab >> 27) & 1u;
+        const float nx = lanef(LF_OV + R_NX), ny = lanef(LF_OV + R_NY);
+        const float ma = sm[SC::BIM + a], mb = sm[SC::BIM + b];
+        if (MODE == 2) {
+            correct_pair(sm + SC::BX, sm + SC::BY, a, b, amask, dyn_a, dyn_b, nx, ny, ma, mb,
+                         lanef(LF_OV + R_M0 + M_CORR), lanef(LF_OV + R_M0 + M_WORDS + M_CORR));
+            return;
+        }
+        const float ia = sm[SC::BII + a], ib = sm[SC::BII + b], mu = lanef(LF_OV + R_MU);
+        float vax = sm[SC::BVX + a], vay = sm[SC::BVY + a], wa = sm[SC::BW + a];
+        float vbx = sm[SC::BVX + b], vby = sm[SC::BVY + b], wb = sm[SC::BW + b];
+#pragma unroll
+        for (int mi = 0; mi < 2; ++mi) {
+            if (amask & (1u << mi)) {
+                const int f = LF_OV + R_M0 + mi * M_WORDS;
+                float accn = lanef(f + M_ACCN), acct = lanef(f + M_ACCT);
+                manifold_rows<MODE>(nx, ny, mu, ma, mb, ia, ib, lanef(f + M_RNA), lanef(f + M_RNB), lanef(f + M_RTA), lanef(f + M_RTB),
+                                    lanef(f + M_MASSN), lanef(f + M_MASST), lanef(f + M_TARGET), accn, acct, vax, vay, wa, vbx, vby, wb);
+                if (MODE == 1) { lanef(f + M_ACCN) = accn; lanef(f + M_ACCT) = acct; }
+            }
         }
         if (dyn_a) { sm[SC::BVX + a] = vax; sm[SC::BVY + a] = vay; sm[SC::BW + a] = wa; }
         if (dyn_b) { sm[SC::BVX + b] = vbx; sm[SC::BVY + b] = vby; sm[SC::BW + b] = wb; }
     }
     // records of one level touch disjoint movable bodies; levels in order keep the record order
     template <int MODE>
-    __device__ __forceinline__ void sweep_pairs(int cmax, int clevel) {
+    __device__ __forceinline__ void sweep_pairs(int cmax, int clevel, int clevel2) {
 #pragma unroll 1
         for (int lvl = 1; lvl <= cmax; ++lvl) {
             if (clevel == lvl) visit_pair<MODE>();
+            if (clevel2 == lvl) visit_pair2<MODE>();
             g.sync();
         }
     }
@@ -981,6 +1048,11 @@ struct Scene {
                         st[S_AB * G] = __uint_as_float(ab); st[S_NX * G] = nx; st[S_NY * G] = ny;
                         st[S_PX0 * G] = m[0].px; st[S_PY0 * G] = m[0].py; st[S_PEN0 * G] = m[0].pen;
                         st[S_PX1 * G] = m[1].px; st[S_PY1 * G] = m[1].py; st[S_PEN1 * G] = m[1].pen;
+                    } else if (k < 2 * G) {
+                        float *st = sm + SC::STG + (k - G);
+                        st[ov_stage(S_AB) * G] = __uint_as_float(ab); st[ov_stage(S_NX) * G] = nx; st[ov_stage(S_NY) * G] = ny;
+                        st[ov_stage(S_PX0) * G] = m[0].px; st[ov_stage(S_PY0) * G] = m[0].py; st[ov_stage(S_PEN0) * G] = m[0].pen;
+                        st[ov_stage(S_PX1) * G] = m[1].px; st[ov_stage(S_PY1) * G] = m[1].py; st[ov_stage(S_PEN1) * G] = m[1].pen;
                     } else {
                         uint32_t *st = ovf + (size_t)k * kRecWords;
                         st[S_AB] = ab; st[S_NX] = __float_as_uint(nx); st[S_NY] = __float_as_uint(ny);
@@ -995,40 +1067,49 @@ struct Scene {
         g.sync();
         c_rec += (unsigned)nrec << 16;
 
-        const bool overflow = nrec > G;
-        int cmax = 0, clevel = 0;
+        const bool overflow = nrec > 2 * G;
+        int cmax = 0, clevel = 0, clevel2 = 0;
         if (overflow) {
             cmax = slow_solve<SC, G>(sm, ovf, lv, nrec, jab, jlevel, jmax, prm.solver_iters, prm.warm_start, prm.motor_rho,
                                      rec.accn, rec.acct, contact_consts());
         } else {
-            // every staged pair becomes a record in its own lane: accumulated impulses of the same pair in the
-            // previous step come from the lane that owned it then
             const ContactConsts cc = contact_consts();
-            const bool mine = lane < nrec;
-            uint32_t ab = 0u;
-            int wi = 255;
+            const bool two = nrec > G;      // some lanes get a second record
+            if (two) {
+                if (lane == 0) cmax = levels_by_one_lane<SC, G>(smu, ovf, nrec);
+                g.sync();
+            }
+            // every staged pair becomes a record in its own lane: accumulated impulses of the same pair in the
+            // previous step come from wherever its record was then
+            const bool mine = lane < nrec, mine2 = two && G + lane < nrec;
+            uint32_t ab = 0u, ab2 = 0u;
             float nx = 0.0f, ny = 0.0f, pt[6] = { 0.0f, 0.0f, 0.0f, 0.0f, 0.0f, 0.0f };
-            if (mine) {
-                ab = __float_as_uint(lanef(S_AB)); wi = widx()[(ab >> 12) & 127];
-                nx = lanef(S_NX); ny = lanef(S_NY);
-                pt[0] = lanef(S_PX0); pt[1] = lanef(S_PY0); pt[2] = lanef(S_PEN0); pt[3] = lanef(S_PX1); pt[4] = lanef(S_PY1); pt[5] = lanef(S_PEN1);
+            float w[4], w2[4];
+            {
+                int wi = 255;
+                if (mine) {
+                    ab = __float_as_uint(lanef(S_AB)); wi = widx()[(ab >> 12) & 127];
+                    nx = lanef(S_NX); ny = lanef(S_NY);
+                    pt[0] = lanef(S_PX0); pt[1] = lanef(S_PY0); pt[2] = lanef(S_PEN0); pt[3] = lanef(S_PX1); pt[4] = lanef(S_PY1); pt[5] = lanef(S_PEN1);
+                }
+                const float old_n = rec.accn, old_t = rec.acct;
+                warm_lookup<SC, G>(g, sm, ovf, wi, old_n, old_t, prm.warm_start, w);
+                if (two) {
+                    int wi2 = 255;
+                    if (mine2) { ab2 = __float_as_uint(lanef(ov_stage(S_AB))); wi2 = widx()[(ab2 >> 12) & 127]; }
+                    warm_lookup<SC, G>(g, sm, ovf, wi2, old_n, old_t, prm.warm_start, w2);
+                }
             }
-            const int src = (wi < G) ? wi : 0;
-            float w[4] = { g.shflf(rec.accn, src), g.shflf(rec.acct, src), sm[SC::STG + kStageWords * G + src], sm[SC::STG + (kStageWords + 1) * G + src] };
-            if (wi >= G && wi != 255) {
-                const uint32_t *wr = ovf + SC::SCRATCH_WARM + (size_t)wi * kWarmWords;
-#pragma unroll
-                for (int q = 0; q < 4; ++q) w[q] = __uint_as_float(wr[1 + q]);
-            }
-            if (wi == 255 || !prm.warm_start) { w[0] = 0.0f; w[1] = 0.0f; w[2] = 0.0f; w[3] = 0.0f; }
             g.sync();     // every lane has read the fields it needs from other lanes before they are rewritten
             const int a = ab & 31, b = (ab >> 5) & 31;
             const unsigned amask = (ab >> 10) & 3u;
             rec.ab = ab; rec.nx = nx; rec.ny = ny;
             rec.ma = sm[SC::BIM + a]; rec.mb = sm[SC::BIM + b]; rec.ia = sm[SC::BII + a]; rec.ib = sm[SC::BII + b];
-            const float fra = sm[SC::BFR + a], frb = sm[SC::BFR + b];
+            {
+                const float fra = sm[SC::BFR + a], frb = sm[SC::BFR + b];
+                rec.mu = sqrtf(__fmaf_rn(fra, fra, frb * frb));
+            }
             const float er = fmin_cmp(sm[SC::BRE + a], sm[SC::BRE + b]);
-            rec.mu = sqrtf(__fmaf_rn(fra, fra, frb * frb));
             float corr0 = 0.0f, corr1 = 0.0f;
             rec.rna = 0.0f; rec.rnb = 0.0f; rec.rta = 0.0f; rec.rtb = 0.0f; rec.massn = 0.0f; rec.masst = 0.0f; rec.target = 0.0f;
             rec.accn = 0.0f; rec.acct = 0.0f;
@@ -1046,11 +1127,40 @@ struct Scene {
                 lanef(M2_MASSN) = massn; lanef(M2_MASST) = masst; lanef(M2_TARGET) = target;
                 acc2n = w[2]; acc2t = w[3];
             }
-            lanef(kStageWords) = acc2n; lanef(kStageWords + 1) = acc2t;
-            lanef(kStageWords + 2) = corr0; lanef(kStageWords + 3) = corr1;
-            // levels of the records (canonical order = record order): one more than the highest level of an
-            // earlier record that shares a movable body
-            {
+            lanef(LF_ACC2N) = acc2n; lanef(LF_ACC2T) = acc2t;
+            lanef(LF_CORR0) = corr0; lanef(LF_CORR1) = corr1;
+            if (two) {
+                // the second record of this lane, built in place in its memory-form fields
+                if (mine2) {
+                    const int a2 = ab2 & 31, b2 = (ab2 >> 5) & 31;
+                    const float nx2 = lanef(ov_stage(S_NX)), ny2 = lanef(ov_stage(S_NY));
+                    const float pt2[6] = { lanef(ov_stage(S_PX0)), lanef(ov_stage(S_PY0)), lanef(ov_stage(S_PEN0)),
+                                           lanef(ov_stage(S_PX1)), lanef(ov_stage(S_PY1)), lanef(ov_stage(S_PEN1)) };
+                    const float ma = sm[SC::BIM + a2], mb = sm[SC::BIM + b2], ia = sm[SC::BII + a2], ib = sm[SC::BII + b2];
+                    const float fra = sm[SC::BFR + a2], frb = sm[SC::BFR + b2];
+                    const float er2 = fmin_cmp(sm[SC::BRE + a2], sm[SC::BRE + b2]);
+                    lanef(LF_OV + R_MU) = sqrtf(__fmaf_rn(fra, fra, frb * frb));
+#pragma unroll
+                    for (int mi = 0; mi < 2; ++mi) {
+                        float rna = 0.0f, rnb = 0.0f, rta = 0.0f, rtb = 0.0f, massn = 0.0f, masst = 0.0f, target = 0.0f, corr = 0.0f, an = 0.0f, at = 0.0f;
+                        if ((ab2 >> 10) & (1u << mi)) {
+                            prestep_manifold<SC>(a2, b2, nx2, ny2, ma, mb, ia, ib, pt2[3 * mi], pt2[3 * mi + 1], pt2[3 * mi + 2], er2, sm, cc,
+                                                 rna, rnb, rta, rtb, massn, masst, target, corr);
+                            an = w2[2 * mi]; at = w2[2 * mi + 1];
+                        }
+                        const int f = LF_OV + R_M0 + mi * M_WORDS;
+                        lanef(f + M_RNA) = rna; lanef(f + M_RNB) = rnb; lanef(f + M_RTA) = rta; lanef(f + M_RTB) = rtb;
+                        lanef(f + M_MASSN) = massn; lanef(f + M_MASST) = masst; lanef(f + M_TARGET) = target; lanef(f + M_CORR) = corr;
+                        lanef(f + M_ACCN) = an; lanef(f + M_ACCT) = at;
+                    }
+                    clevel2 = (int)((ab2 >> 19) & 127u);
+                }
+                clevel = (int)((ab >> 19) & 127u);
+                cmax = g.shfl(cmax, 0);
+                c_man += (unsigned)(__popc(g.ballot((ab2 >> 10) & 1u)) + __popc(g.ballot((ab2 >> 11) & 1u)));
+            } else {
+                // levels of the records (canonical order = record order): one more than the highest level of an
+                // earlier record that shares a movable body
                 int lvl = mine ? 1 : 0;
                 const bool da = (ab >> 26) & 1u, db = (ab >> 27) & 1u;
 #pragma unroll 1
@@ -1066,13 +1176,13 @@ struct Scene {
             }
             c_man += (unsigned)(__popc(g.ballot(amask & 1u)) + __popc(g.ballot(amask & 2u)));
             // warm start: contacts, then joints
-            sweep_pairs<0>(cmax, clevel);
+            sweep_pairs<0>(cmax, clevel, clevel2);
             sweep_joints<SC, G, 0>(sm, jab, lane, jlevel, jmax, lv, prm.motor_rho);
             // solver iterations: joints, then contacts
 #pragma unroll 1
             for (int it = 0; it < prm.solver_iters; ++it) {
                 sweep_joints<SC, G, 1>(sm, jab, lane, jlevel, jmax, lv, prm.motor_rho);
-                sweep_pairs<1>(cmax, clevel);
+                sweep_pairs<1>(cmax, clevel, clevel2);
             }
         }
         // Euler step with the solved velocities
@@ -1085,7 +1195,7 @@ struct Scene {
         }
         g.sync();
         if (overflow) slow_correct<SC, G>(sm, ovf, nrec, cmax);
-        else sweep_pairs<2>(cmax, clevel);
+        else sweep_pairs<2>(cmax, clevel, clevel2);
         sweep_joints<SC, G, 2>(sm, jab, lane, jlevel, jmax, lv, prm.motor_rho);
         bool finite = true;
         for (int i = lane; i < SC::N; i += G)
@@ -1099,12 +1209,18 @@ struct Scene {
         g.sync();
         if (overflow) {
             c_man += (unsigned)slow_finish<SC, G>(sm, ovf, nrec);
-            // the first G pairs go back to their lanes
-            const uint32_t *wr = ovf + SC::SCRATCH_WARM + (size_t)lane * kWarmWords;
+            // the first 2 G pairs go back to their lanes
+            const uint32_t *wr = ovf + SC::SCRATCH_WARM + (size_t)lane * kWarmWords, *wr2 = wr + (size_t)G * kWarmWords;
             rec.ab = wr[0] << 12;
             rec.accn = __uint_as_float(wr[1]); rec.acct = __uint_as_float(wr[2]);
-            lanef(kStageWords) = __uint_as_float(wr[3]); lanef(kStageWords + 1) = __uint_as_float(wr[4]);
-        } else if (lane < nrec) widx()[(rec.ab >> 12) & 127] = (uint8_t)lane;
+            lanef(LF_ACC2N) = __uint_as_float(wr[3]); lanef(LF_ACC2T) = __uint_as_float(wr[4]);
+            lanef(LF_OV + R_AB) = __uint_as_float(wr2[0] << 12);
+            lanef(LF_OV_ACC0N) = __uint_as_float(wr2[1]); lanef(LF_OV_ACC0T) = __uint_as_float(wr2[2]);
+            lanef(LF_OV_ACC1N) = __uint_as_float(wr2[3]); lanef(LF_OV_ACC1T) = __uint_as_float(wr2[4]);
+        } else {
+            if (lane < nrec) widx()[(rec.ab >> 12) & 127] = (uint8_t)lane;
+            if (clevel2 != 0) widx()[(__float_as_uint(lanef(LF_OV + R_AB)) >> 12) & 127] = (uint8_t)(G + lane);
+        }
 
         // reward, termination, counters, auto-reset
         const bool timeout = prm.max_episode_steps > 0 && step_count >= prm.max_episode_steps;
@@ -1156,15 +1272,22 @@ struct Scene {
         g.sync();
         // accumulated impulses of the previous launch: entry k goes to lane k
         rec.ab = 0u; rec.accn = 0.0f; rec.acct = 0.0f;
-        lanef(kStageWords) = 0.0f; lanef(kStageWords + 1) = 0.0f;
+        lanef(LF_ACC2N) = 0.0f; lanef(LF_ACC2T) = 0.0f;
         if (lane < nwarm) {
             const uint32_t *wr = st + SC::ST_WARM + kWarmWords * lane;
             rec.ab = wr[0] << 12;
             rec.accn = __uint_as_float(wr[1]); rec.acct = __uint_as_float(wr[2]);
-            lanef(kStageWords) = __uint_as_float(wr[3]); lanef(kStageWords + 1) = __uint_as_float(wr[4]);
+            lanef(LF_ACC2N) = __uint_as_float(wr[3]); lanef(LF_ACC2T) = __uint_as_float(wr[4]);
             widx()[wr[0]] = (uint8_t)lane;
         }
-        if (nwarm > G) warm_in<SC, G>(sm, ovf, st + SC::ST_WARM, nwarm);
+        if (G + lane < nwarm) {
+            const uint32_t *wr = st + SC::ST_WARM + kWarmWords * (G + lane);
+            lanef(LF_OV + R_AB) = __uint_as_float(wr[0] << 12);
+            lanef(LF_OV_ACC0N) = __uint_as_float(wr[1]); lanef(LF_OV_ACC0T) = __uint_as_float(wr[2]);
+            lanef(LF_OV_ACC1N) = __uint_as_float(wr[3]); lanef(LF_OV_ACC1T) = __uint_as_float(wr[4]);
+            widx()[wr[0]] = (uint8_t)(G + lane);
+        }
+        if (nwarm > 2 * G) warm_in<SC, G>(sm, ovf, st + SC::ST_WARM, nwarm);
         g.sync();
 #pragma unroll 1
         for (int s = 0; s < prm.n_steps; ++s) {
@@ -1184,9 +1307,15 @@ struct Scene {
             uint32_t *wr = st + SC::ST_WARM + kWarmWords * lane;
             wr[0] = (rec.ab >> 12) & 127u;
             wr[1] = __float_as_uint(rec.accn); wr[2] = __float_as_uint(rec.acct);
-            wr[3] = __float_as_uint(lanef(kStageWords)); wr[4] = __float_as_uint(lanef(kStageWords + 1));
+            wr[3] = __float_as_uint(lanef(LF_ACC2N)); wr[4] = __float_as_uint(lanef(LF_ACC2T));
         }
-        if (nw > G) warm_out<SC, G>(ovf, st + SC::ST_WARM, nw);
+        if (G + lane < nw) {
+            uint32_t *wr = st + SC::ST_WARM + kWarmWords * (G + lane);
+            wr[0] = (__float_as_uint(lanef(LF_OV + R_AB)) >> 12) & 127u;
+            wr[1] = __float_as_uint(lanef(LF_OV_ACC0N)); wr[2] = __float_as_uint(lanef(LF_OV_ACC0T));
+            wr[3] = __float_as_uint(lanef(LF_OV_ACC1N)); wr[4] = __float_as_uint(lanef(LF_OV_ACC1T));
+        }
+        if (nw > 2 * G) warm_out<SC, G>(ovf, st + SC::ST_WARM, nw);
         flush_counters();
         g.sync();
     }

@@ -138,15 +138,17 @@ def test_custom_dimensions_and_inactive_entities():
     assert np.array_equal(r, rr) and np.array_equal(d, dr)
 
 
-def test_more_active_pairs_than_lanes_and_than_shared_memory_records():
-    # every shape of an L scene dropped on the same spot: far more than 32 touching pairs, so the
-    # records beyond the shared-memory capacity go through the global-memory scratch
+@pytest.mark.parametrize("lanes", [8, 16, 32])
+def test_more_active_pairs_than_lanes_and_than_shared_memory_records(lanes):
+    # every shape of an L scene dropped on the same spot: far more touching pairs than twice the lanes
+    # of a scene, so the step's contacts go through the global-memory scratch; as the pile spreads the
+    # count falls through the range where lanes hold two records each, then one
     lv = scenes.make_levels("L", 6, 51)
     rng = np.random.default_rng(51)
     lv["pos"][:, 1:, 0] = rng.uniform(-0.3, 0.3, (6, 15)).astype(np.float32)
     lv["pos"][:, 1:, 1] = rng.uniform(0.8, 1.4, (6, 15)).astype(np.float32)
     lv["joint_active"][:] = 0
-    env, ref = parity.make_pair(lv, 6)
+    env, ref = parity.make_pair(lv, 6, lanes_per_scene=lanes)
     trace = env.enable_trace()
     act = scenes.make_actions(12, 6, env.n_actions, 51)
     (r, d), (rr, dr) = parity.step_both(env, ref, act[:1])
