@@ -297,7 +297,7 @@ def run_gpu(args) -> dict:
         "dtype": "f32", "data": "synthetic",
         "config": {"workload": f"{w['size']} scenes, {n_envs} envs per GPU, {FUSED} fused engine steps + 1 observation per bench step "
                                f"(config {args.workload}: pool of {w['n_levels']} levels, horizon {w['max_episode_steps']})",
-                   "lanes_per_scene": env.cfg.lanes_per_scene or 32, "fused_steps": FUSED,
+                   "lanes_per_scene": env.cfg.lanes_per_scene or 16, "fused_steps": FUSED,
                    "l2": "flushed between timed iterations (256 MiB write, untimed); K distinct action buffers"},
         "clocks": clk,
         "e2e": {"value": e2e_value, "unit": UNIT,

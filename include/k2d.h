@@ -43,6 +43,7 @@ extern "C" {
 #define K2D_ERR_CUDA (-6)          /* a CUDA runtime call failed                         */
 #define K2D_ERR_ARG (-7)           /* another argument is invalid                        */
 #define K2D_ERR_LIMIT (-8)         /* a size is beyond a limit built into the library    */
+#define K2D_ERR_WAIT (-9)          /* k2d_status: a wait inside k2d_step ran out (see there) */
 
 #define K2D_MAX_POLYGONS 12
 #define K2D_MAX_CIRCLES 4
@@ -148,12 +149,13 @@ int k2d_reset(k2d_state *s, const int32_t *host_level_ids);
 int k2d_step(k2d_state *s, const float *dev_actions, int32_t n_steps, float *dev_reward, uint8_t *dev_done);
 
 /* The paper has no counterpart of this call; it exists for one kind of user of this library.
- * k2d_step keeps the contact records of a crowded scene (more than 32 touching pairs) in the
- * scratch tail of the state buffer, which the caller has to allocate.  Some callers cannot: a
- * process whose device memory is one arena fixed at start-up, a plug-in handed a pre-sized
- * buffer by its host, code running where cudaMalloc is forbidden (a real-time loop).  For them this variant does exactly what k2d_step does, with the same
+ * k2d_step keeps the contact records of a very crowded scene (far more touching pairs than
+ * lanes working on the scene) in the scratch tail of the state buffer, which the caller has to
+ * allocate.  Some callers cannot: a process whose device memory is one arena fixed at start-up,
+ * a plug-in handed a pre-sized buffer by its host, code running where cudaMalloc is forbidden
+ * (a real-time loop).  For them this variant does exactly what k2d_step does, with the same
  * arguments and bit-identical results, but keeps those records in an array compiled into the
- * library (K2D_STATIC_SCRATCH_MAX_ENVS x 10208 bytes, about 10 MB, resident on every GPU that
+ * library (K2D_STATIC_SCRATCH_MAX_ENVS x 13920 bytes, about 14 MB, resident on every GPU that
  * loads the library until the process exits) and never touches the scratch tail.  It allocates
  * and frees nothing, on the host side of CUDA or on the device.
  *  - n_envs above K2D_STATIC_SCRATCH_MAX_ENVS is refused with K2D_ERR_LIMIT (and a line on
@@ -184,7 +186,11 @@ int k2d_set_state(k2d_state *s, const void *host_canonical);
 
 /* host_counts[8] (int64), all since the last k2d_reset: non-finite events, auto-resets, active
  * manifolds summed over env-steps, env-steps, pairs that passed the bounding-box test (polygon-
- * polygon, polygon-circle, circle-circle), pairs with at least one active manifold. */
+ * polygon, polygon-circle, circle-circle), pairs with at least one active manifold.
+ * Returns K2D_ERR_WAIT (with the counts filled in) if, in some k2d_step since the last k2d_reset,
+ * a group of lanes waited longer than its limit (seconds) for another group to finish an earlier
+ * part of the same env's steps: the kernel then gave up on that env instead of hanging, and the
+ * states are not valid any more; k2d_reset clears the condition. */
 int k2d_status(k2d_state *s, int64_t *host_counts);
 
 /* Host only, no device needed: validates one level against the config and returns the constants

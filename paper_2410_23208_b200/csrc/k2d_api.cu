@@ -17,7 +17,9 @@ using ClassM = SizeClass<6, 3, 2, 2>;
 using ClassL = SizeClass<12, 4, 6, 2>;
 
 constexpr int kMaxSlots = 8192;      // resident scene groups a launch may use (bounds the overflow scratch)
-constexpr size_t kCtrlBytes = 256;   // control block at the start of the state buffer: 8 x uint64 counters
+constexpr size_t kCtrlBytes = 256;   // control block at the start of the state buffer: 8 x uint64 counters, then the work queue words
+constexpr size_t kQueueOffset = 128;
+constexpr int kChunkSteps = 8;       // steps per work item when there are more envs than resident scene groups
 
 // run-time view of a size class
 struct ClassInfo {
@@ -83,11 +85,12 @@ using namespace k2d;
 struct k2d_state {
     k2d_config cfg;
     ClassInfo ci;
-    int G, grid, slots;
+    int G, grid, groups, slots;
     size_t smem_bytes;
     cudaStream_t stream;
     unsigned char *dev_base;
     unsigned long long *dev_counters;
+    unsigned int *dev_queue, *dev_chunks;
     int *dev_ids;
     uint32_t *dev_env, *dev_scratch, *dev_levels;
     float *dev_trace;
@@ -100,12 +103,14 @@ namespace k2d {
 
 static size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
-struct BufLayout { size_t ids_off, env_off, scratch_off, total; int slots; };
+struct BufLayout { size_t ids_off, chunks_off, env_off, scratch_off, total; int slots; };
 static BufLayout buffer_layout(const k2d_config *cfg, const ClassInfo &ci) {
     BufLayout b{};
-    b.slots = cfg->n_envs < kMaxSlots ? cfg->n_envs : kMaxSlots;
+    // every scene group of a launch can end up stepping an env, so the scratch covers whole blocks (up to 16 groups each)
+    b.slots = ((cfg->n_envs < kMaxSlots ? cfg->n_envs : kMaxSlots) + 15) / 16 * 16;
     b.ids_off = kCtrlBytes;
-    b.env_off = align_up(b.ids_off + (size_t)cfg->n_envs * 4, 256);
+    b.chunks_off = align_up(b.ids_off + (size_t)cfg->n_envs * 4, 256);
+    b.env_off = align_up(b.chunks_off + (size_t)cfg->n_envs * 4, 256);
     b.scratch_off = align_up(b.env_off + (size_t)cfg->n_envs * ci.ST_WORDS * 4, 256);
     b.total = align_up(b.scratch_off + (size_t)b.slots * ci.SCRATCH_WORDS * 4, 256);
     return b;
@@ -257,7 +262,31 @@ static cudaError_t setup_step(k2d_state *s, int num_sms) {
     if (grid * GPB > s->slots) grid = s->slots / GPB;
     if (grid < 1) grid = 1;
     s->grid = grid;
+    s->groups = grid * GPB;
     return cudaSuccess;
+}
+
+// Kernel arguments of one k2d_step launch.  With more envs than resident scene groups the launch is cut
+// into chunks of kChunkSteps steps, so that the groups can balance the work between them.
+static StepParams step_params(const k2d_state *s, const float *dev_actions, int n_steps, float *dev_reward, uint8_t *dev_done,
+                              uint32_t *scratch) {
+    const k2d_config &c = s->cfg;
+    StepParams prm{};
+    prm.state = s->dev_env; prm.levels = s->dev_levels; prm.actions = dev_actions; prm.reward = dev_reward; prm.done = dev_done;
+    prm.counters = s->dev_counters; prm.queue = s->dev_queue; prm.chunks_done = s->dev_chunks; prm.scratch = scratch; prm.trace = s->dev_trace;
+    prm.n_envs = c.n_envs; prm.n_steps = n_steps; prm.n_actions = c.n_actions; prm.n_levels = c.n_levels;
+    prm.chunk_steps = n_steps; prm.n_chunks = 1;
+    if (c.n_envs > s->groups && n_steps > kChunkSteps) {
+        const int n_chunks = (n_steps + kChunkSteps - 1) / kChunkSteps;
+        if ((unsigned long long)c.n_envs * (unsigned long long)n_chunks + (unsigned long long)s->groups < 0xffffffffULL) {
+            prm.chunk_steps = kChunkSteps; prm.n_chunks = n_chunks;
+        }
+    }
+    prm.solver_iters = c.solver_iters; prm.warm_start = c.warm_start; prm.auto_reset = c.auto_reset; prm.max_episode_steps = c.max_episode_steps;
+    prm.dt = c.dt; prm.gdt = c.gravity_y * c.dt; prm.contact_alpha = c.contact_alpha; prm.contact_beta = c.contact_beta; prm.slop = c.slop;
+    prm.rest_thr = c.restitution_threshold; prm.face_tol = c.face_tol; prm.joint_alpha = c.joint_alpha; prm.joint_beta = c.joint_beta;
+    prm.motor_rho = c.motor_rho; prm.aabb_margin = c.aabb_margin; prm.seed = c.seed; prm.env_offset = c.env_offset;
+    return prm;
 }
 
 #define K2D_DISPATCH(FN, s, ...)                                                                      \
@@ -319,7 +348,7 @@ int k2d_create(const k2d_config *cfg, void *dev_state_buf, void *dev_level_pool_
     k2d_state *s = new (std::nothrow) k2d_state();
     if (!s) return K2D_ERR_ARG;
     s->cfg = *cfg; s->ci = ci;
-    s->G = cfg->lanes_per_scene ? cfg->lanes_per_scene : 32;
+    s->G = cfg->lanes_per_scene ? cfg->lanes_per_scene : 16;
     s->stream = (cudaStream_t)cfg->cuda_stream;
     s->dev_trace = nullptr;
     // index maps between the caller's scene dimensions and the internal size class
@@ -339,6 +368,8 @@ int k2d_create(const k2d_config *cfg, void *dev_state_buf, void *dev_level_pool_
     s->slots = bl.slots;
     s->dev_base = (unsigned char *)dev_state_buf;
     s->dev_counters = (unsigned long long *)s->dev_base;
+    s->dev_queue = (unsigned int *)(s->dev_base + kQueueOffset);
+    s->dev_chunks = (unsigned int *)(s->dev_base + bl.chunks_off);
     s->dev_ids = (int *)(s->dev_base + bl.ids_off);
     s->dev_env = (uint32_t *)(s->dev_base + bl.env_off);
     s->dev_scratch = (uint32_t *)(s->dev_base + bl.scratch_off);
@@ -363,6 +394,7 @@ int k2d_reset(k2d_state *s, const int32_t *host_level_ids) {
         for (int e = 0; e < E; ++e) if (host_level_ids[e] < 0 || host_level_ids[e] >= s->cfg.n_levels) return K2D_ERR_ARG;
     CUDA_OK(cudaSetDevice(s->cfg.device));
     CUDA_OK(cudaMemsetAsync(s->dev_base, 0, kCtrlBytes, s->stream));
+    CUDA_OK(cudaMemsetAsync(s->dev_chunks, 0, (size_t)E * 4, s->stream));
     if (host_level_ids) CUDA_OK(cudaMemcpyAsync(s->dev_ids, host_level_ids, (size_t)E * 4, cudaMemcpyHostToDevice, s->stream));
     const int *ids = host_level_ids ? s->dev_ids : nullptr;
     if (s->ci.id == 0) k2d_reset_kernel<ClassS><<<E, 64, 0, s->stream>>>(s->dev_env, s->dev_levels, ids, E, s->cfg.n_levels);
@@ -377,15 +409,7 @@ int k2d_step(k2d_state *s, const float *dev_actions, int32_t n_steps, float *dev
     if (!s || !dev_actions || !dev_reward || !dev_done) return K2D_ERR_NULL;
     if (n_steps < 1 || n_steps > s->cfg.max_fused_steps) return K2D_ERR_STEPS;
     if (((uintptr_t)dev_actions & 3) || ((uintptr_t)dev_reward & 3)) return K2D_ERR_ALIGN;
-    const k2d_config &c = s->cfg;
-    StepParams prm{};
-    prm.state = s->dev_env; prm.levels = s->dev_levels; prm.actions = dev_actions; prm.reward = dev_reward; prm.done = dev_done;
-    prm.counters = s->dev_counters; prm.scratch = s->dev_scratch; prm.trace = s->dev_trace;
-    prm.n_envs = c.n_envs; prm.n_steps = n_steps; prm.n_actions = c.n_actions; prm.n_levels = c.n_levels;
-    prm.solver_iters = c.solver_iters; prm.warm_start = c.warm_start; prm.auto_reset = c.auto_reset; prm.max_episode_steps = c.max_episode_steps;
-    prm.dt = c.dt; prm.gdt = c.gravity_y * c.dt; prm.contact_alpha = c.contact_alpha; prm.contact_beta = c.contact_beta; prm.slop = c.slop;
-    prm.rest_thr = c.restitution_threshold; prm.face_tol = c.face_tol; prm.joint_alpha = c.joint_alpha; prm.joint_beta = c.joint_beta;
-    prm.motor_rho = c.motor_rho; prm.aabb_margin = c.aabb_margin; prm.seed = c.seed; prm.env_offset = c.env_offset;
+    const StepParams prm = step_params(s, dev_actions, n_steps, dev_reward, dev_done, s->dev_scratch);
     CUDA_OK(K2D_DISPATCH(launch_step, s, s, prm));
     return K2D_OK;
 }
@@ -497,7 +521,9 @@ int k2d_status(k2d_state *s, int64_t *host_counts) {
     CUDA_OK(cudaSetDevice(s->cfg.device));
     CUDA_OK(cudaStreamSynchronize(s->stream));
     CUDA_OK(cudaMemcpy(host_counts, s->dev_counters, 8 * sizeof(int64_t), cudaMemcpyDeviceToHost));
-    return K2D_OK;
+    unsigned int queue[4] = { 0u, 0u, 0u, 0u };
+    CUDA_OK(cudaMemcpy(queue, s->dev_queue, sizeof(queue), cudaMemcpyDeviceToHost));
+    return queue[Q_ERROR] ? K2D_ERR_WAIT : K2D_OK;
 }
 
 int k2d_level_info(const k2d_config *cfg, const k2d_level *host_level, float *host_inv_mass, float *host_inv_inertia, uint8_t *host_collide) {
@@ -552,7 +578,7 @@ int k2d_step_static_scratch(k2d_state *s, const float *dev_actions, int32_t n_st
     if (n_steps < 1 || n_steps > s->cfg.max_fused_steps) return K2D_ERR_STEPS;
     if (((uintptr_t)dev_actions & 3) || ((uintptr_t)dev_reward & 3)) return K2D_ERR_ALIGN;
     const k2d_config &c = s->cfg;
-    if (c.n_envs > K2D_STATIC_SCRATCH_MAX_ENVS || c.device >= 64) {
+    if (c.n_envs > K2D_STATIC_SCRATCH_MAX_ENVS || s->groups > K2D_STATIC_SCRATCH_MAX_ENVS || c.device >= 64) {
         std::fprintf(stderr, "k2d_step_static_scratch: n_envs = %d is beyond the built-in scratch (at most %d envs); use k2d_step\n",
                      c.n_envs, K2D_STATIC_SCRATCH_MAX_ENVS);
         return K2D_ERR_LIMIT;
@@ -569,15 +595,8 @@ int k2d_step_static_scratch(k2d_state *s, const float *dev_actions, int32_t n_st
         }
         scratch = k2d_static_ptr[c.device];
     }
-    StepParams prm{};
-    prm.state = s->dev_env; prm.levels = s->dev_levels; prm.actions = dev_actions; prm.reward = dev_reward; prm.done = dev_done;
-    prm.counters = s->dev_counters; prm.scratch = scratch; prm.trace = s->dev_trace;
-    prm.n_envs = c.n_envs; prm.n_steps = n_steps; prm.n_actions = c.n_actions; prm.n_levels = c.n_levels;
-    prm.solver_iters = c.solver_iters; prm.warm_start = c.warm_start; prm.auto_reset = c.auto_reset; prm.max_episode_steps = c.max_episode_steps;
-    prm.dt = c.dt; prm.gdt = c.gravity_y * c.dt; prm.contact_alpha = c.contact_alpha; prm.contact_beta = c.contact_beta; prm.slop = c.slop;
-    prm.rest_thr = c.restitution_threshold; prm.face_tol = c.face_tol; prm.joint_alpha = c.joint_alpha; prm.joint_beta = c.joint_beta;
-    prm.motor_rho = c.motor_rho; prm.aabb_margin = c.aabb_margin; prm.seed = c.seed; prm.env_offset = c.env_offset;
-    // the launch of k2d_step never uses more scene groups than envs, so n_envs bounds the scratch slots it touches
+    const StepParams prm = step_params(s, dev_actions, n_steps, dev_reward, dev_done, scratch);
+    // a launch never has more scene groups than envs rounded up to a whole block, so the limit on n_envs bounds the scratch slots
     CUDA_OK(K2D_DISPATCH(launch_step, s, s, prm));
     return K2D_OK;
 }
@@ -593,6 +612,7 @@ const char *k2d_error_string(int code) {
         case K2D_ERR_CUDA: return "CUDA runtime error";
         case K2D_ERR_ARG: return "invalid argument";
         case K2D_ERR_LIMIT: return "size beyond a built-in limit";
+        case K2D_ERR_WAIT: return "a scene group gave up waiting for another; the last step is incomplete";
         default: return "unknown error";
     }
 }

@@ -22,6 +22,8 @@ namespace k2d {
 
 constexpr int kBlockThreads = 128;
 constexpr int kMaxActions = 16;
+enum { Q_TICKET = 0, Q_LEFT = 1, Q_ERROR = 2 };
+constexpr unsigned kWaitLimit = 1u << 24;   // polls (about 100 ns apart) before a wait for another group's chunk gives up
 constexpr int kRecWords = 24;   // contact pair record
 constexpr int kWarmWords = 5;   // pair index + 4 accumulated impulses
 constexpr int kStageWords = 9;  // packed pair word, normal, two contact points with penetration
@@ -110,9 +112,12 @@ struct StepParams {
     float *reward;
     uint8_t *done;
     unsigned long long *counters;
+    unsigned int *queue;       // work queue words: next ticket, groups that have left, error flag
+    unsigned int *chunks_done; // per env: chunks of this launch already stepped (0 again when the launch is over)
     uint32_t *scratch;
     float *trace;
     int n_envs, n_steps, n_actions, n_levels;
+    int chunk_steps, n_chunks;   // a launch is cut into n_chunks pieces of chunk_steps steps; work items are (chunk, env)
     int solver_iters, warm_start, auto_reset, max_episode_steps;
     float dt, gdt, contact_alpha, contact_beta, slop, rest_thr, face_tol, joint_alpha, joint_beta, motor_rho, aabb_margin;
     unsigned long long seed;
@@ -596,7 +601,7 @@ __device__ __noinline__ void warm_in(float *sm, uint32_t *ovf, const uint32_t *s
     for (int k = 2 * G + g.lane; k < nwarm; k += G) {
         uint32_t *wr = ovf + SC::SCRATCH_WARM + (size_t)k * kWarmWords;
 #pragma unroll
-        for (int q = 0; q < kWarmWords; ++q) wr[q] = st_warm[kWarmWords * k + q];
+        for (int q = 0; q < kWarmWords; ++q) wr[q] = __ldcg(st_warm + kWarmWords * k + q);
         widx[wr[0]] = (uint8_t)k;
     }
 }
@@ -1257,17 +1262,19 @@ struct Scene {
     }
 
     // ---- whole launch for one scene
-    __device__ __forceinline__ void run(int e) {
+    // steps s0 .. s1-1 of env e.  The state record may have been written by another SM earlier in this
+    // launch, so it is read past the (non-coherent) L1.
+    __device__ __forceinline__ void run(int e, int s0, int s1) {
         uint32_t *st = prm.state + (size_t)e * SC::ST_WORDS;
-        for (int i = lane; i < 6 * SC::N; i += G) smu[SC::BX + i] = st[SC::ST_BODY + i];
-        if (lane < 5) smu[SC::META + lane] = st[SC::ST_META + lane];
+        for (int i = lane; i < 6 * SC::N; i += G) smu[SC::BX + i] = __ldcg(st + SC::ST_BODY + i);
+        if (lane < 5) smu[SC::META + lane] = __ldcg(st + SC::ST_META + lane);
         if (SC::J > 0 && lane < SC::J) {
-            smu[SC::JROW + JR_ACCX * SC::J + lane] = st[SC::ST_JACC + 2 * lane];
-            smu[SC::JROW + JR_ACCY * SC::J + lane] = st[SC::ST_JACC + 2 * lane + 1];
+            smu[SC::JROW + JR_ACCX * SC::J + lane] = __ldcg(st + SC::ST_JACC + 2 * lane);
+            smu[SC::JROW + JR_ACCY * SC::J + lane] = __ldcg(st + SC::ST_JACC + 2 * lane + 1);
         }
         for (int i = lane; i < (SC::NPAIRS + 3) / 4; i += G) smu[SC::WIDX + i] = 0xffffffffu;
-        const int level = (int)st[SC::ST_META + META_LEVEL];
-        const int nwarm = (int)st[SC::ST_META + META_NWARM];
+        const int level = (int)__ldcg(st + SC::ST_META + META_LEVEL);
+        const int nwarm = (int)__ldcg(st + SC::ST_META + META_NWARM);
         load_level_consts(prm.levels + (size_t)level * SC::LV_WORDS);
         g.sync();
         // accumulated impulses of the previous launch: entry k goes to lane k
@@ -1275,25 +1282,27 @@ struct Scene {
         lanef(LF_ACC2N) = 0.0f; lanef(LF_ACC2T) = 0.0f;
         if (lane < nwarm) {
             const uint32_t *wr = st + SC::ST_WARM + kWarmWords * lane;
-            rec.ab = wr[0] << 12;
-            rec.accn = __uint_as_float(wr[1]); rec.acct = __uint_as_float(wr[2]);
-            lanef(LF_ACC2N) = __uint_as_float(wr[3]); lanef(LF_ACC2T) = __uint_as_float(wr[4]);
-            widx()[wr[0]] = (uint8_t)lane;
+            const uint32_t p = __ldcg(wr);
+            rec.ab = p << 12;
+            rec.accn = __uint_as_float(__ldcg(wr + 1)); rec.acct = __uint_as_float(__ldcg(wr + 2));
+            lanef(LF_ACC2N) = __uint_as_float(__ldcg(wr + 3)); lanef(LF_ACC2T) = __uint_as_float(__ldcg(wr + 4));
+            widx()[p] = (uint8_t)lane;
         }
         if (G + lane < nwarm) {
             const uint32_t *wr = st + SC::ST_WARM + kWarmWords * (G + lane);
-            lanef(LF_OV + R_AB) = __uint_as_float(wr[0] << 12);
-            lanef(LF_OV_ACC0N) = __uint_as_float(wr[1]); lanef(LF_OV_ACC0T) = __uint_as_float(wr[2]);
-            lanef(LF_OV_ACC1N) = __uint_as_float(wr[3]); lanef(LF_OV_ACC1T) = __uint_as_float(wr[4]);
-            widx()[wr[0]] = (uint8_t)(G + lane);
+            const uint32_t p = __ldcg(wr);
+            lanef(LF_OV + R_AB) = __uint_as_float(p << 12);
+            lanef(LF_OV_ACC0N) = __uint_as_float(__ldcg(wr + 1)); lanef(LF_OV_ACC0T) = __uint_as_float(__ldcg(wr + 2));
+            lanef(LF_OV_ACC1N) = __uint_as_float(__ldcg(wr + 3)); lanef(LF_OV_ACC1T) = __uint_as_float(__ldcg(wr + 4));
+            widx()[p] = (uint8_t)(G + lane);
         }
         if (nwarm > 2 * G) warm_in<SC, G>(sm, ovf, st + SC::ST_WARM, nwarm);
         g.sync();
 #pragma unroll 1
-        for (int s = 0; s < prm.n_steps; ++s) {
+        for (int s = s0; s < s1; ++s) {
             step(e, s);
             g.sync();
-            if ((s & 255) == 255) flush_counters();
+            if (((s - s0) & 255) == 255) flush_counters();
         }
         // write back
         for (int i = lane; i < 6 * SC::N; i += G) st[SC::ST_BODY + i] = smu[SC::BX + i];
@@ -1342,8 +1351,52 @@ __global__ void __launch_bounds__(kBlockThreads) k2d_step_kernel(const StepParam
     uint32_t *region = smem_raw + SC::PTAB_WORDS + gib * region_words<SC, G>();
     uint32_t *scratch = prm.scratch + (size_t)slot * SC::SCRATCH_WORDS;
     Scene<SC, G> scene(region, ptab, scratch, prm);
+    // Work items are (chunk, env), handed out in that order by one ticket counter: a group that is done
+    // takes the next item, so groups with cheap scenes take more of them.  Chunk c of an env may start
+    // only when its chunk c - 1 is stepped and its state is back in memory (another group may have done
+    // it); with items handed out chunk by chunk that is almost always long past, else the group waits for
+    // the group that holds it, which is running.
+    const Group<G> &g = scene.g;
+    const unsigned items = (unsigned)prm.n_envs * (unsigned)prm.n_chunks;
 #pragma unroll 1
-    for (int e = slot; e < prm.n_envs; e += nslots) scene.run(e);
+    for (;;) {
+        unsigned t = 0u;
+        if (g.lane == 0) t = atomicAdd(prm.queue + Q_TICKET, 1u);
+        t = g.shflu(t, 0);
+        if (t >= items) break;
+        const int c = (int)(t / (unsigned)prm.n_envs), e = (int)(t - (unsigned)c * (unsigned)prm.n_envs);
+        bool ok = true;
+        if (c > 0) {
+            if (g.lane == 0) {
+                const volatile unsigned int *flag = prm.chunks_done + e;
+                const volatile unsigned int *err = prm.queue + Q_ERROR;
+                unsigned polls = 0u;
+                while (*flag != (unsigned)c) {
+                    if (*err != 0u || ++polls > kWaitLimit) { atomicExch(prm.queue + Q_ERROR, 1u); ok = false; break; }
+                    __nanosleep(100);
+                }
+            }
+            ok = g.shfl(ok ? 1 : 0, 0) != 0;
+            __threadfence();
+        }
+        if (ok) {
+            const int s0 = c * prm.chunk_steps;
+            scene.run(e, s0, min(prm.n_steps, s0 + prm.chunk_steps));
+        }
+        if (prm.n_chunks > 1) {
+            __threadfence();      // this lane's part of the state record is visible before the count moves
+            g.sync();
+            if (g.lane == 0) atomicExch(prm.chunks_done + e, (c + 1 == prm.n_chunks) ? 0u : (unsigned)(c + 1));
+        }
+    }
+    // the last group to leave rewinds the queue for the next launch
+    if (g.lane == 0) {
+        __threadfence();
+        if (atomicAdd(prm.queue + Q_LEFT, 1u) == (unsigned)nslots - 1u) {
+            atomicExch(prm.queue + Q_TICKET, 0u);
+            atomicExch(prm.queue + Q_LEFT, 0u);
+        }
+    }
 }
 
 // ---------------------------------------------------------------- reset kernel: one thread per (env, word)

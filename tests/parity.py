@@ -42,12 +42,12 @@ def errors(env, ref):
     return out, exact
 
 
-def step_both(env, ref, actions_np, chunk=None):
+def step_both(env, ref, actions_np, chunk=None, n_threads=1):
     """Steps both by all rows of actions_np; the GPU in launches of `chunk` fused steps."""
     import torch
     n = actions_np.shape[0]
     chunk = chunk or n
-    r_ref, d_ref = ref.step(actions_np)
+    r_ref, d_ref = ref.step(actions_np, n_threads=n_threads)
     rs, ds = [], []
     for s0 in range(0, n, chunk):
         a = torch.from_numpy(np.ascontiguousarray(actions_np[s0:s0 + chunk])).to(env.device)

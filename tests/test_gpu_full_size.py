@@ -1,0 +1,32 @@
+"""GPU parity at the size and launch configuration the benchmark times: L scenes, 16384 envs, 32 fused
+steps per launch, auto-reset from a pool of 1024 levels with horizon 256.  With more envs than scene
+groups resident on the device, a launch is cut into chunks that the groups hand to one another, so this
+is also the test of that hand-over.  The oracle steps every env (threads over envs)."""
+import os
+
+import numpy as np
+import pytest
+
+from paper_2410_23208_b200 import scenes
+from tests import parity
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.mark.parametrize("lanes,horizon", [(0, 256), (32, 12)])
+def test_benchmark_configuration_matches_the_oracle_on_every_env(lanes, horizon):
+    w = scenes.WORKLOADS[3]
+    seed = scenes.workload_seed(3)
+    lv = scenes.make_levels(w["size"], w["n_levels"], seed, static_prob=w["static_prob"])
+    n_envs, fused = w["n_envs"], 32
+    env, ref = parity.make_pair(lv, n_envs, auto_reset=w["auto_reset"], max_episode_steps=horizon, seed=seed,
+                                max_fused_steps=fused, lanes_per_scene=lanes)
+    act = scenes.make_actions(2 * fused + 5, n_envs, env.n_actions, seed)
+    # two full launches and a short one; the library's default lanes with the benchmark's horizon, and one
+    # warp per scene with a horizon of 12, under which every env resets several times
+    (r, d), (rr, dr) = parity.step_both(env, ref, act, chunk=fused, n_threads=os.cpu_count() or 1)
+    assert np.array_equal(r, rr) and np.array_equal(d, dr)
+    err, exact = parity.errors(env, ref)
+    assert exact, err
+    assert np.array_equal(env.status(), ref.counters)
+    assert d.sum() >= (n_envs * 5 if horizon == 12 else 1)
