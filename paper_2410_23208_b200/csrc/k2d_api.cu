@@ -19,7 +19,10 @@ using ClassL = SizeClass<12, 4, 6, 2>;
 constexpr int kMaxSlots = 8192;      // resident scene groups a launch may use (bounds the overflow scratch)
 constexpr size_t kCtrlBytes = 256;   // control block at the start of the state buffer: 8 x uint64 counters, then the work queue words
 constexpr size_t kQueueOffset = 128;
-constexpr int kChunkSteps = 8;       // steps per work item when there are more envs than resident scene groups
+#ifndef K2D_CHUNK_STEPS
+#define K2D_CHUNK_STEPS 8
+#endif
+constexpr int kChunkSteps = K2D_CHUNK_STEPS;       // steps per work item when there are more envs than resident scene groups
 
 // run-time view of a size class
 struct ClassInfo {

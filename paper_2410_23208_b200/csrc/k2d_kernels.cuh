@@ -21,6 +21,10 @@
 namespace k2d {
 
 constexpr int kBlockThreads = 128;
+#ifndef K2D_MIN_BLOCKS
+#define K2D_MIN_BLOCKS 5
+#endif
+constexpr int kMinBlocks = K2D_MIN_BLOCKS;   // resident blocks per SM the step kernel is compiled for (bounds its registers)
 constexpr int kMaxActions = 16;
 enum { Q_TICKET = 0, Q_LEFT = 1, Q_ERROR = 2 };
 constexpr unsigned kWaitLimit = 1u << 24;   // polls (about 100 ns apart) before a wait for another group's chunk gives up
@@ -67,10 +71,11 @@ struct SizeClass {
     static constexpr int WIDX = SURV + (NPAIRS + 3) / 4; // bytes: pair -> record index of the previous step
     // then, per lane of the group (field-major, G words per field):
     //   STG  kStageWords fields: manifolds on their way to the owning lane; afterwards the second manifold's constants
-    //   ACC2 2 fields: accumulated impulses of the second manifold;  CORR 2 fields: positional corrections
-    //   OV   kRecWords fields: the lane's second record (pair number G + lane of a crowded scene) in memory form
+    //   ACC2 2 fields: accumulated impulses of the second manifold
+    // (the positional corrections of a lane's record, 2 x G words, reuse the world-frame vertex arrays after the narrowphase)
+    // then kRecWords fields of G / 2 words: second records of the lower half of the lanes
     static constexpr int STG = WIDX + (NPAIRS + 3) / 4;
-    static constexpr int LANE_FIELDS = kStageWords + 4 + kRecWords;
+    static constexpr int LANE_FIELDS = kStageWords + 2;
     static constexpr int PTAB_WORDS = ((NPAIRS + 1) / 2 + 3) / 4 * 4;  // block-shared pair table, 16 bits per pair
 };
 // memory form of a contact pair record (the overflow path keeps records in global scratch)
@@ -83,11 +88,12 @@ static_assert(S_PEN1 + 1 == kStageWords, "stage size");
 // second-manifold constants reuse the stage fields of the same lane
 enum { M2_RNA = 0, M2_RNB, M2_RTA, M2_RTB, M2_MASSN, M2_MASST, M2_TARGET };
 // per-lane fields after the stage fields
-enum { LF_ACC2N = kStageWords, LF_ACC2T, LF_CORR0, LF_CORR1, LF_OV };
-// where stage field f of a lane's second record waits inside its memory-form fields (clear of the accumulated impulses)
-__host__ __device__ constexpr int ov_stage(int f) { return LF_OV + (f < 3 ? f : f + 1); }
-constexpr int LF_OV_ACC0N = LF_OV + R_M0 + M_ACCN, LF_OV_ACC0T = LF_OV + R_M0 + M_ACCT;
-constexpr int LF_OV_ACC1N = LF_OV + R_M0 + M_WORDS + M_ACCN, LF_OV_ACC1T = LF_OV + R_M0 + M_WORDS + M_ACCT;
+enum { LF_ACC2N = kStageWords, LF_ACC2T, LF_COUNT };
+// The lower half of the lanes can hold a second record each (pair number G + lane of a crowded scene),
+// in memory form: kRecWords fields of G / 2 words after the per-lane fields.  Stage field f of such a
+// record waits in record field ovs(f), clear of the accumulated impulses.
+__host__ __device__ constexpr int ovs(int f) { return f < 3 ? f : f + 1; }
+constexpr int OV_ACC0N = R_M0 + M_ACCN, OV_ACC0T = R_M0 + M_ACCT, OV_ACC1N = R_M0 + M_WORDS + M_ACCN, OV_ACC1T = R_M0 + M_WORDS + M_ACCT;
 // joint row fields
 enum { JR_RAX = 0, JR_RAY, JR_RBX, JR_RBY, JR_I11, JR_I12, JR_I22, JR_BX, JR_BY, JR_CX, JR_CY, JR_ACCX, JR_ACCY };
 static_assert(JR_ACCY + 1 == kJointWords, "joint row size");
@@ -95,7 +101,10 @@ enum { META_STEP = 0, META_EPISODE, META_LEVEL, META_STATUS, META_NWARM };
 
 // shared-memory words per scene: padded so that the groups of one warp start in different banks
 template <class SC, int G>
-__host__ __device__ constexpr int region_words() { return (SC::STG + SC::LANE_FIELDS * G + 31) / 32 * 32 + (G < 32 ? G : 0); }
+__host__ __device__ constexpr int region_words() {
+    constexpr int raw = SC::STG + SC::LANE_FIELDS * G + kRecWords * (G / 2);
+    return G < 32 ? (raw - G + 31) / 32 * 32 + G : (raw + 3) / 4 * 4;
+}
 
 // body flag word
 constexpr uint32_t F_ACTIVE = 1u, F_DYNAMIC = 2u;
@@ -384,7 +393,7 @@ __device__ __forceinline__ void sweep_joints(float *sm, uint32_t jab, int lane, 
 // Accumulated impulses that pair record `wi` of the previous step left behind (255: the pair was not
 // touching).  Records 0..G-1 live with lane wi (first manifold in its registers: old_n / old_t are the
 // calling lane's own, fetched across lanes here, so every lane of the group must call; second manifold
-// in its shared-memory fields), records G..2G-1 in the second-record fields of lane wi - G, later ones
+// in its shared-memory fields), the next G / 2 records in the second-record fields of lane wi - G, later ones
 // in the warm entries of the global scratch.
 template <class SC, int G>
 __device__ __forceinline__ void warm_lookup(const Group<G> &g, const float *sm, const uint32_t *ovf, int wi, float old_n, float old_t,
@@ -394,9 +403,9 @@ __device__ __forceinline__ void warm_lookup(const Group<G> &g, const float *sm, 
     w[0] = g.shflf(old_n, src); w[1] = g.shflf(old_t, src);
     w[2] = lf[LF_ACC2N * G + src]; w[3] = lf[LF_ACC2T * G + src];
     if (wi >= G && wi != 255) {
-        if (wi < 2 * G) {
-            const float *o = lf + (wi - G);
-            w[0] = o[LF_OV_ACC0N * G]; w[1] = o[LF_OV_ACC0T * G]; w[2] = o[LF_OV_ACC1N * G]; w[3] = o[LF_OV_ACC1T * G];
+        if (wi < G + G / 2) {
+            const float *o = lf + LF_COUNT * G + (wi - G);
+            w[0] = o[OV_ACC0N * (G / 2)]; w[1] = o[OV_ACC0T * (G / 2)]; w[2] = o[OV_ACC1N * (G / 2)]; w[3] = o[OV_ACC1T * (G / 2)];
         } else {
             const uint32_t *wr = ovf + SC::SCRATCH_WARM + (size_t)wi * kWarmWords;
 #pragma unroll
@@ -408,7 +417,7 @@ __device__ __forceinline__ void warm_lookup(const Group<G> &g, const float *sm, 
 
 // Levels of nrec staged pairs by one lane with a per-body table (used when there are more pairs than
 // lanes): a pair's level is one more than the highest level of an earlier pair sharing a movable body.
-// The packed pair words of pairs 0..G-1 are in the stage fields, of G..2G-1 in the second-record
+// The packed pair words of pairs 0..G-1 are in the stage fields, of the next G / 2 in the second-record
 // fields, of later ones in global scratch; the level goes into bits 19.. of each word.
 template <class SC, int G>
 __device__ __forceinline__ int levels_by_one_lane(uint32_t *smu, uint32_t *ovf, int nrec) {
@@ -417,7 +426,7 @@ __device__ __forceinline__ int levels_by_one_lane(uint32_t *smu, uint32_t *ovf, 
     for (int i = 0; i < SC::N; ++i) bl[i] = 0;
     for (int k = 0; k < nrec; ++k) {
         uint32_t *w = (k < G) ? (smu + SC::STG + S_AB * G + k)
-                    : (k < 2 * G) ? (smu + SC::STG + ov_stage(S_AB) * G + (k - G)) : (ovf + (size_t)k * kRecWords + S_AB);
+                    : (k < G + G / 2) ? (smu + SC::STG + LF_COUNT * G + ovs(S_AB) * (G / 2) + (k - G)) : (ovf + (size_t)k * kRecWords + S_AB);
         const uint32_t ab = *w;
         const int a = ab & 31, b = (ab >> 5) & 31;
         int lvl = 1;
@@ -509,11 +518,14 @@ __device__ __noinline__ int slow_solve(float *sm, uint32_t *ovf, const uint32_t 
     __threadfence_block();
     g.sync();
     cmax = g.shfl(cmax, 0);
-    // the staged manifolds of the first 2 G pairs join the others in scratch
+    // the staged manifolds of the first G + G / 2 pairs join the others in scratch
     {
         uint32_t *r = ovf + (size_t)lane * kRecWords, *r2 = ovf + (size_t)(G + lane) * kRecWords;
 #pragma unroll
-        for (int f = 0; f < kStageWords; ++f) { r[f] = smu[SC::STG + f * G + lane]; r2[f] = smu[SC::STG + ov_stage(f) * G + lane]; }
+        for (int f = 0; f < kStageWords; ++f) {
+            r[f] = smu[SC::STG + f * G + lane];
+            if (lane < G / 2) r2[f] = smu[SC::STG + LF_COUNT * G + ovs(f) * (G / 2) + lane];
+        }
     }
     g.sync();
     // pre-step of every pair; accumulated impulses of the previous step come from the lane that
@@ -593,12 +605,12 @@ __device__ __noinline__ int slow_finish(float *sm, uint32_t *ovf, int nrec) {
     return nman;
 }
 
-// Launch boundaries: warm entries 2 G.. between the state record and the scratch.
+// Launch boundaries: warm entries G + G / 2 .. between the state record and the scratch.
 template <class SC, int G>
 __device__ __noinline__ void warm_in(float *sm, uint32_t *ovf, const uint32_t *st_warm, int nwarm) {
     Group<G> g;
     uint8_t *widx = reinterpret_cast<uint8_t *>(reinterpret_cast<uint32_t *>(sm) + SC::WIDX);
-    for (int k = 2 * G + g.lane; k < nwarm; k += G) {
+    for (int k = G + G / 2 + g.lane; k < nwarm; k += G) {
         uint32_t *wr = ovf + SC::SCRATCH_WARM + (size_t)k * kWarmWords;
 #pragma unroll
         for (int q = 0; q < kWarmWords; ++q) wr[q] = __ldcg(st_warm + kWarmWords * k + q);
@@ -608,7 +620,7 @@ __device__ __noinline__ void warm_in(float *sm, uint32_t *ovf, const uint32_t *s
 template <class SC, int G>
 __device__ __noinline__ void warm_out(const uint32_t *ovf, uint32_t *st_warm, int nwarm) {
     Group<G> g;
-    for (int k = 2 * G + g.lane; k < nwarm; k += G) {
+    for (int k = G + G / 2 + g.lane; k < nwarm; k += G) {
         const uint32_t *wr = ovf + SC::SCRATCH_WARM + (size_t)k * kWarmWords;
 #pragma unroll
         for (int q = 0; q < kWarmWords; ++q) st_warm[kWarmWords * k + q] = wr[q];
@@ -619,6 +631,7 @@ __device__ __noinline__ void warm_out(const uint32_t *ovf, uint32_t *st_warm, in
 template <class SC, int G>
 struct Scene {
     static_assert(SC::J <= G && SC::T <= G && kMaxActions <= 2 * G, "one lane per joint / thruster");
+    static_assert(2 * G <= 5 * SC::P4, "positional corrections reuse the world-frame vertex arrays");
     float *sm;            // this scene's shared-memory region
     uint32_t *smu;
     const uint16_t *ptab; // block-shared pair table
@@ -641,6 +654,8 @@ struct Scene {
     __device__ __forceinline__ float4 &box4(int i) { return *reinterpret_cast<float4 *>(sm + SC::BOX + 4 * i); }
     // this lane's word of per-lane field f
     __device__ __forceinline__ float &lanef(int f) { return sm[SC::STG + f * G + lane]; }
+    // this lane's word of field f of its second record (lanes below G / 2 only)
+    __device__ __forceinline__ float &ovl(int f) { return sm[SC::STG + LF_COUNT * G + f * (G / 2) + lane]; }
     __device__ __forceinline__ ContactConsts contact_consts() const {
         ContactConsts cc; cc.slop = prm.slop; cc.rest_thr = prm.rest_thr; cc.alpha = prm.contact_alpha; cc.beta = prm.contact_beta; return cc;
     }
@@ -810,7 +825,7 @@ struct Scene {
         const bool dyn_a = (ab >> 26) & 1u, dyn_b = (ab >> 27) & 1u;
         if (MODE == 2) {
             correct_pair(sm + SC::BX, sm + SC::BY, a, b, amask, dyn_a, dyn_b, rec.nx, rec.ny, rec.ma, rec.mb,
-                         lanef(LF_CORR0), lanef(LF_CORR1));
+                         sm[SC::WVX + lane], sm[SC::WVX + G + lane]);
             return;
         }
         float vax = sm[SC::BVX + a], vay = sm[SC::BVY + a], wa = sm[SC::BW + a];
@@ -831,28 +846,28 @@ struct Scene {
     // pairs), which is in memory form in the lane's shared-memory fields
     template <int MODE>
     __device__ __forceinline__ void visit_pair2() {
-        const uint32_t ab = __float_as_uint(lanef(LF_OV + R_AB));
+        const uint32_t ab = __float_as_uint(ovl(R_AB));
         const int a = ab & 31, b = (ab >> 5) & 31;
         const unsigned amask = (ab >> 10) & 3u;
         const bool dyn_a = (ab >> 26) & 1u, dyn_b = (ab >> 27) & 1u;
-        const float nx = lanef(LF_OV + R_NX), ny = lanef(LF_OV + R_NY);
+        const float nx = ovl(R_NX), ny = ovl(R_NY);
         const float ma = sm[SC::BIM + a], mb = sm[SC::BIM + b];
         if (MODE == 2) {
             correct_pair(sm + SC::BX, sm + SC::BY, a, b, amask, dyn_a, dyn_b, nx, ny, ma, mb,
-                         lanef(LF_OV + R_M0 + M_CORR), lanef(LF_OV + R_M0 + M_WORDS + M_CORR));
+                         ovl(R_M0 + M_CORR), ovl(R_M0 + M_WORDS + M_CORR));
             return;
         }
-        const float ia = sm[SC::BII + a], ib = sm[SC::BII + b], mu = lanef(LF_OV + R_MU);
+        const float ia = sm[SC::BII + a], ib = sm[SC::BII + b], mu = ovl(R_MU);
         float vax = sm[SC::BVX + a], vay = sm[SC::BVY + a], wa = sm[SC::BW + a];
         float vbx = sm[SC::BVX + b], vby = sm[SC::BVY + b], wb = sm[SC::BW + b];
 #pragma unroll
         for (int mi = 0; mi < 2; ++mi) {
             if (amask & (1u << mi)) {
-                const int f = LF_OV + R_M0 + mi * M_WORDS;
-                float accn = lanef(f + M_ACCN), acct = lanef(f + M_ACCT);
-                manifold_rows<MODE>(nx, ny, mu, ma, mb, ia, ib, lanef(f + M_RNA), lanef(f + M_RNB), lanef(f + M_RTA), lanef(f + M_RTB),
-                                    lanef(f + M_MASSN), lanef(f + M_MASST), lanef(f + M_TARGET), accn, acct, vax, vay, wa, vbx, vby, wb);
-                if (MODE == 1) { lanef(f + M_ACCN) = accn; lanef(f + M_ACCT) = acct; }
+                const int f = R_M0 + mi * M_WORDS;
+                float accn = ovl(f + M_ACCN), acct = ovl(f + M_ACCT);
+                manifold_rows<MODE>(nx, ny, mu, ma, mb, ia, ib, ovl(f + M_RNA), ovl(f + M_RNB), ovl(f + M_RTA), ovl(f + M_RTB),
+                                    ovl(f + M_MASSN), ovl(f + M_MASST), ovl(f + M_TARGET), accn, acct, vax, vay, wa, vbx, vby, wb);
+                if (MODE == 1) { ovl(f + M_ACCN) = accn; ovl(f + M_ACCT) = acct; }
             }
         }
         if (dyn_a) { sm[SC::BVX + a] = vax; sm[SC::BVY + a] = vay; sm[SC::BW + a] = wa; }
@@ -1053,11 +1068,12 @@ struct Scene {
                         st[S_AB * G] = __uint_as_float(ab); st[S_NX * G] = nx; st[S_NY * G] = ny;
                         st[S_PX0 * G] = m[0].px; st[S_PY0 * G] = m[0].py; st[S_PEN0 * G] = m[0].pen;
                         st[S_PX1 * G] = m[1].px; st[S_PY1 * G] = m[1].py; st[S_PEN1 * G] = m[1].pen;
-                    } else if (k < 2 * G) {
-                        float *st = sm + SC::STG + (k - G);
-                        st[ov_stage(S_AB) * G] = __uint_as_float(ab); st[ov_stage(S_NX) * G] = nx; st[ov_stage(S_NY) * G] = ny;
-                        st[ov_stage(S_PX0) * G] = m[0].px; st[ov_stage(S_PY0) * G] = m[0].py; st[ov_stage(S_PEN0) * G] = m[0].pen;
-                        st[ov_stage(S_PX1) * G] = m[1].px; st[ov_stage(S_PY1) * G] = m[1].py; st[ov_stage(S_PEN1) * G] = m[1].pen;
+                    } else if (k < G + G / 2) {
+                        float *st = sm + SC::STG + LF_COUNT * G + (k - G);
+                        constexpr int H = G / 2;
+                        st[ovs(S_AB) * H] = __uint_as_float(ab); st[ovs(S_NX) * H] = nx; st[ovs(S_NY) * H] = ny;
+                        st[ovs(S_PX0) * H] = m[0].px; st[ovs(S_PY0) * H] = m[0].py; st[ovs(S_PEN0) * H] = m[0].pen;
+                        st[ovs(S_PX1) * H] = m[1].px; st[ovs(S_PY1) * H] = m[1].py; st[ovs(S_PEN1) * H] = m[1].pen;
                     } else {
                         uint32_t *st = ovf + (size_t)k * kRecWords;
                         st[S_AB] = ab; st[S_NX] = __float_as_uint(nx); st[S_NY] = __float_as_uint(ny);
@@ -1072,7 +1088,7 @@ struct Scene {
         g.sync();
         c_rec += (unsigned)nrec << 16;
 
-        const bool overflow = nrec > 2 * G;
+        const bool overflow = nrec > G + G / 2;
         int cmax = 0, clevel = 0, clevel2 = 0;
         if (overflow) {
             cmax = slow_solve<SC, G>(sm, ovf, lv, nrec, jab, jlevel, jmax, prm.solver_iters, prm.warm_start, prm.motor_rho,
@@ -1101,7 +1117,7 @@ struct Scene {
                 warm_lookup<SC, G>(g, sm, ovf, wi, old_n, old_t, prm.warm_start, w);
                 if (two) {
                     int wi2 = 255;
-                    if (mine2) { ab2 = __float_as_uint(lanef(ov_stage(S_AB))); wi2 = widx()[(ab2 >> 12) & 127]; }
+                    if (mine2) { ab2 = __float_as_uint(ovl(ovs(S_AB))); wi2 = widx()[(ab2 >> 12) & 127]; }
                     warm_lookup<SC, G>(g, sm, ovf, wi2, old_n, old_t, prm.warm_start, w2);
                 }
             }
@@ -1133,18 +1149,17 @@ struct Scene {
                 acc2n = w[2]; acc2t = w[3];
             }
             lanef(LF_ACC2N) = acc2n; lanef(LF_ACC2T) = acc2t;
-            lanef(LF_CORR0) = corr0; lanef(LF_CORR1) = corr1;
+            sm[SC::WVX + lane] = corr0; sm[SC::WVX + G + lane] = corr1;
             if (two) {
                 // the second record of this lane, built in place in its memory-form fields
                 if (mine2) {
                     const int a2 = ab2 & 31, b2 = (ab2 >> 5) & 31;
-                    const float nx2 = lanef(ov_stage(S_NX)), ny2 = lanef(ov_stage(S_NY));
-                    const float pt2[6] = { lanef(ov_stage(S_PX0)), lanef(ov_stage(S_PY0)), lanef(ov_stage(S_PEN0)),
-                                           lanef(ov_stage(S_PX1)), lanef(ov_stage(S_PY1)), lanef(ov_stage(S_PEN1)) };
+                    const float nx2 = ovl(ovs(S_NX)), ny2 = ovl(ovs(S_NY));
+                    const float pt2[6] = { ovl(ovs(S_PX0)), ovl(ovs(S_PY0)), ovl(ovs(S_PEN0)), ovl(ovs(S_PX1)), ovl(ovs(S_PY1)), ovl(ovs(S_PEN1)) };
                     const float ma = sm[SC::BIM + a2], mb = sm[SC::BIM + b2], ia = sm[SC::BII + a2], ib = sm[SC::BII + b2];
                     const float fra = sm[SC::BFR + a2], frb = sm[SC::BFR + b2];
                     const float er2 = fmin_cmp(sm[SC::BRE + a2], sm[SC::BRE + b2]);
-                    lanef(LF_OV + R_MU) = sqrtf(__fmaf_rn(fra, fra, frb * frb));
+                    ovl(R_MU) = sqrtf(__fmaf_rn(fra, fra, frb * frb));
 #pragma unroll
                     for (int mi = 0; mi < 2; ++mi) {
                         float rna = 0.0f, rnb = 0.0f, rta = 0.0f, rtb = 0.0f, massn = 0.0f, masst = 0.0f, target = 0.0f, corr = 0.0f, an = 0.0f, at = 0.0f;
@@ -1153,10 +1168,10 @@ struct Scene {
                                                  rna, rnb, rta, rtb, massn, masst, target, corr);
                             an = w2[2 * mi]; at = w2[2 * mi + 1];
                         }
-                        const int f = LF_OV + R_M0 + mi * M_WORDS;
-                        lanef(f + M_RNA) = rna; lanef(f + M_RNB) = rnb; lanef(f + M_RTA) = rta; lanef(f + M_RTB) = rtb;
-                        lanef(f + M_MASSN) = massn; lanef(f + M_MASST) = masst; lanef(f + M_TARGET) = target; lanef(f + M_CORR) = corr;
-                        lanef(f + M_ACCN) = an; lanef(f + M_ACCT) = at;
+                        const int f = R_M0 + mi * M_WORDS;
+                        ovl(f + M_RNA) = rna; ovl(f + M_RNB) = rnb; ovl(f + M_RTA) = rta; ovl(f + M_RTB) = rtb;
+                        ovl(f + M_MASSN) = massn; ovl(f + M_MASST) = masst; ovl(f + M_TARGET) = target; ovl(f + M_CORR) = corr;
+                        ovl(f + M_ACCN) = an; ovl(f + M_ACCT) = at;
                     }
                     clevel2 = (int)((ab2 >> 19) & 127u);
                 }
@@ -1214,17 +1229,19 @@ struct Scene {
         g.sync();
         if (overflow) {
             c_man += (unsigned)slow_finish<SC, G>(sm, ovf, nrec);
-            // the first 2 G pairs go back to their lanes
+            // the first G + G / 2 pairs go back to their lanes
             const uint32_t *wr = ovf + SC::SCRATCH_WARM + (size_t)lane * kWarmWords, *wr2 = wr + (size_t)G * kWarmWords;
             rec.ab = wr[0] << 12;
             rec.accn = __uint_as_float(wr[1]); rec.acct = __uint_as_float(wr[2]);
             lanef(LF_ACC2N) = __uint_as_float(wr[3]); lanef(LF_ACC2T) = __uint_as_float(wr[4]);
-            lanef(LF_OV + R_AB) = __uint_as_float(wr2[0] << 12);
-            lanef(LF_OV_ACC0N) = __uint_as_float(wr2[1]); lanef(LF_OV_ACC0T) = __uint_as_float(wr2[2]);
-            lanef(LF_OV_ACC1N) = __uint_as_float(wr2[3]); lanef(LF_OV_ACC1T) = __uint_as_float(wr2[4]);
+            if (lane < G / 2) {
+                ovl(R_AB) = __uint_as_float(wr2[0] << 12);
+                ovl(OV_ACC0N) = __uint_as_float(wr2[1]); ovl(OV_ACC0T) = __uint_as_float(wr2[2]);
+                ovl(OV_ACC1N) = __uint_as_float(wr2[3]); ovl(OV_ACC1T) = __uint_as_float(wr2[4]);
+            }
         } else {
             if (lane < nrec) widx()[(rec.ab >> 12) & 127] = (uint8_t)lane;
-            if (clevel2 != 0) widx()[(__float_as_uint(lanef(LF_OV + R_AB)) >> 12) & 127] = (uint8_t)(G + lane);
+            if (clevel2 != 0) widx()[(__float_as_uint(ovl(R_AB)) >> 12) & 127] = (uint8_t)(G + lane);
         }
 
         // reward, termination, counters, auto-reset
@@ -1288,15 +1305,15 @@ struct Scene {
             lanef(LF_ACC2N) = __uint_as_float(__ldcg(wr + 3)); lanef(LF_ACC2T) = __uint_as_float(__ldcg(wr + 4));
             widx()[p] = (uint8_t)lane;
         }
-        if (G + lane < nwarm) {
+        if (lane < G / 2 && G + lane < nwarm) {
             const uint32_t *wr = st + SC::ST_WARM + kWarmWords * (G + lane);
             const uint32_t p = __ldcg(wr);
-            lanef(LF_OV + R_AB) = __uint_as_float(p << 12);
-            lanef(LF_OV_ACC0N) = __uint_as_float(__ldcg(wr + 1)); lanef(LF_OV_ACC0T) = __uint_as_float(__ldcg(wr + 2));
-            lanef(LF_OV_ACC1N) = __uint_as_float(__ldcg(wr + 3)); lanef(LF_OV_ACC1T) = __uint_as_float(__ldcg(wr + 4));
+            ovl(R_AB) = __uint_as_float(p << 12);
+            ovl(OV_ACC0N) = __uint_as_float(__ldcg(wr + 1)); ovl(OV_ACC0T) = __uint_as_float(__ldcg(wr + 2));
+            ovl(OV_ACC1N) = __uint_as_float(__ldcg(wr + 3)); ovl(OV_ACC1T) = __uint_as_float(__ldcg(wr + 4));
             widx()[p] = (uint8_t)(G + lane);
         }
-        if (nwarm > 2 * G) warm_in<SC, G>(sm, ovf, st + SC::ST_WARM, nwarm);
+        if (nwarm > G + G / 2) warm_in<SC, G>(sm, ovf, st + SC::ST_WARM, nwarm);
         g.sync();
 #pragma unroll 1
         for (int s = s0; s < s1; ++s) {
@@ -1318,13 +1335,13 @@ struct Scene {
             wr[1] = __float_as_uint(rec.accn); wr[2] = __float_as_uint(rec.acct);
             wr[3] = __float_as_uint(lanef(LF_ACC2N)); wr[4] = __float_as_uint(lanef(LF_ACC2T));
         }
-        if (G + lane < nw) {
+        if (lane < G / 2 && G + lane < nw) {
             uint32_t *wr = st + SC::ST_WARM + kWarmWords * (G + lane);
-            wr[0] = (__float_as_uint(lanef(LF_OV + R_AB)) >> 12) & 127u;
-            wr[1] = __float_as_uint(lanef(LF_OV_ACC0N)); wr[2] = __float_as_uint(lanef(LF_OV_ACC0T));
-            wr[3] = __float_as_uint(lanef(LF_OV_ACC1N)); wr[4] = __float_as_uint(lanef(LF_OV_ACC1T));
+            wr[0] = (__float_as_uint(ovl(R_AB)) >> 12) & 127u;
+            wr[1] = __float_as_uint(ovl(OV_ACC0N)); wr[2] = __float_as_uint(ovl(OV_ACC0T));
+            wr[3] = __float_as_uint(ovl(OV_ACC1N)); wr[4] = __float_as_uint(ovl(OV_ACC1T));
         }
-        if (nw > 2 * G) warm_out<SC, G>(ovf, st + SC::ST_WARM, nw);
+        if (nw > G + G / 2) warm_out<SC, G>(ovf, st + SC::ST_WARM, nw);
         flush_counters();
         g.sync();
     }
@@ -1340,7 +1357,7 @@ __device__ __forceinline__ uint16_t pair_code(int p) {
 }
 
 template <class SC, int G>
-__global__ void __launch_bounds__(kBlockThreads) k2d_step_kernel(const StepParams prm) {
+__global__ void __launch_bounds__(kBlockThreads, kMinBlocks) k2d_step_kernel(const StepParams prm) {
     extern __shared__ __align__(16) uint32_t smem_raw[];
     constexpr int GPB = kBlockThreads / G;
     uint16_t *ptab = reinterpret_cast<uint16_t *>(smem_raw);
