@@ -420,7 +420,7 @@ __device__ __forceinline__ void warm_lookup(const Group<G> &g, const float *sm, 
 // The packed pair words of pairs 0..G-1 are in the stage fields, of the next G / 2 in the second-record
 // fields, of later ones in global scratch; the level goes into bits 19.. of each word.
 template <class SC, int G>
-__device__ __forceinline__ int levels_by_one_lane(uint32_t *smu, uint32_t *ovf, int nrec) {
+__device__ __noinline__ int levels_by_one_lane(uint32_t *smu, uint32_t *ovf, int nrec) {
     uint8_t *bl = reinterpret_cast<uint8_t *>(smu + SC::SURV);   // the survivor list is no longer needed
     int cmax = 0;
     for (int i = 0; i < SC::N; ++i) bl[i] = 0;
@@ -627,6 +627,160 @@ __device__ __noinline__ void warm_out(const uint32_t *ovf, uint32_t *st_warm, in
     }
 }
 
+// ---- one visit of the calling lane's second record (pair number G + lane of a scene with more than G
+// touching pairs), which is in memory form in the lane's shared-memory fields.  MODE as for the first record.
+template <class SC, int G, int MODE>
+__device__ __noinline__ void visit_second(float *sm) {
+    float *ov = sm + SC::STG + LF_COUNT * G + Group<G>().lane;
+    constexpr int H = G / 2;
+    const uint32_t ab = __float_as_uint(ov[R_AB * H]);
+    const int a = ab & 31, b = (ab >> 5) & 31;
+    const unsigned amask = (ab >> 10) & 3u;
+    const bool dyn_a = (ab >> 26) & 1u, dyn_b = (ab >> 27) & 1u;
+    const float nx = ov[R_NX * H], ny = ov[R_NY * H];
+    const float ma = sm[SC::BIM + a], mb = sm[SC::BIM + b];
+    if (MODE == 2) {
+        correct_pair(sm + SC::BX, sm + SC::BY, a, b, amask, dyn_a, dyn_b, nx, ny, ma, mb, ov[(R_M0 + M_CORR) * H], ov[(R_M0 + M_WORDS + M_CORR) * H]);
+        return;
+    }
+    const float ia = sm[SC::BII + a], ib = sm[SC::BII + b], mu = ov[R_MU * H];
+    float vax = sm[SC::BVX + a], vay = sm[SC::BVY + a], wa = sm[SC::BW + a];
+    float vbx = sm[SC::BVX + b], vby = sm[SC::BVY + b], wb = sm[SC::BW + b];
+#pragma unroll 1
+    for (int mi = 0; mi < 2; ++mi) {
+        if (amask & (1u << mi)) {
+            float *m = ov + (R_M0 + mi * M_WORDS) * H;
+            float accn = m[M_ACCN * H], acct = m[M_ACCT * H];
+            manifold_rows<MODE>(nx, ny, mu, ma, mb, ia, ib, m[M_RNA * H], m[M_RNB * H], m[M_RTA * H], m[M_RTB * H],
+                                m[M_MASSN * H], m[M_MASST * H], m[M_TARGET * H], accn, acct, vax, vay, wa, vbx, vby, wb);
+            if (MODE == 1) { m[M_ACCN * H] = accn; m[M_ACCT * H] = acct; }
+        }
+    }
+    if (dyn_a) { sm[SC::BVX + a] = vax; sm[SC::BVY + a] = vay; sm[SC::BW + a] = wa; }
+    if (dyn_b) { sm[SC::BVX + b] = vbx; sm[SC::BVY + b] = vby; sm[SC::BW + b] = wb; }
+}
+
+// Second records, first half: the accumulated impulses the staged pair G + lane carried out of the
+// previous step, parked in four of the lane's second-record fields that are free until the record is built.
+template <class SC, int G>
+__device__ __noinline__ void second_lookup(float *sm, const uint32_t *ovf, int nrec, float old_n, float old_t, int warm_start) {
+    const Group<G> g;
+    constexpr int H = G / 2;
+    float *ov = sm + SC::STG + LF_COUNT * G + g.lane;
+    const uint8_t *widx = reinterpret_cast<const uint8_t *>(reinterpret_cast<const uint32_t *>(sm) + SC::WIDX);
+    const bool mine2 = g.lane < H && G + g.lane < nrec;
+    int wi2 = 255;
+    if (mine2) wi2 = widx[(__float_as_uint(ov[ovs(S_AB) * H]) >> 12) & 127];
+    float w2[4];
+    warm_lookup<SC, G>(g, sm, ovf, wi2, old_n, old_t, warm_start, w2);
+    if (mine2) {
+#pragma unroll
+        for (int q = 0; q < 4; ++q) ov[(R_M0 + M_WORDS + q) * H] = w2[q];
+    }
+}
+// Second half, after every lane has read what it needs from other lanes: the record is built in place.
+// Returns its level | its number of active manifolds << 8 (0 for a lane without a second record).
+template <class SC, int G>
+__device__ __noinline__ unsigned second_build(float *sm, int nrec, ContactConsts cc) {
+    const int lane = Group<G>().lane;
+    constexpr int H = G / 2;
+    if (!(lane < H && G + lane < nrec)) return 0u;
+    float *ov = sm + SC::STG + LF_COUNT * G + lane;
+    const uint32_t ab2 = __float_as_uint(ov[ovs(S_AB) * H]);
+    const int a2 = ab2 & 31, b2 = (ab2 >> 5) & 31;
+    const float nx2 = ov[ovs(S_NX) * H], ny2 = ov[ovs(S_NY) * H];
+    const float pt2[6] = { ov[ovs(S_PX0) * H], ov[ovs(S_PY0) * H], ov[ovs(S_PEN0) * H], ov[ovs(S_PX1) * H], ov[ovs(S_PY1) * H], ov[ovs(S_PEN1) * H] };
+    float w2[4];
+#pragma unroll
+    for (int q = 0; q < 4; ++q) w2[q] = ov[(R_M0 + M_WORDS + q) * H];
+    const float ma = sm[SC::BIM + a2], mb = sm[SC::BIM + b2], ia = sm[SC::BII + a2], ib = sm[SC::BII + b2];
+    const float fra = sm[SC::BFR + a2], frb = sm[SC::BFR + b2];
+    const float er2 = fmin_cmp(sm[SC::BRE + a2], sm[SC::BRE + b2]);
+    ov[R_MU * H] = sqrtf(__fmaf_rn(fra, fra, frb * frb));
+#pragma unroll 1
+    for (int mi = 0; mi < 2; ++mi) {
+        float rna = 0.0f, rnb = 0.0f, rta = 0.0f, rtb = 0.0f, massn = 0.0f, masst = 0.0f, target = 0.0f, corr = 0.0f, an = 0.0f, at = 0.0f;
+        if ((ab2 >> 10) & (1u << mi)) {
+            prestep_manifold<SC>(a2, b2, nx2, ny2, ma, mb, ia, ib, pt2[3 * mi], pt2[3 * mi + 1], pt2[3 * mi + 2], er2, sm, cc,
+                                 rna, rnb, rta, rtb, massn, masst, target, corr);
+            an = w2[2 * mi]; at = w2[2 * mi + 1];
+        }
+        float *m = ov + (R_M0 + mi * M_WORDS) * H;
+        m[M_RNA * H] = rna; m[M_RNB * H] = rnb; m[M_RTA * H] = rta; m[M_RTB * H] = rtb;
+        m[M_MASSN * H] = massn; m[M_MASST * H] = masst; m[M_TARGET * H] = target; m[M_CORR * H] = corr;
+        m[M_ACCN * H] = an; m[M_ACCT * H] = at;
+    }
+    return ((ab2 >> 19) & 127u) | ((unsigned)__popc((ab2 >> 10) & 3u) << 8);
+}
+
+// ================================================================ rarely run code, kept out of line
+// so that the code a step normally runs stays small
+// level constants into shared memory; returns the packed word of joint number `lane` (0 beyond the last joint)
+template <class SC, int G>
+__device__ __noinline__ uint32_t load_level_consts(uint32_t *smu, const uint32_t *lv) {
+    const int lane = Group<G>().lane;
+    for (int i = lane; i < SC::N; i += G) {
+        smu[SC::BIM + i] = lv[SC::LV_IM + i];
+        smu[SC::BII + i] = lv[SC::LV_II + i];
+        smu[SC::BFR + i] = lv[SC::LV_FR + i];
+        smu[SC::BRE + i] = lv[SC::LV_RE + i];
+        smu[SC::BFL + i] = lv[SC::LV_FLAGS + i];
+    }
+    for (int i = lane; i < SC::C; i += G) smu[SC::RAD + i] = lv[SC::LV_RAD + i];
+    for (int i = lane; i < SC::MASKW; i += G) smu[SC::MASK + i] = lv[SC::LV_MASK + i];
+    return (SC::J > 0 && lane < SC::J) ? lv[SC::LV_JOINT + 8 * lane] : 0u;
+}
+
+// Auto-reset of a finished env: next level (its own, or drawn from the pool by the hash of seed,
+// global env index and episode), pose from the level, no accumulated impulses, counters.  Returns the
+// packed word of joint number `lane` of the level the env is on afterwards.
+template <class SC, int G>
+__device__ __noinline__ uint32_t reset_env(uint32_t *smu, const uint32_t *levels, int n_levels, int auto_reset, unsigned long long seed,
+                                           long long env_index, unsigned long long *counters, uint32_t jab) {
+    Group<G> g;
+    const int lane = g.lane;
+    const int episode = (int)smu[SC::META + META_EPISODE] + 1;
+    int level = (int)smu[SC::META + META_LEVEL];
+    g.sync();
+    if (auto_reset == 2) {
+        const unsigned long long h = mix64(seed + ((unsigned long long)env_index + 1ULL) * 0x9E3779B97F4A7C15ULL +
+                                           (unsigned long long)episode * 0xD1B54A32D192ED03ULL);
+        const int nl = (int)(h % (unsigned long long)n_levels);
+        if (nl != level) { level = nl; jab = load_level_consts<SC, G>(smu, levels + (size_t)nl * SC::LV_WORDS); }
+    }
+    const uint32_t *lv = levels + (size_t)level * SC::LV_WORDS;
+    for (int i = lane; i < 6 * SC::N; i += G) smu[SC::BX + i] = lv[SC::LV_X + i];
+    if (SC::J > 0 && lane < SC::J) { smu[SC::JROW + JR_ACCX * SC::J + lane] = 0u; smu[SC::JROW + JR_ACCY * SC::J + lane] = 0u; }
+    for (int i = lane; i < (SC::NPAIRS + 3) / 4; i += G) smu[SC::WIDX + i] = 0xffffffffu;
+    if (lane == 0) {
+        smu[SC::META + META_STEP] = 0u; smu[SC::META + META_EPISODE] = (uint32_t)episode; smu[SC::META + META_LEVEL] = (uint32_t)level;
+        smu[SC::META + META_STATUS] = 0u; smu[SC::META + META_NWARM] = 0u;
+        atomicAdd(counters + 1, 1ULL);
+    }
+    g.sync();
+    return jab;
+}
+
+// packed work counters of a group to the global ones (lane 0)
+__device__ __noinline__ void flush_counters(unsigned long long *counters, unsigned c_surv, unsigned c_rec, unsigned c_man) {
+    const unsigned v[6] = { c_man & 0xffffu, c_man >> 16, c_surv & 0xffffu, c_surv >> 16, c_rec & 0xffffu, c_rec >> 16 };
+#pragma unroll 1
+    for (int q = 0; q < 6; ++q) if (v[q]) atomicAdd(counters + 2 + q, (unsigned long long)v[q]);
+}
+
+// debug trace of one pair's manifolds
+__device__ __noinline__ void trace_pair(float *t, int nm, unsigned act, float px0, float py0, float pen0, float px1, float py1, float pen1,
+                                        float nx0, float ny0, float nx1, float ny1) {
+    t[0] = px0; t[1] = py0; t[2] = nx0; t[3] = ny0; t[4] = pen0; t[5] = (act & 1u) ? 1.0f : 0.0f;
+    if (nm > 1) { t[6] = px1; t[7] = py1; t[8] = nx1; t[9] = ny1; t[10] = pen1; t[11] = (act & 2u) ? 1.0f : 0.0f; }
+}
+template <class SC, int G>
+__device__ __noinline__ void trace_clear(float *trace) {
+    const Group<G> g;
+    for (int i = g.lane; i < SC::NSLOTS * 6; i += G) trace[i] = ((i % 6) == 3) ? 1.0f : ((i % 6) == 4 ? -1.0f : 0.0f);
+    g.sync();
+}
+
 // ---------------------------------------------------------------- scene processing
 template <class SC, int G>
 struct Scene {
@@ -659,36 +813,9 @@ struct Scene {
     __device__ __forceinline__ ContactConsts contact_consts() const {
         ContactConsts cc; cc.slop = prm.slop; cc.rest_thr = prm.rest_thr; cc.alpha = prm.contact_alpha; cc.beta = prm.contact_beta; return cc;
     }
-    __device__ __forceinline__ void flush_counters() {
-        if (lane == 0) {
-            const unsigned v[5] = { c_man & 0xffffu, c_man >> 16, c_surv & 0xffffu, c_surv >> 16, c_rec & 0xffffu };
-            if (v[0]) atomicAdd(prm.counters + 2, (unsigned long long)v[0]);
-            if (v[1]) atomicAdd(prm.counters + 3, (unsigned long long)v[1]);
-            if (v[2]) atomicAdd(prm.counters + 4, (unsigned long long)v[2]);
-            if (v[3]) atomicAdd(prm.counters + 5, (unsigned long long)v[3]);
-            if (v[4]) atomicAdd(prm.counters + 6, (unsigned long long)v[4]);
-            if (c_rec >> 16) atomicAdd(prm.counters + 7, (unsigned long long)(c_rec >> 16));
-        }
+    __device__ __forceinline__ void flush() {
+        if (lane == 0) flush_counters(prm.counters, c_surv, c_rec, c_man);
         c_surv = 0u; c_rec = 0u; c_man = 0u;
-    }
-
-    // ---- level constants into shared memory / registers
-    __device__ __forceinline__ void load_level_consts(const uint32_t *lv) {
-        for (int i = lane; i < SC::N; i += G) {
-            smu[SC::BIM + i] = lv[SC::LV_IM + i];
-            smu[SC::BII + i] = lv[SC::LV_II + i];
-            smu[SC::BFR + i] = lv[SC::LV_FR + i];
-            smu[SC::BRE + i] = lv[SC::LV_RE + i];
-            smu[SC::BFL + i] = lv[SC::LV_FLAGS + i];
-        }
-        for (int i = lane; i < SC::C; i += G) smu[SC::RAD + i] = lv[SC::LV_RAD + i];
-        for (int i = lane; i < SC::MASKW; i += G) smu[SC::MASK + i] = lv[SC::LV_MASK + i];
-        jab = (SC::J > 0 && lane < SC::J) ? lv[SC::LV_JOINT + 8 * lane] : 0u;
-    }
-    __device__ __forceinline__ void load_level_pose(const uint32_t *lv) {
-        for (int i = lane; i < 6 * SC::N; i += G) smu[SC::BX + i] = lv[SC::LV_X + i];
-        if (SC::J > 0 && lane < SC::J) { sm[SC::JROW + JR_ACCX * SC::J + lane] = 0.0f; sm[SC::JROW + JR_ACCY * SC::J + lane] = 0.0f; }
-        for (int i = lane; i < (SC::NPAIRS + 3) / 4; i += G) smu[SC::WIDX + i] = 0xffffffffu;
     }
 
     // ---- narrowphase: polygon a against polygon b (world data in shared memory)
@@ -842,44 +969,13 @@ struct Scene {
         if (dyn_a) { sm[SC::BVX + a] = vax; sm[SC::BVY + a] = vay; sm[SC::BW + a] = wa; }
         if (dyn_b) { sm[SC::BVX + b] = vbx; sm[SC::BVY + b] = vby; sm[SC::BW + b] = wb; }
     }
-    // ---- the same for the lane's second record (pair number G + lane of a scene with more than G touching
-    // pairs), which is in memory form in the lane's shared-memory fields
-    template <int MODE>
-    __device__ __forceinline__ void visit_pair2() {
-        const uint32_t ab = __float_as_uint(ovl(R_AB));
-        const int a = ab & 31, b = (ab >> 5) & 31;
-        const unsigned amask = (ab >> 10) & 3u;
-        const bool dyn_a = (ab >> 26) & 1u, dyn_b = (ab >> 27) & 1u;
-        const float nx = ovl(R_NX), ny = ovl(R_NY);
-        const float ma = sm[SC::BIM + a], mb = sm[SC::BIM + b];
-        if (MODE == 2) {
-            correct_pair(sm + SC::BX, sm + SC::BY, a, b, amask, dyn_a, dyn_b, nx, ny, ma, mb,
-                         ovl(R_M0 + M_CORR), ovl(R_M0 + M_WORDS + M_CORR));
-            return;
-        }
-        const float ia = sm[SC::BII + a], ib = sm[SC::BII + b], mu = ovl(R_MU);
-        float vax = sm[SC::BVX + a], vay = sm[SC::BVY + a], wa = sm[SC::BW + a];
-        float vbx = sm[SC::BVX + b], vby = sm[SC::BVY + b], wb = sm[SC::BW + b];
-#pragma unroll
-        for (int mi = 0; mi < 2; ++mi) {
-            if (amask & (1u << mi)) {
-                const int f = R_M0 + mi * M_WORDS;
-                float accn = ovl(f + M_ACCN), acct = ovl(f + M_ACCT);
-                manifold_rows<MODE>(nx, ny, mu, ma, mb, ia, ib, ovl(f + M_RNA), ovl(f + M_RNB), ovl(f + M_RTA), ovl(f + M_RTB),
-                                    ovl(f + M_MASSN), ovl(f + M_MASST), ovl(f + M_TARGET), accn, acct, vax, vay, wa, vbx, vby, wb);
-                if (MODE == 1) { ovl(f + M_ACCN) = accn; ovl(f + M_ACCT) = acct; }
-            }
-        }
-        if (dyn_a) { sm[SC::BVX + a] = vax; sm[SC::BVY + a] = vay; sm[SC::BW + a] = wa; }
-        if (dyn_b) { sm[SC::BVX + b] = vbx; sm[SC::BVY + b] = vby; sm[SC::BW + b] = wb; }
-    }
     // records of one level touch disjoint movable bodies; levels in order keep the record order
     template <int MODE>
     __device__ __forceinline__ void sweep_pairs(int cmax, int clevel, int clevel2) {
 #pragma unroll 1
         for (int lvl = 1; lvl <= cmax; ++lvl) {
             if (clevel == lvl) visit_pair<MODE>();
-            if (clevel2 == lvl) visit_pair2<MODE>();
+            if (clevel2 == lvl) visit_second<SC, G, MODE>(sm);
             g.sync();
         }
     }
@@ -1022,10 +1118,7 @@ struct Scene {
         int nrec = 0;
         bool t_gb = false, t_gr = false;
         float *trace = prm.trace ? prm.trace + (size_t)e * SC::NSLOTS * 6 : nullptr;
-        if (trace) {
-            for (int i = lane; i < SC::NSLOTS * 6; i += G) trace[i] = ((i % 6) == 3) ? 1.0f : ((i % 6) == 4 ? -1.0f : 0.0f);
-            g.sync();
-        }
+        if (trace) trace_clear<SC, G>(trace);
 #pragma unroll 1
         for (int kind = 0; kind < 3; ++kind) {
             const int lo = kind == 0 ? 0 : (kind == 1 ? ns_pp : ns_pc);
@@ -1043,15 +1136,9 @@ struct Scene {
                     else if (kind == 1) act = manifold_pc(a, b, m[0], lv);
                     else act = manifold_cc(a, b, m[0]);
                     // a polygon pair rejected before its manifolds exist leaves its slots at the default
-                    if (trace && !(kind == 0 && act == 0u)) {
-                        const int slot = (p < SC::NPP) ? 2 * p : SC::NPP + p;
-                        const int nm = (kind == 0) ? 2 : 1;
-                        for (int mi = 0; mi < nm; ++mi) {
-                            float *t = trace + (slot + mi) * 6;
-                            t[0] = m[mi].px; t[1] = m[mi].py; t[2] = m[mi].nx; t[3] = m[mi].ny; t[4] = m[mi].pen;
-                            t[5] = ((act >> mi) & 1u) ? 1.0f : 0.0f;
-                        }
-                    }
+                    if (trace && !(kind == 0 && act == 0u))
+                        trace_pair(trace + ((p < SC::NPP) ? 2 * p : SC::NPP + p) * 6, (kind == 0) ? 2 : 1, act, m[0].px, m[0].py, m[0].pen,
+                                   m[1].px, m[1].py, m[1].pen, m[0].nx, m[0].ny, m[1].nx, m[1].ny);
                 }
                 const unsigned bal = g.ballot(act != 0u);
                 if (act) {
@@ -1102,10 +1189,10 @@ struct Scene {
             }
             // every staged pair becomes a record in its own lane: accumulated impulses of the same pair in the
             // previous step come from wherever its record was then
-            const bool mine = lane < nrec, mine2 = two && G + lane < nrec;
-            uint32_t ab = 0u, ab2 = 0u;
+            const bool mine = lane < nrec;
+            uint32_t ab = 0u;
             float nx = 0.0f, ny = 0.0f, pt[6] = { 0.0f, 0.0f, 0.0f, 0.0f, 0.0f, 0.0f };
-            float w[4], w2[4];
+            float w[4];
             {
                 int wi = 255;
                 if (mine) {
@@ -1115,11 +1202,7 @@ struct Scene {
                 }
                 const float old_n = rec.accn, old_t = rec.acct;
                 warm_lookup<SC, G>(g, sm, ovf, wi, old_n, old_t, prm.warm_start, w);
-                if (two) {
-                    int wi2 = 255;
-                    if (mine2) { ab2 = __float_as_uint(ovl(ovs(S_AB))); wi2 = widx()[(ab2 >> 12) & 127]; }
-                    warm_lookup<SC, G>(g, sm, ovf, wi2, old_n, old_t, prm.warm_start, w2);
-                }
+                if (two) second_lookup<SC, G>(sm, ovf, nrec, old_n, old_t, prm.warm_start);
             }
             g.sync();     // every lane has read the fields it needs from other lanes before they are rewritten
             const int a = ab & 31, b = (ab >> 5) & 31;
@@ -1151,33 +1234,11 @@ struct Scene {
             lanef(LF_ACC2N) = acc2n; lanef(LF_ACC2T) = acc2t;
             sm[SC::WVX + lane] = corr0; sm[SC::WVX + G + lane] = corr1;
             if (two) {
-                // the second record of this lane, built in place in its memory-form fields
-                if (mine2) {
-                    const int a2 = ab2 & 31, b2 = (ab2 >> 5) & 31;
-                    const float nx2 = ovl(ovs(S_NX)), ny2 = ovl(ovs(S_NY));
-                    const float pt2[6] = { ovl(ovs(S_PX0)), ovl(ovs(S_PY0)), ovl(ovs(S_PEN0)), ovl(ovs(S_PX1)), ovl(ovs(S_PY1)), ovl(ovs(S_PEN1)) };
-                    const float ma = sm[SC::BIM + a2], mb = sm[SC::BIM + b2], ia = sm[SC::BII + a2], ib = sm[SC::BII + b2];
-                    const float fra = sm[SC::BFR + a2], frb = sm[SC::BFR + b2];
-                    const float er2 = fmin_cmp(sm[SC::BRE + a2], sm[SC::BRE + b2]);
-                    ovl(R_MU) = sqrtf(__fmaf_rn(fra, fra, frb * frb));
-#pragma unroll
-                    for (int mi = 0; mi < 2; ++mi) {
-                        float rna = 0.0f, rnb = 0.0f, rta = 0.0f, rtb = 0.0f, massn = 0.0f, masst = 0.0f, target = 0.0f, corr = 0.0f, an = 0.0f, at = 0.0f;
-                        if ((ab2 >> 10) & (1u << mi)) {
-                            prestep_manifold<SC>(a2, b2, nx2, ny2, ma, mb, ia, ib, pt2[3 * mi], pt2[3 * mi + 1], pt2[3 * mi + 2], er2, sm, cc,
-                                                 rna, rnb, rta, rtb, massn, masst, target, corr);
-                            an = w2[2 * mi]; at = w2[2 * mi + 1];
-                        }
-                        const int f = R_M0 + mi * M_WORDS;
-                        ovl(f + M_RNA) = rna; ovl(f + M_RNB) = rnb; ovl(f + M_RTA) = rta; ovl(f + M_RTB) = rtb;
-                        ovl(f + M_MASSN) = massn; ovl(f + M_MASST) = masst; ovl(f + M_TARGET) = target; ovl(f + M_CORR) = corr;
-                        ovl(f + M_ACCN) = an; ovl(f + M_ACCT) = at;
-                    }
-                    clevel2 = (int)((ab2 >> 19) & 127u);
-                }
+                const unsigned r2 = second_build<SC, G>(sm, nrec, cc);     // level | active manifolds << 8
+                clevel2 = (int)(r2 & 127u);
                 clevel = (int)((ab >> 19) & 127u);
                 cmax = g.shfl(cmax, 0);
-                c_man += (unsigned)(__popc(g.ballot((ab2 >> 10) & 1u)) + __popc(g.ballot((ab2 >> 11) & 1u)));
+                c_man += (unsigned)g.sum_int((int)(r2 >> 8));
             } else {
                 // levels of the records (canonical order = record order): one more than the highest level of an
                 // earlier record that shares a movable body
@@ -1258,24 +1319,8 @@ struct Scene {
         }
         c_man += 1u << 16;
         g.sync();
-        if (done && prm.auto_reset != 0) {
-            const int episode = (int)smu[SC::META + META_EPISODE] + 1;
-            int level = (int)smu[SC::META + META_LEVEL];
-            g.sync();
-            if (prm.auto_reset == 2) {
-                const unsigned long long h = mix64(prm.seed + ((unsigned long long)(prm.env_offset + e) + 1ULL) * 0x9E3779B97F4A7C15ULL +
-                                                   (unsigned long long)episode * 0xD1B54A32D192ED03ULL);
-                const int nl = (int)(h % (unsigned long long)prm.n_levels);
-                if (nl != level) { level = nl; load_level_consts(prm.levels + (size_t)nl * SC::LV_WORDS); }
-            }
-            load_level_pose(prm.levels + (size_t)level * SC::LV_WORDS);
-            if (lane == 0) {
-                smu[SC::META + META_STEP] = 0u; smu[SC::META + META_EPISODE] = (uint32_t)episode; smu[SC::META + META_LEVEL] = (uint32_t)level;
-                smu[SC::META + META_STATUS] = 0u; smu[SC::META + META_NWARM] = 0u;
-                atomicAdd(prm.counters + 1, 1ULL);
-            }
-            g.sync();
-        }
+        if (done && prm.auto_reset != 0)
+            jab = reset_env<SC, G>(smu, prm.levels, prm.n_levels, prm.auto_reset, prm.seed, prm.env_offset + e, prm.counters, jab);
     }
 
     // ---- whole launch for one scene
@@ -1292,7 +1337,7 @@ struct Scene {
         for (int i = lane; i < (SC::NPAIRS + 3) / 4; i += G) smu[SC::WIDX + i] = 0xffffffffu;
         const int level = (int)__ldcg(st + SC::ST_META + META_LEVEL);
         const int nwarm = (int)__ldcg(st + SC::ST_META + META_NWARM);
-        load_level_consts(prm.levels + (size_t)level * SC::LV_WORDS);
+        jab = load_level_consts<SC, G>(smu, prm.levels + (size_t)level * SC::LV_WORDS);
         g.sync();
         // accumulated impulses of the previous launch: entry k goes to lane k
         rec.ab = 0u; rec.accn = 0.0f; rec.acct = 0.0f;
@@ -1319,7 +1364,7 @@ struct Scene {
         for (int s = s0; s < s1; ++s) {
             step(e, s);
             g.sync();
-            if (((s - s0) & 255) == 255) flush_counters();
+            if (((s - s0) & 255) == 255) flush();
         }
         // write back
         for (int i = lane; i < 6 * SC::N; i += G) st[SC::ST_BODY + i] = smu[SC::BX + i];
@@ -1342,7 +1387,7 @@ struct Scene {
             wr[3] = __float_as_uint(ovl(OV_ACC1N)); wr[4] = __float_as_uint(ovl(OV_ACC1T));
         }
         if (nw > G + G / 2) warm_out<SC, G>(ovf, st + SC::ST_WARM, nw);
-        flush_counters();
+        flush();
         g.sync();
     }
 };
