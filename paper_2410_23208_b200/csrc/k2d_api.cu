@@ -269,6 +269,17 @@ static cudaError_t setup_step(k2d_state *s, int num_sms) {
     return cudaSuccess;
 }
 
+template <class SC>
+static cudaError_t launch_obs(const k2d_state *s, float *dev_obs) {
+    const k2d_config &c = s->cfg;
+    const int wpb = kObsThreads / 32, grid = (c.n_envs + wpb - 1) / wpb;
+    const int width = (c.n_polygons + c.n_circles) * 29 + c.n_joints * 2 * (11 + c.n_actions) + c.n_thrusters * 6;
+    const size_t smem = sizeof(float) * wpb * ((width + 2 * SC::N + 3) / 4 * 4);
+    k2d_obs_kernel<SC><<<grid, kObsThreads, smem, s->stream>>>(s->dev_env, s->dev_levels, dev_obs, c.n_envs, c.n_actions, c.n_polygons,
+                                                              c.n_circles, c.n_joints, c.n_thrusters);
+    return cudaGetLastError();
+}
+
 // Kernel arguments of one k2d_step launch.  With more envs than resident scene groups the launch is cut
 // into chunks of kChunkSteps steps, so that the groups can balance the work between them.
 static StepParams step_params(const k2d_state *s, const float *dev_actions, int n_steps, float *dev_reward, uint8_t *dev_done,
@@ -420,12 +431,7 @@ int k2d_step(k2d_state *s, const float *dev_actions, int32_t n_steps, float *dev
 int k2d_obs(k2d_state *s, float *dev_obs) {
     if (!s || !dev_obs) return K2D_ERR_NULL;
     if ((uintptr_t)dev_obs & 3) return K2D_ERR_ALIGN;
-    const k2d_config &c = s->cfg;
-    const int wpb = kBlockThreads / 32, grid = (c.n_envs + wpb - 1) / wpb;
-    if (s->ci.id == 0) k2d_obs_kernel<ClassS><<<grid, kBlockThreads, 0, s->stream>>>(s->dev_env, s->dev_levels, dev_obs, c.n_envs, c.n_actions, c.n_polygons, c.n_circles, c.n_joints, c.n_thrusters);
-    else if (s->ci.id == 1) k2d_obs_kernel<ClassM><<<grid, kBlockThreads, 0, s->stream>>>(s->dev_env, s->dev_levels, dev_obs, c.n_envs, c.n_actions, c.n_polygons, c.n_circles, c.n_joints, c.n_thrusters);
-    else k2d_obs_kernel<ClassL><<<grid, kBlockThreads, 0, s->stream>>>(s->dev_env, s->dev_levels, dev_obs, c.n_envs, c.n_actions, c.n_polygons, c.n_circles, c.n_joints, c.n_thrusters);
-    CUDA_OK(cudaGetLastError());
+    CUDA_OK(s->ci.id == 0 ? launch_obs<ClassS>(s, dev_obs) : s->ci.id == 1 ? launch_obs<ClassM>(s, dev_obs) : launch_obs<ClassL>(s, dev_obs));
     return K2D_OK;
 }
 

@@ -25,6 +25,7 @@ constexpr int kBlockThreads = 128;
 #define K2D_MIN_BLOCKS 5
 #endif
 constexpr int kMinBlocks = K2D_MIN_BLOCKS;   // resident blocks per SM the step kernel is compiled for (bounds its registers)
+constexpr int kObsThreads = 128;   // observation kernel: one warp per env, four envs per block
 constexpr int kMaxActions = 16;
 enum { Q_TICKET = 0, Q_LEFT = 1, Q_ERROR = 2 };
 constexpr unsigned kWaitLimit = 1u << 24;   // polls (about 100 ns apart) before a wait for another group's chunk gives up
@@ -1478,92 +1479,99 @@ __global__ void k2d_reset_kernel(uint32_t *state, const uint32_t *levels, const 
 }
 
 // ---------------------------------------------------------------- observation kernel: one warp per env
+// Each lane writes whole entity rows (a shape, one side of a joint, a thruster) into the warp's
+// shared-memory image of the observation, then the warp copies the image out with coalesced stores.
 template <class SC>
-__global__ void __launch_bounds__(kBlockThreads) k2d_obs_kernel(const uint32_t *state, const uint32_t *levels, float *obs,
-                                                                int n_envs, int n_actions, int n_polygons, int n_circles,
-                                                                int n_joints, int n_thrusters) {
-    __shared__ float cs[kBlockThreads / 32][2 * SC::N];
+__global__ void __launch_bounds__(kObsThreads) k2d_obs_kernel(const uint32_t *state, const uint32_t *levels, float *obs,
+                                                              int n_envs, int n_actions, int n_polygons, int n_circles,
+                                                              int n_joints, int n_thrusters) {
+    extern __shared__ __align__(16) float obs_smem[];
     const int w = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int e = blockIdx.x * (kBlockThreads / 32) + w;
+    const int e = blockIdx.x * (kObsThreads / 32) + w;
     if (e >= n_envs) return;
+    const int n_shapes = n_polygons + n_circles;
+    const int jw = 11 + n_actions;
+    const int width = n_shapes * 29 + 2 * n_joints * jw + 6 * n_thrusters;
+    float *img = obs_smem + (size_t)w * ((width + 2 * SC::N + 3) / 4 * 4);
+    float *cs = img + width;                 // cos, sin of every shape's angle
     const uint32_t *st = state + (size_t)e * SC::ST_WORDS;
     const uint32_t *lv = levels + (size_t)st[SC::ST_META + 2] * SC::LV_WORDS;
     const float *stf = reinterpret_cast<const float *>(st);
     const float *lvf = reinterpret_cast<const float *>(lv);
-    for (int i = lane; i < SC::N; i += 32) {
-        float c, s;
-        sincos_spec(stf[2 * SC::N + i], c, s);
-        cs[w][i] = c; cs[w][SC::N + i] = s;
+    for (int ci = lane; ci < n_shapes; ci += 32) {
+        const int i = ci < n_polygons ? ci : SC::P + (ci - n_polygons);     // internal shape index
+        float c, sn;
+        sincos_spec(stf[2 * SC::N + i], c, sn);
+        cs[i] = c; cs[SC::N + i] = sn;
+        float *o = img + ci * 29;
+        const uint32_t fl = lv[SC::LV_FLAGS + i];
+        if (!(fl & F_ACTIVE)) {
+            for (int f = 0; f < 29; ++f) o[f] = 0.0f;
+            continue;
+        }
+        const int nv = flag_nverts(fl);
+        const uint32_t role = flag_role(fl);
+        const bool poly = i < SC::P;
+        o[0] = stf[i]; o[1] = stf[SC::N + i]; o[2] = stf[3 * SC::N + i]; o[3] = stf[4 * SC::N + i];
+        o[4] = lvf[SC::LV_IM + i]; o[5] = lvf[SC::LV_II + i]; o[6] = lvf[SC::LV_DENS + i];
+        o[7] = tanh_spec(stf[5 * SC::N + i] * 0.1f);
+#pragma unroll
+        for (int r = 0; r < 4; ++r) o[8 + r] = (role == (uint32_t)r) ? 1.0f : 0.0f;
+        o[12] = sn; o[13] = c; o[14] = lvf[SC::LV_FR + i]; o[15] = lvf[SC::LV_RE + i];
+        o[16] = poly ? 1.0f : 0.0f; o[17] = poly ? 0.0f : 1.0f;
+        o[18] = poly ? 0.0f : lvf[SC::LV_RAD + (poly ? 0 : i - SC::P)];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const bool on = poly && k < nv;
+            o[19 + 2 * k] = on ? lvf[SC::LV_PVX + 4 * (poly ? i : 0) + k] : 0.0f;
+            o[20 + 2 * k] = on ? lvf[SC::LV_PVY + 4 * (poly ? i : 0) + k] : 0.0f;
+        }
+        o[27] = (poly && nv == 3) ? 1.0f : 0.0f;
+        o[28] = (poly && nv != 3) ? 1.0f : 0.0f;
     }
     __syncwarp();
-    const int n_shapes = n_polygons + n_circles;
-    const int jw = 11 + n_actions;
-    const int width = n_shapes * 29 + 2 * n_joints * jw + 6 * n_thrusters;
-    float *o = obs + (size_t)e * width;
-    for (int idx = lane; idx < width; idx += 32) {
-        float v = 0.0f;
-        if (idx < n_shapes * 29) {
-            const int ci = idx / 29, f = idx - ci * 29;
-            const int i = ci < n_polygons ? ci : SC::P + (ci - n_polygons);     // internal shape index
-            const uint32_t fl = lv[SC::LV_FLAGS + i];
-            if (fl & F_ACTIVE) {
-                const int nv = flag_nverts(fl);
-                if (f == 0) v = stf[i];
-                else if (f == 1) v = stf[SC::N + i];
-                else if (f == 2) v = stf[3 * SC::N + i];
-                else if (f == 3) v = stf[4 * SC::N + i];
-                else if (f == 4) v = lvf[SC::LV_IM + i];
-                else if (f == 5) v = lvf[SC::LV_II + i];
-                else if (f == 6) v = lvf[SC::LV_DENS + i];
-                else if (f == 7) v = tanh_spec(stf[5 * SC::N + i] * 0.1f);
-                else if (f < 12) v = (flag_role(fl) == (uint32_t)(f - 8)) ? 1.0f : 0.0f;
-                else if (f == 12) v = cs[w][SC::N + i];
-                else if (f == 13) v = cs[w][i];
-                else if (f == 14) v = lvf[SC::LV_FR + i];
-                else if (f == 15) v = lvf[SC::LV_RE + i];
-                else if (f == 16) v = i < SC::P ? 1.0f : 0.0f;
-                else if (f == 17) v = i < SC::P ? 0.0f : 1.0f;
-                else if (f == 18) v = i < SC::P ? 0.0f : lvf[SC::LV_RAD + (i - SC::P)];
-                else if (f < 27) {
-                    const int q = f - 19, k = q >> 1;
-                    if (i < SC::P && k < nv) v = (q & 1) ? lvf[SC::LV_PVY + 4 * i + k] : lvf[SC::LV_PVX + 4 * i + k];
-                } else if (i < SC::P) v = ((f == 27) == (nv == 3)) ? 1.0f : 0.0f;
-            }
-        } else if (idx < n_shapes * 29 + 2 * n_joints * jw) {
-            const int q = idx - n_shapes * 29;
-            const int row = q / jw, f = q - row * jw;
-            const int j = row >> 1, d = row & 1;
-            const uint32_t *jl = lv + SC::LV_JOINT + 8 * j;
-            const uint32_t jab = jl[0];
-            if ((jab >> 28) & 1u) {
-                const int a = jab & 255, b = (jab >> 8) & 255;
-                const int from = d ? b : a, to = d ? a : b;
-                if (f == 0) v = 1.0f;
-                else if (f >= 2 && f < 6) { const int side = ((f - 2) >> 1) ^ d; v = __uint_as_float(jl[1 + 2 * side + ((f - 2) & 1)]); }
-                else if (f == 6) v = __uint_as_float(jl[6]);
-                else if (f == 7) v = __uint_as_float(jl[5]);
-                else if (f >= 9 && f < 9 + n_actions) v = ((int)((jab >> 16) & 255) == f - 9) ? 1.0f : 0.0f;
-                else if (f == 9 + n_actions) v = __fmaf_rn(cs[w][SC::N + to], cs[w][from], -(cs[w][to] * cs[w][SC::N + from]));
-                else if (f == 10 + n_actions) v = __fmaf_rn(cs[w][to], cs[w][from], cs[w][SC::N + to] * cs[w][SC::N + from]);
-            }
-        } else {
-            const int q = idx - n_shapes * 29 - 2 * n_joints * jw;
-            const int t = q / 6, f = q - t * 6;
-            const uint32_t *th = lv + SC::LV_THR + 8 * t;
-            const uint32_t tp = th[0];
-            if ((tp >> 20) & 1u) {
-                const int i = tp & 255;
-                float dx, dy;
-                rot2(cs[w][i], cs[w][SC::N + i], __uint_as_float(th[3]), __uint_as_float(th[4]), dx, dy);
-                if (f == 0) v = 1.0f;
-                else if (f == 1) v = __uint_as_float(th[1]);
-                else if (f == 2) v = __uint_as_float(th[2]);
-                else if (f == 3) v = __uint_as_float(th[5]);
-                else if (f == 4) v = dy;
-                else v = dx;
-            }
+    float *jrows = img + n_shapes * 29;
+    for (int row = lane; row < 2 * n_joints; row += 32) {
+        const int j = row >> 1, d = row & 1;
+        const uint32_t *jl = lv + SC::LV_JOINT + 8 * j;
+        const uint32_t jab = jl[0];
+        float *o = jrows + row * jw;
+        for (int f = 0; f < jw; ++f) o[f] = 0.0f;
+        if ((jab >> 28) & 1u) {
+            const int a = jab & 255, b = (jab >> 8) & 255;
+            const int from = d ? b : a, to = d ? a : b;
+            o[0] = 1.0f;
+#pragma unroll
+            for (int f = 2; f < 6; ++f) { const int side = ((f - 2) >> 1) ^ d; o[f] = __uint_as_float(jl[1 + 2 * side + ((f - 2) & 1)]); }
+            o[6] = __uint_as_float(jl[6]); o[7] = __uint_as_float(jl[5]);
+            const int bind = (int)((jab >> 16) & 255);
+            if (bind < n_actions) o[9 + bind] = 1.0f;
+            o[9 + n_actions] = __fmaf_rn(cs[SC::N + to], cs[from], -(cs[to] * cs[SC::N + from]));
+            o[10 + n_actions] = __fmaf_rn(cs[to], cs[from], cs[SC::N + to] * cs[SC::N + from]);
         }
-        o[idx] = v;
+    }
+    float *trows = jrows + 2 * n_joints * jw;
+    for (int t = lane; t < n_thrusters; t += 32) {
+        const uint32_t *th = lv + SC::LV_THR + 8 * t;
+        const uint32_t tp = th[0];
+        float *o = trows + t * 6;
+        for (int f = 0; f < 6; ++f) o[f] = 0.0f;
+        if ((tp >> 20) & 1u) {
+            const int i = tp & 255;
+            float dx, dy;
+            rot2(cs[i], cs[SC::N + i], __uint_as_float(th[3]), __uint_as_float(th[4]), dx, dy);
+            o[0] = 1.0f; o[1] = __uint_as_float(th[1]); o[2] = __uint_as_float(th[2]); o[3] = __uint_as_float(th[5]);
+            o[4] = dy; o[5] = dx;
+        }
+    }
+    __syncwarp();
+    float *out = obs + (size_t)e * width;
+    if (((width & 3) == 0) && ((reinterpret_cast<uintptr_t>(obs) & 15) == 0)) {
+        const float4 *src = reinterpret_cast<const float4 *>(img);
+        float4 *dst = reinterpret_cast<float4 *>(out);
+        for (int q = lane; q < width / 4; q += 32) dst[q] = src[q];
+    } else {
+        for (int q = lane; q < width; q += 32) out[q] = img[q];
     }
 }
 
