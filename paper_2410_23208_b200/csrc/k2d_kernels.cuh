@@ -32,7 +32,7 @@ constexpr unsigned kWaitLimit = 1u << 24;   // polls (about 100 ns apart) before
 constexpr int kRecWords = 24;   // contact pair record
 constexpr int kWarmWords = 5;   // pair index + 4 accumulated impulses
 constexpr int kStageWords = 9;  // packed pair word, normal, two contact points with penetration
-constexpr int kJointWords = 13; // joint row kept in shared memory
+constexpr int kJointWords = 20; // joint row kept in shared memory: five 16-byte groups
 
 // ---------------------------------------------------------------- size classes and layouts
 template <int P_, int C_, int J_, int T_>
@@ -59,15 +59,16 @@ struct SizeClass {
     static constexpr int SCRATCH_WORDS = NPAIRS * (kRecWords + kWarmWords);
     static constexpr int SCRATCH_WARM = NPAIRS * kRecWords;
     // shared memory region of one scene (words)
-    static constexpr int BX = 0, BY = N, BTH = 2 * N, BVX = 3 * N, BVY = 4 * N, BW = 5 * N;
-    static constexpr int BIM = 6 * N, BII = 7 * N, BFR = 8 * N, BRE = 9 * N, BC = 10 * N, BS = 11 * N, BFL = 12 * N;
-    static constexpr int RAD = 13 * N;
+    // per body 16-byte groups (x, y, angle, -) and (vx, vy, angular velocity, -), then per-body arrays
+    static constexpr int BPOS = 0, BVEL = 4 * N;
+    static constexpr int BIM = 8 * N, BII = 9 * N, BFR = 10 * N, BRE = 11 * N, BC = 12 * N, BS = 13 * N, BFL = 14 * N;
+    static constexpr int RAD = 15 * N;
     static constexpr int WVX = RAD + C, WVY = WVX + P4, WNX = WVY + P4, WNY = WNX + P4, WOFF = WNY + P4;
     static constexpr int BOX = (WOFF + P4 + 3) / 4 * 4;  // N x (min x, min y, max x, max y), 16-byte aligned
     static constexpr int MASK = BOX + 4 * N;
     static constexpr int ACT = MASK + MASKW;
     static constexpr int META = ACT + kMaxActions;       // step_count, episode_count, level_id, status, warm entries
-    static constexpr int JROW = META + 8;                // kJointWords x J, field-major
+    static constexpr int JROW = (META + 8 + 3) / 4 * 4;  // J rows of kJointWords, 16-byte aligned
     static constexpr int SURV = JROW + kJointWords * J;  // bytes: pairs that passed the box test
     static constexpr int WIDX = SURV + (NPAIRS + 3) / 4; // bytes: pair -> record index of the previous step
     // then, per lane of the group (field-major, G words per field):
@@ -96,10 +97,17 @@ enum { LF_ACC2N = kStageWords, LF_ACC2T, LF_COUNT };
 __host__ __device__ constexpr int ovs(int f) { return f < 3 ? f : f + 1; }
 constexpr int OV_ACC0N = R_M0 + M_ACCN, OV_ACC0T = R_M0 + M_ACCT, OV_ACC1N = R_M0 + M_WORDS + M_ACCN, OV_ACC1T = R_M0 + M_WORDS + M_ACCT;
 // joint row fields
-enum { JR_RAX = 0, JR_RAY, JR_RBX, JR_RBY, JR_I11, JR_I12, JR_I22, JR_BX, JR_BY, JR_CX, JR_CY, JR_ACCX, JR_ACCY };
-static_assert(JR_ACCY + 1 == kJointWords, "joint row size");
+enum { JR_RAX = 0, JR_RAY, JR_RBX, JR_RBY, JR_I11, JR_I12, JR_I22, JR_PAD0, JR_BX, JR_BY, JR_CX, JR_CY, JR_MA, JR_MB, JR_IA, JR_IB,
+       JR_ACCX, JR_ACCY, JR_PAD1, JR_PAD2 };
+static_assert(JR_PAD2 + 1 == kJointWords, "joint row size");
 enum { META_STEP = 0, META_EPISODE, META_LEVEL, META_STATUS, META_NWARM };
 
+// shared-memory word of word i of a state record's body block (x[N], y[N], angle[N], vx[N], vy[N], w[N])
+template <class SC>
+__device__ __forceinline__ int body_word(int i) {
+    const int f = i / SC::N, b = i - f * SC::N;
+    return (f < 3 ? SC::BPOS + f : SC::BVEL + f - 3) + 4 * b;
+}
 // shared-memory words per scene: padded so that the groups of one warp start in different banks
 template <class SC, int G>
 __host__ __device__ constexpr int region_words() {
@@ -143,6 +151,8 @@ __device__ __forceinline__ void rot2(float c, float s, float vx, float vy, float
     ox = __fmaf_rn(c, vx, -(s * vy));
     oy = __fmaf_rn(s, vx, c * vy);
 }
+__device__ __forceinline__ float4 ld4(const float *p) { return *reinterpret_cast<const float4 *>(p); }
+__device__ __forceinline__ void st4(float *p, float a, float b, float c) { *reinterpret_cast<float4 *>(p) = make_float4(a, b, c, 0.0f); }
 __device__ __forceinline__ bool finite_bits(float v) { return (__float_as_uint(v) & 0x7f800000u) != 0x7f800000u; }
 
 // Sine and cosine: reduction by multiples of pi/2 with a three-part constant and FMA, then the
@@ -253,17 +263,19 @@ __device__ __forceinline__ void prestep_manifold(int a, int b, float nx, float n
                                                  float px, float py, float pen, float er, const float *sm, const ContactConsts &cc,
                                                  float &rna, float &rnb, float &rta, float &rtb, float &massn, float &masst,
                                                  float &target, float &corr) {
-    const float rax = px - sm[SC::BX + a], ray = py - sm[SC::BY + a];
-    const float rbx = px - sm[SC::BX + b], rby = py - sm[SC::BY + b];
+    const float4 pa4 = ld4(sm + SC::BPOS + 4 * a), pb4 = ld4(sm + SC::BPOS + 4 * b);
+    const float4 va4 = ld4(sm + SC::BVEL + 4 * a), vb4 = ld4(sm + SC::BVEL + 4 * b);
+    const float rax = px - pa4.x, ray = py - pa4.y;
+    const float rbx = px - pb4.x, rby = py - pb4.y;
     const float tx = -ny, ty = nx;
     rna = cross2(rax, ray, nx, ny); rnb = cross2(rbx, rby, nx, ny);
     rta = cross2(rax, ray, tx, ty); rtb = cross2(rbx, rby, tx, ty);
     float kn = ma + mb; kn = __fmaf_rn(ia * rna, rna, kn); kn = __fmaf_rn(ib * rnb, rnb, kn);
     float kt = ma + mb; kt = __fmaf_rn(ia * rta, rta, kt); kt = __fmaf_rn(ib * rtb, rtb, kt);
     // normal approach speed before warm starting
-    float vn0 = dot2(nx, ny, sm[SC::BVX + b] - sm[SC::BVX + a], sm[SC::BVY + b] - sm[SC::BVY + a]);
-    vn0 = __fmaf_rn(sm[SC::BW + b], rnb, vn0);
-    vn0 = __fmaf_rn(-sm[SC::BW + a], rna, vn0);
+    float vn0 = dot2(nx, ny, vb4.x - va4.x, vb4.y - va4.y);
+    vn0 = __fmaf_rn(vb4.z, rnb, vn0);
+    vn0 = __fmaf_rn(-va4.z, rna, vn0);
     const float depth = fmax_cmp(pen - cc.slop, 0.0f);
     const float bounce = (vn0 < -cc.rest_thr) ? (-er * vn0) : 0.0f;
     massn = 1.0f / kn; masst = 1.0f / kt;
@@ -313,9 +325,9 @@ __device__ __forceinline__ void manifold_rows(float nx, float ny, float mu, floa
 }
 
 // positional correction of one pair: each active manifold moves the two bodies apart along the normal
-__device__ __forceinline__ void correct_pair(float *bx, float *by, int a, int b, unsigned amask, bool dyn_a, bool dyn_b,
+__device__ __forceinline__ void correct_pair(float *pos, int a, int b, unsigned amask, bool dyn_a, bool dyn_b,
                                              float nx, float ny, float ma, float mb, float corr0, float corr1) {
-    float xa = bx[a], ya = by[a], xb = bx[b], yb = by[b];
+    float xa = pos[4 * a], ya = pos[4 * a + 1], xb = pos[4 * b], yb = pos[4 * b + 1];
     if (amask & 1u) {
         const float ca = ma * corr0, cb = mb * corr0;
         xa = __fmaf_rn(-ca, nx, xa); ya = __fmaf_rn(-ca, ny, ya);
@@ -326,8 +338,8 @@ __device__ __forceinline__ void correct_pair(float *bx, float *by, int a, int b,
         xa = __fmaf_rn(-ca, nx, xa); ya = __fmaf_rn(-ca, ny, ya);
         xb = __fmaf_rn(cb, nx, xb); yb = __fmaf_rn(cb, ny, yb);
     }
-    if (dyn_a) { bx[a] = xa; by[a] = ya; }
-    if (dyn_b) { bx[b] = xb; by[b] = yb; }
+    if (dyn_a) { pos[4 * a] = xa; pos[4 * a + 1] = ya; }
+    if (dyn_b) { pos[4 * b] = xb; pos[4 * b + 1] = yb; }
 }
 
 // ---- joints; the row of joint j is in shared memory.  MODE 0: warm start, 1: solver iteration,
@@ -336,48 +348,44 @@ template <class SC, int MODE>
 __device__ __forceinline__ void visit_joint(float *sm, uint32_t jab, int j, const uint32_t *lv, float motor_rho) {
     const int a = jab & 255, b = (jab >> 8) & 255;
     const bool dyn_a = (jab >> 29) & 1u, dyn_b = (jab >> 30) & 1u;
-    float *jr = sm + SC::JROW + j;
+    float *jr = sm + SC::JROW + kJointWords * j;
     if (MODE == 3) {
         const float A = fmax_cmp(fmin_cmp(sm[SC::ACT + ((jab >> 16) & 255)], 1.0f), -1.0f);
         const float speed = __uint_as_float(lv[SC::LV_JOINT + 8 * j + 5]), power = __uint_as_float(lv[SC::LV_JOINT + 8 * j + 6]);
-        const float wa = sm[SC::BW + a], wb = sm[SC::BW + b];
+        const float wa = sm[SC::BVEL + 4 * a + 2], wb = sm[SC::BVEL + 4 * b + 2];
         const float arg = __fmaf_rn(-speed, A, wa - wb) * motor_rho;
         const float jr_ = power * tanh_spec(arg);
-        if (dyn_a) sm[SC::BW + a] = __fmaf_rn(-jr_, sm[SC::BII + a], wa);
-        if (dyn_b) sm[SC::BW + b] = __fmaf_rn(jr_, sm[SC::BII + b], wb);
+        if (dyn_a) sm[SC::BVEL + 4 * a + 2] = __fmaf_rn(-jr_, sm[SC::BII + a], wa);
+        if (dyn_b) sm[SC::BVEL + 4 * b + 2] = __fmaf_rn(jr_, sm[SC::BII + b], wb);
         return;
     }
-    const float ma = sm[SC::BIM + a], mb = sm[SC::BIM + b];
+    const float4 mi4 = ld4(jr + JR_MA);       // inverse masses and inertias of the two bodies
+    const float ma = mi4.x, mb = mi4.y, ia = mi4.z, ib = mi4.w;
     if (MODE == 2) {
-        const float cx = jr[JR_CX * SC::J], cy = jr[JR_CY * SC::J];
-        if (dyn_a) { sm[SC::BX + a] = __fmaf_rn(ma, cx, sm[SC::BX + a]); sm[SC::BY + a] = __fmaf_rn(ma, cy, sm[SC::BY + a]); }
-        if (dyn_b) { sm[SC::BX + b] = __fmaf_rn(-mb, cx, sm[SC::BX + b]); sm[SC::BY + b] = __fmaf_rn(-mb, cy, sm[SC::BY + b]); }
+        const float cx = jr[JR_CX], cy = jr[JR_CY];
+        if (dyn_a) { sm[SC::BPOS + 4 * a] = __fmaf_rn(ma, cx, sm[SC::BPOS + 4 * a]); sm[SC::BPOS + 4 * a + 1] = __fmaf_rn(ma, cy, sm[SC::BPOS + 4 * a + 1]); }
+        if (dyn_b) { sm[SC::BPOS + 4 * b] = __fmaf_rn(-mb, cx, sm[SC::BPOS + 4 * b]); sm[SC::BPOS + 4 * b + 1] = __fmaf_rn(-mb, cy, sm[SC::BPOS + 4 * b + 1]); }
         return;
     }
-    const float ia = sm[SC::BII + a], ib = sm[SC::BII + b];
-    const float rax = jr[JR_RAX * SC::J], ray = jr[JR_RAY * SC::J], rbx = jr[JR_RBX * SC::J], rby = jr[JR_RBY * SC::J];
-    float vax = sm[SC::BVX + a], vay = sm[SC::BVY + a], wa = sm[SC::BW + a];
-    float vbx = sm[SC::BVX + b], vby = sm[SC::BVY + b], wb = sm[SC::BW + b];
+    const float4 r4 = ld4(jr + JR_RAX);
+    const float rax = r4.x, ray = r4.y, rbx = r4.z, rby = r4.w;
+    const float4 va4 = ld4(sm + SC::BVEL + 4 * a), vb4 = ld4(sm + SC::BVEL + 4 * b);
+    float vax = va4.x, vay = va4.y, wa = va4.z, vbx = vb4.x, vby = vb4.y, wb = vb4.z;
     float lx, ly;
-    if (MODE == 0) { lx = jr[JR_ACCX * SC::J]; ly = jr[JR_ACCY * SC::J]; }
+    if (MODE == 0) { lx = jr[JR_ACCX]; ly = jr[JR_ACCY]; }
     else {
+        const float4 k4 = ld4(jr + JR_I11), b4 = ld4(jr + JR_BX);
+        const float2 acc = *reinterpret_cast<const float2 *>(jr + JR_ACCX);
         const float cx = __fmaf_rn(-wb, rby, vbx) - __fmaf_rn(-wa, ray, vax);
         const float cy = __fmaf_rn(wb, rbx, vby) - __fmaf_rn(wa, rax, vay);
-        const float rx = -(cx + jr[JR_BX * SC::J]), ry = -(cy + jr[JR_BY * SC::J]);
-        const float i11 = jr[JR_I11 * SC::J], i12 = jr[JR_I12 * SC::J], i22 = jr[JR_I22 * SC::J];
+        const float rx = -(cx + b4.x), ry = -(cy + b4.y);
+        const float i11 = k4.x, i12 = k4.y, i22 = k4.z;
         lx = __fmaf_rn(i11, rx, i12 * ry);
         ly = __fmaf_rn(i12, rx, i22 * ry);
-        jr[JR_ACCX * SC::J] = jr[JR_ACCX * SC::J] + lx;
-        jr[JR_ACCY * SC::J] = jr[JR_ACCY * SC::J] + ly;
+        *reinterpret_cast<float2 *>(jr + JR_ACCX) = make_float2(acc.x + lx, acc.y + ly);
     }
-    if (dyn_a) {
-        sm[SC::BVX + a] = __fmaf_rn(-ma, lx, vax); sm[SC::BVY + a] = __fmaf_rn(-ma, ly, vay);
-        sm[SC::BW + a] = __fmaf_rn(-ia, cross2(rax, ray, lx, ly), wa);
-    }
-    if (dyn_b) {
-        sm[SC::BVX + b] = __fmaf_rn(mb, lx, vbx); sm[SC::BVY + b] = __fmaf_rn(mb, ly, vby);
-        sm[SC::BW + b] = __fmaf_rn(ib, cross2(rbx, rby, lx, ly), wb);
-    }
+    if (dyn_a) st4(sm + SC::BVEL + 4 * a, __fmaf_rn(-ma, lx, vax), __fmaf_rn(-ma, ly, vay), __fmaf_rn(-ia, cross2(rax, ray, lx, ly), wa));
+    if (dyn_b) st4(sm + SC::BVEL + 4 * b, __fmaf_rn(mb, lx, vbx), __fmaf_rn(mb, ly, vby), __fmaf_rn(ib, cross2(rbx, rby, lx, ly), wb));
 }
 // joints of one level touch disjoint movable bodies; levels in order keep the joint order
 template <class SC, int G, int MODE>
@@ -482,10 +490,10 @@ __device__ __forceinline__ void slow_sweep_pairs(float *sm, uint32_t *ovf, int n
             const unsigned amask = (c.ab >> 10) & 3u;
             const bool dyn_a = (c.ab >> 26) & 1u, dyn_b = (c.ab >> 27) & 1u;
             const float ma = sm[SC::BIM + a], mb = sm[SC::BIM + b];
-            if (MODE == 2) { correct_pair(sm + SC::BX, sm + SC::BY, a, b, amask, dyn_a, dyn_b, c.nx, c.ny, ma, mb, c.corr[0], c.corr[1]); continue; }
+            if (MODE == 2) { correct_pair(sm + SC::BPOS, a, b, amask, dyn_a, dyn_b, c.nx, c.ny, ma, mb, c.corr[0], c.corr[1]); continue; }
             const float ia = sm[SC::BII + a], ib = sm[SC::BII + b];
-            float vax = sm[SC::BVX + a], vay = sm[SC::BVY + a], wa = sm[SC::BW + a];
-            float vbx = sm[SC::BVX + b], vby = sm[SC::BVY + b], wb = sm[SC::BW + b];
+            const float4 va4 = ld4(sm + SC::BVEL + 4 * a), vb4 = ld4(sm + SC::BVEL + 4 * b);
+            float vax = va4.x, vay = va4.y, wa = va4.z, vbx = vb4.x, vby = vb4.y, wb = vb4.z;
 #pragma unroll
             for (int mi = 0; mi < 2; ++mi) {
                 if (amask & (1u << mi)) {
@@ -497,8 +505,8 @@ __device__ __forceinline__ void slow_sweep_pairs(float *sm, uint32_t *ovf, int n
                     }
                 }
             }
-            if (dyn_a) { sm[SC::BVX + a] = vax; sm[SC::BVY + a] = vay; sm[SC::BW + a] = wa; }
-            if (dyn_b) { sm[SC::BVX + b] = vbx; sm[SC::BVY + b] = vby; sm[SC::BW + b] = wb; }
+            if (dyn_a) st4(sm + SC::BVEL + 4 * a, vax, vay, wa);
+            if (dyn_b) st4(sm + SC::BVEL + 4 * b, vbx, vby, wb);
         }
         g.sync();
     }
@@ -641,12 +649,12 @@ __device__ __noinline__ void visit_second(float *sm) {
     const float nx = ov[R_NX * H], ny = ov[R_NY * H];
     const float ma = sm[SC::BIM + a], mb = sm[SC::BIM + b];
     if (MODE == 2) {
-        correct_pair(sm + SC::BX, sm + SC::BY, a, b, amask, dyn_a, dyn_b, nx, ny, ma, mb, ov[(R_M0 + M_CORR) * H], ov[(R_M0 + M_WORDS + M_CORR) * H]);
+        correct_pair(sm + SC::BPOS, a, b, amask, dyn_a, dyn_b, nx, ny, ma, mb, ov[(R_M0 + M_CORR) * H], ov[(R_M0 + M_WORDS + M_CORR) * H]);
         return;
     }
     const float ia = sm[SC::BII + a], ib = sm[SC::BII + b], mu = ov[R_MU * H];
-    float vax = sm[SC::BVX + a], vay = sm[SC::BVY + a], wa = sm[SC::BW + a];
-    float vbx = sm[SC::BVX + b], vby = sm[SC::BVY + b], wb = sm[SC::BW + b];
+    const float4 va4 = ld4(sm + SC::BVEL + 4 * a), vb4 = ld4(sm + SC::BVEL + 4 * b);
+    float vax = va4.x, vay = va4.y, wa = va4.z, vbx = vb4.x, vby = vb4.y, wb = vb4.z;
 #pragma unroll 1
     for (int mi = 0; mi < 2; ++mi) {
         if (amask & (1u << mi)) {
@@ -657,8 +665,8 @@ __device__ __noinline__ void visit_second(float *sm) {
             if (MODE == 1) { m[M_ACCN * H] = accn; m[M_ACCT * H] = acct; }
         }
     }
-    if (dyn_a) { sm[SC::BVX + a] = vax; sm[SC::BVY + a] = vay; sm[SC::BW + a] = wa; }
-    if (dyn_b) { sm[SC::BVX + b] = vbx; sm[SC::BVY + b] = vby; sm[SC::BW + b] = wb; }
+    if (dyn_a) st4(sm + SC::BVEL + 4 * a, vax, vay, wa);
+    if (dyn_b) st4(sm + SC::BVEL + 4 * b, vbx, vby, wb);
 }
 
 // Second records, first half: the accumulated impulses the staged pair G + lane carried out of the
@@ -750,8 +758,8 @@ __device__ __noinline__ uint32_t reset_env(uint32_t *smu, const uint32_t *levels
         if (nl != level) { level = nl; jab = load_level_consts<SC, G>(smu, levels + (size_t)nl * SC::LV_WORDS); }
     }
     const uint32_t *lv = levels + (size_t)level * SC::LV_WORDS;
-    for (int i = lane; i < 6 * SC::N; i += G) smu[SC::BX + i] = lv[SC::LV_X + i];
-    if (SC::J > 0 && lane < SC::J) { smu[SC::JROW + JR_ACCX * SC::J + lane] = 0u; smu[SC::JROW + JR_ACCY * SC::J + lane] = 0u; }
+    for (int i = lane; i < 6 * SC::N; i += G) smu[body_word<SC>(i)] = lv[SC::LV_X + i];
+    if (SC::J > 0 && lane < SC::J) { smu[SC::JROW + kJointWords * lane + JR_ACCX] = 0u; smu[SC::JROW + kJointWords * lane + JR_ACCY] = 0u; }
     for (int i = lane; i < (SC::NPAIRS + 3) / 4; i += G) smu[SC::WIDX + i] = 0xffffffffu;
     if (lane == 0) {
         smu[SC::META + META_STEP] = 0u; smu[SC::META + META_EPISODE] = (uint32_t)episode; smu[SC::META + META_LEVEL] = (uint32_t)level;
@@ -901,7 +909,7 @@ struct Scene {
     // polygon a against circle b
     __device__ unsigned manifold_pc(int a, int b, Manifold &m, const uint32_t *lv) const {
         const int cnt = flag_nverts(smu[SC::BFL + a]);
-        const float cx = sm[SC::BX + b], cy = sm[SC::BY + b], r = sm[SC::RAD + (b - SC::P)];
+        const float cx = sm[SC::BPOS + 4 * b], cy = sm[SC::BPOS + 4 * b + 1], r = sm[SC::RAD + (b - SC::P)];
         float maxsep = 0.0f, mind2 = 0.0f, qx = 0.0f, qy = 0.0f, dqx = 0.0f, dqy = 0.0f;
         int kmax = 0, kmin = 0;
 #pragma unroll
@@ -934,8 +942,8 @@ struct Scene {
     }
 
     __device__ unsigned manifold_cc(int a, int b, Manifold &m) const {
-        const float ax = sm[SC::BX + a], ay = sm[SC::BY + a], ra = sm[SC::RAD + (a - SC::P)];
-        const float dx = sm[SC::BX + b] - ax, dy = sm[SC::BY + b] - ay, rb = sm[SC::RAD + (b - SC::P)];
+        const float ax = sm[SC::BPOS + 4 * a], ay = sm[SC::BPOS + 4 * a + 1], ra = sm[SC::RAD + (a - SC::P)];
+        const float dx = sm[SC::BPOS + 4 * b] - ax, dy = sm[SC::BPOS + 4 * b + 1] - ay, rb = sm[SC::RAD + (b - SC::P)];
         const float dist = sqrtf(dot2(dx, dy, dx, dy));
         if (dist < 1e-9f) { m.nx = 0.0f; m.ny = 1.0f; }
         else { const float inv = 1.0f / dist; m.nx = dx * inv; m.ny = dy * inv; }
@@ -952,12 +960,12 @@ struct Scene {
         const unsigned amask = (ab >> 10) & 3u;
         const bool dyn_a = (ab >> 26) & 1u, dyn_b = (ab >> 27) & 1u;
         if (MODE == 2) {
-            correct_pair(sm + SC::BX, sm + SC::BY, a, b, amask, dyn_a, dyn_b, rec.nx, rec.ny, rec.ma, rec.mb,
+            correct_pair(sm + SC::BPOS, a, b, amask, dyn_a, dyn_b, rec.nx, rec.ny, rec.ma, rec.mb,
                          sm[SC::WVX + lane], sm[SC::WVX + G + lane]);
             return;
         }
-        float vax = sm[SC::BVX + a], vay = sm[SC::BVY + a], wa = sm[SC::BW + a];
-        float vbx = sm[SC::BVX + b], vby = sm[SC::BVY + b], wb = sm[SC::BW + b];
+        const float4 va4 = ld4(sm + SC::BVEL + 4 * a), vb4 = ld4(sm + SC::BVEL + 4 * b);
+        float vax = va4.x, vay = va4.y, wa = va4.z, vbx = vb4.x, vby = vb4.y, wb = vb4.z;
         if (amask & 1u)
             manifold_rows<MODE>(rec.nx, rec.ny, rec.mu, rec.ma, rec.mb, rec.ia, rec.ib, rec.rna, rec.rnb, rec.rta, rec.rtb,
                                 rec.massn, rec.masst, rec.target, rec.accn, rec.acct, vax, vay, wa, vbx, vby, wb);
@@ -967,8 +975,8 @@ struct Scene {
                                 lanef(M2_RTB), lanef(M2_MASSN), lanef(M2_MASST), lanef(M2_TARGET), accn, acct, vax, vay, wa, vbx, vby, wb);
             if (MODE == 1) { lanef(LF_ACC2N) = accn; lanef(LF_ACC2T) = acct; }
         }
-        if (dyn_a) { sm[SC::BVX + a] = vax; sm[SC::BVY + a] = vay; sm[SC::BW + a] = wa; }
-        if (dyn_b) { sm[SC::BVX + b] = vbx; sm[SC::BVY + b] = vby; sm[SC::BW + b] = wb; }
+        if (dyn_a) st4(sm + SC::BVEL + 4 * a, vax, vay, wa);
+        if (dyn_b) st4(sm + SC::BVEL + 4 * b, vbx, vby, wb);
     }
     // records of one level touch disjoint movable bodies; levels in order keep the record order
     template <int MODE>
@@ -995,12 +1003,12 @@ struct Scene {
         // gravity, rotation, circle boxes
         for (int i = lane; i < SC::N; i += G) {
             const uint32_t fl = smu[SC::BFL + i];
-            if ((fl & F_ACTIVE) && (fl & F_DYNAMIC)) sm[SC::BVY + i] = sm[SC::BVY + i] + prm.gdt;
+            if ((fl & F_ACTIVE) && (fl & F_DYNAMIC)) sm[SC::BVEL + 4 * i + 1] = sm[SC::BVEL + 4 * i + 1] + prm.gdt;
             float c, sn;
-            sincos_spec(sm[SC::BTH + i], c, sn);
+            sincos_spec(sm[SC::BPOS + 4 * i + 2], c, sn);
             sm[SC::BC + i] = c; sm[SC::BS + i] = sn;
             if (i >= SC::P) {
-                const float r = sm[SC::RAD + (i - SC::P)], x = sm[SC::BX + i], y = sm[SC::BY + i];
+                const float r = sm[SC::RAD + (i - SC::P)], x = sm[SC::BPOS + 4 * i], y = sm[SC::BPOS + 4 * i + 1];
                 box4(i) = make_float4(x - r, y - r, x + r, y + r);
             }
         }
@@ -1013,7 +1021,7 @@ struct Scene {
                 float rx, ry, nx, ny;
                 rot2(c, sn, __uint_as_float(lv[SC::LV_PVX + v]), __uint_as_float(lv[SC::LV_PVY + v]), rx, ry);
                 rot2(c, sn, __uint_as_float(lv[SC::LV_PNX + v]), __uint_as_float(lv[SC::LV_PNY + v]), nx, ny);
-                const float wx = rx + sm[SC::BX + i], wy = ry + sm[SC::BY + i];
+                const float wx = rx + sm[SC::BPOS + 4 * i], wy = ry + sm[SC::BPOS + 4 * i + 1];
                 sm[SC::WVX + v] = wx; sm[SC::WVY + v] = wy; sm[SC::WNX + v] = nx; sm[SC::WNY + v] = ny;
                 sm[SC::WOFF + v] = dot2(nx, ny, wx, wy);
             }
@@ -1054,17 +1062,17 @@ struct Scene {
                     const float imp = (__uint_as_float(th[5]) * A) * prm.dt;
                     const float jx = imp * dx, jy = imp * dy;
                     const float im = sm[SC::BIM + i];
-                    sm[SC::BVX + i] = __fmaf_rn(jx, im, sm[SC::BVX + i]);
-                    sm[SC::BVY + i] = __fmaf_rn(jy, im, sm[SC::BVY + i]);
-                    sm[SC::BW + i] = __fmaf_rn(cross2(rx, ry, jx, jy), sm[SC::BII + i], sm[SC::BW + i]);
+                    sm[SC::BVEL + 4 * i] = __fmaf_rn(jx, im, sm[SC::BVEL + 4 * i]);
+                    sm[SC::BVEL + 4 * i + 1] = __fmaf_rn(jy, im, sm[SC::BVEL + 4 * i + 1]);
+                    sm[SC::BVEL + 4 * i + 2] = __fmaf_rn(cross2(rx, ry, jx, jy), sm[SC::BII + i], sm[SC::BVEL + 4 * i + 2]);
                 }
                 g.sync();
             }
         }
         // joint pre-step (poses only; velocities are not read): the row goes to shared memory
         if (SC::J > 0 && lane < SC::J) {
-            float *jr = sm + SC::JROW + lane;
-            if (!((jab >> 24) & 1u) || !prm.warm_start) { jr[JR_ACCX * SC::J] = 0.0f; jr[JR_ACCY * SC::J] = 0.0f; }
+            float *jr = sm + SC::JROW + kJointWords * lane;
+            if (!((jab >> 24) & 1u) || !prm.warm_start) { jr[JR_ACCX] = 0.0f; jr[JR_ACCY] = 0.0f; }
             if ((jab >> 24) & 1u) {
                 const int a = jab & 255, b = (jab >> 8) & 255;
                 const uint32_t *jl = lv + SC::LV_JOINT + 8 * lane;
@@ -1072,18 +1080,19 @@ struct Scene {
                 rot2(sm[SC::BC + a], sm[SC::BS + a], __uint_as_float(jl[1]), __uint_as_float(jl[2]), rax, ray);
                 rot2(sm[SC::BC + b], sm[SC::BS + b], __uint_as_float(jl[3]), __uint_as_float(jl[4]), rbx, rby);
                 const float ma = sm[SC::BIM + a], mb = sm[SC::BIM + b], ia = sm[SC::BII + a], ib = sm[SC::BII + b];
-                const float gx = (sm[SC::BX + b] + rbx) - (sm[SC::BX + a] + rax), gy = (sm[SC::BY + b] + rby) - (sm[SC::BY + a] + ray);
+                jr[JR_MA] = ma; jr[JR_MB] = mb; jr[JR_IA] = ia; jr[JR_IB] = ib;
+                const float gx = (sm[SC::BPOS + 4 * b] + rbx) - (sm[SC::BPOS + 4 * a] + rax), gy = (sm[SC::BPOS + 4 * b + 1] + rby) - (sm[SC::BPOS + 4 * a + 1] + ray);
                 const float msum = ma + mb;
                 float k11 = msum; k11 = __fmaf_rn(ia * ray, ray, k11); k11 = __fmaf_rn(ib * rby, rby, k11);
                 float k22 = msum; k22 = __fmaf_rn(ia * rax, rax, k22); k22 = __fmaf_rn(ib * rbx, rbx, k22);
                 float k12 = -((ia * rax) * ray); k12 = __fmaf_rn(-(ib * rbx), rby, k12);
                 const float det = __fmaf_rn(k11, k22, -(k12 * k12));
                 const float inv_det = 1.0f / det;
-                jr[JR_RAX * SC::J] = rax; jr[JR_RAY * SC::J] = ray; jr[JR_RBX * SC::J] = rbx; jr[JR_RBY * SC::J] = rby;
-                jr[JR_I11 * SC::J] = k22 * inv_det; jr[JR_I22 * SC::J] = k11 * inv_det; jr[JR_I12 * SC::J] = -(k12 * inv_det);
-                jr[JR_BX * SC::J] = prm.joint_alpha * gx; jr[JR_BY * SC::J] = prm.joint_alpha * gy;
+                jr[JR_RAX] = rax; jr[JR_RAY] = ray; jr[JR_RBX] = rbx; jr[JR_RBY] = rby;
+                jr[JR_I11] = k22 * inv_det; jr[JR_I22] = k11 * inv_det; jr[JR_I12] = -(k12 * inv_det);
+                jr[JR_BX] = prm.joint_alpha * gx; jr[JR_BY] = prm.joint_alpha * gy;
                 const float share = prm.joint_beta / msum;
-                jr[JR_CX * SC::J] = share * gx; jr[JR_CY * SC::J] = share * gy;
+                jr[JR_CX] = share * gx; jr[JR_CY] = share * gy;
             }
         }
         g.sync();
@@ -1270,9 +1279,8 @@ struct Scene {
         // Euler step with the solved velocities
         for (int i = lane; i < SC::N; i += G) {
             if (smu[SC::BFL + i] & F_ACTIVE) {
-                sm[SC::BX + i] = __fmaf_rn(prm.dt, sm[SC::BVX + i], sm[SC::BX + i]);
-                sm[SC::BY + i] = __fmaf_rn(prm.dt, sm[SC::BVY + i], sm[SC::BY + i]);
-                sm[SC::BTH + i] = __fmaf_rn(prm.dt, sm[SC::BW + i], sm[SC::BTH + i]);
+                const float4 p4 = ld4(sm + SC::BPOS + 4 * i), v4 = ld4(sm + SC::BVEL + 4 * i);
+                st4(sm + SC::BPOS + 4 * i, __fmaf_rn(prm.dt, v4.x, p4.x), __fmaf_rn(prm.dt, v4.y, p4.y), __fmaf_rn(prm.dt, v4.z, p4.z));
             }
         }
         g.sync();
@@ -1280,9 +1288,10 @@ struct Scene {
         else sweep_pairs<2>(cmax, clevel, clevel2);
         sweep_joints<SC, G, 2>(sm, jab, lane, jlevel, jmax, lv, prm.motor_rho);
         bool finite = true;
-        for (int i = lane; i < SC::N; i += G)
-            finite = finite && finite_bits(sm[SC::BX + i]) && finite_bits(sm[SC::BY + i]) && finite_bits(sm[SC::BTH + i]) &&
-                     finite_bits(sm[SC::BVX + i]) && finite_bits(sm[SC::BVY + i]) && finite_bits(sm[SC::BW + i]);
+        for (int i = lane; i < SC::N; i += G) {
+            const float4 p4 = ld4(sm + SC::BPOS + 4 * i), v4 = ld4(sm + SC::BVEL + 4 * i);
+            finite = finite && finite_bits(p4.x) && finite_bits(p4.y) && finite_bits(p4.z) && finite_bits(v4.x) && finite_bits(v4.y) && finite_bits(v4.z);
+        }
         finite = !g.any(!finite);
 
         // where the pairs of this step keep their accumulated impulses for the next one
@@ -1329,11 +1338,11 @@ struct Scene {
     // launch, so it is read past the (non-coherent) L1.
     __device__ __forceinline__ void run(int e, int s0, int s1) {
         uint32_t *st = prm.state + (size_t)e * SC::ST_WORDS;
-        for (int i = lane; i < 6 * SC::N; i += G) smu[SC::BX + i] = __ldcg(st + SC::ST_BODY + i);
+        for (int i = lane; i < 6 * SC::N; i += G) smu[body_word<SC>(i)] = __ldcg(st + SC::ST_BODY + i);
         if (lane < 5) smu[SC::META + lane] = __ldcg(st + SC::ST_META + lane);
         if (SC::J > 0 && lane < SC::J) {
-            smu[SC::JROW + JR_ACCX * SC::J + lane] = __ldcg(st + SC::ST_JACC + 2 * lane);
-            smu[SC::JROW + JR_ACCY * SC::J + lane] = __ldcg(st + SC::ST_JACC + 2 * lane + 1);
+            smu[SC::JROW + kJointWords * lane + JR_ACCX] = __ldcg(st + SC::ST_JACC + 2 * lane);
+            smu[SC::JROW + kJointWords * lane + JR_ACCY] = __ldcg(st + SC::ST_JACC + 2 * lane + 1);
         }
         for (int i = lane; i < (SC::NPAIRS + 3) / 4; i += G) smu[SC::WIDX + i] = 0xffffffffu;
         const int level = (int)__ldcg(st + SC::ST_META + META_LEVEL);
@@ -1368,10 +1377,10 @@ struct Scene {
             if (((s - s0) & 255) == 255) flush();
         }
         // write back
-        for (int i = lane; i < 6 * SC::N; i += G) st[SC::ST_BODY + i] = smu[SC::BX + i];
+        for (int i = lane; i < 6 * SC::N; i += G) st[SC::ST_BODY + i] = smu[body_word<SC>(i)];
         if (SC::J > 0 && lane < SC::J) {
-            st[SC::ST_JACC + 2 * lane] = smu[SC::JROW + JR_ACCX * SC::J + lane];
-            st[SC::ST_JACC + 2 * lane + 1] = smu[SC::JROW + JR_ACCY * SC::J + lane];
+            st[SC::ST_JACC + 2 * lane] = smu[SC::JROW + kJointWords * lane + JR_ACCX];
+            st[SC::ST_JACC + 2 * lane + 1] = smu[SC::JROW + kJointWords * lane + JR_ACCY];
         }
         if (lane < 5) st[SC::ST_META + lane] = smu[SC::META + lane];
         const int nw = (int)smu[SC::META + META_NWARM];
