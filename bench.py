@@ -29,7 +29,7 @@ sys.path.insert(0, ROOT)
 
 from paper_2410_23208_b200 import scenes  # noqa: E402
 
-FUSED = 32
+FUSED = 32   # default number of engine steps fused per k2d_step launch (--fused)
 METRIC = "env-steps/sec on 1 B200 (L scenes, 16384 envs); % of FP32 roofline"
 UNIT = "env-steps/s"
 
@@ -39,7 +39,7 @@ FLOPS = dict(body=37, circle_box=4, polygon=84, box_test=8, cc=16, pc=94, pp=190
              pair_prestep=5, man_prestep=54, man_warm=28, man_iter=57, man_pos=10,
              joint_fixed=48 + 33 + 18 + 8, joint_iter=38, thruster=27)
 # DRAM bytes one ncu capture measured for one k2d_step launch of the benchmark workload, per env
-NCU_DRAM_BYTES_PER_ENV_LAUNCH = 2216.4   # profiles/k2d_step_kernel_L_16384envs_32steps.md: (35.447 MB + 0.867 MB) / 16384 envs
+NCU_DRAM_BYTES_PER_ENV_LAUNCH = 1991.0   # profiles/k2d_step_kernel_L_16384envs_32steps.md: (32.210 MB + 0.411 MB) / 16384 envs; None once the kernel has changed since
 
 
 def fp32_peak_tflops(sm_count: int = 148, sm_mhz: float = 1965.0) -> float:
@@ -146,6 +146,7 @@ def run_reference(args) -> dict:
     cores = os.cpu_count() or 1
     sim = k2d_ref.RefSim(levels, sample_envs, auto_reset=w["auto_reset"], max_episode_steps=w["max_episode_steps"],
                          seed=scenes.workload_seed(args.workload))
+    FUSED = args.fused
     acts = scenes.make_actions(FUSED, sample_envs, dims.n_actions, 7)
     for _ in range(args.warmup):
         sim.step(acts, n_threads=cores)
@@ -180,13 +181,14 @@ def cpu_baseline(args, w, dims, levels) -> dict:
     t0 = time.perf_counter()
     sim.step(acts, n_threads=cores)
     dt = time.perf_counter() - t0
-    one = k2d_ref.RefSim(levels, 256, auto_reset=w["auto_reset"], max_episode_steps=w["max_episode_steps"])
+    n1 = min(256, sample_envs)
+    one = k2d_ref.RefSim(levels, n1, auto_reset=w["auto_reset"], max_episode_steps=w["max_episode_steps"])
     t1 = time.perf_counter()
-    one.step(acts[:32, :256], n_threads=1)
+    one.step(acts[:32, :n1], n_threads=1)
     dt1 = time.perf_counter() - t1
     return {"value": sample_envs * sample_steps / dt, "unit": UNIT, "cores": cores, "kind": "oracle",
             "sample": f"first {sample_envs} envs x {sample_steps} engine steps of the workload, {cores} threads over envs",
-            "one_core_value": 256 * 32 / dt1}
+            "one_core_value": n1 * 32 / dt1}
 
 
 def run_gpu(args) -> dict:
@@ -202,6 +204,7 @@ def run_gpu(args) -> dict:
     torch.cuda.set_device(local)
     dev = torch.device("cuda", local)
 
+    FUSED = args.fused
     w, dims, levels = workload_levels(args.workload)
     n_envs = args.envs or w["n_envs"]
     # weak scaling: every rank steps its own n_envs; env_offset makes level draws global
@@ -328,6 +331,7 @@ def main():
     ap.add_argument("--workload", type=int, default=3, choices=sorted(scenes.WORKLOADS))
     ap.add_argument("--envs", type=int, default=0, help="override the workload's env count (per GPU)")
     ap.add_argument("--lanes", type=int, default=0, help="lanes per scene (0 = library default)")
+    ap.add_argument("--fused", type=int, default=FUSED, help="engine steps per k2d_step launch (1 = one launch and one observation per step)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "k2d" else args.warmup
