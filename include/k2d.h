@@ -5,7 +5,8 @@
  * kind (arxiv 2410.23208): circles, convex polygons of 3 or 4 vertices, revolute joints with
  * motors, thrusters.  One call of k2d_step runs, for every scene and for n_steps steps, the
  * paper's Algorithm 1 (gravity, collision manifolds, motors, thrusters, warm start, a fixed
- * number of sequential-impulse solver iterations over joints then contacts, Euler step),
+ * number of sequential-impulse solver iterations over joints (revolute, fixed, with rotation
+ * limits) then contacts, Euler step),
  * followed by Kinetix's touch reward / termination ("Reward" paragraph: green touches blue
  * = +1 and done, green touches red = -1 and done) and the auto-reset.
  *
@@ -65,8 +66,8 @@ extern "C" {
 /* Engine and environment parameters.  The paper leaves dt, the iteration count and the
  * correction coefficients open; the defaults written by k2d_default_config are dt = 1/60,
  * gravity_y = -9.81, 8 solver iterations, contact_alpha = joint_alpha = 6 /s,
- * contact_beta = joint_beta = 0.1, slop = 0.005 m, restitution_threshold = 1 m/s,
- * face_tol = 1e-3 m, motor_rho = 1, aabb_margin = 0.01 m, warm starting on. */
+ * contact_beta = joint_beta = 0.1, joint_gamma = 6 /s, slop = 0.005 m,
+ * restitution_threshold = 1 m/s, face_tol = 1e-3 m, motor_rho = 1, aabb_margin = 0.01 m, warm starting on. */
 typedef struct k2d_config {
     int32_t n_envs;                /* >= 1                                                      */
     int32_t n_polygons;            /* 1 .. K2D_MAX_POLYGONS                                     */
@@ -89,6 +90,7 @@ typedef struct k2d_config {
     float joint_alpha, joint_beta; /* the same two corrections for the joint's point constraint */
     float motor_rho;               /* rho of the motor law j = p tanh((wa - wb - s A) rho)      */
     float aabb_margin;             /* bounding boxes further apart than this skip narrowphase   */
+    float joint_gamma;             /* angular correction of fixed joints and joint limits: gamma * angle error */
     uint64_t seed;                 /* seed of the K2D_RESET_POOL hash                           */
     int64_t env_offset;            /* global index of env 0 (sharding over several GPUs)        */
     int32_t device;                /* CUDA device ordinal                                       */
@@ -112,6 +114,10 @@ typedef struct k2d_level {
     float joint_anchor_a[K2D_MAX_JOINTS][2], joint_anchor_b[K2D_MAX_JOINTS][2]; /* body frame   */
     float motor_speed[K2D_MAX_JOINTS], motor_power[K2D_MAX_JOINTS];
     int32_t motor_binding[K2D_MAX_JOINTS], joint_active[K2D_MAX_JOINTS];
+    /* paper, "Fixed Joints" / "Joint Limits"; the relative rotation of a joint is angle[a] - angle[b] */
+    int32_t joint_fixed[K2D_MAX_JOINTS];             /* 1: also holds the relative rotation at joint_fixed_angle */
+    int32_t joint_limited[K2D_MAX_JOINTS];           /* 1: revolute, relative rotation kept in [min, max]       */
+    float joint_fixed_angle[K2D_MAX_JOINTS], joint_min[K2D_MAX_JOINTS], joint_max[K2D_MAX_JOINTS];
     int32_t thr_shape[K2D_MAX_THRUSTERS];
     float thr_pos[K2D_MAX_THRUSTERS][2], thr_rot[K2D_MAX_THRUSTERS], thr_power[K2D_MAX_THRUSTERS];
     int32_t thr_binding[K2D_MAX_THRUSTERS], thr_active[K2D_MAX_THRUSTERS];
@@ -171,13 +177,16 @@ int k2d_step_static_scratch(k2d_state *s, const float *dev_actions, int32_t n_st
 
 /* Symbolic per-entity observation (paper, tables "Information provided for shapes / joints /
  * thrusters"): dev_obs is [n_envs][k2d_obs_floats] floats; per env the shape rows (29 floats
- * each), two rows per joint (11 + n_actions floats each), one row per thruster (6 floats). */
+ * each), two rows per joint (11 + n_actions floats each), one row per thruster (6 floats).
+ * The buffer is plain row-major, so the same memory read as [n_envs][k2d_obs_floats] is the
+ * paper's Symbolic-Flat observation (the rows concatenated). */
 int k2d_obs(k2d_state *s, float *dev_obs);
 int k2d_obs_floats(const k2d_config *cfg);
 
 /* Canonical host copy of the dynamic state, for checkpoints and comparisons: per env
  * k2d_canonical_words 4-byte words: pos[N][2], angle[N], vel[N][2], angvel[N] (floats),
- * acc[n_slots][2] (accumulated normal, tangent impulse per manifold slot), jacc[n_joints][2],
+ * acc[n_slots][2] (accumulated normal, tangent impulse per manifold slot), jacc[n_joints][3]
+ * (accumulated impulse of the joint's point constraint x, y and of a fixed joint's angular row),
  * then int32 step_count, episode_count, level_id, status.  set_state followed by k2d_step
  * continues bit-identically. */
 int k2d_canonical_words(const k2d_config *cfg);

@@ -61,7 +61,7 @@ typedef struct {
     int32_t n_polygons, n_circles, n_joints, n_thrusters, n_actions, n_levels, n_envs;
     int32_t solver_iters, warm_start, auto_reset, max_episode_steps, broadphase;
     real dt, gravity_y, contact_alpha, contact_beta, slop, restitution_threshold, face_tol;
-    real joint_alpha, joint_beta, motor_rho, aabb_margin;
+    real joint_alpha, joint_beta, motor_rho, aabb_margin, joint_gamma;
     uint64_t seed;
     int64_t env_offset;
 } ref_config;
@@ -77,6 +77,8 @@ typedef struct {
     const real *joint_anchor_a, *joint_anchor_b;    /* [L][J][2] body-frame */
     const real *motor_speed, *motor_power;          /* [L][J] */
     const int32_t *motor_binding, *joint_active;    /* [L][J] */
+    const int32_t *joint_fixed, *joint_limited;     /* [L][J] fixed joint / revolute joint with rotation limits */
+    const real *joint_fixed_angle, *joint_min, *joint_max; /* [L][J] relative rotation (angle a - angle b) held / allowed */
     const int32_t *thr_shape;                       /* [L][T] */
     const real *thr_pos, *thr_rot, *thr_power;      /* [L][T][2], [L][T], [L][T] */
     const int32_t *thr_binding, *thr_active;        /* [L][T] */
@@ -94,13 +96,15 @@ typedef struct {
     int32_t *lv_static, *lv_role, *lv_active;
     int32_t *lv_joint_a, *lv_joint_b, *lv_motor_binding, *lv_joint_active;
     real *lv_anchor_a, *lv_anchor_b, *lv_motor_speed, *lv_motor_power;
+    int32_t *lv_joint_fixed, *lv_joint_limited;
+    real *lv_fixed_angle, *lv_joint_min, *lv_joint_max;
     int32_t *lv_thr_shape, *lv_thr_binding, *lv_thr_active;
     real *lv_thr_pos, *lv_thr_rot, *lv_thr_dir, *lv_thr_power;
     uint8_t *lv_collide; /* [L][n_pairs] */
     /* per env state */
     real *pos, *angle, *vel, *angvel;  /* [E][N][2] ... */
     real *acc;        /* [E][n_slots][2] accumulated normal, tangent impulse */
-    real *jacc;       /* [E][J][2] accumulated joint impulse */
+    real *jacc;       /* [E][J][3] accumulated joint impulse: point constraint x, y; fixed joint's angular impulse */
     int32_t *step_count, *episode_count, *level_id, *status;
     /* per env trace of the last step's manifolds: [E][n_slots][6] = px,py,nx,ny,pen,active */
     real *manifold;
@@ -446,7 +450,7 @@ static void reset_env(ref_sim *S, int e, int level) {
     memcpy(S->angle + (size_t)e * N, S->lv_angle + (size_t)level * N, sizeof(real) * N);
     memcpy(S->angvel + (size_t)e * N, S->lv_angvel + (size_t)level * N, sizeof(real) * N);
     memset(S->acc + (size_t)e * S->n_slots * 2, 0, sizeof(real) * S->n_slots * 2);
-    memset(S->jacc + (size_t)e * S->J * 2, 0, sizeof(real) * S->J * 2);
+    memset(S->jacc + (size_t)e * S->J * 3, 0, sizeof(real) * S->J * 3);
     S->step_count[e] = 0;
     S->level_id[e] = level;
     S->status[e] = 0;
@@ -489,6 +493,11 @@ ref_sim *k2d_ref_create(const ref_config *cfg, const ref_levels *L) {
     COPY_ARR(S->lv_motor_power, L->motor_power, nl * J, real);
     COPY_ARR(S->lv_motor_binding, L->motor_binding, nl * J, int32_t);
     COPY_ARR(S->lv_joint_active, L->joint_active, nl * J, int32_t);
+    COPY_ARR(S->lv_joint_fixed, L->joint_fixed, nl * J, int32_t);
+    COPY_ARR(S->lv_joint_limited, L->joint_limited, nl * J, int32_t);
+    COPY_ARR(S->lv_fixed_angle, L->joint_fixed_angle, nl * J, real);
+    COPY_ARR(S->lv_joint_min, L->joint_min, nl * J, real);
+    COPY_ARR(S->lv_joint_max, L->joint_max, nl * J, real);
     COPY_ARR(S->lv_thr_shape, L->thr_shape, nl * T, int32_t);
     COPY_ARR(S->lv_thr_pos, L->thr_pos, nl * T * 2, real);
     COPY_ARR(S->lv_thr_rot, L->thr_rot, nl * T, real);
@@ -510,7 +519,7 @@ ref_sim *k2d_ref_create(const ref_config *cfg, const ref_levels *L) {
 
     NEW_ARR(S->pos, (size_t)E * N * 2, real); NEW_ARR(S->vel, (size_t)E * N * 2, real);
     NEW_ARR(S->angle, (size_t)E * N, real); NEW_ARR(S->angvel, (size_t)E * N, real);
-    NEW_ARR(S->acc, (size_t)E * S->n_slots * 2, real); NEW_ARR(S->jacc, (size_t)E * J * 2, real);
+    NEW_ARR(S->acc, (size_t)E * S->n_slots * 2, real); NEW_ARR(S->jacc, (size_t)E * J * 3, real);
     NEW_ARR(S->step_count, E, int32_t); NEW_ARR(S->episode_count, E, int32_t);
     NEW_ARR(S->level_id, E, int32_t); NEW_ARR(S->status, E, int32_t);
     NEW_ARR(S->manifold, (size_t)E * S->n_slots * 6, real);
@@ -527,7 +536,7 @@ void k2d_ref_destroy(ref_sim *S) {
         S->lv_joint_a, S->lv_joint_b, S->lv_motor_binding, S->lv_joint_active, S->lv_anchor_a, S->lv_anchor_b,
         S->lv_motor_speed, S->lv_motor_power, S->lv_thr_shape, S->lv_thr_binding, S->lv_thr_active, S->lv_thr_pos,
         S->lv_thr_rot, S->lv_thr_dir, S->lv_thr_power, S->lv_collide, S->pos, S->angle, S->vel, S->angvel, S->acc,
-        S->jacc, S->step_count, S->episode_count, S->level_id, S->status, S->manifold, S->counters };
+        S->jacc, S->lv_joint_fixed, S->lv_joint_limited, S->lv_fixed_angle, S->lv_joint_min, S->lv_joint_max, S->step_count, S->episode_count, S->level_id, S->status, S->manifold, S->counters };
     for (size_t i = 0; i < sizeof(ptrs) / sizeof(ptrs[0]); ++i) free(ptrs[i]);
     free(S);
 }
@@ -584,6 +593,9 @@ typedef struct {
     vec2 ra, rb, bias, corr_dir;
     real i11, i12, i22;              /* inverse of the 2x2 effective mass matrix */
     real ma, mb, ia, ib;
+    /* angular row (paper, "Fixed Joints" and "Joint Limits"): 0 none, 1 fixed, 2 beyond the upper limit, 3 beyond the lower */
+    int ang;
+    real kr, bias_r;                 /* 1 / (1/I_a + 1/I_b); gamma * angular error */
 } joint_row;
 
 static void step_env(ref_sim *S, int e, const real *act, real *out_reward, uint8_t *out_done, int64_t *cnt) {
@@ -591,7 +603,7 @@ static void step_env(ref_sim *S, int e, const real *act, real *out_reward, uint8
     const int P = S->P, C = S->C, N = S->N, J = S->J, T = S->T;
     real *pos = S->pos + (size_t)e * N * 2, *vel = S->vel + (size_t)e * N * 2;
     real *ang = S->angle + (size_t)e * N, *angvel = S->angvel + (size_t)e * N;
-    real *acc = S->acc + (size_t)e * S->n_slots * 2, *jacc = S->jacc + (size_t)e * J * 2;
+    real *acc = S->acc + (size_t)e * S->n_slots * 2, *jacc = S->jacc + (size_t)e * J * 3;
     real *trace = S->manifold + (size_t)e * S->n_slots * 6;
 
     /* a frozen env (non-finite state, no auto-reset) reports done and nothing else */
@@ -749,8 +761,9 @@ static void step_env(ref_sim *S, int e, const real *act, real *out_reward, uint8
         int a = S->lv_joint_a[l * J + j], b = S->lv_joint_b[l * J + j];
         q->a = a; q->b = b;
         q->on = S->lv_joint_active[l * J + j] && active[a] && active[b] && (inv_mass[a] + inv_mass[b] > RC(0));
-        if (!q->on) { jacc[2 * j] = jacc[2 * j + 1] = RC(0); continue; }
-        if (!cf->warm_start) jacc[2 * j] = jacc[2 * j + 1] = RC(0);
+        q->ang = 0;
+        if (!q->on) { jacc[3 * j] = jacc[3 * j + 1] = jacc[3 * j + 2] = RC(0); continue; }
+        if (!cf->warm_start) jacc[3 * j] = jacc[3 * j + 1] = jacc[3 * j + 2] = RC(0);
         vec2 la = { S->lv_anchor_a[(size_t)(l * J + j) * 2], S->lv_anchor_a[(size_t)(l * J + j) * 2 + 1] };
         vec2 lb = { S->lv_anchor_b[(size_t)(l * J + j) * 2], S->lv_anchor_b[(size_t)(l * J + j) * 2 + 1] };
         q->ra = rot2(cs[a], sn[a], la); q->rb = rot2(cs[b], sn[b], lb);
@@ -766,6 +779,25 @@ static void step_env(ref_sim *S, int e, const real *act, real *out_reward, uint8
         q->bias.x = cf->joint_alpha * gap.x; q->bias.y = cf->joint_alpha * gap.y;
         real share = cf->joint_beta / msum;
         q->corr_dir.x = share * gap.x; q->corr_dir.y = share * gap.y;
+        /* angular row.  Fixed joint ("Fixed Joints"): the relative rotation angle_a - angle_b is held at
+         * the joint's angle, error C, velocity correction gamma * C, accumulated and warm-started.
+         * Limited revolute joint ("Joint Limits"): a row only while the relative rotation is beyond a
+         * limit, C measured from that limit, never accumulated.  Both from the poses at the start of
+         * the step, like the manifolds. */
+        real isum = q->ia + q->ib;
+        q->kr = RC(0); q->bias_r = RC(0);
+        if (isum > RC(0)) {
+            real rel = ang[a] - ang[b];
+            if (S->lv_joint_fixed[l * J + j]) {
+                q->ang = 1; q->kr = RC(1) / isum;
+                q->bias_r = cf->joint_gamma * (rel - S->lv_fixed_angle[l * J + j]);
+            } else if (S->lv_joint_limited[l * J + j]) {
+                real hi = S->lv_joint_max[l * J + j], lo = S->lv_joint_min[l * J + j];
+                if (rel > hi) { q->ang = 2; q->kr = RC(1) / isum; q->bias_r = cf->joint_gamma * (rel - hi); }
+                else if (rel < lo) { q->ang = 3; q->kr = RC(1) / isum; q->bias_r = cf->joint_gamma * (rel - lo); }
+            }
+        }
+        if (q->ang != 1) jacc[3 * j + 2] = RC(0);
     }
 
     /* Alg. 1 lines 6-9: warm start, contacts first, then joints */
@@ -779,12 +811,17 @@ static void step_env(ref_sim *S, int e, const real *act, real *out_reward, uint8
     for (int j = 0; j < J; ++j) {
         joint_row *q = &jr[j];
         if (!q->on) continue;
-        vec2 lam = { jacc[2 * j], jacc[2 * j + 1] };
+        vec2 lam = { jacc[3 * j], jacc[3 * j + 1] };
         real *va = vel + 2 * q->a, *vb = vel + 2 * q->b;
         va[0] = R_FMA(-q->ma, lam.x, va[0]); va[1] = R_FMA(-q->ma, lam.y, va[1]);
         angvel[q->a] = R_FMA(-q->ia, cross2(q->ra, lam), angvel[q->a]);
         vb[0] = R_FMA(q->mb, lam.x, vb[0]); vb[1] = R_FMA(q->mb, lam.y, vb[1]);
         angvel[q->b] = R_FMA(q->ib, cross2(q->rb, lam), angvel[q->b]);
+        if (q->ang == 1) {
+            real lr = jacc[3 * j + 2];
+            angvel[q->a] = R_FMA(-lr, q->ia, angvel[q->a]);
+            angvel[q->b] = R_FMA(lr, q->ib, angvel[q->b]);
+        }
     }
 
     /* Alg. 1 lines 10-13: solver iterations, joints then contacts, sequential */
@@ -799,11 +836,29 @@ static void step_env(ref_sim *S, int e, const real *act, real *out_reward, uint8
             real cy = (R_FMA(wb, q->rb.x, vb[1])) - (R_FMA(wa, q->ra.x, va[1]));
             real rx = -(cx + q->bias.x), ry = -(cy + q->bias.y);
             vec2 lam = { R_FMA(q->i11, rx, q->i12 * ry), R_FMA(q->i12, rx, q->i22 * ry) };
-            jacc[2 * j] = jacc[2 * j] + lam.x; jacc[2 * j + 1] = jacc[2 * j + 1] + lam.y;
+            jacc[3 * j] = jacc[3 * j] + lam.x; jacc[3 * j + 1] = jacc[3 * j + 1] + lam.y;
             va[0] = R_FMA(-q->ma, lam.x, va[0]); va[1] = R_FMA(-q->ma, lam.y, va[1]);
             angvel[q->a] = R_FMA(-q->ia, cross2(q->ra, lam), wa);
             vb[0] = R_FMA(q->mb, lam.x, vb[0]); vb[1] = R_FMA(q->mb, lam.y, vb[1]);
             angvel[q->b] = R_FMA(q->ib, cross2(q->rb, lam), wb);
+            if (q->ang) {
+                /* angular impulse j_r = (w_a - w_b + correction) / (1/I_a + 1/I_b): a loses j_r / I_a, b gains j_r / I_b */
+                real wrel = angvel[q->a] - angvel[q->b];
+                real v;
+                if (q->ang == 1) v = wrel + q->bias_r;
+                else if (q->ang == 2) {
+                    /* beyond the upper limit: no correction if already returning; only ever pushes back */
+                    v = (wrel < RC(0)) ? wrel : wrel + q->bias_r;
+                    v = rmax(v, RC(0));
+                } else {
+                    v = (wrel > RC(0)) ? wrel : wrel + q->bias_r;
+                    v = rmin(v, RC(0));
+                }
+                real lr = v * q->kr;
+                if (q->ang == 1) jacc[3 * j + 2] = jacc[3 * j + 2] + lr;
+                angvel[q->a] = R_FMA(-lr, q->ia, angvel[q->a]);
+                angvel[q->b] = R_FMA(lr, q->ib, angvel[q->b]);
+            }
         }
         for (int i = 0; i < n_rows; ++i) {
             contact_row *r = &rows[i];
@@ -960,7 +1015,7 @@ void k2d_ref_obs(ref_sim *S, real *obs) {
                 real *r = o + N * 29 + (2 * j + d) * jw;
                 int from = d ? b : a, to = d ? a : b;
                 const real *lf = d ? lb : la, *lt = d ? la : lb;
-                r[0] = RC(1); r[1] = RC(0);
+                r[0] = RC(1); r[1] = S->lv_joint_fixed[l * J + j] ? RC(1) : RC(0);
                 r[2] = lf[0]; r[3] = lf[1]; r[4] = lt[0]; r[5] = lt[1];
                 r[6] = S->lv_motor_power[l * J + j]; r[7] = S->lv_motor_speed[l * J + j]; r[8] = RC(0);
                 r[9 + S->lv_motor_binding[l * J + j]] = RC(1);

@@ -18,20 +18,22 @@ _LIBS = {}
 DEFAULTS = dict(
     solver_iters=8, warm_start=1, auto_reset=0, max_episode_steps=0, broadphase=1,
     dt=1.0 / 60.0, gravity_y=-9.81, contact_alpha=6.0, contact_beta=0.1, slop=0.005,
-    restitution_threshold=1.0, face_tol=1e-3, joint_alpha=6.0, joint_beta=0.1, motor_rho=1.0,
+    restitution_threshold=1.0, face_tol=1e-3, joint_alpha=6.0, joint_beta=0.1, joint_gamma=6.0, motor_rho=1.0,
     aabb_margin=0.01, seed=0, env_offset=0,
 )
 
 _REAL_FIELDS = ("dt", "gravity_y", "contact_alpha", "contact_beta", "slop", "restitution_threshold", "face_tol",
-                "joint_alpha", "joint_beta", "motor_rho", "aabb_margin")
+                "joint_alpha", "joint_beta", "motor_rho", "aabb_margin", "joint_gamma")
 _INT_FIELDS = ("n_polygons", "n_circles", "n_joints", "n_thrusters", "n_actions", "n_levels", "n_envs",
                "solver_iters", "warm_start", "auto_reset", "max_episode_steps", "broadphase")
 
 _LEVEL_REAL = ("poly_verts", "circle_radius", "pos", "angle", "vel", "angvel", "density", "friction", "restitution",
-               "joint_anchor_a", "joint_anchor_b", "motor_speed", "motor_power", "thr_pos", "thr_rot", "thr_power")
+               "joint_anchor_a", "joint_anchor_b", "motor_speed", "motor_power", "joint_fixed_angle", "joint_min", "joint_max",
+               "thr_pos", "thr_rot", "thr_power")
 _LEVEL_ORDER = ("poly_verts", "poly_nverts", "circle_radius", "pos", "angle", "vel", "angvel", "density", "friction",
                 "restitution", "is_static", "role", "active", "joint_a", "joint_b", "joint_anchor_a",
-                "joint_anchor_b", "motor_speed", "motor_power", "motor_binding", "joint_active", "thr_shape",
+                "joint_anchor_b", "motor_speed", "motor_power", "motor_binding", "joint_active", "joint_fixed",
+                "joint_limited", "joint_fixed_angle", "joint_min", "joint_max", "thr_shape",
                 "thr_pos", "thr_rot", "thr_power", "thr_binding", "thr_active")
 
 
@@ -136,7 +138,7 @@ class RefSim:
         self.vel = _as(v.vel, (E, N, 2), r)
         self.angvel = _as(v.angvel, (E, N), r)
         self.acc = _as(v.acc, (E, self.n_slots, 2), r)
-        self.jacc = _as(v.jacc, (E, J, 2), r)
+        self.jacc = _as(v.jacc, (E, J, 3), r)
         self.step_count = _as(v.step_count, (E,), np.int32)
         self.episode_count = _as(v.episode_count, (E,), np.int32)
         self.level_id = _as(v.level_id, (E,), np.int32)

@@ -61,7 +61,7 @@ static int check_config(const k2d_config *c) {
         !(c->lanes_per_scene == 0 || c->lanes_per_scene == 8 || c->lanes_per_scene == 16 || c->lanes_per_scene == 32))
         return K2D_ERR_CONFIG;
     const float f[] = { c->dt, c->gravity_y, c->contact_alpha, c->contact_beta, c->slop, c->restitution_threshold, c->face_tol,
-                        c->joint_alpha, c->joint_beta, c->motor_rho, c->aabb_margin };
+                        c->joint_alpha, c->joint_beta, c->motor_rho, c->aabb_margin, c->joint_gamma };
     for (float v : f) if (!std::isfinite(v)) return K2D_ERR_CONFIG;
     if (!(c->dt > 0.0f) || c->aabb_margin < 0.0f || c->slop < 0.0f) return K2D_ERR_CONFIG;
     return K2D_OK;
@@ -191,14 +191,15 @@ static int pack_level(const k2d_config *cfg, const ClassInfo &ci, const k2d_leve
     std::vector<int> body_level(ci.N, 0);
     std::vector<std::pair<int, int>> joined;
     for (int j = 0; j < nJ; ++j) {
-        uint32_t *jw = w + ci.LV_JOINT + 8 * j;
+        uint32_t *jw = w + ci.LV_JOINT + kJointLevelWords * j;
         if (!L->joint_active[j]) continue;
         const int a0 = L->joint_a[j], b0 = L->joint_b[j];
         if (a0 < 0 || a0 >= nN || b0 < 0 || b0 >= nN || a0 == b0) return K2D_ERR_LEVEL;
         if (L->motor_binding[j] < 0 || L->motor_binding[j] >= cfg->n_actions) return K2D_ERR_LEVEL;
-        const float v[6] = { L->joint_anchor_a[j][0], L->joint_anchor_a[j][1], L->joint_anchor_b[j][0], L->joint_anchor_b[j][1],
-                             L->motor_speed[j], L->motor_power[j] };
+        const float v[9] = { L->joint_anchor_a[j][0], L->joint_anchor_a[j][1], L->joint_anchor_b[j][0], L->joint_anchor_b[j][1],
+                             L->motor_speed[j], L->motor_power[j], L->joint_fixed_angle[j], L->joint_min[j], L->joint_max[j] };
         for (float x : v) if (!std::isfinite(x)) return K2D_ERR_LEVEL;
+        if (L->joint_limited[j] && !L->joint_fixed[j] && L->joint_min[j] > L->joint_max[j]) return K2D_ERR_LEVEL;
         const int a = internal(a0), b = internal(b0);
         const bool on = is_active[a] && is_active[b] && !(is_static[a] && is_static[b]);
         int lvl = 0;
@@ -210,8 +211,10 @@ static int pack_level(const k2d_config *cfg, const ClassInfo &ci, const k2d_leve
             if (!is_static[b]) body_level[b] = lvl;
         }
         jw[0] = (uint32_t)a | ((uint32_t)b << 8) | ((uint32_t)L->motor_binding[j] << 16) | ((on ? 1u : 0u) << 24) | ((uint32_t)lvl << 25) | (1u << 28) |
-                ((is_static[a] ? 0u : 1u) << 29) | ((is_static[b] ? 0u : 1u) << 30);
-        for (int k = 0; k < 6; ++k) jw[1 + k] = f2u(v[k]);
+                ((is_static[a] ? 0u : 1u) << 29) | ((is_static[b] ? 0u : 1u) << 30) |
+                (((L->joint_fixed[j] || L->joint_limited[j]) ? 1u : 0u) << 31);
+        for (int k = 0; k < 9; ++k) jw[1 + k] = f2u(v[k]);
+        jw[10] = L->joint_fixed[j] ? 1u : (L->joint_limited[j] ? 2u : 0u);
         joined.emplace_back(a, b);
     }
     std::fill(body_level.begin(), body_level.end(), 0);
@@ -298,7 +301,7 @@ static StepParams step_params(const k2d_state *s, const float *dev_actions, int 
     }
     prm.solver_iters = c.solver_iters; prm.warm_start = c.warm_start; prm.auto_reset = c.auto_reset; prm.max_episode_steps = c.max_episode_steps;
     prm.dt = c.dt; prm.gdt = c.gravity_y * c.dt; prm.contact_alpha = c.contact_alpha; prm.contact_beta = c.contact_beta; prm.slop = c.slop;
-    prm.rest_thr = c.restitution_threshold; prm.face_tol = c.face_tol; prm.joint_alpha = c.joint_alpha; prm.joint_beta = c.joint_beta;
+    prm.rest_thr = c.restitution_threshold; prm.face_tol = c.face_tol; prm.joint_alpha = c.joint_alpha; prm.joint_beta = c.joint_beta; prm.joint_gamma = c.joint_gamma;
     prm.motor_rho = c.motor_rho; prm.aabb_margin = c.aabb_margin; prm.seed = c.seed; prm.env_offset = c.env_offset;
     return prm;
 }
@@ -323,7 +326,7 @@ int k2d_default_config(k2d_config *cfg, int32_t n_envs, int32_t n_polygons, int3
     cfg->solver_iters = 8; cfg->warm_start = 1; cfg->auto_reset = K2D_RESET_NONE; cfg->max_episode_steps = 0; cfg->max_fused_steps = 64;
     cfg->dt = 1.0f / 60.0f; cfg->gravity_y = -9.81f;
     cfg->contact_alpha = 6.0f; cfg->contact_beta = 0.1f; cfg->slop = 0.005f; cfg->restitution_threshold = 1.0f; cfg->face_tol = 1e-3f;
-    cfg->joint_alpha = 6.0f; cfg->joint_beta = 0.1f; cfg->motor_rho = 1.0f; cfg->aabb_margin = 0.01f;
+    cfg->joint_alpha = 6.0f; cfg->joint_beta = 0.1f; cfg->joint_gamma = 6.0f; cfg->motor_rho = 1.0f; cfg->aabb_margin = 0.01f;
     return check_config(cfg);
 }
 
@@ -348,7 +351,7 @@ int k2d_canonical_words(const k2d_config *cfg) {
     if (check_config(cfg) != K2D_OK) return 0;
     const int P = cfg->n_polygons, C = cfg->n_circles, N = P + C;
     const int slots = P * (P - 1) + P * C + C * (C - 1) / 2;
-    return 6 * N + 2 * slots + 2 * cfg->n_joints + 4;
+    return 6 * N + 2 * slots + 3 * cfg->n_joints + 4;
 }
 
 int k2d_create(const k2d_config *cfg, void *dev_state_buf, void *dev_level_pool_buf, const k2d_level *host_levels, k2d_state **out) {
@@ -470,8 +473,8 @@ int k2d_get_state(k2d_state *s, void *host_canonical) {
             if (p < nP * (nP - 1) / 2) { acc[2 * slot + 2] = wr[3]; acc[2 * slot + 3] = wr[4]; }
         }
         uint32_t *jacc = acc + 2 * n_slots;
-        for (int j = 0; j < 2 * nJ; ++j) jacc[j] = st[ci.ST_JACC + j];
-        uint32_t *meta = jacc + 2 * nJ;
+        for (int j = 0; j < 3 * nJ; ++j) jacc[j] = st[ci.ST_JACC + j];
+        uint32_t *meta = jacc + 3 * nJ;
         for (int k = 0; k < 4; ++k) meta[k] = st[ci.ST_META + k];
     }
     return K2D_OK;
@@ -514,8 +517,8 @@ int k2d_set_state(k2d_state *s, const void *host_canonical) {
             wr[0] = (uint32_t)s->pair_map[p]; wr[1] = v[0]; wr[2] = v[1]; wr[3] = v[2]; wr[4] = v[3];
         }
         const uint32_t *jacc = acc + 2 * n_slots;
-        for (int j = 0; j < 2 * nJ; ++j) st[ci.ST_JACC + j] = jacc[j];
-        const uint32_t *meta = jacc + 2 * nJ;
+        for (int j = 0; j < 3 * nJ; ++j) st[ci.ST_JACC + j] = jacc[j];
+        const uint32_t *meta = jacc + 3 * nJ;
         for (int k = 0; k < 4; ++k) st[ci.ST_META + k] = meta[k];
         st[ci.ST_META + 4] = (uint32_t)nwarm;
     }

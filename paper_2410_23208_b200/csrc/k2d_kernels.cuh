@@ -32,7 +32,8 @@ constexpr unsigned kWaitLimit = 1u << 24;   // polls (about 100 ns apart) before
 constexpr int kRecWords = 24;   // contact pair record
 constexpr int kWarmWords = 5;   // pair index + 4 accumulated impulses
 constexpr int kStageWords = 9;  // packed pair word, normal, two contact points with penetration
-constexpr int kJointWords = 20; // joint row kept in shared memory: five 16-byte groups
+constexpr int kJointWords = 24; // joint row kept in shared memory: six 16-byte groups
+constexpr int kJointLevelWords = 12;  // joint record of a level
 
 // ---------------------------------------------------------------- size classes and layouts
 template <int P_, int C_, int J_, int T_>
@@ -47,12 +48,13 @@ struct SizeClass {
     static constexpr int LV_IM = 6 * N, LV_II = 7 * N, LV_FR = 8 * N, LV_RE = 9 * N, LV_FLAGS = 10 * N, LV_DENS = 11 * N;
     static constexpr int LV_RAD = 12 * N;
     static constexpr int LV_PVX = LV_RAD + C, LV_PVY = LV_PVX + P4, LV_PNX = LV_PVY + P4, LV_PNY = LV_PNX + P4, LV_ELEN = LV_PNY + P4;
-    static constexpr int LV_JOINT = LV_ELEN + P4;        // J x 8: packed, anchor a xy, anchor b xy, speed, power, pad
-    static constexpr int LV_THR = LV_JOINT + 8 * J;      // T x 8: packed, pos xy, dir xy, power, pad, pad
+    // J x 12: packed, anchor a xy, anchor b xy, speed, power, fixed angle, lower limit, upper limit, kind (1 fixed, 2 limited), pad
+    static constexpr int LV_JOINT = LV_ELEN + P4;
+    static constexpr int LV_THR = LV_JOINT + kJointLevelWords * J;      // T x 8: packed, pos xy, dir xy, power, pad, pad
     static constexpr int LV_MASK = LV_THR + 8 * T;
     static constexpr int LV_WORDS = (LV_MASK + MASKW + 3) / 4 * 4;
     // state record: bodies (same order as shared memory), joint impulses, meta, warm list
-    static constexpr int ST_BODY = 0, ST_JACC = 6 * N, ST_META = ST_JACC + 2 * J, ST_WARM = ST_META + 8;
+    static constexpr int ST_BODY = 0, ST_JACC = 6 * N, ST_META = ST_JACC + 3 * J, ST_WARM = ST_META + 8;
     static constexpr int ST_WORDS = (ST_WARM + kWarmWords * NPAIRS + 3) / 4 * 4;
     // A scene with more touching pairs than lanes takes the step's contact solve through global
     // scratch: one memory record and one warm entry per pair.
@@ -98,8 +100,9 @@ __host__ __device__ constexpr int ovs(int f) { return f < 3 ? f : f + 1; }
 constexpr int OV_ACC0N = R_M0 + M_ACCN, OV_ACC0T = R_M0 + M_ACCT, OV_ACC1N = R_M0 + M_WORDS + M_ACCN, OV_ACC1T = R_M0 + M_WORDS + M_ACCT;
 // joint row fields
 enum { JR_RAX = 0, JR_RAY, JR_RBX, JR_RBY, JR_I11, JR_I12, JR_I22, JR_PAD0, JR_BX, JR_BY, JR_CX, JR_CY, JR_MA, JR_MB, JR_IA, JR_IB,
-       JR_ACCX, JR_ACCY, JR_PAD1, JR_PAD2 };
-static_assert(JR_PAD2 + 1 == kJointWords, "joint row size");
+       JR_ACCX, JR_ACCY, JR_PAD1, JR_PAD2,
+       JR_ANG, JR_KR, JR_BIASR, JR_ACCR };   // angular row: kind (0 none, 1 fixed, 2 beyond the upper limit, 3 beyond the lower), 1 / (1/I_a + 1/I_b), gamma x error, accumulated
+static_assert(JR_ACCR + 1 == kJointWords, "joint row size");
 enum { META_STEP = 0, META_EPISODE, META_LEVEL, META_STATUS, META_NWARM };
 
 // shared-memory word of word i of a state record's body block (x[N], y[N], angle[N], vx[N], vy[N], w[N])
@@ -119,7 +122,7 @@ __host__ __device__ constexpr int region_words() {
 constexpr uint32_t F_ACTIVE = 1u, F_DYNAMIC = 2u;
 __host__ __device__ inline uint32_t flag_role(uint32_t f) { return (f >> 2) & 3u; }
 __host__ __device__ inline uint32_t flag_nverts(uint32_t f) { return (f >> 4) & 7u; }
-// joint packed word: a | b<<8 | binding<<16 | on<<24 | level<<25 | active<<28 | a movable<<29 | b movable<<30
+// joint packed word: a | b<<8 | binding<<16 | on<<24 | level<<25 | active<<28 | a movable<<29 | b movable<<30 | fixed or limited<<31
 // thruster packed word: shape | binding<<8 | on<<16 | level<<17 | active<<20
 // record AB word: a | b<<5 | amask<<10 | pair<<12 | level<<19 | dynA<<26 | dynB<<27
 
@@ -137,7 +140,7 @@ struct StepParams {
     int n_envs, n_steps, n_actions, n_levels;
     int chunk_steps, n_chunks;   // a launch is cut into n_chunks pieces of chunk_steps steps; work items are (chunk, env)
     int solver_iters, warm_start, auto_reset, max_episode_steps;
-    float dt, gdt, contact_alpha, contact_beta, slop, rest_thr, face_tol, joint_alpha, joint_beta, motor_rho, aabb_margin;
+    float dt, gdt, contact_alpha, contact_beta, slop, rest_thr, face_tol, joint_alpha, joint_beta, joint_gamma, motor_rho, aabb_margin;
     unsigned long long seed;
     long long env_offset;
 };
@@ -351,7 +354,7 @@ __device__ __forceinline__ void visit_joint(float *sm, uint32_t jab, int j, cons
     float *jr = sm + SC::JROW + kJointWords * j;
     if (MODE == 3) {
         const float A = fmax_cmp(fmin_cmp(sm[SC::ACT + ((jab >> 16) & 255)], 1.0f), -1.0f);
-        const float speed = __uint_as_float(lv[SC::LV_JOINT + 8 * j + 5]), power = __uint_as_float(lv[SC::LV_JOINT + 8 * j + 6]);
+        const float speed = __uint_as_float(lv[SC::LV_JOINT + kJointLevelWords * j + 5]), power = __uint_as_float(lv[SC::LV_JOINT + kJointLevelWords * j + 6]);
         const float wa = sm[SC::BVEL + 4 * a + 2], wb = sm[SC::BVEL + 4 * b + 2];
         const float arg = __fmaf_rn(-speed, A, wa - wb) * motor_rho;
         const float jr_ = power * tanh_spec(arg);
@@ -371,6 +374,10 @@ __device__ __forceinline__ void visit_joint(float *sm, uint32_t jab, int j, cons
     const float rax = r4.x, ray = r4.y, rbx = r4.z, rby = r4.w;
     const float4 va4 = ld4(sm + SC::BVEL + 4 * a), vb4 = ld4(sm + SC::BVEL + 4 * b);
     float vax = va4.x, vay = va4.y, wa = va4.z, vbx = vb4.x, vby = vb4.y, wb = vb4.z;
+    // angular row of a fixed or limited joint (bit 31 of the packed word): kind this step, inverse angular mass,
+    // correction, accumulated angular impulse
+    const float4 ang4 = (jab >> 31) ? ld4(jr + JR_ANG) : make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+    const int ang = __float_as_int(ang4.x);
     float lx, ly;
     if (MODE == 0) { lx = jr[JR_ACCX]; ly = jr[JR_ACCY]; }
     else {
@@ -384,8 +391,25 @@ __device__ __forceinline__ void visit_joint(float *sm, uint32_t jab, int j, cons
         ly = __fmaf_rn(i12, rx, i22 * ry);
         *reinterpret_cast<float2 *>(jr + JR_ACCX) = make_float2(acc.x + lx, acc.y + ly);
     }
-    if (dyn_a) st4(sm + SC::BVEL + 4 * a, __fmaf_rn(-ma, lx, vax), __fmaf_rn(-ma, ly, vay), __fmaf_rn(-ia, cross2(rax, ray, lx, ly), wa));
-    if (dyn_b) st4(sm + SC::BVEL + 4 * b, __fmaf_rn(mb, lx, vbx), __fmaf_rn(mb, ly, vby), __fmaf_rn(ib, cross2(rbx, rby, lx, ly), wb));
+    wa = __fmaf_rn(-ia, cross2(rax, ray, lx, ly), wa);
+    wb = __fmaf_rn(ib, cross2(rbx, rby, lx, ly), wb);
+    if (ang != 0) {
+        // angular row after the point row (paper, "Fixed Joints", "Joint Limits"): j_r = (w_a - w_b + correction) / (1/I_a + 1/I_b)
+        float lr;
+        if (MODE == 0) lr = (ang == 1) ? ang4.w : 0.0f;
+        else {
+            const float wrel = wa - wb;
+            float v;
+            if (ang == 1) v = wrel + ang4.z;
+            else if (ang == 2) { v = (wrel < 0.0f) ? wrel : wrel + ang4.z; v = fmax_cmp(v, 0.0f); }
+            else { v = (wrel > 0.0f) ? wrel : wrel + ang4.z; v = fmin_cmp(v, 0.0f); }
+            lr = v * ang4.y;
+            if (ang == 1) jr[JR_ACCR] = ang4.w + lr;
+        }
+        if (MODE == 1 || ang == 1) { wa = __fmaf_rn(-lr, ia, wa); wb = __fmaf_rn(lr, ib, wb); }
+    }
+    if (dyn_a) st4(sm + SC::BVEL + 4 * a, __fmaf_rn(-ma, lx, vax), __fmaf_rn(-ma, ly, vay), wa);
+    if (dyn_b) st4(sm + SC::BVEL + 4 * b, __fmaf_rn(mb, lx, vbx), __fmaf_rn(mb, ly, vby), wb);
 }
 // joints of one level touch disjoint movable bodies; levels in order keep the joint order
 template <class SC, int G, int MODE>
@@ -737,7 +761,7 @@ __device__ __noinline__ uint32_t load_level_consts(uint32_t *smu, const uint32_t
     }
     for (int i = lane; i < SC::C; i += G) smu[SC::RAD + i] = lv[SC::LV_RAD + i];
     for (int i = lane; i < SC::MASKW; i += G) smu[SC::MASK + i] = lv[SC::LV_MASK + i];
-    return (SC::J > 0 && lane < SC::J) ? lv[SC::LV_JOINT + 8 * lane] : 0u;
+    return (SC::J > 0 && lane < SC::J) ? lv[SC::LV_JOINT + kJointLevelWords * lane] : 0u;
 }
 
 // Auto-reset of a finished env: next level (its own, or drawn from the pool by the hash of seed,
@@ -759,7 +783,7 @@ __device__ __noinline__ uint32_t reset_env(uint32_t *smu, const uint32_t *levels
     }
     const uint32_t *lv = levels + (size_t)level * SC::LV_WORDS;
     for (int i = lane; i < 6 * SC::N; i += G) smu[body_word<SC>(i)] = lv[SC::LV_X + i];
-    if (SC::J > 0 && lane < SC::J) { smu[SC::JROW + kJointWords * lane + JR_ACCX] = 0u; smu[SC::JROW + kJointWords * lane + JR_ACCY] = 0u; }
+    if (SC::J > 0 && lane < SC::J) { smu[SC::JROW + kJointWords * lane + JR_ACCX] = 0u; smu[SC::JROW + kJointWords * lane + JR_ACCY] = 0u; smu[SC::JROW + kJointWords * lane + JR_ACCR] = 0u; }
     for (int i = lane; i < (SC::NPAIRS + 3) / 4; i += G) smu[SC::WIDX + i] = 0xffffffffu;
     if (lane == 0) {
         smu[SC::META + META_STEP] = 0u; smu[SC::META + META_EPISODE] = (uint32_t)episode; smu[SC::META + META_LEVEL] = (uint32_t)level;
@@ -1072,10 +1096,12 @@ struct Scene {
         // joint pre-step (poses only; velocities are not read): the row goes to shared memory
         if (SC::J > 0 && lane < SC::J) {
             float *jr = sm + SC::JROW + kJointWords * lane;
-            if (!((jab >> 24) & 1u) || !prm.warm_start) { jr[JR_ACCX] = 0.0f; jr[JR_ACCY] = 0.0f; }
+            if (!((jab >> 24) & 1u) || !prm.warm_start) { jr[JR_ACCX] = 0.0f; jr[JR_ACCY] = 0.0f; jr[JR_ACCR] = 0.0f; }
+            int ang = 0;
+            float kr = 0.0f, bias_r = 0.0f;
             if ((jab >> 24) & 1u) {
                 const int a = jab & 255, b = (jab >> 8) & 255;
-                const uint32_t *jl = lv + SC::LV_JOINT + 8 * lane;
+                const uint32_t *jl = lv + SC::LV_JOINT + kJointLevelWords * lane;
                 float rax, ray, rbx, rby;
                 rot2(sm[SC::BC + a], sm[SC::BS + a], __uint_as_float(jl[1]), __uint_as_float(jl[2]), rax, ray);
                 rot2(sm[SC::BC + b], sm[SC::BS + b], __uint_as_float(jl[3]), __uint_as_float(jl[4]), rbx, rby);
@@ -1093,7 +1119,21 @@ struct Scene {
                 jr[JR_BX] = prm.joint_alpha * gx; jr[JR_BY] = prm.joint_alpha * gy;
                 const float share = prm.joint_beta / msum;
                 jr[JR_CX] = share * gx; jr[JR_CY] = share * gy;
+                // angular row from the relative rotation at the start of the step
+                const float isum = ia + ib;
+                const uint32_t kind = jl[10];
+                if (isum > 0.0f && kind != 0u) {
+                    const float rel = sm[SC::BPOS + 4 * a + 2] - sm[SC::BPOS + 4 * b + 2];
+                    if (kind & 1u) { ang = 1; kr = 1.0f / isum; bias_r = prm.joint_gamma * (rel - __uint_as_float(jl[7])); }
+                    else {
+                        const float lo = __uint_as_float(jl[8]), hi = __uint_as_float(jl[9]);
+                        if (rel > hi) { ang = 2; kr = 1.0f / isum; bias_r = prm.joint_gamma * (rel - hi); }
+                        else if (rel < lo) { ang = 3; kr = 1.0f / isum; bias_r = prm.joint_gamma * (rel - lo); }
+                    }
+                }
             }
+            if (ang != 1) jr[JR_ACCR] = 0.0f;
+            jr[JR_ANG] = __int_as_float(ang); jr[JR_KR] = kr; jr[JR_BIASR] = bias_r;
         }
         g.sync();
 
@@ -1341,8 +1381,9 @@ struct Scene {
         for (int i = lane; i < 6 * SC::N; i += G) smu[body_word<SC>(i)] = __ldcg(st + SC::ST_BODY + i);
         if (lane < 5) smu[SC::META + lane] = __ldcg(st + SC::ST_META + lane);
         if (SC::J > 0 && lane < SC::J) {
-            smu[SC::JROW + kJointWords * lane + JR_ACCX] = __ldcg(st + SC::ST_JACC + 2 * lane);
-            smu[SC::JROW + kJointWords * lane + JR_ACCY] = __ldcg(st + SC::ST_JACC + 2 * lane + 1);
+            smu[SC::JROW + kJointWords * lane + JR_ACCX] = __ldcg(st + SC::ST_JACC + 3 * lane);
+            smu[SC::JROW + kJointWords * lane + JR_ACCY] = __ldcg(st + SC::ST_JACC + 3 * lane + 1);
+            smu[SC::JROW + kJointWords * lane + JR_ACCR] = __ldcg(st + SC::ST_JACC + 3 * lane + 2);
         }
         for (int i = lane; i < (SC::NPAIRS + 3) / 4; i += G) smu[SC::WIDX + i] = 0xffffffffu;
         const int level = (int)__ldcg(st + SC::ST_META + META_LEVEL);
@@ -1379,8 +1420,9 @@ struct Scene {
         // write back
         for (int i = lane; i < 6 * SC::N; i += G) st[SC::ST_BODY + i] = smu[body_word<SC>(i)];
         if (SC::J > 0 && lane < SC::J) {
-            st[SC::ST_JACC + 2 * lane] = smu[SC::JROW + kJointWords * lane + JR_ACCX];
-            st[SC::ST_JACC + 2 * lane + 1] = smu[SC::JROW + kJointWords * lane + JR_ACCY];
+            st[SC::ST_JACC + 3 * lane] = smu[SC::JROW + kJointWords * lane + JR_ACCX];
+            st[SC::ST_JACC + 3 * lane + 1] = smu[SC::JROW + kJointWords * lane + JR_ACCY];
+            st[SC::ST_JACC + 3 * lane + 2] = smu[SC::JROW + kJointWords * lane + JR_ACCR];
         }
         if (lane < 5) st[SC::ST_META + lane] = smu[SC::META + lane];
         const int nw = (int)smu[SC::META + META_NWARM];
@@ -1542,14 +1584,14 @@ __global__ void __launch_bounds__(kObsThreads) k2d_obs_kernel(const uint32_t *st
     float *jrows = img + n_shapes * 29;
     for (int row = lane; row < 2 * n_joints; row += 32) {
         const int j = row >> 1, d = row & 1;
-        const uint32_t *jl = lv + SC::LV_JOINT + 8 * j;
+        const uint32_t *jl = lv + SC::LV_JOINT + kJointLevelWords * j;
         const uint32_t jab = jl[0];
         float *o = jrows + row * jw;
         for (int f = 0; f < jw; ++f) o[f] = 0.0f;
         if ((jab >> 28) & 1u) {
             const int a = jab & 255, b = (jab >> 8) & 255;
             const int from = d ? b : a, to = d ? a : b;
-            o[0] = 1.0f;
+            o[0] = 1.0f; o[1] = (jl[10] & 1u) ? 1.0f : 0.0f;
 #pragma unroll
             for (int f = 2; f < 6; ++f) { const int side = ((f - 2) >> 1) ^ d; o[f] = __uint_as_float(jl[1 + 2 * side + ((f - 2) & 1)]); }
             o[6] = __uint_as_float(jl[6]); o[7] = __uint_as_float(jl[5]);

@@ -29,7 +29,7 @@ class Config(C.Structure):
         [(n, C.c_int32) for n in ("n_envs", "n_polygons", "n_circles", "n_joints", "n_thrusters", "n_actions", "n_levels",
                                   "solver_iters", "warm_start", "auto_reset", "max_episode_steps", "max_fused_steps")] +
         [(n, C.c_float) for n in ("dt", "gravity_y", "contact_alpha", "contact_beta", "slop", "restitution_threshold",
-                                  "face_tol", "joint_alpha", "joint_beta", "motor_rho", "aabb_margin")] +
+                                  "face_tol", "joint_alpha", "joint_beta", "motor_rho", "aabb_margin", "joint_gamma")] +
         [("seed", C.c_uint64), ("env_offset", C.c_int64), ("device", C.c_int32), ("lanes_per_scene", C.c_int32),
          ("cuda_stream", C.c_void_p)])
 
@@ -45,6 +45,8 @@ LEVEL_DTYPE = np.dtype([
     ("joint_anchor_a", np.float32, (MAX_JOINTS, 2)), ("joint_anchor_b", np.float32, (MAX_JOINTS, 2)),
     ("motor_speed", np.float32, (MAX_JOINTS,)), ("motor_power", np.float32, (MAX_JOINTS,)),
     ("motor_binding", np.int32, (MAX_JOINTS,)), ("joint_active", np.int32, (MAX_JOINTS,)),
+    ("joint_fixed", np.int32, (MAX_JOINTS,)), ("joint_limited", np.int32, (MAX_JOINTS,)),
+    ("joint_fixed_angle", np.float32, (MAX_JOINTS,)), ("joint_min", np.float32, (MAX_JOINTS,)), ("joint_max", np.float32, (MAX_JOINTS,)),
     ("thr_shape", np.int32, (MAX_THRUSTERS,)), ("thr_pos", np.float32, (MAX_THRUSTERS, 2)),
     ("thr_rot", np.float32, (MAX_THRUSTERS,)), ("thr_power", np.float32, (MAX_THRUSTERS,)),
     ("thr_binding", np.int32, (MAX_THRUSTERS,)), ("thr_active", np.int32, (MAX_THRUSTERS,)),
@@ -199,7 +201,7 @@ class Env:
         f = raw.view(np.float32)
         o = 0
         out = {}
-        for name, shape in (("pos", (N, 2)), ("angle", (N,)), ("vel", (N, 2)), ("angvel", (N,)), ("acc", (S, 2)), ("jacc", (J, 2))):
+        for name, shape in (("pos", (N, 2)), ("angle", (N,)), ("vel", (N, 2)), ("angvel", (N,)), ("acc", (S, 2)), ("jacc", (J, 3))):
             n = int(np.prod(shape))
             out[name] = f[:, o:o + n].reshape((-1,) + shape).copy()
             o += n

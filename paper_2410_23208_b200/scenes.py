@@ -77,6 +77,8 @@ LEVEL_FIELDS = (
     ("is_static", np.int32), ("role", np.int32), ("active", np.int32),
     ("joint_a", np.int32), ("joint_b", np.int32), ("joint_anchor_a", np.float32), ("joint_anchor_b", np.float32),
     ("motor_speed", np.float32), ("motor_power", np.float32), ("motor_binding", np.int32), ("joint_active", np.int32),
+    ("joint_fixed", np.int32), ("joint_limited", np.int32), ("joint_fixed_angle", np.float32),
+    ("joint_min", np.float32), ("joint_max", np.float32),
     ("thr_shape", np.int32), ("thr_pos", np.float32), ("thr_rot", np.float32), ("thr_power", np.float32),
     ("thr_binding", np.int32), ("thr_active", np.int32),
 )
@@ -92,6 +94,7 @@ def empty_levels(dims: SceneDims, n_levels: int) -> dict:
         "is_static": (N,), "role": (N,), "active": (N,),
         "joint_a": (J,), "joint_b": (J,), "joint_anchor_a": (J, 2), "joint_anchor_b": (J, 2),
         "motor_speed": (J,), "motor_power": (J,), "motor_binding": (J,), "joint_active": (J,),
+        "joint_fixed": (J,), "joint_limited": (J,), "joint_fixed_angle": (J,), "joint_min": (J,), "joint_max": (J,),
         "thr_shape": (T,), "thr_pos": (T, 2), "thr_rot": (T,), "thr_power": (T,),
         "thr_binding": (T,), "thr_active": (T,),
     }
@@ -133,7 +136,8 @@ def _rot(c: float, s: float, v):
     return (c * v[0] - s * v[1], s * v[0] + c * v[1])
 
 
-def _one_level(dims: SceneDims, seed: int, index: int, static_prob: float, with_red, triangle_prob: float, out: dict):
+def _one_level(dims: SceneDims, seed: int, index: int, static_prob: float, with_red, triangle_prob: float, out: dict,
+               fixed_prob: float = 0.0, limit_prob: float = 0.0):
     P, C, N, J, T = dims.n_polygons, dims.n_circles, dims.n_shapes, dims.n_joints, dims.n_thrusters
     d = _Draws(seed, index)
     verts = [None] * P
@@ -285,6 +289,22 @@ def _one_level(dims: SceneDims, seed: int, index: int, static_prob: float, with_
         o["motor_power"][index, j] = d.u(0.1, 0.8) / inv_i
         o["motor_binding"][index, j] = j
         o["joint_active"][index, j] = 1
+    if fixed_prob > 0.0 or limit_prob > 0.0:
+        # joint kinds come from a stream of their own, so that levels drawn without them do not change:
+        # a fixed joint holds the relative rotation the level starts with, a limited one allows a
+        # range of 0.2 .. 1 rad to either side of it
+        dj = _Draws(seed ^ 0x51F1, index)
+        for j, ch in enumerate(children):
+            rel0 = ang[partner[ch]] - ang[ch]
+            u = dj.u()
+            lo, hi = dj.u(0.2, 1.0), dj.u(0.2, 1.0)
+            if u < fixed_prob:
+                o["joint_fixed"][index, j] = 1
+                o["joint_fixed_angle"][index, j] = rel0
+            elif u < fixed_prob + limit_prob:
+                o["joint_limited"][index, j] = 1
+                o["joint_min"][index, j] = rel0 - lo
+                o["joint_max"][index, j] = rel0 + hi
     movable = [k for k in range(1, N) if not static[k]] or list(range(1, N))
     for t in range(T):
         k = movable[d.integer(0, len(movable))]
@@ -298,10 +318,12 @@ def _one_level(dims: SceneDims, seed: int, index: int, static_prob: float, with_
 
 
 def make_levels(size, n_levels: int, seed: int, static_prob: float = 0.0, with_red=None,
-                triangle_prob: float = 0.0) -> dict:
+                triangle_prob: float = 0.0, fixed_prob: float = 0.0, limit_prob: float = 0.0) -> dict:
     """Draw ``n_levels`` scenes of size class ``size`` ("S", "M", "L" or a SceneDims).
 
     ``with_red``: True / False, or a probability; default is always for L and 1/2 otherwise.
+    ``fixed_prob`` / ``limit_prob``: probability that a joint is a fixed joint / a revolute joint with
+    rotation limits (the benchmark workloads use neither).
     Level ``k`` depends only on ``(seed, k)`` and the other arguments, not on ``n_levels``.
     """
     dims = SIZES[size] if isinstance(size, str) else size
@@ -309,7 +331,7 @@ def make_levels(size, n_levels: int, seed: int, static_prob: float = 0.0, with_r
         with_red = True if dims == SIZES["L"] else 0.5
     out = empty_levels(dims, n_levels)
     for k in range(n_levels):
-        _one_level(dims, seed, k, static_prob, with_red, triangle_prob, out)
+        _one_level(dims, seed, k, static_prob, with_red, triangle_prob, out, fixed_prob, limit_prob)
     return out
 
 
@@ -348,7 +370,8 @@ def custom_level(dims: SceneDims, polygons=(), circles=(), joints=(), thrusters=
     origin), plus optional pos, angle, vel, angvel, density, friction, restitution, static, role.
     circles: dicts with ``radius`` and the same optional keys.  Shape indices: polygons first, in the
     order given, then circles at ``dims.n_polygons + k``.
-    joints: dicts with a, b, anchor_a, anchor_b and optional speed, power, binding.
+    joints: dicts with a, b, anchor_a, anchor_b and optional speed, power, binding, fixed (the relative
+    rotation angle_a - angle_b a fixed joint holds), limits ((min, max) of that relative rotation).
     thrusters: dicts with shape and optional pos, rot, power, binding.
     """
     lv = empty_levels(dims, 1)
@@ -385,6 +408,12 @@ def custom_level(dims: SceneDims, polygons=(), circles=(), joints=(), thrusters=
         lv["motor_power"][0, j] = d.get("power", 0.0)
         lv["motor_binding"][0, j] = d.get("binding", j)
         lv["joint_active"][0, j] = 1
+        if "fixed" in d:
+            lv["joint_fixed"][0, j] = 1
+            lv["joint_fixed_angle"][0, j] = d["fixed"]
+        if "limits" in d:
+            lv["joint_limited"][0, j] = 1
+            lv["joint_min"][0, j], lv["joint_max"][0, j] = d["limits"]
     for t, d in enumerate(thrusters):
         lv["thr_shape"][0, t] = d["shape"]
         lv["thr_pos"][0, t] = d.get("pos", (0.0, 0.0))

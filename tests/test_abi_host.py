@@ -24,9 +24,9 @@ def test_library_exports_every_declared_symbol():
 
 def test_struct_layouts_match_the_header():
     # sizes computed from the header's field lists
-    assert C.sizeof(k2d.Config) == 12 * 4 + 11 * 4 + 4 + 8 + 8 + 4 + 4 + 8
-    n_float = 12 * 4 * 2 + 4 + 16 * 2 + 16 + 16 * 2 + 16 + 3 * 16 + 6 * 2 * 2 + 6 * 2 + 2 * 2 + 2 + 2
-    n_int = 12 + 3 * 16 + 2 * 6 + 2 * 6 + 2 + 2 * 2
+    assert C.sizeof(k2d.Config) == 12 * 4 + 12 * 4 + 8 + 8 + 4 + 4 + 8
+    n_float = 12 * 4 * 2 + 4 + 16 * 2 + 16 + 16 * 2 + 16 + 3 * 16 + 6 * 2 * 2 + 6 * 2 + 6 * 3 + 2 * 2 + 2 + 2
+    n_int = 12 + 3 * 16 + 2 * 6 + 2 * 6 + 2 * 6 + 2 + 2 * 2
     assert k2d.LEVEL_DTYPE.itemsize == 4 * (n_float + n_int)
 
 
@@ -37,7 +37,7 @@ def test_sizes_and_defaults():
     assert (cfg.n_actions, cfg.solver_iters, cfg.warm_start) == (8, 8, 1)
     assert cfg.dt == pytest.approx(1 / 60) and cfg.gravity_y == pytest.approx(-9.81)
     assert lib.k2d_obs_floats(C.byref(cfg)) == 704
-    assert lib.k2d_canonical_words(C.byref(cfg)) == 6 * 16 + 2 * 186 + 12 + 4
+    assert lib.k2d_canonical_words(C.byref(cfg)) == 6 * 16 + 2 * 186 + 18 + 4
     sb = lib.k2d_state_bytes(C.byref(cfg))
     assert sb > 16384 * 6 * 16 * 4 and sb % 256 == 0
     for dims, width in (((5, 2, 1, 1), 235), ((6, 3, 2, 2), 333)):

@@ -211,3 +211,42 @@ def test_step_rejects_too_many_fused_steps():
     act = torch.zeros((5, 4, env.n_actions), device="cuda")
     with pytest.raises(k2d.K2DError):
         env.step(act)
+
+
+@pytest.mark.parametrize("size,lanes", [("L", 16), ("L", 32), ("M", 8), ("S", 16)])
+def test_fixed_joints_and_joint_limits_match_the_oracle(size, lanes):
+    # a third of the joints fixed, a third with rotation limits; motors push the limited ones against their stops
+    n_envs = 96
+    lv = scenes.make_levels(size, n_envs, 71, static_prob=0.1, triangle_prob=0.2, fixed_prob=0.34, limit_prob=0.33)
+    assert lv["joint_fixed"].sum() > 0 and lv["joint_limited"].sum() > 0
+    env, ref = parity.make_pair(lv, n_envs, lanes_per_scene=lanes, max_fused_steps=128)
+    act = scenes.make_actions(120, n_envs, env.n_actions, 71)
+    (r, d), (rr, dr) = parity.step_both(env, ref, act[:1])
+    err, exact = parity.errors(env, ref)
+    _check_tolerances(err, 1)
+    assert exact, err
+    (r, d), (rr, dr) = parity.step_both(env, ref, act[1:], chunk=17)
+    err, exact = parity.errors(env, ref)
+    _check_tolerances(err, 120)
+    assert exact, err
+    assert np.array_equal(r, rr) and np.array_equal(d, dr)
+    assert np.abs(ref.jacc[:, :, 2]).max() > 0                    # fixed joints carry accumulated angular impulses
+    assert np.array_equal(env.obs().cpu().numpy().view(np.uint32), ref.obs().view(np.uint32))
+
+
+def test_joint_kinds_with_auto_reset_and_checkpoint():
+    lv = scenes.make_levels("L", 32, 72, static_prob=0.1, fixed_prob=0.5, limit_prob=0.5)
+    env, ref = parity.make_pair(lv, 64, auto_reset=2, max_episode_steps=7, seed=3, joint_gamma=3.0)
+    act = scenes.make_actions(40, 64, env.n_actions, 72)
+    (r, d), (rr, dr) = parity.step_both(env, ref, act[:20], chunk=5)
+    st = env.get_state()
+    env2 = k2d.Env(lv, 64, auto_reset=2, max_episode_steps=7, seed=3, joint_gamma=3.0)
+    env2.set_state(st)
+    parity.step_both(env, ref, act[20:], chunk=20)
+    import torch
+    env2.step(torch.from_numpy(act[20:]).cuda())
+    err, exact = parity.errors(env, ref)
+    assert exact, err
+    sa, sb = env.get_state(), env2.get_state()
+    for k in sa:
+        assert np.array_equal(sa[k], sb[k], equal_nan=True), k
