@@ -345,6 +345,32 @@ __device__ __forceinline__ void correct_pair(float *pos, int a, int b, unsigned 
     if (dyn_b) { pos[4 * b] = xb; pos[4 * b + 1] = yb; }
 }
 
+// ---- angular row of a fixed joint or of a revolute joint beyond one of its limits (paper, "Fixed Joints",
+// "Joint Limits"): j_r = (w_a - w_b + correction) / (1/I_a + 1/I_b), a loses j_r / I_a, b gains j_r / I_b.  A fixed
+// joint's impulse is accumulated and warm-started; a limit only ever pushes back, applies no correction while the
+// joint is already returning, and is not accumulated.  Returns the two angular velocities.  Out of line: most
+// joints are plain revolute joints.
+template <int MODE>
+__device__ __noinline__ float2 angular_row(float *jr, float ia, float ib, float wa, float wb) {
+    const float4 ang4 = ld4(jr + JR_ANG);      // kind this step, inverse angular mass, correction, accumulated impulse
+    const int ang = __float_as_int(ang4.x);
+    if (ang == 0) return make_float2(wa, wb);
+    float lr;
+    if (MODE == 0) {
+        if (ang != 1) return make_float2(wa, wb);
+        lr = ang4.w;
+    } else {
+        const float wrel = wa - wb;
+        float v;
+        if (ang == 1) v = wrel + ang4.z;
+        else if (ang == 2) { v = (wrel < 0.0f) ? wrel : wrel + ang4.z; v = fmax_cmp(v, 0.0f); }
+        else { v = (wrel > 0.0f) ? wrel : wrel + ang4.z; v = fmin_cmp(v, 0.0f); }
+        lr = v * ang4.y;
+        if (ang == 1) jr[JR_ACCR] = ang4.w + lr;
+    }
+    return make_float2(__fmaf_rn(-lr, ia, wa), __fmaf_rn(lr, ib, wb));
+}
+
 // ---- joints; the row of joint j is in shared memory.  MODE 0: warm start, 1: solver iteration,
 // 2: positional correction, 3: motor
 template <class SC, int MODE>
@@ -374,10 +400,6 @@ __device__ __forceinline__ void visit_joint(float *sm, uint32_t jab, int j, cons
     const float rax = r4.x, ray = r4.y, rbx = r4.z, rby = r4.w;
     const float4 va4 = ld4(sm + SC::BVEL + 4 * a), vb4 = ld4(sm + SC::BVEL + 4 * b);
     float vax = va4.x, vay = va4.y, wa = va4.z, vbx = vb4.x, vby = vb4.y, wb = vb4.z;
-    // angular row of a fixed or limited joint (bit 31 of the packed word): kind this step, inverse angular mass,
-    // correction, accumulated angular impulse
-    const float4 ang4 = (jab >> 31) ? ld4(jr + JR_ANG) : make_float4(0.0f, 0.0f, 0.0f, 0.0f);
-    const int ang = __float_as_int(ang4.x);
     float lx, ly;
     if (MODE == 0) { lx = jr[JR_ACCX]; ly = jr[JR_ACCY]; }
     else {
@@ -393,20 +415,9 @@ __device__ __forceinline__ void visit_joint(float *sm, uint32_t jab, int j, cons
     }
     wa = __fmaf_rn(-ia, cross2(rax, ray, lx, ly), wa);
     wb = __fmaf_rn(ib, cross2(rbx, rby, lx, ly), wb);
-    if (ang != 0) {
-        // angular row after the point row (paper, "Fixed Joints", "Joint Limits"): j_r = (w_a - w_b + correction) / (1/I_a + 1/I_b)
-        float lr;
-        if (MODE == 0) lr = (ang == 1) ? ang4.w : 0.0f;
-        else {
-            const float wrel = wa - wb;
-            float v;
-            if (ang == 1) v = wrel + ang4.z;
-            else if (ang == 2) { v = (wrel < 0.0f) ? wrel : wrel + ang4.z; v = fmax_cmp(v, 0.0f); }
-            else { v = (wrel > 0.0f) ? wrel : wrel + ang4.z; v = fmin_cmp(v, 0.0f); }
-            lr = v * ang4.y;
-            if (ang == 1) jr[JR_ACCR] = ang4.w + lr;
-        }
-        if (MODE == 1 || ang == 1) { wa = __fmaf_rn(-lr, ia, wa); wb = __fmaf_rn(lr, ib, wb); }
+    if (jab >> 31) {      // fixed or limited joint: its angular row follows the point row
+        const float2 w2 = angular_row<MODE>(jr, ia, ib, wa, wb);
+        wa = w2.x; wb = w2.y;
     }
     if (dyn_a) st4(sm + SC::BVEL + 4 * a, __fmaf_rn(-ma, lx, vax), __fmaf_rn(-ma, ly, vay), wa);
     if (dyn_b) st4(sm + SC::BVEL + 4 * b, __fmaf_rn(mb, lx, vbx), __fmaf_rn(mb, ly, vby), wb);
