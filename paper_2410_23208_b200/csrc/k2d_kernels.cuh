@@ -65,7 +65,7 @@ struct SizeClass {
     static constexpr int BPOS = 0, BVEL = 4 * N;
     static constexpr int BIM = 8 * N, BII = 9 * N, BFR = 10 * N, BRE = 11 * N, BC = 12 * N, BS = 13 * N, BFL = 14 * N;
     static constexpr int RAD = 15 * N;
-    static constexpr int WVX = RAD + C, WVY = WVX + P4, WNX = WVY + P4, WNY = WNX + P4, WOFF = WNY + P4;
+    static constexpr int WVX = (RAD + C + 3) / 4 * 4, WVY = WVX + P4, WNX = WVY + P4, WNY = WNX + P4, WOFF = WNY + P4;
     static constexpr int BOX = (WOFF + P4 + 3) / 4 * 4;  // N x (min x, min y, max x, max y), 16-byte aligned
     static constexpr int MASK = BOX + 4 * N;
     static constexpr int ACT = MASK + MASKW;
@@ -863,34 +863,33 @@ struct Scene {
     }
 
     // ---- narrowphase: polygon a against polygon b (world data in shared memory)
-    __device__ __forceinline__ void max_separation(int x, int cntx, const float (&yx)[4], const float (&yy)[4], int cnty,
-                                                   float &best, int &edge) const {
-        best = 0.0f; edge = 0;
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            if (i < cntx) {
-                float nx = sm[SC::WNX + 4 * x + i], ny = sm[SC::WNY + 4 * x + i];
-                float lo = dot2(nx, ny, yx[0], yy[0]);
-#pragma unroll
-                for (int j = 1; j < 4; ++j)
-                    if (j < cnty) lo = fmin_cmp(lo, dot2(nx, ny, yx[j], yy[j]));
-                float sep = lo - sm[SC::WOFF + 4 * x + i];
-                if (i == 0 || sep > best) { best = sep; edge = i; }
-            }
-        }
-    }
-
     __device__ unsigned manifold_pp(int a, int b, Manifold (&m)[2]) const {
         const int cnta = flag_nverts(smu[SC::BFL + a]), cntb = flag_nverts(smu[SC::BFL + b]);
-        float ax[4], ay[4], bx[4], by[4];
+        // largest separation of the other polygon's vertices along each polygon's face normals, first face on ties
+        float sa = 0.0f, sb = 0.0f; int ea = 0, eb = 0;
+#pragma unroll 1
+        for (int side = 0; side < 2; ++side) {
+            const int x = side ? b : a, y = side ? a : b;
+            const int cntx = side ? cntb : cnta, cnty = side ? cnta : cntb;
+            const float4 nx4 = ld4(sm + SC::WNX + 4 * x), ny4 = ld4(sm + SC::WNY + 4 * x), off4 = ld4(sm + SC::WOFF + 4 * x);
+            const float4 yx4 = ld4(sm + SC::WVX + 4 * y), yy4 = ld4(sm + SC::WVY + 4 * y);
+            const float nxs[4] = { nx4.x, nx4.y, nx4.z, nx4.w }, nys[4] = { ny4.x, ny4.y, ny4.z, ny4.w };
+            const float offs[4] = { off4.x, off4.y, off4.z, off4.w };
+            const float yx[4] = { yx4.x, yx4.y, yx4.z, yx4.w }, yy[4] = { yy4.x, yy4.y, yy4.z, yy4.w };
+            float best = 0.0f; int edge = 0;
 #pragma unroll
-        for (int k = 0; k < 4; ++k) {
-            ax[k] = sm[SC::WVX + 4 * a + k]; ay[k] = sm[SC::WVY + 4 * a + k];
-            bx[k] = sm[SC::WVX + 4 * b + k]; by[k] = sm[SC::WVY + 4 * b + k];
+            for (int i = 0; i < 4; ++i) {
+                if (i < cntx) {
+                    float lo = dot2(nxs[i], nys[i], yx[0], yy[0]);
+#pragma unroll
+                    for (int j = 1; j < 4; ++j)
+                        if (j < cnty) lo = fmin_cmp(lo, dot2(nxs[i], nys[i], yx[j], yy[j]));
+                    const float sep = lo - offs[i];
+                    if (i == 0 || sep > best) { best = sep; edge = i; }
+                }
+            }
+            if (side == 0) { sa = best; ea = edge; } else { sb = best; eb = edge; }
         }
-        float sa, sb; int ea, eb;
-        max_separation(a, cnta, bx, by, cntb, sa, ea);
-        max_separation(b, cntb, ax, ay, cnta, sb, eb);
         if (sa > 0.0f || sb > 0.0f) return 0u;
         const bool ref_b = sb > sa + prm.face_tol;
         const int R = ref_b ? b : a, I = ref_b ? a : b;
