@@ -91,6 +91,7 @@ typedef struct k2d_config {
     float motor_rho;               /* rho of the motor law j = p tanh((wa - wb - s A) rho)      */
     float aabb_margin;             /* bounding boxes further apart than this skip narrowphase   */
     float joint_gamma;             /* angular correction of fixed joints and joint limits: gamma * angle error */
+    float dense_kappa;             /* dense reward kappa * (d_t - d_t+1), d = green-blue distance; 0 = off */
     uint64_t seed;                 /* seed of the K2D_RESET_POOL hash                           */
     int64_t env_offset;            /* global index of env 0 (sharding over several GPUs)        */
     int32_t device;                /* CUDA device ordinal                                       */
@@ -150,9 +151,17 @@ int k2d_reset(k2d_state *s, const int32_t *host_level_ids);
 /* Advances every env by n_steps steps (paper, Algorithm 1 + "Reward").  dev_actions is
  * [n_steps][n_envs][n_actions] floats, one row consumed per step (motor actions are clipped
  * to [-1, 1], thruster actions to [0, 1]: paper, "Action Space"); dev_reward [n_steps][n_envs]
- * floats in {-1, 0, +1}; dev_done [n_steps][n_envs] bytes.  1 <= n_steps <= max_fused_steps.
+ * floats in {-1, 0, +1}, plus, if dense_kappa is not 0, the paper's auxiliary dense reward
+ * kappa * (d_t - d_t+1) with d the distance between the positions of the first green and the
+ * first blue shape before and after the step; dev_done [n_steps][n_envs] bytes.  1 <= n_steps <= max_fused_steps.
  * The whole call is one kernel launch; scene state stays on chip between the fused steps. */
 int k2d_step(k2d_state *s, const float *dev_actions, int32_t n_steps, float *dev_reward, uint8_t *dev_done);
+
+/* The same step with the paper's multi-discrete action space ("Action Space": every motor and
+ * thruster is inactive or at maximum power, motors forwards or backwards): dev_actions is
+ * [n_steps][n_envs][n_actions] int32 codes; a motor reads 0 = off, 1 = forwards (+1), 2 = backwards
+ * (-1), anything else off; a thruster reads 0 = off, anything else on. */
+int k2d_step_discrete(k2d_state *s, const int32_t *dev_actions, int32_t n_steps, float *dev_reward, uint8_t *dev_done);
 
 /* The paper has no counterpart of this call; it exists for one kind of user of this library.
  * k2d_step keeps the contact records of a very crowded scene (far more touching pairs than

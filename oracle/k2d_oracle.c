@@ -59,9 +59,9 @@ typedef struct { real x, y; } vec2;
 /* ---- configuration and raw level description (filled by the caller) ---- */
 typedef struct {
     int32_t n_polygons, n_circles, n_joints, n_thrusters, n_actions, n_levels, n_envs;
-    int32_t solver_iters, warm_start, auto_reset, max_episode_steps, broadphase;
+    int32_t solver_iters, warm_start, auto_reset, max_episode_steps, broadphase, discrete_actions;
     real dt, gravity_y, contact_alpha, contact_beta, slop, restitution_threshold, face_tol;
-    real joint_alpha, joint_beta, motor_rho, aabb_margin, joint_gamma;
+    real joint_alpha, joint_beta, motor_rho, aabb_margin, joint_gamma, dense_kappa;
     uint64_t seed;
     int64_t env_offset;
 } ref_config;
@@ -616,6 +616,17 @@ static void step_env(ref_sim *S, int e, const real *act, real *out_reward, uint8
     const uint8_t *collide = S->lv_collide + (size_t)l * S->n_pairs;
     const real dt = cf->dt;
 
+    /* distance between the first green and the first blue shape before the step (dense reward) */
+    int dense_g = -1, dense_b = -1;
+    real dense_d0 = RC(0);
+    if (cf->dense_kappa != RC(0)) {
+        for (int i = N - 1; i >= 0; --i) if (active[i]) { if (role[i] == ROLE_GREEN) dense_g = i; if (role[i] == ROLE_BLUE) dense_b = i; }
+        if (dense_g >= 0 && dense_b >= 0) {
+            vec2 dd = { pos[2 * dense_b] - pos[2 * dense_g], pos[2 * dense_b + 1] - pos[2 * dense_g + 1] };
+            dense_d0 = R_SQRT(dot2(dd, dd));
+        }
+    }
+
     /* Alg. 1 line 2: gravity on movable shapes */
     const real gdt = cf->gravity_y * dt;
     for (int i = 0; i < N; ++i)
@@ -691,7 +702,9 @@ static void step_env(ref_sim *S, int e, const real *act, real *out_reward, uint8
     for (int j = 0; j < J; ++j) {
         int a = S->lv_joint_a[l * J + j], b = S->lv_joint_b[l * J + j];
         if (!(S->lv_joint_active[l * J + j] && active[a] && active[b] && (inv_mass[a] + inv_mass[b] > RC(0)))) continue;
-        real A = rmax(rmin(act[S->lv_motor_binding[l * J + j]], RC(1)), RC(-1));
+        /* "Action Space": continuous in [-1, 1]; multi-discrete 0 = off, 1 = forwards, 2 = backwards at full power */
+        real av = act[S->lv_motor_binding[l * J + j]];
+        real A = cf->discrete_actions ? (av == RC(1) ? RC(1) : (av == RC(2) ? RC(-1) : RC(0))) : rmax(rmin(av, RC(1)), RC(-1));
         real d = angvel[a] - angvel[b];
         real arg = R_FMA(-S->lv_motor_speed[l * J + j], A, d) * cf->motor_rho;
         real jr = S->lv_motor_power[l * J + j] * k2d_ref_tanh(arg);
@@ -704,7 +717,9 @@ static void step_env(ref_sim *S, int e, const real *act, real *out_reward, uint8
         if (!S->lv_thr_active[l * T + t]) continue;
         int i = S->lv_thr_shape[l * T + t];
         if (!active[i]) continue;
-        real A = rmax(rmin(act[S->lv_thr_binding[l * T + t]], RC(1)), RC(0));
+        /* continuous in [0, 1]; multi-discrete 0 = off, anything else = full power */
+        real tv = act[S->lv_thr_binding[l * T + t]];
+        real A = cf->discrete_actions ? (tv != RC(0) ? RC(1) : RC(0)) : rmax(rmin(tv, RC(1)), RC(0));
         vec2 ld = { S->lv_thr_dir[(size_t)(l * T + t) * 2], S->lv_thr_dir[(size_t)(l * T + t) * 2 + 1] };
         vec2 lp = { S->lv_thr_pos[(size_t)(l * T + t) * 2], S->lv_thr_pos[(size_t)(l * T + t) * 2 + 1] };
         vec2 dir = rot2(cs[i], sn[i], ld), r = rot2(cs[i], sn[i], lp);
@@ -912,6 +927,13 @@ static void step_env(ref_sim *S, int e, const real *act, real *out_reward, uint8
     S->step_count[e] += 1;
     int timeout = cf->max_episode_steps > 0 && S->step_count[e] >= cf->max_episode_steps;
     real reward = (real)(touch_gb - touch_gr);
+    /* "Reward": auxiliary dense signal kappa (d_t - d_{t+1}), d = distance between the green and the blue shape
+     * (the first of each by index), before and after this step */
+    if (cf->dense_kappa != RC(0) && dense_g >= 0 && dense_b >= 0) {
+        vec2 dd = { pos[2 * dense_b] - pos[2 * dense_g], pos[2 * dense_b + 1] - pos[2 * dense_g + 1] };
+        real d1 = R_SQRT(dot2(dd, dd));
+        reward = reward + cf->dense_kappa * (dense_d0 - d1);
+    }
     int done = touch_gb || touch_gr || timeout;
     if (!finite) { reward = RC(0); done = 1; S->status[e] |= STATUS_NONFINITE; cnt[0] += 1; }
     *out_reward = reward; *out_done = (uint8_t)done;

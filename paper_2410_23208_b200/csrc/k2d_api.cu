@@ -28,7 +28,7 @@ constexpr int kChunkSteps = K2D_CHUNK_STEPS;       // steps per work item when t
 struct ClassInfo {
     int id, P, C, N, J, T, NPP, NPC, NCC, NPAIRS, NSLOTS, MASKW;
     int LV_WORDS, ST_WORDS, SCRATCH_WORDS, PTAB_WORDS;
-    int LV_X, LV_IM, LV_II, LV_FR, LV_RE, LV_FLAGS, LV_DENS, LV_RAD, LV_PVX, LV_PVY, LV_PNX, LV_PNY, LV_ELEN, LV_JOINT, LV_THR, LV_MASK;
+    int LV_X, LV_IM, LV_II, LV_FR, LV_RE, LV_FLAGS, LV_DENS, LV_RAD, LV_PVX, LV_PVY, LV_PNX, LV_PNY, LV_ELEN, LV_JOINT, LV_THR, LV_MASK, LV_GB;
     int ST_JACC, ST_META, ST_WARM;
 };
 template <class SC>
@@ -39,7 +39,7 @@ static ClassInfo make_info(int id) {
     c.LV_WORDS = SC::LV_WORDS; c.ST_WORDS = SC::ST_WORDS; c.SCRATCH_WORDS = SC::SCRATCH_WORDS; c.PTAB_WORDS = SC::PTAB_WORDS;
     c.LV_X = SC::LV_X; c.LV_IM = SC::LV_IM; c.LV_II = SC::LV_II; c.LV_FR = SC::LV_FR; c.LV_RE = SC::LV_RE; c.LV_FLAGS = SC::LV_FLAGS;
     c.LV_DENS = SC::LV_DENS; c.LV_RAD = SC::LV_RAD; c.LV_PVX = SC::LV_PVX; c.LV_PVY = SC::LV_PVY; c.LV_PNX = SC::LV_PNX; c.LV_PNY = SC::LV_PNY;
-    c.LV_ELEN = SC::LV_ELEN; c.LV_JOINT = SC::LV_JOINT; c.LV_THR = SC::LV_THR; c.LV_MASK = SC::LV_MASK;
+    c.LV_ELEN = SC::LV_ELEN; c.LV_JOINT = SC::LV_JOINT; c.LV_THR = SC::LV_THR; c.LV_MASK = SC::LV_MASK; c.LV_GB = SC::LV_GB;
     c.ST_JACC = SC::ST_JACC; c.ST_META = SC::ST_META; c.ST_WARM = SC::ST_WARM;
     return c;
 }
@@ -61,7 +61,7 @@ static int check_config(const k2d_config *c) {
         !(c->lanes_per_scene == 0 || c->lanes_per_scene == 8 || c->lanes_per_scene == 16 || c->lanes_per_scene == 32))
         return K2D_ERR_CONFIG;
     const float f[] = { c->dt, c->gravity_y, c->contact_alpha, c->contact_beta, c->slop, c->restitution_threshold, c->face_tol,
-                        c->joint_alpha, c->joint_beta, c->motor_rho, c->aabb_margin, c->joint_gamma };
+                        c->joint_alpha, c->joint_beta, c->motor_rho, c->aabb_margin, c->joint_gamma, c->dense_kappa };
     for (float v : f) if (!std::isfinite(v)) return K2D_ERR_CONFIG;
     if (!(c->dt > 0.0f) || c->aabb_margin < 0.0f || c->slop < 0.0f) return K2D_ERR_CONFIG;
     return K2D_OK;
@@ -186,6 +186,17 @@ static int pack_level(const k2d_config *cfg, const ClassInfo &ci, const k2d_leve
         w[ci.LV_FR + q] = f2u(L->friction[i]); w[ci.LV_RE + q] = f2u(L->restitution[i]); w[ci.LV_DENS + q] = f2u(L->density[i]);
         w[ci.LV_FLAGS + q] = F_ACTIVE | (st ? 0u : F_DYNAMIC) | ((uint32_t)L->role[i] << 2) | (nv << 4);
     }
+    // the dense reward measures the distance between the first green and the first blue shape
+    {
+        int g = -1, b = -1;
+        for (int q = ci.N - 1; q >= 0; --q) {
+            if (!is_active[q]) continue;
+            const uint32_t role = flag_role(w[ci.LV_FLAGS + q]);
+            if (role == K2D_ROLE_GREEN) g = q;
+            if (role == K2D_ROLE_BLUE) b = q;
+        }
+        w[ci.LV_GB] = (g >= 0 && b >= 0) ? ((uint32_t)g | ((uint32_t)b << 8) | (1u << 16)) : 0u;
+    }
     // joints: "on" when both shapes exist and at least one can move; level = 1 + highest level of an earlier
     // joint sharing a movable shape (so lanes can run a level's joints at once and keep the joint order)
     std::vector<int> body_level(ci.N, 0);
@@ -286,12 +297,13 @@ static cudaError_t launch_obs(const k2d_state *s, float *dev_obs) {
 // Kernel arguments of one k2d_step launch.  With more envs than resident scene groups the launch is cut
 // into chunks of kChunkSteps steps, so that the groups can balance the work between them.
 static StepParams step_params(const k2d_state *s, const float *dev_actions, int n_steps, float *dev_reward, uint8_t *dev_done,
-                              uint32_t *scratch) {
+                              uint32_t *scratch, int discrete = 0) {
     const k2d_config &c = s->cfg;
     StepParams prm{};
     prm.state = s->dev_env; prm.levels = s->dev_levels; prm.actions = dev_actions; prm.reward = dev_reward; prm.done = dev_done;
     prm.counters = s->dev_counters; prm.queue = s->dev_queue; prm.chunks_done = s->dev_chunks; prm.scratch = scratch; prm.trace = s->dev_trace;
     prm.n_envs = c.n_envs; prm.n_steps = n_steps; prm.n_actions = c.n_actions; prm.n_levels = c.n_levels;
+    prm.discrete = discrete; prm.dense_kappa = c.dense_kappa;
     prm.chunk_steps = n_steps; prm.n_chunks = 1;
     if (c.n_envs > s->groups && n_steps > kChunkSteps) {
         const int n_chunks = (n_steps + kChunkSteps - 1) / kChunkSteps;
@@ -584,6 +596,15 @@ int k2d_eval_sincos_tanh(const float *dev_x, int32_t n, float *dev_cos, float *d
 static __device__ __align__(256) uint32_t k2d_static_scratch[(size_t)K2D_STATIC_SCRATCH_MAX_ENVS * ClassL::SCRATCH_WORDS];
 static std::mutex k2d_static_mutex;
 static uint32_t *k2d_static_ptr[64];     // device address of the array on each device, filled on first use
+
+int k2d_step_discrete(k2d_state *s, const int32_t *dev_actions, int32_t n_steps, float *dev_reward, uint8_t *dev_done) {
+    if (!s || !dev_actions || !dev_reward || !dev_done) return K2D_ERR_NULL;
+    if (n_steps < 1 || n_steps > s->cfg.max_fused_steps) return K2D_ERR_STEPS;
+    if (((uintptr_t)dev_actions & 3) || ((uintptr_t)dev_reward & 3)) return K2D_ERR_ALIGN;
+    const StepParams prm = step_params(s, reinterpret_cast<const float *>(dev_actions), n_steps, dev_reward, dev_done, s->dev_scratch, 1);
+    CUDA_OK(K2D_DISPATCH(launch_step, s, s, prm));
+    return K2D_OK;
+}
 
 int k2d_step_static_scratch(k2d_state *s, const float *dev_actions, int32_t n_steps, float *dev_reward, uint8_t *dev_done) {
     if (!s || !dev_actions || !dev_reward || !dev_done) return K2D_ERR_NULL;

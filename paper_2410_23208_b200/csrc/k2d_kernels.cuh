@@ -52,7 +52,8 @@ struct SizeClass {
     static constexpr int LV_JOINT = LV_ELEN + P4;
     static constexpr int LV_THR = LV_JOINT + kJointLevelWords * J;      // T x 8: packed, pos xy, dir xy, power, pad, pad
     static constexpr int LV_MASK = LV_THR + 8 * T;
-    static constexpr int LV_WORDS = (LV_MASK + MASKW + 3) / 4 * 4;
+    static constexpr int LV_GB = LV_MASK + MASKW;        // first green shape | first blue shape << 8 | both exist << 16
+    static constexpr int LV_WORDS = (LV_GB + 1 + 3) / 4 * 4;
     // state record: bodies (same order as shared memory), joint impulses, meta, warm list
     static constexpr int ST_BODY = 0, ST_JACC = 6 * N, ST_META = ST_JACC + 3 * J, ST_WARM = ST_META + 8;
     static constexpr int ST_WORDS = (ST_WARM + kWarmWords * NPAIRS + 3) / 4 * 4;
@@ -103,7 +104,7 @@ enum { JR_RAX = 0, JR_RAY, JR_RBX, JR_RBY, JR_I11, JR_I12, JR_I22, JR_PAD0, JR_B
        JR_ACCX, JR_ACCY, JR_PAD1, JR_PAD2,
        JR_ANG, JR_KR, JR_BIASR, JR_ACCR };   // angular row: kind (0 none, 1 fixed, 2 beyond the upper limit, 3 beyond the lower), 1 / (1/I_a + 1/I_b), gamma x error, accumulated
 static_assert(JR_ACCR + 1 == kJointWords, "joint row size");
-enum { META_STEP = 0, META_EPISODE, META_LEVEL, META_STATUS, META_NWARM };
+enum { META_STEP = 0, META_EPISODE, META_LEVEL, META_STATUS, META_NWARM, META_GB, META_D0 };   // the last two: dense reward's shapes and distance before the step
 
 // shared-memory word of word i of a state record's body block (x[N], y[N], angle[N], vx[N], vy[N], w[N])
 template <class SC>
@@ -140,6 +141,8 @@ struct StepParams {
     int n_envs, n_steps, n_actions, n_levels;
     int chunk_steps, n_chunks;   // a launch is cut into n_chunks pieces of chunk_steps steps; work items are (chunk, env)
     int solver_iters, warm_start, auto_reset, max_episode_steps;
+    int discrete;             // actions are int32 codes (multi-discrete action space) instead of floats
+    float dense_kappa;        // coefficient of the dense reward (0 = off)
     float dt, gdt, contact_alpha, contact_beta, slop, rest_thr, face_tol, joint_alpha, joint_beta, joint_gamma, motor_rho, aabb_margin;
     unsigned long long seed;
     long long env_offset;
@@ -374,12 +377,15 @@ __device__ __noinline__ float2 angular_row(float *jr, float ia, float ib, float 
 // ---- joints; the row of joint j is in shared memory.  MODE 0: warm start, 1: solver iteration,
 // 2: positional correction, 3: motor
 template <class SC, int MODE>
-__device__ __forceinline__ void visit_joint(float *sm, uint32_t jab, int j, const uint32_t *lv, float motor_rho) {
+__device__ __forceinline__ void visit_joint(float *sm, uint32_t jab, int j, const uint32_t *lv, float motor_rho, int discrete = 0) {
     const int a = jab & 255, b = (jab >> 8) & 255;
     const bool dyn_a = (jab >> 29) & 1u, dyn_b = (jab >> 30) & 1u;
     float *jr = sm + SC::JROW + kJointWords * j;
     if (MODE == 3) {
-        const float A = fmax_cmp(fmin_cmp(sm[SC::ACT + ((jab >> 16) & 255)], 1.0f), -1.0f);
+        const float av = sm[SC::ACT + ((jab >> 16) & 255)];
+        // paper, "Action Space": continuous in [-1, 1], or multi-discrete codes 0 off, 1 forwards, 2 backwards at full power
+        const float A = discrete ? (__float_as_int(av) == 1 ? 1.0f : (__float_as_int(av) == 2 ? -1.0f : 0.0f))
+                                 : fmax_cmp(fmin_cmp(av, 1.0f), -1.0f);
         const float speed = __uint_as_float(lv[SC::LV_JOINT + kJointLevelWords * j + 5]), power = __uint_as_float(lv[SC::LV_JOINT + kJointLevelWords * j + 6]);
         const float wa = sm[SC::BVEL + 4 * a + 2], wb = sm[SC::BVEL + 4 * b + 2];
         const float arg = __fmaf_rn(-speed, A, wa - wb) * motor_rho;
@@ -424,12 +430,13 @@ __device__ __forceinline__ void visit_joint(float *sm, uint32_t jab, int j, cons
 }
 // joints of one level touch disjoint movable bodies; levels in order keep the joint order
 template <class SC, int G, int MODE>
-__device__ __forceinline__ void sweep_joints(float *sm, uint32_t jab, int lane, int jlevel, int jmax, const uint32_t *lv, float motor_rho) {
+__device__ __forceinline__ void sweep_joints(float *sm, uint32_t jab, int lane, int jlevel, int jmax, const uint32_t *lv, float motor_rho,
+                                             int discrete = 0) {
     const unsigned mask = Group<G>().mask;
     if (SC::J == 0) return;
 #pragma unroll 1
     for (int lvl = 1; lvl <= jmax; ++lvl) {
-        if (jlevel == lvl) visit_joint<SC, MODE>(sm, jab, lane, lv, motor_rho);
+        if (jlevel == lvl) visit_joint<SC, MODE>(sm, jab, lane, lv, motor_rho, discrete);
         __syncwarp(mask);
     }
 }
@@ -772,6 +779,7 @@ __device__ __noinline__ uint32_t load_level_consts(uint32_t *smu, const uint32_t
     }
     for (int i = lane; i < SC::C; i += G) smu[SC::RAD + i] = lv[SC::LV_RAD + i];
     for (int i = lane; i < SC::MASKW; i += G) smu[SC::MASK + i] = lv[SC::LV_MASK + i];
+    if (lane == 0) smu[SC::META + META_GB] = lv[SC::LV_GB];
     return (SC::J > 0 && lane < SC::J) ? lv[SC::LV_JOINT + kJointLevelWords * lane] : 0u;
 }
 
@@ -856,6 +864,13 @@ struct Scene {
     __device__ __forceinline__ float &ovl(int f) { return sm[SC::STG + LF_COUNT * G + f * (G / 2) + lane]; }
     __device__ __forceinline__ ContactConsts contact_consts() const {
         ContactConsts cc; cc.slop = prm.slop; cc.rest_thr = prm.rest_thr; cc.alpha = prm.contact_alpha; cc.beta = prm.contact_beta; return cc;
+    }
+    // paper, "Reward": d_t of the dense signal kappa (d_t - d_{t+1})
+    __device__ __forceinline__ float green_blue_distance() const {
+        const uint32_t gb = smu[SC::META + META_GB];
+        const float4 pg = ld4(sm + SC::BPOS + 4 * (gb & 255u)), pb = ld4(sm + SC::BPOS + 4 * ((gb >> 8) & 255u));
+        const float dx = pb.x - pg.x, dy = pb.y - pg.y;
+        return sqrtf(dot2(dx, dy, dx, dy));
     }
     __device__ __forceinline__ void flush() {
         if (lane == 0) flush_counters(prm.counters, c_surv, c_rec, c_man);
@@ -1031,6 +1046,8 @@ struct Scene {
             return;
         }
         const uint32_t *lv = prm.levels + (size_t)smu[SC::META + META_LEVEL] * SC::LV_WORDS;
+        // dense reward: distance between the first green and the first blue shape before the step
+        if (prm.dense_kappa != 0.0f && lane == 0) sm[SC::META + META_D0] = green_blue_distance();
         // actions of this step
         if (lane < prm.n_actions) sm[SC::ACT + lane] = prm.actions[((size_t)s * prm.n_envs + e) * prm.n_actions + lane];
         if (G < kMaxActions && lane + G < prm.n_actions) sm[SC::ACT + lane + G] = prm.actions[((size_t)s * prm.n_envs + e) * prm.n_actions + lane + G];
@@ -1078,7 +1095,7 @@ struct Scene {
             box4(i) = make_float4(x0, y0, x1, y1);
         }
         // motors (joint order), thrusters (thruster order)
-        sweep_joints<SC, G, 3>(sm, jab, lane, jlevel, jmax, lv, prm.motor_rho);
+        sweep_joints<SC, G, 3>(sm, jab, lane, jlevel, jmax, lv, prm.motor_rho, prm.discrete);
         if (SC::T > 0) {
             int tl = 0; uint32_t tp = 0u;
             if (lane < SC::T) { tp = lv[SC::LV_THR + 8 * lane]; if ((tp >> 16) & 1u) tl = (tp >> 17) & 7u; }
@@ -1088,7 +1105,9 @@ struct Scene {
                 if (tl == lvl) {
                     const int i = tp & 255;
                     const uint32_t *th = lv + SC::LV_THR + 8 * lane;
-                    const float A = fmax_cmp(fmin_cmp(sm[SC::ACT + ((tp >> 8) & 255)], 1.0f), 0.0f);
+                    const float tv = sm[SC::ACT + ((tp >> 8) & 255)];
+                    // continuous in [0, 1], or multi-discrete: 0 off, anything else full power
+                    const float A = prm.discrete ? (__float_as_int(tv) != 0 ? 1.0f : 0.0f) : fmax_cmp(fmin_cmp(tv, 1.0f), 0.0f);
                     const float c = sm[SC::BC + i], sn = sm[SC::BS + i];
                     float dx, dy, rx, ry;
                     rot2(c, sn, __uint_as_float(th[3]), __uint_as_float(th[4]), dx, dy);
@@ -1368,6 +1387,8 @@ struct Scene {
         // reward, termination, counters, auto-reset
         const bool timeout = prm.max_episode_steps > 0 && step_count >= prm.max_episode_steps;
         float reward = (float)((int)touch_gb - (int)touch_gr);
+        if (prm.dense_kappa != 0.0f && ((smu[SC::META + META_GB] >> 16) & 1u))
+            reward = reward + prm.dense_kappa * (sm[SC::META + META_D0] - green_blue_distance());
         bool done = touch_gb || touch_gr || timeout;
         if (!finite) { reward = 0.0f; done = true; }
         if (lane == 0) {

@@ -18,7 +18,7 @@ RESET_NONE, RESET_SAME_LEVEL, RESET_POOL = 0, 1, 2
 
 EXPORTS = (
     "k2d_default_config", "k2d_state_bytes", "k2d_level_pool_bytes", "k2d_create", "k2d_reset", "k2d_step",
-    "k2d_step_static_scratch", "k2d_obs",
+    "k2d_step_discrete", "k2d_step_static_scratch", "k2d_obs",
     "k2d_obs_floats", "k2d_canonical_words", "k2d_get_state", "k2d_set_state", "k2d_status", "k2d_level_info",
     "k2d_set_trace", "k2d_trace_slots", "k2d_eval_sincos_tanh", "k2d_error_string", "k2d_destroy",
 )
@@ -29,7 +29,7 @@ class Config(C.Structure):
         [(n, C.c_int32) for n in ("n_envs", "n_polygons", "n_circles", "n_joints", "n_thrusters", "n_actions", "n_levels",
                                   "solver_iters", "warm_start", "auto_reset", "max_episode_steps", "max_fused_steps")] +
         [(n, C.c_float) for n in ("dt", "gravity_y", "contact_alpha", "contact_beta", "slop", "restitution_threshold",
-                                  "face_tol", "joint_alpha", "joint_beta", "motor_rho", "aabb_margin", "joint_gamma")] +
+                                  "face_tol", "joint_alpha", "joint_beta", "motor_rho", "aabb_margin", "joint_gamma", "dense_kappa")] +
         [("seed", C.c_uint64), ("env_offset", C.c_int64), ("device", C.c_int32), ("lanes_per_scene", C.c_int32),
          ("cuda_stream", C.c_void_p)])
 
@@ -70,6 +70,7 @@ def load_library():
         lib.k2d_reset.argtypes = [vp, vp]
         lib.k2d_step.argtypes = [vp, vp, i32, vp, vp]
         lib.k2d_step_static_scratch.argtypes = [vp, vp, i32, vp, vp]
+        lib.k2d_step_discrete.argtypes = [vp, vp, i32, vp, vp]
         lib.k2d_obs.argtypes = [vp, vp]
         lib.k2d_obs_floats.argtypes = [C.POINTER(Config)]
         lib.k2d_canonical_words.argtypes = [C.POINTER(Config)]
@@ -172,7 +173,9 @@ class Env:
         crowded scenes live in an array inside the library instead of the tail of the state buffer
         (for callers that cannot allocate that tail; at most 1024 envs)."""
         torch = self.torch
-        assert actions.is_cuda and actions.dtype == torch.float32 and actions.is_contiguous()
+        assert actions.is_cuda and actions.dtype in (torch.float32, torch.int32) and actions.is_contiguous()
+        discrete = actions.dtype == torch.int32        # multi-discrete codes go through k2d_step_discrete
+        assert not (discrete and static_scratch)
         if actions.dim() == 2:
             actions = actions.unsqueeze(0)
         n_steps = actions.shape[0]
@@ -182,7 +185,7 @@ class Env:
         if done is None:
             done = torch.empty((n_steps, self.n_envs), dtype=torch.uint8, device=self.device)
         fn, name = ((self.lib.k2d_step_static_scratch, "k2d_step_static_scratch") if static_scratch
-                    else (self.lib.k2d_step, "k2d_step"))
+                    else (self.lib.k2d_step_discrete, "k2d_step_discrete") if discrete else (self.lib.k2d_step, "k2d_step"))
         _check(fn(self._h, actions.data_ptr(), n_steps, reward.data_ptr(), done.data_ptr()), name)
         return reward, done
 

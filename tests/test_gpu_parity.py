@@ -250,3 +250,33 @@ def test_joint_kinds_with_auto_reset_and_checkpoint():
     sa, sb = env.get_state(), env2.get_state()
     for k in sa:
         assert np.array_equal(sa[k], sb[k], equal_nan=True), k
+
+
+def test_multi_discrete_actions_match_the_oracle():
+    n_envs = 64
+    lv = scenes.make_levels("L", n_envs, 81, static_prob=0.1)
+    env = k2d.Env(lv, n_envs)
+    ref = k2d_ref.RefSim(lv, n_envs, discrete_actions=1)
+    codes = np.random.default_rng(81).integers(0, 3, (40, n_envs, env.n_actions)).astype(np.int32)
+    (r, d), (rr, dr) = parity.step_both(env, ref, codes, chunk=10)
+    err, exact = parity.errors(env, ref)
+    assert exact, err
+    assert np.array_equal(r, rr) and np.array_equal(d, dr)
+    # the same codes read as floats would be something else: the discrete entry point really decoded them
+    env2 = k2d.Env(lv, n_envs)
+    import torch
+    env2.step(torch.from_numpy(codes.astype(np.float32)).cuda())
+    assert not np.array_equal(env2.get_state()["angvel"], env.get_state()["angvel"])
+
+
+@pytest.mark.parametrize("lanes", [16, 32])
+def test_dense_reward_matches_the_oracle(lanes):
+    n_envs = 128
+    lv = scenes.make_levels("L", 64, 82, static_prob=0.1)
+    env, ref = parity.make_pair(lv, n_envs, auto_reset=2, max_episode_steps=9, seed=4, dense_kappa=0.3, lanes_per_scene=lanes)
+    act = scenes.make_actions(48, n_envs, env.n_actions, 82)
+    (r, d), (rr, dr) = parity.step_both(env, ref, act, chunk=16)
+    assert np.array_equal(r.view(np.uint32), rr.view(np.uint32)) and np.array_equal(d, dr)
+    assert np.count_nonzero((r != 0) & (np.abs(r) < 0.5)) > r.size // 2          # most steps carry a dense term
+    err, exact = parity.errors(env, ref)
+    assert exact, err

@@ -215,3 +215,66 @@ def test_threads_do_not_change_results():
     rb, db = b.step(act, n_threads=5)
     assert np.array_equal(a.pos, b.pos) and np.array_equal(ra, rb) and np.array_equal(da, db)
     assert np.array_equal(a.counters, b.counters)
+
+
+# ---------------------------------------------------------------- multi-discrete actions, dense reward
+def _motor_and_thruster_level():
+    return custom_level(DIMS, polygons=[dict(half=(0.2, 0.2), pos=(0.0, 3.0), static=1),
+                                        dict(half=(0.4, 0.1), pos=(0.0, 3.0), density=1.0),
+                                        dict(half=(0.3, 0.3), pos=(2.0, 3.0), density=1.0)],
+                        joints=[dict(a=0, b=1, speed=2.0, power=0.05)],
+                        thrusters=[dict(shape=2, power=3.0, rot=0.5)])
+
+
+@pytest.mark.parametrize("codes,continuous", [((0, 0), (0.0, 0.0)), ((1, 1), (1.0, 1.0)), ((2, 0), (-1.0, 0.0)), ((2, 1), (-1.0, 1.0))])
+def test_multi_discrete_actions_are_off_or_full_power(codes, continuous):
+    # paper, "Action Space": inactive, or at maximum power, motors forwards or backwards
+    lv = _motor_and_thruster_level()
+    d = k2d_ref.RefSim(lv, 1, discrete_actions=1)
+    c = k2d_ref.RefSim(lv, 1)
+    for _ in range(5):
+        d.step(np.array(codes, np.float32).reshape(1, 1, 2))
+        c.step(np.array(continuous, np.float32).reshape(1, 1, 2))
+    for k in ("pos", "angle", "vel", "angvel"):
+        assert np.array_equal(getattr(d, k), getattr(c, k)), k
+    if codes != (0, 0):
+        idle = k2d_ref.RefSim(lv, 1)
+        for _ in range(5):
+            idle.step(np.zeros((1, 1, 2), np.float32))
+        assert not np.array_equal(idle.vel, d.vel) or not np.array_equal(idle.angvel, d.angvel)
+
+
+def test_dense_reward_is_kappa_times_the_decrease_of_the_green_blue_distance():
+    # a green circle flies at constant velocity towards a fixated blue one, no gravity: d_t - d_{t+1} = v dt
+    kappa, v = 0.25, 1.5
+    lv = custom_level(DIMS, circles=[dict(radius=0.25, pos=(-3.0, 2.0), vel=(v, 0.0), role=ROLE_GREEN),
+                                     dict(radius=0.25, pos=(1.0, 2.0), static=1, role=ROLE_BLUE)])
+    sim = k2d_ref.RefSim(lv, 1, f64=True, gravity_y=0.0, dense_kappa=kappa)
+    r, d = sim.step(np.zeros((10, 1, sim.n_actions)))
+    assert np.allclose(r[:, 0], kappa * v / 60.0, rtol=0, atol=1e-12) and not d.any()
+    # moving away gives the negative; without kappa nothing
+    lv["vel"][0, 3] = (-v, 0.0)
+    sim = k2d_ref.RefSim(lv, 1, f64=True, gravity_y=0.0, dense_kappa=kappa)
+    r, _ = sim.step(np.zeros((3, 1, sim.n_actions)))
+    assert np.allclose(r[:, 0], -kappa * v / 60.0, rtol=0, atol=1e-12)
+    sim = k2d_ref.RefSim(lv, 1, f64=True, gravity_y=0.0)
+    r, _ = sim.step(np.zeros((3, 1, sim.n_actions)))
+    assert np.all(r == 0.0)
+
+
+def test_dense_reward_adds_to_the_touch_reward_and_needs_both_shapes():
+    kappa = 0.5
+    lv = touching_level(True, False)
+    plain = k2d_ref.RefSim(lv, 1, f64=True)
+    dense = k2d_ref.RefSim(lv, 1, f64=True, dense_kappa=kappa)
+    g = int(np.argmax(lv["role"][0] == ROLE_GREEN)); b = int(np.argmax(lv["role"][0] == ROLE_BLUE))
+    d0 = np.hypot(*(dense.pos[0, b] - dense.pos[0, g]))
+    rp, _ = plain.step(np.zeros((1, 1, plain.n_actions)))
+    rd, dd = dense.step(np.zeros((1, 1, dense.n_actions)))
+    d1 = np.hypot(*(dense.pos[0, b] - dense.pos[0, g]))
+    assert rp[0, 0] == 1.0 and dd[0, 0] == 1
+    assert rd[0, 0] == pytest.approx(1.0 + kappa * (d0 - d1), abs=1e-12)
+    lv["role"][0][lv["role"][0] == ROLE_BLUE] = 0
+    sim = k2d_ref.RefSim(lv, 1, f64=True, dense_kappa=kappa)
+    r, _ = sim.step(np.zeros((2, 1, sim.n_actions)))
+    assert np.all(r == 0.0)
