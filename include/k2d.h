@@ -192,6 +192,16 @@ int k2d_step_static_scratch(k2d_state *s, const float *dev_actions, int32_t n_st
 int k2d_obs(k2d_state *s, float *dev_obs);
 int k2d_obs_floats(const k2d_config *cfg);
 
+/* Pixel observation (paper: the "Pixels" observation space, a 125 x 125 image; the paper gives
+ * no more than the size).  dev_pixels is [n_envs][K2D_PIXELS][K2D_PIXELS][4] bytes, RGBA, row 0
+ * at the top, 4-byte aligned.  The centre of pixel (row r, column c) is the world point
+ * x = -3.125 + (c + 0.5) * 0.05, y = 5.75 - (r + 0.5) * 0.05.  A pixel has the colour of the
+ * highest-index active shape whose interior or boundary contains its centre, white otherwise:
+ * green (0, 200, 0), blue (0, 0, 220), red (220, 0, 0), no role (128, 128, 128) or, if fixated,
+ * (64, 64, 64); alpha is 255.  Joints and thrusters are not drawn.  Asynchronous on the stream. */
+#define K2D_PIXELS 125
+int k2d_render(k2d_state *s, uint8_t *dev_pixels);
+
 /* Canonical host copy of the dynamic state, for checkpoints and comparisons: per env
  * k2d_canonical_words 4-byte words: pos[N][2], angle[N], vel[N][2], angvel[N] (floats),
  * acc[n_slots][2] (accumulated normal, tangent impulse per manifold slot), jacc[n_joints][3]

@@ -23,8 +23,10 @@
  * momentum/restitution, circle-plane and corner distances by brute force,
  * polygon overlap by Sutherland-Hodgman brute force, resting box impulse
  * m*g*dt, sliding-block Coulomb deceleration, pendulum period and energy,
- * motor recurrence, thruster closed form, solver invariants, splitmix64
- * vectors, sincos/tanh against libm.  The whole step has no Jax2D trajectory
+ * motor recurrence, thruster closed form, fixed-joint common angular velocity
+ * and error decay, joint-limit stops, multi-discrete codes, dense reward of a
+ * body at constant speed, rendered areas and draw order, solver invariants,
+ * splitmix64 vectors, sincos/tanh against libm.  The whole step has no Jax2D trajectory
  * to compare with: "parity unpinned" against the paper's own implementation.
  */
 #include <math.h>
@@ -1057,6 +1059,71 @@ void k2d_ref_obs(ref_sim *S, real *obs) {
             r[3] = S->lv_thr_power[l * T + t];
             r[4] = d.y; r[5] = d.x;
         }
+    }
+}
+
+/* ---- pixel observation ---------------------------------------------------
+ * The paper gives the size only ("125 x 125 observation", section "Pixels" of
+ * the network details).  Reading: an RGBA byte image per env, row 0 at the top;
+ * the centre of pixel (row r, column c) is the world point
+ * x = -3.125 + (c + 0.5) * 0.05, y = 5.75 - (r + 0.5) * 0.05 (a 6.25 m window
+ * with the floor's top edge half a metre above its bottom); a pixel takes the
+ * colour of the highest-index active shape that contains its centre (polygon:
+ * not outside any face; circle: squared distance <= radius squared), white
+ * otherwise; colours by role (none: grey, darker if fixated; green; blue;
+ * red), alpha 255.  Joints and thrusters are not drawn. */
+#define PIX 125
+void k2d_ref_render(ref_sim *S, uint8_t *out) {
+    const ref_config *cf = &S->cfg;
+    const int P = S->P, C = S->C, N = S->N;
+    const real scale = RC(0.05), x0 = RC(-3.125), y1 = RC(5.75);
+    static const uint8_t role_rgb[4][3] = { { 128, 128, 128 }, { 0, 200, 0 }, { 0, 0, 220 }, { 220, 0, 0 } };
+    for (int e = 0; e < cf->n_envs; ++e) {
+        const int l = S->level_id[e];
+        const real *pos = S->pos + (size_t)e * N * 2, *ang = S->angle + (size_t)e * N;
+        real cs[32], sn[32];
+        wpoly W[16];
+        for (int i = 0; i < N; ++i) k2d_ref_sincos(ang[i], &cs[i], &sn[i]);
+        for (int i = 0; i < P; ++i) {
+            wpoly *w = &W[i];
+            w->cnt = S->lv_nverts[l * P + i];
+            const real *lv = S->lv_verts + ((size_t)(l * P + i) * MAX_VERTS) * 2;
+            const real *ln = S->lv_normals + ((size_t)(l * P + i) * MAX_VERTS) * 2;
+            for (int k = 0; k < w->cnt; ++k) {
+                vec2 loc = { lv[2 * k], lv[2 * k + 1] }, nl = { ln[2 * k], ln[2 * k + 1] };
+                vec2 r = rot2(cs[i], sn[i], loc);
+                w->w[k].x = r.x + pos[2 * i]; w->w[k].y = r.y + pos[2 * i + 1];
+                w->nrm[k] = rot2(cs[i], sn[i], nl);
+                w->off[k] = dot2(w->nrm[k], w->w[k]);
+            }
+        }
+        uint8_t *img = out + (size_t)e * PIX * PIX * 4;
+        for (int r = 0; r < PIX; ++r)
+            for (int c = 0; c < PIX; ++c) {
+                vec2 p = { x0 + ((real)c + RC(0.5)) * scale, y1 - ((real)r + RC(0.5)) * scale };
+                int hit = -1;
+                for (int i = N - 1; i >= 0 && hit < 0; --i) {
+                    if (!S->lv_active[l * N + i]) continue;
+                    if (i < P) {
+                        int inside = 1;
+                        for (int k = 0; k < W[i].cnt; ++k) if (dot2(W[i].nrm[k], p) - W[i].off[k] > RC(0)) inside = 0;
+                        if (inside) hit = i;
+                    } else {
+                        vec2 d = { p.x - pos[2 * i], p.y - pos[2 * i + 1] };
+                        real rad = S->lv_radius[l * C + (i - P)];
+                        if (dot2(d, d) <= rad * rad) hit = i;
+                    }
+                }
+                uint8_t *px = img + ((size_t)r * PIX + c) * 4;
+                if (hit < 0) { px[0] = px[1] = px[2] = 255; }
+                else {
+                    int role = S->lv_role[l * N + hit];
+                    const uint8_t *rgb = role_rgb[role];
+                    int dark = (role == 0 && S->lv_static[l * N + hit]);
+                    px[0] = dark ? 64 : rgb[0]; px[1] = dark ? 64 : rgb[1]; px[2] = dark ? 64 : rgb[2];
+                }
+                px[3] = 255;
+            }
     }
 }
 

@@ -62,6 +62,7 @@ def _lib(f64: bool):
         lib.k2d_ref_views.argtypes = [C.c_void_p, C.c_void_p]
         lib.k2d_ref_step.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_int]
         lib.k2d_ref_obs.argtypes = [C.c_void_p, C.c_void_p]
+        lib.k2d_ref_render.argtypes = [C.c_void_p, C.c_void_p]
         lib.k2d_ref_obs_floats.argtypes = [C.c_void_p]
         lib.k2d_ref_obs_floats.restype = C.c_int
         lib.k2d_ref_sincos.argtypes = [real, C.c_void_p, C.c_void_p]
@@ -179,6 +180,12 @@ class RefSim:
         o = np.zeros((self.n_envs, self.obs_floats), self.real)
         self.lib.k2d_ref_obs(self._h, o.ctypes.data)
         return o
+
+    def render(self):
+        """RGBA byte images [n_envs][125][125][4] of the scenes (the pixel observation)"""
+        img = np.zeros((self.n_envs, 125, 125, 4), np.uint8)
+        self.lib.k2d_ref_render(self._h, img.ctypes.data)
+        return img
 
     def snapshot(self) -> dict:
         return {k: getattr(self, k).copy() for k in ("pos", "angle", "vel", "angvel", "acc", "jacc", "step_count",

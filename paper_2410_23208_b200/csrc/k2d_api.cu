@@ -450,6 +450,18 @@ int k2d_obs(k2d_state *s, float *dev_obs) {
     return K2D_OK;
 }
 
+int k2d_render(k2d_state *s, uint8_t *dev_pixels) {
+    if (!s || !dev_pixels) return K2D_ERR_NULL;
+    if ((uintptr_t)dev_pixels & 3) return K2D_ERR_ALIGN;
+    const int E = s->cfg.n_envs;
+    uint32_t *out = reinterpret_cast<uint32_t *>(dev_pixels);
+    if (s->ci.id == 0) k2d_render_kernel<ClassS><<<E, kRenderThreads, 0, s->stream>>>(s->dev_env, s->dev_levels, out, E);
+    else if (s->ci.id == 1) k2d_render_kernel<ClassM><<<E, kRenderThreads, 0, s->stream>>>(s->dev_env, s->dev_levels, out, E);
+    else k2d_render_kernel<ClassL><<<E, kRenderThreads, 0, s->stream>>>(s->dev_env, s->dev_levels, out, E);
+    CUDA_OK(cudaGetLastError());
+    return K2D_OK;
+}
+
 int k2d_get_state(k2d_state *s, void *host_canonical) {
     if (!s || !host_canonical) return K2D_ERR_NULL;
     const k2d_config &c = s->cfg; const ClassInfo &ci = s->ci;

@@ -1657,6 +1657,97 @@ __global__ void __launch_bounds__(kObsThreads) k2d_obs_kernel(const uint32_t *st
     }
 }
 
+// ---------------------------------------------------------------- pixel observation: one block per env
+// A 125 x 125 RGBA image of the scene: the centre of pixel (row r, column c) is the world point
+// (-3.125 + (c + 0.5) * 0.05, 5.75 - (r + 0.5) * 0.05); a pixel takes the colour of the highest-index active
+// shape that contains its centre (polygon: not outside any face; circle: squared distance <= radius squared),
+// white otherwise.  Each warp takes rows; per row it first finds the shapes whose box reaches the row.
+constexpr int kPix = 125;
+constexpr int kRenderThreads = 128;
+template <class SC>
+__global__ void __launch_bounds__(kRenderThreads) k2d_render_kernel(const uint32_t *state, const uint32_t *levels, uint32_t *pixels, int n_envs) {
+    __shared__ float4 s_box[SC::N];          // min x, min y, max x, max y, a little enlarged (culling only)
+    __shared__ float4 s_nx[SC::N], s_ny[SC::N], s_off[SC::N];   // polygon: face normals and offsets; circle: centre x, y, radius^2 in .x
+    __shared__ uint32_t s_col[SC::N];
+    __shared__ int s_nv[SC::N];              // vertices of a polygon, 0 for a circle, -1 for a shape that is not drawn
+    const int e = blockIdx.x;
+    if (e >= n_envs) return;
+    const uint32_t *st = state + (size_t)e * SC::ST_WORDS;
+    const uint32_t *lv = levels + (size_t)st[SC::ST_META + META_LEVEL] * SC::LV_WORDS;
+    const float *stf = reinterpret_cast<const float *>(st);
+    const float *lvf = reinterpret_cast<const float *>(lv);
+    for (int i = threadIdx.x; i < SC::N; i += kRenderThreads) {
+        const uint32_t fl = lv[SC::LV_FLAGS + i];
+        int nv = -1;
+        if (fl & F_ACTIVE) {
+            const float x = stf[i], y = stf[SC::N + i];
+            const uint32_t role = flag_role(fl);
+            uint32_t rgb = role == 1u ? (200u << 8) : role == 2u ? (220u << 16) : role == 3u ? 220u : ((fl & F_DYNAMIC) ? 0x808080u : 0x404040u);
+            s_col[i] = rgb | 0xff000000u;
+            if (i < SC::P) {
+                nv = (int)flag_nverts(fl);
+                float c, sn;
+                sincos_spec(stf[2 * SC::N + i], c, sn);
+                float nxs[4] = { 0.0f, 0.0f, 0.0f, 0.0f }, nys[4] = { 0.0f, 0.0f, 0.0f, 0.0f }, offs[4] = { 0.0f, 0.0f, 0.0f, 0.0f };
+                float x0 = 0.0f, y0 = 0.0f, x1 = 0.0f, y1 = 0.0f;
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    if (k < nv) {
+                        float rx, ry;
+                        rot2(c, sn, lvf[SC::LV_PVX + 4 * i + k], lvf[SC::LV_PVY + 4 * i + k], rx, ry);
+                        rot2(c, sn, lvf[SC::LV_PNX + 4 * i + k], lvf[SC::LV_PNY + 4 * i + k], nxs[k], nys[k]);
+                        const float wx = rx + x, wy = ry + y;
+                        offs[k] = dot2(nxs[k], nys[k], wx, wy);
+                        if (k == 0) { x0 = x1 = wx; y0 = y1 = wy; }
+                        else { x0 = fmin_cmp(x0, wx); x1 = fmax_cmp(x1, wx); y0 = fmin_cmp(y0, wy); y1 = fmax_cmp(y1, wy); }
+                    }
+                }
+                s_nx[i] = make_float4(nxs[0], nxs[1], nxs[2], nxs[3]); s_ny[i] = make_float4(nys[0], nys[1], nys[2], nys[3]);
+                s_off[i] = make_float4(offs[0], offs[1], offs[2], offs[3]);
+                s_box[i] = make_float4(x0 - 0.01f, y0 - 0.01f, x1 + 0.01f, y1 + 0.01f);
+            } else {
+                nv = 0;
+                const float r = lvf[SC::LV_RAD + (i - SC::P)];
+                s_nx[i] = make_float4(x, 0.0f, 0.0f, 0.0f); s_ny[i] = make_float4(y, 0.0f, 0.0f, 0.0f); s_off[i] = make_float4(r * r, 0.0f, 0.0f, 0.0f);
+                s_box[i] = make_float4(x - r - 0.01f, y - r - 0.01f, x + r + 0.01f, y + r + 0.01f);
+            }
+        }
+        s_nv[i] = nv;
+    }
+    __syncthreads();
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    uint32_t *img = pixels + (size_t)e * kPix * kPix;
+    for (int r = warp; r < kPix; r += kRenderThreads / 32) {
+        const float py = 5.75f - ((float)r + 0.5f) * 0.05f;
+        bool reach = false;
+        if (lane < SC::N && s_nv[lane] >= 0) reach = s_box[lane].y <= py && py <= s_box[lane].w;
+        const unsigned row_mask = __ballot_sync(0xffffffffu, reach);
+        for (int c = lane; c < kPix; c += 32) {
+            const float px = -3.125f + ((float)c + 0.5f) * 0.05f;
+            uint32_t col = 0xffffffffu;
+            unsigned m = row_mask;
+            while (m) {
+                const int i = 31 - __clz(m);
+                m &= ~(1u << i);
+                const float4 bx = s_box[i];
+                if (px < bx.x || px > bx.z) continue;
+                bool inside;
+                const int nv = s_nv[i];
+                if (nv > 0) {
+                    const float4 nx = s_nx[i], ny = s_ny[i], off = s_off[i];
+                    inside = !(dot2(nx.x, ny.x, px, py) - off.x > 0.0f) && !(dot2(nx.y, ny.y, px, py) - off.y > 0.0f) &&
+                             !(dot2(nx.z, ny.z, px, py) - off.z > 0.0f) && (nv < 4 || !(dot2(nx.w, ny.w, px, py) - off.w > 0.0f));
+                } else {
+                    const float dx = px - s_nx[i].x, dy = py - s_ny[i].x;
+                    inside = dot2(dx, dy, dx, dy) <= s_off[i].x;
+                }
+                if (inside) { col = s_col[i]; break; }
+            }
+            img[r * kPix + c] = col;
+        }
+    }
+}
+
 __global__ void k2d_eval_kernel(const float *x, int n, float *c, float *s, float *t) {
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= n) return;

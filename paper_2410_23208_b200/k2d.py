@@ -18,7 +18,7 @@ RESET_NONE, RESET_SAME_LEVEL, RESET_POOL = 0, 1, 2
 
 EXPORTS = (
     "k2d_default_config", "k2d_state_bytes", "k2d_level_pool_bytes", "k2d_create", "k2d_reset", "k2d_step",
-    "k2d_step_discrete", "k2d_step_static_scratch", "k2d_obs",
+    "k2d_step_discrete", "k2d_step_static_scratch", "k2d_obs", "k2d_render",
     "k2d_obs_floats", "k2d_canonical_words", "k2d_get_state", "k2d_set_state", "k2d_status", "k2d_level_info",
     "k2d_set_trace", "k2d_trace_slots", "k2d_eval_sincos_tanh", "k2d_error_string", "k2d_destroy",
 )
@@ -72,6 +72,7 @@ def load_library():
         lib.k2d_step_static_scratch.argtypes = [vp, vp, i32, vp, vp]
         lib.k2d_step_discrete.argtypes = [vp, vp, i32, vp, vp]
         lib.k2d_obs.argtypes = [vp, vp]
+        lib.k2d_render.argtypes = [vp, vp]
         lib.k2d_obs_floats.argtypes = [C.POINTER(Config)]
         lib.k2d_canonical_words.argtypes = [C.POINTER(Config)]
         lib.k2d_get_state.argtypes = [vp, vp]
@@ -194,6 +195,14 @@ class Env:
         if out is None:
             out = torch.empty((self.n_envs, self.obs_floats), dtype=torch.float32, device=self.device)
         _check(self.lib.k2d_obs(self._h, out.data_ptr()), "k2d_obs")
+        return out
+
+    def render(self, out=None):
+        """RGBA byte images [n_envs, 125, 125, 4] of the scenes (the pixel observation)"""
+        torch = self.torch
+        if out is None:
+            out = torch.empty((self.n_envs, 125, 125, 4), dtype=torch.uint8, device=self.device)
+        _check(self.lib.k2d_render(self._h, out.data_ptr()), "k2d_render")
         return out
 
     # ---- canonical state

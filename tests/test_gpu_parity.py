@@ -280,3 +280,17 @@ def test_dense_reward_matches_the_oracle(lanes):
     assert np.count_nonzero((r != 0) & (np.abs(r) < 0.5)) > r.size // 2          # most steps carry a dense term
     err, exact = parity.errors(env, ref)
     assert exact, err
+
+
+@pytest.mark.parametrize("size", ["S", "M", "L"])
+def test_pixel_observation_matches_the_oracle(size):
+    n_envs = 24
+    lv = scenes.make_levels(size, n_envs, 91, static_prob=0.2, triangle_prob=0.3)
+    lv["active"][3, 2] = 0
+    env, ref = parity.make_pair(lv, n_envs)
+    assert np.array_equal(env.render().cpu().numpy(), ref.render())       # the levels as placed
+    act = scenes.make_actions(30, n_envs, env.n_actions, 91)
+    parity.step_both(env, ref, act)
+    img, want = env.render().cpu().numpy(), ref.render()
+    assert np.array_equal(img, want)                                      # byte for byte after 30 steps
+    assert (want[..., :3] != 255).any(-1).mean() > 0.05 and np.all(img[..., 3] == 255)
