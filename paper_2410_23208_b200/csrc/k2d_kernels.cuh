@@ -1661,7 +1661,7 @@ __global__ void __launch_bounds__(kObsThreads) k2d_obs_kernel(const uint32_t *st
 // A 125 x 125 RGBA image of the scene: the centre of pixel (row r, column c) is the world point
 // (-3.125 + (c + 0.5) * 0.05, 5.75 - (r + 0.5) * 0.05); a pixel takes the colour of the highest-index active
 // shape that contains its centre (polygon: not outside any face; circle: squared distance <= radius squared),
-// white otherwise.  Each warp takes rows; per row it first finds the shapes whose box reaches the row.
+// white otherwise.
 constexpr int kPix = 125;
 constexpr int kRenderThreads = 128;
 template <class SC>
@@ -1717,34 +1717,43 @@ __global__ void __launch_bounds__(kRenderThreads) k2d_render_kernel(const uint32
     __syncthreads();
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     uint32_t *img = pixels + (size_t)e * kPix * kPix;
+    // a warp paints one row at a time in registers: lane l holds the pixels of columns l, l + 32, l + 64, l + 96;
+    // the shapes whose box reaches the row go over it in index order, each only over the 32-column blocks its box
+    // touches, so the highest index ends up on top
     for (int r = warp; r < kPix; r += kRenderThreads / 32) {
         const float py = 5.75f - ((float)r + 0.5f) * 0.05f;
         bool reach = false;
         if (lane < SC::N && s_nv[lane] >= 0) reach = s_box[lane].y <= py && py <= s_box[lane].w;
-        const unsigned row_mask = __ballot_sync(0xffffffffu, reach);
-        for (int c = lane; c < kPix; c += 32) {
-            const float px = -3.125f + ((float)c + 0.5f) * 0.05f;
-            uint32_t col = 0xffffffffu;
-            unsigned m = row_mask;
-            while (m) {
-                const int i = 31 - __clz(m);
-                m &= ~(1u << i);
-                const float4 bx = s_box[i];
-                if (px < bx.x || px > bx.z) continue;
+        unsigned m = __ballot_sync(0xffffffffu, reach);
+        uint32_t col[4] = { 0xffffffffu, 0xffffffffu, 0xffffffffu, 0xffffffffu };
+        while (m) {
+            const int i = __ffs(m) - 1;
+            m &= m - 1u;
+            const float4 bx = s_box[i];
+            // columns that certainly cover the (enlarged) box; the exact test decides
+            const int c_lo = (int)fmax_cmp(fmin_cmp((bx.x + 3.125f) * 20.0f - 1.0f, 126.0f), 0.0f);
+            const int c_hi = (int)fmax_cmp(fmin_cmp((bx.z + 3.125f) * 20.0f + 1.0f, 124.0f), -1.0f);
+            const int nv = s_nv[i];
+            const float4 nx = s_nx[i], ny = s_ny[i], off = s_off[i];
+            const uint32_t shape_col = s_col[i];
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                if (c_hi < 32 * k || c_lo > 32 * k + 31) continue;       // the same for the whole warp
+                const float px = -3.125f + ((float)(32 * k + lane) + 0.5f) * 0.05f;
                 bool inside;
-                const int nv = s_nv[i];
                 if (nv > 0) {
-                    const float4 nx = s_nx[i], ny = s_ny[i], off = s_off[i];
                     inside = !(dot2(nx.x, ny.x, px, py) - off.x > 0.0f) && !(dot2(nx.y, ny.y, px, py) - off.y > 0.0f) &&
                              !(dot2(nx.z, ny.z, px, py) - off.z > 0.0f) && (nv < 4 || !(dot2(nx.w, ny.w, px, py) - off.w > 0.0f));
                 } else {
-                    const float dx = px - s_nx[i].x, dy = py - s_ny[i].x;
-                    inside = dot2(dx, dy, dx, dy) <= s_off[i].x;
+                    const float dx = px - nx.x, dy = py - ny.x;
+                    inside = dot2(dx, dy, dx, dy) <= off.x;
                 }
-                if (inside) { col = s_col[i]; break; }
+                if (inside) col[k] = shape_col;
             }
-            img[r * kPix + c] = col;
         }
+#pragma unroll
+        for (int k = 0; k < 4; ++k)
+            if (32 * k + lane < kPix) img[r * kPix + 32 * k + lane] = col[k];
     }
 }
 
