@@ -255,19 +255,50 @@ def run_gpu(args) -> dict:
     total_ms = float(sum(step_ms) + sum(obs_ms))
     counts = env.status() - counts0
 
-    # ---- end to end through the public API with host buffers: H2D actions, step, obs, D2H reward + done
-    for i in range(2):
-        stage.copy_(host_actions[i % len(host_actions)], non_blocking=True)
-        env.step(stage, reward, done)
+    # ---- end to end through the public API with host buffers: every step uploads its actions from pinned host
+    # memory and reads reward + done back; a second stream carries the copies, so the upload of step i + 1 and
+    # the read-back of step i - 1 overlap the launches of step i (two sets of device buffers)
+    copy_stream = torch.cuda.Stream(dev)
+    main_stream = torch.cuda.current_stream(dev)
+    stages = [stage, torch.empty_like(stage)]
+    rewards, dones = [reward, torch.empty_like(reward)], [done, torch.empty_like(done)]
+    ev_up = [torch.cuda.Event() for _ in range(K + 3)]
+    ev_done = [torch.cuda.Event() for _ in range(K + 3)]
+    ev_down = [torch.cuda.Event() for _ in range(K + 3)]
+
+    def upload(i):
+        with torch.cuda.stream(copy_stream):
+            if i >= 2:
+                copy_stream.wait_event(ev_done[i - 2])       # the launch that last read this staging buffer
+            stages[i % 2].copy_(host_actions[i % len(host_actions)], non_blocking=True)
+            ev_up[i].record(copy_stream)
+
+    def run(i):
+        main_stream.wait_event(ev_up[i])
+        if i >= 2:
+            main_stream.wait_event(ev_down[i - 2])           # its results have been read back
+        env.step(stages[i % 2], rewards[i % 2], dones[i % 2])
+        env.obs(obs)
+        ev_done[i].record(main_stream)
+
+    def download(i):
+        with torch.cuda.stream(copy_stream):
+            copy_stream.wait_event(ev_done[i])
+            host_reward.copy_(rewards[i % 2], non_blocking=True)
+            host_done.copy_(dones[i % 2], non_blocking=True)
+            ev_down[i].record(copy_stream)
+
     barrier()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
+    copy_stream.wait_event(e0)
+    upload(0)
     for i in range(K):
-        stage.copy_(host_actions[i % len(host_actions)], non_blocking=True)
-        env.step(stage, reward, done)
-        env.obs(obs)
-        host_reward.copy_(reward, non_blocking=True)
-        host_done.copy_(done, non_blocking=True)
+        run(i)
+        if i + 1 < K:
+            upload(i + 1)
+        download(i)
+    main_stream.wait_event(ev_down[K - 1])
     e1.record()
     barrier()
     e2e_ms = e0.elapsed_time(e1)
