@@ -72,8 +72,10 @@ struct SizeClass {
     static constexpr int ACT = MASK + MASKW;
     static constexpr int META = ACT + kMaxActions;       // step_count, episode_count, level_id, status, warm entries
     static constexpr int JROW = (META + 8 + 3) / 4 * 4;  // J rows of kJointWords, 16-byte aligned
-    static constexpr int SURV = JROW + kJointWords * J;  // bytes: pairs that passed the box test
-    static constexpr int WIDX = SURV + (NPAIRS + 3) / 4; // bytes: pair -> record index of the previous step
+    static constexpr int LVC = JROW + kJointWords * J;   // copy of the level record's edge lengths, joint and thruster records
+    static constexpr int LVC_WORDS = LV_MASK - LV_ELEN;
+    static constexpr int SURV = LVC + LVC_WORDS;         // bytes: pairs that passed the box test
+    static constexpr int WIDX = SURV + ((NPAIRS + 3) / 4 > N ? (NPAIRS + 3) / 4 : N); // bytes: pair -> record index of the previous step (the survivor area is reused as N words)
     // then, per lane of the group (field-major, G words per field):
     //   STG  kStageWords fields: manifolds on their way to the owning lane; afterwards the second manifold's constants
     //   ACC2 2 fields: accumulated impulses of the second manifold
@@ -377,7 +379,7 @@ __device__ __noinline__ float2 angular_row(float *jr, float ia, float ib, float 
 // ---- joints; the row of joint j is in shared memory.  MODE 0: warm start, 1: solver iteration,
 // 2: positional correction, 3: motor
 template <class SC, int MODE>
-__device__ __forceinline__ void visit_joint(float *sm, uint32_t jab, int j, const uint32_t *lv, float motor_rho, int discrete = 0) {
+__device__ __forceinline__ void visit_joint(float *sm, uint32_t jab, int j, float motor_rho, int discrete = 0) {
     const int a = jab & 255, b = (jab >> 8) & 255;
     const bool dyn_a = (jab >> 29) & 1u, dyn_b = (jab >> 30) & 1u;
     float *jr = sm + SC::JROW + kJointWords * j;
@@ -386,7 +388,8 @@ __device__ __forceinline__ void visit_joint(float *sm, uint32_t jab, int j, cons
         // paper, "Action Space": continuous in [-1, 1], or multi-discrete codes 0 off, 1 forwards, 2 backwards at full power
         const float A = discrete ? (__float_as_int(av) == 1 ? 1.0f : (__float_as_int(av) == 2 ? -1.0f : 0.0f))
                                  : fmax_cmp(fmin_cmp(av, 1.0f), -1.0f);
-        const float speed = __uint_as_float(lv[SC::LV_JOINT + kJointLevelWords * j + 5]), power = __uint_as_float(lv[SC::LV_JOINT + kJointLevelWords * j + 6]);
+        const float *jl = sm + SC::LVC + (SC::LV_JOINT - SC::LV_ELEN) + kJointLevelWords * j;
+        const float speed = jl[5], power = jl[6];
         const float wa = sm[SC::BVEL + 4 * a + 2], wb = sm[SC::BVEL + 4 * b + 2];
         const float arg = __fmaf_rn(-speed, A, wa - wb) * motor_rho;
         const float jr_ = power * tanh_spec(arg);
@@ -430,13 +433,13 @@ __device__ __forceinline__ void visit_joint(float *sm, uint32_t jab, int j, cons
 }
 // joints of one level touch disjoint movable bodies; levels in order keep the joint order
 template <class SC, int G, int MODE>
-__device__ __forceinline__ void sweep_joints(float *sm, uint32_t jab, int lane, int jlevel, int jmax, const uint32_t *lv, float motor_rho,
+__device__ __forceinline__ void sweep_joints(float *sm, uint32_t jab, int lane, int jlevel, int jmax, float motor_rho,
                                              int discrete = 0) {
     const unsigned mask = Group<G>().mask;
     if (SC::J == 0) return;
 #pragma unroll 1
     for (int lvl = 1; lvl <= jmax; ++lvl) {
-        if (jlevel == lvl) visit_joint<SC, MODE>(sm, jab, lane, lv, motor_rho, discrete);
+        if (jlevel == lvl) visit_joint<SC, MODE>(sm, jab, lane, motor_rho, discrete);
         __syncwarp(mask);
     }
 }
@@ -558,7 +561,7 @@ __device__ __forceinline__ void slow_sweep_pairs(float *sm, uint32_t *ovf, int n
 // their levels, warm start and all solver iterations, joints included.  old_n / old_t: this lane's
 // first-manifold accumulated impulses of the previous step.  Returns the highest contact level.
 template <class SC, int G>
-__device__ __noinline__ int slow_solve(float *sm, uint32_t *ovf, const uint32_t *lv, int nrec, uint32_t jab, int jlevel, int jmax,
+__device__ __noinline__ int slow_solve(float *sm, uint32_t *ovf, int nrec, uint32_t jab, int jlevel, int jmax,
                                        int solver_iters, int warm_start, float motor_rho, float old_n, float old_t, ContactConsts cc) {
     Group<G> g;
     const int lane = g.lane;
@@ -617,9 +620,9 @@ __device__ __noinline__ int slow_solve(float *sm, uint32_t *ovf, const uint32_t 
     }
     g.sync();
     slow_sweep_pairs<SC, G, 0>(sm, ovf, nrec, cmax);
-    sweep_joints<SC, G, 0>(sm, jab, lane, jlevel, jmax, lv, motor_rho);
+    sweep_joints<SC, G, 0>(sm, jab, lane, jlevel, jmax, motor_rho);
     for (int it = 0; it < solver_iters; ++it) {
-        sweep_joints<SC, G, 1>(sm, jab, lane, jlevel, jmax, lv, motor_rho);
+        sweep_joints<SC, G, 1>(sm, jab, lane, jlevel, jmax, motor_rho);
         slow_sweep_pairs<SC, G, 1>(sm, ovf, nrec, cmax);
     }
     return cmax;
@@ -780,6 +783,7 @@ __device__ __noinline__ uint32_t load_level_consts(uint32_t *smu, const uint32_t
     for (int i = lane; i < SC::C; i += G) smu[SC::RAD + i] = lv[SC::LV_RAD + i];
     for (int i = lane; i < SC::MASKW; i += G) smu[SC::MASK + i] = lv[SC::LV_MASK + i];
     if (lane == 0) smu[SC::META + META_GB] = lv[SC::LV_GB];
+    for (int i = lane; i < SC::LVC_WORDS; i += G) smu[SC::LVC + i] = lv[SC::LV_ELEN + i];
     return (SC::J > 0 && lane < SC::J) ? lv[SC::LV_JOINT + kJointLevelWords * lane] : 0u;
 }
 
@@ -956,7 +960,7 @@ struct Scene {
     }
 
     // polygon a against circle b
-    __device__ unsigned manifold_pc(int a, int b, Manifold &m, const uint32_t *lv) const {
+    __device__ unsigned manifold_pc(int a, int b, Manifold &m) const {
         const int cnt = flag_nverts(smu[SC::BFL + a]);
         const float cx = sm[SC::BPOS + 4 * b], cy = sm[SC::BPOS + 4 * b + 1], r = sm[SC::RAD + (b - SC::P)];
         float maxsep = 0.0f, mind2 = 0.0f, qx = 0.0f, qy = 0.0f, dqx = 0.0f, dqy = 0.0f;
@@ -969,7 +973,7 @@ struct Scene {
                 const float sep = dot2(nx, ny, cx, cy) - sm[SC::WOFF + 4 * a + k];
                 const float tx = -ny, ty = nx;
                 float s = dot2(tx, ty, cx - wx, cy - wy);
-                s = fmax_cmp(fmin_cmp(s, __uint_as_float(lv[SC::LV_ELEN + 4 * a + k])), 0.0f);
+                s = fmax_cmp(fmin_cmp(s, sm[SC::LVC + 4 * a + k]), 0.0f);
                 const float px = __fmaf_rn(s, tx, wx), py = __fmaf_rn(s, ty, wy);
                 const float ex = cx - px, ey = cy - py;
                 const float d2 = dot2(ex, ey, ex, ey);
@@ -1095,16 +1099,16 @@ struct Scene {
             box4(i) = make_float4(x0, y0, x1, y1);
         }
         // motors (joint order), thrusters (thruster order)
-        sweep_joints<SC, G, 3>(sm, jab, lane, jlevel, jmax, lv, prm.motor_rho, prm.discrete);
+        sweep_joints<SC, G, 3>(sm, jab, lane, jlevel, jmax, prm.motor_rho, prm.discrete);
         if (SC::T > 0) {
             int tl = 0; uint32_t tp = 0u;
-            if (lane < SC::T) { tp = lv[SC::LV_THR + 8 * lane]; if ((tp >> 16) & 1u) tl = (tp >> 17) & 7u; }
+            const uint32_t *th = smu + SC::LVC + (SC::LV_THR - SC::LV_ELEN) + 8 * lane;
+            if (lane < SC::T) { tp = th[0]; if ((tp >> 16) & 1u) tl = (tp >> 17) & 7u; }
             const int tmax = g.max_int(tl);
 #pragma unroll 1
             for (int lvl = 1; lvl <= tmax; ++lvl) {
                 if (tl == lvl) {
                     const int i = tp & 255;
-                    const uint32_t *th = lv + SC::LV_THR + 8 * lane;
                     const float tv = sm[SC::ACT + ((tp >> 8) & 255)];
                     // continuous in [0, 1], or multi-discrete: 0 off, anything else full power
                     const float A = prm.discrete ? (__float_as_int(tv) != 0 ? 1.0f : 0.0f) : fmax_cmp(fmin_cmp(tv, 1.0f), 0.0f);
@@ -1130,7 +1134,7 @@ struct Scene {
             float kr = 0.0f, bias_r = 0.0f;
             if ((jab >> 24) & 1u) {
                 const int a = jab & 255, b = (jab >> 8) & 255;
-                const uint32_t *jl = lv + SC::LV_JOINT + kJointLevelWords * lane;
+                const uint32_t *jl = smu + SC::LVC + (SC::LV_JOINT - SC::LV_ELEN) + kJointLevelWords * lane;
                 float rax, ray, rbx, rby;
                 rot2(sm[SC::BC + a], sm[SC::BS + a], __uint_as_float(jl[1]), __uint_as_float(jl[2]), rax, ray);
                 rot2(sm[SC::BC + b], sm[SC::BS + b], __uint_as_float(jl[3]), __uint_as_float(jl[4]), rbx, rby);
@@ -1212,7 +1216,7 @@ struct Scene {
                 if (idx < hi) {
                     p = surv()[idx]; a = ptab[p] & 255; b = ptab[p] >> 8;
                     if (kind == 0) act = manifold_pp(a, b, m);
-                    else if (kind == 1) act = manifold_pc(a, b, m[0], lv);
+                    else if (kind == 1) act = manifold_pc(a, b, m[0]);
                     else act = manifold_cc(a, b, m[0]);
                     // a polygon pair rejected before its manifolds exist leaves its slots at the default
                     if (trace && !(kind == 0 && act == 0u))
@@ -1257,7 +1261,7 @@ struct Scene {
         const bool overflow = nrec > G + G / 2;
         int cmax = 0, clevel = 0, clevel2 = 0;
         if (overflow) {
-            cmax = slow_solve<SC, G>(sm, ovf, lv, nrec, jab, jlevel, jmax, prm.solver_iters, prm.warm_start, prm.motor_rho,
+            cmax = slow_solve<SC, G>(sm, ovf, nrec, jab, jlevel, jmax, prm.solver_iters, prm.warm_start, prm.motor_rho,
                                      rec.accn, rec.acct, contact_consts());
         } else {
             const ContactConsts cc = contact_consts();
@@ -1320,16 +1324,25 @@ struct Scene {
                 c_man += (unsigned)g.sum_int((int)(r2 >> 8));
             } else {
                 // levels of the records (canonical order = record order): one more than the highest level of an
-                // earlier record that shares a movable body
-                int lvl = mine ? 1 : 0;
+                // earlier record that shares a movable body.  Every movable body collects the set of records that
+                // touch it; a record's conflicts are the earlier members of its bodies' sets; then level r goes to
+                // the records whose conflicts all have a level already, round after round.
+                uint32_t *touch = smu + SC::SURV;            // the survivor list is no longer needed
+                for (int i = lane; i < SC::N; i += G) touch[i] = 0u;
+                g.sync();
                 const bool da = (ab >> 26) & 1u, db = (ab >> 27) & 1u;
+                if (mine && da) atomicOr(touch + a, 1u << lane);
+                if (mine && db) atomicOr(touch + b, 1u << lane);
+                g.sync();
+                const unsigned conflicts = ((da ? touch[a] : 0u) | (db ? touch[b] : 0u)) & g.lanes_below();
+                const unsigned all = g.ballot(mine);
+                unsigned assigned = 0u;
+                int lvl = 0;
 #pragma unroll 1
-                for (int q = 0; q + 1 < nrec; ++q) {
-                    const uint32_t abq = g.shflu(ab, q);
-                    const int lq = g.shfl(lvl, q);
-                    const int aq = abq & 31, bq = (abq >> 5) & 31;
-                    const bool hit = (da && (a == aq || a == bq)) || (db && (b == aq || b == bq));
-                    if (q < lane && mine && hit) lvl = max(lvl, lq + 1);
+                for (int r = 1; assigned != all; ++r) {
+                    const bool ready = mine && lvl == 0 && (conflicts & ~assigned) == 0u;
+                    if (ready) lvl = r;
+                    assigned |= g.ballot(ready);
                 }
                 clevel = lvl;
                 cmax = g.max_int(lvl);
@@ -1337,11 +1350,11 @@ struct Scene {
             c_man += (unsigned)(__popc(g.ballot(amask & 1u)) + __popc(g.ballot(amask & 2u)));
             // warm start: contacts, then joints
             sweep_pairs<0>(cmax, clevel, clevel2);
-            sweep_joints<SC, G, 0>(sm, jab, lane, jlevel, jmax, lv, prm.motor_rho);
+            sweep_joints<SC, G, 0>(sm, jab, lane, jlevel, jmax, prm.motor_rho);
             // solver iterations: joints, then contacts
 #pragma unroll 1
             for (int it = 0; it < prm.solver_iters; ++it) {
-                sweep_joints<SC, G, 1>(sm, jab, lane, jlevel, jmax, lv, prm.motor_rho);
+                sweep_joints<SC, G, 1>(sm, jab, lane, jlevel, jmax, prm.motor_rho);
                 sweep_pairs<1>(cmax, clevel, clevel2);
             }
         }
@@ -1355,7 +1368,7 @@ struct Scene {
         g.sync();
         if (overflow) slow_correct<SC, G>(sm, ovf, nrec, cmax);
         else sweep_pairs<2>(cmax, clevel, clevel2);
-        sweep_joints<SC, G, 2>(sm, jab, lane, jlevel, jmax, lv, prm.motor_rho);
+        sweep_joints<SC, G, 2>(sm, jab, lane, jlevel, jmax, prm.motor_rho);
         bool finite = true;
         for (int i = lane; i < SC::N; i += G) {
             const float4 p4 = ld4(sm + SC::BPOS + 4 * i), v4 = ld4(sm + SC::BVEL + 4 * i);
