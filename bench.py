@@ -39,7 +39,7 @@ FLOPS = dict(body=37, circle_box=4, polygon=84, box_test=8, cc=16, pc=94, pp=190
              pair_prestep=5, man_prestep=54, man_warm=28, man_iter=57, man_pos=10,
              joint_fixed=48 + 33 + 18 + 8, joint_iter=38, thruster=27)
 # DRAM bytes one ncu capture measured for one k2d_step launch of the benchmark workload, per env
-NCU_DRAM_BYTES_PER_ENV_LAUNCH = 1991.0   # profiles/k2d_step_kernel_L_16384envs_32steps.md: (32.210 MB + 0.411 MB) / 16384 envs; None once the kernel has changed since
+NCU_DRAM_BYTES_PER_ENV_LAUNCH = 2064.0   # profiles/k2d_step_kernel_L_16384envs_32steps.md: (33.369 MB + 0.448 MB) / 16384 envs; None once the kernel has changed since
 
 
 def fp32_peak_tflops(sm_count: int = 148, sm_mhz: float = 1965.0) -> float:
