@@ -30,3 +30,20 @@ def test_benchmark_configuration_matches_the_oracle_on_every_env(lanes, horizon)
     assert exact, err
     assert np.array_equal(env.status(), ref.counters)
     assert d.sum() >= (n_envs * 5 if horizon == 12 else 1)
+
+
+@pytest.mark.parametrize("lanes,n_envs", [(0, 6000), (32, 3000)])
+def test_a_few_more_envs_than_resident_groups(lanes, n_envs):
+    # just above the number of scene groups a B200 holds at once (5920 half-warps, 2960 warps for L scenes):
+    # the second chunk of the first envs is handed out while their first chunk may still be running on another
+    # group, so groups really wait for one another here
+    w = scenes.WORKLOADS[3]
+    seed = 77
+    lv = scenes.make_levels(w["size"], 256, seed, static_prob=w["static_prob"])
+    env, ref = parity.make_pair(lv, n_envs, auto_reset=2, max_episode_steps=10, seed=seed, max_fused_steps=24, lanes_per_scene=lanes)
+    act = scenes.make_actions(48, n_envs, env.n_actions, seed)
+    (r, d), (rr, dr) = parity.step_both(env, ref, act, chunk=24, n_threads=os.cpu_count() or 1)
+    assert np.array_equal(r, rr) and np.array_equal(d, dr)
+    err, exact = parity.errors(env, ref)
+    assert exact, err
+    assert np.array_equal(env.status(), ref.counters)       # also says that no wait ran out
