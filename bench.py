@@ -219,6 +219,9 @@ def run_gpu(args) -> dict:
     reward = torch.empty((FUSED, n_envs), dtype=torch.float32, device=dev)
     done = torch.empty((FUSED, n_envs), dtype=torch.uint8, device=dev)
     obs = torch.empty((n_envs, env.obs_floats), dtype=torch.float32, device=dev)
+    if args.pixels:
+        obs = torch.empty((n_envs, 125, 125, 4), dtype=torch.uint8, device=dev)
+        env.obs = env.render                      # same call shape: writes into the buffer it is given
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
     host_reward = torch.empty((FUSED, n_envs), dtype=torch.float32).pin_memory()
     host_done = torch.empty((FUSED, n_envs), dtype=torch.uint8).pin_memory()
@@ -320,6 +323,8 @@ def run_gpu(args) -> dict:
     flops_step = algorithmic_flops_per_env_step(dims, levels, counts, env.cfg.solver_iters)
     mean_pairs = float(counts[7]) / max(1, int(counts[3]))
     bytes_ = algorithmic_bytes_per_env_launch(dims, FUSED, mean_pairs, env.obs_floats)
+    if args.pixels:
+        bytes_["obs"] = 125 * 125 * 4 + 4 * 6 * dims.n_shapes      # the image out, the poses in
     achieved_tflops = flops_step * env_steps_per_launch / (mean_step_ms * 1e-3) / 1e12
     peak = fp32_peak_tflops()
     hbm_peak, hbm_src = measured_hbm_gbs()
@@ -332,6 +337,7 @@ def run_gpu(args) -> dict:
         "config": {"workload": f"{w['size']} scenes, {n_envs} envs per GPU, {FUSED} fused engine steps + 1 observation per bench step "
                                f"(config {args.workload}: pool of {w['n_levels']} levels, horizon {w['max_episode_steps']})",
                    "lanes_per_scene": env.cfg.lanes_per_scene or 16, "fused_steps": FUSED,
+                   "observation": "pixels 125x125 RGBA (k2d_render)" if args.pixels else "symbolic entity rows (k2d_obs)",
                    "l2": "flushed between timed iterations (256 MiB write, untimed); K distinct action buffers"},
         "clocks": clk,
         "e2e": {"value": e2e_value, "unit": UNIT,
@@ -363,6 +369,7 @@ def main():
     ap.add_argument("--envs", type=int, default=0, help="override the workload's env count (per GPU)")
     ap.add_argument("--lanes", type=int, default=0, help="lanes per scene (0 = library default)")
     ap.add_argument("--fused", type=int, default=FUSED, help="engine steps per k2d_step launch (1 = one launch and one observation per step)")
+    ap.add_argument("--pixels", action="store_true", help="the observation of a bench step is the 125 x 125 pixel image (k2d_render) instead of the entity rows")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "k2d" else args.warmup
