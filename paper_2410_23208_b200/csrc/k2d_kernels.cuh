@@ -1677,9 +1677,17 @@ __global__ void __launch_bounds__(kObsThreads) k2d_obs_kernel(const uint32_t *st
 // white otherwise.
 constexpr int kPix = 125;
 constexpr int kRenderThreads = 128;
+// pixel columns and rows that certainly cover a world-frame box (one pixel and 1 cm to spare); the exact tests decide
+__device__ __forceinline__ int4 pixel_range(float x0, float y0, float x1, float y1) {
+    const int c_lo = (int)fmax_cmp(fmin_cmp((x0 - 0.01f + 3.125f) * 20.0f - 1.5f, 126.0f), 0.0f);
+    const int c_hi = (int)fmax_cmp(fmin_cmp((x1 + 0.01f + 3.125f) * 20.0f + 1.5f, 124.0f), -1.0f);
+    const int r_lo = (int)fmax_cmp(fmin_cmp((5.75f - (y1 + 0.01f)) * 20.0f - 1.5f, 126.0f), 0.0f);
+    const int r_hi = (int)fmax_cmp(fmin_cmp((5.75f - (y0 - 0.01f)) * 20.0f + 1.5f, 124.0f), -1.0f);
+    return make_int4(c_lo, c_hi, r_lo, r_hi);
+}
 template <class SC>
 __global__ void __launch_bounds__(kRenderThreads) k2d_render_kernel(const uint32_t *state, const uint32_t *levels, uint32_t *pixels, int n_envs) {
-    __shared__ float4 s_box[SC::N];          // min x, min y, max x, max y, a little enlarged (culling only)
+    __shared__ int4 s_rng[SC::N];            // first and last column, first and last row that the shape's box can reach (culling only)
     __shared__ float4 s_nx[SC::N], s_ny[SC::N], s_off[SC::N];   // polygon: face normals and offsets; circle: centre x, y, radius^2 in .x
     __shared__ uint32_t s_col[SC::N];
     __shared__ int s_nv[SC::N];              // vertices of a polygon, 0 for a circle, -1 for a shape that is not drawn
@@ -1717,12 +1725,12 @@ __global__ void __launch_bounds__(kRenderThreads) k2d_render_kernel(const uint32
                 }
                 s_nx[i] = make_float4(nxs[0], nxs[1], nxs[2], nxs[3]); s_ny[i] = make_float4(nys[0], nys[1], nys[2], nys[3]);
                 s_off[i] = make_float4(offs[0], offs[1], offs[2], offs[3]);
-                s_box[i] = make_float4(x0 - 0.01f, y0 - 0.01f, x1 + 0.01f, y1 + 0.01f);
+                s_rng[i] = pixel_range(x0, y0, x1, y1);
             } else {
                 nv = 0;
                 const float r = lvf[SC::LV_RAD + (i - SC::P)];
                 s_nx[i] = make_float4(x, 0.0f, 0.0f, 0.0f); s_ny[i] = make_float4(y, 0.0f, 0.0f, 0.0f); s_off[i] = make_float4(r * r, 0.0f, 0.0f, 0.0f);
-                s_box[i] = make_float4(x - r - 0.01f, y - r - 0.01f, x + r + 0.01f, y + r + 0.01f);
+                s_rng[i] = pixel_range(x - r, y - r, x + r, y + r);
             }
         }
         s_nv[i] = nv;
@@ -1736,30 +1744,30 @@ __global__ void __launch_bounds__(kRenderThreads) k2d_render_kernel(const uint32
     for (int r = warp; r < kPix; r += kRenderThreads / 32) {
         const float py = 5.75f - ((float)r + 0.5f) * 0.05f;
         bool reach = false;
-        if (lane < SC::N && s_nv[lane] >= 0) reach = s_box[lane].y <= py && py <= s_box[lane].w;
+        if (lane < SC::N && s_nv[lane] >= 0) reach = s_rng[lane].z <= r && r <= s_rng[lane].w;
         unsigned m = __ballot_sync(0xffffffffu, reach);
         uint32_t col[4] = { 0xffffffffu, 0xffffffffu, 0xffffffffu, 0xffffffffu };
         while (m) {
             const int i = __ffs(m) - 1;
             m &= m - 1u;
-            const float4 bx = s_box[i];
-            // columns that certainly cover the (enlarged) box; the exact test decides
-            const int c_lo = (int)fmax_cmp(fmin_cmp((bx.x + 3.125f) * 20.0f - 1.0f, 126.0f), 0.0f);
-            const int c_hi = (int)fmax_cmp(fmin_cmp((bx.z + 3.125f) * 20.0f + 1.0f, 124.0f), -1.0f);
+            const int4 rng = s_rng[i];
             const int nv = s_nv[i];
             const float4 nx = s_nx[i], ny = s_ny[i], off = s_off[i];
             const uint32_t shape_col = s_col[i];
+            // the row's share of every face's dot product (polygon) or of the squared distance (circle)
+            const float t0 = ny.x * py, t1 = ny.y * py, t2 = ny.z * py, t3 = ny.w * py;
+            const float dy = py - ny.x, dy2 = dy * dy;
 #pragma unroll
             for (int k = 0; k < 4; ++k) {
-                if (c_hi < 32 * k || c_lo > 32 * k + 31) continue;       // the same for the whole warp
+                if (rng.y < 32 * k || rng.x > 32 * k + 31) continue;       // the same for the whole warp
                 const float px = -3.125f + ((float)(32 * k + lane) + 0.5f) * 0.05f;
                 bool inside;
                 if (nv > 0) {
-                    inside = !(dot2(nx.x, ny.x, px, py) - off.x > 0.0f) && !(dot2(nx.y, ny.y, px, py) - off.y > 0.0f) &&
-                             !(dot2(nx.z, ny.z, px, py) - off.z > 0.0f) && (nv < 4 || !(dot2(nx.w, ny.w, px, py) - off.w > 0.0f));
+                    inside = !(__fmaf_rn(nx.x, px, t0) - off.x > 0.0f) && !(__fmaf_rn(nx.y, px, t1) - off.y > 0.0f) &&
+                             !(__fmaf_rn(nx.z, px, t2) - off.z > 0.0f) && (nv < 4 || !(__fmaf_rn(nx.w, px, t3) - off.w > 0.0f));
                 } else {
-                    const float dx = px - nx.x, dy = py - ny.x;
-                    inside = dot2(dx, dy, dx, dy) <= off.x;
+                    const float dx = px - nx.x;
+                    inside = __fmaf_rn(dx, dx, dy2) <= off.x;
                 }
                 if (inside) col[k] = shape_col;
             }
