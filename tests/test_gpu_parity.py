@@ -294,3 +294,44 @@ def test_pixel_observation_matches_the_oracle(size):
     img, want = env.render().cpu().numpy(), ref.render()
     assert np.array_equal(img, want)                                      # byte for byte after 30 steps
     assert (want[..., :3] != 255).any(-1).mean() > 0.05 and np.all(img[..., 3] == 255)
+
+
+def test_degenerate_and_edge_cases_match_the_oracle():
+    # hand-made scenes around the narrowphase's special cases, one env each: coincident circle centres, a circle
+    # centre inside a polygon and exactly on a face, boxes resting with exactly parallel faces, a triangle tip in
+    # a box, a lone floor (nothing to do), an all-fixated scene, and a single env on its own
+    dims = scenes.SceneDims(4, 3, 1, 1)
+    floor = dict(half=(5.0, 0.5), pos=(0.0, -0.5), static=1)
+    cases = [
+        scenes.custom_level(dims, polygons=[floor], circles=[dict(radius=0.3, pos=(0.0, 2.0)), dict(radius=0.2, pos=(0.0, 2.0))]),
+        scenes.custom_level(dims, polygons=[floor, dict(half=(0.5, 0.5), pos=(0.0, 0.5))],
+                            circles=[dict(radius=0.1, pos=(0.1, 0.6)), dict(radius=0.2, pos=(0.0, 1.0)), dict(radius=0.2, pos=(0.5, 0.5))]),
+        scenes.custom_level(dims, polygons=[floor, dict(half=(0.5, 0.25), pos=(0.0, 0.25)), dict(half=(0.5, 0.25), pos=(0.0, 0.75)),
+                                            dict(half=(0.25, 0.25), pos=(0.25, 1.25))]),
+        scenes.custom_level(dims, polygons=[floor, dict(half=(0.6, 0.3), pos=(0.0, 0.3)),
+                                            dict(verts=[(-0.3, 0.2), (0.0, -0.4), (0.3, 0.2)], pos=(0.1, 0.95))]),
+        scenes.custom_level(dims, polygons=[floor]),
+        scenes.custom_level(dims, polygons=[floor, dict(half=(0.3, 0.3), pos=(0.0, 0.2), static=1)],
+                            circles=[dict(radius=0.2, pos=(0.1, 0.3), static=1)]),
+    ]
+    lv = scenes.concat_levels(cases)
+    n = len(cases)
+    env, ref = parity.make_pair(lv, n)
+    act = scenes.make_actions(40, n, env.n_actions, 5)
+    (r, d), (rr, dr) = parity.step_both(env, ref, act[:1])
+    err, exact = parity.errors(env, ref)
+    _check_tolerances(err, 1)
+    assert exact, err
+    (r, d), (rr, dr) = parity.step_both(env, ref, act[1:], chunk=13)
+    err, exact = parity.errors(env, ref)
+    assert exact, err
+    assert np.array_equal(r, rr) and np.array_equal(d, dr)
+    assert np.array_equal(env.obs().cpu().numpy().view(np.uint32), ref.obs().view(np.uint32))
+    assert np.array_equal(env.render().cpu().numpy(), ref.render())
+    # one env alone, one step at a time and the largest fused launch the handle allows
+    one, one_ref = parity.make_pair(scenes.take_levels(lv, [2]), 1, max_fused_steps=64)
+    a1 = scenes.make_actions(64 + 3, 1, one.n_actions, 6)
+    parity.step_both(one, one_ref, a1[:3], chunk=1)
+    parity.step_both(one, one_ref, a1[3:], chunk=64)
+    err, exact = parity.errors(one, one_ref)
+    assert exact, err
