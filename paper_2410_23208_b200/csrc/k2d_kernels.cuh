@@ -20,7 +20,10 @@
 
 namespace k2d {
 
-constexpr int kBlockThreads = 128;
+#ifndef K2D_BLOCK_THREADS
+#define K2D_BLOCK_THREADS 128
+#endif
+constexpr int kBlockThreads = K2D_BLOCK_THREADS;
 #ifndef K2D_MIN_BLOCKS
 #define K2D_MIN_BLOCKS 5
 #endif
