@@ -271,6 +271,33 @@ def eval_sincos_tanh(x):
     return c, s, t
 
 
+def first_outcomes(reward: np.ndarray, done: np.ndarray) -> np.ndarray:
+    """Per env, the reward at its first done step of a rollout without auto-reset ([n_steps][n_envs] arrays):
+    +1 solved, -1 failed, 0 timed out or never done.  Host logic only."""
+    reward, done = np.asarray(reward), np.asarray(done).astype(bool)
+    first = np.argmax(done, axis=0)
+    out = reward[first, np.arange(reward.shape[1])]
+    return np.where(done.any(axis=0), np.sign(out), 0).astype(np.int8)
+
+
+def noop_outcomes(levels: dict, n_steps: int, device: int = 0, chunk: int = 32, **cfg_kw) -> np.ndarray:
+    """What doing nothing achieves on every level: one env per level, zero actions for ``n_steps`` steps, no
+    auto-reset; returns +1 / -1 / 0 per level (see first_outcomes).  The paper's level generator rejects levels
+    that the no-op policy solves ("trivially solvable"); this is that rollout, run by the CUDA library."""
+    import torch
+    n = levels["pos"].shape[0]
+    env = Env(levels, n, device=device, auto_reset=RESET_NONE, max_fused_steps=chunk, **cfg_kw)
+    zeros = torch.zeros((chunk, n, env.n_actions), dtype=torch.float32, device=env.device)
+    rs, ds = [], []
+    for s0 in range(0, n_steps, chunk):
+        k = min(chunk, n_steps - s0)
+        r, d = env.step(zeros[:k])
+        rs.append(r.cpu().numpy())
+        ds.append(d.cpu().numpy())
+    env.close()
+    return first_outcomes(np.concatenate(rs), np.concatenate(ds))
+
+
 def shard_envs(n_envs_total: int, rank: int, world_size: int):
     """Contiguous env range of ``rank``: (offset, count).  Envs are independent, so ranks never
     exchange data; the offset goes into ``env_offset`` so that level draws on auto-reset do not

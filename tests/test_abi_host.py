@@ -113,3 +113,11 @@ def test_shard_envs_partitions_contiguously():
         assert spans[0][0] == 0 and sum(c for _, c in spans) == total
         for (o0, c0), (o1, _) in zip(spans, spans[1:]):
             assert o1 == o0 + c0
+
+
+def test_first_outcomes_takes_the_reward_at_the_first_done_step():
+    reward = np.array([[0, 0, 0, 0], [1, 0, -1, 0], [1, -1, 1, 0]], np.float32)
+    done = np.array([[0, 0, 0, 0], [1, 0, 1, 0], [1, 1, 1, 0]], np.uint8)
+    assert k2d.first_outcomes(reward, done).tolist() == [1, -1, -1, 0]
+    # a done without reward (horizon) counts as neither
+    assert k2d.first_outcomes(np.zeros((2, 1), np.float32), np.array([[0], [1]], np.uint8)).tolist() == [0]

@@ -335,3 +335,12 @@ def test_degenerate_and_edge_cases_match_the_oracle():
     parity.step_both(one, one_ref, a1[3:], chunk=64)
     err, exact = parity.errors(one, one_ref)
     assert exact, err
+
+
+def test_noop_rollout_outcomes_match_the_oracle():
+    lv = scenes.make_levels("M", 96, 95, static_prob=0.1)
+    got = k2d.noop_outcomes(lv, 90, chunk=32)
+    ref = k2d_ref.RefSim(lv, 96)
+    r, d = ref.step(np.zeros((90, 96, ref.n_actions), np.float32))
+    assert np.array_equal(got, k2d.first_outcomes(r, d))
+    assert (got != 0).any()
