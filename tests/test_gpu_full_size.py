@@ -41,8 +41,9 @@ def test_a_few_more_envs_than_resident_groups(lanes, n_envs):
     seed = 77
     lv = scenes.make_levels(w["size"], 256, seed, static_prob=w["static_prob"])
     env, ref = parity.make_pair(lv, n_envs, auto_reset=2, max_episode_steps=10, seed=seed, max_fused_steps=24, lanes_per_scene=lanes)
-    act = scenes.make_actions(48, n_envs, env.n_actions, seed)
-    (r, d), (rr, dr) = parity.step_both(env, ref, act, chunk=24, n_threads=os.cpu_count() or 1)
+    act = scenes.make_actions(40, n_envs, env.n_actions, seed)
+    # launches of 20 steps: work items of 8, 8 and 4 steps
+    (r, d), (rr, dr) = parity.step_both(env, ref, act, chunk=20, n_threads=os.cpu_count() or 1)
     assert np.array_equal(r, rr) and np.array_equal(d, dr)
     err, exact = parity.errors(env, ref)
     assert exact, err
