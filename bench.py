@@ -173,7 +173,7 @@ def run_reference(args) -> dict:
 def cpu_baseline(args, w, dims, levels) -> dict:
     from oracle import k2d_ref
     cores = os.cpu_count() or 1
-    sample_envs, sample_steps = min(w["n_envs"], 2048), 256
+    sample_envs, sample_steps = min(w["n_envs"], 4096), 512      # about 20 core-seconds of oracle work for L scenes
     sim = k2d_ref.RefSim(levels, sample_envs, auto_reset=w["auto_reset"], max_episode_steps=w["max_episode_steps"],
                          seed=scenes.workload_seed(args.workload))
     acts = scenes.make_actions(sample_steps, sample_envs, dims.n_actions, 7)
