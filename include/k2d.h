@@ -95,7 +95,7 @@ typedef struct k2d_config {
     uint64_t seed;                 /* seed of the K2D_RESET_POOL hash                           */
     int64_t env_offset;            /* global index of env 0 (sharding over several GPUs)        */
     int32_t device;                /* CUDA device ordinal                                       */
-    int32_t lanes_per_scene;       /* 0 = library default; else 8, 16 or 32                     */
+    int32_t lanes_per_scene;       /* 0 = library default (32 for few envs, else 16); or 8, 16, 32 */
     void *cuda_stream;             /* cudaStream_t of the caller (NULL = default stream)        */
 } k2d_config;
 
