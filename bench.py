@@ -336,7 +336,7 @@ def run_gpu(args) -> dict:
         "dtype": "f32", "data": "synthetic",
         "config": {"workload": f"{w['size']} scenes, {n_envs} envs per GPU, {FUSED} fused engine steps + 1 observation per bench step "
                                f"(config {args.workload}: pool of {w['n_levels']} levels, horizon {w['max_episode_steps']})",
-                   "lanes_per_scene": env.cfg.lanes_per_scene or (32 if n_envs < 48 * torch.cuda.get_device_properties(dev).multi_processor_count else 16), "fused_steps": FUSED,
+                   "lanes_per_scene": env.cfg.lanes_per_scene or (32 if n_envs < (48 if w["size"] == "L" else 24) * torch.cuda.get_device_properties(dev).multi_processor_count else 16), "fused_steps": FUSED,
                    "observation": "pixels 125x125 RGBA (k2d_render)" if args.pixels else "symbolic entity rows (k2d_obs)",
                    "l2": "flushed between timed iterations (256 MiB write, untimed); K distinct action buffers"},
         "clocks": clk,

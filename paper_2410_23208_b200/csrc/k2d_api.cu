@@ -407,8 +407,8 @@ int k2d_create(const k2d_config *cfg, void *dev_state_buf, void *dev_level_pool_
     int num_sms = 0;
     if (err == cudaSuccess) err = cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, cfg->device);
     // default lanes per scene: a warp per scene while the device has warps to spare (measured on B200: faster below
-    // about 48 envs per SM), two scenes per warp beyond
-    if (err == cudaSuccess && !cfg->lanes_per_scene) s->G = (cfg->n_envs < 48 * num_sms) ? 32 : 16;
+    // about 48 envs per SM for the largest size class, 24 for the smaller ones), two scenes per warp beyond
+    if (err == cudaSuccess && !cfg->lanes_per_scene) s->G = (cfg->n_envs < (ci.id == 2 ? 48 : 24) * num_sms) ? 32 : 16;
     if (err == cudaSuccess) err = K2D_DISPATCH(setup_step, s, s, num_sms);
     if (err == cudaSuccess) err = cudaMemcpyAsync(s->dev_levels, s->host_levels.data(), s->host_levels.size() * 4, cudaMemcpyHostToDevice, s->stream);
     if (err == cudaSuccess) err = cudaStreamSynchronize(s->stream);
