@@ -1,9 +1,11 @@
 // k2d_kernels.cuh -- device code of the batched 2D rigid-body environment step (sm_100a).
 //
-// One group of G lanes (G = 32: one warp; 16 or 8: two or four scenes per warp) owns one scene.
-// The scene's state is loaded from HBM once per launch, kept in shared memory across all fused
-// steps, and written back once.  Within a step the lanes of the group work on bodies, polygon
-// vertices, shape pairs (bounding-box test, narrowphase, contact pre-step) and constraint rows.
+// One group of G lanes (G = 16: two scenes per warp; 32: one warp per scene; 8: four scenes per warp)
+// owns one scene.  A group takes work items (a run of consecutive steps of one env) from a ticket queue;
+// for an item it loads the scene's state from memory once, keeps it in shared memory (bodies, joint rows,
+// world-frame geometry) and in registers (the contact pair record of every lane) across the item's steps,
+// and writes it back once.  Within a step the lanes of the group work on bodies, polygon vertices, shape
+// pairs (bounding-box test, narrowphase), contact pair records (one per lane) and joints (one per lane).
 //
 // Arithmetic contract: every +,-,*,/,sqrt is an individually rounded IEEE binary32 operation
 // (the file is compiled with --fmad=false --prec-div=true --prec-sqrt=true --ftz=false), a fused
