@@ -278,3 +278,14 @@ def test_dense_reward_adds_to_the_touch_reward_and_needs_both_shapes():
     sim = k2d_ref.RefSim(lv, 1, f64=True, dense_kappa=kappa)
     r, _ = sim.step(np.zeros((2, 1, sim.n_actions)))
     assert np.all(r == 0.0)
+
+
+def test_oracle_trajectories_have_not_changed():
+    # digests written by tests/golden/make_oracle_trajectories.py from the oracle alone
+    import importlib.util
+    here = os.path.dirname(os.path.abspath(__file__))
+    spec = importlib.util.spec_from_file_location("make_oracle_trajectories", os.path.join(here, "golden", "make_oracle_trajectories.py"))
+    mod = importlib.util.module_from_spec(spec)
+    spec.loader.exec_module(mod)
+    stored = [ln.strip() for ln in open(os.path.join(here, "golden", "oracle_trajectories.txt")) if ln.strip() and not ln.startswith("#")]
+    assert mod.lines() == stored
