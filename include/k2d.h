@@ -81,6 +81,7 @@ typedef struct k2d_config {
     int32_t auto_reset;            /* K2D_RESET_*                                               */
     int32_t max_episode_steps;     /* 0 = no horizon; else done when step_count reaches it      */
     int32_t max_fused_steps;       /* largest n_steps k2d_step accepts                          */
+    int32_t frame_skip;            /* >= 1: engine steps each action row is held for (paper: 2)  */
     float dt, gravity_y;
     float contact_alpha;           /* velocity correction: bias = alpha * max(pen - slop, 0)    */
     float contact_beta;            /* positional correction: beta * max(pen - slop, 0)          */
@@ -127,7 +128,8 @@ typedef struct k2d_level {
 typedef struct k2d_state k2d_state;   /* opaque host handle */
 
 /* Fills *cfg with the defaults listed above for the given scene dimensions (n_actions =
- * n_joints + n_thrusters, n_levels = n_envs, auto_reset = NONE, max_fused_steps = 64). */
+ * n_joints + n_thrusters, n_levels = n_envs, auto_reset = NONE, max_fused_steps = 64,
+ * frame_skip = 1). */
 int k2d_default_config(k2d_config *cfg, int32_t n_envs, int32_t n_polygons, int32_t n_circles,
                        int32_t n_joints, int32_t n_thrusters);
 
@@ -149,7 +151,9 @@ int k2d_create(const k2d_config *cfg, void *dev_state_buf, void *dev_level_pool_
 int k2d_reset(k2d_state *s, const int32_t *host_level_ids);
 
 /* Advances every env by n_steps steps (paper, Algorithm 1 + "Reward").  dev_actions is
- * [n_steps][n_envs][n_actions] floats, one row consumed per step (motor actions are clipped
+ * [ceil(n_steps / frame_skip)][n_envs][n_actions] floats, one row per frame_skip steps of this
+ * call (frame_skip = 1: one row consumed per step; the paper trains with a frame skip of 2;
+ * reward and done are still written for every engine step) (motor actions are clipped
  * to [-1, 1], thruster actions to [0, 1]: paper, "Action Space"); dev_reward [n_steps][n_envs]
  * floats in {-1, 0, +1}, plus, if dense_kappa is not 0, the paper's auxiliary dense reward
  * kappa * (d_t - d_t+1) with d the distance between the positions of the first green and the

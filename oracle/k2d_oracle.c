@@ -61,7 +61,7 @@ typedef struct { real x, y; } vec2;
 /* ---- configuration and raw level description (filled by the caller) ---- */
 typedef struct {
     int32_t n_polygons, n_circles, n_joints, n_thrusters, n_actions, n_levels, n_envs;
-    int32_t solver_iters, warm_start, auto_reset, max_episode_steps, broadphase, discrete_actions;
+    int32_t solver_iters, warm_start, auto_reset, max_episode_steps, broadphase, discrete_actions, frame_skip;
     real dt, gravity_y, contact_alpha, contact_beta, slop, restitution_threshold, face_tol;
     real joint_alpha, joint_beta, motor_rho, aabb_margin, joint_gamma, dense_kappa;
     uint64_t seed;
@@ -951,12 +951,13 @@ static void step_env(ref_sim *S, int e, const real *act, real *out_reward, uint8
     }
 }
 
-/* actions [n_steps][n_envs][n_actions]; reward, done [n_steps][n_envs] */
+/* actions [ceil(n_steps / frame_skip)][n_envs][n_actions]: every row is held for frame_skip steps (the paper's
+ * frame skip; 1 = a row per step); reward, done [n_steps][n_envs] */
 static void step_range(ref_sim *S, int e0, int e1, const real *actions, int n_steps, real *reward, uint8_t *done, int64_t *cnt) {
-    int E = S->cfg.n_envs, A = S->cfg.n_actions;
+    int E = S->cfg.n_envs, A = S->cfg.n_actions, fs = S->cfg.frame_skip > 0 ? S->cfg.frame_skip : 1;
     for (int e = e0; e < e1; ++e)
         for (int s = 0; s < n_steps; ++s)
-            step_env(S, e, actions + ((size_t)s * E + e) * A, reward + (size_t)s * E + e, done + (size_t)s * E + e, cnt);
+            step_env(S, e, actions + ((size_t)(s / fs) * E + e) * A, reward + (size_t)s * E + e, done + (size_t)s * E + e, cnt);
 }
 
 typedef struct { ref_sim *S; int e0, e1, n_steps; const real *actions; real *reward; uint8_t *done; int64_t cnt[8]; } job;

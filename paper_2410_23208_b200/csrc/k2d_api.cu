@@ -57,7 +57,7 @@ static int check_config(const k2d_config *c) {
         c->n_joints < 0 || c->n_joints > K2D_MAX_JOINTS || c->n_thrusters < 0 || c->n_thrusters > K2D_MAX_THRUSTERS ||
         c->n_actions < 1 || c->n_actions > kMaxActions || c->n_levels < 1 || c->solver_iters < 0 || c->solver_iters > 1024 ||
         (c->warm_start != 0 && c->warm_start != 1) || c->auto_reset < 0 || c->auto_reset > 2 || c->max_episode_steps < 0 ||
-        c->max_fused_steps < 1 || c->device < 0 ||
+        c->max_fused_steps < 1 || c->frame_skip < 1 || c->device < 0 ||
         !(c->lanes_per_scene == 0 || c->lanes_per_scene == 8 || c->lanes_per_scene == 16 || c->lanes_per_scene == 32))
         return K2D_ERR_CONFIG;
     const float f[] = { c->dt, c->gravity_y, c->contact_alpha, c->contact_beta, c->slop, c->restitution_threshold, c->face_tol,
@@ -303,7 +303,7 @@ static StepParams step_params(const k2d_state *s, const float *dev_actions, int 
     prm.state = s->dev_env; prm.levels = s->dev_levels; prm.actions = dev_actions; prm.reward = dev_reward; prm.done = dev_done;
     prm.counters = s->dev_counters; prm.queue = s->dev_queue; prm.chunks_done = s->dev_chunks; prm.scratch = scratch; prm.trace = s->dev_trace;
     prm.n_envs = c.n_envs; prm.n_steps = n_steps; prm.n_actions = c.n_actions; prm.n_levels = c.n_levels;
-    prm.discrete = discrete; prm.dense_kappa = c.dense_kappa;
+    prm.discrete = discrete; prm.dense_kappa = c.dense_kappa; prm.frame_skip = c.frame_skip;
     prm.chunk_steps = n_steps; prm.n_chunks = 1;
     if (c.n_envs > s->groups && n_steps > kChunkSteps) {
         const int n_chunks = (n_steps + kChunkSteps - 1) / kChunkSteps;
@@ -335,7 +335,7 @@ int k2d_default_config(k2d_config *cfg, int32_t n_envs, int32_t n_polygons, int3
     cfg->n_envs = n_envs; cfg->n_polygons = n_polygons; cfg->n_circles = n_circles; cfg->n_joints = n_joints; cfg->n_thrusters = n_thrusters;
     cfg->n_actions = n_joints + n_thrusters > 0 ? n_joints + n_thrusters : 1;
     cfg->n_levels = n_envs;
-    cfg->solver_iters = 8; cfg->warm_start = 1; cfg->auto_reset = K2D_RESET_NONE; cfg->max_episode_steps = 0; cfg->max_fused_steps = 64;
+    cfg->solver_iters = 8; cfg->warm_start = 1; cfg->auto_reset = K2D_RESET_NONE; cfg->max_episode_steps = 0; cfg->max_fused_steps = 64; cfg->frame_skip = 1;
     cfg->dt = 1.0f / 60.0f; cfg->gravity_y = -9.81f;
     cfg->contact_alpha = 6.0f; cfg->contact_beta = 0.1f; cfg->slop = 0.005f; cfg->restitution_threshold = 1.0f; cfg->face_tol = 1e-3f;
     cfg->joint_alpha = 6.0f; cfg->joint_beta = 0.1f; cfg->joint_gamma = 6.0f; cfg->motor_rho = 1.0f; cfg->aabb_margin = 0.01f;

@@ -149,6 +149,7 @@ struct StepParams {
     int chunk_steps, n_chunks;   // a launch is cut into n_chunks pieces of chunk_steps steps; work items are (chunk, env)
     int solver_iters, warm_start, auto_reset, max_episode_steps;
     int discrete;             // actions are int32 codes (multi-discrete action space) instead of floats
+    int frame_skip;           // engine steps each action row is held for
     float dense_kappa;        // coefficient of the dense reward (0 = off)
     float dt, gdt, contact_alpha, contact_beta, slop, rest_thr, face_tol, joint_alpha, joint_beta, joint_gamma, motor_rho, aabb_margin;
     unsigned long long seed;
@@ -1058,8 +1059,9 @@ struct Scene {
         // dense reward: distance between the first green and the first blue shape before the step
         if (prm.dense_kappa != 0.0f && lane == 0) sm[SC::META + META_D0] = green_blue_distance();
         // actions of this step
-        if (lane < prm.n_actions) sm[SC::ACT + lane] = prm.actions[((size_t)s * prm.n_envs + e) * prm.n_actions + lane];
-        if (G < kMaxActions && lane + G < prm.n_actions) sm[SC::ACT + lane + G] = prm.actions[((size_t)s * prm.n_envs + e) * prm.n_actions + lane + G];
+        const float *act_row = prm.actions + ((size_t)(s / prm.frame_skip) * prm.n_envs + e) * prm.n_actions;
+        if (lane < prm.n_actions) sm[SC::ACT + lane] = act_row[lane];
+        if (G < kMaxActions && lane + G < prm.n_actions) sm[SC::ACT + lane + G] = act_row[lane + G];
         // gravity, rotation, circle boxes
         for (int i = lane; i < SC::N; i += G) {
             const uint32_t fl = smu[SC::BFL + i];

@@ -27,7 +27,7 @@ EXPORTS = (
 class Config(C.Structure):
     _fields_ = (
         [(n, C.c_int32) for n in ("n_envs", "n_polygons", "n_circles", "n_joints", "n_thrusters", "n_actions", "n_levels",
-                                  "solver_iters", "warm_start", "auto_reset", "max_episode_steps", "max_fused_steps")] +
+                                  "solver_iters", "warm_start", "auto_reset", "max_episode_steps", "max_fused_steps", "frame_skip")] +
         [(n, C.c_float) for n in ("dt", "gravity_y", "contact_alpha", "contact_beta", "slop", "restitution_threshold",
                                   "face_tol", "joint_alpha", "joint_beta", "motor_rho", "aabb_margin", "joint_gamma", "dense_kappa")] +
         [("seed", C.c_uint64), ("env_offset", C.c_int64), ("device", C.c_int32), ("lanes_per_scene", C.c_int32),
@@ -167,7 +167,7 @@ class Env:
         ids = None if level_ids is None else np.ascontiguousarray(level_ids, np.int32)
         _check(self.lib.k2d_reset(self._h, None if ids is None else ids.ctypes.data), "k2d_reset")
 
-    def step(self, actions, reward=None, done=None, static_scratch=False):
+    def step(self, actions, reward=None, done=None, static_scratch=False, n_steps=None):
         """actions: CUDA float32 [n_steps, n_envs, n_actions]; returns (reward, done) CUDA tensors [n_steps, n_envs].
 
         ``static_scratch=True`` goes through k2d_step_static_scratch: same results, but the records of
@@ -179,8 +179,9 @@ class Env:
         assert not (discrete and static_scratch)
         if actions.dim() == 2:
             actions = actions.unsqueeze(0)
-        n_steps = actions.shape[0]
-        assert tuple(actions.shape) == (n_steps, self.n_envs, self.n_actions), tuple(actions.shape)
+        fs = max(1, int(self.cfg.frame_skip))
+        n_steps = actions.shape[0] * fs if n_steps is None else int(n_steps)      # every action row is held for frame_skip steps
+        assert tuple(actions.shape) == (-(-n_steps // fs), self.n_envs, self.n_actions), tuple(actions.shape)
         if reward is None:
             reward = torch.empty((n_steps, self.n_envs), dtype=torch.float32, device=self.device)
         if done is None:

@@ -359,3 +359,16 @@ def test_status_reports_a_wait_that_ran_out_and_reset_clears_it():
         env.status()
     env.reset()
     assert env.status().sum() == 0
+
+
+def test_frame_skip_matches_the_oracle():
+    n_envs = 64
+    lv = scenes.make_levels("L", n_envs, 97, static_prob=0.1)
+    env, ref = parity.make_pair(lv, n_envs, frame_skip=2, auto_reset=2, max_episode_steps=9, seed=2)
+    import torch
+    rows = scenes.make_actions(20, n_envs, env.n_actions, 97)
+    r_ref, d_ref = ref.step(rows, n_steps=39)                         # the last row is held for one step only
+    r, d = env.step(torch.from_numpy(rows).cuda(), n_steps=39)
+    assert np.array_equal(r.cpu().numpy(), r_ref) and np.array_equal(d.cpu().numpy(), d_ref)
+    err, exact = parity.errors(env, ref)
+    assert exact, err

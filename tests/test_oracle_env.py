@@ -289,3 +289,17 @@ def test_oracle_trajectories_have_not_changed():
     spec.loader.exec_module(mod)
     stored = [ln.strip() for ln in open(os.path.join(here, "golden", "oracle_trajectories.txt")) if ln.strip() and not ln.startswith("#")]
     assert mod.lines() == stored
+
+
+def test_frame_skip_holds_every_action_row():
+    # paper, hyperparameter table: frame skip 2.  Holding a row for k steps equals repeating it k times.
+    lv = _motor_and_thruster_level()
+    rng = np.random.default_rng(3)
+    rows = rng.uniform(-1, 1, (4, 1, 2)).astype(np.float32)
+    held = k2d_ref.RefSim(lv, 1, frame_skip=3)
+    rep = k2d_ref.RefSim(lv, 1)
+    rh, dh = held.step(rows[:3], n_steps=8)               # 3 + 3 + 2 steps
+    rr, dr = rep.step(np.repeat(rows[:3], 3, axis=0)[:8])
+    assert np.array_equal(rh, rr) and np.array_equal(dh, dr) and rh.shape == (8, 1)
+    for k in ("pos", "angle", "vel", "angvel"):
+        assert np.array_equal(getattr(held, k), getattr(rep, k)), k
