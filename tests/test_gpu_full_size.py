@@ -48,3 +48,17 @@ def test_a_few_more_envs_than_resident_groups(lanes, n_envs):
     err, exact = parity.errors(env, ref)
     assert exact, err
     assert np.array_equal(env.status(), ref.counters)       # also says that no wait ran out
+
+
+def test_a_thousand_steps_stay_bit_identical():
+    # long horizon: 1024 L envs x 1024 steps with pool resets, fixed joints, limits and a dense reward
+    seed = 123
+    lv = scenes.make_levels("L", 128, seed, static_prob=0.1, triangle_prob=0.2, fixed_prob=0.15, limit_prob=0.25)
+    n_envs = 1024
+    env, ref = parity.make_pair(lv, n_envs, auto_reset=2, max_episode_steps=300, seed=seed, dense_kappa=0.1, max_fused_steps=64)
+    act = scenes.make_actions(1024, n_envs, env.n_actions, seed)
+    (r, d), (rr, dr) = parity.step_both(env, ref, act, chunk=64, n_threads=os.cpu_count() or 1)
+    assert np.array_equal(r.view(np.uint32), rr.view(np.uint32)) and np.array_equal(d, dr)
+    err, exact = parity.errors(env, ref)
+    assert exact, err
+    assert np.array_equal(env.status(), ref.counters) and ref.counters[0] == 0      # and nothing went non-finite
