@@ -17,7 +17,10 @@
  *    handle; it never allocates or frees device memory.  k2d_step and k2d_obs are asynchronous
  *    on the stream given in the config; k2d_create, k2d_reset, k2d_get_state, k2d_set_state
  *    and k2d_status synchronise that stream.
- *  - "dev_" pointers are device memory, 16-byte aligned; "host_" pointers are host memory.
+ *  - "dev_" pointers are device memory on the config's device; the state buffer and the level pool
+ *    must be 16-byte aligned, every other device pointer 4-byte aligned.  "host_" pointers are host
+ *    memory.  Every call that touches the device makes the config's device current (cudaSetDevice)
+ *    and leaves it current, so handles on several devices can be used from one thread.
  *  - Shape index inside a scene: polygons 0 .. n_polygons-1, then circles.  Pair order (used by
  *    the solver and by the accumulated-impulse slots): polygon-polygon pairs (i<j,
  *    lexicographic), polygon-circle pairs (polygon major), circle-circle pairs (i<j);
@@ -38,7 +41,7 @@ extern "C" {
 #define K2D_OK 0
 #define K2D_ERR_NULL (-1)          /* a required pointer is null                         */
 #define K2D_ERR_CONFIG (-2)        /* a config field is out of range                     */
-#define K2D_ERR_ALIGN (-3)         /* a device pointer is not 16-byte aligned            */
+#define K2D_ERR_ALIGN (-3)         /* a device pointer is not aligned as required        */
 #define K2D_ERR_LEVEL (-4)         /* level data invalid (non-finite, bad index, ...)    */
 #define K2D_ERR_STEPS (-5)         /* n_steps < 1 or > max_fused_steps                   */
 #define K2D_ERR_CUDA (-6)          /* a CUDA runtime call failed                         */
@@ -138,6 +141,10 @@ int k2d_default_config(k2d_config *cfg, int32_t n_envs, int32_t n_polygons, int3
  * Host-only; 0 on an invalid config. */
 size_t k2d_state_bytes(const k2d_config *cfg);
 size_t k2d_level_pool_bytes(const k2d_config *cfg);
+/* The state buffer without its overflow-scratch tail, which is its last part: what a caller who steps only
+ * through k2d_step_static_scratch (below) has to provide.  A handle created over a buffer of this size must
+ * never be given to k2d_step or k2d_step_discrete, which write the tail.  Host-only; 0 on an invalid config. */
+size_t k2d_state_bytes_no_scratch(const k2d_config *cfg);
 
 /* Validates the config and the n_levels host levels, derives mass properties and the pair
  * collision mask (joined shapes do not collide: paper, "Joints"), uploads the level pool to
@@ -163,7 +170,7 @@ int k2d_step(k2d_state *s, const float *dev_actions, int32_t n_steps, float *dev
 
 /* The same step with the paper's multi-discrete action space ("Action Space": every motor and
  * thruster is inactive or at maximum power, motors forwards or backwards): dev_actions is
- * [n_steps][n_envs][n_actions] int32 codes; a motor reads 0 = off, 1 = forwards (+1), 2 = backwards
+ * [ceil(n_steps / frame_skip)][n_envs][n_actions] int32 codes (one row per frame_skip steps, as for k2d_step); a motor reads 0 = off, 1 = forwards (+1), 2 = backwards
  * (-1), anything else off; a thruster reads 0 = off, anything else on. */
 int k2d_step_discrete(k2d_state *s, const int32_t *dev_actions, int32_t n_steps, float *dev_reward, uint8_t *dev_done);
 

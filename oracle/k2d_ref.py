@@ -152,7 +152,7 @@ class RefSim:
         self.pair_slot = _as(v.pair_slot, (self.n_pairs,), np.int32)
         self.collide = _as(v.collide, (L, self.n_pairs), np.uint8)
         self.counters = _as(v.counters, (8,), np.int64)
-        self.n_envs, self.n_actions = E, J + T
+        self.n_envs, self.n_actions = E, int(full["n_actions"])
         self.obs_floats = self.lib.k2d_ref_obs_floats(C.byref(self._c))
 
     def __del__(self):

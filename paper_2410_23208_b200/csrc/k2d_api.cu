@@ -348,6 +348,12 @@ size_t k2d_state_bytes(const k2d_config *cfg) {
     return buffer_layout(cfg, ci).total;
 }
 
+size_t k2d_state_bytes_no_scratch(const k2d_config *cfg) {
+    ClassInfo ci;
+    if (check_config(cfg) != K2D_OK || !pick_class(cfg, &ci)) return 0;
+    return buffer_layout(cfg, ci).scratch_off;
+}
+
 size_t k2d_level_pool_bytes(const k2d_config *cfg) {
     ClassInfo ci;
     if (check_config(cfg) != K2D_OK || !pick_class(cfg, &ci)) return 0;
@@ -441,6 +447,7 @@ int k2d_step(k2d_state *s, const float *dev_actions, int32_t n_steps, float *dev
     if (!s || !dev_actions || !dev_reward || !dev_done) return K2D_ERR_NULL;
     if (n_steps < 1 || n_steps > s->cfg.max_fused_steps) return K2D_ERR_STEPS;
     if (((uintptr_t)dev_actions & 3) || ((uintptr_t)dev_reward & 3)) return K2D_ERR_ALIGN;
+    CUDA_OK(cudaSetDevice(s->cfg.device));
     const StepParams prm = step_params(s, dev_actions, n_steps, dev_reward, dev_done, s->dev_scratch);
     CUDA_OK(K2D_DISPATCH(launch_step, s, s, prm));
     return K2D_OK;
@@ -449,6 +456,7 @@ int k2d_step(k2d_state *s, const float *dev_actions, int32_t n_steps, float *dev
 int k2d_obs(k2d_state *s, float *dev_obs) {
     if (!s || !dev_obs) return K2D_ERR_NULL;
     if ((uintptr_t)dev_obs & 3) return K2D_ERR_ALIGN;
+    CUDA_OK(cudaSetDevice(s->cfg.device));
     CUDA_OK(s->ci.id == 0 ? launch_obs<ClassS>(s, dev_obs) : s->ci.id == 1 ? launch_obs<ClassM>(s, dev_obs) : launch_obs<ClassL>(s, dev_obs));
     return K2D_OK;
 }
@@ -456,6 +464,7 @@ int k2d_obs(k2d_state *s, float *dev_obs) {
 int k2d_render(k2d_state *s, uint8_t *dev_pixels) {
     if (!s || !dev_pixels) return K2D_ERR_NULL;
     if ((uintptr_t)dev_pixels & 3) return K2D_ERR_ALIGN;
+    CUDA_OK(cudaSetDevice(s->cfg.device));
     const int E = s->cfg.n_envs;
     uint32_t *out = reinterpret_cast<uint32_t *>(dev_pixels);
     if (s->ci.id == 0) k2d_render_kernel<ClassS><<<E, kRenderThreads, 0, s->stream>>>(s->dev_env, s->dev_levels, out, E);
@@ -616,6 +625,7 @@ int k2d_step_discrete(k2d_state *s, const int32_t *dev_actions, int32_t n_steps,
     if (!s || !dev_actions || !dev_reward || !dev_done) return K2D_ERR_NULL;
     if (n_steps < 1 || n_steps > s->cfg.max_fused_steps) return K2D_ERR_STEPS;
     if (((uintptr_t)dev_actions & 3) || ((uintptr_t)dev_reward & 3)) return K2D_ERR_ALIGN;
+    CUDA_OK(cudaSetDevice(s->cfg.device));
     const StepParams prm = step_params(s, reinterpret_cast<const float *>(dev_actions), n_steps, dev_reward, dev_done, s->dev_scratch, 1);
     CUDA_OK(K2D_DISPATCH(launch_step, s, s, prm));
     return K2D_OK;

@@ -17,7 +17,7 @@ MAX_POLYGONS, MAX_CIRCLES, MAX_SHAPES, MAX_JOINTS, MAX_THRUSTERS = 12, 4, 16, 6,
 RESET_NONE, RESET_SAME_LEVEL, RESET_POOL = 0, 1, 2
 
 EXPORTS = (
-    "k2d_default_config", "k2d_state_bytes", "k2d_level_pool_bytes", "k2d_create", "k2d_reset", "k2d_step",
+    "k2d_default_config", "k2d_state_bytes", "k2d_state_bytes_no_scratch", "k2d_level_pool_bytes", "k2d_create", "k2d_reset", "k2d_step",
     "k2d_step_discrete", "k2d_step_static_scratch", "k2d_obs", "k2d_render",
     "k2d_obs_floats", "k2d_canonical_words", "k2d_get_state", "k2d_set_state", "k2d_status", "k2d_level_info",
     "k2d_set_trace", "k2d_trace_slots", "k2d_eval_sincos_tanh", "k2d_error_string", "k2d_destroy",
@@ -64,6 +64,8 @@ def load_library():
         lib.k2d_default_config.argtypes = [C.POINTER(Config), i32, i32, i32, i32, i32]
         lib.k2d_state_bytes.argtypes = [C.POINTER(Config)]
         lib.k2d_state_bytes.restype = C.c_size_t
+        lib.k2d_state_bytes_no_scratch.argtypes = [C.POINTER(Config)]
+        lib.k2d_state_bytes_no_scratch.restype = C.c_size_t
         lib.k2d_level_pool_bytes.argtypes = [C.POINTER(Config)]
         lib.k2d_level_pool_bytes.restype = C.c_size_t
         lib.k2d_create.argtypes = [C.POINTER(Config), vp, vp, vp, C.POINTER(vp)]

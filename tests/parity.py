@@ -13,15 +13,28 @@ META_KEYS = ("step_count", "episode_count", "level_id", "status")
 
 ORACLE_CFG = ("solver_iters", "warm_start", "auto_reset", "max_episode_steps", "dt", "gravity_y", "contact_alpha",
               "contact_beta", "slop", "restitution_threshold", "face_tol", "joint_alpha", "joint_beta", "joint_gamma", "motor_rho",
-              "aabb_margin", "dense_kappa", "seed", "env_offset", "frame_skip")
+              "aabb_margin", "dense_kappa", "seed", "env_offset", "frame_skip", "n_actions")
 
 
-def make_pair(levels, n_envs, **cfg):
-    """(Env on cuda:0, RefSim) with the same configuration."""
+def make_pair(levels, n_envs, broadphase=0, **cfg):
+    """(Env on cuda:0, RefSim) with the same configuration.  The oracle runs the narrowphase on every pair that
+    may collide (``broadphase=0``): the library's bounding-box test in front of its narrowphase is thereby checked
+    against a reference that has no such test.  ``broadphase=1`` gives the oracle the same test, which makes its
+    counters of pairs past the test comparable too."""
     env = k2d.Env(levels, n_envs, **cfg)
     ocfg = {k: getattr(env.cfg, k) for k in ORACLE_CFG}
-    ref = k2d_ref.RefSim(levels, n_envs, **ocfg)
+    ref = k2d_ref.RefSim(levels, n_envs, broadphase=broadphase, **ocfg)
     return env, ref
+
+
+def counters_match(env, ref) -> bool:
+    """k2d_status against the oracle's counters; the three counts of pairs past the bounding-box test only when the
+    oracle runs that test"""
+    got, want = env.status(), ref.counters
+    keep = np.ones(8, bool)
+    if not ref.cfg["broadphase"]:
+        keep[4:7] = False
+    return bool(np.array_equal(got[keep], want[keep]))
 
 
 def errors(env, ref):

@@ -27,13 +27,20 @@ def _crowded_levels(n_levels, seed):
     return lv
 
 
-def test_static_scratch_step_equals_step_on_two_calls_in_a_row():
+@pytest.mark.parametrize("lanes", [32, 16])
+def test_static_scratch_step_equals_step_on_two_calls_in_a_row(lanes):
+    import ctypes
     import torch
     n_envs = 24
     calls = ((0, 1), (1, 7))     # action rows of the first call (one step, the pile at its densest) and of the second
     lv = _crowded_levels(n_envs, 77)
-    a = k2d.Env(lv, n_envs)
-    b = k2d.Env(lv, n_envs)
+    a = k2d.Env(lv, n_envs, lanes_per_scene=lanes)
+    b = k2d.Env(lv, n_envs, lanes_per_scene=lanes)
+    # the variant must leave the scratch tail of its state buffer alone: the tail is filled with a pattern here and
+    # looked at again after every call
+    tail = a.lib.k2d_state_bytes_no_scratch(ctypes.byref(b.cfg))
+    assert 0 < tail < b.state_buf.numel()
+    b.state_buf[tail:] = 0xA5
     trace = a.enable_trace()
     act = scenes.make_actions(calls[-1][1], n_envs, a.n_actions, 77)
     for call, (lo, hi) in enumerate(calls):
@@ -41,11 +48,12 @@ def test_static_scratch_step_equals_step_on_two_calls_in_a_row():
         ra, da = a.step(x)
         rb, db = b.step(x, static_scratch=True)
         torch.cuda.synchronize()
-        # touching pairs in the latest step: 66 polygon pairs own two manifold slots each, the others one;
-        # beyond 32 of them the records go to the scratch
+        # touching pairs in the latest step: 66 polygon pairs own two manifold slots each, the others one.  A scene keeps
+        # the records of its first lanes + lanes / 2 touching pairs on chip; with more, all of the step's records go
+        # through the scratch, which is what the first call must reach
         on = trace.cpu().numpy()[:, :, 5] > 0
         pairs = (on[:, :132:2] | on[:, 1:132:2]).sum(1) + on[:, 132:].sum(1)
-        assert call > 0 or pairs.max() > 32, pairs
+        assert call > 0 or pairs.max() > lanes + lanes // 2, pairs
         assert torch.equal(ra, rb) and torch.equal(da, db)
         sa, sb = a.get_state(), b.get_state()
         for key in parity.STATE_KEYS:
@@ -53,6 +61,7 @@ def test_static_scratch_step_equals_step_on_two_calls_in_a_row():
         for key in parity.META_KEYS:
             assert np.array_equal(sa[key], sb[key]), (call, key)
         assert np.array_equal(a.status(), b.status())
+        assert bool((b.state_buf[tail:] == 0xA5).all())
 
 
 def test_static_scratch_step_refuses_more_envs_than_its_array_holds():
