@@ -1,21 +1,29 @@
 // k2d_kernels.cuh -- device code of the batched 2D rigid-body environment step (sm_100a).
 //
-// One group of G lanes (G = 16: two scenes per warp; 32: one warp per scene; 8: four scenes per warp)
-// owns one scene.  A group takes work items (a run of consecutive steps of one env) from a ticket queue;
-// for an item it loads the scene's state from memory once, keeps it in shared memory (bodies, joint rows,
-// world-frame geometry) and in registers (the contact pair record of every lane) across the item's steps,
-// and writes it back once.  Within a step the lanes of the group work on bodies, polygon vertices, shape
-// pairs (bounding-box test, narrowphase), contact pair records (one per lane) and joints (one per lane).
+// One engine step of every env is two kernel launches.
+//
+//   k2d_prep_kernel   A group of G lanes (G = 16: two scenes per warp; 32: one warp per scene; 8: four per warp)
+//                     takes one scene at a time from a ticket queue.  Its lanes work on bodies, polygon vertices,
+//                     shape pairs (bounding-box test, narrowphase) and contact manifolds (one per lane): gravity,
+//                     world-frame geometry, motors, thrusters, joint pre-step, manifolds, touch flags, and the
+//                     pre-step of every active manifold.  It leaves the step's constraint rows (one 80-byte row per
+//                     active manifold, in canonical order, and one 96-byte row per joint) in the env's scratch
+//                     area and the velocities in the env's state record.
+//   k2d_solve_kernel  One thread per env walks that env's rows strictly in the canonical order (warm start, solver
+//                     iterations of joints then contacts, Euler step, positional corrections), then does the
+//                     reward, the termination and the auto-reset.  The velocities of the env's bodies sit in shared
+//                     memory as one 16-byte group per (body, thread), which no two threads of a warp share a bank
+//                     for, whatever body each of them addresses.
+//
+// The sequential-impulse solver is a chain of dependent rows per scene, so a scene offers little to the lanes of a
+// warp; 32 scenes side by side offer 32 independent chains.  The geometry of a scene, on the other hand, is wide
+// (120 pairs to test for the largest size class) and needs its working set in shared memory, which is why that
+// part keeps several lanes per scene.
 //
 // Arithmetic contract: every +,-,*,/,sqrt is an individually rounded IEEE binary32 operation
 // (the file is compiled with --fmad=false --prec-div=true --prec-sqrt=true --ftz=false), a fused
-// multiply-add appears only where the code says __fmaf_rn, and min/max are comparisons.  The
-// sequential-impulse solver keeps the canonical constraint order (joints, then contacts by pair
-// index) by "level scheduling": a row's level is one more than the highest level of an earlier
-// row that shares a movable body with it, rows of one level touch disjoint movable bodies and
-// run on different lanes at once, and levels run in order -- every body sees exactly the
-// sequence of updates a one-row-at-a-time sweep would give it, so results are bit-identical to
-// that sweep.
+// multiply-add appears only where the code says __fmaf_rn, and min/max are comparisons.  The solver visits
+// the rows one after the other in the canonical order (joints by index, then manifolds by pair index and slot).
 #pragma once
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -27,17 +35,20 @@ namespace k2d {
 #endif
 constexpr int kBlockThreads = K2D_BLOCK_THREADS;
 #ifndef K2D_MIN_BLOCKS
-#define K2D_MIN_BLOCKS 5
+#define K2D_MIN_BLOCKS 6
 #endif
-constexpr int kMinBlocks = K2D_MIN_BLOCKS;   // resident blocks per SM the step kernel is compiled for (bounds its registers)
+constexpr int kMinBlocks = K2D_MIN_BLOCKS;   // resident blocks per SM the prep kernel is compiled for (bounds its registers)
+#ifndef K2D_SOLVE_THREADS
+#define K2D_SOLVE_THREADS 32
+#endif
+constexpr int kSolveThreads = K2D_SOLVE_THREADS;   // solve kernel: one env per thread
 constexpr int kObsThreads = 128;   // observation kernel: one warp per env, four envs per block
 constexpr int kMaxActions = 16;
-enum { Q_TICKET = 0, Q_LEFT = 1, Q_ERROR = 2 };
-constexpr unsigned kWaitLimit = 1u << 24;   // polls (about 100 ns apart) before a wait for another group's chunk gives up
-constexpr int kRecWords = 24;   // contact pair record
-constexpr int kWarmWords = 5;   // pair index + 4 accumulated impulses
+enum { Q_TICKET = 0, Q_LEFT = 1 };
+constexpr int kRowWords = 20;   // one active manifold: five 16-byte groups
+constexpr int kWarmWords = 3;   // slot key, accumulated normal and tangent impulse
 constexpr int kStageWords = 9;  // packed pair word, normal, two contact points with penetration
-constexpr int kJointWords = 24; // joint row kept in shared memory: six 16-byte groups
+constexpr int kJointWords = 24; // joint row: six 16-byte groups
 constexpr int kJointLevelWords = 12;  // joint record of a level
 
 // ---------------------------------------------------------------- size classes and layouts
@@ -59,14 +70,17 @@ struct SizeClass {
     static constexpr int LV_MASK = LV_THR + 8 * T;
     static constexpr int LV_GB = LV_MASK + MASKW;        // first green shape | first blue shape << 8 | both exist << 16
     static constexpr int LV_WORDS = (LV_GB + 1 + 3) / 4 * 4;
-    // state record: bodies (same order as shared memory), joint impulses, meta, warm list
-    static constexpr int ST_BODY = 0, ST_JACC = 6 * N, ST_META = ST_JACC + 3 * J, ST_WARM = ST_META + 8;
-    static constexpr int ST_WORDS = (ST_WARM + kWarmWords * NPAIRS + 3) / 4 * 4;
-    // A scene with more touching pairs than lanes takes the step's contact solve through global
-    // scratch: one memory record and one warm entry per pair.
-    static constexpr int SCRATCH_WORDS = NPAIRS * (kRecWords + kWarmWords);
-    static constexpr int SCRATCH_WARM = NPAIRS * kRecWords;
-    // shared memory region of one scene (words)
+    // state record of an env: per body the 16-byte groups (x, y, angle, -) and (vx, vy, angular velocity, -), meta,
+    // accumulated joint impulses, and the accumulated impulses of the manifolds that were active in the latest step
+    static constexpr int ST_POS = 0, ST_VEL = 4 * N, ST_META = 8 * N, ST_JACC = ST_META + 8;
+    static constexpr int ST_WARM = (ST_JACC + 3 * J + 3) / 4 * 4;
+    static constexpr int ST_WORDS = (ST_WARM + kWarmWords * NSLOTS + 3) / 4 * 4;
+    // scratch of an env, valid from the prep kernel of a step to its solve kernel: manifold rows, then joint rows.
+    // Room for two rows per pair: a pair staged beyond the first G of a scene waits in the row slot 2 k + 1.
+    static constexpr int ROW_CAP = 2 * NPAIRS;
+    static constexpr int SCR_ROWS = 0, SCR_JROW = ROW_CAP * kRowWords;
+    static constexpr int SCRATCH_WORDS = SCR_JROW + kJointWords * J;
+    // shared memory region of one scene in the prep kernel (words)
     // per body 16-byte groups (x, y, angle, -) and (vx, vy, angular velocity, -), then per-body arrays
     static constexpr int BPOS = 0, BVEL = 4 * N;
     static constexpr int BIM = 8 * N, BII = 9 * N, BFR = 10 * N, BRE = 11 * N, BC = 12 * N, BS = 13 * N, BFL = 14 * N;
@@ -75,54 +89,38 @@ struct SizeClass {
     static constexpr int BOX = (WOFF + P4 + 3) / 4 * 4;  // N x (min x, min y, max x, max y), 16-byte aligned
     static constexpr int MASK = BOX + 4 * N;
     static constexpr int ACT = MASK + MASKW;
-    static constexpr int META = ACT + kMaxActions;       // step_count, episode_count, level_id, status, warm entries
-    static constexpr int JROW = (META + 8 + 3) / 4 * 4;  // J rows of kJointWords, 16-byte aligned
-    static constexpr int LVC = JROW + kJointWords * J;   // copy of the level record's edge lengths, joint and thruster records
-    static constexpr int LVC_WORDS = LV_MASK - LV_ELEN;
-    static constexpr int SURV = LVC + LVC_WORDS;         // bytes: pairs that passed the box test
-    static constexpr int WIDX = SURV + ((NPAIRS + 3) / 4 > N ? (NPAIRS + 3) / 4 : N); // bytes: pair -> record index of the previous step (the survivor area is reused as N words)
-    // then, per lane of the group (field-major, G words per field):
-    //   STG  kStageWords fields: manifolds on their way to the owning lane; afterwards the second manifold's constants
-    //   ACC2 2 fields: accumulated impulses of the second manifold
-    // (the positional corrections of a lane's record, 2 x G words, reuse the world-frame vertex arrays after the narrowphase)
-    // then kRecWords fields of G / 2 words: second records of the lower half of the lanes
-    static constexpr int STG = WIDX + (NPAIRS + 3) / 4;
-    static constexpr int LANE_FIELDS = kStageWords + 2;
+    static constexpr int META = ACT + kMaxActions;       // the state record's meta words
+    static constexpr int ELEN = (META + 8 + 3) / 4 * 4;  // edge lengths of the level's polygons
+    static constexpr int SURV = ELEN + P4;               // bytes: pairs that passed the box test
+    static constexpr int WIDX = SURV + (NPAIRS + 3) / 4; // bytes: manifold slot key -> entry of the previous step's warm list
+    // then, per lane of the group (field-major, G words per field): kStageWords fields, manifolds on their way to the
+    // lane that builds their rows
+    static constexpr int STG = WIDX + (2 * NPAIRS + 3) / 4;
     static constexpr int PTAB_WORDS = ((NPAIRS + 1) / 2 + 3) / 4 * 4;  // block-shared pair table, 16 bits per pair
 };
-// memory form of a contact pair record (the overflow path keeps records in global scratch)
-enum { R_AB = 0, R_NX, R_NY, R_MU, R_M0 = 4 };
-enum { M_RNA = 0, M_RNB, M_RTA, M_RTB, M_MASSN, M_MASST, M_TARGET, M_CORR, M_ACCN, M_ACCT, M_WORDS };
-static_assert(R_M0 + 2 * M_WORDS == kRecWords, "record size");
+// manifold row (scratch): what the solver needs of one active manifold
+enum { R_AB = 0, R_NX, R_NY, R_MU, R_MA, R_MB, R_IA, R_IB, R_RNA, R_RNB, R_RTA, R_RTB, R_MASSN, R_MASST, R_TARGET, R_CORR,
+       R_ACCN, R_ACCT, R_KEY, R_PAD };
+static_assert(R_PAD + 1 == kRowWords, "row size");
+// row AB word: a | b<<5 | a movable<<10 | b movable<<11
 // staged manifold fields
 enum { S_AB = 0, S_NX, S_NY, S_PX0, S_PY0, S_PEN0, S_PX1, S_PY1, S_PEN1 };
 static_assert(S_PEN1 + 1 == kStageWords, "stage size");
-// second-manifold constants reuse the stage fields of the same lane
-enum { M2_RNA = 0, M2_RNB, M2_RTA, M2_RTB, M2_MASSN, M2_MASST, M2_TARGET };
-// per-lane fields after the stage fields
-enum { LF_ACC2N = kStageWords, LF_ACC2T, LF_COUNT };
-// The lower half of the lanes can hold a second record each (pair number G + lane of a crowded scene),
-// in memory form: kRecWords fields of G / 2 words after the per-lane fields.  Stage field f of such a
-// record waits in record field ovs(f), clear of the accumulated impulses.
-__host__ __device__ constexpr int ovs(int f) { return f < 3 ? f : f + 1; }
-constexpr int OV_ACC0N = R_M0 + M_ACCN, OV_ACC0T = R_M0 + M_ACCT, OV_ACC1N = R_M0 + M_WORDS + M_ACCN, OV_ACC1T = R_M0 + M_WORDS + M_ACCT;
+// staged AB word: a | b<<5 | active manifolds<<10 | pair<<12 | a movable<<26 | b movable<<27
 // joint row fields
-enum { JR_RAX = 0, JR_RAY, JR_RBX, JR_RBY, JR_I11, JR_I12, JR_I22, JR_PAD0, JR_BX, JR_BY, JR_CX, JR_CY, JR_MA, JR_MB, JR_IA, JR_IB,
+enum { JR_RAX = 0, JR_RAY, JR_RBX, JR_RBY, JR_I11, JR_I12, JR_I22, JR_JAB, JR_BX, JR_BY, JR_CX, JR_CY, JR_MA, JR_MB, JR_IA, JR_IB,
        JR_ACCX, JR_ACCY, JR_PAD1, JR_PAD2,
        JR_ANG, JR_KR, JR_BIASR, JR_ACCR };   // angular row: kind (0 none, 1 fixed, 2 beyond the upper limit, 3 beyond the lower), 1 / (1/I_a + 1/I_b), gamma x error, accumulated
 static_assert(JR_ACCR + 1 == kJointWords, "joint row size");
-enum { META_STEP = 0, META_EPISODE, META_LEVEL, META_STATUS, META_NWARM, META_GB, META_D0 };   // the last two: dense reward's shapes and distance before the step
+// meta words of a state record.  FLAGS, D0 and ACTIVE are messages from the prep kernel to the solve kernel of the same step:
+// touch flags (green-blue | green-red << 1), the dense reward's shapes (both exist << 2 | green << 8 | blue << 16) and their
+// distance before the step, and the bit mask of the shapes that exist.
+enum { META_STEP = 0, META_EPISODE, META_LEVEL, META_STATUS, META_NROWS, META_FLAGS, META_D0, META_ACTIVE };
 
-// shared-memory word of word i of a state record's body block (x[N], y[N], angle[N], vx[N], vy[N], w[N])
-template <class SC>
-__device__ __forceinline__ int body_word(int i) {
-    const int f = i / SC::N, b = i - f * SC::N;
-    return (f < 3 ? SC::BPOS + f : SC::BVEL + f - 3) + 4 * b;
-}
 // shared-memory words per scene: padded so that the groups of one warp start in different banks
 template <class SC, int G>
 __host__ __device__ constexpr int region_words() {
-    constexpr int raw = SC::STG + SC::LANE_FIELDS * G + kRecWords * (G / 2);
+    constexpr int raw = SC::STG + kStageWords * G;
     return G < 32 ? (raw - G + 31) / 32 * 32 + G : (raw + 3) / 4 * 4;
 }
 
@@ -132,24 +130,20 @@ __host__ __device__ inline uint32_t flag_role(uint32_t f) { return (f >> 2) & 3u
 __host__ __device__ inline uint32_t flag_nverts(uint32_t f) { return (f >> 4) & 7u; }
 // joint packed word: a | b<<8 | binding<<16 | on<<24 | level<<25 | active<<28 | a movable<<29 | b movable<<30 | fixed or limited<<31
 // thruster packed word: shape | binding<<8 | on<<16 | level<<17 | active<<20
-// record AB word: a | b<<5 | amask<<10 | pair<<12 | level<<19 | dynA<<26 | dynB<<27
 
 struct StepParams {
     uint32_t *state;
     const uint32_t *levels;
-    const float *actions;
-    float *reward;
+    const float *actions;      // the action row of this step, [n_envs][n_actions]
+    float *reward;             // this step's [n_envs]
     uint8_t *done;
     unsigned long long *counters;
-    unsigned int *queue;       // work queue words: next ticket, groups that have left, error flag
-    unsigned int *chunks_done; // per env: chunks of this launch already stepped (0 again when the launch is over)
-    uint32_t *scratch;
+    unsigned int *queue;       // work queue words of the prep kernel: next ticket, groups that have left
+    uint32_t *scratch;         // [n_envs][SCRATCH_WORDS]
     float *trace;
-    int n_envs, n_steps, n_actions, n_levels;
-    int chunk_steps, n_chunks;   // a launch is cut into n_chunks pieces of chunk_steps steps; work items are (chunk, env)
+    int n_envs, n_actions, n_levels;
     int solver_iters, warm_start, auto_reset, max_episode_steps;
     int discrete;             // actions are int32 codes (multi-discrete action space) instead of floats
-    int frame_skip;           // engine steps each action row is held for
     float dense_kappa;        // coefficient of the dense reward (0 = off)
     float dt, gdt, contact_alpha, contact_beta, slop, rest_thr, face_tol, joint_alpha, joint_beta, joint_gamma, motor_rho, aabb_margin;
     unsigned long long seed;
@@ -223,7 +217,6 @@ __device__ __forceinline__ unsigned long long mix64(unsigned long long z) {
     z ^= z >> 31;
     return z;
 }
-
 // ---------------------------------------------------------------- group of G lanes
 template <int G>
 struct Group {
@@ -251,24 +244,6 @@ struct Group {
 
 // one manifold as the narrowphase leaves it
 struct Manifold { float px, py, nx, ny, pen; };
-
-// What the lane that owns a contact pair record keeps in registers for the whole step: the pair
-// (packed word), the shared normal, the friction coefficient, the inverse masses and inertias of
-// the two bodies, and the first manifold's lever-arm cross products, effective masses, target
-// normal velocity and accumulated impulses.  The second manifold (polygon-polygon pairs only) is
-// in the lane's shared-memory fields.
-struct Rec {
-    uint32_t ab;
-    float nx, ny, mu, ma, mb, ia, ib;
-    float rna, rnb, rta, rtb, massn, masst, target, accn, acct;
-};
-// memory form (overflow path)
-struct RecM {
-    uint32_t ab;
-    float nx, ny, mu;
-    float rna[2], rnb[2], rta[2], rtb[2], massn[2], masst[2], target[2], corr[2], accn[2], acct[2];
-};
-
 struct ContactConsts { float slop, rest_thr, alpha, beta; };
 
 // ---- contact pre-step for one manifold of pair (a, b) with normal (nx, ny)
@@ -337,447 +312,19 @@ __device__ __forceinline__ void manifold_rows(float nx, float ny, float mu, floa
         vbx = __fmaf_rn(mb, px, vbx); vby = __fmaf_rn(mb, py, vby); wb = __fmaf_rn(wtb, dt_, wb);
     }
 }
-
-// positional correction of one pair: each active manifold moves the two bodies apart along the normal
-__device__ __forceinline__ void correct_pair(float *pos, int a, int b, unsigned amask, bool dyn_a, bool dyn_b,
-                                             float nx, float ny, float ma, float mb, float corr0, float corr1) {
-    float xa = pos[4 * a], ya = pos[4 * a + 1], xb = pos[4 * b], yb = pos[4 * b + 1];
-    if (amask & 1u) {
-        const float ca = ma * corr0, cb = mb * corr0;
-        xa = __fmaf_rn(-ca, nx, xa); ya = __fmaf_rn(-ca, ny, ya);
-        xb = __fmaf_rn(cb, nx, xb); yb = __fmaf_rn(cb, ny, yb);
-    }
-    if (amask & 2u) {
-        const float ca = ma * corr1, cb = mb * corr1;
-        xa = __fmaf_rn(-ca, nx, xa); ya = __fmaf_rn(-ca, ny, ya);
-        xb = __fmaf_rn(cb, nx, xb); yb = __fmaf_rn(cb, ny, yb);
-    }
-    if (dyn_a) { pos[4 * a] = xa; pos[4 * a + 1] = ya; }
-    if (dyn_b) { pos[4 * b] = xb; pos[4 * b + 1] = yb; }
-}
-
-// ---- angular row of a fixed joint or of a revolute joint beyond one of its limits (paper, "Fixed Joints",
-// "Joint Limits"): j_r = (w_a - w_b + correction) / (1/I_a + 1/I_b), a loses j_r / I_a, b gains j_r / I_b.  A fixed
-// joint's impulse is accumulated and warm-started; a limit only ever pushes back, applies no correction while the
-// joint is already returning, and is not accumulated.  Returns the two angular velocities.  Out of line: most
-// joints are plain revolute joints.
-template <int MODE>
-__device__ __noinline__ float2 angular_row(float *jr, float ia, float ib, float wa, float wb) {
-    const float4 ang4 = ld4(jr + JR_ANG);      // kind this step, inverse angular mass, correction, accumulated impulse
-    const int ang = __float_as_int(ang4.x);
-    if (ang == 0) return make_float2(wa, wb);
-    float lr;
-    if (MODE == 0) {
-        if (ang != 1) return make_float2(wa, wb);
-        lr = ang4.w;
-    } else {
-        const float wrel = wa - wb;
-        float v;
-        if (ang == 1) v = wrel + ang4.z;
-        else if (ang == 2) { v = (wrel < 0.0f) ? wrel : wrel + ang4.z; v = fmax_cmp(v, 0.0f); }
-        else { v = (wrel > 0.0f) ? wrel : wrel + ang4.z; v = fmin_cmp(v, 0.0f); }
-        lr = v * ang4.y;
-        if (ang == 1) jr[JR_ACCR] = ang4.w + lr;
-    }
-    return make_float2(__fmaf_rn(-lr, ia, wa), __fmaf_rn(lr, ib, wb));
-}
-
-// ---- joints; the row of joint j is in shared memory.  MODE 0: warm start, 1: solver iteration,
-// 2: positional correction, 3: motor
-template <class SC, int MODE>
-__device__ __forceinline__ void visit_joint(float *sm, uint32_t jab, int j, float motor_rho, int discrete = 0) {
-    const int a = jab & 255, b = (jab >> 8) & 255;
-    const bool dyn_a = (jab >> 29) & 1u, dyn_b = (jab >> 30) & 1u;
-    float *jr = sm + SC::JROW + kJointWords * j;
-    if (MODE == 3) {
-        const float av = sm[SC::ACT + ((jab >> 16) & 255)];
-        // paper, "Action Space": continuous in [-1, 1], or multi-discrete codes 0 off, 1 forwards, 2 backwards at full power
-        const float A = discrete ? (__float_as_int(av) == 1 ? 1.0f : (__float_as_int(av) == 2 ? -1.0f : 0.0f))
-                                 : fmax_cmp(fmin_cmp(av, 1.0f), -1.0f);
-        const float *jl = sm + SC::LVC + (SC::LV_JOINT - SC::LV_ELEN) + kJointLevelWords * j;
-        const float speed = jl[5], power = jl[6];
-        const float wa = sm[SC::BVEL + 4 * a + 2], wb = sm[SC::BVEL + 4 * b + 2];
-        const float arg = __fmaf_rn(-speed, A, wa - wb) * motor_rho;
-        const float jr_ = power * tanh_spec(arg);
-        if (dyn_a) sm[SC::BVEL + 4 * a + 2] = __fmaf_rn(-jr_, sm[SC::BII + a], wa);
-        if (dyn_b) sm[SC::BVEL + 4 * b + 2] = __fmaf_rn(jr_, sm[SC::BII + b], wb);
-        return;
-    }
-    const float4 mi4 = ld4(jr + JR_MA);       // inverse masses and inertias of the two bodies
-    const float ma = mi4.x, mb = mi4.y, ia = mi4.z, ib = mi4.w;
-    if (MODE == 2) {
-        const float cx = jr[JR_CX], cy = jr[JR_CY];
-        if (dyn_a) { sm[SC::BPOS + 4 * a] = __fmaf_rn(ma, cx, sm[SC::BPOS + 4 * a]); sm[SC::BPOS + 4 * a + 1] = __fmaf_rn(ma, cy, sm[SC::BPOS + 4 * a + 1]); }
-        if (dyn_b) { sm[SC::BPOS + 4 * b] = __fmaf_rn(-mb, cx, sm[SC::BPOS + 4 * b]); sm[SC::BPOS + 4 * b + 1] = __fmaf_rn(-mb, cy, sm[SC::BPOS + 4 * b + 1]); }
-        return;
-    }
-    const float4 r4 = ld4(jr + JR_RAX);
-    const float rax = r4.x, ray = r4.y, rbx = r4.z, rby = r4.w;
-    const float4 va4 = ld4(sm + SC::BVEL + 4 * a), vb4 = ld4(sm + SC::BVEL + 4 * b);
-    float vax = va4.x, vay = va4.y, wa = va4.z, vbx = vb4.x, vby = vb4.y, wb = vb4.z;
-    float lx, ly;
-    if (MODE == 0) { lx = jr[JR_ACCX]; ly = jr[JR_ACCY]; }
-    else {
-        const float4 k4 = ld4(jr + JR_I11), b4 = ld4(jr + JR_BX);
-        const float2 acc = *reinterpret_cast<const float2 *>(jr + JR_ACCX);
-        const float cx = __fmaf_rn(-wb, rby, vbx) - __fmaf_rn(-wa, ray, vax);
-        const float cy = __fmaf_rn(wb, rbx, vby) - __fmaf_rn(wa, rax, vay);
-        const float rx = -(cx + b4.x), ry = -(cy + b4.y);
-        const float i11 = k4.x, i12 = k4.y, i22 = k4.z;
-        lx = __fmaf_rn(i11, rx, i12 * ry);
-        ly = __fmaf_rn(i12, rx, i22 * ry);
-        *reinterpret_cast<float2 *>(jr + JR_ACCX) = make_float2(acc.x + lx, acc.y + ly);
-    }
-    wa = __fmaf_rn(-ia, cross2(rax, ray, lx, ly), wa);
-    wb = __fmaf_rn(ib, cross2(rbx, rby, lx, ly), wb);
-    if (jab >> 31) {      // fixed or limited joint: its angular row follows the point row
-        const float2 w2 = angular_row<MODE>(jr, ia, ib, wa, wb);
-        wa = w2.x; wb = w2.y;
-    }
-    if (dyn_a) st4(sm + SC::BVEL + 4 * a, __fmaf_rn(-ma, lx, vax), __fmaf_rn(-ma, ly, vay), wa);
-    if (dyn_b) st4(sm + SC::BVEL + 4 * b, __fmaf_rn(mb, lx, vbx), __fmaf_rn(mb, ly, vby), wb);
-}
-// joints of one level touch disjoint movable bodies; levels in order keep the joint order
-template <class SC, int G, int MODE>
-__device__ __forceinline__ void sweep_joints(float *sm, uint32_t jab, int lane, int jlevel, int jmax, float motor_rho,
-                                             int discrete = 0) {
-    const unsigned mask = Group<G>().mask;
-    if (SC::J == 0) return;
-#pragma unroll 1
-    for (int lvl = 1; lvl <= jmax; ++lvl) {
-        if (jlevel == lvl) visit_joint<SC, MODE>(sm, jab, lane, motor_rho, discrete);
-        __syncwarp(mask);
-    }
-}
-
-// Accumulated impulses that pair record `wi` of the previous step left behind (255: the pair was not
-// touching).  Records 0..G-1 live with lane wi (first manifold in its registers: old_n / old_t are the
-// calling lane's own, fetched across lanes here, so every lane of the group must call; second manifold
-// in its shared-memory fields), the next G / 2 records in the second-record fields of lane wi - G, later ones
-// in the warm entries of the global scratch.
-template <class SC, int G>
-__device__ __forceinline__ void warm_lookup(const Group<G> &g, const float *sm, const uint32_t *ovf, int wi, float old_n, float old_t,
-                                            int warm_start, float (&w)[4]) {
-    const int src = (wi < G) ? wi : 0;
-    const float *lf = sm + SC::STG;
-    w[0] = g.shflf(old_n, src); w[1] = g.shflf(old_t, src);
-    w[2] = lf[LF_ACC2N * G + src]; w[3] = lf[LF_ACC2T * G + src];
-    if (wi >= G && wi != 255) {
-        if (wi < G + G / 2) {
-            const float *o = lf + LF_COUNT * G + (wi - G);
-            w[0] = o[OV_ACC0N * (G / 2)]; w[1] = o[OV_ACC0T * (G / 2)]; w[2] = o[OV_ACC1N * (G / 2)]; w[3] = o[OV_ACC1T * (G / 2)];
-        } else {
-            const uint32_t *wr = ovf + SC::SCRATCH_WARM + (size_t)wi * kWarmWords;
-#pragma unroll
-            for (int q = 0; q < 4; ++q) w[q] = __uint_as_float(wr[1 + q]);
-        }
-    }
-    if (wi == 255 || !warm_start) { w[0] = 0.0f; w[1] = 0.0f; w[2] = 0.0f; w[3] = 0.0f; }
-}
-
-// Levels of nrec staged pairs by one lane with a per-body table (used when there are more pairs than
-// lanes): a pair's level is one more than the highest level of an earlier pair sharing a movable body.
-// The packed pair words of pairs 0..G-1 are in the stage fields, of the next G / 2 in the second-record
-// fields, of later ones in global scratch; the level goes into bits 19.. of each word.
-template <class SC, int G>
-__device__ __noinline__ int levels_by_one_lane(uint32_t *smu, uint32_t *ovf, int nrec) {
-    uint8_t *bl = reinterpret_cast<uint8_t *>(smu + SC::SURV);   // the survivor list is no longer needed
-    int cmax = 0;
-    for (int i = 0; i < SC::N; ++i) bl[i] = 0;
-    for (int k = 0; k < nrec; ++k) {
-        uint32_t *w = (k < G) ? (smu + SC::STG + S_AB * G + k)
-                    : (k < G + G / 2) ? (smu + SC::STG + LF_COUNT * G + ovs(S_AB) * (G / 2) + (k - G)) : (ovf + (size_t)k * kRecWords + S_AB);
-        const uint32_t ab = *w;
-        const int a = ab & 31, b = (ab >> 5) & 31;
-        int lvl = 1;
-        if ((ab >> 26) & 1u) lvl = max(lvl, bl[a] + 1);
-        if ((ab >> 27) & 1u) lvl = max(lvl, bl[b] + 1);
-        if ((ab >> 26) & 1u) bl[a] = (uint8_t)lvl;
-        if ((ab >> 27) & 1u) bl[b] = (uint8_t)lvl;
-        *w = ab | ((uint32_t)lvl << 19);
-        cmax = max(cmax, lvl);
-    }
-    return cmax;
-}
-
-// ================================================================ overflow path (cold code)
-// A scene with more touching pairs than lanes (nrec > G) solves this step's contacts from memory
-// records in global scratch, one loop over records per level, with the same row arithmetic.
-__device__ __forceinline__ void recm_load(const uint32_t *r, RecM &c) {
-    c.ab = r[R_AB]; c.nx = __uint_as_float(r[R_NX]); c.ny = __uint_as_float(r[R_NY]); c.mu = __uint_as_float(r[R_MU]);
-#pragma unroll
-    for (int mi = 0; mi < 2; ++mi) {
-        const uint32_t *m = r + R_M0 + mi * M_WORDS;
-        c.rna[mi] = __uint_as_float(m[M_RNA]); c.rnb[mi] = __uint_as_float(m[M_RNB]);
-        c.rta[mi] = __uint_as_float(m[M_RTA]); c.rtb[mi] = __uint_as_float(m[M_RTB]);
-        c.massn[mi] = __uint_as_float(m[M_MASSN]); c.masst[mi] = __uint_as_float(m[M_MASST]);
-        c.target[mi] = __uint_as_float(m[M_TARGET]); c.corr[mi] = __uint_as_float(m[M_CORR]);
-        c.accn[mi] = __uint_as_float(m[M_ACCN]); c.acct[mi] = __uint_as_float(m[M_ACCT]);
-    }
-}
-__device__ __forceinline__ void recm_store(uint32_t *r, const RecM &c) {
-    r[R_AB] = c.ab; r[R_NX] = __float_as_uint(c.nx); r[R_NY] = __float_as_uint(c.ny); r[R_MU] = __float_as_uint(c.mu);
-#pragma unroll
-    for (int mi = 0; mi < 2; ++mi) {
-        uint32_t *m = r + R_M0 + mi * M_WORDS;
-        m[M_RNA] = __float_as_uint(c.rna[mi]); m[M_RNB] = __float_as_uint(c.rnb[mi]);
-        m[M_RTA] = __float_as_uint(c.rta[mi]); m[M_RTB] = __float_as_uint(c.rtb[mi]);
-        m[M_MASSN] = __float_as_uint(c.massn[mi]); m[M_MASST] = __float_as_uint(c.masst[mi]);
-        m[M_TARGET] = __float_as_uint(c.target[mi]); m[M_CORR] = __float_as_uint(c.corr[mi]);
-        m[M_ACCN] = __float_as_uint(c.accn[mi]); m[M_ACCT] = __float_as_uint(c.acct[mi]);
-    }
-}
-
-template <class SC, int G, int MODE>
-__device__ __forceinline__ void slow_sweep_pairs(float *sm, uint32_t *ovf, int nrec, int cmax) {
-    Group<G> g;
-    for (int lvl = 1; lvl <= cmax; ++lvl) {
-        for (int k = g.lane; k < nrec; k += G) {
-            uint32_t *r = ovf + (size_t)k * kRecWords;
-            if (((r[R_AB] >> 19) & 127u) != (unsigned)lvl) continue;
-            RecM c;
-            recm_load(r, c);
-            const int a = c.ab & 31, b = (c.ab >> 5) & 31;
-            const unsigned amask = (c.ab >> 10) & 3u;
-            const bool dyn_a = (c.ab >> 26) & 1u, dyn_b = (c.ab >> 27) & 1u;
-            const float ma = sm[SC::BIM + a], mb = sm[SC::BIM + b];
-            if (MODE == 2) { correct_pair(sm + SC::BPOS, a, b, amask, dyn_a, dyn_b, c.nx, c.ny, ma, mb, c.corr[0], c.corr[1]); continue; }
-            const float ia = sm[SC::BII + a], ib = sm[SC::BII + b];
-            const float4 va4 = ld4(sm + SC::BVEL + 4 * a), vb4 = ld4(sm + SC::BVEL + 4 * b);
-            float vax = va4.x, vay = va4.y, wa = va4.z, vbx = vb4.x, vby = vb4.y, wb = vb4.z;
-#pragma unroll
-            for (int mi = 0; mi < 2; ++mi) {
-                if (amask & (1u << mi)) {
-                    manifold_rows<MODE>(c.nx, c.ny, c.mu, ma, mb, ia, ib, c.rna[mi], c.rnb[mi], c.rta[mi], c.rtb[mi], c.massn[mi], c.masst[mi],
-                                        c.target[mi], c.accn[mi], c.acct[mi], vax, vay, wa, vbx, vby, wb);
-                    if (MODE == 1) {
-                        r[R_M0 + mi * M_WORDS + M_ACCN] = __float_as_uint(c.accn[mi]);
-                        r[R_M0 + mi * M_WORDS + M_ACCT] = __float_as_uint(c.acct[mi]);
-                    }
-                }
-            }
-            if (dyn_a) st4(sm + SC::BVEL + 4 * a, vax, vay, wa);
-            if (dyn_b) st4(sm + SC::BVEL + 4 * b, vbx, vby, wb);
-        }
-        g.sync();
-    }
-}
-
-// Records from the staged manifolds (the first G in shared memory, the rest already in scratch),
-// their levels, warm start and all solver iterations, joints included.  old_n / old_t: this lane's
-// first-manifold accumulated impulses of the previous step.  Returns the highest contact level.
-template <class SC, int G>
-__device__ __noinline__ int slow_solve(float *sm, uint32_t *ovf, int nrec, uint32_t jab, int jlevel, int jmax,
-                                       int solver_iters, int warm_start, float motor_rho, float old_n, float old_t, ContactConsts cc) {
-    Group<G> g;
-    const int lane = g.lane;
-    uint32_t *smu = reinterpret_cast<uint32_t *>(sm);
-    const uint8_t *widx = reinterpret_cast<const uint8_t *>(smu + SC::WIDX);
-    int cmax = 0;
-    if (lane == 0) cmax = levels_by_one_lane<SC, G>(smu, ovf, nrec);
-    __threadfence_block();
-    g.sync();
-    cmax = g.shfl(cmax, 0);
-    // the staged manifolds of the first G + G / 2 pairs join the others in scratch
-    {
-        uint32_t *r = ovf + (size_t)lane * kRecWords, *r2 = ovf + (size_t)(G + lane) * kRecWords;
-#pragma unroll
-        for (int f = 0; f < kStageWords; ++f) {
-            r[f] = smu[SC::STG + f * G + lane];
-            if (lane < G / 2) r2[f] = smu[SC::STG + LF_COUNT * G + ovs(f) * (G / 2) + lane];
-        }
-    }
-    g.sync();
-    // pre-step of every pair; accumulated impulses of the previous step come from the lane that
-    // owned the pair then (first manifold in its registers, second in its shared-memory fields)
-    // or from the warm entries in scratch
-    for (int base = 0; base < nrec; base += G) {
-        const int k = base + lane;
-        const bool valid = k < nrec;
-        uint32_t *r = ovf + (size_t)(valid ? k : 0) * kRecWords;
-        uint32_t ab = 0u;
-        int wi = 255;
-        if (valid) { ab = r[S_AB]; wi = widx[(ab >> 12) & 127]; }
-        float w[4];
-        warm_lookup<SC, G>(g, sm, ovf, wi, old_n, old_t, warm_start, w);
-        if (valid) {
-            RecM c;
-            c.ab = ab; c.nx = __uint_as_float(r[S_NX]); c.ny = __uint_as_float(r[S_NY]);
-            const float pt[6] = { __uint_as_float(r[S_PX0]), __uint_as_float(r[S_PY0]), __uint_as_float(r[S_PEN0]),
-                                  __uint_as_float(r[S_PX1]), __uint_as_float(r[S_PY1]), __uint_as_float(r[S_PEN1]) };
-            const int a = ab & 31, b = (ab >> 5) & 31;
-            const float ma = sm[SC::BIM + a], mb = sm[SC::BIM + b], ia = sm[SC::BII + a], ib = sm[SC::BII + b];
-            const float fra = sm[SC::BFR + a], frb = sm[SC::BFR + b];
-            const float er = fmin_cmp(sm[SC::BRE + a], sm[SC::BRE + b]);
-            c.mu = sqrtf(__fmaf_rn(fra, fra, frb * frb));
-#pragma unroll
-            for (int mi = 0; mi < 2; ++mi) {
-                if ((ab >> 10) & (1u << mi)) {
-                    prestep_manifold<SC>(a, b, c.nx, c.ny, ma, mb, ia, ib, pt[3 * mi], pt[3 * mi + 1], pt[3 * mi + 2], er, sm, cc,
-                                         c.rna[mi], c.rnb[mi], c.rta[mi], c.rtb[mi], c.massn[mi], c.masst[mi], c.target[mi], c.corr[mi]);
-                    c.accn[mi] = w[2 * mi]; c.acct[mi] = w[2 * mi + 1];
-                } else {
-                    c.rna[mi] = 0.0f; c.rnb[mi] = 0.0f; c.rta[mi] = 0.0f; c.rtb[mi] = 0.0f; c.massn[mi] = 0.0f; c.masst[mi] = 0.0f;
-                    c.target[mi] = 0.0f; c.corr[mi] = 0.0f; c.accn[mi] = 0.0f; c.acct[mi] = 0.0f;
-                }
-            }
-            recm_store(r, c);
-        }
-    }
-    g.sync();
-    slow_sweep_pairs<SC, G, 0>(sm, ovf, nrec, cmax);
-    sweep_joints<SC, G, 0>(sm, jab, lane, jlevel, jmax, motor_rho);
-    for (int it = 0; it < solver_iters; ++it) {
-        sweep_joints<SC, G, 1>(sm, jab, lane, jlevel, jmax, motor_rho);
-        slow_sweep_pairs<SC, G, 1>(sm, ovf, nrec, cmax);
-    }
-    return cmax;
-}
-
-template <class SC, int G>
-__device__ __noinline__ void slow_correct(float *sm, uint32_t *ovf, int nrec, int cmax) {
-    slow_sweep_pairs<SC, G, 2>(sm, ovf, nrec, cmax);
-}
-
-// End of an overflow step: every pair's accumulated impulses become warm entries in scratch and the
-// pair index table learns where they are; returns the number of active manifolds.
-template <class SC, int G>
-__device__ __noinline__ int slow_finish(float *sm, uint32_t *ovf, int nrec) {
-    Group<G> g;
-    uint8_t *widx = reinterpret_cast<uint8_t *>(reinterpret_cast<uint32_t *>(sm) + SC::WIDX);
-    int nman = 0;
-    for (int k = g.lane; k < nrec; k += G) {
-        const uint32_t *r = ovf + (size_t)k * kRecWords;
-        uint32_t *wr = ovf + SC::SCRATCH_WARM + (size_t)k * kWarmWords;
-        const uint32_t ab = r[R_AB];
-        const int p = (ab >> 12) & 127;
-        const unsigned am = (ab >> 10) & 3u;
-        wr[0] = (uint32_t)p;
-        wr[1] = (am & 1u) ? r[R_M0 + M_ACCN] : 0u;
-        wr[2] = (am & 1u) ? r[R_M0 + M_ACCT] : 0u;
-        wr[3] = (am & 2u) ? r[R_M0 + M_WORDS + M_ACCN] : 0u;
-        wr[4] = (am & 2u) ? r[R_M0 + M_WORDS + M_ACCT] : 0u;
-        widx[p] = (uint8_t)k;
-        nman += __popc(am);
-    }
-    nman = g.sum_int(nman);
-    g.sync();
-    return nman;
-}
-
-// Launch boundaries: warm entries G + G / 2 .. between the state record and the scratch.
-template <class SC, int G>
-__device__ __noinline__ void warm_in(float *sm, uint32_t *ovf, const uint32_t *st_warm, int nwarm) {
-    Group<G> g;
-    uint8_t *widx = reinterpret_cast<uint8_t *>(reinterpret_cast<uint32_t *>(sm) + SC::WIDX);
-    for (int k = G + G / 2 + g.lane; k < nwarm; k += G) {
-        uint32_t *wr = ovf + SC::SCRATCH_WARM + (size_t)k * kWarmWords;
-#pragma unroll
-        for (int q = 0; q < kWarmWords; ++q) wr[q] = __ldcg(st_warm + kWarmWords * k + q);
-        widx[wr[0]] = (uint8_t)k;
-    }
-}
-template <class SC, int G>
-__device__ __noinline__ void warm_out(const uint32_t *ovf, uint32_t *st_warm, int nwarm) {
-    Group<G> g;
-    for (int k = G + G / 2 + g.lane; k < nwarm; k += G) {
-        const uint32_t *wr = ovf + SC::SCRATCH_WARM + (size_t)k * kWarmWords;
-#pragma unroll
-        for (int q = 0; q < kWarmWords; ++q) st_warm[kWarmWords * k + q] = wr[q];
-    }
-}
-
-// ---- one visit of the calling lane's second record (pair number G + lane of a scene with more than G
-// touching pairs), which is in memory form in the lane's shared-memory fields.  MODE as for the first record.
-template <class SC, int G, int MODE>
-__device__ __noinline__ void visit_second(float *sm) {
-    float *ov = sm + SC::STG + LF_COUNT * G + Group<G>().lane;
-    constexpr int H = G / 2;
-    const uint32_t ab = __float_as_uint(ov[R_AB * H]);
-    const int a = ab & 31, b = (ab >> 5) & 31;
-    const unsigned amask = (ab >> 10) & 3u;
-    const bool dyn_a = (ab >> 26) & 1u, dyn_b = (ab >> 27) & 1u;
-    const float nx = ov[R_NX * H], ny = ov[R_NY * H];
-    const float ma = sm[SC::BIM + a], mb = sm[SC::BIM + b];
-    if (MODE == 2) {
-        correct_pair(sm + SC::BPOS, a, b, amask, dyn_a, dyn_b, nx, ny, ma, mb, ov[(R_M0 + M_CORR) * H], ov[(R_M0 + M_WORDS + M_CORR) * H]);
-        return;
-    }
-    const float ia = sm[SC::BII + a], ib = sm[SC::BII + b], mu = ov[R_MU * H];
-    const float4 va4 = ld4(sm + SC::BVEL + 4 * a), vb4 = ld4(sm + SC::BVEL + 4 * b);
-    float vax = va4.x, vay = va4.y, wa = va4.z, vbx = vb4.x, vby = vb4.y, wb = vb4.z;
-#pragma unroll 1
-    for (int mi = 0; mi < 2; ++mi) {
-        if (amask & (1u << mi)) {
-            float *m = ov + (R_M0 + mi * M_WORDS) * H;
-            float accn = m[M_ACCN * H], acct = m[M_ACCT * H];
-            manifold_rows<MODE>(nx, ny, mu, ma, mb, ia, ib, m[M_RNA * H], m[M_RNB * H], m[M_RTA * H], m[M_RTB * H],
-                                m[M_MASSN * H], m[M_MASST * H], m[M_TARGET * H], accn, acct, vax, vay, wa, vbx, vby, wb);
-            if (MODE == 1) { m[M_ACCN * H] = accn; m[M_ACCT * H] = acct; }
-        }
-    }
-    if (dyn_a) st4(sm + SC::BVEL + 4 * a, vax, vay, wa);
-    if (dyn_b) st4(sm + SC::BVEL + 4 * b, vbx, vby, wb);
-}
-
-// Second records, first half: the accumulated impulses the staged pair G + lane carried out of the
-// previous step, parked in four of the lane's second-record fields that are free until the record is built.
-template <class SC, int G>
-__device__ __noinline__ void second_lookup(float *sm, const uint32_t *ovf, int nrec, float old_n, float old_t, int warm_start) {
-    const Group<G> g;
-    constexpr int H = G / 2;
-    float *ov = sm + SC::STG + LF_COUNT * G + g.lane;
-    const uint8_t *widx = reinterpret_cast<const uint8_t *>(reinterpret_cast<const uint32_t *>(sm) + SC::WIDX);
-    const bool mine2 = g.lane < H && G + g.lane < nrec;
-    int wi2 = 255;
-    if (mine2) wi2 = widx[(__float_as_uint(ov[ovs(S_AB) * H]) >> 12) & 127];
-    float w2[4];
-    warm_lookup<SC, G>(g, sm, ovf, wi2, old_n, old_t, warm_start, w2);
-    if (mine2) {
-#pragma unroll
-        for (int q = 0; q < 4; ++q) ov[(R_M0 + M_WORDS + q) * H] = w2[q];
-    }
-}
-// Second half, after every lane has read what it needs from other lanes: the record is built in place.
-// Returns its level | its number of active manifolds << 8 (0 for a lane without a second record).
-template <class SC, int G>
-__device__ __noinline__ unsigned second_build(float *sm, int nrec, ContactConsts cc) {
-    const int lane = Group<G>().lane;
-    constexpr int H = G / 2;
-    if (!(lane < H && G + lane < nrec)) return 0u;
-    float *ov = sm + SC::STG + LF_COUNT * G + lane;
-    const uint32_t ab2 = __float_as_uint(ov[ovs(S_AB) * H]);
-    const int a2 = ab2 & 31, b2 = (ab2 >> 5) & 31;
-    const float nx2 = ov[ovs(S_NX) * H], ny2 = ov[ovs(S_NY) * H];
-    const float pt2[6] = { ov[ovs(S_PX0) * H], ov[ovs(S_PY0) * H], ov[ovs(S_PEN0) * H], ov[ovs(S_PX1) * H], ov[ovs(S_PY1) * H], ov[ovs(S_PEN1) * H] };
-    float w2[4];
-#pragma unroll
-    for (int q = 0; q < 4; ++q) w2[q] = ov[(R_M0 + M_WORDS + q) * H];
-    const float ma = sm[SC::BIM + a2], mb = sm[SC::BIM + b2], ia = sm[SC::BII + a2], ib = sm[SC::BII + b2];
-    const float fra = sm[SC::BFR + a2], frb = sm[SC::BFR + b2];
-    const float er2 = fmin_cmp(sm[SC::BRE + a2], sm[SC::BRE + b2]);
-    ov[R_MU * H] = sqrtf(__fmaf_rn(fra, fra, frb * frb));
-#pragma unroll 1
-    for (int mi = 0; mi < 2; ++mi) {
-        float rna = 0.0f, rnb = 0.0f, rta = 0.0f, rtb = 0.0f, massn = 0.0f, masst = 0.0f, target = 0.0f, corr = 0.0f, an = 0.0f, at = 0.0f;
-        if ((ab2 >> 10) & (1u << mi)) {
-            prestep_manifold<SC>(a2, b2, nx2, ny2, ma, mb, ia, ib, pt2[3 * mi], pt2[3 * mi + 1], pt2[3 * mi + 2], er2, sm, cc,
-                                 rna, rnb, rta, rtb, massn, masst, target, corr);
-            an = w2[2 * mi]; at = w2[2 * mi + 1];
-        }
-        float *m = ov + (R_M0 + mi * M_WORDS) * H;
-        m[M_RNA * H] = rna; m[M_RNB * H] = rnb; m[M_RTA * H] = rta; m[M_RTB * H] = rtb;
-        m[M_MASSN * H] = massn; m[M_MASST * H] = masst; m[M_TARGET * H] = target; m[M_CORR * H] = corr;
-        m[M_ACCN * H] = an; m[M_ACCT * H] = at;
-    }
-    return ((ab2 >> 19) & 127u) | ((unsigned)__popc((ab2 >> 10) & 3u) << 8);
+template <class SC>
+__device__ __forceinline__ uint16_t pair_code(int p) {
+    int a, b;
+    if (p < SC::NPP) { int i = 0, rem = p; while (rem >= SC::P - 1 - i) { rem -= SC::P - 1 - i; ++i; } a = i; b = i + 1 + rem; }
+    else if (p < SC::NPP + SC::NPC) { const int q = p - SC::NPP; a = q / SC::C; b = SC::P + q % SC::C; }
+    else { int i = 0, rem = p - SC::NPP - SC::NPC; while (rem >= SC::C - 1 - i) { rem -= SC::C - 1 - i; ++i; } a = SC::P + i; b = SC::P + i + 1 + rem; }
+    return (uint16_t)(a | (b << 8));
 }
 
 // ================================================================ rarely run code, kept out of line
-// so that the code a step normally runs stays small
 // level constants into shared memory; returns the packed word of joint number `lane` (0 beyond the last joint)
 template <class SC, int G>
-__device__ __noinline__ uint32_t load_level_consts(uint32_t *smu, const uint32_t *lv) {
+__device__ __forceinline__ uint32_t load_level_consts(uint32_t *smu, const uint32_t *lv) {
     const int lane = Group<G>().lane;
     for (int i = lane; i < SC::N; i += G) {
         smu[SC::BIM + i] = lv[SC::LV_IM + i];
@@ -788,39 +335,8 @@ __device__ __noinline__ uint32_t load_level_consts(uint32_t *smu, const uint32_t
     }
     for (int i = lane; i < SC::C; i += G) smu[SC::RAD + i] = lv[SC::LV_RAD + i];
     for (int i = lane; i < SC::MASKW; i += G) smu[SC::MASK + i] = lv[SC::LV_MASK + i];
-    if (lane == 0) smu[SC::META + META_GB] = lv[SC::LV_GB];
-    for (int i = lane; i < SC::LVC_WORDS; i += G) smu[SC::LVC + i] = lv[SC::LV_ELEN + i];
+    for (int i = lane; i < SC::P4; i += G) smu[SC::ELEN + i] = lv[SC::LV_ELEN + i];
     return (SC::J > 0 && lane < SC::J) ? lv[SC::LV_JOINT + kJointLevelWords * lane] : 0u;
-}
-
-// Auto-reset of a finished env: next level (its own, or drawn from the pool by the hash of seed,
-// global env index and episode), pose from the level, no accumulated impulses, counters.  Returns the
-// packed word of joint number `lane` of the level the env is on afterwards.
-template <class SC, int G>
-__device__ __noinline__ uint32_t reset_env(uint32_t *smu, const uint32_t *levels, int n_levels, int auto_reset, unsigned long long seed,
-                                           long long env_index, unsigned long long *counters, uint32_t jab) {
-    Group<G> g;
-    const int lane = g.lane;
-    const int episode = (int)smu[SC::META + META_EPISODE] + 1;
-    int level = (int)smu[SC::META + META_LEVEL];
-    g.sync();
-    if (auto_reset == 2) {
-        const unsigned long long h = mix64(seed + ((unsigned long long)env_index + 1ULL) * 0x9E3779B97F4A7C15ULL +
-                                           (unsigned long long)episode * 0xD1B54A32D192ED03ULL);
-        const int nl = (int)(h % (unsigned long long)n_levels);
-        if (nl != level) { level = nl; jab = load_level_consts<SC, G>(smu, levels + (size_t)nl * SC::LV_WORDS); }
-    }
-    const uint32_t *lv = levels + (size_t)level * SC::LV_WORDS;
-    for (int i = lane; i < 6 * SC::N; i += G) smu[body_word<SC>(i)] = lv[SC::LV_X + i];
-    if (SC::J > 0 && lane < SC::J) { smu[SC::JROW + kJointWords * lane + JR_ACCX] = 0u; smu[SC::JROW + kJointWords * lane + JR_ACCY] = 0u; smu[SC::JROW + kJointWords * lane + JR_ACCR] = 0u; }
-    for (int i = lane; i < (SC::NPAIRS + 3) / 4; i += G) smu[SC::WIDX + i] = 0xffffffffu;
-    if (lane == 0) {
-        smu[SC::META + META_STEP] = 0u; smu[SC::META + META_EPISODE] = (uint32_t)episode; smu[SC::META + META_LEVEL] = (uint32_t)level;
-        smu[SC::META + META_STATUS] = 0u; smu[SC::META + META_NWARM] = 0u;
-        atomicAdd(counters + 1, 1ULL);
-    }
-    g.sync();
-    return jab;
 }
 
 // packed work counters of a group to the global ones (lane 0)
@@ -843,44 +359,29 @@ __device__ __noinline__ void trace_clear(float *trace) {
     g.sync();
 }
 
-// ---------------------------------------------------------------- scene processing
+// ---------------------------------------------------------------- first half of a step: one scene per group of G lanes
 template <class SC, int G>
 struct Scene {
     static_assert(SC::J <= G && SC::T <= G && kMaxActions <= 2 * G, "one lane per joint / thruster");
-    static_assert(2 * G <= 5 * SC::P4, "positional corrections reuse the world-frame vertex arrays");
+    static_assert(2 * SC::NPAIRS < 255, "manifold slot keys are bytes");
     float *sm;            // this scene's shared-memory region
     uint32_t *smu;
     const uint16_t *ptab; // block-shared pair table
-    uint32_t *ovf;        // this group's overflow scratch in global memory
     const StepParams &prm;
     Group<G> g;
     int lane;
-    // state a lane keeps in registers from step to step
-    Rec rec;              // contact pair record number `lane` of the latest step (its accumulated impulses warm-start the next)
-    uint32_t jab;         // packed word of joint number `lane` (0 beyond the last joint)
     unsigned c_surv, c_rec, c_man;   // packed work counters: pp | pc << 16, cc | active pairs << 16, manifolds | env-steps << 16
 
-    __device__ __forceinline__ Scene(uint32_t *region, const uint16_t *pt, uint32_t *scratch, const StepParams &p)
-        : sm(reinterpret_cast<float *>(region)), smu(region), ptab(pt), ovf(scratch), prm(p), g() {
-        lane = g.lane; jab = 0u; c_surv = 0u; c_rec = 0u; c_man = 0u;
+    __device__ __forceinline__ Scene(uint32_t *region, const uint16_t *pt, const StepParams &p)
+        : sm(reinterpret_cast<float *>(region)), smu(region), ptab(pt), prm(p), g() {
+        lane = g.lane; c_surv = 0u; c_rec = 0u; c_man = 0u;
     }
 
     __device__ __forceinline__ uint8_t *surv() { return reinterpret_cast<uint8_t *>(smu + SC::SURV); }
     __device__ __forceinline__ uint8_t *widx() { return reinterpret_cast<uint8_t *>(smu + SC::WIDX); }
     __device__ __forceinline__ float4 &box4(int i) { return *reinterpret_cast<float4 *>(sm + SC::BOX + 4 * i); }
-    // this lane's word of per-lane field f
-    __device__ __forceinline__ float &lanef(int f) { return sm[SC::STG + f * G + lane]; }
-    // this lane's word of field f of its second record (lanes below G / 2 only)
-    __device__ __forceinline__ float &ovl(int f) { return sm[SC::STG + LF_COUNT * G + f * (G / 2) + lane]; }
     __device__ __forceinline__ ContactConsts contact_consts() const {
         ContactConsts cc; cc.slop = prm.slop; cc.rest_thr = prm.rest_thr; cc.alpha = prm.contact_alpha; cc.beta = prm.contact_beta; return cc;
-    }
-    // paper, "Reward": d_t of the dense signal kappa (d_t - d_{t+1})
-    __device__ __forceinline__ float green_blue_distance() const {
-        const uint32_t gb = smu[SC::META + META_GB];
-        const float4 pg = ld4(sm + SC::BPOS + 4 * (gb & 255u)), pb = ld4(sm + SC::BPOS + 4 * ((gb >> 8) & 255u));
-        const float dx = pb.x - pg.x, dy = pb.y - pg.y;
-        return sqrtf(dot2(dx, dy, dx, dy));
     }
     __device__ __forceinline__ void flush() {
         if (lane == 0) flush_counters(prm.counters, c_surv, c_rec, c_man);
@@ -979,7 +480,7 @@ struct Scene {
                 const float sep = dot2(nx, ny, cx, cy) - sm[SC::WOFF + 4 * a + k];
                 const float tx = -ny, ty = nx;
                 float s = dot2(tx, ty, cx - wx, cy - wy);
-                s = fmax_cmp(fmin_cmp(s, sm[SC::LVC + 4 * a + k]), 0.0f);
+                s = fmax_cmp(fmin_cmp(s, sm[SC::ELEN + 4 * a + k]), 0.0f);
                 const float px = __fmaf_rn(s, tx, wx), py = __fmaf_rn(s, ty, wy);
                 const float ex = cx - px, ey = cy - py;
                 const float d2 = dot2(ex, ey, ex, ey);
@@ -1011,68 +512,51 @@ struct Scene {
         return m.pen > 0.0f ? 1u : 0u;
     }
 
-    // ---- one visit of this lane's contact pair record.  MODE 0: warm start, 1: solver iteration, 2: positional correction
-    template <int MODE>
-    __device__ __forceinline__ void visit_pair() {
-        const uint32_t ab = rec.ab;
-        const int a = ab & 31, b = (ab >> 5) & 31;
-        const unsigned amask = (ab >> 10) & 3u;
-        const bool dyn_a = (ab >> 26) & 1u, dyn_b = (ab >> 27) & 1u;
-        if (MODE == 2) {
-            correct_pair(sm + SC::BPOS, a, b, amask, dyn_a, dyn_b, rec.nx, rec.ny, rec.ma, rec.mb,
-                         sm[SC::WVX + lane], sm[SC::WVX + G + lane]);
-            return;
-        }
-        const float4 va4 = ld4(sm + SC::BVEL + 4 * a), vb4 = ld4(sm + SC::BVEL + 4 * b);
-        float vax = va4.x, vay = va4.y, wa = va4.z, vbx = vb4.x, vby = vb4.y, wb = vb4.z;
-        if (amask & 1u)
-            manifold_rows<MODE>(rec.nx, rec.ny, rec.mu, rec.ma, rec.mb, rec.ia, rec.ib, rec.rna, rec.rnb, rec.rta, rec.rtb,
-                                rec.massn, rec.masst, rec.target, rec.accn, rec.acct, vax, vay, wa, vbx, vby, wb);
-        if (amask & 2u) {
-            float accn = lanef(LF_ACC2N), acct = lanef(LF_ACC2T);
-            manifold_rows<MODE>(rec.nx, rec.ny, rec.mu, rec.ma, rec.mb, rec.ia, rec.ib, lanef(M2_RNA), lanef(M2_RNB), lanef(M2_RTA),
-                                lanef(M2_RTB), lanef(M2_MASSN), lanef(M2_MASST), lanef(M2_TARGET), accn, acct, vax, vay, wa, vbx, vby, wb);
-            if (MODE == 1) { lanef(LF_ACC2N) = accn; lanef(LF_ACC2T) = acct; }
-        }
-        if (dyn_a) st4(sm + SC::BVEL + 4 * a, vax, vay, wa);
-        if (dyn_b) st4(sm + SC::BVEL + 4 * b, vbx, vby, wb);
-    }
-    // records of one level touch disjoint movable bodies; levels in order keep the record order
-    template <int MODE>
-    __device__ __forceinline__ void sweep_pairs(int cmax, int clevel, int clevel2) {
-#pragma unroll 1
-        for (int lvl = 1; lvl <= cmax; ++lvl) {
-            if (clevel == lvl) visit_pair<MODE>();
-            if (clevel2 == lvl) visit_second<SC, G, MODE>(sm);
-            g.sync();
-        }
-    }
-
-    // ---- one environment step
-    __device__ __forceinline__ void step(int e, int s) {
-        // frozen env: reports done, nothing else
-        if (smu[SC::META + META_STATUS] & 1u) {
-            if (lane == 0) { prm.reward[(size_t)s * prm.n_envs + e] = 0.0f; prm.done[(size_t)s * prm.n_envs + e] = 1; }
-            return;
-        }
-        const uint32_t *lv = prm.levels + (size_t)smu[SC::META + META_LEVEL] * SC::LV_WORDS;
-        // dense reward: distance between the first green and the first blue shape before the step
-        if (prm.dense_kappa != 0.0f && lane == 0) sm[SC::META + META_D0] = green_blue_distance();
+    // ---- the first half of one environment step of env e
+    __device__ __forceinline__ void prepare(int e) {
+        uint32_t *st = prm.state + (size_t)e * SC::ST_WORDS;
+        uint32_t *scr = prm.scratch + (size_t)e * SC::SCRATCH_WORDS;
+        // frozen env: nothing to prepare (the solve kernel reports done)
+        if (__ldcg(st + SC::ST_META + META_STATUS) & 1u) return;
+        const uint32_t *lv = prm.levels + (size_t)__ldcg(st + SC::ST_META + META_LEVEL) * SC::LV_WORDS;
+        const int nprev = (int)__ldcg(st + SC::ST_META + META_NROWS);
+        // state record -> shared memory (the same 16-byte groups), level constants, index of the previous step's impulses
+        for (int i = lane; i < 2 * SC::N; i += G)
+            reinterpret_cast<float4 *>(sm + SC::BPOS)[i] = __ldcg(reinterpret_cast<const float4 *>(st + SC::ST_POS) + i);
+        const uint32_t jab = load_level_consts<SC, G>(smu, lv);
+        for (int i = lane; i < (2 * SC::NPAIRS + 3) / 4; i += G) smu[SC::WIDX + i] = 0xffffffffu;
         // actions of this step
-        const float *act_row = prm.actions + ((size_t)(s / prm.frame_skip) * prm.n_envs + e) * prm.n_actions;
+        const float *act_row = prm.actions + (size_t)e * prm.n_actions;
         if (lane < prm.n_actions) sm[SC::ACT + lane] = act_row[lane];
         if (G < kMaxActions && lane + G < prm.n_actions) sm[SC::ACT + lane + G] = act_row[lane + G];
+        g.sync();
+        for (int k = lane; k < nprev; k += G) widx()[__ldcg(st + SC::ST_WARM + kWarmWords * k)] = (uint8_t)k;
+        // dense reward: the first green and the first blue shape, and their distance before the step
+        const uint32_t gb = lv[SC::LV_GB];
+        float d0 = 0.0f;
+        if (prm.dense_kappa != 0.0f && ((gb >> 16) & 1u)) {
+            const float4 pg = ld4(sm + SC::BPOS + 4 * (gb & 255u)), pb = ld4(sm + SC::BPOS + 4 * ((gb >> 8) & 255u));
+            const float dx = pb.x - pg.x, dy = pb.y - pg.y;
+            d0 = sqrtf(dot2(dx, dy, dx, dy));
+        }
         // gravity, rotation, circle boxes
-        for (int i = lane; i < SC::N; i += G) {
-            const uint32_t fl = smu[SC::BFL + i];
-            if ((fl & F_ACTIVE) && (fl & F_DYNAMIC)) sm[SC::BVEL + 4 * i + 1] = sm[SC::BVEL + 4 * i + 1] + prm.gdt;
-            float c, sn;
-            sincos_spec(sm[SC::BPOS + 4 * i + 2], c, sn);
-            sm[SC::BC + i] = c; sm[SC::BS + i] = sn;
-            if (i >= SC::P) {
-                const float r = sm[SC::RAD + (i - SC::P)], x = sm[SC::BPOS + 4 * i], y = sm[SC::BPOS + 4 * i + 1];
-                box4(i) = make_float4(x - r, y - r, x + r, y + r);
+        unsigned active_mask = 0u;
+        for (int base = 0; base < SC::N; base += G) {
+            const int i = base + lane;
+            bool act_i = false;
+            if (i < SC::N) {
+                const uint32_t fl = smu[SC::BFL + i];
+                act_i = (fl & F_ACTIVE) != 0u;
+                if (act_i && (fl & F_DYNAMIC)) sm[SC::BVEL + 4 * i + 1] = sm[SC::BVEL + 4 * i + 1] + prm.gdt;
+                float c, sn;
+                sincos_spec(sm[SC::BPOS + 4 * i + 2], c, sn);
+                sm[SC::BC + i] = c; sm[SC::BS + i] = sn;
+                if (i >= SC::P) {
+                    const float r = sm[SC::RAD + (i - SC::P)], x = sm[SC::BPOS + 4 * i], y = sm[SC::BPOS + 4 * i + 1];
+                    box4(i) = make_float4(x - r, y - r, x + r, y + r);
+                }
             }
+            active_mask |= g.ballot(act_i) << base;
         }
         g.sync();
         // world-frame polygon vertices, normals, face offsets
@@ -1089,8 +573,10 @@ struct Scene {
             }
         }
         // this lane's joint: "on" bit and level come with the level record
-        const int jlevel = ((jab >> 24) & 1u) ? (int)((jab >> 25) & 7u) : 0;
+        const bool jon = ((jab >> 24) & 1u) != 0u;
+        const int jlevel = jon ? (int)((jab >> 25) & 7u) : 0;
         const int jmax = (SC::J > 0) ? g.max_int(jlevel) : 0;
+        const uint32_t *jl = lv + SC::LV_JOINT + kJointLevelWords * (lane < SC::J ? lane : 0);
         g.sync();
         // polygon boxes
         for (int i = lane; i < SC::P; i += G) {
@@ -1105,11 +591,30 @@ struct Scene {
             }
             box4(i) = make_float4(x0, y0, x1, y1);
         }
-        // motors (joint order), thrusters (thruster order)
-        sweep_joints<SC, G, 3>(sm, jab, lane, jlevel, jmax, prm.motor_rho, prm.discrete);
+        // motors in joint order: joints of one level touch disjoint movable shapes, levels in order keep the joint order
+        if (SC::J > 0) {
+#pragma unroll 1
+            for (int lvl = 1; lvl <= jmax; ++lvl) {
+                if (jlevel == lvl) {
+                    const int a = jab & 255, b = (jab >> 8) & 255;
+                    const float av = sm[SC::ACT + ((jab >> 16) & 255)];
+                    // paper, "Action Space": continuous in [-1, 1], or multi-discrete codes 0 off, 1 forwards, 2 backwards at full power
+                    const float A = prm.discrete ? (__float_as_int(av) == 1 ? 1.0f : (__float_as_int(av) == 2 ? -1.0f : 0.0f))
+                                                 : fmax_cmp(fmin_cmp(av, 1.0f), -1.0f);
+                    const float speed = __uint_as_float(jl[5]), power = __uint_as_float(jl[6]);
+                    const float wa = sm[SC::BVEL + 4 * a + 2], wb = sm[SC::BVEL + 4 * b + 2];
+                    const float arg = __fmaf_rn(-speed, A, wa - wb) * prm.motor_rho;
+                    const float jr_ = power * tanh_spec(arg);
+                    if ((jab >> 29) & 1u) sm[SC::BVEL + 4 * a + 2] = __fmaf_rn(-jr_, sm[SC::BII + a], wa);
+                    if ((jab >> 30) & 1u) sm[SC::BVEL + 4 * b + 2] = __fmaf_rn(jr_, sm[SC::BII + b], wb);
+                }
+                g.sync();
+            }
+        }
+        // thrusters in thruster order, by level in the same way
         if (SC::T > 0) {
             int tl = 0; uint32_t tp = 0u;
-            const uint32_t *th = smu + SC::LVC + (SC::LV_THR - SC::LV_ELEN) + 8 * lane;
+            const uint32_t *th = lv + SC::LV_THR + 8 * (lane < SC::T ? lane : 0);
             if (lane < SC::T) { tp = th[0]; if ((tp >> 16) & 1u) tl = (tp >> 17) & 7u; }
             const int tmax = g.max_int(tl);
 #pragma unroll 1
@@ -1133,20 +638,22 @@ struct Scene {
                 g.sync();
             }
         }
-        // joint pre-step (poses only; velocities are not read): the row goes to shared memory
+        // joint pre-step (poses only; velocities are not read): the row goes to the env's scratch
         if (SC::J > 0 && lane < SC::J) {
-            float *jr = sm + SC::JROW + kJointWords * lane;
-            if (!((jab >> 24) & 1u) || !prm.warm_start) { jr[JR_ACCX] = 0.0f; jr[JR_ACCY] = 0.0f; jr[JR_ACCR] = 0.0f; }
+            float4 q[6];
+#pragma unroll
+            for (int f = 0; f < 6; ++f) q[f] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+            float accx = __uint_as_float(__ldcg(st + SC::ST_JACC + 3 * lane)), accy = __uint_as_float(__ldcg(st + SC::ST_JACC + 3 * lane + 1));
+            float accr = __uint_as_float(__ldcg(st + SC::ST_JACC + 3 * lane + 2));
+            if (!jon || !prm.warm_start) { accx = 0.0f; accy = 0.0f; accr = 0.0f; }
             int ang = 0;
             float kr = 0.0f, bias_r = 0.0f;
-            if ((jab >> 24) & 1u) {
+            if (jon) {
                 const int a = jab & 255, b = (jab >> 8) & 255;
-                const uint32_t *jl = smu + SC::LVC + (SC::LV_JOINT - SC::LV_ELEN) + kJointLevelWords * lane;
                 float rax, ray, rbx, rby;
                 rot2(sm[SC::BC + a], sm[SC::BS + a], __uint_as_float(jl[1]), __uint_as_float(jl[2]), rax, ray);
                 rot2(sm[SC::BC + b], sm[SC::BS + b], __uint_as_float(jl[3]), __uint_as_float(jl[4]), rbx, rby);
                 const float ma = sm[SC::BIM + a], mb = sm[SC::BIM + b], ia = sm[SC::BII + a], ib = sm[SC::BII + b];
-                jr[JR_MA] = ma; jr[JR_MB] = mb; jr[JR_IA] = ia; jr[JR_IB] = ib;
                 const float gx = (sm[SC::BPOS + 4 * b] + rbx) - (sm[SC::BPOS + 4 * a] + rax), gy = (sm[SC::BPOS + 4 * b + 1] + rby) - (sm[SC::BPOS + 4 * a + 1] + ray);
                 const float msum = ma + mb;
                 float k11 = msum; k11 = __fmaf_rn(ia * ray, ray, k11); k11 = __fmaf_rn(ib * rby, rby, k11);
@@ -1154,11 +661,11 @@ struct Scene {
                 float k12 = -((ia * rax) * ray); k12 = __fmaf_rn(-(ib * rbx), rby, k12);
                 const float det = __fmaf_rn(k11, k22, -(k12 * k12));
                 const float inv_det = 1.0f / det;
-                jr[JR_RAX] = rax; jr[JR_RAY] = ray; jr[JR_RBX] = rbx; jr[JR_RBY] = rby;
-                jr[JR_I11] = k22 * inv_det; jr[JR_I22] = k11 * inv_det; jr[JR_I12] = -(k12 * inv_det);
-                jr[JR_BX] = prm.joint_alpha * gx; jr[JR_BY] = prm.joint_alpha * gy;
                 const float share = prm.joint_beta / msum;
-                jr[JR_CX] = share * gx; jr[JR_CY] = share * gy;
+                q[0] = make_float4(rax, ray, rbx, rby);
+                q[1] = make_float4(k22 * inv_det, -(k12 * inv_det), k11 * inv_det, 0.0f);
+                q[2] = make_float4(prm.joint_alpha * gx, prm.joint_alpha * gy, share * gx, share * gy);
+                q[3] = make_float4(ma, mb, ia, ib);
                 // angular row from the relative rotation at the start of the step
                 const float isum = ia + ib;
                 const uint32_t kind = jl[10];
@@ -1172,8 +679,13 @@ struct Scene {
                     }
                 }
             }
-            if (ang != 1) jr[JR_ACCR] = 0.0f;
-            jr[JR_ANG] = __int_as_float(ang); jr[JR_KR] = kr; jr[JR_BIASR] = bias_r;
+            if (ang != 1) accr = 0.0f;
+            q[1].w = __uint_as_float(jab);
+            q[4] = make_float4(accx, accy, 0.0f, 0.0f);
+            q[5] = make_float4(__int_as_float(ang), kr, bias_r, accr);
+            float4 *jr = reinterpret_cast<float4 *>(scr + SC::SCR_JROW + kJointWords * lane);
+#pragma unroll
+            for (int f = 0; f < 6; ++f) jr[f] = q[f];
         }
         g.sync();
 
@@ -1204,7 +716,8 @@ struct Scene {
         c_surv += (unsigned)ns_pp | ((unsigned)(ns_pc - ns_pp) << 16);
         c_rec += (unsigned)(nsurv - ns_pc);
 
-        // narrowphase: survivors of one kind at a time; active pairs are staged in pair order
+        // narrowphase: survivors of one kind at a time; pairs with an active manifold are staged in pair order, the
+        // first G of them in shared memory, later ones in the row slots 2 k + 1 of the env's scratch
         int nrec = 0;
         bool t_gb = false, t_gr = false;
         float *trace = prm.trace ? prm.trace + (size_t)e * SC::NSLOTS * 6 : nullptr;
@@ -1241,21 +754,15 @@ struct Scene {
                                         (((fa & F_DYNAMIC) ? 1u : 0u) << 26) | (((fb & F_DYNAMIC) ? 1u : 0u) << 27);
                     const float nx = (act & 1u) ? m[0].nx : m[1].nx, ny = (act & 1u) ? m[0].ny : m[1].ny;
                     if (k < G) {
-                        float *st = sm + SC::STG + k;
-                        st[S_AB * G] = __uint_as_float(ab); st[S_NX * G] = nx; st[S_NY * G] = ny;
-                        st[S_PX0 * G] = m[0].px; st[S_PY0 * G] = m[0].py; st[S_PEN0 * G] = m[0].pen;
-                        st[S_PX1 * G] = m[1].px; st[S_PY1 * G] = m[1].py; st[S_PEN1 * G] = m[1].pen;
-                    } else if (k < G + G / 2) {
-                        float *st = sm + SC::STG + LF_COUNT * G + (k - G);
-                        constexpr int H = G / 2;
-                        st[ovs(S_AB) * H] = __uint_as_float(ab); st[ovs(S_NX) * H] = nx; st[ovs(S_NY) * H] = ny;
-                        st[ovs(S_PX0) * H] = m[0].px; st[ovs(S_PY0) * H] = m[0].py; st[ovs(S_PEN0) * H] = m[0].pen;
-                        st[ovs(S_PX1) * H] = m[1].px; st[ovs(S_PY1) * H] = m[1].py; st[ovs(S_PEN1) * H] = m[1].pen;
+                        float *sg = sm + SC::STG + k;
+                        sg[S_AB * G] = __uint_as_float(ab); sg[S_NX * G] = nx; sg[S_NY * G] = ny;
+                        sg[S_PX0 * G] = m[0].px; sg[S_PY0 * G] = m[0].py; sg[S_PEN0 * G] = m[0].pen;
+                        sg[S_PX1 * G] = m[1].px; sg[S_PY1 * G] = m[1].py; sg[S_PEN1 * G] = m[1].pen;
                     } else {
-                        uint32_t *st = ovf + (size_t)k * kRecWords;
-                        st[S_AB] = ab; st[S_NX] = __float_as_uint(nx); st[S_NY] = __float_as_uint(ny);
-                        st[S_PX0] = __float_as_uint(m[0].px); st[S_PY0] = __float_as_uint(m[0].py); st[S_PEN0] = __float_as_uint(m[0].pen);
-                        st[S_PX1] = __float_as_uint(m[1].px); st[S_PY1] = __float_as_uint(m[1].py); st[S_PEN1] = __float_as_uint(m[1].pen);
+                        uint32_t *sg = scr + SC::SCR_ROWS + (size_t)(2 * k + 1) * kRowWords;
+                        sg[S_AB] = ab; sg[S_NX] = __float_as_uint(nx); sg[S_NY] = __float_as_uint(ny);
+                        sg[S_PX0] = __float_as_uint(m[0].px); sg[S_PY0] = __float_as_uint(m[0].py); sg[S_PEN0] = __float_as_uint(m[0].pen);
+                        sg[S_PX1] = __float_as_uint(m[1].px); sg[S_PY1] = __float_as_uint(m[1].py); sg[S_PEN1] = __float_as_uint(m[1].pen);
                     }
                 }
                 nrec += __popc(bal);
@@ -1265,295 +772,102 @@ struct Scene {
         g.sync();
         c_rec += (unsigned)nrec << 16;
 
-        const bool overflow = nrec > G + G / 2;
-        int cmax = 0, clevel = 0, clevel2 = 0;
-        if (overflow) {
-            cmax = slow_solve<SC, G>(sm, ovf, nrec, jab, jlevel, jmax, prm.solver_iters, prm.warm_start, prm.motor_rho,
-                                     rec.accn, rec.acct, contact_consts());
-        } else {
-            const ContactConsts cc = contact_consts();
-            const bool two = nrec > G;      // some lanes get a second record
-            if (two) {
-                if (lane == 0) cmax = levels_by_one_lane<SC, G>(smu, ovf, nrec);
-                g.sync();
-            }
-            // every staged pair becomes a record in its own lane: accumulated impulses of the same pair in the
-            // previous step come from wherever its record was then
-            const bool mine = lane < nrec;
+        // rows: lane k of a round takes staged pair k, runs the pre-step of its active manifolds and writes one row per
+        // manifold; the accumulated impulses of the same manifold slot in the previous step come from the warm list
+        int nrows = 0;
+        const ContactConsts cc = contact_consts();
+#pragma unroll 1
+        for (int base = 0; base < nrec; base += G) {
+            const int k = base + lane;
+            const bool mine = k < nrec;
             uint32_t ab = 0u;
             float nx = 0.0f, ny = 0.0f, pt[6] = { 0.0f, 0.0f, 0.0f, 0.0f, 0.0f, 0.0f };
-            float w[4];
-            {
-                int wi = 255;
-                if (mine) {
-                    ab = __float_as_uint(lanef(S_AB)); wi = widx()[(ab >> 12) & 127];
-                    nx = lanef(S_NX); ny = lanef(S_NY);
-                    pt[0] = lanef(S_PX0); pt[1] = lanef(S_PY0); pt[2] = lanef(S_PEN0); pt[3] = lanef(S_PX1); pt[4] = lanef(S_PY1); pt[5] = lanef(S_PEN1);
+            if (mine) {
+                if (base == 0) {
+                    const float *sg = sm + SC::STG + lane;
+                    ab = __float_as_uint(sg[S_AB * G]); nx = sg[S_NX * G]; ny = sg[S_NY * G];
+                    pt[0] = sg[S_PX0 * G]; pt[1] = sg[S_PY0 * G]; pt[2] = sg[S_PEN0 * G]; pt[3] = sg[S_PX1 * G]; pt[4] = sg[S_PY1 * G]; pt[5] = sg[S_PEN1 * G];
+                } else {
+                    const uint32_t *sg = scr + SC::SCR_ROWS + (size_t)(2 * k + 1) * kRowWords;
+                    ab = __ldcg(sg + S_AB); nx = __uint_as_float(__ldcg(sg + S_NX)); ny = __uint_as_float(__ldcg(sg + S_NY));
+                    pt[0] = __uint_as_float(__ldcg(sg + S_PX0)); pt[1] = __uint_as_float(__ldcg(sg + S_PY0)); pt[2] = __uint_as_float(__ldcg(sg + S_PEN0));
+                    pt[3] = __uint_as_float(__ldcg(sg + S_PX1)); pt[4] = __uint_as_float(__ldcg(sg + S_PY1)); pt[5] = __uint_as_float(__ldcg(sg + S_PEN1));
                 }
-                const float old_n = rec.accn, old_t = rec.acct;
-                warm_lookup<SC, G>(g, sm, ovf, wi, old_n, old_t, prm.warm_start, w);
-                if (two) second_lookup<SC, G>(sm, ovf, nrec, old_n, old_t, prm.warm_start);
             }
-            g.sync();     // every lane has read the fields it needs from other lanes before they are rewritten
-            const int a = ab & 31, b = (ab >> 5) & 31;
             const unsigned amask = (ab >> 10) & 3u;
-            rec.ab = ab; rec.nx = nx; rec.ny = ny;
-            rec.ma = sm[SC::BIM + a]; rec.mb = sm[SC::BIM + b]; rec.ia = sm[SC::BII + a]; rec.ib = sm[SC::BII + b];
-            {
+            const unsigned b0 = g.ballot((amask & 1u) != 0u), b1 = g.ballot((amask & 2u) != 0u);
+            int row = nrows + __popc(b0 & g.lanes_below()) + __popc(b1 & g.lanes_below());
+            nrows += __popc(b0) + __popc(b1);
+            g.sync();       // every lane of the round has its staged pair before rows are written over the staging slots
+            if (mine) {
+                const int a = ab & 31, b = (ab >> 5) & 31, p = (ab >> 12) & 127;
+                const float ma = sm[SC::BIM + a], mb = sm[SC::BIM + b], ia = sm[SC::BII + a], ib = sm[SC::BII + b];
                 const float fra = sm[SC::BFR + a], frb = sm[SC::BFR + b];
-                rec.mu = sqrtf(__fmaf_rn(fra, fra, frb * frb));
-            }
-            const float er = fmin_cmp(sm[SC::BRE + a], sm[SC::BRE + b]);
-            float corr0 = 0.0f, corr1 = 0.0f;
-            rec.rna = 0.0f; rec.rnb = 0.0f; rec.rta = 0.0f; rec.rtb = 0.0f; rec.massn = 0.0f; rec.masst = 0.0f; rec.target = 0.0f;
-            rec.accn = 0.0f; rec.acct = 0.0f;
-            if (amask & 1u) {
-                prestep_manifold<SC>(a, b, nx, ny, rec.ma, rec.mb, rec.ia, rec.ib, pt[0], pt[1], pt[2], er, sm, cc,
-                                     rec.rna, rec.rnb, rec.rta, rec.rtb, rec.massn, rec.masst, rec.target, corr0);
-                rec.accn = w[0]; rec.acct = w[1];
-            }
-            float acc2n = 0.0f, acc2t = 0.0f;
-            if (amask & 2u) {
-                float rna, rnb, rta, rtb, massn, masst, target;
-                prestep_manifold<SC>(a, b, nx, ny, rec.ma, rec.mb, rec.ia, rec.ib, pt[3], pt[4], pt[5], er, sm, cc,
-                                     rna, rnb, rta, rtb, massn, masst, target, corr1);
-                lanef(M2_RNA) = rna; lanef(M2_RNB) = rnb; lanef(M2_RTA) = rta; lanef(M2_RTB) = rtb;
-                lanef(M2_MASSN) = massn; lanef(M2_MASST) = masst; lanef(M2_TARGET) = target;
-                acc2n = w[2]; acc2t = w[3];
-            }
-            lanef(LF_ACC2N) = acc2n; lanef(LF_ACC2T) = acc2t;
-            sm[SC::WVX + lane] = corr0; sm[SC::WVX + G + lane] = corr1;
-            if (two) {
-                const unsigned r2 = second_build<SC, G>(sm, nrec, cc);     // level | active manifolds << 8
-                clevel2 = (int)(r2 & 127u);
-                clevel = (int)((ab >> 19) & 127u);
-                cmax = g.shfl(cmax, 0);
-                c_man += (unsigned)g.sum_int((int)(r2 >> 8));
-            } else {
-                // levels of the records (canonical order = record order): one more than the highest level of an
-                // earlier record that shares a movable body.  Every movable body collects the set of records that
-                // touch it; a record's conflicts are the earlier members of its bodies' sets; then level r goes to
-                // the records whose conflicts all have a level already, round after round.
-                uint32_t *touch = smu + SC::SURV;            // the survivor list is no longer needed
-                for (int i = lane; i < SC::N; i += G) touch[i] = 0u;
-                g.sync();
-                const bool da = (ab >> 26) & 1u, db = (ab >> 27) & 1u;
-                if (mine && da) atomicOr(touch + a, 1u << lane);
-                if (mine && db) atomicOr(touch + b, 1u << lane);
-                g.sync();
-                const unsigned conflicts = ((da ? touch[a] : 0u) | (db ? touch[b] : 0u)) & g.lanes_below();
-                const unsigned all = g.ballot(mine);
-                unsigned assigned = 0u;
-                int lvl = 0;
+                const float mu = sqrtf(__fmaf_rn(fra, fra, frb * frb));
+                const float er = fmin_cmp(sm[SC::BRE + a], sm[SC::BRE + b]);
+                const uint32_t rab = (uint32_t)a | ((uint32_t)b << 5) | (((ab >> 26) & 3u) << 10);
 #pragma unroll 1
-                for (int r = 1; assigned != all; ++r) {
-                    const bool ready = mine && lvl == 0 && (conflicts & ~assigned) == 0u;
-                    if (ready) lvl = r;
-                    assigned |= g.ballot(ready);
+                for (int mi = 0; mi < 2; ++mi) {
+                    if (amask & (1u << mi)) {
+                        float rna, rnb, rta, rtb, massn, masst, target, corr;
+                        prestep_manifold<SC>(a, b, nx, ny, ma, mb, ia, ib, pt[3 * mi], pt[3 * mi + 1], pt[3 * mi + 2], er, sm, cc,
+                                             rna, rnb, rta, rtb, massn, masst, target, corr);
+                        const int key = 2 * p + mi;
+                        const int wi = widx()[key];
+                        float accn = 0.0f, acct = 0.0f;
+                        if (wi != 255 && prm.warm_start) {
+                            accn = __uint_as_float(__ldcg(st + SC::ST_WARM + kWarmWords * wi + 1));
+                            acct = __uint_as_float(__ldcg(st + SC::ST_WARM + kWarmWords * wi + 2));
+                        }
+                        float4 *r = reinterpret_cast<float4 *>(scr + SC::SCR_ROWS + (size_t)row * kRowWords);
+                        r[0] = make_float4(__uint_as_float(rab), nx, ny, mu);
+                        r[1] = make_float4(ma, mb, ia, ib);
+                        r[2] = make_float4(rna, rnb, rta, rtb);
+                        r[3] = make_float4(massn, masst, target, corr);
+                        r[4] = make_float4(accn, acct, __int_as_float(key), 0.0f);
+                        ++row;
+                    }
                 }
-                clevel = lvl;
-                cmax = g.max_int(lvl);
-            }
-            c_man += (unsigned)(__popc(g.ballot(amask & 1u)) + __popc(g.ballot(amask & 2u)));
-            // warm start: contacts, then joints
-            sweep_pairs<0>(cmax, clevel, clevel2);
-            sweep_joints<SC, G, 0>(sm, jab, lane, jlevel, jmax, prm.motor_rho);
-            // solver iterations: joints, then contacts
-#pragma unroll 1
-            for (int it = 0; it < prm.solver_iters; ++it) {
-                sweep_joints<SC, G, 1>(sm, jab, lane, jlevel, jmax, prm.motor_rho);
-                sweep_pairs<1>(cmax, clevel, clevel2);
             }
         }
-        // Euler step with the solved velocities
-        for (int i = lane; i < SC::N; i += G) {
-            if (smu[SC::BFL + i] & F_ACTIVE) {
-                const float4 p4 = ld4(sm + SC::BPOS + 4 * i), v4 = ld4(sm + SC::BVEL + 4 * i);
-                st4(sm + SC::BPOS + 4 * i, __fmaf_rn(prm.dt, v4.x, p4.x), __fmaf_rn(prm.dt, v4.y, p4.y), __fmaf_rn(prm.dt, v4.z, p4.z));
-            }
-        }
-        g.sync();
-        if (overflow) slow_correct<SC, G>(sm, ovf, nrec, cmax);
-        else sweep_pairs<2>(cmax, clevel, clevel2);
-        sweep_joints<SC, G, 2>(sm, jab, lane, jlevel, jmax, prm.motor_rho);
-        bool finite = true;
-        for (int i = lane; i < SC::N; i += G) {
-            const float4 p4 = ld4(sm + SC::BPOS + 4 * i), v4 = ld4(sm + SC::BVEL + 4 * i);
-            finite = finite && finite_bits(p4.x) && finite_bits(p4.y) && finite_bits(p4.z) && finite_bits(v4.x) && finite_bits(v4.y) && finite_bits(v4.z);
-        }
-        finite = !g.any(!finite);
-
-        // where the pairs of this step keep their accumulated impulses for the next one
-        for (int i = lane; i < (SC::NPAIRS + 3) / 4; i += G) smu[SC::WIDX + i] = 0xffffffffu;
-        const int step_count = (int)smu[SC::META + META_STEP] + 1;
-        g.sync();
-        if (overflow) {
-            c_man += (unsigned)slow_finish<SC, G>(sm, ovf, nrec);
-            // the first G + G / 2 pairs go back to their lanes
-            const uint32_t *wr = ovf + SC::SCRATCH_WARM + (size_t)lane * kWarmWords, *wr2 = wr + (size_t)G * kWarmWords;
-            rec.ab = wr[0] << 12;
-            rec.accn = __uint_as_float(wr[1]); rec.acct = __uint_as_float(wr[2]);
-            lanef(LF_ACC2N) = __uint_as_float(wr[3]); lanef(LF_ACC2T) = __uint_as_float(wr[4]);
-            if (lane < G / 2) {
-                ovl(R_AB) = __uint_as_float(wr2[0] << 12);
-                ovl(OV_ACC0N) = __uint_as_float(wr2[1]); ovl(OV_ACC0T) = __uint_as_float(wr2[2]);
-                ovl(OV_ACC1N) = __uint_as_float(wr2[3]); ovl(OV_ACC1T) = __uint_as_float(wr2[4]);
-            }
-        } else {
-            if (lane < nrec) widx()[(rec.ab >> 12) & 127] = (uint8_t)lane;
-            if (clevel2 != 0) widx()[(__float_as_uint(ovl(R_AB)) >> 12) & 127] = (uint8_t)(G + lane);
-        }
-
-        // reward, termination, counters, auto-reset
-        const bool timeout = prm.max_episode_steps > 0 && step_count >= prm.max_episode_steps;
-        float reward = (float)((int)touch_gb - (int)touch_gr);
-        if (prm.dense_kappa != 0.0f && ((smu[SC::META + META_GB] >> 16) & 1u))
-            reward = reward + prm.dense_kappa * (sm[SC::META + META_D0] - green_blue_distance());
-        bool done = touch_gb || touch_gr || timeout;
-        if (!finite) { reward = 0.0f; done = true; }
+        c_man += (unsigned)nrows | (1u << 16);
+        // velocities (gravity, motors, thrusters) and this step's messages to the solve kernel
+        for (int i = lane; i < SC::N; i += G)
+            reinterpret_cast<float4 *>(st + SC::ST_VEL)[i] = reinterpret_cast<const float4 *>(sm + SC::BVEL)[i];
         if (lane == 0) {
-            prm.reward[(size_t)s * prm.n_envs + e] = reward;
-            prm.done[(size_t)s * prm.n_envs + e] = done ? 1 : 0;
-            smu[SC::META + META_STEP] = (uint32_t)step_count;
-            smu[SC::META + META_NWARM] = (uint32_t)nrec;
-            if (!finite) { smu[SC::META + META_STATUS] |= 1u; atomicAdd(prm.counters + 0, 1ULL); }
+            const uint32_t flags = (touch_gb ? 1u : 0u) | (touch_gr ? 2u : 0u) | (((gb >> 16) & 1u) << 2) | ((gb & 255u) << 8) | (((gb >> 8) & 255u) << 16);
+            *reinterpret_cast<uint4 *>(st + SC::ST_META + META_NROWS) = make_uint4((uint32_t)nrows, flags, __float_as_uint(d0), active_mask);
         }
-        c_man += 1u << 16;
-        g.sync();
-        if (done && prm.auto_reset != 0)
-            jab = reset_env<SC, G>(smu, prm.levels, prm.n_levels, prm.auto_reset, prm.seed, prm.env_offset + e, prm.counters, jab);
-    }
-
-    // ---- whole launch for one scene
-    // steps s0 .. s1-1 of env e.  The state record may have been written by another SM earlier in this
-    // launch, so it is read past the (non-coherent) L1.
-    __device__ __forceinline__ void run(int e, int s0, int s1) {
-        uint32_t *st = prm.state + (size_t)e * SC::ST_WORDS;
-        for (int i = lane; i < 6 * SC::N; i += G) smu[body_word<SC>(i)] = __ldcg(st + SC::ST_BODY + i);
-        if (lane < 5) smu[SC::META + lane] = __ldcg(st + SC::ST_META + lane);
-        if (SC::J > 0 && lane < SC::J) {
-            smu[SC::JROW + kJointWords * lane + JR_ACCX] = __ldcg(st + SC::ST_JACC + 3 * lane);
-            smu[SC::JROW + kJointWords * lane + JR_ACCY] = __ldcg(st + SC::ST_JACC + 3 * lane + 1);
-            smu[SC::JROW + kJointWords * lane + JR_ACCR] = __ldcg(st + SC::ST_JACC + 3 * lane + 2);
-        }
-        for (int i = lane; i < (SC::NPAIRS + 3) / 4; i += G) smu[SC::WIDX + i] = 0xffffffffu;
-        const int level = (int)__ldcg(st + SC::ST_META + META_LEVEL);
-        const int nwarm = (int)__ldcg(st + SC::ST_META + META_NWARM);
-        jab = load_level_consts<SC, G>(smu, prm.levels + (size_t)level * SC::LV_WORDS);
-        g.sync();
-        // accumulated impulses of the previous launch: entry k goes to lane k
-        rec.ab = 0u; rec.accn = 0.0f; rec.acct = 0.0f;
-        lanef(LF_ACC2N) = 0.0f; lanef(LF_ACC2T) = 0.0f;
-        if (lane < nwarm) {
-            const uint32_t *wr = st + SC::ST_WARM + kWarmWords * lane;
-            const uint32_t p = __ldcg(wr);
-            rec.ab = p << 12;
-            rec.accn = __uint_as_float(__ldcg(wr + 1)); rec.acct = __uint_as_float(__ldcg(wr + 2));
-            lanef(LF_ACC2N) = __uint_as_float(__ldcg(wr + 3)); lanef(LF_ACC2T) = __uint_as_float(__ldcg(wr + 4));
-            widx()[p] = (uint8_t)lane;
-        }
-        if (lane < G / 2 && G + lane < nwarm) {
-            const uint32_t *wr = st + SC::ST_WARM + kWarmWords * (G + lane);
-            const uint32_t p = __ldcg(wr);
-            ovl(R_AB) = __uint_as_float(p << 12);
-            ovl(OV_ACC0N) = __uint_as_float(__ldcg(wr + 1)); ovl(OV_ACC0T) = __uint_as_float(__ldcg(wr + 2));
-            ovl(OV_ACC1N) = __uint_as_float(__ldcg(wr + 3)); ovl(OV_ACC1T) = __uint_as_float(__ldcg(wr + 4));
-            widx()[p] = (uint8_t)(G + lane);
-        }
-        if (nwarm > G + G / 2) warm_in<SC, G>(sm, ovf, st + SC::ST_WARM, nwarm);
-        g.sync();
-#pragma unroll 1
-        for (int s = s0; s < s1; ++s) {
-            step(e, s);
-            g.sync();
-            if (((s - s0) & 255) == 255) flush();
-        }
-        // write back
-        for (int i = lane; i < 6 * SC::N; i += G) st[SC::ST_BODY + i] = smu[body_word<SC>(i)];
-        if (SC::J > 0 && lane < SC::J) {
-            st[SC::ST_JACC + 3 * lane] = smu[SC::JROW + kJointWords * lane + JR_ACCX];
-            st[SC::ST_JACC + 3 * lane + 1] = smu[SC::JROW + kJointWords * lane + JR_ACCY];
-            st[SC::ST_JACC + 3 * lane + 2] = smu[SC::JROW + kJointWords * lane + JR_ACCR];
-        }
-        if (lane < 5) st[SC::ST_META + lane] = smu[SC::META + lane];
-        const int nw = (int)smu[SC::META + META_NWARM];
-        if (lane < nw) {
-            uint32_t *wr = st + SC::ST_WARM + kWarmWords * lane;
-            wr[0] = (rec.ab >> 12) & 127u;
-            wr[1] = __float_as_uint(rec.accn); wr[2] = __float_as_uint(rec.acct);
-            wr[3] = __float_as_uint(lanef(LF_ACC2N)); wr[4] = __float_as_uint(lanef(LF_ACC2T));
-        }
-        if (lane < G / 2 && G + lane < nw) {
-            uint32_t *wr = st + SC::ST_WARM + kWarmWords * (G + lane);
-            wr[0] = (__float_as_uint(ovl(R_AB)) >> 12) & 127u;
-            wr[1] = __float_as_uint(ovl(OV_ACC0N)); wr[2] = __float_as_uint(ovl(OV_ACC0T));
-            wr[3] = __float_as_uint(ovl(OV_ACC1N)); wr[4] = __float_as_uint(ovl(OV_ACC1T));
-        }
-        if (nw > G + G / 2) warm_out<SC, G>(ovf, st + SC::ST_WARM, nw);
-        flush();
-        g.sync();
     }
 };
 
-template <class SC>
-__device__ __forceinline__ uint16_t pair_code(int p) {
-    int a, b;
-    if (p < SC::NPP) { int i = 0, rem = p; while (rem >= SC::P - 1 - i) { rem -= SC::P - 1 - i; ++i; } a = i; b = i + 1 + rem; }
-    else if (p < SC::NPP + SC::NPC) { const int q = p - SC::NPP; a = q / SC::C; b = SC::P + q % SC::C; }
-    else { int i = 0, rem = p - SC::NPP - SC::NPC; while (rem >= SC::C - 1 - i) { rem -= SC::C - 1 - i; ++i; } a = SC::P + i; b = SC::P + i + 1 + rem; }
-    return (uint16_t)(a | (b << 8));
-}
 
 template <class SC, int G>
-__global__ void __launch_bounds__(kBlockThreads, kMinBlocks) k2d_step_kernel(const StepParams prm) {
+__global__ void __launch_bounds__(kBlockThreads, kMinBlocks) k2d_prep_kernel(const StepParams prm) {
     extern __shared__ __align__(16) uint32_t smem_raw[];
     constexpr int GPB = kBlockThreads / G;
     uint16_t *ptab = reinterpret_cast<uint16_t *>(smem_raw);
     for (int p = threadIdx.x; p < SC::NPAIRS; p += kBlockThreads) ptab[p] = pair_code<SC>(p);
     __syncthreads();
     const int gib = threadIdx.x / G;
-    const int slot = blockIdx.x * GPB + gib, nslots = gridDim.x * GPB;
+    const int nslots = gridDim.x * GPB;
     uint32_t *region = smem_raw + SC::PTAB_WORDS + gib * region_words<SC, G>();
-    uint32_t *scratch = prm.scratch + (size_t)slot * SC::SCRATCH_WORDS;
-    Scene<SC, G> scene(region, ptab, scratch, prm);
-    // Work items are (chunk, env), handed out in that order by one ticket counter: a group that is done
-    // takes the next item, so groups with cheap scenes take more of them.  Chunk c of an env may start
-    // only when its chunk c - 1 is stepped and its state is back in memory (another group may have done
-    // it); with items handed out chunk by chunk that is almost always long past, else the group waits for
-    // the group that holds it, which is running.
+    Scene<SC, G> scene(region, ptab, prm);
+    // Envs are handed out one at a time by a ticket counter: a group that is done takes the next one, so groups with
+    // cheap scenes take more of them.
     const Group<G> &g = scene.g;
-    const unsigned items = (unsigned)prm.n_envs * (unsigned)prm.n_chunks;
+    int taken = 0;
 #pragma unroll 1
     for (;;) {
         unsigned t = 0u;
         if (g.lane == 0) t = atomicAdd(prm.queue + Q_TICKET, 1u);
         t = g.shflu(t, 0);
-        if (t >= items) break;
-        const int c = (int)(t / (unsigned)prm.n_envs), e = (int)(t - (unsigned)c * (unsigned)prm.n_envs);
-        bool ok = true;
-        if (c > 0) {
-            if (g.lane == 0) {
-                const volatile unsigned int *flag = prm.chunks_done + e;
-                const volatile unsigned int *err = prm.queue + Q_ERROR;
-                unsigned polls = 0u;
-                while (*flag != (unsigned)c) {
-                    if (*err != 0u || ++polls > kWaitLimit) { atomicExch(prm.queue + Q_ERROR, 1u); ok = false; break; }
-                    __nanosleep(100);
-                }
-            }
-            ok = g.shfl(ok ? 1 : 0, 0) != 0;
-            __threadfence();
-        }
-        if (ok) {
-            const int s0 = c * prm.chunk_steps;
-            scene.run(e, s0, min(prm.n_steps, s0 + prm.chunk_steps));
-        }
-        if (prm.n_chunks > 1) {
-            __threadfence();      // this lane's part of the state record is visible before the count moves
-            g.sync();
-            if (g.lane == 0) atomicExch(prm.chunks_done + e, (c + 1 == prm.n_chunks) ? 0u : (unsigned)(c + 1));
-        }
+        if (t >= (unsigned)prm.n_envs) break;
+        scene.prepare((int)t);
+        g.sync();
+        if ((++taken & 63) == 0) scene.flush();
     }
+    scene.flush();
     // the last group to leave rewinds the queue for the next launch
     if (g.lane == 0) {
         __threadfence();
@@ -1564,7 +878,263 @@ __global__ void __launch_bounds__(kBlockThreads, kMinBlocks) k2d_step_kernel(con
     }
 }
 
-// ---------------------------------------------------------------- reset kernel: one thread per (env, word)
+// ================================================================ second half of a step: one thread per env
+// The constants of a joint row and of a manifold row as the solver reads them (read-only loads: the rows were written by
+// the prep kernel of the same step and nothing writes them while the solve kernel runs; the accumulated impulses, which the
+// solver does write, are copied to shared memory first).
+struct JointConsts { float4 r, k, b, m; };       // lever arms; inverse effective mass and packed joint word; bias and correction; inverse masses
+struct RowConsts { float4 h0, h1, c0, c1; };      // pair word, normal, friction; inverse masses; lever-arm cross products; effective masses, target, correction
+__device__ __forceinline__ JointConsts load_joint(const float *jr) {
+    const float4 *q = reinterpret_cast<const float4 *>(jr);
+    JointConsts c; c.r = __ldg(q); c.k = __ldg(q + 1); c.b = __ldg(q + 2); c.m = __ldg(q + 3);
+    return c;
+}
+__device__ __forceinline__ RowConsts load_row(const float *r) {
+    const float4 *q = reinterpret_cast<const float4 *>(r);
+    RowConsts c; c.h0 = __ldg(q); c.h1 = __ldg(q + 1); c.c0 = __ldg(q + 2); c.c1 = __ldg(q + 3);
+    return c;
+}
+
+// ---- angular row of a fixed joint or of a revolute joint beyond one of its limits (paper, "Fixed Joints",
+// "Joint Limits"): j_r = (w_a - w_b + correction) / (1/I_a + 1/I_b), a loses j_r / I_a, b gains j_r / I_b.  A fixed
+// joint's impulse is accumulated and warm-started; a limit only ever pushes back, applies no correction while the
+// joint is already returning, and is not accumulated.  ang4: kind this step, inverse angular mass, correction, -;
+// accr: the accumulated impulse.  Out of line: most joints are plain revolute joints.
+template <int MODE>
+__device__ __noinline__ float2 angular_row(const float *jr, float *accr, float ia, float ib, float wa, float wb) {
+    const float4 ang4 = __ldg(reinterpret_cast<const float4 *>(jr + JR_ANG));
+    const int ang = __float_as_int(ang4.x);
+    if (ang == 0) return make_float2(wa, wb);
+    float lr;
+    if (MODE == 0) {
+        if (ang != 1) return make_float2(wa, wb);
+        lr = *accr;
+    } else {
+        const float wrel = wa - wb;
+        float v;
+        if (ang == 1) v = wrel + ang4.z;
+        else if (ang == 2) { v = (wrel < 0.0f) ? wrel : wrel + ang4.z; v = fmax_cmp(v, 0.0f); }
+        else { v = (wrel > 0.0f) ? wrel : wrel + ang4.z; v = fmin_cmp(v, 0.0f); }
+        lr = v * ang4.y;
+        if (ang == 1) *accr = *accr + lr;
+    }
+    return make_float2(__fmaf_rn(-lr, ia, wa), __fmaf_rn(lr, ib, wb));
+}
+
+// one visit of a joint row.  MODE 0: apply the accumulated impulses (warm start); 1: one solver iteration.
+// sv: the calling thread's column of the block's velocity array (stride kSolveThreads groups per body);
+// acc: the joint's accumulated impulses (x, y, angular, -) in shared memory.
+template <int MODE>
+__device__ __forceinline__ void solve_joint(const JointConsts &c, const float *jr, float4 *acc, float4 *sv) {
+    const uint32_t jab = __float_as_uint(c.k.w);
+    if (!((jab >> 24) & 1u)) return;
+    const int a = jab & 255, b = (jab >> 8) & 255;
+    const float ma = c.m.x, mb = c.m.y, ia = c.m.z, ib = c.m.w;
+    const float rax = c.r.x, ray = c.r.y, rbx = c.r.z, rby = c.r.w;
+    const float4 va4 = sv[a * kSolveThreads], vb4 = sv[b * kSolveThreads];
+    float vax = va4.x, vay = va4.y, wa = va4.z, vbx = vb4.x, vby = vb4.y, wb = vb4.z;
+    float4 ac = *acc;
+    float lx, ly;
+    if (MODE == 0) { lx = ac.x; ly = ac.y; }
+    else {
+        const float cx = __fmaf_rn(-wb, rby, vbx) - __fmaf_rn(-wa, ray, vax);
+        const float cy = __fmaf_rn(wb, rbx, vby) - __fmaf_rn(wa, rax, vay);
+        const float rx = -(cx + c.b.x), ry = -(cy + c.b.y);
+        const float i11 = c.k.x, i12 = c.k.y, i22 = c.k.z;
+        lx = __fmaf_rn(i11, rx, i12 * ry);
+        ly = __fmaf_rn(i12, rx, i22 * ry);
+        ac.x = ac.x + lx; ac.y = ac.y + ly;
+    }
+    wa = __fmaf_rn(-ia, cross2(rax, ray, lx, ly), wa);
+    wb = __fmaf_rn(ib, cross2(rbx, rby, lx, ly), wb);
+    if (jab >> 31) {      // fixed or limited joint: its angular row follows the point row
+        const float2 w2 = angular_row<MODE>(jr, &ac.z, ia, ib, wa, wb);
+        wa = w2.x; wb = w2.y;
+    }
+    if (MODE == 1) *acc = ac;
+    if ((jab >> 29) & 1u) sv[a * kSolveThreads] = make_float4(__fmaf_rn(-ma, lx, vax), __fmaf_rn(-ma, ly, vay), wa, 0.0f);
+    if ((jab >> 30) & 1u) sv[b * kSolveThreads] = make_float4(__fmaf_rn(mb, lx, vbx), __fmaf_rn(mb, ly, vby), wb, 0.0f);
+}
+
+// one visit of a manifold row (normal then friction), same modes; acc: its accumulated normal and tangent impulse
+template <int MODE>
+__device__ __forceinline__ void solve_row(const RowConsts &c, float2 *accp, float4 *sv) {
+    float2 acc = *accp;
+    const uint32_t ab = __float_as_uint(c.h0.x);
+    const int a = ab & 31, b = (ab >> 5) & 31;
+    const float4 va4 = sv[a * kSolveThreads], vb4 = sv[b * kSolveThreads];
+    float vax = va4.x, vay = va4.y, wa = va4.z, vbx = vb4.x, vby = vb4.y, wb = vb4.z;
+    manifold_rows<MODE>(c.h0.y, c.h0.z, c.h0.w, c.h1.x, c.h1.y, c.h1.z, c.h1.w, c.c0.x, c.c0.y, c.c0.z, c.c0.w, c.c1.x, c.c1.y, c.c1.z,
+                        acc.x, acc.y, vax, vay, wa, vbx, vby, wb);
+    if (MODE == 1) *accp = acc;
+    if ((ab >> 10) & 1u) sv[a * kSolveThreads] = make_float4(vax, vay, wa, 0.0f);
+    if ((ab >> 11) & 1u) sv[b * kSolveThreads] = make_float4(vbx, vby, wb, 0.0f);
+}
+
+constexpr int kAccCap = 32;   // manifold rows of an env whose accumulated impulses sit in shared memory during the solve; later rows use their scratch row
+
+template <class SC>
+__global__ void __launch_bounds__(kSolveThreads) k2d_solve_kernel(const StepParams prm) {
+    // velocities (later positions) of the block's envs: one 16-byte group per (body, thread); a thread's groups are
+    // kSolveThreads groups apart, so the threads of a warp never meet in a bank, whichever bodies they address
+    __shared__ float4 s_body[SC::N * kSolveThreads];
+    __shared__ float4 s_jacc[(SC::J > 0 ? SC::J : 1) * kSolveThreads];
+    __shared__ float2 s_racc[kAccCap * kSolveThreads];
+    const int e = blockIdx.x * kSolveThreads + threadIdx.x;
+    if (e >= prm.n_envs) return;
+    float4 *sv = s_body + threadIdx.x;
+    float4 *sj = s_jacc + threadIdx.x;
+    float2 *sa = s_racc + threadIdx.x;
+    uint32_t *st = prm.state + (size_t)e * SC::ST_WORDS;
+    float *stf = reinterpret_cast<float *>(st);
+    float *rows = reinterpret_cast<float *>(prm.scratch + (size_t)e * SC::SCRATCH_WORDS + SC::SCR_ROWS);
+    float *jrows = reinterpret_cast<float *>(prm.scratch + (size_t)e * SC::SCRATCH_WORDS + SC::SCR_JROW);
+    const uint4 m0 = *reinterpret_cast<const uint4 *>(st + SC::ST_META), m1 = *reinterpret_cast<const uint4 *>(st + SC::ST_META + 4);
+    // frozen env: reports done, nothing else
+    if (m0.w & 1u) { prm.reward[e] = 0.0f; prm.done[e] = 1; return; }
+    const int nrows = (int)m1.x;
+    const uint32_t flags = m1.y, active = m1.w;
+#pragma unroll
+    for (int i = 0; i < SC::N; ++i) sv[i * kSolveThreads] = ld4(stf + SC::ST_VEL + 4 * i);
+#pragma unroll
+    for (int j = 0; j < SC::J; ++j) {
+        const float2 a2 = *reinterpret_cast<const float2 *>(jrows + j * kJointWords + JR_ACCX);
+        sj[j * kSolveThreads] = make_float4(a2.x, a2.y, jrows[j * kJointWords + JR_ACCR], 0.0f);
+    }
+    const int ncap = nrows < kAccCap ? nrows : kAccCap;
+#pragma unroll 1
+    for (int k = 0; k < ncap; ++k) sa[k * kSolveThreads] = *reinterpret_cast<const float2 *>(rows + k * kRowWords + R_ACCN);
+#define K2D_ACC_OF(k) ((k) < kAccCap ? sa + (k) * kSolveThreads : reinterpret_cast<float2 *>(rows + (k) * kRowWords + R_ACCN))
+    // warm start: contacts, then joints (Algorithm 1)
+    {
+        RowConsts cur = load_row(rows);
+#pragma unroll 1
+        for (int k = 0; k < nrows; ++k) {
+            const RowConsts nxt = load_row(rows + (k + 1 < nrows ? k + 1 : k) * kRowWords);
+            solve_row<0>(cur, K2D_ACC_OF(k), sv);
+            cur = nxt;
+        }
+    }
+#pragma unroll 1
+    for (int j = 0; j < SC::J; ++j) solve_joint<0>(load_joint(jrows + j * kJointWords), jrows + j * kJointWords, sj + j * kSolveThreads, sv);
+    // solver iterations: joints by index, then manifolds in pair order; the next row's constants are fetched while a row is solved
+#pragma unroll 1
+    for (int it = 0; it < prm.solver_iters; ++it) {
+        if (SC::J > 0) {
+            JointConsts cur = load_joint(jrows);
+#pragma unroll 1
+            for (int j = 0; j < SC::J; ++j) {
+                const JointConsts nxt = load_joint(jrows + (j + 1 < SC::J ? j + 1 : j) * kJointWords);
+                solve_joint<1>(cur, jrows + j * kJointWords, sj + j * kSolveThreads, sv);
+                cur = nxt;
+            }
+        }
+        RowConsts cur = load_row(rows);
+#pragma unroll 1
+        for (int k = 0; k < nrows; ++k) {
+            const RowConsts nxt = load_row(rows + (k + 1 < nrows ? k + 1 : k) * kRowWords);
+            solve_row<1>(cur, K2D_ACC_OF(k), sv);
+            cur = nxt;
+        }
+    }
+    // Euler step with the solved velocities; the velocities go back to the state record and the array holds positions from here on
+    bool finite = true;
+#pragma unroll
+    for (int i = 0; i < SC::N; ++i) {
+        const float4 v4 = sv[i * kSolveThreads];
+        float4 p4 = ld4(stf + SC::ST_POS + 4 * i);
+        if ((active >> i) & 1u) { p4.x = __fmaf_rn(prm.dt, v4.x, p4.x); p4.y = __fmaf_rn(prm.dt, v4.y, p4.y); p4.z = __fmaf_rn(prm.dt, v4.z, p4.z); }
+        finite = finite && finite_bits(v4.x) && finite_bits(v4.y) && finite_bits(v4.z);
+        st4(stf + SC::ST_VEL + 4 * i, v4.x, v4.y, v4.z);
+        sv[i * kSolveThreads] = p4;
+    }
+    // positional corrections: every active manifold moves its two bodies apart along the normal, then the joints close their gaps
+#pragma unroll 1
+    for (int k = 0; k < nrows; ++k) {
+        const float *r = rows + k * kRowWords;
+        const float4 h0 = __ldg(reinterpret_cast<const float4 *>(r + R_AB));
+        const float2 mm = __ldg(reinterpret_cast<const float2 *>(r + R_MA));
+        const float corr = __ldg(r + R_CORR);
+        const uint32_t ab = __float_as_uint(h0.x);
+        const int a = ab & 31, b = (ab >> 5) & 31;
+        const float ca = mm.x * corr, cb = mm.y * corr;
+        if ((ab >> 10) & 1u) { float4 p = sv[a * kSolveThreads]; p.x = __fmaf_rn(-ca, h0.y, p.x); p.y = __fmaf_rn(-ca, h0.z, p.y); sv[a * kSolveThreads] = p; }
+        if ((ab >> 11) & 1u) { float4 p = sv[b * kSolveThreads]; p.x = __fmaf_rn(cb, h0.y, p.x); p.y = __fmaf_rn(cb, h0.z, p.y); sv[b * kSolveThreads] = p; }
+    }
+#pragma unroll 1
+    for (int j = 0; j < SC::J; ++j) {
+        const JointConsts c = load_joint(jrows + j * kJointWords);
+        const uint32_t jab = __float_as_uint(c.k.w);
+        if (!((jab >> 24) & 1u)) continue;
+        const int a = jab & 255, b = (jab >> 8) & 255;
+        const float cx = c.b.z, cy = c.b.w, ma = c.m.x, mb = c.m.y;
+        if ((jab >> 29) & 1u) { float4 p = sv[a * kSolveThreads]; p.x = __fmaf_rn(ma, cx, p.x); p.y = __fmaf_rn(ma, cy, p.y); sv[a * kSolveThreads] = p; }
+        if ((jab >> 30) & 1u) { float4 p = sv[b * kSolveThreads]; p.x = __fmaf_rn(-mb, cx, p.x); p.y = __fmaf_rn(-mb, cy, p.y); sv[b * kSolveThreads] = p; }
+    }
+#pragma unroll
+    for (int i = 0; i < SC::N; ++i) {
+        const float4 p4 = sv[i * kSolveThreads];
+        finite = finite && finite_bits(p4.x) && finite_bits(p4.y) && finite_bits(p4.z);
+        st4(stf + SC::ST_POS + 4 * i, p4.x, p4.y, p4.z);
+    }
+    // reward and termination (paper, "Reward"): green touches blue = +1, green touches red = -1, either ends the episode
+    const int step_count = (int)m0.x + 1;
+    const bool touch_gb = (flags & 1u) != 0u, touch_gr = (flags & 2u) != 0u;
+    const bool timeout = prm.max_episode_steps > 0 && step_count >= prm.max_episode_steps;
+    float reward = (float)((int)touch_gb - (int)touch_gr);
+    if (prm.dense_kappa != 0.0f && ((flags >> 2) & 1u)) {
+        const float4 pg = sv[((flags >> 8) & 255u) * kSolveThreads], pb = sv[((flags >> 16) & 255u) * kSolveThreads];
+        const float dx = pb.x - pg.x, dy = pb.y - pg.y;
+        reward = reward + prm.dense_kappa * (__uint_as_float(m1.z) - sqrtf(dot2(dx, dy, dx, dy)));
+    }
+    bool done = touch_gb || touch_gr || timeout;
+    uint32_t status = m0.w;
+    if (!finite) { reward = 0.0f; done = true; status |= 1u; atomicAdd(prm.counters + 0, 1ULL); }
+    prm.reward[e] = reward;
+    prm.done[e] = done ? 1 : 0;
+    if (!(done && prm.auto_reset != 0)) {
+        // the accumulated impulses of this step's rows warm-start the next step
+#pragma unroll 1
+        for (int k = 0; k < nrows; ++k) {
+            const float2 acc = *K2D_ACC_OF(k);
+            st[SC::ST_WARM + kWarmWords * k] = __float_as_uint(__ldg(rows + k * kRowWords + R_KEY));
+            st[SC::ST_WARM + kWarmWords * k + 1] = __float_as_uint(acc.x);
+            st[SC::ST_WARM + kWarmWords * k + 2] = __float_as_uint(acc.y);
+        }
+#pragma unroll
+        for (int j = 0; j < SC::J; ++j) {
+            const float4 a4 = sj[j * kSolveThreads];
+            st[SC::ST_JACC + 3 * j] = __float_as_uint(a4.x);
+            st[SC::ST_JACC + 3 * j + 1] = __float_as_uint(a4.y);
+            st[SC::ST_JACC + 3 * j + 2] = __float_as_uint(a4.z);
+        }
+        st[SC::ST_META + META_STEP] = (uint32_t)step_count;
+        st[SC::ST_META + META_STATUS] = status;
+        return;
+    }
+#undef K2D_ACC_OF
+    // auto-reset of a finished env: next level (its own, or drawn from the pool by the hash of seed, global env index
+    // and episode), pose from the level, no accumulated impulses
+    const int episode = (int)m0.y + 1;
+    int level = (int)m0.z;
+    if (prm.auto_reset == 2) {
+        const unsigned long long h = mix64(prm.seed + ((unsigned long long)(prm.env_offset + e) + 1ULL) * 0x9E3779B97F4A7C15ULL +
+                                           (unsigned long long)episode * 0xD1B54A32D192ED03ULL);
+        level = (int)(h % (unsigned long long)prm.n_levels);
+    }
+    const float *lv = reinterpret_cast<const float *>(prm.levels + (size_t)level * SC::LV_WORDS);
+#pragma unroll 1
+    for (int i = 0; i < SC::N; ++i) {
+        st4(stf + SC::ST_POS + 4 * i, lv[SC::LV_X + i], lv[SC::LV_Y + i], lv[SC::LV_TH + i]);
+        st4(stf + SC::ST_VEL + 4 * i, lv[SC::LV_VX + i], lv[SC::LV_VY + i], lv[SC::LV_W + i]);
+    }
+    for (int j = 0; j < 3 * SC::J; ++j) st[SC::ST_JACC + j] = 0u;
+    *reinterpret_cast<uint4 *>(st + SC::ST_META) = make_uint4(0u, (uint32_t)episode, (uint32_t)level, 0u);
+    st[SC::ST_META + META_NROWS] = 0u;
+    atomicAdd(prm.counters + 1, 1ULL);
+}
+
+// ---------------------------------------------------------------- reset kernel: one block per env
 template <class SC>
 __global__ void k2d_reset_kernel(uint32_t *state, const uint32_t *levels, const int *level_ids, int n_envs, int n_levels) {
     const int e = blockIdx.x;
@@ -1574,8 +1144,10 @@ __global__ void k2d_reset_kernel(uint32_t *state, const uint32_t *levels, const 
     const uint32_t *lv = levels + (size_t)l * SC::LV_WORDS;
     for (int i = threadIdx.x; i < SC::ST_WARM; i += blockDim.x) {
         uint32_t v = 0u;
-        if (i < 6 * SC::N) v = lv[SC::LV_X + i];
-        else if (i == SC::ST_META + 2) v = (uint32_t)l;
+        if (i < 8 * SC::N) {
+            const int half = i / (4 * SC::N), r = i - half * 4 * SC::N, body = r >> 2, f = r & 3;     // position or velocity group, body, component
+            if (f < 3) v = lv[SC::LV_X + (3 * half + f) * SC::N + body];
+        } else if (i == SC::ST_META + META_LEVEL) v = (uint32_t)l;
         st[i] = v;
     }
 }
@@ -1597,13 +1169,13 @@ __global__ void __launch_bounds__(kObsThreads) k2d_obs_kernel(const uint32_t *st
     float *img = obs_smem + (size_t)w * ((width + 2 * SC::N + 3) / 4 * 4);
     float *cs = img + width;                 // cos, sin of every shape's angle
     const uint32_t *st = state + (size_t)e * SC::ST_WORDS;
-    const uint32_t *lv = levels + (size_t)st[SC::ST_META + 2] * SC::LV_WORDS;
+    const uint32_t *lv = levels + (size_t)st[SC::ST_META + META_LEVEL] * SC::LV_WORDS;
     const float *stf = reinterpret_cast<const float *>(st);
     const float *lvf = reinterpret_cast<const float *>(lv);
     for (int ci = lane; ci < n_shapes; ci += 32) {
         const int i = ci < n_polygons ? ci : SC::P + (ci - n_polygons);     // internal shape index
         float c, sn;
-        sincos_spec(stf[2 * SC::N + i], c, sn);
+        sincos_spec(stf[SC::ST_POS + 4 * i + 2], c, sn);
         cs[i] = c; cs[SC::N + i] = sn;
         float *o = img + ci * 29;
         const uint32_t fl = lv[SC::LV_FLAGS + i];
@@ -1614,9 +1186,9 @@ __global__ void __launch_bounds__(kObsThreads) k2d_obs_kernel(const uint32_t *st
         const int nv = flag_nverts(fl);
         const uint32_t role = flag_role(fl);
         const bool poly = i < SC::P;
-        o[0] = stf[i]; o[1] = stf[SC::N + i]; o[2] = stf[3 * SC::N + i]; o[3] = stf[4 * SC::N + i];
+        o[0] = stf[SC::ST_POS + 4 * i]; o[1] = stf[SC::ST_POS + 4 * i + 1]; o[2] = stf[SC::ST_VEL + 4 * i]; o[3] = stf[SC::ST_VEL + 4 * i + 1];
         o[4] = lvf[SC::LV_IM + i]; o[5] = lvf[SC::LV_II + i]; o[6] = lvf[SC::LV_DENS + i];
-        o[7] = tanh_spec(stf[5 * SC::N + i] * 0.1f);
+        o[7] = tanh_spec(stf[SC::ST_VEL + 4 * i + 2] * 0.1f);
 #pragma unroll
         for (int r = 0; r < 4; ++r) o[8 + r] = (role == (uint32_t)r) ? 1.0f : 0.0f;
         o[12] = sn; o[13] = c; o[14] = lvf[SC::LV_FR + i]; o[15] = lvf[SC::LV_RE + i];
@@ -1708,14 +1280,14 @@ __global__ void __launch_bounds__(kRenderThreads) k2d_render_kernel(const uint32
         const uint32_t fl = lv[SC::LV_FLAGS + i];
         int nv = -1;
         if (fl & F_ACTIVE) {
-            const float x = stf[i], y = stf[SC::N + i];
+            const float x = stf[SC::ST_POS + 4 * i], y = stf[SC::ST_POS + 4 * i + 1];
             const uint32_t role = flag_role(fl);
             uint32_t rgb = role == 1u ? (200u << 8) : role == 2u ? (220u << 16) : role == 3u ? 220u : ((fl & F_DYNAMIC) ? 0x808080u : 0x404040u);
             s_col[i] = rgb | 0xff000000u;
             if (i < SC::P) {
                 nv = (int)flag_nverts(fl);
                 float c, sn;
-                sincos_spec(stf[2 * SC::N + i], c, sn);
+                sincos_spec(stf[SC::ST_POS + 4 * i + 2], c, sn);
                 float nxs[4] = { 0.0f, 0.0f, 0.0f, 0.0f }, nys[4] = { 0.0f, 0.0f, 0.0f, 0.0f }, offs[4] = { 0.0f, 0.0f, 0.0f, 0.0f };
                 float x0 = 0.0f, y0 = 0.0f, x1 = 0.0f, y1 = 0.0f;
 #pragma unroll
