@@ -178,12 +178,12 @@ int k2d_step_discrete(k2d_state *s, const int32_t *dev_actions, int32_t n_steps,
 
 /* The paper has no counterpart of this call; it exists for one kind of user of this library.
  * k2d_step hands the constraint rows of a step from its first kernel to its second through the
- * scratch tail of the state buffer (19776 bytes per env for the largest scenes), which the caller
+ * scratch tail of the state buffer (19904 bytes per env for the largest scenes), which the caller
  * has to allocate.  Some callers cannot: a process whose device memory is one arena fixed at start-up,
  * a plug-in handed a pre-sized buffer by its host, code running where cudaMalloc is forbidden
  * (a real-time loop).  For them this variant does exactly what k2d_step does, with the same
  * arguments and bit-identical results, but keeps those rows in an array compiled into the
- * library (K2D_STATIC_SCRATCH_MAX_ENVS x 19776 bytes, about 20 MB, resident on every GPU that
+ * library (K2D_STATIC_SCRATCH_MAX_ENVS x 19904 bytes, about 20 MB, resident on every GPU that
  * loads the library until the process exits) and never touches the scratch tail; a state buffer of
  * k2d_state_bytes_no_scratch bytes is enough for a handle that is only ever stepped this way.  It
  * allocates and frees nothing, on the host side of CUDA or on the device.

@@ -258,7 +258,8 @@ static cudaError_t launch_step(const k2d_state *s, const StepParams &prm) {
     k2d_prep_kernel<SC, G><<<s->grid, kBlockThreads, s->smem_bytes, s->stream>>>(prm);
     cudaError_t err = cudaGetLastError();
     if (err != cudaSuccess) return err;
-    k2d_solve_kernel<SC><<<(prm.n_envs + kSolveThreads - 1) / kSolveThreads, kSolveThreads, 0, s->stream>>>(prm);
+    constexpr int SPB = kSolveThreads / kSolveLanes;      // scenes per block of the solve kernel
+    k2d_solve_kernel<SC><<<(prm.n_envs + SPB - 1) / SPB, kSolveThreads, 0, s->stream>>>(prm);
     return cudaGetLastError();
 }
 template <class SC, int G>
@@ -497,16 +498,16 @@ int k2d_get_state(k2d_state *s, void *host_canonical) {
             o[3 * nN + 2 * i] = vq[0]; o[3 * nN + 2 * i + 1] = vq[1];
             o[5 * nN + i] = vq[2];
         }
-        // the warm list holds (slot key = 2 x pair + manifold, accumulated normal, tangent impulse) of the latest step's rows
+        // the warm list holds (pair, accumulated normal and tangent impulse of its two manifolds) of the latest step's rows
         uint32_t *acc = o + 6 * nN;
         const int nrows = (int)st[ci.ST_META + META_NROWS];
-        for (int k = 0; k < nrows && k < ci.NSLOTS; ++k) {
+        for (int k = 0; k < nrows && k < ci.NPAIRS; ++k) {
             const uint32_t *wr = st + ci.ST_WARM + kWarmWords * k;
-            const uint32_t key = wr[0];
-            const int p = (key < 2u * (uint32_t)ci.NPAIRS) ? inv_pair[key >> 1] : -1;
+            const int p = (wr[0] < (uint32_t)ci.NPAIRS) ? inv_pair[wr[0]] : -1;
             if (p < 0) continue;
-            const int slot = pair_slot(nP, nC, p) + (int)(key & 1u);
+            const int slot = pair_slot(nP, nC, p);
             acc[2 * slot] = wr[1]; acc[2 * slot + 1] = wr[2];
+            if (p < nP * (nP - 1) / 2) { acc[2 * slot + 2] = wr[3]; acc[2 * slot + 3] = wr[4]; }
         }
         uint32_t *jacc = acc + 2 * n_slots;
         for (int j = 0; j < 3 * nJ; ++j) jacc[j] = st[ci.ST_JACC + j];
@@ -549,13 +550,11 @@ int k2d_set_state(k2d_state *s, const void *host_canonical) {
         int nrows = 0;
         for (int p = 0; p < n_pairs; ++p) {
             const int slot = pair_slot(nP, nC, p);
-            const int n_man = p < nP * (nP - 1) / 2 ? 2 : 1;
-            for (int mi = 0; mi < n_man; ++mi) {
-                const uint32_t vn = acc[2 * (slot + mi)], vt = acc[2 * (slot + mi) + 1];
-                if (!((vn | vt) & 0x7fffffffu)) continue;
-                uint32_t *wr = st + ci.ST_WARM + kWarmWords * nrows++;
-                wr[0] = 2u * (uint32_t)s->pair_map[p] + (uint32_t)mi; wr[1] = vn; wr[2] = vt;
-            }
+            const bool two = p < nP * (nP - 1) / 2;
+            const uint32_t v[4] = { acc[2 * slot], acc[2 * slot + 1], two ? acc[2 * slot + 2] : 0u, two ? acc[2 * slot + 3] : 0u };
+            if (!((v[0] | v[1] | v[2] | v[3]) & 0x7fffffffu)) continue;
+            uint32_t *wr = st + ci.ST_WARM + kWarmWords * nrows++;
+            wr[0] = (uint32_t)s->pair_map[p]; wr[1] = v[0]; wr[2] = v[1]; wr[3] = v[2]; wr[4] = v[3];
         }
         const uint32_t *jacc = acc + 2 * n_slots;
         for (int j = 0; j < 3 * nJ; ++j) st[ci.ST_JACC + j] = jacc[j];

@@ -4,26 +4,28 @@
 //
 //   k2d_prep_kernel   A group of G lanes (G = 16: two scenes per warp; 32: one warp per scene; 8: four per warp)
 //                     takes one scene at a time from a ticket queue.  Its lanes work on bodies, polygon vertices,
-//                     shape pairs (bounding-box test, narrowphase) and contact manifolds (one per lane): gravity,
+//                     shape pairs (bounding-box test, narrowphase) and touching pairs (one per lane): gravity,
 //                     world-frame geometry, motors, thrusters, joint pre-step, manifolds, touch flags, and the
-//                     pre-step of every active manifold.  It leaves the step's constraint rows (one 80-byte row per
-//                     active manifold, in canonical order, and one 96-byte row per joint) in the env's scratch
+//                     pre-step of every touching pair.  It leaves the step's constraint rows (one 112-byte row per
+//                     touching pair, sorted by solver level, and one 96-byte row per joint) in the env's scratch
 //                     area and the velocities in the env's state record.
-//   k2d_solve_kernel  One thread per env walks that env's rows strictly in the canonical order (warm start, solver
-//                     iterations of joints then contacts, Euler step, positional corrections), then does the
-//                     reward, the termination and the auto-reset.  The velocities of the env's bodies sit in shared
-//                     memory as one 16-byte group per (body, thread), which no two threads of a warp share a bank
-//                     for, whatever body each of them addresses.
+//   k2d_solve_kernel  A group of 4 lanes (eight scenes per warp) runs the warm start, the solver iterations, the Euler
+//                     step and the positional corrections over those rows, then the reward, the termination and the
+//                     auto-reset.  Only the bodies' velocities (later positions) and the accumulated impulses are in
+//                     shared memory; the rows' constants are read through the read-only cache.
 //
-// The sequential-impulse solver is a chain of dependent rows per scene, so a scene offers little to the lanes of a
-// warp; 32 scenes side by side offer 32 independent chains.  The geometry of a scene, on the other hand, is wide
-// (120 pairs to test for the largest size class) and needs its working set in shared memory, which is why that
-// part keeps several lanes per scene.
+// The sequential-impulse solver of a scene is a chain of dependent rows with two or three independent rows per link,
+// so it can feed few lanes; its working set is small.  The geometry of a scene is wide (120 pairs to test for the
+// largest size class) and needs a working set of several kilobytes in shared memory.  Hence two kernels with
+// different lanes per scene and different occupancy.
 //
 // Arithmetic contract: every +,-,*,/,sqrt is an individually rounded IEEE binary32 operation
 // (the file is compiled with --fmad=false --prec-div=true --prec-sqrt=true --ftz=false), a fused
 // multiply-add appears only where the code says __fmaf_rn, and min/max are comparisons.  The solver visits
-// the rows one after the other in the canonical order (joints by index, then manifolds by pair index and slot).
+// rows in an order equivalent to the canonical one (joints by index, then touching pairs by pair index): "level
+// scheduling": a row's level is one more than the highest level of an earlier row that shares a movable body with it;
+// rows of one level touch disjoint movable bodies and run on different lanes at once, and levels run in order, so every
+// body sees exactly the sequence of updates a one-row-at-a-time sweep would give it: results are bit-identical to that sweep.
 #pragma once
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -39,15 +41,20 @@ constexpr int kBlockThreads = K2D_BLOCK_THREADS;
 #endif
 constexpr int kMinBlocks = K2D_MIN_BLOCKS;   // resident blocks per SM the prep kernel is compiled for (bounds its registers)
 #ifndef K2D_SOLVE_THREADS
-#define K2D_SOLVE_THREADS 32
+#define K2D_SOLVE_THREADS 64
 #endif
-constexpr int kSolveThreads = K2D_SOLVE_THREADS;   // solve kernel: one env per thread
+constexpr int kSolveThreads = K2D_SOLVE_THREADS;
+#ifndef K2D_SOLVE_LANES
+#define K2D_SOLVE_LANES 4
+#endif
+constexpr int kSolveLanes = K2D_SOLVE_LANES;       // solve kernel: lanes per scene
 constexpr int kObsThreads = 128;   // observation kernel: one warp per env, four envs per block
 constexpr int kMaxActions = 16;
 enum { Q_TICKET = 0, Q_LEFT = 1 };
-constexpr int kRowWords = 20;   // one active manifold: five 16-byte groups
-constexpr int kWarmWords = 3;   // slot key, accumulated normal and tangent impulse
+constexpr int kRowWords = 28;   // one touching pair: seven 16-byte groups
+constexpr int kWarmWords = 5;   // pair index + 4 accumulated impulses
 constexpr int kStageWords = 9;  // packed pair word, normal, two contact points with penetration
+constexpr int kStageStride = 12; // a staged pair in scratch: the stage words, then the row slot it is to fill
 constexpr int kJointWords = 24; // joint row: six 16-byte groups
 constexpr int kJointLevelWords = 12;  // joint record of a level
 
@@ -74,12 +81,14 @@ struct SizeClass {
     // accumulated joint impulses, and the accumulated impulses of the manifolds that were active in the latest step
     static constexpr int ST_POS = 0, ST_VEL = 4 * N, ST_META = 8 * N, ST_JACC = ST_META + 8;
     static constexpr int ST_WARM = (ST_JACC + 3 * J + 3) / 4 * 4;
-    static constexpr int ST_WORDS = (ST_WARM + kWarmWords * NSLOTS + 3) / 4 * 4;
-    // scratch of an env, valid from the prep kernel of a step to its solve kernel: manifold rows, then joint rows.
-    // Room for two rows per pair: a pair staged beyond the first G of a scene waits in the row slot 2 k + 1.
-    static constexpr int ROW_CAP = 2 * NPAIRS;
-    static constexpr int SCR_ROWS = 0, SCR_JROW = ROW_CAP * kRowWords;
-    static constexpr int SCRATCH_WORDS = SCR_JROW + kJointWords * J;
+    static constexpr int ST_WORDS = (ST_WARM + kWarmWords * NPAIRS + 3) / 4 * 4;
+    // scratch of an env, valid from the prep kernel of a step to its solve kernel: pair rows sorted by level, joint rows,
+    // the first row of every level (bytes; entry L for level L, entry highest level + 1 = number of rows), and a
+    // staging area for the pairs of a scene with more touching pairs than lanes
+    static constexpr int SCR_ROWS = 0, SCR_JROW = NPAIRS * kRowWords;
+    static constexpr int SCR_LSTART = SCR_JROW + kJointWords * J;
+    static constexpr int SCR_STAGE = SCR_LSTART + ((NPAIRS + 2 + 3) / 4 + 3) / 4 * 4;
+    static constexpr int SCRATCH_WORDS = SCR_STAGE + kStageStride * NPAIRS;
     // shared memory region of one scene in the prep kernel (words)
     // per body 16-byte groups (x, y, angle, -) and (vx, vy, angular velocity, -), then per-body arrays
     static constexpr int BPOS = 0, BVEL = 4 * N;
@@ -90,31 +99,36 @@ struct SizeClass {
     static constexpr int MASK = BOX + 4 * N;
     static constexpr int ACT = MASK + MASKW;
     static constexpr int META = ACT + kMaxActions;       // the state record's meta words
-    static constexpr int ELEN = (META + 8 + 3) / 4 * 4;  // edge lengths of the level's polygons
-    static constexpr int SURV = ELEN + P4;               // bytes: pairs that passed the box test
-    static constexpr int WIDX = SURV + (NPAIRS + 3) / 4; // bytes: manifold slot key -> entry of the previous step's warm list
-    // then, per lane of the group (field-major, G words per field): kStageWords fields, manifolds on their way to the
-    // lane that builds their rows
-    static constexpr int STG = WIDX + (2 * NPAIRS + 3) / 4;
+    static constexpr int LVC = (META + 8 + 3) / 4 * 4;   // copy of the level record's edge lengths, joint and thruster records
+    static constexpr int LVC_WORDS = LV_MASK - LV_ELEN;
+    static constexpr int ELEN = LVC, LVC_JOINT = LVC + (LV_JOINT - LV_ELEN), LVC_THR = LVC + (LV_THR - LV_ELEN);
+    static constexpr int SURV = LVC + LVC_WORDS;         // bytes: pairs that passed the box test; afterwards per-body words of the level search
+    static constexpr int WIDX = SURV + ((NPAIRS + 3) / 4 > N ? (NPAIRS + 3) / 4 : N); // bytes: pair -> entry of the previous step's warm list
+    // then, per lane of the group (field-major, G words per field): kStageWords fields, touching pairs on their way to
+    // the lane that builds their rows
+    static constexpr int STG = WIDX + (NPAIRS + 3) / 4;
     static constexpr int PTAB_WORDS = ((NPAIRS + 1) / 2 + 3) / 4 * 4;  // block-shared pair table, 16 bits per pair
 };
-// manifold row (scratch): what the solver needs of one active manifold
-enum { R_AB = 0, R_NX, R_NY, R_MU, R_MA, R_MB, R_IA, R_IB, R_RNA, R_RNB, R_RTA, R_RTB, R_MASSN, R_MASST, R_TARGET, R_CORR,
-       R_ACCN, R_ACCT, R_KEY, R_PAD };
-static_assert(R_PAD + 1 == kRowWords, "row size");
-// row AB word: a | b<<5 | a movable<<10 | b movable<<11
+// pair row (scratch): what the solver needs of one touching pair: pair word, normal, friction | inverse masses and inertias |
+// per manifold the lever-arm cross products, effective masses, target normal velocity, positional correction | the four
+// accumulated impulses
+enum { R_AB = 0, R_NX, R_NY, R_MU, R_MA, R_MB, R_IA, R_IB, R_M0 = 8, R_M1 = 16, R_ACC = 24 };
+enum { M_RNA = 0, M_RNB, M_RTA, M_RTB, M_MASSN, M_MASST, M_TARGET, M_CORR };
+static_assert(R_ACC + 4 == kRowWords, "row size");
+// row AB word = staged AB word
 // staged manifold fields
 enum { S_AB = 0, S_NX, S_NY, S_PX0, S_PY0, S_PEN0, S_PX1, S_PY1, S_PEN1 };
 static_assert(S_PEN1 + 1 == kStageWords, "stage size");
-// staged AB word: a | b<<5 | active manifolds<<10 | pair<<12 | a movable<<26 | b movable<<27
+// staged AB word: a | b<<5 | active manifolds<<10 | pair<<12 | level<<19 | a movable<<26 | b movable<<27
 // joint row fields
 enum { JR_RAX = 0, JR_RAY, JR_RBX, JR_RBY, JR_I11, JR_I12, JR_I22, JR_JAB, JR_BX, JR_BY, JR_CX, JR_CY, JR_MA, JR_MB, JR_IA, JR_IB,
        JR_ACCX, JR_ACCY, JR_PAD1, JR_PAD2,
        JR_ANG, JR_KR, JR_BIASR, JR_ACCR };   // angular row: kind (0 none, 1 fixed, 2 beyond the upper limit, 3 beyond the lower), 1 / (1/I_a + 1/I_b), gamma x error, accumulated
 static_assert(JR_ACCR + 1 == kJointWords, "joint row size");
-// meta words of a state record.  FLAGS, D0 and ACTIVE are messages from the prep kernel to the solve kernel of the same step:
-// touch flags (green-blue | green-red << 1), the dense reward's shapes (both exist << 2 | green << 8 | blue << 16) and their
-// distance before the step, and the bit mask of the shapes that exist.
+// meta words of a state record.  NROWS is the number of pair rows of the latest step (= entries of the warm list).  FLAGS, D0
+// and ACTIVE are messages from the prep kernel to the solve kernel of the same step: touch flags (green-blue | green-red << 1),
+// the dense reward's shapes (both exist << 2 | green << 8 | blue << 16), the highest contact level << 24; the distance of
+// those shapes before the step; the bit mask of the shapes that exist | the highest joint level << 16.
 enum { META_STEP = 0, META_EPISODE, META_LEVEL, META_STATUS, META_NROWS, META_FLAGS, META_D0, META_ACTIVE };
 
 // shared-memory words per scene: padded so that the groups of one warp start in different banks
@@ -322,21 +336,12 @@ __device__ __forceinline__ uint16_t pair_code(int p) {
 }
 
 // ================================================================ rarely run code, kept out of line
-// level constants into shared memory; returns the packed word of joint number `lane` (0 beyond the last joint)
-template <class SC, int G>
-__device__ __forceinline__ uint32_t load_level_consts(uint32_t *smu, const uint32_t *lv) {
-    const int lane = Group<G>().lane;
-    for (int i = lane; i < SC::N; i += G) {
-        smu[SC::BIM + i] = lv[SC::LV_IM + i];
-        smu[SC::BII + i] = lv[SC::LV_II + i];
-        smu[SC::BFR + i] = lv[SC::LV_FR + i];
-        smu[SC::BRE + i] = lv[SC::LV_RE + i];
-        smu[SC::BFL + i] = lv[SC::LV_FLAGS + i];
-    }
-    for (int i = lane; i < SC::C; i += G) smu[SC::RAD + i] = lv[SC::LV_RAD + i];
-    for (int i = lane; i < SC::MASKW; i += G) smu[SC::MASK + i] = lv[SC::LV_MASK + i];
-    for (int i = lane; i < SC::P4; i += G) smu[SC::ELEN + i] = lv[SC::LV_ELEN + i];
-    return (SC::J > 0 && lane < SC::J) ? lv[SC::LV_JOINT + kJointLevelWords * lane] : 0u;
+// what the prep kernel reads of an env's meta words before it starts on the env
+struct MetaHead { uint32_t level, status, nprev; };
+__device__ __forceinline__ MetaHead load_meta_head(const uint32_t *st_meta) {
+    const uint4 m = __ldcg(reinterpret_cast<const uint4 *>(st_meta));
+    MetaHead h; h.level = m.z; h.status = m.w; h.nprev = __ldcg(st_meta + META_NROWS);
+    return h;
 }
 
 // packed work counters of a group to the global ones (lane 0)
@@ -359,11 +364,52 @@ __device__ __noinline__ void trace_clear(float *trace) {
     g.sync();
 }
 
+// A scene with more touching pairs than lanes: one lane walks the staged pairs in the scratch (in staging order), gives
+// each its level (into bits 19.. of its packed word) and its row slot (the word after the stage words), and fills the
+// table of level starts.  Returns the highest level.  bl: N bytes of shared memory.
+template <class SC>
+__device__ __noinline__ int place_crowded_impl(uint32_t *scr, uint8_t *lstart, uint8_t *bl, int nrec) {
+    uint32_t *stage = scr + SC::SCR_STAGE;
+    int cmax = 0;
+    for (int i = 0; i < SC::N; ++i) bl[i] = 0;
+    for (int L = 0; L <= nrec + 1; ++L) lstart[L] = 0;
+    for (int k = 0; k < nrec; ++k) {
+        uint32_t *w = stage + (size_t)k * kStageStride;
+        const uint32_t ab = w[S_AB];
+        const int a = ab & 31, b = (ab >> 5) & 31;
+        int lvl = 1;
+        if ((ab >> 26) & 1u) lvl = max(lvl, bl[a] + 1);
+        if ((ab >> 27) & 1u) lvl = max(lvl, bl[b] + 1);
+        if ((ab >> 26) & 1u) bl[a] = (uint8_t)lvl;
+        if ((ab >> 27) & 1u) bl[b] = (uint8_t)lvl;
+        w[S_AB] = ab | ((uint32_t)lvl << 19);
+        lstart[lvl] = (uint8_t)(lstart[lvl] + 1);
+        cmax = max(cmax, lvl);
+    }
+    // counts -> starts; a cursor per level in the spare word of stage entry level - 1
+    int run = 0;
+    for (int L = 1; L <= cmax; ++L) {
+        const int c = lstart[L];
+        lstart[L] = (uint8_t)run;
+        stage[(size_t)(L - 1) * kStageStride + kStageWords + 1] = (uint32_t)run;
+        run += c;
+    }
+    lstart[cmax + 1] = (uint8_t)run;
+    for (int k = 0; k < nrec; ++k) {
+        uint32_t *w = stage + (size_t)k * kStageStride;
+        const int lvl = (int)((w[S_AB] >> 19) & 127u);
+        uint32_t *cur = stage + (size_t)(lvl - 1) * kStageStride + kStageWords + 1;
+        w[kStageWords] = *cur;
+        *cur = *cur + 1u;
+    }
+    return cmax;
+}
+
 // ---------------------------------------------------------------- first half of a step: one scene per group of G lanes
 template <class SC, int G>
 struct Scene {
     static_assert(SC::J <= G && SC::T <= G && kMaxActions <= 2 * G, "one lane per joint / thruster");
-    static_assert(2 * SC::NPAIRS < 255, "manifold slot keys are bytes");
+    static_assert(SC::NPAIRS < 255, "pair indices are bytes");
     float *sm;            // this scene's shared-memory region
     uint32_t *smu;
     const uint16_t *ptab; // block-shared pair table
@@ -512,27 +558,88 @@ struct Scene {
         return m.pen > 0.0f ? 1u : 0u;
     }
 
-    // ---- the first half of one environment step of env e
-    __device__ __forceinline__ void prepare(int e) {
+    // ---- the first half of one environment step of env e (not frozen), whose meta head has been read already.
+    // tn_raw: lane 0's ticket for the group's next env, still in flight; on return next_e is that ticket for all lanes
+    // and next_head the env's meta head (if there is such an env), fetched while this env's pairs are tested.
+    __device__ __forceinline__ void prepare(int e, const MetaHead &head, unsigned tn_raw, unsigned &next_e, MetaHead &next_head) {
         uint32_t *st = prm.state + (size_t)e * SC::ST_WORDS;
         uint32_t *scr = prm.scratch + (size_t)e * SC::SCRATCH_WORDS;
-        // frozen env: nothing to prepare (the solve kernel reports done)
-        if (__ldcg(st + SC::ST_META + META_STATUS) & 1u) return;
-        const uint32_t *lv = prm.levels + (size_t)__ldcg(st + SC::ST_META + META_LEVEL) * SC::LV_WORDS;
-        const int nprev = (int)__ldcg(st + SC::ST_META + META_NROWS);
-        // state record -> shared memory (the same 16-byte groups), level constants, index of the previous step's impulses
-        for (int i = lane; i < 2 * SC::N; i += G)
-            reinterpret_cast<float4 *>(sm + SC::BPOS)[i] = __ldcg(reinterpret_cast<const float4 *>(st + SC::ST_POS) + i);
-        const uint32_t jab = load_level_consts<SC, G>(smu, lv);
-        for (int i = lane; i < (2 * SC::NPAIRS + 3) / 4; i += G) smu[SC::WIDX + i] = 0xffffffffu;
-        // actions of this step
-        const float *act_row = prm.actions + (size_t)e * prm.n_actions;
-        if (lane < prm.n_actions) sm[SC::ACT + lane] = act_row[lane];
-        if (G < kMaxActions && lane + G < prm.n_actions) sm[SC::ACT + lane + G] = act_row[lane + G];
+        const uint32_t *lv = prm.levels + (size_t)head.level * SC::LV_WORDS;
+        const int nprev = (int)head.nprev;
+        // Everything this step reads from memory is asked for here, in two volleys of loads that are all in flight before the
+        // first of them is used, so that the group waits for memory twice per step and not once per word: the state record
+        // (the same 16-byte groups as in shared memory), the level's constants, the body-frame vertices and normals (parked
+        // where their world-frame images will go), the action row, the previous step's warm list.
+        constexpr int KB = (2 * SC::N + G - 1) / G, KN = (SC::N + G - 1) / G, KV = (SC::P4 + G - 1) / G, KL = (SC::LVC_WORDS + G - 1) / G;
+        {
+            float4 body[KB];
+            uint32_t cim[KN], cii[KN], cfr[KN], cre[KN], cfl[KN], pvx[KV], pvy[KV], pnx[KV], pny[KV];
+#pragma unroll
+            for (int k = 0; k < KB; ++k) { const int i = lane + k * G; body[k] = (i < 2 * SC::N) ? __ldcg(reinterpret_cast<const float4 *>(st + SC::ST_POS) + i) : make_float4(0.0f, 0.0f, 0.0f, 0.0f); }
+#pragma unroll
+            for (int k = 0; k < KN; ++k) {
+                const int i = lane + k * G; const bool in = i < SC::N;
+                cim[k] = in ? __ldg(lv + SC::LV_IM + i) : 0u; cii[k] = in ? __ldg(lv + SC::LV_II + i) : 0u; cfr[k] = in ? __ldg(lv + SC::LV_FR + i) : 0u;
+                cre[k] = in ? __ldg(lv + SC::LV_RE + i) : 0u; cfl[k] = in ? __ldg(lv + SC::LV_FLAGS + i) : 0u;
+            }
+#pragma unroll
+            for (int k = 0; k < KV; ++k) {
+                const int v = lane + k * G; const bool in = v < SC::P4;
+                pvx[k] = in ? __ldg(lv + SC::LV_PVX + v) : 0u; pvy[k] = in ? __ldg(lv + SC::LV_PVY + v) : 0u;
+                pnx[k] = in ? __ldg(lv + SC::LV_PNX + v) : 0u; pny[k] = in ? __ldg(lv + SC::LV_PNY + v) : 0u;
+            }
+#pragma unroll
+            for (int k = 0; k < KB; ++k) { const int i = lane + k * G; if (i < 2 * SC::N) reinterpret_cast<float4 *>(sm + SC::BPOS)[i] = body[k]; }
+#pragma unroll
+            for (int k = 0; k < KN; ++k) {
+                const int i = lane + k * G;
+                if (i < SC::N) { smu[SC::BIM + i] = cim[k]; smu[SC::BII + i] = cii[k]; smu[SC::BFR + i] = cfr[k]; smu[SC::BRE + i] = cre[k]; smu[SC::BFL + i] = cfl[k]; }
+            }
+#pragma unroll
+            for (int k = 0; k < KV; ++k) {
+                const int v = lane + k * G;
+                if (v < SC::P4) { smu[SC::WVX + v] = pvx[k]; smu[SC::WVY + v] = pvy[k]; smu[SC::WNX + v] = pnx[k]; smu[SC::WNY + v] = pny[k]; }
+            }
+        }
+        uint32_t gb;
+        uint32_t wpair = 255u;
+        float4 wacc = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+        float jacc0 = 0.0f, jacc1 = 0.0f, jacc2 = 0.0f;
+        {
+            uint32_t lvc[KL], rad = 0u, msk = 0u, act0 = 0u, act1 = 0u;
+#pragma unroll
+            for (int k = 0; k < KL; ++k) { const int i = lane + k * G; lvc[k] = (i < SC::LVC_WORDS) ? __ldg(lv + SC::LV_ELEN + i) : 0u; }
+            static_assert(SC::C <= G && SC::MASKW <= G, "one lane per circle / mask word");
+            if (lane < SC::C) rad = __ldg(lv + SC::LV_RAD + lane);
+            if (lane < SC::MASKW) msk = __ldg(lv + SC::LV_MASK + lane);
+            const uint32_t *act_row = reinterpret_cast<const uint32_t *>(prm.actions) + (size_t)e * prm.n_actions;
+            if (lane < prm.n_actions) act0 = __ldg(act_row + lane);
+            if (G < kMaxActions && lane + G < prm.n_actions) act1 = __ldg(act_row + lane + G);
+            gb = __ldg(lv + SC::LV_GB);
+            // the previous step's accumulated impulses: entry k stays with lane k (entries beyond the lanes are read from the
+            // state record when needed); the byte table maps a pair to its entry
+            if (lane < nprev) {
+                const uint32_t *wr = st + SC::ST_WARM + kWarmWords * lane;
+                wpair = __ldcg(wr);
+                wacc = make_float4(__uint_as_float(__ldcg(wr + 1)), __uint_as_float(__ldcg(wr + 2)), __uint_as_float(__ldcg(wr + 3)), __uint_as_float(__ldcg(wr + 4)));
+            }
+            if (SC::J > 0 && lane < SC::J) {
+                jacc0 = __uint_as_float(__ldcg(st + SC::ST_JACC + 3 * lane)); jacc1 = __uint_as_float(__ldcg(st + SC::ST_JACC + 3 * lane + 1));
+                jacc2 = __uint_as_float(__ldcg(st + SC::ST_JACC + 3 * lane + 2));
+            }
+#pragma unroll
+            for (int k = 0; k < KL; ++k) { const int i = lane + k * G; if (i < SC::LVC_WORDS) smu[SC::LVC + i] = lvc[k]; }
+            if (lane < SC::C) smu[SC::RAD + lane] = rad;
+            if (lane < SC::MASKW) smu[SC::MASK + lane] = msk;
+            if (lane < prm.n_actions) smu[SC::ACT + lane] = act0;
+            if (G < kMaxActions && lane + G < prm.n_actions) smu[SC::ACT + lane + G] = act1;
+        }
+        for (int i = lane; i < (SC::NPAIRS + 3) / 4; i += G) smu[SC::WIDX + i] = 0xffffffffu;
         g.sync();
-        for (int k = lane; k < nprev; k += G) widx()[__ldcg(st + SC::ST_WARM + kWarmWords * k)] = (uint8_t)k;
+        if (wpair != 255u) widx()[wpair] = (uint8_t)lane;
+        for (int k = G + lane; k < nprev; k += G) widx()[__ldcg(st + SC::ST_WARM + kWarmWords * k)] = (uint8_t)k;
+        const uint32_t jab = (SC::J > 0 && lane < SC::J) ? smu[SC::LVC_JOINT + kJointLevelWords * lane] : 0u;
         // dense reward: the first green and the first blue shape, and their distance before the step
-        const uint32_t gb = lv[SC::LV_GB];
         float d0 = 0.0f;
         if (prm.dense_kappa != 0.0f && ((gb >> 16) & 1u)) {
             const float4 pg = ld4(sm + SC::BPOS + 4 * (gb & 255u)), pb = ld4(sm + SC::BPOS + 4 * ((gb >> 8) & 255u));
@@ -559,14 +666,14 @@ struct Scene {
             active_mask |= g.ballot(act_i) << base;
         }
         g.sync();
-        // world-frame polygon vertices, normals, face offsets
+        // world-frame polygon vertices, normals, face offsets (each lane turns the body-frame values it parked)
         for (int v = lane; v < SC::P4; v += G) {
             const int i = v >> 2, k = v & 3;
             if (k < (int)flag_nverts(smu[SC::BFL + i])) {
                 const float c = sm[SC::BC + i], sn = sm[SC::BS + i];
                 float rx, ry, nx, ny;
-                rot2(c, sn, __uint_as_float(lv[SC::LV_PVX + v]), __uint_as_float(lv[SC::LV_PVY + v]), rx, ry);
-                rot2(c, sn, __uint_as_float(lv[SC::LV_PNX + v]), __uint_as_float(lv[SC::LV_PNY + v]), nx, ny);
+                rot2(c, sn, sm[SC::WVX + v], sm[SC::WVY + v], rx, ry);
+                rot2(c, sn, sm[SC::WNX + v], sm[SC::WNY + v], nx, ny);
                 const float wx = rx + sm[SC::BPOS + 4 * i], wy = ry + sm[SC::BPOS + 4 * i + 1];
                 sm[SC::WVX + v] = wx; sm[SC::WVY + v] = wy; sm[SC::WNX + v] = nx; sm[SC::WNY + v] = ny;
                 sm[SC::WOFF + v] = dot2(nx, ny, wx, wy);
@@ -576,7 +683,7 @@ struct Scene {
         const bool jon = ((jab >> 24) & 1u) != 0u;
         const int jlevel = jon ? (int)((jab >> 25) & 7u) : 0;
         const int jmax = (SC::J > 0) ? g.max_int(jlevel) : 0;
-        const uint32_t *jl = lv + SC::LV_JOINT + kJointLevelWords * (lane < SC::J ? lane : 0);
+        const uint32_t *jl = smu + SC::LVC_JOINT + kJointLevelWords * (lane < SC::J ? lane : 0);
         g.sync();
         // polygon boxes
         for (int i = lane; i < SC::P; i += G) {
@@ -614,7 +721,7 @@ struct Scene {
         // thrusters in thruster order, by level in the same way
         if (SC::T > 0) {
             int tl = 0; uint32_t tp = 0u;
-            const uint32_t *th = lv + SC::LV_THR + 8 * (lane < SC::T ? lane : 0);
+            const uint32_t *th = smu + SC::LVC_THR + 8 * (lane < SC::T ? lane : 0);
             if (lane < SC::T) { tp = th[0]; if ((tp >> 16) & 1u) tl = (tp >> 17) & 7u; }
             const int tmax = g.max_int(tl);
 #pragma unroll 1
@@ -638,13 +745,13 @@ struct Scene {
                 g.sync();
             }
         }
+        g.sync();       // boxes and velocities are final
         // joint pre-step (poses only; velocities are not read): the row goes to the env's scratch
         if (SC::J > 0 && lane < SC::J) {
             float4 q[6];
 #pragma unroll
             for (int f = 0; f < 6; ++f) q[f] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
-            float accx = __uint_as_float(__ldcg(st + SC::ST_JACC + 3 * lane)), accy = __uint_as_float(__ldcg(st + SC::ST_JACC + 3 * lane + 1));
-            float accr = __uint_as_float(__ldcg(st + SC::ST_JACC + 3 * lane + 2));
+            float accx = jacc0, accy = jacc1, accr = jacc2;
             if (!jon || !prm.warm_start) { accx = 0.0f; accy = 0.0f; accr = 0.0f; }
             int ang = 0;
             float kr = 0.0f, bias_r = 0.0f;
@@ -687,7 +794,6 @@ struct Scene {
 #pragma unroll
             for (int f = 0; f < 6; ++f) jr[f] = q[f];
         }
-        g.sync();
 
         // bounding-box test over all pairs -> compact list of surviving pairs, in pair order
         int nsurv = 0, ns_pp, ns_pc;
@@ -715,9 +821,12 @@ struct Scene {
         g.sync();
         c_surv += (unsigned)ns_pp | ((unsigned)(ns_pc - ns_pp) << 16);
         c_rec += (unsigned)(nsurv - ns_pc);
+        // the group's next env: its ticket has arrived by now; its meta head will have by the end of this env
+        next_e = g.shflu(tn_raw, 0);
+        if (next_e < (unsigned)prm.n_envs) next_head = load_meta_head(prm.state + (size_t)next_e * SC::ST_WORDS + SC::ST_META);
 
         // narrowphase: survivors of one kind at a time; pairs with an active manifold are staged in pair order, the
-        // first G of them in shared memory, later ones in the row slots 2 k + 1 of the env's scratch
+        // first G of them in shared memory, later ones in the staging area of the env's scratch
         int nrec = 0;
         bool t_gb = false, t_gr = false;
         float *trace = prm.trace ? prm.trace + (size_t)e * SC::NSLOTS * 6 : nullptr;
@@ -759,7 +868,7 @@ struct Scene {
                         sg[S_PX0 * G] = m[0].px; sg[S_PY0 * G] = m[0].py; sg[S_PEN0 * G] = m[0].pen;
                         sg[S_PX1 * G] = m[1].px; sg[S_PY1 * G] = m[1].py; sg[S_PEN1 * G] = m[1].pen;
                     } else {
-                        uint32_t *sg = scr + SC::SCR_ROWS + (size_t)(2 * k + 1) * kRowWords;
+                        uint32_t *sg = scr + SC::SCR_STAGE + (size_t)k * kStageStride;
                         sg[S_AB] = ab; sg[S_NX] = __float_as_uint(nx); sg[S_NY] = __float_as_uint(ny);
                         sg[S_PX0] = __float_as_uint(m[0].px); sg[S_PY0] = __float_as_uint(m[0].py); sg[S_PEN0] = __float_as_uint(m[0].pen);
                         sg[S_PX1] = __float_as_uint(m[1].px); sg[S_PY1] = __float_as_uint(m[1].py); sg[S_PEN1] = __float_as_uint(m[1].pen);
@@ -772,71 +881,125 @@ struct Scene {
         g.sync();
         c_rec += (unsigned)nrec << 16;
 
-        // rows: lane k of a round takes staged pair k, runs the pre-step of its active manifolds and writes one row per
-        // manifold; the accumulated impulses of the same manifold slot in the previous step come from the warm list
-        int nrows = 0;
+        // Levels of the touching pairs (canonical order = staging order): one more than the highest level of an earlier pair
+        // that shares a movable body.  Then every pair gets its row slot: rows are sorted by level, in staging order within
+        // a level, and a byte table in the scratch says where each level starts.
+        uint8_t *lstart = reinterpret_cast<uint8_t *>(scr + SC::SCR_LSTART);
+        const bool crowded = nrec > G;      // more touching pairs than lanes: rare, handled by one lane through the scratch
+        int cmax = 0, lvl = 0, slot = 0;
+        uint32_t ab = 0u;
+        if (!crowded) {
+            const bool mine = lane < nrec;
+            if (mine) ab = __float_as_uint(sm[SC::STG + S_AB * G + lane]);
+            const int a = ab & 31, b = (ab >> 5) & 31;
+            // every movable body collects the set of pairs that touch it; a pair's conflicts are the earlier members of its
+            // bodies' sets; level r goes to the pairs whose conflicts all have a level already, round after round
+            uint32_t *touch = smu + SC::SURV;            // the survivor list is no longer needed
+            for (int i = lane; i < SC::N; i += G) touch[i] = 0u;
+            g.sync();
+            const bool da = (ab >> 26) & 1u, db = (ab >> 27) & 1u;
+            if (mine && da) atomicOr(touch + a, 1u << lane);
+            if (mine && db) atomicOr(touch + b, 1u << lane);
+            g.sync();
+            const unsigned conflicts = ((da ? touch[a] : 0u) | (db ? touch[b] : 0u)) & g.lanes_below();
+            const unsigned all = g.ballot(mine);
+            unsigned assigned = 0u;
+#pragma unroll 1
+            for (int r = 1; assigned != all; ++r) {
+                const bool ready = mine && lvl == 0 && (conflicts & ~assigned) == 0u;
+                if (ready) lvl = r;
+                assigned |= g.ballot(ready);
+            }
+            cmax = g.max_int(lvl);
+            int run = 0;
+#pragma unroll 1
+            for (int L = 1; L <= cmax; ++L) {
+                const unsigned bal = g.ballot(lvl == L);
+                if (lvl == L) slot = run + __popc(bal & g.lanes_below());
+                if (lane == 0) lstart[L] = (uint8_t)run;
+                run += __popc(bal);
+            }
+            if (lane == 0) lstart[cmax + 1] = (uint8_t)run;
+        } else {
+            // the pairs staged in shared memory join the others in the scratch
+            {
+                uint32_t *sg = scr + SC::SCR_STAGE + (size_t)lane * kStageStride;
+#pragma unroll
+                for (int f = 0; f < kStageWords; ++f) sg[f] = smu[SC::STG + f * G + lane];
+            }
+            g.sync();
+            if (lane == 0) cmax = place_crowded_impl<SC>(scr, lstart, reinterpret_cast<uint8_t *>(smu + SC::SURV), nrec);
+            g.sync();
+            cmax = g.shfl(cmax, 0);
+        }
+
+        // rows: lane k of a round takes staged pair k, runs the pre-step of its active manifolds and writes the pair's row
+        // into its slot; the accumulated impulses of the same pair in the previous step come from the lane that holds that
+        // entry of the warm list (or from the state record beyond the lanes)
+        int nman = 0;
         const ContactConsts cc = contact_consts();
 #pragma unroll 1
         for (int base = 0; base < nrec; base += G) {
             const int k = base + lane;
             const bool mine = k < nrec;
-            uint32_t ab = 0u;
             float nx = 0.0f, ny = 0.0f, pt[6] = { 0.0f, 0.0f, 0.0f, 0.0f, 0.0f, 0.0f };
             if (mine) {
-                if (base == 0) {
+                if (!crowded) {
                     const float *sg = sm + SC::STG + lane;
-                    ab = __float_as_uint(sg[S_AB * G]); nx = sg[S_NX * G]; ny = sg[S_NY * G];
+                    nx = sg[S_NX * G]; ny = sg[S_NY * G];
                     pt[0] = sg[S_PX0 * G]; pt[1] = sg[S_PY0 * G]; pt[2] = sg[S_PEN0 * G]; pt[3] = sg[S_PX1 * G]; pt[4] = sg[S_PY1 * G]; pt[5] = sg[S_PEN1 * G];
                 } else {
-                    const uint32_t *sg = scr + SC::SCR_ROWS + (size_t)(2 * k + 1) * kRowWords;
+                    const uint32_t *sg = scr + SC::SCR_STAGE + (size_t)k * kStageStride;
                     ab = __ldcg(sg + S_AB); nx = __uint_as_float(__ldcg(sg + S_NX)); ny = __uint_as_float(__ldcg(sg + S_NY));
                     pt[0] = __uint_as_float(__ldcg(sg + S_PX0)); pt[1] = __uint_as_float(__ldcg(sg + S_PY0)); pt[2] = __uint_as_float(__ldcg(sg + S_PEN0));
                     pt[3] = __uint_as_float(__ldcg(sg + S_PX1)); pt[4] = __uint_as_float(__ldcg(sg + S_PY1)); pt[5] = __uint_as_float(__ldcg(sg + S_PEN1));
+                    slot = (int)__ldcg(sg + kStageWords);
                 }
-            }
+            } else ab = 0u;
             const unsigned amask = (ab >> 10) & 3u;
-            const unsigned b0 = g.ballot((amask & 1u) != 0u), b1 = g.ballot((amask & 2u) != 0u);
-            int row = nrows + __popc(b0 & g.lanes_below()) + __popc(b1 & g.lanes_below());
-            nrows += __popc(b0) + __popc(b1);
-            g.sync();       // every lane of the round has its staged pair before rows are written over the staging slots
+            const int p = (ab >> 12) & 127;
+            // warm start values of this pair
+            const int wi = mine ? (int)widx()[p] : 255;
+            const int src = wi < G ? wi : 0;
+            float4 w4 = make_float4(g.shflf(wacc.x, src), g.shflf(wacc.y, src), g.shflf(wacc.z, src), g.shflf(wacc.w, src));
+            if (wi >= G && wi != 255) {
+                const uint32_t *wr = st + SC::ST_WARM + kWarmWords * wi;
+                w4 = make_float4(__uint_as_float(__ldcg(wr + 1)), __uint_as_float(__ldcg(wr + 2)), __uint_as_float(__ldcg(wr + 3)), __uint_as_float(__ldcg(wr + 4)));
+            }
+            if (wi == 255 || !prm.warm_start) w4 = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+            if (!(amask & 1u)) { w4.x = 0.0f; w4.y = 0.0f; }
+            if (!(amask & 2u)) { w4.z = 0.0f; w4.w = 0.0f; }
+            nman += __popc(amask);
             if (mine) {
-                const int a = ab & 31, b = (ab >> 5) & 31, p = (ab >> 12) & 127;
+                const int a = ab & 31, b = (ab >> 5) & 31;
                 const float ma = sm[SC::BIM + a], mb = sm[SC::BIM + b], ia = sm[SC::BII + a], ib = sm[SC::BII + b];
                 const float fra = sm[SC::BFR + a], frb = sm[SC::BFR + b];
                 const float mu = sqrtf(__fmaf_rn(fra, fra, frb * frb));
                 const float er = fmin_cmp(sm[SC::BRE + a], sm[SC::BRE + b]);
-                const uint32_t rab = (uint32_t)a | ((uint32_t)b << 5) | (((ab >> 26) & 3u) << 10);
+                float4 *r = reinterpret_cast<float4 *>(scr + SC::SCR_ROWS + (size_t)slot * kRowWords);
+                r[0] = make_float4(__uint_as_float(ab), nx, ny, mu);
+                r[1] = make_float4(ma, mb, ia, ib);
 #pragma unroll 1
                 for (int mi = 0; mi < 2; ++mi) {
-                    if (amask & (1u << mi)) {
-                        float rna, rnb, rta, rtb, massn, masst, target, corr;
-                        prestep_manifold<SC>(a, b, nx, ny, ma, mb, ia, ib, pt[3 * mi], pt[3 * mi + 1], pt[3 * mi + 2], er, sm, cc,
+                    float rna = 0.0f, rnb = 0.0f, rta = 0.0f, rtb = 0.0f, massn = 0.0f, masst = 0.0f, target = 0.0f, corr = 0.0f;
+                    if (amask & (1u << mi))
+                        prestep_manifold<SC>(a, b, nx, ny, ma, mb, ia, ib, mi ? pt[3] : pt[0], mi ? pt[4] : pt[1], mi ? pt[5] : pt[2], er, sm, cc,
                                              rna, rnb, rta, rtb, massn, masst, target, corr);
-                        const int key = 2 * p + mi;
-                        const int wi = widx()[key];
-                        float accn = 0.0f, acct = 0.0f;
-                        if (wi != 255 && prm.warm_start) {
-                            accn = __uint_as_float(__ldcg(st + SC::ST_WARM + kWarmWords * wi + 1));
-                            acct = __uint_as_float(__ldcg(st + SC::ST_WARM + kWarmWords * wi + 2));
-                        }
-                        float4 *r = reinterpret_cast<float4 *>(scr + SC::SCR_ROWS + (size_t)row * kRowWords);
-                        r[0] = make_float4(__uint_as_float(rab), nx, ny, mu);
-                        r[1] = make_float4(ma, mb, ia, ib);
-                        r[2] = make_float4(rna, rnb, rta, rtb);
-                        r[3] = make_float4(massn, masst, target, corr);
-                        r[4] = make_float4(accn, acct, __int_as_float(key), 0.0f);
-                        ++row;
-                    }
+                    r[2 + 2 * mi] = make_float4(rna, rnb, rta, rtb);
+                    r[3 + 2 * mi] = make_float4(massn, masst, target, corr);
                 }
+                r[6] = w4;
             }
         }
-        c_man += (unsigned)nrows | (1u << 16);
+        nman = g.sum_int(nman);
+        c_man += (unsigned)nman | (1u << 16);
         // velocities (gravity, motors, thrusters) and this step's messages to the solve kernel
         for (int i = lane; i < SC::N; i += G)
             reinterpret_cast<float4 *>(st + SC::ST_VEL)[i] = reinterpret_cast<const float4 *>(sm + SC::BVEL)[i];
         if (lane == 0) {
-            const uint32_t flags = (touch_gb ? 1u : 0u) | (touch_gr ? 2u : 0u) | (((gb >> 16) & 1u) << 2) | ((gb & 255u) << 8) | (((gb >> 8) & 255u) << 16);
-            *reinterpret_cast<uint4 *>(st + SC::ST_META + META_NROWS) = make_uint4((uint32_t)nrows, flags, __float_as_uint(d0), active_mask);
+            const uint32_t flags = (touch_gb ? 1u : 0u) | (touch_gr ? 2u : 0u) | (((gb >> 16) & 1u) << 2) | ((gb & 255u) << 8) | (((gb >> 8) & 255u) << 16) |
+                                   ((uint32_t)cmax << 24);
+            *reinterpret_cast<uint4 *>(st + SC::ST_META + META_NROWS) = make_uint4((uint32_t)nrec, flags, __float_as_uint(d0), active_mask | ((uint32_t)jmax << 16));
         }
     }
 };
@@ -854,17 +1017,28 @@ __global__ void __launch_bounds__(kBlockThreads, kMinBlocks) k2d_prep_kernel(con
     uint32_t *region = smem_raw + SC::PTAB_WORDS + gib * region_words<SC, G>();
     Scene<SC, G> scene(region, ptab, prm);
     // Envs are handed out one at a time by a ticket counter: a group that is done takes the next one, so groups with
-    // cheap scenes take more of them.
+    // cheap scenes take more of them.  A group draws the ticket of its next env when it starts on an env and reads that
+    // env's meta words half way through, so neither the counter nor the memory is waited for between envs.
     const Group<G> &g = scene.g;
+    unsigned t = 0u;
+    if (g.lane == 0) t = atomicAdd(prm.queue + Q_TICKET, 1u);
+    t = g.shflu(t, 0);
+    MetaHead head = { 0u, 0u, 0u };
+    if (t < (unsigned)prm.n_envs) head = load_meta_head(prm.state + (size_t)t * SC::ST_WORDS + SC::ST_META);
     int taken = 0;
 #pragma unroll 1
-    for (;;) {
-        unsigned t = 0u;
-        if (g.lane == 0) t = atomicAdd(prm.queue + Q_TICKET, 1u);
-        t = g.shflu(t, 0);
-        if (t >= (unsigned)prm.n_envs) break;
-        scene.prepare((int)t);
+    while (t < (unsigned)prm.n_envs) {
+        unsigned tn_raw = 0u, next_e = 0u;
+        if (g.lane == 0) tn_raw = atomicAdd(prm.queue + Q_TICKET, 1u);
+        MetaHead next_head = { 0u, 0u, 0u };
+        if (head.status & 1u) {      // frozen env: nothing to prepare (the solve kernel reports done)
+            next_e = g.shflu(tn_raw, 0);
+            if (next_e < (unsigned)prm.n_envs) next_head = load_meta_head(prm.state + (size_t)next_e * SC::ST_WORDS + SC::ST_META);
+        } else {
+            scene.prepare((int)t, head, tn_raw, next_e, next_head);
+        }
         g.sync();
+        t = next_e; head = next_head;
         if ((++taken & 63) == 0) scene.flush();
     }
     scene.flush();
@@ -878,37 +1052,25 @@ __global__ void __launch_bounds__(kBlockThreads, kMinBlocks) k2d_prep_kernel(con
     }
 }
 
-// ================================================================ second half of a step: one thread per env
-// The constants of a joint row and of a manifold row as the solver reads them (read-only loads: the rows were written by
-// the prep kernel of the same step and nothing writes them while the solve kernel runs; the accumulated impulses, which the
-// solver does write, are copied to shared memory first).
-struct JointConsts { float4 r, k, b, m; };       // lever arms; inverse effective mass and packed joint word; bias and correction; inverse masses
-struct RowConsts { float4 h0, h1, c0, c1; };      // pair word, normal, friction; inverse masses; lever-arm cross products; effective masses, target, correction
-__device__ __forceinline__ JointConsts load_joint(const float *jr) {
-    const float4 *q = reinterpret_cast<const float4 *>(jr);
-    JointConsts c; c.r = __ldg(q); c.k = __ldg(q + 1); c.b = __ldg(q + 2); c.m = __ldg(q + 3);
-    return c;
-}
-__device__ __forceinline__ RowConsts load_row(const float *r) {
-    const float4 *q = reinterpret_cast<const float4 *>(r);
-    RowConsts c; c.h0 = __ldg(q); c.h1 = __ldg(q + 1); c.c0 = __ldg(q + 2); c.c1 = __ldg(q + 3);
-    return c;
-}
+// ================================================================ second half of a step: a group of kSolveLanes lanes per env
+// The rows of a scene are copied to shared memory when its group starts (the first kRowCap pair rows and all joint rows;
+// later pair rows, which few scenes have, are used where they are, in the scratch), so the sweeps below read and update
+// them at shared-memory latency.  A row pointer is therefore a generic pointer.
 
 // ---- angular row of a fixed joint or of a revolute joint beyond one of its limits (paper, "Fixed Joints",
 // "Joint Limits"): j_r = (w_a - w_b + correction) / (1/I_a + 1/I_b), a loses j_r / I_a, b gains j_r / I_b.  A fixed
 // joint's impulse is accumulated and warm-started; a limit only ever pushes back, applies no correction while the
-// joint is already returning, and is not accumulated.  ang4: kind this step, inverse angular mass, correction, -;
-// accr: the accumulated impulse.  Out of line: most joints are plain revolute joints.
+// joint is already returning, and is not accumulated.  The row's last group: kind this step, inverse angular mass,
+// correction, accumulated impulse.  Out of line: most joints are plain revolute joints.
 template <int MODE>
-__device__ __noinline__ float2 angular_row(const float *jr, float *accr, float ia, float ib, float wa, float wb) {
-    const float4 ang4 = __ldg(reinterpret_cast<const float4 *>(jr + JR_ANG));
+__device__ __noinline__ float2 angular_row(float *jr, float ia, float ib, float wa, float wb) {
+    const float4 ang4 = ld4(jr + JR_ANG);
     const int ang = __float_as_int(ang4.x);
     if (ang == 0) return make_float2(wa, wb);
     float lr;
     if (MODE == 0) {
         if (ang != 1) return make_float2(wa, wb);
-        lr = *accr;
+        lr = ang4.w;
     } else {
         const float wrel = wa - wb;
         float v;
@@ -916,203 +1078,285 @@ __device__ __noinline__ float2 angular_row(const float *jr, float *accr, float i
         else if (ang == 2) { v = (wrel < 0.0f) ? wrel : wrel + ang4.z; v = fmax_cmp(v, 0.0f); }
         else { v = (wrel > 0.0f) ? wrel : wrel + ang4.z; v = fmin_cmp(v, 0.0f); }
         lr = v * ang4.y;
-        if (ang == 1) *accr = *accr + lr;
+        if (ang == 1) jr[JR_ACCR] = ang4.w + lr;
     }
     return make_float2(__fmaf_rn(-lr, ia, wa), __fmaf_rn(lr, ib, wb));
 }
 
-// one visit of a joint row.  MODE 0: apply the accumulated impulses (warm start); 1: one solver iteration.
-// sv: the calling thread's column of the block's velocity array (stride kSolveThreads groups per body);
-// acc: the joint's accumulated impulses (x, y, angular, -) in shared memory.
+// one visit of a joint row.  MODE 0: apply the accumulated impulses (warm start); 1: one solver iteration; 2: positional
+// correction.  sv: the scene's bodies in shared memory (velocities; positions in mode 2).
 template <int MODE>
-__device__ __forceinline__ void solve_joint(const JointConsts &c, const float *jr, float4 *acc, float4 *sv) {
-    const uint32_t jab = __float_as_uint(c.k.w);
-    if (!((jab >> 24) & 1u)) return;
+__device__ __forceinline__ void solve_joint(float *jr, float4 *sv) {
+    const float4 k4 = ld4(jr + JR_I11), mi4 = ld4(jr + JR_MA);
+    const uint32_t jab = __float_as_uint(k4.w);
     const int a = jab & 255, b = (jab >> 8) & 255;
-    const float ma = c.m.x, mb = c.m.y, ia = c.m.z, ib = c.m.w;
-    const float rax = c.r.x, ray = c.r.y, rbx = c.r.z, rby = c.r.w;
-    const float4 va4 = sv[a * kSolveThreads], vb4 = sv[b * kSolveThreads];
+    const float ma = mi4.x, mb = mi4.y, ia = mi4.z, ib = mi4.w;
+    if (MODE == 2) {
+        const float cx = jr[JR_CX], cy = jr[JR_CY];
+        if ((jab >> 29) & 1u) { float4 p = sv[a]; p.x = __fmaf_rn(ma, cx, p.x); p.y = __fmaf_rn(ma, cy, p.y); sv[a] = p; }
+        if ((jab >> 30) & 1u) { float4 p = sv[b]; p.x = __fmaf_rn(-mb, cx, p.x); p.y = __fmaf_rn(-mb, cy, p.y); sv[b] = p; }
+        return;
+    }
+    const float4 r4 = ld4(jr + JR_RAX);
+    const float rax = r4.x, ray = r4.y, rbx = r4.z, rby = r4.w;
+    const float4 va4 = sv[a], vb4 = sv[b];
     float vax = va4.x, vay = va4.y, wa = va4.z, vbx = vb4.x, vby = vb4.y, wb = vb4.z;
-    float4 ac = *acc;
+    const float2 acc = *reinterpret_cast<const float2 *>(jr + JR_ACCX);
     float lx, ly;
-    if (MODE == 0) { lx = ac.x; ly = ac.y; }
+    if (MODE == 0) { lx = acc.x; ly = acc.y; }
     else {
+        const float2 b2 = *reinterpret_cast<const float2 *>(jr + JR_BX);
         const float cx = __fmaf_rn(-wb, rby, vbx) - __fmaf_rn(-wa, ray, vax);
         const float cy = __fmaf_rn(wb, rbx, vby) - __fmaf_rn(wa, rax, vay);
-        const float rx = -(cx + c.b.x), ry = -(cy + c.b.y);
-        const float i11 = c.k.x, i12 = c.k.y, i22 = c.k.z;
+        const float rx = -(cx + b2.x), ry = -(cy + b2.y);
+        const float i11 = k4.x, i12 = k4.y, i22 = k4.z;
         lx = __fmaf_rn(i11, rx, i12 * ry);
         ly = __fmaf_rn(i12, rx, i22 * ry);
-        ac.x = ac.x + lx; ac.y = ac.y + ly;
+        *reinterpret_cast<float2 *>(jr + JR_ACCX) = make_float2(acc.x + lx, acc.y + ly);
     }
     wa = __fmaf_rn(-ia, cross2(rax, ray, lx, ly), wa);
     wb = __fmaf_rn(ib, cross2(rbx, rby, lx, ly), wb);
     if (jab >> 31) {      // fixed or limited joint: its angular row follows the point row
-        const float2 w2 = angular_row<MODE>(jr, &ac.z, ia, ib, wa, wb);
+        const float2 w2 = angular_row<MODE>(jr, ia, ib, wa, wb);
         wa = w2.x; wb = w2.y;
     }
-    if (MODE == 1) *acc = ac;
-    if ((jab >> 29) & 1u) sv[a * kSolveThreads] = make_float4(__fmaf_rn(-ma, lx, vax), __fmaf_rn(-ma, ly, vay), wa, 0.0f);
-    if ((jab >> 30) & 1u) sv[b * kSolveThreads] = make_float4(__fmaf_rn(mb, lx, vbx), __fmaf_rn(mb, ly, vby), wb, 0.0f);
+    if ((jab >> 29) & 1u) sv[a] = make_float4(__fmaf_rn(-ma, lx, vax), __fmaf_rn(-ma, ly, vay), wa, 0.0f);
+    if ((jab >> 30) & 1u) sv[b] = make_float4(__fmaf_rn(mb, lx, vbx), __fmaf_rn(mb, ly, vby), wb, 0.0f);
 }
 
-// one visit of a manifold row (normal then friction), same modes; acc: its accumulated normal and tangent impulse
+// one visit of a pair row (per active manifold the normal row, then the friction row), same modes
 template <int MODE>
-__device__ __forceinline__ void solve_row(const RowConsts &c, float2 *accp, float4 *sv) {
-    float2 acc = *accp;
-    const uint32_t ab = __float_as_uint(c.h0.x);
+__device__ __forceinline__ void solve_pair(float *r, float4 *sv) {
+    const float4 h0 = ld4(r + R_AB), h1 = ld4(r + R_MA);
+    const uint32_t ab = __float_as_uint(h0.x);
     const int a = ab & 31, b = (ab >> 5) & 31;
-    const float4 va4 = sv[a * kSolveThreads], vb4 = sv[b * kSolveThreads];
+    const unsigned amask = (ab >> 10) & 3u;
+    const bool dyn_a = (ab >> 26) & 1u, dyn_b = (ab >> 27) & 1u;
+    if (MODE == 2) {
+        const float corr0 = r[R_M0 + M_CORR], corr1 = r[R_M1 + M_CORR];
+        float4 pa = sv[a], pb = sv[b];
+        if (amask & 1u) {
+            const float ca = h1.x * corr0, cb = h1.y * corr0;
+            pa.x = __fmaf_rn(-ca, h0.y, pa.x); pa.y = __fmaf_rn(-ca, h0.z, pa.y);
+            pb.x = __fmaf_rn(cb, h0.y, pb.x); pb.y = __fmaf_rn(cb, h0.z, pb.y);
+        }
+        if (amask & 2u) {
+            const float ca = h1.x * corr1, cb = h1.y * corr1;
+            pa.x = __fmaf_rn(-ca, h0.y, pa.x); pa.y = __fmaf_rn(-ca, h0.z, pa.y);
+            pb.x = __fmaf_rn(cb, h0.y, pb.x); pb.y = __fmaf_rn(cb, h0.z, pb.y);
+        }
+        if (dyn_a) sv[a] = pa;
+        if (dyn_b) sv[b] = pb;
+        return;
+    }
+    const float4 va4 = sv[a], vb4 = sv[b];
     float vax = va4.x, vay = va4.y, wa = va4.z, vbx = vb4.x, vby = vb4.y, wb = vb4.z;
-    manifold_rows<MODE>(c.h0.y, c.h0.z, c.h0.w, c.h1.x, c.h1.y, c.h1.z, c.h1.w, c.c0.x, c.c0.y, c.c0.z, c.c0.w, c.c1.x, c.c1.y, c.c1.z,
-                        acc.x, acc.y, vax, vay, wa, vbx, vby, wb);
-    if (MODE == 1) *accp = acc;
-    if ((ab >> 10) & 1u) sv[a * kSolveThreads] = make_float4(vax, vay, wa, 0.0f);
-    if ((ab >> 11) & 1u) sv[b * kSolveThreads] = make_float4(vbx, vby, wb, 0.0f);
+    float4 acc = ld4(r + R_ACC);
+    if (amask & 1u) {
+        const float4 c0 = ld4(r + R_M0), c1 = ld4(r + R_M0 + 4);
+        manifold_rows<MODE>(h0.y, h0.z, h0.w, h1.x, h1.y, h1.z, h1.w, c0.x, c0.y, c0.z, c0.w, c1.x, c1.y, c1.z, acc.x, acc.y,
+                            vax, vay, wa, vbx, vby, wb);
+    }
+    if (amask & 2u) {
+        const float4 c0 = ld4(r + R_M1), c1 = ld4(r + R_M1 + 4);
+        manifold_rows<MODE>(h0.y, h0.z, h0.w, h1.x, h1.y, h1.z, h1.w, c0.x, c0.y, c0.z, c0.w, c1.x, c1.y, c1.z, acc.z, acc.w,
+                            vax, vay, wa, vbx, vby, wb);
+    }
+    if (MODE == 1) *reinterpret_cast<float4 *>(r + R_ACC) = acc;
+    if (dyn_a) sv[a] = make_float4(vax, vay, wa, 0.0f);
+    if (dyn_b) sv[b] = make_float4(vbx, vby, wb, 0.0f);
 }
 
-constexpr int kAccCap = 32;   // manifold rows of an env whose accumulated impulses sit in shared memory during the solve; later rows use their scratch row
+constexpr int kRowCap = 12;   // pair rows of an env that are copied to shared memory for the solve; later rows are used in the scratch
+constexpr int kLevCap = 32;   // level starts of an env kept in shared memory; a scene with more levels reads the table in its scratch
+
+// n groups of 16 bytes from memory to shared memory by the GS lanes of a group, B per lane in flight at a time
+template <int B, int GS>
+__device__ __forceinline__ void stage_groups(float4 *dst, const float4 *src, int n, int lane) {
+#pragma unroll 1
+    for (int base = 0; base < n; base += B * GS) {
+        float4 v[B];
+#pragma unroll
+        for (int k = 0; k < B; ++k) { const int i = base + lane + k * GS; v[k] = (i < n) ? __ldcg(src + i) : make_float4(0.0f, 0.0f, 0.0f, 0.0f); }
+#pragma unroll
+        for (int k = 0; k < B; ++k) { const int i = base + lane + k * GS; if (i < n) dst[i] = v[k]; }
+    }
+}
 
 template <class SC>
 __global__ void __launch_bounds__(kSolveThreads) k2d_solve_kernel(const StepParams prm) {
-    // velocities (later positions) of the block's envs: one 16-byte group per (body, thread); a thread's groups are
-    // kSolveThreads groups apart, so the threads of a warp never meet in a bank, whichever bodies they address
-    __shared__ float4 s_body[SC::N * kSolveThreads];
-    __shared__ float4 s_jacc[(SC::J > 0 ? SC::J : 1) * kSolveThreads];
-    __shared__ float2 s_racc[kAccCap * kSolveThreads];
-    const int e = blockIdx.x * kSolveThreads + threadIdx.x;
-    if (e >= prm.n_envs) return;
-    float4 *sv = s_body + threadIdx.x;
-    float4 *sj = s_jacc + threadIdx.x;
-    float2 *sa = s_racc + threadIdx.x;
-    uint32_t *st = prm.state + (size_t)e * SC::ST_WORDS;
+    constexpr int GS = kSolveLanes, SPB = kSolveThreads / GS;     // lanes per scene, scenes per block
+    constexpr int JPL = (SC::J + GS - 1) / GS;                    // joints a lane may own: lane, lane + GS, ...
+    // per scene: the bodies' velocities (later positions), the joint rows, the first kRowCap pair rows, the first row of every level
+    constexpr int S_BODY = 0, S_JROW = 4 * SC::N, S_ROWS = S_JROW + kJointWords * SC::J, S_LSTART = S_ROWS + kRowWords * kRowCap;
+    constexpr int S_WORDS = S_LSTART + kLevCap / 4;
+    __shared__ __align__(16) float s_scene[SPB * S_WORDS];
+    const Group<GS> g;
+    const int lane = g.lane, sb = threadIdx.x / GS;
+    const int e = blockIdx.x * SPB + sb;
+    const bool in_range = e < prm.n_envs;
+    uint32_t *st = prm.state + (size_t)(in_range ? e : 0) * SC::ST_WORDS;
     float *stf = reinterpret_cast<float *>(st);
-    float *rows = reinterpret_cast<float *>(prm.scratch + (size_t)e * SC::SCRATCH_WORDS + SC::SCR_ROWS);
-    float *jrows = reinterpret_cast<float *>(prm.scratch + (size_t)e * SC::SCRATCH_WORDS + SC::SCR_JROW);
-    const uint4 m0 = *reinterpret_cast<const uint4 *>(st + SC::ST_META), m1 = *reinterpret_cast<const uint4 *>(st + SC::ST_META + 4);
+    uint4 m0 = make_uint4(0u, 0u, 0u, 0u), m1 = m0;
+    if (in_range) { m0 = *reinterpret_cast<const uint4 *>(st + SC::ST_META); m1 = *reinterpret_cast<const uint4 *>(st + SC::ST_META + 4); }
     // frozen env: reports done, nothing else
-    if (m0.w & 1u) { prm.reward[e] = 0.0f; prm.done[e] = 1; return; }
+    const bool frozen = in_range && (m0.w & 1u);
+    if (frozen && lane == 0) { prm.reward[e] = 0.0f; prm.done[e] = 1; }
+    const bool live = in_range && !frozen;
+    const unsigned wmask = __ballot_sync(0xffffffffu, live);      // the warp's lanes that go on: its groups stay in step level by level
+    if (!live) return;
+    float *ss = s_scene + sb * S_WORDS;
+    float4 *sv = reinterpret_cast<float4 *>(ss + S_BODY);
+    float *sj = ss + S_JROW, *sr = ss + S_ROWS;
+    uint8_t *sl = reinterpret_cast<uint8_t *>(ss + S_LSTART);
+    uint32_t *scr = prm.scratch + (size_t)e * SC::SCRATCH_WORDS;
+    float *rows = reinterpret_cast<float *>(scr + SC::SCR_ROWS);
+    const uint8_t *lstart = reinterpret_cast<const uint8_t *>(scr + SC::SCR_LSTART);
     const int nrows = (int)m1.x;
-    const uint32_t flags = m1.y, active = m1.w;
-#pragma unroll
-    for (int i = 0; i < SC::N; ++i) sv[i * kSolveThreads] = ld4(stf + SC::ST_VEL + 4 * i);
-#pragma unroll
-    for (int j = 0; j < SC::J; ++j) {
-        const float2 a2 = *reinterpret_cast<const float2 *>(jrows + j * kJointWords + JR_ACCX);
-        sj[j * kSolveThreads] = make_float4(a2.x, a2.y, jrows[j * kJointWords + JR_ACCR], 0.0f);
-    }
-    const int ncap = nrows < kAccCap ? nrows : kAccCap;
-#pragma unroll 1
-    for (int k = 0; k < ncap; ++k) sa[k * kSolveThreads] = *reinterpret_cast<const float2 *>(rows + k * kRowWords + R_ACCN);
-#define K2D_ACC_OF(k) ((k) < kAccCap ? sa + (k) * kSolveThreads : reinterpret_cast<float2 *>(rows + (k) * kRowWords + R_ACCN))
-    // warm start: contacts, then joints (Algorithm 1)
+    const uint32_t flags = m1.y, active = m1.w & 0xffffu;
+    const int cmax = (int)(flags >> 24), jmax = (int)((m1.w >> 16) & 15u);
+    const int cmax_w = __reduce_max_sync(wmask, cmax), jmax_w = __reduce_max_sync(wmask, jmax);
+    // velocities, joint rows, level starts, pair rows -> shared memory
     {
-        RowConsts cur = load_row(rows);
-#pragma unroll 1
-        for (int k = 0; k < nrows; ++k) {
-            const RowConsts nxt = load_row(rows + (k + 1 < nrows ? k + 1 : k) * kRowWords);
-            solve_row<0>(cur, K2D_ACC_OF(k), sv);
-            cur = nxt;
+        constexpr int NB = SC::N + 6 * SC::J;       // the velocities and the joint rows are contiguous neither in memory nor here: two sources, one volley
+        constexpr int KB = (NB + GS - 1) / GS;
+        float4 v[KB];
+        uint32_t lw = 0u;
+        const float4 *src_v = reinterpret_cast<const float4 *>(stf + SC::ST_VEL), *src_j = reinterpret_cast<const float4 *>(scr + SC::SCR_JROW);
+#pragma unroll
+        for (int k = 0; k < KB; ++k) {
+            const int i = lane + k * GS;
+            v[k] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+            if (i < SC::N) v[k] = __ldcg(src_v + i); else if (i < NB) v[k] = __ldcg(src_j + (i - SC::N));
+        }
+        static_assert(kLevCap / 4 <= 2 * GS, "level starts: at most two words per lane");
+        uint32_t lw2 = 0u;
+        if (lane < kLevCap / 4) lw = __ldcg(scr + SC::SCR_LSTART + lane);
+        if (lane + GS < kLevCap / 4) lw2 = __ldcg(scr + SC::SCR_LSTART + lane + GS);
+#pragma unroll
+        for (int k = 0; k < KB; ++k) {
+            const int i = lane + k * GS;
+            if (i < SC::N) sv[i] = v[k]; else if (i < NB) reinterpret_cast<float4 *>(sj)[i - SC::N] = v[k];
+        }
+        if (lane < kLevCap / 4) reinterpret_cast<uint32_t *>(sl)[lane] = lw;
+        if (lane + GS < kLevCap / 4) reinterpret_cast<uint32_t *>(sl)[lane + GS] = lw2;
+    }
+    stage_groups<6, GS>(reinterpret_cast<float4 *>(sr), reinterpret_cast<const float4 *>(rows), 7 * (nrows < kRowCap ? nrows : kRowCap), lane);
+    g.sync();
+    // this lane's joints and their levels (0: the joint takes no part)
+    int jlev[JPL > 0 ? JPL : 1];
+#pragma unroll
+    for (int q = 0; q < JPL; ++q) {
+        const int j = lane + q * GS;
+        jlev[q] = 0;
+        if (j < SC::J) {
+            const uint32_t jab = __float_as_uint(sj[j * kJointWords + JR_JAB]);
+            if ((jab >> 24) & 1u) jlev[q] = (int)((jab >> 25) & 7u);
         }
     }
-#pragma unroll 1
-    for (int j = 0; j < SC::J; ++j) solve_joint<0>(load_joint(jrows + j * kJointWords), jrows + j * kJointWords, sj + j * kSolveThreads, sv);
-    // solver iterations: joints by index, then manifolds in pair order; the next row's constants are fetched while a row is solved
+#define K2D_ROW(r) ((r) < kRowCap ? sr + (r) * kRowWords : rows + (r) * kRowWords)
+#define K2D_LSTART(L) ((L) < kLevCap ? (int)sl[L] : (int)lstart[L])
+    // One sweep over the pair rows / the joint rows, level by level; the rows of a level go to the lanes round robin.  All
+    // groups of the warp walk the same number of levels and meet after each, so that they execute the rows together.
+#define K2D_SWEEP_PAIRS(MODE)                                                                         \
+    _Pragma("unroll 1") for (int L = 1; L <= cmax_w; ++L) {                                           \
+        int r = 0, r1 = 0;                                                                            \
+        if (L <= cmax) { r = K2D_LSTART(L); r1 = K2D_LSTART(L + 1); }                                 \
+        const int rounds = (__reduce_max_sync(wmask, r1 - r) + GS - 1) / GS;                          \
+        r += lane;                                                                                    \
+        _Pragma("unroll 1") for (int q = 0; q < rounds; ++q, r += GS)                                 \
+            if (r < r1) solve_pair<MODE>(K2D_ROW(r), sv);                                             \
+        __syncwarp(wmask);                                                                            \
+    }
+#define K2D_SWEEP_JOINTS(MODE)                                                                        \
+    if (SC::J > 0) {                                                                                  \
+        _Pragma("unroll 1") for (int L = 1; L <= jmax_w; ++L) {                                       \
+            _Pragma("unroll") for (int q = 0; q < JPL; ++q)                                           \
+                if (jlev[q] == L) solve_joint<MODE>(sj + (lane + q * GS) * kJointWords, sv);          \
+            __syncwarp(wmask);                                                                        \
+        }                                                                                             \
+    }
+    // warm start: contacts, then joints (Algorithm 1); solver iterations: joints, then contacts
+    K2D_SWEEP_PAIRS(0)
+    K2D_SWEEP_JOINTS(0)
 #pragma unroll 1
     for (int it = 0; it < prm.solver_iters; ++it) {
-        if (SC::J > 0) {
-            JointConsts cur = load_joint(jrows);
-#pragma unroll 1
-            for (int j = 0; j < SC::J; ++j) {
-                const JointConsts nxt = load_joint(jrows + (j + 1 < SC::J ? j + 1 : j) * kJointWords);
-                solve_joint<1>(cur, jrows + j * kJointWords, sj + j * kSolveThreads, sv);
-                cur = nxt;
-            }
-        }
-        RowConsts cur = load_row(rows);
-#pragma unroll 1
-        for (int k = 0; k < nrows; ++k) {
-            const RowConsts nxt = load_row(rows + (k + 1 < nrows ? k + 1 : k) * kRowWords);
-            solve_row<1>(cur, K2D_ACC_OF(k), sv);
-            cur = nxt;
-        }
+        K2D_SWEEP_JOINTS(1)
+        K2D_SWEEP_PAIRS(1)
     }
     // Euler step with the solved velocities; the velocities go back to the state record and the array holds positions from here on
     bool finite = true;
+    {
+        constexpr int KN = (SC::N + GS - 1) / GS;
+        float4 p[KN];
 #pragma unroll
-    for (int i = 0; i < SC::N; ++i) {
-        const float4 v4 = sv[i * kSolveThreads];
-        float4 p4 = ld4(stf + SC::ST_POS + 4 * i);
-        if ((active >> i) & 1u) { p4.x = __fmaf_rn(prm.dt, v4.x, p4.x); p4.y = __fmaf_rn(prm.dt, v4.y, p4.y); p4.z = __fmaf_rn(prm.dt, v4.z, p4.z); }
-        finite = finite && finite_bits(v4.x) && finite_bits(v4.y) && finite_bits(v4.z);
-        st4(stf + SC::ST_VEL + 4 * i, v4.x, v4.y, v4.z);
-        sv[i * kSolveThreads] = p4;
+        for (int k = 0; k < KN; ++k) { const int i = lane + k * GS; p[k] = (i < SC::N) ? ld4(stf + SC::ST_POS + 4 * i) : make_float4(0.0f, 0.0f, 0.0f, 0.0f); }
+#pragma unroll
+        for (int k = 0; k < KN; ++k) {
+            const int i = lane + k * GS;
+            if (i < SC::N) {
+                const float4 v4 = sv[i];
+                float4 p4 = p[k];
+                if ((active >> i) & 1u) { p4.x = __fmaf_rn(prm.dt, v4.x, p4.x); p4.y = __fmaf_rn(prm.dt, v4.y, p4.y); p4.z = __fmaf_rn(prm.dt, v4.z, p4.z); }
+                finite = finite && finite_bits(v4.x) && finite_bits(v4.y) && finite_bits(v4.z);
+                st4(stf + SC::ST_VEL + 4 * i, v4.x, v4.y, v4.z);
+                sv[i] = p4;
+            }
+        }
     }
+    __syncwarp(wmask);
     // positional corrections: every active manifold moves its two bodies apart along the normal, then the joints close their gaps
-#pragma unroll 1
-    for (int k = 0; k < nrows; ++k) {
-        const float *r = rows + k * kRowWords;
-        const float4 h0 = __ldg(reinterpret_cast<const float4 *>(r + R_AB));
-        const float2 mm = __ldg(reinterpret_cast<const float2 *>(r + R_MA));
-        const float corr = __ldg(r + R_CORR);
-        const uint32_t ab = __float_as_uint(h0.x);
-        const int a = ab & 31, b = (ab >> 5) & 31;
-        const float ca = mm.x * corr, cb = mm.y * corr;
-        if ((ab >> 10) & 1u) { float4 p = sv[a * kSolveThreads]; p.x = __fmaf_rn(-ca, h0.y, p.x); p.y = __fmaf_rn(-ca, h0.z, p.y); sv[a * kSolveThreads] = p; }
-        if ((ab >> 11) & 1u) { float4 p = sv[b * kSolveThreads]; p.x = __fmaf_rn(cb, h0.y, p.x); p.y = __fmaf_rn(cb, h0.z, p.y); sv[b * kSolveThreads] = p; }
-    }
-#pragma unroll 1
-    for (int j = 0; j < SC::J; ++j) {
-        const JointConsts c = load_joint(jrows + j * kJointWords);
-        const uint32_t jab = __float_as_uint(c.k.w);
-        if (!((jab >> 24) & 1u)) continue;
-        const int a = jab & 255, b = (jab >> 8) & 255;
-        const float cx = c.b.z, cy = c.b.w, ma = c.m.x, mb = c.m.y;
-        if ((jab >> 29) & 1u) { float4 p = sv[a * kSolveThreads]; p.x = __fmaf_rn(ma, cx, p.x); p.y = __fmaf_rn(ma, cy, p.y); sv[a * kSolveThreads] = p; }
-        if ((jab >> 30) & 1u) { float4 p = sv[b * kSolveThreads]; p.x = __fmaf_rn(-mb, cx, p.x); p.y = __fmaf_rn(-mb, cy, p.y); sv[b * kSolveThreads] = p; }
-    }
-#pragma unroll
-    for (int i = 0; i < SC::N; ++i) {
-        const float4 p4 = sv[i * kSolveThreads];
+    K2D_SWEEP_PAIRS(2)
+    K2D_SWEEP_JOINTS(2)
+    for (int i = lane; i < SC::N; i += GS) {
+        const float4 p4 = sv[i];
         finite = finite && finite_bits(p4.x) && finite_bits(p4.y) && finite_bits(p4.z);
         st4(stf + SC::ST_POS + 4 * i, p4.x, p4.y, p4.z);
     }
+    finite = !g.any(!finite);
     // reward and termination (paper, "Reward"): green touches blue = +1, green touches red = -1, either ends the episode
     const int step_count = (int)m0.x + 1;
     const bool touch_gb = (flags & 1u) != 0u, touch_gr = (flags & 2u) != 0u;
     const bool timeout = prm.max_episode_steps > 0 && step_count >= prm.max_episode_steps;
     float reward = (float)((int)touch_gb - (int)touch_gr);
     if (prm.dense_kappa != 0.0f && ((flags >> 2) & 1u)) {
-        const float4 pg = sv[((flags >> 8) & 255u) * kSolveThreads], pb = sv[((flags >> 16) & 255u) * kSolveThreads];
+        const float4 pg = sv[(flags >> 8) & 255u], pb = sv[(flags >> 16) & 255u];
         const float dx = pb.x - pg.x, dy = pb.y - pg.y;
         reward = reward + prm.dense_kappa * (__uint_as_float(m1.z) - sqrtf(dot2(dx, dy, dx, dy)));
     }
     bool done = touch_gb || touch_gr || timeout;
     uint32_t status = m0.w;
-    if (!finite) { reward = 0.0f; done = true; status |= 1u; atomicAdd(prm.counters + 0, 1ULL); }
-    prm.reward[e] = reward;
-    prm.done[e] = done ? 1 : 0;
+    if (!finite) { reward = 0.0f; done = true; status |= 1u; }
+    if (lane == 0) {
+        prm.reward[e] = reward;
+        prm.done[e] = done ? 1 : 0;
+        if (!finite) atomicAdd(prm.counters + 0, 1ULL);
+    }
     if (!(done && prm.auto_reset != 0)) {
         // the accumulated impulses of this step's rows warm-start the next step
-#pragma unroll 1
-        for (int k = 0; k < nrows; ++k) {
-            const float2 acc = *K2D_ACC_OF(k);
-            st[SC::ST_WARM + kWarmWords * k] = __float_as_uint(__ldg(rows + k * kRowWords + R_KEY));
-            st[SC::ST_WARM + kWarmWords * k + 1] = __float_as_uint(acc.x);
-            st[SC::ST_WARM + kWarmWords * k + 2] = __float_as_uint(acc.y);
+        for (int r = lane; r < nrows; r += GS) {
+            const float *row = K2D_ROW(r);
+            const float4 acc = ld4(row + R_ACC);
+            uint32_t *wr = st + SC::ST_WARM + kWarmWords * r;
+            wr[0] = (__float_as_uint(row[R_AB]) >> 12) & 127u;
+            wr[1] = __float_as_uint(acc.x); wr[2] = __float_as_uint(acc.y); wr[3] = __float_as_uint(acc.z); wr[4] = __float_as_uint(acc.w);
         }
-#pragma unroll
-        for (int j = 0; j < SC::J; ++j) {
-            const float4 a4 = sj[j * kSolveThreads];
-            st[SC::ST_JACC + 3 * j] = __float_as_uint(a4.x);
-            st[SC::ST_JACC + 3 * j + 1] = __float_as_uint(a4.y);
-            st[SC::ST_JACC + 3 * j + 2] = __float_as_uint(a4.z);
+        for (int j = lane; j < SC::J; j += GS) {
+            const float *jr = sj + j * kJointWords;
+            st[SC::ST_JACC + 3 * j] = __float_as_uint(jr[JR_ACCX]);
+            st[SC::ST_JACC + 3 * j + 1] = __float_as_uint(jr[JR_ACCY]);
+            st[SC::ST_JACC + 3 * j + 2] = __float_as_uint(jr[JR_ACCR]);
         }
-        st[SC::ST_META + META_STEP] = (uint32_t)step_count;
-        st[SC::ST_META + META_STATUS] = status;
+        if (lane == 0) {
+            st[SC::ST_META + META_STEP] = (uint32_t)step_count;
+            st[SC::ST_META + META_STATUS] = status;
+        }
         return;
     }
-#undef K2D_ACC_OF
+#undef K2D_SWEEP_JOINTS
+#undef K2D_SWEEP_PAIRS
+#undef K2D_LSTART
+#undef K2D_ROW
     // auto-reset of a finished env: next level (its own, or drawn from the pool by the hash of seed, global env index
     // and episode), pose from the level, no accumulated impulses
     const int episode = (int)m0.y + 1;
@@ -1123,15 +1367,16 @@ __global__ void __launch_bounds__(kSolveThreads) k2d_solve_kernel(const StepPara
         level = (int)(h % (unsigned long long)prm.n_levels);
     }
     const float *lv = reinterpret_cast<const float *>(prm.levels + (size_t)level * SC::LV_WORDS);
-#pragma unroll 1
-    for (int i = 0; i < SC::N; ++i) {
+    for (int i = lane; i < SC::N; i += GS) {
         st4(stf + SC::ST_POS + 4 * i, lv[SC::LV_X + i], lv[SC::LV_Y + i], lv[SC::LV_TH + i]);
         st4(stf + SC::ST_VEL + 4 * i, lv[SC::LV_VX + i], lv[SC::LV_VY + i], lv[SC::LV_W + i]);
     }
-    for (int j = 0; j < 3 * SC::J; ++j) st[SC::ST_JACC + j] = 0u;
-    *reinterpret_cast<uint4 *>(st + SC::ST_META) = make_uint4(0u, (uint32_t)episode, (uint32_t)level, 0u);
-    st[SC::ST_META + META_NROWS] = 0u;
-    atomicAdd(prm.counters + 1, 1ULL);
+    for (int j = lane; j < 3 * SC::J; j += GS) st[SC::ST_JACC + j] = 0u;
+    if (lane == 0) {
+        *reinterpret_cast<uint4 *>(st + SC::ST_META) = make_uint4(0u, (uint32_t)episode, (uint32_t)level, 0u);
+        st[SC::ST_META + META_NROWS] = 0u;
+        atomicAdd(prm.counters + 1, 1ULL);
+    }
 }
 
 // ---------------------------------------------------------------- reset kernel: one block per env
