@@ -47,6 +47,7 @@ extern "C" {
 #define K2D_ERR_CUDA (-6)          /* a CUDA runtime call failed                         */
 #define K2D_ERR_ARG (-7)           /* another argument is invalid                        */
 #define K2D_ERR_LIMIT (-8)         /* a size is beyond a limit built into the library    */
+#define K2D_ERR_WAIT (-9)          /* k2d_status: a wait inside k2d_step ran out (see there) */
 
 #define K2D_MAX_POLYGONS 12
 #define K2D_MAX_CIRCLES 4
@@ -164,10 +165,7 @@ int k2d_reset(k2d_state *s, const int32_t *host_level_ids);
  * floats in {-1, 0, +1}, plus, if dense_kappa is not 0, the paper's auxiliary dense reward
  * kappa * (d_t - d_t+1) with d the distance between the positions of the first green and the
  * first blue shape before and after the step; dev_done [n_steps][n_envs] bytes.  1 <= n_steps <= max_fused_steps.
- * The call enqueues two kernel launches per engine step and returns; nothing in them waits for anything but
- * stream order.  The first kernel of a step works with several lanes per scene (geometry, manifolds, the
- * constraint rows of the step), the second with one thread per scene (the sequential solver, Euler step,
- * reward, termination, auto-reset); between the two the rows sit in the scratch part of the state buffer. */
+ * The whole call is one kernel launch; scene state stays on chip between the fused steps. */
 int k2d_step(k2d_state *s, const float *dev_actions, int32_t n_steps, float *dev_reward, uint8_t *dev_done);
 
 /* The same step with the paper's multi-discrete action space ("Action Space": every motor and
@@ -177,24 +175,22 @@ int k2d_step(k2d_state *s, const float *dev_actions, int32_t n_steps, float *dev
 int k2d_step_discrete(k2d_state *s, const int32_t *dev_actions, int32_t n_steps, float *dev_reward, uint8_t *dev_done);
 
 /* The paper has no counterpart of this call; it exists for one kind of user of this library.
- * k2d_step hands the constraint rows of a step from its first kernel to its second through the
- * scratch tail of the state buffer (19904 bytes per env for the largest scenes), which the caller
- * has to allocate.  Some callers cannot: a process whose device memory is one arena fixed at start-up,
+ * k2d_step keeps the contact records of a very crowded scene (far more touching pairs than
+ * lanes working on the scene) in the scratch tail of the state buffer, which the caller has to
+ * allocate.  Some callers cannot: a process whose device memory is one arena fixed at start-up,
  * a plug-in handed a pre-sized buffer by its host, code running where cudaMalloc is forbidden
  * (a real-time loop).  For them this variant does exactly what k2d_step does, with the same
- * arguments and bit-identical results, but keeps those rows in an array compiled into the
- * library (K2D_STATIC_SCRATCH_MAX_ENVS x 19904 bytes, about 20 MB, resident on every GPU that
- * loads the library until the process exits) and never touches the scratch tail; a state buffer of
- * k2d_state_bytes_no_scratch bytes is enough for a handle that is only ever stepped this way.  It
- * allocates and frees nothing, on the host side of CUDA or on the device.
+ * arguments and bit-identical results, but keeps those records in an array compiled into the
+ * library (K2D_STATIC_SCRATCH_MAX_ENVS x 13920 bytes, about 14 MB, resident on every GPU that
+ * loads the library until the process exits) and never touches the scratch tail.  It allocates
+ * and frees nothing, on the host side of CUDA or on the device.
  *  - n_envs above K2D_STATIC_SCRATCH_MAX_ENVS is refused with K2D_ERR_LIMIT (and a line on
  *    stderr); nothing is enqueued.
  *  - The first call on each device looks up the array's device address (with that device made
  *    current); make that first call before any stream capture begins.
- *  - All handles and streams of a process share the one array per device.  It carries nothing from
- *    one call to the next and nothing in it has to start at zero (every row is written by a step's
- *    first kernel before its second kernel reads it), so calls one after another, of one handle or of
- *    several, need no clearing; calls that overlap on the GPU (two streams, two handles) race on it
+ *  - All handles and streams of a process share the one array per device.  Nothing in it has
+ *    to start at zero (every record is written before it is read), so calls one after another
+ *    need no clearing; calls that overlap on the GPU (two streams, two handles) race on it
  *    and must be serialised by the caller. */
 #define K2D_STATIC_SCRATCH_MAX_ENVS 1024
 int k2d_step_static_scratch(k2d_state *s, const float *dev_actions, int32_t n_steps, float *dev_reward, uint8_t *dev_done);
@@ -229,7 +225,11 @@ int k2d_set_state(k2d_state *s, const void *host_canonical);
 
 /* host_counts[8] (int64), all since the last k2d_reset: non-finite events, auto-resets, active
  * manifolds summed over env-steps, env-steps, pairs that passed the bounding-box test (polygon-
- * polygon, polygon-circle, circle-circle), pairs with at least one active manifold. */
+ * polygon, polygon-circle, circle-circle), pairs with at least one active manifold.
+ * Returns K2D_ERR_WAIT (with the counts filled in) if, in some k2d_step since the last k2d_reset,
+ * a group of lanes waited longer than its limit (seconds) for another group to finish an earlier
+ * part of the same env's steps: the kernel then gave up on that env instead of hanging, and the
+ * states are not valid any more; k2d_reset clears the condition. */
 int k2d_status(k2d_state *s, int64_t *host_counts);
 
 /* Host only, no device needed: validates one level against the config and returns the constants

@@ -3,7 +3,6 @@
 #include <cmath>
 #include <cstdio>
 #include <cstring>
-#include <cstdlib>
 #include <mutex>
 #include <new>
 #include <vector>
@@ -17,15 +16,20 @@ using ClassS = SizeClass<5, 2, 1, 1>;
 using ClassM = SizeClass<6, 3, 2, 2>;
 using ClassL = SizeClass<12, 4, 6, 2>;
 
+constexpr int kMaxSlots = 8192;      // resident scene groups a launch may use (bounds the overflow scratch)
 constexpr size_t kCtrlBytes = 256;   // control block at the start of the state buffer: 8 x uint64 counters, then the work queue words
 constexpr size_t kQueueOffset = 128;
+#ifndef K2D_CHUNK_STEPS
+#define K2D_CHUNK_STEPS 8
+#endif
+constexpr int kChunkSteps = K2D_CHUNK_STEPS;       // steps per work item when there are more envs than resident scene groups
 
 // run-time view of a size class
 struct ClassInfo {
     int id, P, C, N, J, T, NPP, NPC, NCC, NPAIRS, NSLOTS, MASKW;
     int LV_WORDS, ST_WORDS, SCRATCH_WORDS, PTAB_WORDS;
     int LV_X, LV_IM, LV_II, LV_FR, LV_RE, LV_FLAGS, LV_DENS, LV_RAD, LV_PVX, LV_PVY, LV_PNX, LV_PNY, LV_ELEN, LV_JOINT, LV_THR, LV_MASK, LV_GB;
-    int ST_POS, ST_VEL, ST_JACC, ST_META, ST_WARM;
+    int ST_JACC, ST_META, ST_WARM;
 };
 template <class SC>
 static ClassInfo make_info(int id) {
@@ -36,7 +40,7 @@ static ClassInfo make_info(int id) {
     c.LV_X = SC::LV_X; c.LV_IM = SC::LV_IM; c.LV_II = SC::LV_II; c.LV_FR = SC::LV_FR; c.LV_RE = SC::LV_RE; c.LV_FLAGS = SC::LV_FLAGS;
     c.LV_DENS = SC::LV_DENS; c.LV_RAD = SC::LV_RAD; c.LV_PVX = SC::LV_PVX; c.LV_PVY = SC::LV_PVY; c.LV_PNX = SC::LV_PNX; c.LV_PNY = SC::LV_PNY;
     c.LV_ELEN = SC::LV_ELEN; c.LV_JOINT = SC::LV_JOINT; c.LV_THR = SC::LV_THR; c.LV_MASK = SC::LV_MASK; c.LV_GB = SC::LV_GB;
-    c.ST_POS = SC::ST_POS; c.ST_VEL = SC::ST_VEL; c.ST_JACC = SC::ST_JACC; c.ST_META = SC::ST_META; c.ST_WARM = SC::ST_WARM;
+    c.ST_JACC = SC::ST_JACC; c.ST_META = SC::ST_META; c.ST_WARM = SC::ST_WARM;
     return c;
 }
 
@@ -84,12 +88,12 @@ using namespace k2d;
 struct k2d_state {
     k2d_config cfg;
     ClassInfo ci;
-    int G, grid;
+    int G, grid, groups, slots;
     size_t smem_bytes;
     cudaStream_t stream;
     unsigned char *dev_base;
     unsigned long long *dev_counters;
-    unsigned int *dev_queue;
+    unsigned int *dev_queue, *dev_chunks;
     int *dev_ids;
     uint32_t *dev_env, *dev_scratch, *dev_levels;
     float *dev_trace;
@@ -102,14 +106,16 @@ namespace k2d {
 
 static size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
-// control block | reset staging ids | env states | scratch (the constraint rows of every env's current step)
-struct BufLayout { size_t ids_off, env_off, scratch_off, total; };
+struct BufLayout { size_t ids_off, chunks_off, env_off, scratch_off, total; int slots; };
 static BufLayout buffer_layout(const k2d_config *cfg, const ClassInfo &ci) {
     BufLayout b{};
+    // every scene group of a launch can end up stepping an env, so the scratch covers whole blocks (up to 16 groups each)
+    b.slots = ((cfg->n_envs < kMaxSlots ? cfg->n_envs : kMaxSlots) + 15) / 16 * 16;
     b.ids_off = kCtrlBytes;
-    b.env_off = align_up(b.ids_off + (size_t)cfg->n_envs * 4, 256);
+    b.chunks_off = align_up(b.ids_off + (size_t)cfg->n_envs * 4, 256);
+    b.env_off = align_up(b.chunks_off + (size_t)cfg->n_envs * 4, 256);
     b.scratch_off = align_up(b.env_off + (size_t)cfg->n_envs * ci.ST_WORDS * 4, 256);
-    b.total = align_up(b.scratch_off + (size_t)cfg->n_envs * ci.SCRATCH_WORDS * 4, 256);
+    b.total = align_up(b.scratch_off + (size_t)b.slots * ci.SCRATCH_WORDS * 4, 256);
     return b;
 }
 
@@ -252,33 +258,28 @@ static int pack_level(const k2d_config *cfg, const ClassInfo &ci, const k2d_leve
     return K2D_OK;
 }
 
-// One engine step of every env: the prep kernel (geometry, manifolds, constraint rows), then the solve kernel.
 template <class SC, int G>
 static cudaError_t launch_step(const k2d_state *s, const StepParams &prm) {
-    k2d_prep_kernel<SC, G><<<s->grid, kBlockThreads, s->smem_bytes, s->stream>>>(prm);
-    cudaError_t err = cudaGetLastError();
-    if (err != cudaSuccess) return err;
-    constexpr int SPB = kSolveThreads / kSolveLanes;      // scenes per block of the solve kernel
-    k2d_solve_kernel<SC><<<(prm.n_envs + SPB - 1) / SPB, kSolveThreads, 0, s->stream>>>(prm);
+    k2d_step_kernel<SC, G><<<s->grid, kBlockThreads, s->smem_bytes, s->stream>>>(prm);
     return cudaGetLastError();
 }
 template <class SC, int G>
 static cudaError_t setup_step(k2d_state *s, int num_sms) {
     constexpr int GPB = kBlockThreads / G;
     s->smem_bytes = sizeof(uint32_t) * (SC::PTAB_WORDS + GPB * region_words<SC, G>());
-    cudaError_t err = cudaFuncSetAttribute(k2d_prep_kernel<SC, G>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)s->smem_bytes);
+    cudaError_t err = cudaFuncSetAttribute(k2d_step_kernel<SC, G>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)s->smem_bytes);
     if (err != cudaSuccess) return err;
-    { const char *cv = getenv("K2D_PROBE_CARVEOUT");
-      if (cv) { err = cudaFuncSetAttribute(k2d_solve_kernel<SC>, cudaFuncAttributePreferredSharedMemoryCarveout, atoi(cv)); if (err != cudaSuccess) return err; } }
     int per_sm = 0;
-    err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k2d_prep_kernel<SC, G>, kBlockThreads, s->smem_bytes);
+    err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k2d_step_kernel<SC, G>, kBlockThreads, s->smem_bytes);
     if (err != cudaSuccess) return err;
     if (per_sm < 1) per_sm = 1;
     int grid = num_sms * per_sm;
     const int need = (s->cfg.n_envs + GPB - 1) / GPB;
     if (grid > need) grid = need;
+    if (grid * GPB > s->slots) grid = s->slots / GPB;
     if (grid < 1) grid = 1;
     s->grid = grid;
+    s->groups = grid * GPB;
     return cudaSuccess;
 }
 
@@ -293,17 +294,23 @@ static cudaError_t launch_obs(const k2d_state *s, float *dev_obs) {
     return cudaGetLastError();
 }
 
-// Kernel arguments of engine step `step` of a k2d_step call: every action row is held for frame_skip steps.
-static StepParams step_params(const k2d_state *s, const float *dev_actions, int step, float *dev_reward, uint8_t *dev_done,
+// Kernel arguments of one k2d_step launch.  With more envs than resident scene groups the launch is cut
+// into chunks of kChunkSteps steps, so that the groups can balance the work between them.
+static StepParams step_params(const k2d_state *s, const float *dev_actions, int n_steps, float *dev_reward, uint8_t *dev_done,
                               uint32_t *scratch, int discrete = 0) {
     const k2d_config &c = s->cfg;
     StepParams prm{};
-    prm.state = s->dev_env; prm.levels = s->dev_levels;
-    prm.actions = dev_actions + (size_t)(step / c.frame_skip) * c.n_envs * c.n_actions;
-    prm.reward = dev_reward + (size_t)step * c.n_envs; prm.done = dev_done + (size_t)step * c.n_envs;
-    prm.counters = s->dev_counters; prm.queue = s->dev_queue; prm.scratch = scratch; prm.trace = s->dev_trace;
-    prm.n_envs = c.n_envs; prm.n_actions = c.n_actions; prm.n_levels = c.n_levels;
-    prm.discrete = discrete; prm.dense_kappa = c.dense_kappa;
+    prm.state = s->dev_env; prm.levels = s->dev_levels; prm.actions = dev_actions; prm.reward = dev_reward; prm.done = dev_done;
+    prm.counters = s->dev_counters; prm.queue = s->dev_queue; prm.chunks_done = s->dev_chunks; prm.scratch = scratch; prm.trace = s->dev_trace;
+    prm.n_envs = c.n_envs; prm.n_steps = n_steps; prm.n_actions = c.n_actions; prm.n_levels = c.n_levels;
+    prm.discrete = discrete; prm.dense_kappa = c.dense_kappa; prm.frame_skip = c.frame_skip;
+    prm.chunk_steps = n_steps; prm.n_chunks = 1;
+    if (c.n_envs > s->groups && n_steps > kChunkSteps) {
+        const int n_chunks = (n_steps + kChunkSteps - 1) / kChunkSteps;
+        if ((unsigned long long)c.n_envs * (unsigned long long)n_chunks + (unsigned long long)s->groups < 0xffffffffULL) {
+            prm.chunk_steps = kChunkSteps; prm.n_chunks = n_chunks;
+        }
+    }
     prm.solver_iters = c.solver_iters; prm.warm_start = c.warm_start; prm.auto_reset = c.auto_reset; prm.max_episode_steps = c.max_episode_steps;
     prm.dt = c.dt; prm.gdt = c.gravity_y * c.dt; prm.contact_alpha = c.contact_alpha; prm.contact_beta = c.contact_beta; prm.slop = c.slop;
     prm.rest_thr = c.restitution_threshold; prm.face_tol = c.face_tol; prm.joint_alpha = c.joint_alpha; prm.joint_beta = c.joint_beta; prm.joint_gamma = c.joint_gamma;
@@ -311,22 +318,10 @@ static StepParams step_params(const k2d_state *s, const float *dev_actions, int 
     return prm;
 }
 
-// all engine steps of one call, in stream order
-static int run_steps(const k2d_state *s, const float *dev_actions, int n_steps, float *dev_reward, uint8_t *dev_done, uint32_t *scratch, int discrete);
-
 #define K2D_DISPATCH(FN, s, ...)                                                                      \
     ((s)->ci.id == 0 ? ((s)->G == 32 ? FN<ClassS, 32>(__VA_ARGS__) : (s)->G == 16 ? FN<ClassS, 16>(__VA_ARGS__) : FN<ClassS, 8>(__VA_ARGS__)) \
    : (s)->ci.id == 1 ? ((s)->G == 32 ? FN<ClassM, 32>(__VA_ARGS__) : (s)->G == 16 ? FN<ClassM, 16>(__VA_ARGS__) : FN<ClassM, 8>(__VA_ARGS__)) \
                      : ((s)->G == 32 ? FN<ClassL, 32>(__VA_ARGS__) : (s)->G == 16 ? FN<ClassL, 16>(__VA_ARGS__) : FN<ClassL, 8>(__VA_ARGS__)))
-
-static int run_steps(const k2d_state *s, const float *dev_actions, int n_steps, float *dev_reward, uint8_t *dev_done, uint32_t *scratch, int discrete) {
-    for (int step = 0; step < n_steps; ++step) {
-        const StepParams prm = step_params(s, dev_actions, step, dev_reward, dev_done, scratch, discrete);
-        const cudaError_t err = K2D_DISPATCH(launch_step, s, s, prm);
-        if (err != cudaSuccess) { std::fprintf(stderr, "k2d_step: launch failed: %s\n", cudaGetErrorString(err)); return K2D_ERR_CUDA; }
-    }
-    return K2D_OK;
-}
 
 }  // namespace k2d
 
@@ -405,9 +400,11 @@ int k2d_create(const k2d_config *cfg, void *dev_state_buf, void *dev_level_pool_
         if (rc != K2D_OK) { delete s; return rc; }
     }
     const BufLayout bl = buffer_layout(cfg, ci);
+    s->slots = bl.slots;
     s->dev_base = (unsigned char *)dev_state_buf;
     s->dev_counters = (unsigned long long *)s->dev_base;
     s->dev_queue = (unsigned int *)(s->dev_base + kQueueOffset);
+    s->dev_chunks = (unsigned int *)(s->dev_base + bl.chunks_off);
     s->dev_ids = (int *)(s->dev_base + bl.ids_off);
     s->dev_env = (uint32_t *)(s->dev_base + bl.env_off);
     s->dev_scratch = (uint32_t *)(s->dev_base + bl.scratch_off);
@@ -415,7 +412,8 @@ int k2d_create(const k2d_config *cfg, void *dev_state_buf, void *dev_level_pool_
     cudaError_t err = cudaSetDevice(cfg->device);
     int num_sms = 0;
     if (err == cudaSuccess) err = cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, cfg->device);
-    // default lanes per scene of the prep kernel: a warp per scene while the device has warps to spare, two scenes per warp beyond
+    // default lanes per scene: a warp per scene while the device has warps to spare (measured on B200: faster below
+    // about 48 envs per SM for the largest size class, 24 for the smaller ones), two scenes per warp beyond
     if (err == cudaSuccess && !cfg->lanes_per_scene) s->G = (cfg->n_envs < (ci.id == 2 ? 48 : 24) * num_sms) ? 32 : 16;
     if (err == cudaSuccess) err = K2D_DISPATCH(setup_step, s, s, num_sms);
     if (err == cudaSuccess) err = cudaMemcpyAsync(s->dev_levels, s->host_levels.data(), s->host_levels.size() * 4, cudaMemcpyHostToDevice, s->stream);
@@ -434,6 +432,7 @@ int k2d_reset(k2d_state *s, const int32_t *host_level_ids) {
         for (int e = 0; e < E; ++e) if (host_level_ids[e] < 0 || host_level_ids[e] >= s->cfg.n_levels) return K2D_ERR_ARG;
     CUDA_OK(cudaSetDevice(s->cfg.device));
     CUDA_OK(cudaMemsetAsync(s->dev_base, 0, kCtrlBytes, s->stream));
+    CUDA_OK(cudaMemsetAsync(s->dev_chunks, 0, (size_t)E * 4, s->stream));
     if (host_level_ids) CUDA_OK(cudaMemcpyAsync(s->dev_ids, host_level_ids, (size_t)E * 4, cudaMemcpyHostToDevice, s->stream));
     const int *ids = host_level_ids ? s->dev_ids : nullptr;
     if (s->ci.id == 0) k2d_reset_kernel<ClassS><<<E, 64, 0, s->stream>>>(s->dev_env, s->dev_levels, ids, E, s->cfg.n_levels);
@@ -449,7 +448,9 @@ int k2d_step(k2d_state *s, const float *dev_actions, int32_t n_steps, float *dev
     if (n_steps < 1 || n_steps > s->cfg.max_fused_steps) return K2D_ERR_STEPS;
     if (((uintptr_t)dev_actions & 3) || ((uintptr_t)dev_reward & 3)) return K2D_ERR_ALIGN;
     CUDA_OK(cudaSetDevice(s->cfg.device));
-    return run_steps(s, dev_actions, n_steps, dev_reward, dev_done, s->dev_scratch, 0);
+    const StepParams prm = step_params(s, dev_actions, n_steps, dev_reward, dev_done, s->dev_scratch);
+    CUDA_OK(K2D_DISPATCH(launch_step, s, s, prm));
+    return K2D_OK;
 }
 
 int k2d_obs(k2d_state *s, float *dev_obs) {
@@ -492,16 +493,14 @@ int k2d_get_state(k2d_state *s, void *host_canonical) {
         std::memset(o, 0, sizeof(uint32_t) * cw);
         for (int i = 0; i < nN; ++i) {
             const int q = s->shape_map[i];
-            const uint32_t *pq = st + ci.ST_POS + 4 * q, *vq = st + ci.ST_VEL + 4 * q;
-            o[2 * i] = pq[0]; o[2 * i + 1] = pq[1];
-            o[2 * nN + i] = pq[2];
-            o[3 * nN + 2 * i] = vq[0]; o[3 * nN + 2 * i + 1] = vq[1];
-            o[5 * nN + i] = vq[2];
+            o[2 * i] = st[0 * ci.N + q]; o[2 * i + 1] = st[1 * ci.N + q];
+            o[2 * nN + i] = st[2 * ci.N + q];
+            o[3 * nN + 2 * i] = st[3 * ci.N + q]; o[3 * nN + 2 * i + 1] = st[4 * ci.N + q];
+            o[5 * nN + i] = st[5 * ci.N + q];
         }
-        // the warm list holds (pair, accumulated normal and tangent impulse of its two manifolds) of the latest step's rows
         uint32_t *acc = o + 6 * nN;
-        const int nrows = (int)st[ci.ST_META + META_NROWS];
-        for (int k = 0; k < nrows && k < ci.NPAIRS; ++k) {
+        const int nwarm = (int)st[ci.ST_META + 4];
+        for (int k = 0; k < nwarm && k < ci.NPAIRS; ++k) {
             const uint32_t *wr = st + ci.ST_WARM + kWarmWords * k;
             const int p = (wr[0] < (uint32_t)ci.NPAIRS) ? inv_pair[wr[0]] : -1;
             if (p < 0) continue;
@@ -535,32 +534,29 @@ int k2d_set_state(k2d_state *s, const void *host_canonical) {
         const int lvl = (int)o[cw - 2];
         // shapes outside the caller's dimensions keep their level pose
         const uint32_t *lv = s->host_levels.data() + (size_t)lvl * ci.LV_WORDS;
-        for (int q = 0; q < ci.N; ++q)
-            for (int f = 0; f < 3; ++f) {
-                st[ci.ST_POS + 4 * q + f] = lv[ci.LV_X + f * ci.N + q];
-                st[ci.ST_VEL + 4 * q + f] = lv[ci.LV_X + (3 + f) * ci.N + q];
-            }
+        for (int i = 0; i < 6 * ci.N; ++i) st[i] = lv[ci.LV_X + i];
         for (int i = 0; i < nN; ++i) {
             const int q = s->shape_map[i];
-            uint32_t *pq = st + ci.ST_POS + 4 * q, *vq = st + ci.ST_VEL + 4 * q;
-            pq[0] = o[2 * i]; pq[1] = o[2 * i + 1]; pq[2] = o[2 * nN + i];
-            vq[0] = o[3 * nN + 2 * i]; vq[1] = o[3 * nN + 2 * i + 1]; vq[2] = o[5 * nN + i];
+            st[0 * ci.N + q] = o[2 * i]; st[1 * ci.N + q] = o[2 * i + 1];
+            st[2 * ci.N + q] = o[2 * nN + i];
+            st[3 * ci.N + q] = o[3 * nN + 2 * i]; st[4 * ci.N + q] = o[3 * nN + 2 * i + 1];
+            st[5 * ci.N + q] = o[5 * nN + i];
         }
         const uint32_t *acc = o + 6 * nN;
-        int nrows = 0;
-        for (int p = 0; p < n_pairs; ++p) {
+        int nwarm = 0;
+        for (int p = 0; p < n_pairs; ++p) {      // config pair order maps monotonically to internal pair order
             const int slot = pair_slot(nP, nC, p);
             const bool two = p < nP * (nP - 1) / 2;
             const uint32_t v[4] = { acc[2 * slot], acc[2 * slot + 1], two ? acc[2 * slot + 2] : 0u, two ? acc[2 * slot + 3] : 0u };
             if (!((v[0] | v[1] | v[2] | v[3]) & 0x7fffffffu)) continue;
-            uint32_t *wr = st + ci.ST_WARM + kWarmWords * nrows++;
+            uint32_t *wr = st + ci.ST_WARM + kWarmWords * nwarm++;
             wr[0] = (uint32_t)s->pair_map[p]; wr[1] = v[0]; wr[2] = v[1]; wr[3] = v[2]; wr[4] = v[3];
         }
         const uint32_t *jacc = acc + 2 * n_slots;
         for (int j = 0; j < 3 * nJ; ++j) st[ci.ST_JACC + j] = jacc[j];
         const uint32_t *meta = jacc + 3 * nJ;
         for (int k = 0; k < 4; ++k) st[ci.ST_META + k] = meta[k];
-        st[ci.ST_META + META_NROWS] = (uint32_t)nrows;
+        st[ci.ST_META + 4] = (uint32_t)nwarm;
     }
     CUDA_OK(cudaSetDevice(c.device));
     CUDA_OK(cudaStreamSynchronize(s->stream));
@@ -573,7 +569,9 @@ int k2d_status(k2d_state *s, int64_t *host_counts) {
     CUDA_OK(cudaSetDevice(s->cfg.device));
     CUDA_OK(cudaStreamSynchronize(s->stream));
     CUDA_OK(cudaMemcpy(host_counts, s->dev_counters, 8 * sizeof(int64_t), cudaMemcpyDeviceToHost));
-    return K2D_OK;
+    unsigned int queue[4] = { 0u, 0u, 0u, 0u };
+    CUDA_OK(cudaMemcpy(queue, s->dev_queue, sizeof(queue), cudaMemcpyDeviceToHost));
+    return queue[Q_ERROR] ? K2D_ERR_WAIT : K2D_OK;
 }
 
 int k2d_level_info(const k2d_config *cfg, const k2d_level *host_level, float *host_inv_mass, float *host_inv_inertia, uint8_t *host_collide) {
@@ -628,7 +626,9 @@ int k2d_step_discrete(k2d_state *s, const int32_t *dev_actions, int32_t n_steps,
     if (n_steps < 1 || n_steps > s->cfg.max_fused_steps) return K2D_ERR_STEPS;
     if (((uintptr_t)dev_actions & 3) || ((uintptr_t)dev_reward & 3)) return K2D_ERR_ALIGN;
     CUDA_OK(cudaSetDevice(s->cfg.device));
-    return run_steps(s, reinterpret_cast<const float *>(dev_actions), n_steps, dev_reward, dev_done, s->dev_scratch, 1);
+    const StepParams prm = step_params(s, reinterpret_cast<const float *>(dev_actions), n_steps, dev_reward, dev_done, s->dev_scratch, 1);
+    CUDA_OK(K2D_DISPATCH(launch_step, s, s, prm));
+    return K2D_OK;
 }
 
 int k2d_step_static_scratch(k2d_state *s, const float *dev_actions, int32_t n_steps, float *dev_reward, uint8_t *dev_done) {
@@ -636,7 +636,7 @@ int k2d_step_static_scratch(k2d_state *s, const float *dev_actions, int32_t n_st
     if (n_steps < 1 || n_steps > s->cfg.max_fused_steps) return K2D_ERR_STEPS;
     if (((uintptr_t)dev_actions & 3) || ((uintptr_t)dev_reward & 3)) return K2D_ERR_ALIGN;
     const k2d_config &c = s->cfg;
-    if (c.n_envs > K2D_STATIC_SCRATCH_MAX_ENVS || c.device >= 64) {
+    if (c.n_envs > K2D_STATIC_SCRATCH_MAX_ENVS || s->groups > K2D_STATIC_SCRATCH_MAX_ENVS || c.device >= 64) {
         std::fprintf(stderr, "k2d_step_static_scratch: n_envs = %d is beyond the built-in scratch (at most %d envs); use k2d_step\n",
                      c.n_envs, K2D_STATIC_SCRATCH_MAX_ENVS);
         return K2D_ERR_LIMIT;
@@ -653,8 +653,10 @@ int k2d_step_static_scratch(k2d_state *s, const float *dev_actions, int32_t n_st
         }
         scratch = k2d_static_ptr[c.device];
     }
-    // the rows of env e live at e x SCRATCH_WORDS of its size class, which is at most the largest class's: the limit on n_envs bounds the array
-    return run_steps(s, dev_actions, n_steps, dev_reward, dev_done, scratch, 0);
+    const StepParams prm = step_params(s, dev_actions, n_steps, dev_reward, dev_done, scratch);
+    // a launch never has more scene groups than envs rounded up to a whole block, so the limit on n_envs bounds the scratch slots
+    CUDA_OK(K2D_DISPATCH(launch_step, s, s, prm));
+    return K2D_OK;
 }
 
 const char *k2d_error_string(int code) {
@@ -668,6 +670,7 @@ const char *k2d_error_string(int code) {
         case K2D_ERR_CUDA: return "CUDA runtime error";
         case K2D_ERR_ARG: return "invalid argument";
         case K2D_ERR_LIMIT: return "size beyond a built-in limit";
+        case K2D_ERR_WAIT: return "a scene group gave up waiting for another; the last step is incomplete";
         default: return "unknown error";
     }
 }

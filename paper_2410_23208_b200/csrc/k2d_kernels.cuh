@@ -1,31 +1,21 @@
 // k2d_kernels.cuh -- device code of the batched 2D rigid-body environment step (sm_100a).
 //
-// One engine step of every env is two kernel launches.
-//
-//   k2d_prep_kernel   A group of G lanes (G = 16: two scenes per warp; 32: one warp per scene; 8: four per warp)
-//                     takes one scene at a time from a ticket queue.  Its lanes work on bodies, polygon vertices,
-//                     shape pairs (bounding-box test, narrowphase) and touching pairs (one per lane): gravity,
-//                     world-frame geometry, motors, thrusters, joint pre-step, manifolds, touch flags, and the
-//                     pre-step of every touching pair.  It leaves the step's constraint rows (one 112-byte row per
-//                     touching pair, sorted by solver level, and one 96-byte row per joint) in the env's scratch
-//                     area and the velocities in the env's state record.
-//   k2d_solve_kernel  A group of 4 lanes (eight scenes per warp) runs the warm start, the solver iterations, the Euler
-//                     step and the positional corrections over those rows, then the reward, the termination and the
-//                     auto-reset.  Only the bodies' velocities (later positions) and the accumulated impulses are in
-//                     shared memory; the rows' constants are read through the read-only cache.
-//
-// The sequential-impulse solver of a scene is a chain of dependent rows with two or three independent rows per link,
-// so it can feed few lanes; its working set is small.  The geometry of a scene is wide (120 pairs to test for the
-// largest size class) and needs a working set of several kilobytes in shared memory.  Hence two kernels with
-// different lanes per scene and different occupancy.
+// One group of G lanes (G = 16: two scenes per warp; 32: one warp per scene; 8: four scenes per warp)
+// owns one scene.  A group takes work items (a run of consecutive steps of one env) from a ticket queue;
+// for an item it loads the scene's state from memory once, keeps it in shared memory (bodies, joint rows,
+// world-frame geometry) and in registers (the contact pair record of every lane) across the item's steps,
+// and writes it back once.  Within a step the lanes of the group work on bodies, polygon vertices, shape
+// pairs (bounding-box test, narrowphase), contact pair records (one per lane) and joints (one per lane).
 //
 // Arithmetic contract: every +,-,*,/,sqrt is an individually rounded IEEE binary32 operation
 // (the file is compiled with --fmad=false --prec-div=true --prec-sqrt=true --ftz=false), a fused
-// multiply-add appears only where the code says __fmaf_rn, and min/max are comparisons.  The solver visits
-// rows in an order equivalent to the canonical one (joints by index, then touching pairs by pair index): "level
-// scheduling": a row's level is one more than the highest level of an earlier row that shares a movable body with it;
-// rows of one level touch disjoint movable bodies and run on different lanes at once, and levels run in order, so every
-// body sees exactly the sequence of updates a one-row-at-a-time sweep would give it: results are bit-identical to that sweep.
+// multiply-add appears only where the code says __fmaf_rn, and min/max are comparisons.  The
+// sequential-impulse solver keeps the canonical constraint order (joints, then contacts by pair
+// index) by "level scheduling": a row's level is one more than the highest level of an earlier
+// row that shares a movable body with it, rows of one level touch disjoint movable bodies and
+// run on different lanes at once, and levels run in order -- every body sees exactly the
+// sequence of updates a one-row-at-a-time sweep would give it, so results are bit-identical to
+// that sweep.
 #pragma once
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -37,25 +27,17 @@ namespace k2d {
 #endif
 constexpr int kBlockThreads = K2D_BLOCK_THREADS;
 #ifndef K2D_MIN_BLOCKS
-#define K2D_MIN_BLOCKS 6
+#define K2D_MIN_BLOCKS 5
 #endif
-constexpr int kMinBlocks = K2D_MIN_BLOCKS;   // resident blocks per SM the prep kernel is compiled for (bounds its registers)
-#ifndef K2D_SOLVE_THREADS
-#define K2D_SOLVE_THREADS 64
-#endif
-constexpr int kSolveThreads = K2D_SOLVE_THREADS;
-#ifndef K2D_SOLVE_LANES
-#define K2D_SOLVE_LANES 4
-#endif
-constexpr int kSolveLanes = K2D_SOLVE_LANES;       // solve kernel: lanes per scene
+constexpr int kMinBlocks = K2D_MIN_BLOCKS;   // resident blocks per SM the step kernel is compiled for (bounds its registers)
 constexpr int kObsThreads = 128;   // observation kernel: one warp per env, four envs per block
 constexpr int kMaxActions = 16;
-enum { Q_TICKET = 0, Q_LEFT = 1 };
-constexpr int kRowWords = 28;   // one touching pair: seven 16-byte groups
+enum { Q_TICKET = 0, Q_LEFT = 1, Q_ERROR = 2 };
+constexpr unsigned kWaitLimit = 1u << 24;   // polls (about 100 ns apart) before a wait for another group's chunk gives up
+constexpr int kRecWords = 24;   // contact pair record
 constexpr int kWarmWords = 5;   // pair index + 4 accumulated impulses
 constexpr int kStageWords = 9;  // packed pair word, normal, two contact points with penetration
-constexpr int kStageStride = 12; // a staged pair in scratch: the stage words, then the row slot it is to fill
-constexpr int kJointWords = 24; // joint row: six 16-byte groups
+constexpr int kJointWords = 24; // joint row kept in shared memory: six 16-byte groups
 constexpr int kJointLevelWords = 12;  // joint record of a level
 
 // ---------------------------------------------------------------- size classes and layouts
@@ -77,19 +59,14 @@ struct SizeClass {
     static constexpr int LV_MASK = LV_THR + 8 * T;
     static constexpr int LV_GB = LV_MASK + MASKW;        // first green shape | first blue shape << 8 | both exist << 16
     static constexpr int LV_WORDS = (LV_GB + 1 + 3) / 4 * 4;
-    // state record of an env: per body the 16-byte groups (x, y, angle, -) and (vx, vy, angular velocity, -), meta,
-    // accumulated joint impulses, and the accumulated impulses of the manifolds that were active in the latest step
-    static constexpr int ST_POS = 0, ST_VEL = 4 * N, ST_META = 8 * N, ST_JACC = ST_META + 8;
-    static constexpr int ST_WARM = (ST_JACC + 3 * J + 3) / 4 * 4;
+    // state record: bodies (same order as shared memory), joint impulses, meta, warm list
+    static constexpr int ST_BODY = 0, ST_JACC = 6 * N, ST_META = ST_JACC + 3 * J, ST_WARM = ST_META + 8;
     static constexpr int ST_WORDS = (ST_WARM + kWarmWords * NPAIRS + 3) / 4 * 4;
-    // scratch of an env, valid from the prep kernel of a step to its solve kernel: pair rows sorted by level, joint rows,
-    // the first row of every level (bytes; entry L for level L, entry highest level + 1 = number of rows), and a
-    // staging area for the pairs of a scene with more touching pairs than lanes
-    static constexpr int SCR_ROWS = 0, SCR_JROW = NPAIRS * kRowWords;
-    static constexpr int SCR_LSTART = SCR_JROW + kJointWords * J;
-    static constexpr int SCR_STAGE = SCR_LSTART + ((NPAIRS + 2 + 3) / 4 + 3) / 4 * 4;
-    static constexpr int SCRATCH_WORDS = SCR_STAGE + kStageStride * NPAIRS;
-    // shared memory region of one scene in the prep kernel (words)
+    // A scene with more touching pairs than lanes takes the step's contact solve through global
+    // scratch: one memory record and one warm entry per pair.
+    static constexpr int SCRATCH_WORDS = NPAIRS * (kRecWords + kWarmWords);
+    static constexpr int SCRATCH_WARM = NPAIRS * kRecWords;
+    // shared memory region of one scene (words)
     // per body 16-byte groups (x, y, angle, -) and (vx, vy, angular velocity, -), then per-body arrays
     static constexpr int BPOS = 0, BVEL = 4 * N;
     static constexpr int BIM = 8 * N, BII = 9 * N, BFR = 10 * N, BRE = 11 * N, BC = 12 * N, BS = 13 * N, BFL = 14 * N;
@@ -98,43 +75,54 @@ struct SizeClass {
     static constexpr int BOX = (WOFF + P4 + 3) / 4 * 4;  // N x (min x, min y, max x, max y), 16-byte aligned
     static constexpr int MASK = BOX + 4 * N;
     static constexpr int ACT = MASK + MASKW;
-    static constexpr int META = ACT + kMaxActions;       // the state record's meta words
-    static constexpr int LVC = (META + 8 + 3) / 4 * 4;   // copy of the level record's edge lengths, joint and thruster records
+    static constexpr int META = ACT + kMaxActions;       // step_count, episode_count, level_id, status, warm entries
+    static constexpr int JROW = (META + 8 + 3) / 4 * 4;  // J rows of kJointWords, 16-byte aligned
+    static constexpr int LVC = JROW + kJointWords * J;   // copy of the level record's edge lengths, joint and thruster records
     static constexpr int LVC_WORDS = LV_MASK - LV_ELEN;
-    static constexpr int ELEN = LVC, LVC_JOINT = LVC + (LV_JOINT - LV_ELEN), LVC_THR = LVC + (LV_THR - LV_ELEN);
-    static constexpr int SURV = LVC + LVC_WORDS;         // bytes: pairs that passed the box test; afterwards per-body words of the level search
-    static constexpr int WIDX = SURV + ((NPAIRS + 3) / 4 > N ? (NPAIRS + 3) / 4 : N); // bytes: pair -> entry of the previous step's warm list
-    // then, per lane of the group (field-major, G words per field): kStageWords fields, touching pairs on their way to
-    // the lane that builds their rows
+    static constexpr int SURV = LVC + LVC_WORDS;         // bytes: pairs that passed the box test
+    static constexpr int WIDX = SURV + ((NPAIRS + 3) / 4 > N ? (NPAIRS + 3) / 4 : N); // bytes: pair -> record index of the previous step (the survivor area is reused as N words)
+    // then, per lane of the group (field-major, G words per field):
+    //   STG  kStageWords fields: manifolds on their way to the owning lane; afterwards the second manifold's constants
+    //   ACC2 2 fields: accumulated impulses of the second manifold
+    // (the positional corrections of a lane's record, 2 x G words, reuse the world-frame vertex arrays after the narrowphase)
+    // then kRecWords fields of G / 2 words: second records of the lower half of the lanes
     static constexpr int STG = WIDX + (NPAIRS + 3) / 4;
+    static constexpr int LANE_FIELDS = kStageWords + 2;
     static constexpr int PTAB_WORDS = ((NPAIRS + 1) / 2 + 3) / 4 * 4;  // block-shared pair table, 16 bits per pair
 };
-// pair row (scratch): what the solver needs of one touching pair: pair word, normal, friction | inverse masses and inertias |
-// per manifold the lever-arm cross products, effective masses, target normal velocity, positional correction | the four
-// accumulated impulses
-enum { R_AB = 0, R_NX, R_NY, R_MU, R_MA, R_MB, R_IA, R_IB, R_M0 = 8, R_M1 = 16, R_ACC = 24 };
-enum { M_RNA = 0, M_RNB, M_RTA, M_RTB, M_MASSN, M_MASST, M_TARGET, M_CORR };
-static_assert(R_ACC + 4 == kRowWords, "row size");
-// row AB word = staged AB word
+// memory form of a contact pair record (the overflow path keeps records in global scratch)
+enum { R_AB = 0, R_NX, R_NY, R_MU, R_M0 = 4 };
+enum { M_RNA = 0, M_RNB, M_RTA, M_RTB, M_MASSN, M_MASST, M_TARGET, M_CORR, M_ACCN, M_ACCT, M_WORDS };
+static_assert(R_M0 + 2 * M_WORDS == kRecWords, "record size");
 // staged manifold fields
 enum { S_AB = 0, S_NX, S_NY, S_PX0, S_PY0, S_PEN0, S_PX1, S_PY1, S_PEN1 };
 static_assert(S_PEN1 + 1 == kStageWords, "stage size");
-// staged AB word: a | b<<5 | active manifolds<<10 | pair<<12 | level<<19 | a movable<<26 | b movable<<27
+// second-manifold constants reuse the stage fields of the same lane
+enum { M2_RNA = 0, M2_RNB, M2_RTA, M2_RTB, M2_MASSN, M2_MASST, M2_TARGET };
+// per-lane fields after the stage fields
+enum { LF_ACC2N = kStageWords, LF_ACC2T, LF_COUNT };
+// The lower half of the lanes can hold a second record each (pair number G + lane of a crowded scene),
+// in memory form: kRecWords fields of G / 2 words after the per-lane fields.  Stage field f of such a
+// record waits in record field ovs(f), clear of the accumulated impulses.
+__host__ __device__ constexpr int ovs(int f) { return f < 3 ? f : f + 1; }
+constexpr int OV_ACC0N = R_M0 + M_ACCN, OV_ACC0T = R_M0 + M_ACCT, OV_ACC1N = R_M0 + M_WORDS + M_ACCN, OV_ACC1T = R_M0 + M_WORDS + M_ACCT;
 // joint row fields
-enum { JR_RAX = 0, JR_RAY, JR_RBX, JR_RBY, JR_I11, JR_I12, JR_I22, JR_JAB, JR_BX, JR_BY, JR_CX, JR_CY, JR_MA, JR_MB, JR_IA, JR_IB,
+enum { JR_RAX = 0, JR_RAY, JR_RBX, JR_RBY, JR_I11, JR_I12, JR_I22, JR_PAD0, JR_BX, JR_BY, JR_CX, JR_CY, JR_MA, JR_MB, JR_IA, JR_IB,
        JR_ACCX, JR_ACCY, JR_PAD1, JR_PAD2,
        JR_ANG, JR_KR, JR_BIASR, JR_ACCR };   // angular row: kind (0 none, 1 fixed, 2 beyond the upper limit, 3 beyond the lower), 1 / (1/I_a + 1/I_b), gamma x error, accumulated
 static_assert(JR_ACCR + 1 == kJointWords, "joint row size");
-// meta words of a state record.  NROWS is the number of pair rows of the latest step (= entries of the warm list).  FLAGS, D0
-// and ACTIVE are messages from the prep kernel to the solve kernel of the same step: touch flags (green-blue | green-red << 1),
-// the dense reward's shapes (both exist << 2 | green << 8 | blue << 16), the highest contact level << 24; the distance of
-// those shapes before the step; the bit mask of the shapes that exist | the highest joint level << 16.
-enum { META_STEP = 0, META_EPISODE, META_LEVEL, META_STATUS, META_NROWS, META_FLAGS, META_D0, META_ACTIVE };
+enum { META_STEP = 0, META_EPISODE, META_LEVEL, META_STATUS, META_NWARM, META_GB, META_D0 };   // the last two: dense reward's shapes and distance before the step
 
+// shared-memory word of word i of a state record's body block (x[N], y[N], angle[N], vx[N], vy[N], w[N])
+template <class SC>
+__device__ __forceinline__ int body_word(int i) {
+    const int f = i / SC::N, b = i - f * SC::N;
+    return (f < 3 ? SC::BPOS + f : SC::BVEL + f - 3) + 4 * b;
+}
 // shared-memory words per scene: padded so that the groups of one warp start in different banks
 template <class SC, int G>
 __host__ __device__ constexpr int region_words() {
-    constexpr int raw = SC::STG + kStageWords * G;
+    constexpr int raw = SC::STG + SC::LANE_FIELDS * G + kRecWords * (G / 2);
     return G < 32 ? (raw - G + 31) / 32 * 32 + G : (raw + 3) / 4 * 4;
 }
 
@@ -144,20 +132,24 @@ __host__ __device__ inline uint32_t flag_role(uint32_t f) { return (f >> 2) & 3u
 __host__ __device__ inline uint32_t flag_nverts(uint32_t f) { return (f >> 4) & 7u; }
 // joint packed word: a | b<<8 | binding<<16 | on<<24 | level<<25 | active<<28 | a movable<<29 | b movable<<30 | fixed or limited<<31
 // thruster packed word: shape | binding<<8 | on<<16 | level<<17 | active<<20
+// record AB word: a | b<<5 | amask<<10 | pair<<12 | level<<19 | dynA<<26 | dynB<<27
 
 struct StepParams {
     uint32_t *state;
     const uint32_t *levels;
-    const float *actions;      // the action row of this step, [n_envs][n_actions]
-    float *reward;             // this step's [n_envs]
+    const float *actions;
+    float *reward;
     uint8_t *done;
     unsigned long long *counters;
-    unsigned int *queue;       // work queue words of the prep kernel: next ticket, groups that have left
-    uint32_t *scratch;         // [n_envs][SCRATCH_WORDS]
+    unsigned int *queue;       // work queue words: next ticket, groups that have left, error flag
+    unsigned int *chunks_done; // per env: chunks of this launch already stepped (0 again when the launch is over)
+    uint32_t *scratch;
     float *trace;
-    int n_envs, n_actions, n_levels;
+    int n_envs, n_steps, n_actions, n_levels;
+    int chunk_steps, n_chunks;   // a launch is cut into n_chunks pieces of chunk_steps steps; work items are (chunk, env)
     int solver_iters, warm_start, auto_reset, max_episode_steps;
     int discrete;             // actions are int32 codes (multi-discrete action space) instead of floats
+    int frame_skip;           // engine steps each action row is held for
     float dense_kappa;        // coefficient of the dense reward (0 = off)
     float dt, gdt, contact_alpha, contact_beta, slop, rest_thr, face_tol, joint_alpha, joint_beta, joint_gamma, motor_rho, aabb_margin;
     unsigned long long seed;
@@ -231,6 +223,7 @@ __device__ __forceinline__ unsigned long long mix64(unsigned long long z) {
     z ^= z >> 31;
     return z;
 }
+
 // ---------------------------------------------------------------- group of G lanes
 template <int G>
 struct Group {
@@ -258,6 +251,24 @@ struct Group {
 
 // one manifold as the narrowphase leaves it
 struct Manifold { float px, py, nx, ny, pen; };
+
+// What the lane that owns a contact pair record keeps in registers for the whole step: the pair
+// (packed word), the shared normal, the friction coefficient, the inverse masses and inertias of
+// the two bodies, and the first manifold's lever-arm cross products, effective masses, target
+// normal velocity and accumulated impulses.  The second manifold (polygon-polygon pairs only) is
+// in the lane's shared-memory fields.
+struct Rec {
+    uint32_t ab;
+    float nx, ny, mu, ma, mb, ia, ib;
+    float rna, rnb, rta, rtb, massn, masst, target, accn, acct;
+};
+// memory form (overflow path)
+struct RecM {
+    uint32_t ab;
+    float nx, ny, mu;
+    float rna[2], rnb[2], rta[2], rtb[2], massn[2], masst[2], target[2], corr[2], accn[2], acct[2];
+};
+
 struct ContactConsts { float slop, rest_thr, alpha, beta; };
 
 // ---- contact pre-step for one manifold of pair (a, b) with normal (nx, ny)
@@ -326,22 +337,490 @@ __device__ __forceinline__ void manifold_rows(float nx, float ny, float mu, floa
         vbx = __fmaf_rn(mb, px, vbx); vby = __fmaf_rn(mb, py, vby); wb = __fmaf_rn(wtb, dt_, wb);
     }
 }
-template <class SC>
-__device__ __forceinline__ uint16_t pair_code(int p) {
-    int a, b;
-    if (p < SC::NPP) { int i = 0, rem = p; while (rem >= SC::P - 1 - i) { rem -= SC::P - 1 - i; ++i; } a = i; b = i + 1 + rem; }
-    else if (p < SC::NPP + SC::NPC) { const int q = p - SC::NPP; a = q / SC::C; b = SC::P + q % SC::C; }
-    else { int i = 0, rem = p - SC::NPP - SC::NPC; while (rem >= SC::C - 1 - i) { rem -= SC::C - 1 - i; ++i; } a = SC::P + i; b = SC::P + i + 1 + rem; }
-    return (uint16_t)(a | (b << 8));
+
+// positional correction of one pair: each active manifold moves the two bodies apart along the normal
+__device__ __forceinline__ void correct_pair(float *pos, int a, int b, unsigned amask, bool dyn_a, bool dyn_b,
+                                             float nx, float ny, float ma, float mb, float corr0, float corr1) {
+    float xa = pos[4 * a], ya = pos[4 * a + 1], xb = pos[4 * b], yb = pos[4 * b + 1];
+    if (amask & 1u) {
+        const float ca = ma * corr0, cb = mb * corr0;
+        xa = __fmaf_rn(-ca, nx, xa); ya = __fmaf_rn(-ca, ny, ya);
+        xb = __fmaf_rn(cb, nx, xb); yb = __fmaf_rn(cb, ny, yb);
+    }
+    if (amask & 2u) {
+        const float ca = ma * corr1, cb = mb * corr1;
+        xa = __fmaf_rn(-ca, nx, xa); ya = __fmaf_rn(-ca, ny, ya);
+        xb = __fmaf_rn(cb, nx, xb); yb = __fmaf_rn(cb, ny, yb);
+    }
+    if (dyn_a) { pos[4 * a] = xa; pos[4 * a + 1] = ya; }
+    if (dyn_b) { pos[4 * b] = xb; pos[4 * b + 1] = yb; }
+}
+
+// ---- angular row of a fixed joint or of a revolute joint beyond one of its limits (paper, "Fixed Joints",
+// "Joint Limits"): j_r = (w_a - w_b + correction) / (1/I_a + 1/I_b), a loses j_r / I_a, b gains j_r / I_b.  A fixed
+// joint's impulse is accumulated and warm-started; a limit only ever pushes back, applies no correction while the
+// joint is already returning, and is not accumulated.  Returns the two angular velocities.  Out of line: most
+// joints are plain revolute joints.
+template <int MODE>
+__device__ __noinline__ float2 angular_row(float *jr, float ia, float ib, float wa, float wb) {
+    const float4 ang4 = ld4(jr + JR_ANG);      // kind this step, inverse angular mass, correction, accumulated impulse
+    const int ang = __float_as_int(ang4.x);
+    if (ang == 0) return make_float2(wa, wb);
+    float lr;
+    if (MODE == 0) {
+        if (ang != 1) return make_float2(wa, wb);
+        lr = ang4.w;
+    } else {
+        const float wrel = wa - wb;
+        float v;
+        if (ang == 1) v = wrel + ang4.z;
+        else if (ang == 2) { v = (wrel < 0.0f) ? wrel : wrel + ang4.z; v = fmax_cmp(v, 0.0f); }
+        else { v = (wrel > 0.0f) ? wrel : wrel + ang4.z; v = fmin_cmp(v, 0.0f); }
+        lr = v * ang4.y;
+        if (ang == 1) jr[JR_ACCR] = ang4.w + lr;
+    }
+    return make_float2(__fmaf_rn(-lr, ia, wa), __fmaf_rn(lr, ib, wb));
+}
+
+// ---- joints; the row of joint j is in shared memory.  MODE 0: warm start, 1: solver iteration,
+// 2: positional correction, 3: motor
+template <class SC, int MODE>
+__device__ __forceinline__ void visit_joint(float *sm, uint32_t jab, int j, float motor_rho, int discrete = 0) {
+    const int a = jab & 255, b = (jab >> 8) & 255;
+    const bool dyn_a = (jab >> 29) & 1u, dyn_b = (jab >> 30) & 1u;
+    float *jr = sm + SC::JROW + kJointWords * j;
+    if (MODE == 3) {
+        const float av = sm[SC::ACT + ((jab >> 16) & 255)];
+        // paper, "Action Space": continuous in [-1, 1], or multi-discrete codes 0 off, 1 forwards, 2 backwards at full power
+        const float A = discrete ? (__float_as_int(av) == 1 ? 1.0f : (__float_as_int(av) == 2 ? -1.0f : 0.0f))
+                                 : fmax_cmp(fmin_cmp(av, 1.0f), -1.0f);
+        const float *jl = sm + SC::LVC + (SC::LV_JOINT - SC::LV_ELEN) + kJointLevelWords * j;
+        const float speed = jl[5], power = jl[6];
+        const float wa = sm[SC::BVEL + 4 * a + 2], wb = sm[SC::BVEL + 4 * b + 2];
+        const float arg = __fmaf_rn(-speed, A, wa - wb) * motor_rho;
+        const float jr_ = power * tanh_spec(arg);
+        if (dyn_a) sm[SC::BVEL + 4 * a + 2] = __fmaf_rn(-jr_, sm[SC::BII + a], wa);
+        if (dyn_b) sm[SC::BVEL + 4 * b + 2] = __fmaf_rn(jr_, sm[SC::BII + b], wb);
+        return;
+    }
+    const float4 mi4 = ld4(jr + JR_MA);       // inverse masses and inertias of the two bodies
+    const float ma = mi4.x, mb = mi4.y, ia = mi4.z, ib = mi4.w;
+    if (MODE == 2) {
+        const float cx = jr[JR_CX], cy = jr[JR_CY];
+        if (dyn_a) { sm[SC::BPOS + 4 * a] = __fmaf_rn(ma, cx, sm[SC::BPOS + 4 * a]); sm[SC::BPOS + 4 * a + 1] = __fmaf_rn(ma, cy, sm[SC::BPOS + 4 * a + 1]); }
+        if (dyn_b) { sm[SC::BPOS + 4 * b] = __fmaf_rn(-mb, cx, sm[SC::BPOS + 4 * b]); sm[SC::BPOS + 4 * b + 1] = __fmaf_rn(-mb, cy, sm[SC::BPOS + 4 * b + 1]); }
+        return;
+    }
+    const float4 r4 = ld4(jr + JR_RAX);
+    const float rax = r4.x, ray = r4.y, rbx = r4.z, rby = r4.w;
+    const float4 va4 = ld4(sm + SC::BVEL + 4 * a), vb4 = ld4(sm + SC::BVEL + 4 * b);
+    float vax = va4.x, vay = va4.y, wa = va4.z, vbx = vb4.x, vby = vb4.y, wb = vb4.z;
+    float lx, ly;
+    if (MODE == 0) { lx = jr[JR_ACCX]; ly = jr[JR_ACCY]; }
+    else {
+        const float4 k4 = ld4(jr + JR_I11), b4 = ld4(jr + JR_BX);
+        const float2 acc = *reinterpret_cast<const float2 *>(jr + JR_ACCX);
+        const float cx = __fmaf_rn(-wb, rby, vbx) - __fmaf_rn(-wa, ray, vax);
+        const float cy = __fmaf_rn(wb, rbx, vby) - __fmaf_rn(wa, rax, vay);
+        const float rx = -(cx + b4.x), ry = -(cy + b4.y);
+        const float i11 = k4.x, i12 = k4.y, i22 = k4.z;
+        lx = __fmaf_rn(i11, rx, i12 * ry);
+        ly = __fmaf_rn(i12, rx, i22 * ry);
+        *reinterpret_cast<float2 *>(jr + JR_ACCX) = make_float2(acc.x + lx, acc.y + ly);
+    }
+    wa = __fmaf_rn(-ia, cross2(rax, ray, lx, ly), wa);
+    wb = __fmaf_rn(ib, cross2(rbx, rby, lx, ly), wb);
+    if (jab >> 31) {      // fixed or limited joint: its angular row follows the point row
+        const float2 w2 = angular_row<MODE>(jr, ia, ib, wa, wb);
+        wa = w2.x; wb = w2.y;
+    }
+    if (dyn_a) st4(sm + SC::BVEL + 4 * a, __fmaf_rn(-ma, lx, vax), __fmaf_rn(-ma, ly, vay), wa);
+    if (dyn_b) st4(sm + SC::BVEL + 4 * b, __fmaf_rn(mb, lx, vbx), __fmaf_rn(mb, ly, vby), wb);
+}
+// joints of one level touch disjoint movable bodies; levels in order keep the joint order
+template <class SC, int G, int MODE>
+__device__ __forceinline__ void sweep_joints(float *sm, uint32_t jab, int lane, int jlevel, int jmax, float motor_rho,
+                                             int discrete = 0) {
+    const unsigned mask = Group<G>().mask;
+    if (SC::J == 0) return;
+#pragma unroll 1
+    for (int lvl = 1; lvl <= jmax; ++lvl) {
+        if (jlevel == lvl) visit_joint<SC, MODE>(sm, jab, lane, motor_rho, discrete);
+        __syncwarp(mask);
+    }
+}
+
+// Accumulated impulses that pair record `wi` of the previous step left behind (255: the pair was not
+// touching).  Records 0..G-1 live with lane wi (first manifold in its registers: old_n / old_t are the
+// calling lane's own, fetched across lanes here, so every lane of the group must call; second manifold
+// in its shared-memory fields), the next G / 2 records in the second-record fields of lane wi - G, later ones
+// in the warm entries of the global scratch.
+template <class SC, int G>
+__device__ __forceinline__ void warm_lookup(const Group<G> &g, const float *sm, const uint32_t *ovf, int wi, float old_n, float old_t,
+                                            int warm_start, float (&w)[4]) {
+    const int src = (wi < G) ? wi : 0;
+    const float *lf = sm + SC::STG;
+    w[0] = g.shflf(old_n, src); w[1] = g.shflf(old_t, src);
+    w[2] = lf[LF_ACC2N * G + src]; w[3] = lf[LF_ACC2T * G + src];
+    if (wi >= G && wi != 255) {
+        if (wi < G + G / 2) {
+            const float *o = lf + LF_COUNT * G + (wi - G);
+            w[0] = o[OV_ACC0N * (G / 2)]; w[1] = o[OV_ACC0T * (G / 2)]; w[2] = o[OV_ACC1N * (G / 2)]; w[3] = o[OV_ACC1T * (G / 2)];
+        } else {
+            const uint32_t *wr = ovf + SC::SCRATCH_WARM + (size_t)wi * kWarmWords;
+#pragma unroll
+            for (int q = 0; q < 4; ++q) w[q] = __uint_as_float(wr[1 + q]);
+        }
+    }
+    if (wi == 255 || !warm_start) { w[0] = 0.0f; w[1] = 0.0f; w[2] = 0.0f; w[3] = 0.0f; }
+}
+
+// Levels of nrec staged pairs by one lane with a per-body table (used when there are more pairs than
+// lanes): a pair's level is one more than the highest level of an earlier pair sharing a movable body.
+// The packed pair words of pairs 0..G-1 are in the stage fields, of the next G / 2 in the second-record
+// fields, of later ones in global scratch; the level goes into bits 19.. of each word.
+template <class SC, int G>
+__device__ __noinline__ int levels_by_one_lane(uint32_t *smu, uint32_t *ovf, int nrec) {
+    uint8_t *bl = reinterpret_cast<uint8_t *>(smu + SC::SURV);   // the survivor list is no longer needed
+    int cmax = 0;
+    for (int i = 0; i < SC::N; ++i) bl[i] = 0;
+    for (int k = 0; k < nrec; ++k) {
+        uint32_t *w = (k < G) ? (smu + SC::STG + S_AB * G + k)
+                    : (k < G + G / 2) ? (smu + SC::STG + LF_COUNT * G + ovs(S_AB) * (G / 2) + (k - G)) : (ovf + (size_t)k * kRecWords + S_AB);
+        const uint32_t ab = *w;
+        const int a = ab & 31, b = (ab >> 5) & 31;
+        int lvl = 1;
+        if ((ab >> 26) & 1u) lvl = max(lvl, bl[a] + 1);
+        if ((ab >> 27) & 1u) lvl = max(lvl, bl[b] + 1);
+        if ((ab >> 26) & 1u) bl[a] = (uint8_t)lvl;
+        if ((ab >> 27) & 1u) bl[b] = (uint8_t)lvl;
+        *w = ab | ((uint32_t)lvl << 19);
+        cmax = max(cmax, lvl);
+    }
+    return cmax;
+}
+
+// ================================================================ overflow path (cold code)
+// A scene with more touching pairs than lanes (nrec > G) solves this step's contacts from memory
+// records in global scratch, one loop over records per level, with the same row arithmetic.
+__device__ __forceinline__ void recm_load(const uint32_t *r, RecM &c) {
+    c.ab = r[R_AB]; c.nx = __uint_as_float(r[R_NX]); c.ny = __uint_as_float(r[R_NY]); c.mu = __uint_as_float(r[R_MU]);
+#pragma unroll
+    for (int mi = 0; mi < 2; ++mi) {
+        const uint32_t *m = r + R_M0 + mi * M_WORDS;
+        c.rna[mi] = __uint_as_float(m[M_RNA]); c.rnb[mi] = __uint_as_float(m[M_RNB]);
+        c.rta[mi] = __uint_as_float(m[M_RTA]); c.rtb[mi] = __uint_as_float(m[M_RTB]);
+        c.massn[mi] = __uint_as_float(m[M_MASSN]); c.masst[mi] = __uint_as_float(m[M_MASST]);
+        c.target[mi] = __uint_as_float(m[M_TARGET]); c.corr[mi] = __uint_as_float(m[M_CORR]);
+        c.accn[mi] = __uint_as_float(m[M_ACCN]); c.acct[mi] = __uint_as_float(m[M_ACCT]);
+    }
+}
+__device__ __forceinline__ void recm_store(uint32_t *r, const RecM &c) {
+    r[R_AB] = c.ab; r[R_NX] = __float_as_uint(c.nx); r[R_NY] = __float_as_uint(c.ny); r[R_MU] = __float_as_uint(c.mu);
+#pragma unroll
+    for (int mi = 0; mi < 2; ++mi) {
+        uint32_t *m = r + R_M0 + mi * M_WORDS;
+        m[M_RNA] = __float_as_uint(c.rna[mi]); m[M_RNB] = __float_as_uint(c.rnb[mi]);
+        m[M_RTA] = __float_as_uint(c.rta[mi]); m[M_RTB] = __float_as_uint(c.rtb[mi]);
+        m[M_MASSN] = __float_as_uint(c.massn[mi]); m[M_MASST] = __float_as_uint(c.masst[mi]);
+        m[M_TARGET] = __float_as_uint(c.target[mi]); m[M_CORR] = __float_as_uint(c.corr[mi]);
+        m[M_ACCN] = __float_as_uint(c.accn[mi]); m[M_ACCT] = __float_as_uint(c.acct[mi]);
+    }
+}
+
+template <class SC, int G, int MODE>
+__device__ __forceinline__ void slow_sweep_pairs(float *sm, uint32_t *ovf, int nrec, int cmax) {
+    Group<G> g;
+    for (int lvl = 1; lvl <= cmax; ++lvl) {
+        for (int k = g.lane; k < nrec; k += G) {
+            uint32_t *r = ovf + (size_t)k * kRecWords;
+            if (((r[R_AB] >> 19) & 127u) != (unsigned)lvl) continue;
+            RecM c;
+            recm_load(r, c);
+            const int a = c.ab & 31, b = (c.ab >> 5) & 31;
+            const unsigned amask = (c.ab >> 10) & 3u;
+            const bool dyn_a = (c.ab >> 26) & 1u, dyn_b = (c.ab >> 27) & 1u;
+            const float ma = sm[SC::BIM + a], mb = sm[SC::BIM + b];
+            if (MODE == 2) { correct_pair(sm + SC::BPOS, a, b, amask, dyn_a, dyn_b, c.nx, c.ny, ma, mb, c.corr[0], c.corr[1]); continue; }
+            const float ia = sm[SC::BII + a], ib = sm[SC::BII + b];
+            const float4 va4 = ld4(sm + SC::BVEL + 4 * a), vb4 = ld4(sm + SC::BVEL + 4 * b);
+            float vax = va4.x, vay = va4.y, wa = va4.z, vbx = vb4.x, vby = vb4.y, wb = vb4.z;
+#pragma unroll
+            for (int mi = 0; mi < 2; ++mi) {
+                if (amask & (1u << mi)) {
+                    manifold_rows<MODE>(c.nx, c.ny, c.mu, ma, mb, ia, ib, c.rna[mi], c.rnb[mi], c.rta[mi], c.rtb[mi], c.massn[mi], c.masst[mi],
+                                        c.target[mi], c.accn[mi], c.acct[mi], vax, vay, wa, vbx, vby, wb);
+                    if (MODE == 1) {
+                        r[R_M0 + mi * M_WORDS + M_ACCN] = __float_as_uint(c.accn[mi]);
+                        r[R_M0 + mi * M_WORDS + M_ACCT] = __float_as_uint(c.acct[mi]);
+                    }
+                }
+            }
+            if (dyn_a) st4(sm + SC::BVEL + 4 * a, vax, vay, wa);
+            if (dyn_b) st4(sm + SC::BVEL + 4 * b, vbx, vby, wb);
+        }
+        g.sync();
+    }
+}
+
+// Records from the staged manifolds (the first G in shared memory, the rest already in scratch),
+// their levels, warm start and all solver iterations, joints included.  old_n / old_t: this lane's
+// first-manifold accumulated impulses of the previous step.  Returns the highest contact level.
+template <class SC, int G>
+__device__ __noinline__ int slow_solve(float *sm, uint32_t *ovf, int nrec, uint32_t jab, int jlevel, int jmax,
+                                       int solver_iters, int warm_start, float motor_rho, float old_n, float old_t, ContactConsts cc) {
+    Group<G> g;
+    const int lane = g.lane;
+    uint32_t *smu = reinterpret_cast<uint32_t *>(sm);
+    const uint8_t *widx = reinterpret_cast<const uint8_t *>(smu + SC::WIDX);
+    int cmax = 0;
+    if (lane == 0) cmax = levels_by_one_lane<SC, G>(smu, ovf, nrec);
+    __threadfence_block();
+    g.sync();
+    cmax = g.shfl(cmax, 0);
+    // the staged manifolds of the first G + G / 2 pairs join the others in scratch
+    {
+        uint32_t *r = ovf + (size_t)lane * kRecWords, *r2 = ovf + (size_t)(G + lane) * kRecWords;
+#pragma unroll
+        for (int f = 0; f < kStageWords; ++f) {
+            r[f] = smu[SC::STG + f * G + lane];
+            if (lane < G / 2) r2[f] = smu[SC::STG + LF_COUNT * G + ovs(f) * (G / 2) + lane];
+        }
+    }
+    g.sync();
+    // pre-step of every pair; accumulated impulses of the previous step come from the lane that
+    // owned the pair then (first manifold in its registers, second in its shared-memory fields)
+    // or from the warm entries in scratch
+    for (int base = 0; base < nrec; base += G) {
+        const int k = base + lane;
+        const bool valid = k < nrec;
+        uint32_t *r = ovf + (size_t)(valid ? k : 0) * kRecWords;
+        uint32_t ab = 0u;
+        int wi = 255;
+        if (valid) { ab = r[S_AB]; wi = widx[(ab >> 12) & 127]; }
+        float w[4];
+        warm_lookup<SC, G>(g, sm, ovf, wi, old_n, old_t, warm_start, w);
+        if (valid) {
+            RecM c;
+            c.ab = ab; c.nx = __uint_as_float(r[S_NX]); c.ny = __uint_as_float(r[S_NY]);
+            const float pt[6] = { __uint_as_float(r[S_PX0]), __uint_as_float(r[S_PY0]), __uint_as_float(r[S_PEN0]),
+                                  __uint_as_float(r[S_PX1]), __uint_as_float(r[S_PY1]), __uint_as_float(r[S_PEN1]) };
+            const int a = ab & 31, b = (ab >> 5) & 31;
+            const float ma = sm[SC::BIM + a], mb = sm[SC::BIM + b], ia = sm[SC::BII + a], ib = sm[SC::BII + b];
+            const float fra = sm[SC::BFR + a], frb = sm[SC::BFR + b];
+            const float er = fmin_cmp(sm[SC::BRE + a], sm[SC::BRE + b]);
+            c.mu = sqrtf(__fmaf_rn(fra, fra, frb * frb));
+#pragma unroll
+            for (int mi = 0; mi < 2; ++mi) {
+                if ((ab >> 10) & (1u << mi)) {
+                    prestep_manifold<SC>(a, b, c.nx, c.ny, ma, mb, ia, ib, pt[3 * mi], pt[3 * mi + 1], pt[3 * mi + 2], er, sm, cc,
+                                         c.rna[mi], c.rnb[mi], c.rta[mi], c.rtb[mi], c.massn[mi], c.masst[mi], c.target[mi], c.corr[mi]);
+                    c.accn[mi] = w[2 * mi]; c.acct[mi] = w[2 * mi + 1];
+                } else {
+                    c.rna[mi] = 0.0f; c.rnb[mi] = 0.0f; c.rta[mi] = 0.0f; c.rtb[mi] = 0.0f; c.massn[mi] = 0.0f; c.masst[mi] = 0.0f;
+                    c.target[mi] = 0.0f; c.corr[mi] = 0.0f; c.accn[mi] = 0.0f; c.acct[mi] = 0.0f;
+                }
+            }
+            recm_store(r, c);
+        }
+    }
+    g.sync();
+    slow_sweep_pairs<SC, G, 0>(sm, ovf, nrec, cmax);
+    sweep_joints<SC, G, 0>(sm, jab, lane, jlevel, jmax, motor_rho);
+    for (int it = 0; it < solver_iters; ++it) {
+        sweep_joints<SC, G, 1>(sm, jab, lane, jlevel, jmax, motor_rho);
+        slow_sweep_pairs<SC, G, 1>(sm, ovf, nrec, cmax);
+    }
+    return cmax;
+}
+
+template <class SC, int G>
+__device__ __noinline__ void slow_correct(float *sm, uint32_t *ovf, int nrec, int cmax) {
+    slow_sweep_pairs<SC, G, 2>(sm, ovf, nrec, cmax);
+}
+
+// End of an overflow step: every pair's accumulated impulses become warm entries in scratch and the
+// pair index table learns where they are; returns the number of active manifolds.
+template <class SC, int G>
+__device__ __noinline__ int slow_finish(float *sm, uint32_t *ovf, int nrec) {
+    Group<G> g;
+    uint8_t *widx = reinterpret_cast<uint8_t *>(reinterpret_cast<uint32_t *>(sm) + SC::WIDX);
+    int nman = 0;
+    for (int k = g.lane; k < nrec; k += G) {
+        const uint32_t *r = ovf + (size_t)k * kRecWords;
+        uint32_t *wr = ovf + SC::SCRATCH_WARM + (size_t)k * kWarmWords;
+        const uint32_t ab = r[R_AB];
+        const int p = (ab >> 12) & 127;
+        const unsigned am = (ab >> 10) & 3u;
+        wr[0] = (uint32_t)p;
+        wr[1] = (am & 1u) ? r[R_M0 + M_ACCN] : 0u;
+        wr[2] = (am & 1u) ? r[R_M0 + M_ACCT] : 0u;
+        wr[3] = (am & 2u) ? r[R_M0 + M_WORDS + M_ACCN] : 0u;
+        wr[4] = (am & 2u) ? r[R_M0 + M_WORDS + M_ACCT] : 0u;
+        widx[p] = (uint8_t)k;
+        nman += __popc(am);
+    }
+    nman = g.sum_int(nman);
+    g.sync();
+    return nman;
+}
+
+// Launch boundaries: warm entries G + G / 2 .. between the state record and the scratch.
+template <class SC, int G>
+__device__ __noinline__ void warm_in(float *sm, uint32_t *ovf, const uint32_t *st_warm, int nwarm) {
+    Group<G> g;
+    uint8_t *widx = reinterpret_cast<uint8_t *>(reinterpret_cast<uint32_t *>(sm) + SC::WIDX);
+    for (int k = G + G / 2 + g.lane; k < nwarm; k += G) {
+        uint32_t *wr = ovf + SC::SCRATCH_WARM + (size_t)k * kWarmWords;
+#pragma unroll
+        for (int q = 0; q < kWarmWords; ++q) wr[q] = __ldcg(st_warm + kWarmWords * k + q);
+        widx[wr[0]] = (uint8_t)k;
+    }
+}
+template <class SC, int G>
+__device__ __noinline__ void warm_out(const uint32_t *ovf, uint32_t *st_warm, int nwarm) {
+    Group<G> g;
+    for (int k = G + G / 2 + g.lane; k < nwarm; k += G) {
+        const uint32_t *wr = ovf + SC::SCRATCH_WARM + (size_t)k * kWarmWords;
+#pragma unroll
+        for (int q = 0; q < kWarmWords; ++q) st_warm[kWarmWords * k + q] = wr[q];
+    }
+}
+
+// ---- one visit of the calling lane's second record (pair number G + lane of a scene with more than G
+// touching pairs), which is in memory form in the lane's shared-memory fields.  MODE as for the first record.
+template <class SC, int G, int MODE>
+__device__ __noinline__ void visit_second(float *sm) {
+    float *ov = sm + SC::STG + LF_COUNT * G + Group<G>().lane;
+    constexpr int H = G / 2;
+    const uint32_t ab = __float_as_uint(ov[R_AB * H]);
+    const int a = ab & 31, b = (ab >> 5) & 31;
+    const unsigned amask = (ab >> 10) & 3u;
+    const bool dyn_a = (ab >> 26) & 1u, dyn_b = (ab >> 27) & 1u;
+    const float nx = ov[R_NX * H], ny = ov[R_NY * H];
+    const float ma = sm[SC::BIM + a], mb = sm[SC::BIM + b];
+    if (MODE == 2) {
+        correct_pair(sm + SC::BPOS, a, b, amask, dyn_a, dyn_b, nx, ny, ma, mb, ov[(R_M0 + M_CORR) * H], ov[(R_M0 + M_WORDS + M_CORR) * H]);
+        return;
+    }
+    const float ia = sm[SC::BII + a], ib = sm[SC::BII + b], mu = ov[R_MU * H];
+    const float4 va4 = ld4(sm + SC::BVEL + 4 * a), vb4 = ld4(sm + SC::BVEL + 4 * b);
+    float vax = va4.x, vay = va4.y, wa = va4.z, vbx = vb4.x, vby = vb4.y, wb = vb4.z;
+#pragma unroll 1
+    for (int mi = 0; mi < 2; ++mi) {
+        if (amask & (1u << mi)) {
+            float *m = ov + (R_M0 + mi * M_WORDS) * H;
+            float accn = m[M_ACCN * H], acct = m[M_ACCT * H];
+            manifold_rows<MODE>(nx, ny, mu, ma, mb, ia, ib, m[M_RNA * H], m[M_RNB * H], m[M_RTA * H], m[M_RTB * H],
+                                m[M_MASSN * H], m[M_MASST * H], m[M_TARGET * H], accn, acct, vax, vay, wa, vbx, vby, wb);
+            if (MODE == 1) { m[M_ACCN * H] = accn; m[M_ACCT * H] = acct; }
+        }
+    }
+    if (dyn_a) st4(sm + SC::BVEL + 4 * a, vax, vay, wa);
+    if (dyn_b) st4(sm + SC::BVEL + 4 * b, vbx, vby, wb);
+}
+
+// Second records, first half: the accumulated impulses the staged pair G + lane carried out of the
+// previous step, parked in four of the lane's second-record fields that are free until the record is built.
+template <class SC, int G>
+__device__ __noinline__ void second_lookup(float *sm, const uint32_t *ovf, int nrec, float old_n, float old_t, int warm_start) {
+    const Group<G> g;
+    constexpr int H = G / 2;
+    float *ov = sm + SC::STG + LF_COUNT * G + g.lane;
+    const uint8_t *widx = reinterpret_cast<const uint8_t *>(reinterpret_cast<const uint32_t *>(sm) + SC::WIDX);
+    const bool mine2 = g.lane < H && G + g.lane < nrec;
+    int wi2 = 255;
+    if (mine2) wi2 = widx[(__float_as_uint(ov[ovs(S_AB) * H]) >> 12) & 127];
+    float w2[4];
+    warm_lookup<SC, G>(g, sm, ovf, wi2, old_n, old_t, warm_start, w2);
+    if (mine2) {
+#pragma unroll
+        for (int q = 0; q < 4; ++q) ov[(R_M0 + M_WORDS + q) * H] = w2[q];
+    }
+}
+// Second half, after every lane has read what it needs from other lanes: the record is built in place.
+// Returns its level | its number of active manifolds << 8 (0 for a lane without a second record).
+template <class SC, int G>
+__device__ __noinline__ unsigned second_build(float *sm, int nrec, ContactConsts cc) {
+    const int lane = Group<G>().lane;
+    constexpr int H = G / 2;
+    if (!(lane < H && G + lane < nrec)) return 0u;
+    float *ov = sm + SC::STG + LF_COUNT * G + lane;
+    const uint32_t ab2 = __float_as_uint(ov[ovs(S_AB) * H]);
+    const int a2 = ab2 & 31, b2 = (ab2 >> 5) & 31;
+    const float nx2 = ov[ovs(S_NX) * H], ny2 = ov[ovs(S_NY) * H];
+    const float pt2[6] = { ov[ovs(S_PX0) * H], ov[ovs(S_PY0) * H], ov[ovs(S_PEN0) * H], ov[ovs(S_PX1) * H], ov[ovs(S_PY1) * H], ov[ovs(S_PEN1) * H] };
+    float w2[4];
+#pragma unroll
+    for (int q = 0; q < 4; ++q) w2[q] = ov[(R_M0 + M_WORDS + q) * H];
+    const float ma = sm[SC::BIM + a2], mb = sm[SC::BIM + b2], ia = sm[SC::BII + a2], ib = sm[SC::BII + b2];
+    const float fra = sm[SC::BFR + a2], frb = sm[SC::BFR + b2];
+    const float er2 = fmin_cmp(sm[SC::BRE + a2], sm[SC::BRE + b2]);
+    ov[R_MU * H] = sqrtf(__fmaf_rn(fra, fra, frb * frb));
+#pragma unroll 1
+    for (int mi = 0; mi < 2; ++mi) {
+        float rna = 0.0f, rnb = 0.0f, rta = 0.0f, rtb = 0.0f, massn = 0.0f, masst = 0.0f, target = 0.0f, corr = 0.0f, an = 0.0f, at = 0.0f;
+        if ((ab2 >> 10) & (1u << mi)) {
+            prestep_manifold<SC>(a2, b2, nx2, ny2, ma, mb, ia, ib, pt2[3 * mi], pt2[3 * mi + 1], pt2[3 * mi + 2], er2, sm, cc,
+                                 rna, rnb, rta, rtb, massn, masst, target, corr);
+            an = w2[2 * mi]; at = w2[2 * mi + 1];
+        }
+        float *m = ov + (R_M0 + mi * M_WORDS) * H;
+        m[M_RNA * H] = rna; m[M_RNB * H] = rnb; m[M_RTA * H] = rta; m[M_RTB * H] = rtb;
+        m[M_MASSN * H] = massn; m[M_MASST * H] = masst; m[M_TARGET * H] = target; m[M_CORR * H] = corr;
+        m[M_ACCN * H] = an; m[M_ACCT * H] = at;
+    }
+    return ((ab2 >> 19) & 127u) | ((unsigned)__popc((ab2 >> 10) & 3u) << 8);
 }
 
 // ================================================================ rarely run code, kept out of line
-// what the prep kernel reads of an env's meta words before it starts on the env
-struct MetaHead { uint32_t level, status, nprev; };
-__device__ __forceinline__ MetaHead load_meta_head(const uint32_t *st_meta) {
-    const uint4 m = __ldcg(reinterpret_cast<const uint4 *>(st_meta));
-    MetaHead h; h.level = m.z; h.status = m.w; h.nprev = __ldcg(st_meta + META_NROWS);
-    return h;
+// so that the code a step normally runs stays small
+// level constants into shared memory; returns the packed word of joint number `lane` (0 beyond the last joint)
+template <class SC, int G>
+__device__ __noinline__ uint32_t load_level_consts(uint32_t *smu, const uint32_t *lv) {
+    const int lane = Group<G>().lane;
+    for (int i = lane; i < SC::N; i += G) {
+        smu[SC::BIM + i] = lv[SC::LV_IM + i];
+        smu[SC::BII + i] = lv[SC::LV_II + i];
+        smu[SC::BFR + i] = lv[SC::LV_FR + i];
+        smu[SC::BRE + i] = lv[SC::LV_RE + i];
+        smu[SC::BFL + i] = lv[SC::LV_FLAGS + i];
+    }
+    for (int i = lane; i < SC::C; i += G) smu[SC::RAD + i] = lv[SC::LV_RAD + i];
+    for (int i = lane; i < SC::MASKW; i += G) smu[SC::MASK + i] = lv[SC::LV_MASK + i];
+    if (lane == 0) smu[SC::META + META_GB] = lv[SC::LV_GB];
+    for (int i = lane; i < SC::LVC_WORDS; i += G) smu[SC::LVC + i] = lv[SC::LV_ELEN + i];
+    return (SC::J > 0 && lane < SC::J) ? lv[SC::LV_JOINT + kJointLevelWords * lane] : 0u;
+}
+
+// Auto-reset of a finished env: next level (its own, or drawn from the pool by the hash of seed,
+// global env index and episode), pose from the level, no accumulated impulses, counters.  Returns the
+// packed word of joint number `lane` of the level the env is on afterwards.
+template <class SC, int G>
+__device__ __noinline__ uint32_t reset_env(uint32_t *smu, const uint32_t *levels, int n_levels, int auto_reset, unsigned long long seed,
+                                           long long env_index, unsigned long long *counters, uint32_t jab) {
+    Group<G> g;
+    const int lane = g.lane;
+    const int episode = (int)smu[SC::META + META_EPISODE] + 1;
+    int level = (int)smu[SC::META + META_LEVEL];
+    g.sync();
+    if (auto_reset == 2) {
+        const unsigned long long h = mix64(seed + ((unsigned long long)env_index + 1ULL) * 0x9E3779B97F4A7C15ULL +
+                                           (unsigned long long)episode * 0xD1B54A32D192ED03ULL);
+        const int nl = (int)(h % (unsigned long long)n_levels);
+        if (nl != level) { level = nl; jab = load_level_consts<SC, G>(smu, levels + (size_t)nl * SC::LV_WORDS); }
+    }
+    const uint32_t *lv = levels + (size_t)level * SC::LV_WORDS;
+    for (int i = lane; i < 6 * SC::N; i += G) smu[body_word<SC>(i)] = lv[SC::LV_X + i];
+    if (SC::J > 0 && lane < SC::J) { smu[SC::JROW + kJointWords * lane + JR_ACCX] = 0u; smu[SC::JROW + kJointWords * lane + JR_ACCY] = 0u; smu[SC::JROW + kJointWords * lane + JR_ACCR] = 0u; }
+    for (int i = lane; i < (SC::NPAIRS + 3) / 4; i += G) smu[SC::WIDX + i] = 0xffffffffu;
+    if (lane == 0) {
+        smu[SC::META + META_STEP] = 0u; smu[SC::META + META_EPISODE] = (uint32_t)episode; smu[SC::META + META_LEVEL] = (uint32_t)level;
+        smu[SC::META + META_STATUS] = 0u; smu[SC::META + META_NWARM] = 0u;
+        atomicAdd(counters + 1, 1ULL);
+    }
+    g.sync();
+    return jab;
 }
 
 // packed work counters of a group to the global ones (lane 0)
@@ -364,70 +843,44 @@ __device__ __noinline__ void trace_clear(float *trace) {
     g.sync();
 }
 
-// A scene with more touching pairs than lanes: one lane walks the staged pairs in the scratch (in staging order), gives
-// each its level (into bits 19.. of its packed word) and its row slot (the word after the stage words), and fills the
-// table of level starts.  Returns the highest level.  bl: N bytes of shared memory.
-template <class SC>
-__device__ __noinline__ int place_crowded_impl(uint32_t *scr, uint8_t *lstart, uint8_t *bl, int nrec) {
-    uint32_t *stage = scr + SC::SCR_STAGE;
-    int cmax = 0;
-    for (int i = 0; i < SC::N; ++i) bl[i] = 0;
-    for (int L = 0; L <= nrec + 1; ++L) lstart[L] = 0;
-    for (int k = 0; k < nrec; ++k) {
-        uint32_t *w = stage + (size_t)k * kStageStride;
-        const uint32_t ab = w[S_AB];
-        const int a = ab & 31, b = (ab >> 5) & 31;
-        int lvl = 1;
-        if ((ab >> 26) & 1u) lvl = max(lvl, bl[a] + 1);
-        if ((ab >> 27) & 1u) lvl = max(lvl, bl[b] + 1);
-        if ((ab >> 26) & 1u) bl[a] = (uint8_t)lvl;
-        if ((ab >> 27) & 1u) bl[b] = (uint8_t)lvl;
-        w[S_AB] = ab | ((uint32_t)lvl << 19);
-        lstart[lvl] = (uint8_t)(lstart[lvl] + 1);
-        cmax = max(cmax, lvl);
-    }
-    // counts -> starts; a cursor per level in the spare word of stage entry level - 1
-    int run = 0;
-    for (int L = 1; L <= cmax; ++L) {
-        const int c = lstart[L];
-        lstart[L] = (uint8_t)run;
-        stage[(size_t)(L - 1) * kStageStride + kStageWords + 1] = (uint32_t)run;
-        run += c;
-    }
-    lstart[cmax + 1] = (uint8_t)run;
-    for (int k = 0; k < nrec; ++k) {
-        uint32_t *w = stage + (size_t)k * kStageStride;
-        const int lvl = (int)((w[S_AB] >> 19) & 127u);
-        uint32_t *cur = stage + (size_t)(lvl - 1) * kStageStride + kStageWords + 1;
-        w[kStageWords] = *cur;
-        *cur = *cur + 1u;
-    }
-    return cmax;
-}
-
-// ---------------------------------------------------------------- first half of a step: one scene per group of G lanes
+// ---------------------------------------------------------------- scene processing
 template <class SC, int G>
 struct Scene {
     static_assert(SC::J <= G && SC::T <= G && kMaxActions <= 2 * G, "one lane per joint / thruster");
-    static_assert(SC::NPAIRS < 255, "pair indices are bytes");
+    static_assert(2 * G <= 5 * SC::P4, "positional corrections reuse the world-frame vertex arrays");
     float *sm;            // this scene's shared-memory region
     uint32_t *smu;
     const uint16_t *ptab; // block-shared pair table
+    uint32_t *ovf;        // this group's overflow scratch in global memory
     const StepParams &prm;
     Group<G> g;
     int lane;
+    // state a lane keeps in registers from step to step
+    Rec rec;              // contact pair record number `lane` of the latest step (its accumulated impulses warm-start the next)
+    uint32_t jab;         // packed word of joint number `lane` (0 beyond the last joint)
     unsigned c_surv, c_rec, c_man;   // packed work counters: pp | pc << 16, cc | active pairs << 16, manifolds | env-steps << 16
 
-    __device__ __forceinline__ Scene(uint32_t *region, const uint16_t *pt, const StepParams &p)
-        : sm(reinterpret_cast<float *>(region)), smu(region), ptab(pt), prm(p), g() {
-        lane = g.lane; c_surv = 0u; c_rec = 0u; c_man = 0u;
+    __device__ __forceinline__ Scene(uint32_t *region, const uint16_t *pt, uint32_t *scratch, const StepParams &p)
+        : sm(reinterpret_cast<float *>(region)), smu(region), ptab(pt), ovf(scratch), prm(p), g() {
+        lane = g.lane; jab = 0u; c_surv = 0u; c_rec = 0u; c_man = 0u;
     }
 
     __device__ __forceinline__ uint8_t *surv() { return reinterpret_cast<uint8_t *>(smu + SC::SURV); }
     __device__ __forceinline__ uint8_t *widx() { return reinterpret_cast<uint8_t *>(smu + SC::WIDX); }
     __device__ __forceinline__ float4 &box4(int i) { return *reinterpret_cast<float4 *>(sm + SC::BOX + 4 * i); }
+    // this lane's word of per-lane field f
+    __device__ __forceinline__ float &lanef(int f) { return sm[SC::STG + f * G + lane]; }
+    // this lane's word of field f of its second record (lanes below G / 2 only)
+    __device__ __forceinline__ float &ovl(int f) { return sm[SC::STG + LF_COUNT * G + f * (G / 2) + lane]; }
     __device__ __forceinline__ ContactConsts contact_consts() const {
         ContactConsts cc; cc.slop = prm.slop; cc.rest_thr = prm.rest_thr; cc.alpha = prm.contact_alpha; cc.beta = prm.contact_beta; return cc;
+    }
+    // paper, "Reward": d_t of the dense signal kappa (d_t - d_{t+1})
+    __device__ __forceinline__ float green_blue_distance() const {
+        const uint32_t gb = smu[SC::META + META_GB];
+        const float4 pg = ld4(sm + SC::BPOS + 4 * (gb & 255u)), pb = ld4(sm + SC::BPOS + 4 * ((gb >> 8) & 255u));
+        const float dx = pb.x - pg.x, dy = pb.y - pg.y;
+        return sqrtf(dot2(dx, dy, dx, dy));
     }
     __device__ __forceinline__ void flush() {
         if (lane == 0) flush_counters(prm.counters, c_surv, c_rec, c_man);
@@ -526,7 +979,7 @@ struct Scene {
                 const float sep = dot2(nx, ny, cx, cy) - sm[SC::WOFF + 4 * a + k];
                 const float tx = -ny, ty = nx;
                 float s = dot2(tx, ty, cx - wx, cy - wy);
-                s = fmax_cmp(fmin_cmp(s, sm[SC::ELEN + 4 * a + k]), 0.0f);
+                s = fmax_cmp(fmin_cmp(s, sm[SC::LVC + 4 * a + k]), 0.0f);
                 const float px = __fmaf_rn(s, tx, wx), py = __fmaf_rn(s, ty, wy);
                 const float ex = cx - px, ey = cy - py;
                 const float d2 = dot2(ex, ey, ex, ey);
@@ -558,132 +1011,86 @@ struct Scene {
         return m.pen > 0.0f ? 1u : 0u;
     }
 
-    // ---- the first half of one environment step of env e (not frozen), whose meta head has been read already.
-    // tn_raw: lane 0's ticket for the group's next env, still in flight; on return next_e is that ticket for all lanes
-    // and next_head the env's meta head (if there is such an env), fetched while this env's pairs are tested.
-    __device__ __forceinline__ void prepare(int e, const MetaHead &head, unsigned tn_raw, unsigned &next_e, MetaHead &next_head) {
-        uint32_t *st = prm.state + (size_t)e * SC::ST_WORDS;
-        uint32_t *scr = prm.scratch + (size_t)e * SC::SCRATCH_WORDS;
-        const uint32_t *lv = prm.levels + (size_t)head.level * SC::LV_WORDS;
-        const int nprev = (int)head.nprev;
-        // Everything this step reads from memory is asked for here, in two volleys of loads that are all in flight before the
-        // first of them is used, so that the group waits for memory twice per step and not once per word: the state record
-        // (the same 16-byte groups as in shared memory), the level's constants, the body-frame vertices and normals (parked
-        // where their world-frame images will go), the action row, the previous step's warm list.
-        constexpr int KB = (2 * SC::N + G - 1) / G, KN = (SC::N + G - 1) / G, KV = (SC::P4 + G - 1) / G, KL = (SC::LVC_WORDS + G - 1) / G;
-        {
-            float4 body[KB];
-            uint32_t cim[KN], cii[KN], cfr[KN], cre[KN], cfl[KN], pvx[KV], pvy[KV], pnx[KV], pny[KV];
-#pragma unroll
-            for (int k = 0; k < KB; ++k) { const int i = lane + k * G; body[k] = (i < 2 * SC::N) ? __ldcg(reinterpret_cast<const float4 *>(st + SC::ST_POS) + i) : make_float4(0.0f, 0.0f, 0.0f, 0.0f); }
-#pragma unroll
-            for (int k = 0; k < KN; ++k) {
-                const int i = lane + k * G; const bool in = i < SC::N;
-                cim[k] = in ? __ldg(lv + SC::LV_IM + i) : 0u; cii[k] = in ? __ldg(lv + SC::LV_II + i) : 0u; cfr[k] = in ? __ldg(lv + SC::LV_FR + i) : 0u;
-                cre[k] = in ? __ldg(lv + SC::LV_RE + i) : 0u; cfl[k] = in ? __ldg(lv + SC::LV_FLAGS + i) : 0u;
-            }
-#pragma unroll
-            for (int k = 0; k < KV; ++k) {
-                const int v = lane + k * G; const bool in = v < SC::P4;
-                pvx[k] = in ? __ldg(lv + SC::LV_PVX + v) : 0u; pvy[k] = in ? __ldg(lv + SC::LV_PVY + v) : 0u;
-                pnx[k] = in ? __ldg(lv + SC::LV_PNX + v) : 0u; pny[k] = in ? __ldg(lv + SC::LV_PNY + v) : 0u;
-            }
-#pragma unroll
-            for (int k = 0; k < KB; ++k) { const int i = lane + k * G; if (i < 2 * SC::N) reinterpret_cast<float4 *>(sm + SC::BPOS)[i] = body[k]; }
-#pragma unroll
-            for (int k = 0; k < KN; ++k) {
-                const int i = lane + k * G;
-                if (i < SC::N) { smu[SC::BIM + i] = cim[k]; smu[SC::BII + i] = cii[k]; smu[SC::BFR + i] = cfr[k]; smu[SC::BRE + i] = cre[k]; smu[SC::BFL + i] = cfl[k]; }
-            }
-#pragma unroll
-            for (int k = 0; k < KV; ++k) {
-                const int v = lane + k * G;
-                if (v < SC::P4) { smu[SC::WVX + v] = pvx[k]; smu[SC::WVY + v] = pvy[k]; smu[SC::WNX + v] = pnx[k]; smu[SC::WNY + v] = pny[k]; }
-            }
+    // ---- one visit of this lane's contact pair record.  MODE 0: warm start, 1: solver iteration, 2: positional correction
+    template <int MODE>
+    __device__ __forceinline__ void visit_pair() {
+        const uint32_t ab = rec.ab;
+        const int a = ab & 31, b = (ab >> 5) & 31;
+        const unsigned amask = (ab >> 10) & 3u;
+        const bool dyn_a = (ab >> 26) & 1u, dyn_b = (ab >> 27) & 1u;
+        if (MODE == 2) {
+            correct_pair(sm + SC::BPOS, a, b, amask, dyn_a, dyn_b, rec.nx, rec.ny, rec.ma, rec.mb,
+                         sm[SC::WVX + lane], sm[SC::WVX + G + lane]);
+            return;
         }
-        uint32_t gb;
-        uint32_t wpair = 255u;
-        float4 wacc = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
-        float jacc0 = 0.0f, jacc1 = 0.0f, jacc2 = 0.0f;
-        {
-            uint32_t lvc[KL], rad = 0u, msk = 0u, act0 = 0u, act1 = 0u;
-#pragma unroll
-            for (int k = 0; k < KL; ++k) { const int i = lane + k * G; lvc[k] = (i < SC::LVC_WORDS) ? __ldg(lv + SC::LV_ELEN + i) : 0u; }
-            static_assert(SC::C <= G && SC::MASKW <= G, "one lane per circle / mask word");
-            if (lane < SC::C) rad = __ldg(lv + SC::LV_RAD + lane);
-            if (lane < SC::MASKW) msk = __ldg(lv + SC::LV_MASK + lane);
-            const uint32_t *act_row = reinterpret_cast<const uint32_t *>(prm.actions) + (size_t)e * prm.n_actions;
-            if (lane < prm.n_actions) act0 = __ldg(act_row + lane);
-            if (G < kMaxActions && lane + G < prm.n_actions) act1 = __ldg(act_row + lane + G);
-            gb = __ldg(lv + SC::LV_GB);
-            // the previous step's accumulated impulses: entry k stays with lane k (entries beyond the lanes are read from the
-            // state record when needed); the byte table maps a pair to its entry
-            if (lane < nprev) {
-                const uint32_t *wr = st + SC::ST_WARM + kWarmWords * lane;
-                wpair = __ldcg(wr);
-                wacc = make_float4(__uint_as_float(__ldcg(wr + 1)), __uint_as_float(__ldcg(wr + 2)), __uint_as_float(__ldcg(wr + 3)), __uint_as_float(__ldcg(wr + 4)));
-            }
-            if (SC::J > 0 && lane < SC::J) {
-                jacc0 = __uint_as_float(__ldcg(st + SC::ST_JACC + 3 * lane)); jacc1 = __uint_as_float(__ldcg(st + SC::ST_JACC + 3 * lane + 1));
-                jacc2 = __uint_as_float(__ldcg(st + SC::ST_JACC + 3 * lane + 2));
-            }
-#pragma unroll
-            for (int k = 0; k < KL; ++k) { const int i = lane + k * G; if (i < SC::LVC_WORDS) smu[SC::LVC + i] = lvc[k]; }
-            if (lane < SC::C) smu[SC::RAD + lane] = rad;
-            if (lane < SC::MASKW) smu[SC::MASK + lane] = msk;
-            if (lane < prm.n_actions) smu[SC::ACT + lane] = act0;
-            if (G < kMaxActions && lane + G < prm.n_actions) smu[SC::ACT + lane + G] = act1;
+        const float4 va4 = ld4(sm + SC::BVEL + 4 * a), vb4 = ld4(sm + SC::BVEL + 4 * b);
+        float vax = va4.x, vay = va4.y, wa = va4.z, vbx = vb4.x, vby = vb4.y, wb = vb4.z;
+        if (amask & 1u)
+            manifold_rows<MODE>(rec.nx, rec.ny, rec.mu, rec.ma, rec.mb, rec.ia, rec.ib, rec.rna, rec.rnb, rec.rta, rec.rtb,
+                                rec.massn, rec.masst, rec.target, rec.accn, rec.acct, vax, vay, wa, vbx, vby, wb);
+        if (amask & 2u) {
+            float accn = lanef(LF_ACC2N), acct = lanef(LF_ACC2T);
+            manifold_rows<MODE>(rec.nx, rec.ny, rec.mu, rec.ma, rec.mb, rec.ia, rec.ib, lanef(M2_RNA), lanef(M2_RNB), lanef(M2_RTA),
+                                lanef(M2_RTB), lanef(M2_MASSN), lanef(M2_MASST), lanef(M2_TARGET), accn, acct, vax, vay, wa, vbx, vby, wb);
+            if (MODE == 1) { lanef(LF_ACC2N) = accn; lanef(LF_ACC2T) = acct; }
         }
-        for (int i = lane; i < (SC::NPAIRS + 3) / 4; i += G) smu[SC::WIDX + i] = 0xffffffffu;
-        g.sync();
-        if (wpair != 255u) widx()[wpair] = (uint8_t)lane;
-        for (int k = G + lane; k < nprev; k += G) widx()[__ldcg(st + SC::ST_WARM + kWarmWords * k)] = (uint8_t)k;
-        const uint32_t jab = (SC::J > 0 && lane < SC::J) ? smu[SC::LVC_JOINT + kJointLevelWords * lane] : 0u;
-        // dense reward: the first green and the first blue shape, and their distance before the step
-        float d0 = 0.0f;
-        if (prm.dense_kappa != 0.0f && ((gb >> 16) & 1u)) {
-            const float4 pg = ld4(sm + SC::BPOS + 4 * (gb & 255u)), pb = ld4(sm + SC::BPOS + 4 * ((gb >> 8) & 255u));
-            const float dx = pb.x - pg.x, dy = pb.y - pg.y;
-            d0 = sqrtf(dot2(dx, dy, dx, dy));
+        if (dyn_a) st4(sm + SC::BVEL + 4 * a, vax, vay, wa);
+        if (dyn_b) st4(sm + SC::BVEL + 4 * b, vbx, vby, wb);
+    }
+    // records of one level touch disjoint movable bodies; levels in order keep the record order
+    template <int MODE>
+    __device__ __forceinline__ void sweep_pairs(int cmax, int clevel, int clevel2) {
+#pragma unroll 1
+        for (int lvl = 1; lvl <= cmax; ++lvl) {
+            if (clevel == lvl) visit_pair<MODE>();
+            if (clevel2 == lvl) visit_second<SC, G, MODE>(sm);
+            g.sync();
         }
+    }
+
+    // ---- one environment step
+    __device__ __forceinline__ void step(int e, int s) {
+        // frozen env: reports done, nothing else
+        if (smu[SC::META + META_STATUS] & 1u) {
+            if (lane == 0) { prm.reward[(size_t)s * prm.n_envs + e] = 0.0f; prm.done[(size_t)s * prm.n_envs + e] = 1; }
+            return;
+        }
+        const uint32_t *lv = prm.levels + (size_t)smu[SC::META + META_LEVEL] * SC::LV_WORDS;
+        // dense reward: distance between the first green and the first blue shape before the step
+        if (prm.dense_kappa != 0.0f && lane == 0) sm[SC::META + META_D0] = green_blue_distance();
+        // actions of this step
+        const float *act_row = prm.actions + ((size_t)(s / prm.frame_skip) * prm.n_envs + e) * prm.n_actions;
+        if (lane < prm.n_actions) sm[SC::ACT + lane] = act_row[lane];
+        if (G < kMaxActions && lane + G < prm.n_actions) sm[SC::ACT + lane + G] = act_row[lane + G];
         // gravity, rotation, circle boxes
-        unsigned active_mask = 0u;
-        for (int base = 0; base < SC::N; base += G) {
-            const int i = base + lane;
-            bool act_i = false;
-            if (i < SC::N) {
-                const uint32_t fl = smu[SC::BFL + i];
-                act_i = (fl & F_ACTIVE) != 0u;
-                if (act_i && (fl & F_DYNAMIC)) sm[SC::BVEL + 4 * i + 1] = sm[SC::BVEL + 4 * i + 1] + prm.gdt;
-                float c, sn;
-                sincos_spec(sm[SC::BPOS + 4 * i + 2], c, sn);
-                sm[SC::BC + i] = c; sm[SC::BS + i] = sn;
-                if (i >= SC::P) {
-                    const float r = sm[SC::RAD + (i - SC::P)], x = sm[SC::BPOS + 4 * i], y = sm[SC::BPOS + 4 * i + 1];
-                    box4(i) = make_float4(x - r, y - r, x + r, y + r);
-                }
+        for (int i = lane; i < SC::N; i += G) {
+            const uint32_t fl = smu[SC::BFL + i];
+            if ((fl & F_ACTIVE) && (fl & F_DYNAMIC)) sm[SC::BVEL + 4 * i + 1] = sm[SC::BVEL + 4 * i + 1] + prm.gdt;
+            float c, sn;
+            sincos_spec(sm[SC::BPOS + 4 * i + 2], c, sn);
+            sm[SC::BC + i] = c; sm[SC::BS + i] = sn;
+            if (i >= SC::P) {
+                const float r = sm[SC::RAD + (i - SC::P)], x = sm[SC::BPOS + 4 * i], y = sm[SC::BPOS + 4 * i + 1];
+                box4(i) = make_float4(x - r, y - r, x + r, y + r);
             }
-            active_mask |= g.ballot(act_i) << base;
         }
         g.sync();
-        // world-frame polygon vertices, normals, face offsets (each lane turns the body-frame values it parked)
+        // world-frame polygon vertices, normals, face offsets
         for (int v = lane; v < SC::P4; v += G) {
             const int i = v >> 2, k = v & 3;
             if (k < (int)flag_nverts(smu[SC::BFL + i])) {
                 const float c = sm[SC::BC + i], sn = sm[SC::BS + i];
                 float rx, ry, nx, ny;
-                rot2(c, sn, sm[SC::WVX + v], sm[SC::WVY + v], rx, ry);
-                rot2(c, sn, sm[SC::WNX + v], sm[SC::WNY + v], nx, ny);
+                rot2(c, sn, __uint_as_float(lv[SC::LV_PVX + v]), __uint_as_float(lv[SC::LV_PVY + v]), rx, ry);
+                rot2(c, sn, __uint_as_float(lv[SC::LV_PNX + v]), __uint_as_float(lv[SC::LV_PNY + v]), nx, ny);
                 const float wx = rx + sm[SC::BPOS + 4 * i], wy = ry + sm[SC::BPOS + 4 * i + 1];
                 sm[SC::WVX + v] = wx; sm[SC::WVY + v] = wy; sm[SC::WNX + v] = nx; sm[SC::WNY + v] = ny;
                 sm[SC::WOFF + v] = dot2(nx, ny, wx, wy);
             }
         }
         // this lane's joint: "on" bit and level come with the level record
-        const bool jon = ((jab >> 24) & 1u) != 0u;
-        const int jlevel = jon ? (int)((jab >> 25) & 7u) : 0;
+        const int jlevel = ((jab >> 24) & 1u) ? (int)((jab >> 25) & 7u) : 0;
         const int jmax = (SC::J > 0) ? g.max_int(jlevel) : 0;
-        const uint32_t *jl = smu + SC::LVC_JOINT + kJointLevelWords * (lane < SC::J ? lane : 0);
         g.sync();
         // polygon boxes
         for (int i = lane; i < SC::P; i += G) {
@@ -698,30 +1105,11 @@ struct Scene {
             }
             box4(i) = make_float4(x0, y0, x1, y1);
         }
-        // motors in joint order: joints of one level touch disjoint movable shapes, levels in order keep the joint order
-        if (SC::J > 0) {
-#pragma unroll 1
-            for (int lvl = 1; lvl <= jmax; ++lvl) {
-                if (jlevel == lvl) {
-                    const int a = jab & 255, b = (jab >> 8) & 255;
-                    const float av = sm[SC::ACT + ((jab >> 16) & 255)];
-                    // paper, "Action Space": continuous in [-1, 1], or multi-discrete codes 0 off, 1 forwards, 2 backwards at full power
-                    const float A = prm.discrete ? (__float_as_int(av) == 1 ? 1.0f : (__float_as_int(av) == 2 ? -1.0f : 0.0f))
-                                                 : fmax_cmp(fmin_cmp(av, 1.0f), -1.0f);
-                    const float speed = __uint_as_float(jl[5]), power = __uint_as_float(jl[6]);
-                    const float wa = sm[SC::BVEL + 4 * a + 2], wb = sm[SC::BVEL + 4 * b + 2];
-                    const float arg = __fmaf_rn(-speed, A, wa - wb) * prm.motor_rho;
-                    const float jr_ = power * tanh_spec(arg);
-                    if ((jab >> 29) & 1u) sm[SC::BVEL + 4 * a + 2] = __fmaf_rn(-jr_, sm[SC::BII + a], wa);
-                    if ((jab >> 30) & 1u) sm[SC::BVEL + 4 * b + 2] = __fmaf_rn(jr_, sm[SC::BII + b], wb);
-                }
-                g.sync();
-            }
-        }
-        // thrusters in thruster order, by level in the same way
+        // motors (joint order), thrusters (thruster order)
+        sweep_joints<SC, G, 3>(sm, jab, lane, jlevel, jmax, prm.motor_rho, prm.discrete);
         if (SC::T > 0) {
             int tl = 0; uint32_t tp = 0u;
-            const uint32_t *th = smu + SC::LVC_THR + 8 * (lane < SC::T ? lane : 0);
+            const uint32_t *th = smu + SC::LVC + (SC::LV_THR - SC::LV_ELEN) + 8 * lane;
             if (lane < SC::T) { tp = th[0]; if ((tp >> 16) & 1u) tl = (tp >> 17) & 7u; }
             const int tmax = g.max_int(tl);
 #pragma unroll 1
@@ -745,22 +1133,20 @@ struct Scene {
                 g.sync();
             }
         }
-        g.sync();       // boxes and velocities are final
-        // joint pre-step (poses only; velocities are not read): the row goes to the env's scratch
+        // joint pre-step (poses only; velocities are not read): the row goes to shared memory
         if (SC::J > 0 && lane < SC::J) {
-            float4 q[6];
-#pragma unroll
-            for (int f = 0; f < 6; ++f) q[f] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
-            float accx = jacc0, accy = jacc1, accr = jacc2;
-            if (!jon || !prm.warm_start) { accx = 0.0f; accy = 0.0f; accr = 0.0f; }
+            float *jr = sm + SC::JROW + kJointWords * lane;
+            if (!((jab >> 24) & 1u) || !prm.warm_start) { jr[JR_ACCX] = 0.0f; jr[JR_ACCY] = 0.0f; jr[JR_ACCR] = 0.0f; }
             int ang = 0;
             float kr = 0.0f, bias_r = 0.0f;
-            if (jon) {
+            if ((jab >> 24) & 1u) {
                 const int a = jab & 255, b = (jab >> 8) & 255;
+                const uint32_t *jl = smu + SC::LVC + (SC::LV_JOINT - SC::LV_ELEN) + kJointLevelWords * lane;
                 float rax, ray, rbx, rby;
                 rot2(sm[SC::BC + a], sm[SC::BS + a], __uint_as_float(jl[1]), __uint_as_float(jl[2]), rax, ray);
                 rot2(sm[SC::BC + b], sm[SC::BS + b], __uint_as_float(jl[3]), __uint_as_float(jl[4]), rbx, rby);
                 const float ma = sm[SC::BIM + a], mb = sm[SC::BIM + b], ia = sm[SC::BII + a], ib = sm[SC::BII + b];
+                jr[JR_MA] = ma; jr[JR_MB] = mb; jr[JR_IA] = ia; jr[JR_IB] = ib;
                 const float gx = (sm[SC::BPOS + 4 * b] + rbx) - (sm[SC::BPOS + 4 * a] + rax), gy = (sm[SC::BPOS + 4 * b + 1] + rby) - (sm[SC::BPOS + 4 * a + 1] + ray);
                 const float msum = ma + mb;
                 float k11 = msum; k11 = __fmaf_rn(ia * ray, ray, k11); k11 = __fmaf_rn(ib * rby, rby, k11);
@@ -768,11 +1154,11 @@ struct Scene {
                 float k12 = -((ia * rax) * ray); k12 = __fmaf_rn(-(ib * rbx), rby, k12);
                 const float det = __fmaf_rn(k11, k22, -(k12 * k12));
                 const float inv_det = 1.0f / det;
+                jr[JR_RAX] = rax; jr[JR_RAY] = ray; jr[JR_RBX] = rbx; jr[JR_RBY] = rby;
+                jr[JR_I11] = k22 * inv_det; jr[JR_I22] = k11 * inv_det; jr[JR_I12] = -(k12 * inv_det);
+                jr[JR_BX] = prm.joint_alpha * gx; jr[JR_BY] = prm.joint_alpha * gy;
                 const float share = prm.joint_beta / msum;
-                q[0] = make_float4(rax, ray, rbx, rby);
-                q[1] = make_float4(k22 * inv_det, -(k12 * inv_det), k11 * inv_det, 0.0f);
-                q[2] = make_float4(prm.joint_alpha * gx, prm.joint_alpha * gy, share * gx, share * gy);
-                q[3] = make_float4(ma, mb, ia, ib);
+                jr[JR_CX] = share * gx; jr[JR_CY] = share * gy;
                 // angular row from the relative rotation at the start of the step
                 const float isum = ia + ib;
                 const uint32_t kind = jl[10];
@@ -786,14 +1172,10 @@ struct Scene {
                     }
                 }
             }
-            if (ang != 1) accr = 0.0f;
-            q[1].w = __uint_as_float(jab);
-            q[4] = make_float4(accx, accy, 0.0f, 0.0f);
-            q[5] = make_float4(__int_as_float(ang), kr, bias_r, accr);
-            float4 *jr = reinterpret_cast<float4 *>(scr + SC::SCR_JROW + kJointWords * lane);
-#pragma unroll
-            for (int f = 0; f < 6; ++f) jr[f] = q[f];
+            if (ang != 1) jr[JR_ACCR] = 0.0f;
+            jr[JR_ANG] = __int_as_float(ang); jr[JR_KR] = kr; jr[JR_BIASR] = bias_r;
         }
+        g.sync();
 
         // bounding-box test over all pairs -> compact list of surviving pairs, in pair order
         int nsurv = 0, ns_pp, ns_pc;
@@ -821,12 +1203,8 @@ struct Scene {
         g.sync();
         c_surv += (unsigned)ns_pp | ((unsigned)(ns_pc - ns_pp) << 16);
         c_rec += (unsigned)(nsurv - ns_pc);
-        // the group's next env: its ticket has arrived by now; its meta head will have by the end of this env
-        next_e = g.shflu(tn_raw, 0);
-        if (next_e < (unsigned)prm.n_envs) next_head = load_meta_head(prm.state + (size_t)next_e * SC::ST_WORDS + SC::ST_META);
 
-        // narrowphase: survivors of one kind at a time; pairs with an active manifold are staged in pair order, the
-        // first G of them in shared memory, later ones in the staging area of the env's scratch
+        // narrowphase: survivors of one kind at a time; active pairs are staged in pair order
         int nrec = 0;
         bool t_gb = false, t_gr = false;
         float *trace = prm.trace ? prm.trace + (size_t)e * SC::NSLOTS * 6 : nullptr;
@@ -863,15 +1241,21 @@ struct Scene {
                                         (((fa & F_DYNAMIC) ? 1u : 0u) << 26) | (((fb & F_DYNAMIC) ? 1u : 0u) << 27);
                     const float nx = (act & 1u) ? m[0].nx : m[1].nx, ny = (act & 1u) ? m[0].ny : m[1].ny;
                     if (k < G) {
-                        float *sg = sm + SC::STG + k;
-                        sg[S_AB * G] = __uint_as_float(ab); sg[S_NX * G] = nx; sg[S_NY * G] = ny;
-                        sg[S_PX0 * G] = m[0].px; sg[S_PY0 * G] = m[0].py; sg[S_PEN0 * G] = m[0].pen;
-                        sg[S_PX1 * G] = m[1].px; sg[S_PY1 * G] = m[1].py; sg[S_PEN1 * G] = m[1].pen;
+                        float *st = sm + SC::STG + k;
+                        st[S_AB * G] = __uint_as_float(ab); st[S_NX * G] = nx; st[S_NY * G] = ny;
+                        st[S_PX0 * G] = m[0].px; st[S_PY0 * G] = m[0].py; st[S_PEN0 * G] = m[0].pen;
+                        st[S_PX1 * G] = m[1].px; st[S_PY1 * G] = m[1].py; st[S_PEN1 * G] = m[1].pen;
+                    } else if (k < G + G / 2) {
+                        float *st = sm + SC::STG + LF_COUNT * G + (k - G);
+                        constexpr int H = G / 2;
+                        st[ovs(S_AB) * H] = __uint_as_float(ab); st[ovs(S_NX) * H] = nx; st[ovs(S_NY) * H] = ny;
+                        st[ovs(S_PX0) * H] = m[0].px; st[ovs(S_PY0) * H] = m[0].py; st[ovs(S_PEN0) * H] = m[0].pen;
+                        st[ovs(S_PX1) * H] = m[1].px; st[ovs(S_PY1) * H] = m[1].py; st[ovs(S_PEN1) * H] = m[1].pen;
                     } else {
-                        uint32_t *sg = scr + SC::SCR_STAGE + (size_t)k * kStageStride;
-                        sg[S_AB] = ab; sg[S_NX] = __float_as_uint(nx); sg[S_NY] = __float_as_uint(ny);
-                        sg[S_PX0] = __float_as_uint(m[0].px); sg[S_PY0] = __float_as_uint(m[0].py); sg[S_PEN0] = __float_as_uint(m[0].pen);
-                        sg[S_PX1] = __float_as_uint(m[1].px); sg[S_PY1] = __float_as_uint(m[1].py); sg[S_PEN1] = __float_as_uint(m[1].pen);
+                        uint32_t *st = ovf + (size_t)k * kRecWords;
+                        st[S_AB] = ab; st[S_NX] = __float_as_uint(nx); st[S_NY] = __float_as_uint(ny);
+                        st[S_PX0] = __float_as_uint(m[0].px); st[S_PY0] = __float_as_uint(m[0].py); st[S_PEN0] = __float_as_uint(m[0].pen);
+                        st[S_PX1] = __float_as_uint(m[1].px); st[S_PY1] = __float_as_uint(m[1].py); st[S_PEN1] = __float_as_uint(m[1].pen);
                     }
                 }
                 nrec += __popc(bal);
@@ -881,167 +1265,295 @@ struct Scene {
         g.sync();
         c_rec += (unsigned)nrec << 16;
 
-        // Levels of the touching pairs (canonical order = staging order): one more than the highest level of an earlier pair
-        // that shares a movable body.  Then every pair gets its row slot: rows are sorted by level, in staging order within
-        // a level, and a byte table in the scratch says where each level starts.
-        uint8_t *lstart = reinterpret_cast<uint8_t *>(scr + SC::SCR_LSTART);
-        const bool crowded = nrec > G;      // more touching pairs than lanes: rare, handled by one lane through the scratch
-        int cmax = 0, lvl = 0, slot = 0;
-        uint32_t ab = 0u;
-        if (!crowded) {
-            const bool mine = lane < nrec;
-            if (mine) ab = __float_as_uint(sm[SC::STG + S_AB * G + lane]);
-            const int a = ab & 31, b = (ab >> 5) & 31;
-            // every movable body collects the set of pairs that touch it; a pair's conflicts are the earlier members of its
-            // bodies' sets; level r goes to the pairs whose conflicts all have a level already, round after round
-            uint32_t *touch = smu + SC::SURV;            // the survivor list is no longer needed
-            for (int i = lane; i < SC::N; i += G) touch[i] = 0u;
-            g.sync();
-            const bool da = (ab >> 26) & 1u, db = (ab >> 27) & 1u;
-            if (mine && da) atomicOr(touch + a, 1u << lane);
-            if (mine && db) atomicOr(touch + b, 1u << lane);
-            g.sync();
-            const unsigned conflicts = ((da ? touch[a] : 0u) | (db ? touch[b] : 0u)) & g.lanes_below();
-            const unsigned all = g.ballot(mine);
-            unsigned assigned = 0u;
-#pragma unroll 1
-            for (int r = 1; assigned != all; ++r) {
-                const bool ready = mine && lvl == 0 && (conflicts & ~assigned) == 0u;
-                if (ready) lvl = r;
-                assigned |= g.ballot(ready);
-            }
-            cmax = g.max_int(lvl);
-            int run = 0;
-#pragma unroll 1
-            for (int L = 1; L <= cmax; ++L) {
-                const unsigned bal = g.ballot(lvl == L);
-                if (lvl == L) slot = run + __popc(bal & g.lanes_below());
-                if (lane == 0) lstart[L] = (uint8_t)run;
-                run += __popc(bal);
-            }
-            if (lane == 0) lstart[cmax + 1] = (uint8_t)run;
+        const bool overflow = nrec > G + G / 2;
+        int cmax = 0, clevel = 0, clevel2 = 0;
+        if (overflow) {
+            cmax = slow_solve<SC, G>(sm, ovf, nrec, jab, jlevel, jmax, prm.solver_iters, prm.warm_start, prm.motor_rho,
+                                     rec.accn, rec.acct, contact_consts());
         } else {
-            // the pairs staged in shared memory join the others in the scratch
-            {
-                uint32_t *sg = scr + SC::SCR_STAGE + (size_t)lane * kStageStride;
-#pragma unroll
-                for (int f = 0; f < kStageWords; ++f) sg[f] = smu[SC::STG + f * G + lane];
+            const ContactConsts cc = contact_consts();
+            const bool two = nrec > G;      // some lanes get a second record
+            if (two) {
+                if (lane == 0) cmax = levels_by_one_lane<SC, G>(smu, ovf, nrec);
+                g.sync();
             }
-            g.sync();
-            if (lane == 0) cmax = place_crowded_impl<SC>(scr, lstart, reinterpret_cast<uint8_t *>(smu + SC::SURV), nrec);
-            g.sync();
-            cmax = g.shfl(cmax, 0);
+            // every staged pair becomes a record in its own lane: accumulated impulses of the same pair in the
+            // previous step come from wherever its record was then
+            const bool mine = lane < nrec;
+            uint32_t ab = 0u;
+            float nx = 0.0f, ny = 0.0f, pt[6] = { 0.0f, 0.0f, 0.0f, 0.0f, 0.0f, 0.0f };
+            float w[4];
+            {
+                int wi = 255;
+                if (mine) {
+                    ab = __float_as_uint(lanef(S_AB)); wi = widx()[(ab >> 12) & 127];
+                    nx = lanef(S_NX); ny = lanef(S_NY);
+                    pt[0] = lanef(S_PX0); pt[1] = lanef(S_PY0); pt[2] = lanef(S_PEN0); pt[3] = lanef(S_PX1); pt[4] = lanef(S_PY1); pt[5] = lanef(S_PEN1);
+                }
+                const float old_n = rec.accn, old_t = rec.acct;
+                warm_lookup<SC, G>(g, sm, ovf, wi, old_n, old_t, prm.warm_start, w);
+                if (two) second_lookup<SC, G>(sm, ovf, nrec, old_n, old_t, prm.warm_start);
+            }
+            g.sync();     // every lane has read the fields it needs from other lanes before they are rewritten
+            const int a = ab & 31, b = (ab >> 5) & 31;
+            const unsigned amask = (ab >> 10) & 3u;
+            rec.ab = ab; rec.nx = nx; rec.ny = ny;
+            rec.ma = sm[SC::BIM + a]; rec.mb = sm[SC::BIM + b]; rec.ia = sm[SC::BII + a]; rec.ib = sm[SC::BII + b];
+            {
+                const float fra = sm[SC::BFR + a], frb = sm[SC::BFR + b];
+                rec.mu = sqrtf(__fmaf_rn(fra, fra, frb * frb));
+            }
+            const float er = fmin_cmp(sm[SC::BRE + a], sm[SC::BRE + b]);
+            float corr0 = 0.0f, corr1 = 0.0f;
+            rec.rna = 0.0f; rec.rnb = 0.0f; rec.rta = 0.0f; rec.rtb = 0.0f; rec.massn = 0.0f; rec.masst = 0.0f; rec.target = 0.0f;
+            rec.accn = 0.0f; rec.acct = 0.0f;
+            if (amask & 1u) {
+                prestep_manifold<SC>(a, b, nx, ny, rec.ma, rec.mb, rec.ia, rec.ib, pt[0], pt[1], pt[2], er, sm, cc,
+                                     rec.rna, rec.rnb, rec.rta, rec.rtb, rec.massn, rec.masst, rec.target, corr0);
+                rec.accn = w[0]; rec.acct = w[1];
+            }
+            float acc2n = 0.0f, acc2t = 0.0f;
+            if (amask & 2u) {
+                float rna, rnb, rta, rtb, massn, masst, target;
+                prestep_manifold<SC>(a, b, nx, ny, rec.ma, rec.mb, rec.ia, rec.ib, pt[3], pt[4], pt[5], er, sm, cc,
+                                     rna, rnb, rta, rtb, massn, masst, target, corr1);
+                lanef(M2_RNA) = rna; lanef(M2_RNB) = rnb; lanef(M2_RTA) = rta; lanef(M2_RTB) = rtb;
+                lanef(M2_MASSN) = massn; lanef(M2_MASST) = masst; lanef(M2_TARGET) = target;
+                acc2n = w[2]; acc2t = w[3];
+            }
+            lanef(LF_ACC2N) = acc2n; lanef(LF_ACC2T) = acc2t;
+            sm[SC::WVX + lane] = corr0; sm[SC::WVX + G + lane] = corr1;
+            if (two) {
+                const unsigned r2 = second_build<SC, G>(sm, nrec, cc);     // level | active manifolds << 8
+                clevel2 = (int)(r2 & 127u);
+                clevel = (int)((ab >> 19) & 127u);
+                cmax = g.shfl(cmax, 0);
+                c_man += (unsigned)g.sum_int((int)(r2 >> 8));
+            } else {
+                // levels of the records (canonical order = record order): one more than the highest level of an
+                // earlier record that shares a movable body.  Every movable body collects the set of records that
+                // touch it; a record's conflicts are the earlier members of its bodies' sets; then level r goes to
+                // the records whose conflicts all have a level already, round after round.
+                uint32_t *touch = smu + SC::SURV;            // the survivor list is no longer needed
+                for (int i = lane; i < SC::N; i += G) touch[i] = 0u;
+                g.sync();
+                const bool da = (ab >> 26) & 1u, db = (ab >> 27) & 1u;
+                if (mine && da) atomicOr(touch + a, 1u << lane);
+                if (mine && db) atomicOr(touch + b, 1u << lane);
+                g.sync();
+                const unsigned conflicts = ((da ? touch[a] : 0u) | (db ? touch[b] : 0u)) & g.lanes_below();
+                const unsigned all = g.ballot(mine);
+                unsigned assigned = 0u;
+                int lvl = 0;
+#pragma unroll 1
+                for (int r = 1; assigned != all; ++r) {
+                    const bool ready = mine && lvl == 0 && (conflicts & ~assigned) == 0u;
+                    if (ready) lvl = r;
+                    assigned |= g.ballot(ready);
+                }
+                clevel = lvl;
+                cmax = g.max_int(lvl);
+            }
+            c_man += (unsigned)(__popc(g.ballot(amask & 1u)) + __popc(g.ballot(amask & 2u)));
+            // warm start: contacts, then joints
+            sweep_pairs<0>(cmax, clevel, clevel2);
+            sweep_joints<SC, G, 0>(sm, jab, lane, jlevel, jmax, prm.motor_rho);
+            // solver iterations: joints, then contacts
+#pragma unroll 1
+            for (int it = 0; it < prm.solver_iters; ++it) {
+                sweep_joints<SC, G, 1>(sm, jab, lane, jlevel, jmax, prm.motor_rho);
+                sweep_pairs<1>(cmax, clevel, clevel2);
+            }
+        }
+        // Euler step with the solved velocities
+        for (int i = lane; i < SC::N; i += G) {
+            if (smu[SC::BFL + i] & F_ACTIVE) {
+                const float4 p4 = ld4(sm + SC::BPOS + 4 * i), v4 = ld4(sm + SC::BVEL + 4 * i);
+                st4(sm + SC::BPOS + 4 * i, __fmaf_rn(prm.dt, v4.x, p4.x), __fmaf_rn(prm.dt, v4.y, p4.y), __fmaf_rn(prm.dt, v4.z, p4.z));
+            }
+        }
+        g.sync();
+        if (overflow) slow_correct<SC, G>(sm, ovf, nrec, cmax);
+        else sweep_pairs<2>(cmax, clevel, clevel2);
+        sweep_joints<SC, G, 2>(sm, jab, lane, jlevel, jmax, prm.motor_rho);
+        bool finite = true;
+        for (int i = lane; i < SC::N; i += G) {
+            const float4 p4 = ld4(sm + SC::BPOS + 4 * i), v4 = ld4(sm + SC::BVEL + 4 * i);
+            finite = finite && finite_bits(p4.x) && finite_bits(p4.y) && finite_bits(p4.z) && finite_bits(v4.x) && finite_bits(v4.y) && finite_bits(v4.z);
+        }
+        finite = !g.any(!finite);
+
+        // where the pairs of this step keep their accumulated impulses for the next one
+        for (int i = lane; i < (SC::NPAIRS + 3) / 4; i += G) smu[SC::WIDX + i] = 0xffffffffu;
+        const int step_count = (int)smu[SC::META + META_STEP] + 1;
+        g.sync();
+        if (overflow) {
+            c_man += (unsigned)slow_finish<SC, G>(sm, ovf, nrec);
+            // the first G + G / 2 pairs go back to their lanes
+            const uint32_t *wr = ovf + SC::SCRATCH_WARM + (size_t)lane * kWarmWords, *wr2 = wr + (size_t)G * kWarmWords;
+            rec.ab = wr[0] << 12;
+            rec.accn = __uint_as_float(wr[1]); rec.acct = __uint_as_float(wr[2]);
+            lanef(LF_ACC2N) = __uint_as_float(wr[3]); lanef(LF_ACC2T) = __uint_as_float(wr[4]);
+            if (lane < G / 2) {
+                ovl(R_AB) = __uint_as_float(wr2[0] << 12);
+                ovl(OV_ACC0N) = __uint_as_float(wr2[1]); ovl(OV_ACC0T) = __uint_as_float(wr2[2]);
+                ovl(OV_ACC1N) = __uint_as_float(wr2[3]); ovl(OV_ACC1T) = __uint_as_float(wr2[4]);
+            }
+        } else {
+            if (lane < nrec) widx()[(rec.ab >> 12) & 127] = (uint8_t)lane;
+            if (clevel2 != 0) widx()[(__float_as_uint(ovl(R_AB)) >> 12) & 127] = (uint8_t)(G + lane);
         }
 
-        // rows: lane k of a round takes staged pair k, runs the pre-step of its active manifolds and writes the pair's row
-        // into its slot; the accumulated impulses of the same pair in the previous step come from the lane that holds that
-        // entry of the warm list (or from the state record beyond the lanes)
-        int nman = 0;
-        const ContactConsts cc = contact_consts();
-#pragma unroll 1
-        for (int base = 0; base < nrec; base += G) {
-            const int k = base + lane;
-            const bool mine = k < nrec;
-            float nx = 0.0f, ny = 0.0f, pt[6] = { 0.0f, 0.0f, 0.0f, 0.0f, 0.0f, 0.0f };
-            if (mine) {
-                if (!crowded) {
-                    const float *sg = sm + SC::STG + lane;
-                    nx = sg[S_NX * G]; ny = sg[S_NY * G];
-                    pt[0] = sg[S_PX0 * G]; pt[1] = sg[S_PY0 * G]; pt[2] = sg[S_PEN0 * G]; pt[3] = sg[S_PX1 * G]; pt[4] = sg[S_PY1 * G]; pt[5] = sg[S_PEN1 * G];
-                } else {
-                    const uint32_t *sg = scr + SC::SCR_STAGE + (size_t)k * kStageStride;
-                    ab = __ldcg(sg + S_AB); nx = __uint_as_float(__ldcg(sg + S_NX)); ny = __uint_as_float(__ldcg(sg + S_NY));
-                    pt[0] = __uint_as_float(__ldcg(sg + S_PX0)); pt[1] = __uint_as_float(__ldcg(sg + S_PY0)); pt[2] = __uint_as_float(__ldcg(sg + S_PEN0));
-                    pt[3] = __uint_as_float(__ldcg(sg + S_PX1)); pt[4] = __uint_as_float(__ldcg(sg + S_PY1)); pt[5] = __uint_as_float(__ldcg(sg + S_PEN1));
-                    slot = (int)__ldcg(sg + kStageWords);
-                }
-            } else ab = 0u;
-            const unsigned amask = (ab >> 10) & 3u;
-            const int p = (ab >> 12) & 127;
-            // warm start values of this pair
-            const int wi = mine ? (int)widx()[p] : 255;
-            const int src = wi < G ? wi : 0;
-            float4 w4 = make_float4(g.shflf(wacc.x, src), g.shflf(wacc.y, src), g.shflf(wacc.z, src), g.shflf(wacc.w, src));
-            if (wi >= G && wi != 255) {
-                const uint32_t *wr = st + SC::ST_WARM + kWarmWords * wi;
-                w4 = make_float4(__uint_as_float(__ldcg(wr + 1)), __uint_as_float(__ldcg(wr + 2)), __uint_as_float(__ldcg(wr + 3)), __uint_as_float(__ldcg(wr + 4)));
-            }
-            if (wi == 255 || !prm.warm_start) w4 = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
-            if (!(amask & 1u)) { w4.x = 0.0f; w4.y = 0.0f; }
-            if (!(amask & 2u)) { w4.z = 0.0f; w4.w = 0.0f; }
-            nman += __popc(amask);
-            if (mine) {
-                const int a = ab & 31, b = (ab >> 5) & 31;
-                const float ma = sm[SC::BIM + a], mb = sm[SC::BIM + b], ia = sm[SC::BII + a], ib = sm[SC::BII + b];
-                const float fra = sm[SC::BFR + a], frb = sm[SC::BFR + b];
-                const float mu = sqrtf(__fmaf_rn(fra, fra, frb * frb));
-                const float er = fmin_cmp(sm[SC::BRE + a], sm[SC::BRE + b]);
-                float4 *r = reinterpret_cast<float4 *>(scr + SC::SCR_ROWS + (size_t)slot * kRowWords);
-                r[0] = make_float4(__uint_as_float(ab), nx, ny, mu);
-                r[1] = make_float4(ma, mb, ia, ib);
-#pragma unroll 1
-                for (int mi = 0; mi < 2; ++mi) {
-                    float rna = 0.0f, rnb = 0.0f, rta = 0.0f, rtb = 0.0f, massn = 0.0f, masst = 0.0f, target = 0.0f, corr = 0.0f;
-                    if (amask & (1u << mi))
-                        prestep_manifold<SC>(a, b, nx, ny, ma, mb, ia, ib, mi ? pt[3] : pt[0], mi ? pt[4] : pt[1], mi ? pt[5] : pt[2], er, sm, cc,
-                                             rna, rnb, rta, rtb, massn, masst, target, corr);
-                    r[2 + 2 * mi] = make_float4(rna, rnb, rta, rtb);
-                    r[3 + 2 * mi] = make_float4(massn, masst, target, corr);
-                }
-                r[6] = w4;
-            }
-        }
-        nman = g.sum_int(nman);
-        c_man += (unsigned)nman | (1u << 16);
-        // velocities (gravity, motors, thrusters) and this step's messages to the solve kernel
-        for (int i = lane; i < SC::N; i += G)
-            reinterpret_cast<float4 *>(st + SC::ST_VEL)[i] = reinterpret_cast<const float4 *>(sm + SC::BVEL)[i];
+        // reward, termination, counters, auto-reset
+        const bool timeout = prm.max_episode_steps > 0 && step_count >= prm.max_episode_steps;
+        float reward = (float)((int)touch_gb - (int)touch_gr);
+        if (prm.dense_kappa != 0.0f && ((smu[SC::META + META_GB] >> 16) & 1u))
+            reward = reward + prm.dense_kappa * (sm[SC::META + META_D0] - green_blue_distance());
+        bool done = touch_gb || touch_gr || timeout;
+        if (!finite) { reward = 0.0f; done = true; }
         if (lane == 0) {
-            const uint32_t flags = (touch_gb ? 1u : 0u) | (touch_gr ? 2u : 0u) | (((gb >> 16) & 1u) << 2) | ((gb & 255u) << 8) | (((gb >> 8) & 255u) << 16) |
-                                   ((uint32_t)cmax << 24);
-            *reinterpret_cast<uint4 *>(st + SC::ST_META + META_NROWS) = make_uint4((uint32_t)nrec, flags, __float_as_uint(d0), active_mask | ((uint32_t)jmax << 16));
+            prm.reward[(size_t)s * prm.n_envs + e] = reward;
+            prm.done[(size_t)s * prm.n_envs + e] = done ? 1 : 0;
+            smu[SC::META + META_STEP] = (uint32_t)step_count;
+            smu[SC::META + META_NWARM] = (uint32_t)nrec;
+            if (!finite) { smu[SC::META + META_STATUS] |= 1u; atomicAdd(prm.counters + 0, 1ULL); }
         }
+        c_man += 1u << 16;
+        g.sync();
+        if (done && prm.auto_reset != 0)
+            jab = reset_env<SC, G>(smu, prm.levels, prm.n_levels, prm.auto_reset, prm.seed, prm.env_offset + e, prm.counters, jab);
+    }
+
+    // ---- whole launch for one scene
+    // steps s0 .. s1-1 of env e.  The state record may have been written by another SM earlier in this
+    // launch, so it is read past the (non-coherent) L1.
+    __device__ __forceinline__ void run(int e, int s0, int s1) {
+        uint32_t *st = prm.state + (size_t)e * SC::ST_WORDS;
+        for (int i = lane; i < 6 * SC::N; i += G) smu[body_word<SC>(i)] = __ldcg(st + SC::ST_BODY + i);
+        if (lane < 5) smu[SC::META + lane] = __ldcg(st + SC::ST_META + lane);
+        if (SC::J > 0 && lane < SC::J) {
+            smu[SC::JROW + kJointWords * lane + JR_ACCX] = __ldcg(st + SC::ST_JACC + 3 * lane);
+            smu[SC::JROW + kJointWords * lane + JR_ACCY] = __ldcg(st + SC::ST_JACC + 3 * lane + 1);
+            smu[SC::JROW + kJointWords * lane + JR_ACCR] = __ldcg(st + SC::ST_JACC + 3 * lane + 2);
+        }
+        for (int i = lane; i < (SC::NPAIRS + 3) / 4; i += G) smu[SC::WIDX + i] = 0xffffffffu;
+        const int level = (int)__ldcg(st + SC::ST_META + META_LEVEL);
+        const int nwarm = (int)__ldcg(st + SC::ST_META + META_NWARM);
+        jab = load_level_consts<SC, G>(smu, prm.levels + (size_t)level * SC::LV_WORDS);
+        g.sync();
+        // accumulated impulses of the previous launch: entry k goes to lane k
+        rec.ab = 0u; rec.accn = 0.0f; rec.acct = 0.0f;
+        lanef(LF_ACC2N) = 0.0f; lanef(LF_ACC2T) = 0.0f;
+        if (lane < nwarm) {
+            const uint32_t *wr = st + SC::ST_WARM + kWarmWords * lane;
+            const uint32_t p = __ldcg(wr);
+            rec.ab = p << 12;
+            rec.accn = __uint_as_float(__ldcg(wr + 1)); rec.acct = __uint_as_float(__ldcg(wr + 2));
+            lanef(LF_ACC2N) = __uint_as_float(__ldcg(wr + 3)); lanef(LF_ACC2T) = __uint_as_float(__ldcg(wr + 4));
+            widx()[p] = (uint8_t)lane;
+        }
+        if (lane < G / 2 && G + lane < nwarm) {
+            const uint32_t *wr = st + SC::ST_WARM + kWarmWords * (G + lane);
+            const uint32_t p = __ldcg(wr);
+            ovl(R_AB) = __uint_as_float(p << 12);
+            ovl(OV_ACC0N) = __uint_as_float(__ldcg(wr + 1)); ovl(OV_ACC0T) = __uint_as_float(__ldcg(wr + 2));
+            ovl(OV_ACC1N) = __uint_as_float(__ldcg(wr + 3)); ovl(OV_ACC1T) = __uint_as_float(__ldcg(wr + 4));
+            widx()[p] = (uint8_t)(G + lane);
+        }
+        if (nwarm > G + G / 2) warm_in<SC, G>(sm, ovf, st + SC::ST_WARM, nwarm);
+        g.sync();
+#pragma unroll 1
+        for (int s = s0; s < s1; ++s) {
+            step(e, s);
+            g.sync();
+            if (((s - s0) & 255) == 255) flush();
+        }
+        // write back
+        for (int i = lane; i < 6 * SC::N; i += G) st[SC::ST_BODY + i] = smu[body_word<SC>(i)];
+        if (SC::J > 0 && lane < SC::J) {
+            st[SC::ST_JACC + 3 * lane] = smu[SC::JROW + kJointWords * lane + JR_ACCX];
+            st[SC::ST_JACC + 3 * lane + 1] = smu[SC::JROW + kJointWords * lane + JR_ACCY];
+            st[SC::ST_JACC + 3 * lane + 2] = smu[SC::JROW + kJointWords * lane + JR_ACCR];
+        }
+        if (lane < 5) st[SC::ST_META + lane] = smu[SC::META + lane];
+        const int nw = (int)smu[SC::META + META_NWARM];
+        if (lane < nw) {
+            uint32_t *wr = st + SC::ST_WARM + kWarmWords * lane;
+            wr[0] = (rec.ab >> 12) & 127u;
+            wr[1] = __float_as_uint(rec.accn); wr[2] = __float_as_uint(rec.acct);
+            wr[3] = __float_as_uint(lanef(LF_ACC2N)); wr[4] = __float_as_uint(lanef(LF_ACC2T));
+        }
+        if (lane < G / 2 && G + lane < nw) {
+            uint32_t *wr = st + SC::ST_WARM + kWarmWords * (G + lane);
+            wr[0] = (__float_as_uint(ovl(R_AB)) >> 12) & 127u;
+            wr[1] = __float_as_uint(ovl(OV_ACC0N)); wr[2] = __float_as_uint(ovl(OV_ACC0T));
+            wr[3] = __float_as_uint(ovl(OV_ACC1N)); wr[4] = __float_as_uint(ovl(OV_ACC1T));
+        }
+        if (nw > G + G / 2) warm_out<SC, G>(ovf, st + SC::ST_WARM, nw);
+        flush();
+        g.sync();
     }
 };
 
+template <class SC>
+__device__ __forceinline__ uint16_t pair_code(int p) {
+    int a, b;
+    if (p < SC::NPP) { int i = 0, rem = p; while (rem >= SC::P - 1 - i) { rem -= SC::P - 1 - i; ++i; } a = i; b = i + 1 + rem; }
+    else if (p < SC::NPP + SC::NPC) { const int q = p - SC::NPP; a = q / SC::C; b = SC::P + q % SC::C; }
+    else { int i = 0, rem = p - SC::NPP - SC::NPC; while (rem >= SC::C - 1 - i) { rem -= SC::C - 1 - i; ++i; } a = SC::P + i; b = SC::P + i + 1 + rem; }
+    return (uint16_t)(a | (b << 8));
+}
 
 template <class SC, int G>
-__global__ void __launch_bounds__(kBlockThreads, kMinBlocks) k2d_prep_kernel(const StepParams prm) {
+__global__ void __launch_bounds__(kBlockThreads, kMinBlocks) k2d_step_kernel(const StepParams prm) {
     extern __shared__ __align__(16) uint32_t smem_raw[];
     constexpr int GPB = kBlockThreads / G;
     uint16_t *ptab = reinterpret_cast<uint16_t *>(smem_raw);
     for (int p = threadIdx.x; p < SC::NPAIRS; p += kBlockThreads) ptab[p] = pair_code<SC>(p);
     __syncthreads();
     const int gib = threadIdx.x / G;
-    const int nslots = gridDim.x * GPB;
+    const int slot = blockIdx.x * GPB + gib, nslots = gridDim.x * GPB;
     uint32_t *region = smem_raw + SC::PTAB_WORDS + gib * region_words<SC, G>();
-    Scene<SC, G> scene(region, ptab, prm);
-    // Envs are handed out one at a time by a ticket counter: a group that is done takes the next one, so groups with
-    // cheap scenes take more of them.  A group draws the ticket of its next env when it starts on an env and reads that
-    // env's meta words half way through, so neither the counter nor the memory is waited for between envs.
+    uint32_t *scratch = prm.scratch + (size_t)slot * SC::SCRATCH_WORDS;
+    Scene<SC, G> scene(region, ptab, scratch, prm);
+    // Work items are (chunk, env), handed out in that order by one ticket counter: a group that is done
+    // takes the next item, so groups with cheap scenes take more of them.  Chunk c of an env may start
+    // only when its chunk c - 1 is stepped and its state is back in memory (another group may have done
+    // it); with items handed out chunk by chunk that is almost always long past, else the group waits for
+    // the group that holds it, which is running.
     const Group<G> &g = scene.g;
-    unsigned t = 0u;
-    if (g.lane == 0) t = atomicAdd(prm.queue + Q_TICKET, 1u);
-    t = g.shflu(t, 0);
-    MetaHead head = { 0u, 0u, 0u };
-    if (t < (unsigned)prm.n_envs) head = load_meta_head(prm.state + (size_t)t * SC::ST_WORDS + SC::ST_META);
-    int taken = 0;
+    const unsigned items = (unsigned)prm.n_envs * (unsigned)prm.n_chunks;
 #pragma unroll 1
-    while (t < (unsigned)prm.n_envs) {
-        unsigned tn_raw = 0u, next_e = 0u;
-        if (g.lane == 0) tn_raw = atomicAdd(prm.queue + Q_TICKET, 1u);
-        MetaHead next_head = { 0u, 0u, 0u };
-        if (head.status & 1u) {      // frozen env: nothing to prepare (the solve kernel reports done)
-            next_e = g.shflu(tn_raw, 0);
-            if (next_e < (unsigned)prm.n_envs) next_head = load_meta_head(prm.state + (size_t)next_e * SC::ST_WORDS + SC::ST_META);
-        } else {
-            scene.prepare((int)t, head, tn_raw, next_e, next_head);
+    for (;;) {
+        unsigned t = 0u;
+        if (g.lane == 0) t = atomicAdd(prm.queue + Q_TICKET, 1u);
+        t = g.shflu(t, 0);
+        if (t >= items) break;
+        const int c = (int)(t / (unsigned)prm.n_envs), e = (int)(t - (unsigned)c * (unsigned)prm.n_envs);
+        bool ok = true;
+        if (c > 0) {
+            if (g.lane == 0) {
+                const volatile unsigned int *flag = prm.chunks_done + e;
+                const volatile unsigned int *err = prm.queue + Q_ERROR;
+                unsigned polls = 0u;
+                while (*flag != (unsigned)c) {
+                    if (*err != 0u || ++polls > kWaitLimit) { atomicExch(prm.queue + Q_ERROR, 1u); ok = false; break; }
+                    __nanosleep(100);
+                }
+            }
+            ok = g.shfl(ok ? 1 : 0, 0) != 0;
+            __threadfence();
         }
-        g.sync();
-        t = next_e; head = next_head;
-        if ((++taken & 63) == 0) scene.flush();
+        if (ok) {
+            const int s0 = c * prm.chunk_steps;
+            scene.run(e, s0, min(prm.n_steps, s0 + prm.chunk_steps));
+        }
+        if (prm.n_chunks > 1) {
+            __threadfence();      // this lane's part of the state record is visible before the count moves
+            g.sync();
+            if (g.lane == 0) atomicExch(prm.chunks_done + e, (c + 1 == prm.n_chunks) ? 0u : (unsigned)(c + 1));
+        }
     }
-    scene.flush();
     // the last group to leave rewinds the queue for the next launch
     if (g.lane == 0) {
         __threadfence();
@@ -1052,334 +1564,7 @@ __global__ void __launch_bounds__(kBlockThreads, kMinBlocks) k2d_prep_kernel(con
     }
 }
 
-// ================================================================ second half of a step: a group of kSolveLanes lanes per env
-// The rows of a scene are copied to shared memory when its group starts (the first kRowCap pair rows and all joint rows;
-// later pair rows, which few scenes have, are used where they are, in the scratch), so the sweeps below read and update
-// them at shared-memory latency.  A row pointer is therefore a generic pointer.
-
-// ---- angular row of a fixed joint or of a revolute joint beyond one of its limits (paper, "Fixed Joints",
-// "Joint Limits"): j_r = (w_a - w_b + correction) / (1/I_a + 1/I_b), a loses j_r / I_a, b gains j_r / I_b.  A fixed
-// joint's impulse is accumulated and warm-started; a limit only ever pushes back, applies no correction while the
-// joint is already returning, and is not accumulated.  The row's last group: kind this step, inverse angular mass,
-// correction, accumulated impulse.  Out of line: most joints are plain revolute joints.
-template <int MODE>
-__device__ __noinline__ float2 angular_row(float *jr, float ia, float ib, float wa, float wb) {
-    const float4 ang4 = ld4(jr + JR_ANG);
-    const int ang = __float_as_int(ang4.x);
-    if (ang == 0) return make_float2(wa, wb);
-    float lr;
-    if (MODE == 0) {
-        if (ang != 1) return make_float2(wa, wb);
-        lr = ang4.w;
-    } else {
-        const float wrel = wa - wb;
-        float v;
-        if (ang == 1) v = wrel + ang4.z;
-        else if (ang == 2) { v = (wrel < 0.0f) ? wrel : wrel + ang4.z; v = fmax_cmp(v, 0.0f); }
-        else { v = (wrel > 0.0f) ? wrel : wrel + ang4.z; v = fmin_cmp(v, 0.0f); }
-        lr = v * ang4.y;
-        if (ang == 1) jr[JR_ACCR] = ang4.w + lr;
-    }
-    return make_float2(__fmaf_rn(-lr, ia, wa), __fmaf_rn(lr, ib, wb));
-}
-
-// one visit of a joint row.  MODE 0: apply the accumulated impulses (warm start); 1: one solver iteration; 2: positional
-// correction.  sv: the scene's bodies in shared memory (velocities; positions in mode 2).
-template <int MODE>
-__device__ __forceinline__ void solve_joint(float *jr, float4 *sv) {
-    const float4 k4 = ld4(jr + JR_I11), mi4 = ld4(jr + JR_MA);
-    const uint32_t jab = __float_as_uint(k4.w);
-    const int a = jab & 255, b = (jab >> 8) & 255;
-    const float ma = mi4.x, mb = mi4.y, ia = mi4.z, ib = mi4.w;
-    if (MODE == 2) {
-        const float cx = jr[JR_CX], cy = jr[JR_CY];
-        if ((jab >> 29) & 1u) { float4 p = sv[a]; p.x = __fmaf_rn(ma, cx, p.x); p.y = __fmaf_rn(ma, cy, p.y); sv[a] = p; }
-        if ((jab >> 30) & 1u) { float4 p = sv[b]; p.x = __fmaf_rn(-mb, cx, p.x); p.y = __fmaf_rn(-mb, cy, p.y); sv[b] = p; }
-        return;
-    }
-    const float4 r4 = ld4(jr + JR_RAX);
-    const float rax = r4.x, ray = r4.y, rbx = r4.z, rby = r4.w;
-    const float4 va4 = sv[a], vb4 = sv[b];
-    float vax = va4.x, vay = va4.y, wa = va4.z, vbx = vb4.x, vby = vb4.y, wb = vb4.z;
-    const float2 acc = *reinterpret_cast<const float2 *>(jr + JR_ACCX);
-    float lx, ly;
-    if (MODE == 0) { lx = acc.x; ly = acc.y; }
-    else {
-        const float2 b2 = *reinterpret_cast<const float2 *>(jr + JR_BX);
-        const float cx = __fmaf_rn(-wb, rby, vbx) - __fmaf_rn(-wa, ray, vax);
-        const float cy = __fmaf_rn(wb, rbx, vby) - __fmaf_rn(wa, rax, vay);
-        const float rx = -(cx + b2.x), ry = -(cy + b2.y);
-        const float i11 = k4.x, i12 = k4.y, i22 = k4.z;
-        lx = __fmaf_rn(i11, rx, i12 * ry);
-        ly = __fmaf_rn(i12, rx, i22 * ry);
-        *reinterpret_cast<float2 *>(jr + JR_ACCX) = make_float2(acc.x + lx, acc.y + ly);
-    }
-    wa = __fmaf_rn(-ia, cross2(rax, ray, lx, ly), wa);
-    wb = __fmaf_rn(ib, cross2(rbx, rby, lx, ly), wb);
-    if (jab >> 31) {      // fixed or limited joint: its angular row follows the point row
-        const float2 w2 = angular_row<MODE>(jr, ia, ib, wa, wb);
-        wa = w2.x; wb = w2.y;
-    }
-    if ((jab >> 29) & 1u) sv[a] = make_float4(__fmaf_rn(-ma, lx, vax), __fmaf_rn(-ma, ly, vay), wa, 0.0f);
-    if ((jab >> 30) & 1u) sv[b] = make_float4(__fmaf_rn(mb, lx, vbx), __fmaf_rn(mb, ly, vby), wb, 0.0f);
-}
-
-// one visit of a pair row (per active manifold the normal row, then the friction row), same modes
-template <int MODE>
-__device__ __forceinline__ void solve_pair(float *r, float4 *sv) {
-    const float4 h0 = ld4(r + R_AB), h1 = ld4(r + R_MA);
-    const uint32_t ab = __float_as_uint(h0.x);
-    const int a = ab & 31, b = (ab >> 5) & 31;
-    const unsigned amask = (ab >> 10) & 3u;
-    const bool dyn_a = (ab >> 26) & 1u, dyn_b = (ab >> 27) & 1u;
-    if (MODE == 2) {
-        const float corr0 = r[R_M0 + M_CORR], corr1 = r[R_M1 + M_CORR];
-        float4 pa = sv[a], pb = sv[b];
-        if (amask & 1u) {
-            const float ca = h1.x * corr0, cb = h1.y * corr0;
-            pa.x = __fmaf_rn(-ca, h0.y, pa.x); pa.y = __fmaf_rn(-ca, h0.z, pa.y);
-            pb.x = __fmaf_rn(cb, h0.y, pb.x); pb.y = __fmaf_rn(cb, h0.z, pb.y);
-        }
-        if (amask & 2u) {
-            const float ca = h1.x * corr1, cb = h1.y * corr1;
-            pa.x = __fmaf_rn(-ca, h0.y, pa.x); pa.y = __fmaf_rn(-ca, h0.z, pa.y);
-            pb.x = __fmaf_rn(cb, h0.y, pb.x); pb.y = __fmaf_rn(cb, h0.z, pb.y);
-        }
-        if (dyn_a) sv[a] = pa;
-        if (dyn_b) sv[b] = pb;
-        return;
-    }
-    const float4 va4 = sv[a], vb4 = sv[b];
-    float vax = va4.x, vay = va4.y, wa = va4.z, vbx = vb4.x, vby = vb4.y, wb = vb4.z;
-    float4 acc = ld4(r + R_ACC);
-    if (amask & 1u) {
-        const float4 c0 = ld4(r + R_M0), c1 = ld4(r + R_M0 + 4);
-        manifold_rows<MODE>(h0.y, h0.z, h0.w, h1.x, h1.y, h1.z, h1.w, c0.x, c0.y, c0.z, c0.w, c1.x, c1.y, c1.z, acc.x, acc.y,
-                            vax, vay, wa, vbx, vby, wb);
-    }
-    if (amask & 2u) {
-        const float4 c0 = ld4(r + R_M1), c1 = ld4(r + R_M1 + 4);
-        manifold_rows<MODE>(h0.y, h0.z, h0.w, h1.x, h1.y, h1.z, h1.w, c0.x, c0.y, c0.z, c0.w, c1.x, c1.y, c1.z, acc.z, acc.w,
-                            vax, vay, wa, vbx, vby, wb);
-    }
-    if (MODE == 1) *reinterpret_cast<float4 *>(r + R_ACC) = acc;
-    if (dyn_a) sv[a] = make_float4(vax, vay, wa, 0.0f);
-    if (dyn_b) sv[b] = make_float4(vbx, vby, wb, 0.0f);
-}
-
-constexpr int kRowCap = 12;   // pair rows of an env that are copied to shared memory for the solve; later rows are used in the scratch
-constexpr int kLevCap = 32;   // level starts of an env kept in shared memory; a scene with more levels reads the table in its scratch
-
-// n groups of 16 bytes from memory to shared memory by the GS lanes of a group, B per lane in flight at a time
-template <int B, int GS>
-__device__ __forceinline__ void stage_groups(float4 *dst, const float4 *src, int n, int lane) {
-#pragma unroll 1
-    for (int base = 0; base < n; base += B * GS) {
-        float4 v[B];
-#pragma unroll
-        for (int k = 0; k < B; ++k) { const int i = base + lane + k * GS; v[k] = (i < n) ? __ldcg(src + i) : make_float4(0.0f, 0.0f, 0.0f, 0.0f); }
-#pragma unroll
-        for (int k = 0; k < B; ++k) { const int i = base + lane + k * GS; if (i < n) dst[i] = v[k]; }
-    }
-}
-
-template <class SC>
-__global__ void __launch_bounds__(kSolveThreads) k2d_solve_kernel(const StepParams prm) {
-    constexpr int GS = kSolveLanes, SPB = kSolveThreads / GS;     // lanes per scene, scenes per block
-    constexpr int JPL = (SC::J + GS - 1) / GS;                    // joints a lane may own: lane, lane + GS, ...
-    // per scene: the bodies' velocities (later positions), the joint rows, the first kRowCap pair rows, the first row of every level
-    constexpr int S_BODY = 0, S_JROW = 4 * SC::N, S_ROWS = S_JROW + kJointWords * SC::J, S_LSTART = S_ROWS + kRowWords * kRowCap;
-    constexpr int S_WORDS = S_LSTART + kLevCap / 4;
-    __shared__ __align__(16) float s_scene[SPB * S_WORDS];
-    const Group<GS> g;
-    const int lane = g.lane, sb = threadIdx.x / GS;
-    const int e = blockIdx.x * SPB + sb;
-    const bool in_range = e < prm.n_envs;
-    uint32_t *st = prm.state + (size_t)(in_range ? e : 0) * SC::ST_WORDS;
-    float *stf = reinterpret_cast<float *>(st);
-    uint4 m0 = make_uint4(0u, 0u, 0u, 0u), m1 = m0;
-    if (in_range) { m0 = *reinterpret_cast<const uint4 *>(st + SC::ST_META); m1 = *reinterpret_cast<const uint4 *>(st + SC::ST_META + 4); }
-    // frozen env: reports done, nothing else
-    const bool frozen = in_range && (m0.w & 1u);
-    if (frozen && lane == 0) { prm.reward[e] = 0.0f; prm.done[e] = 1; }
-    const bool live = in_range && !frozen;
-    const unsigned wmask = __ballot_sync(0xffffffffu, live);      // the warp's lanes that go on: its groups stay in step level by level
-    if (!live) return;
-    float *ss = s_scene + sb * S_WORDS;
-    float4 *sv = reinterpret_cast<float4 *>(ss + S_BODY);
-    float *sj = ss + S_JROW, *sr = ss + S_ROWS;
-    uint8_t *sl = reinterpret_cast<uint8_t *>(ss + S_LSTART);
-    uint32_t *scr = prm.scratch + (size_t)e * SC::SCRATCH_WORDS;
-    float *rows = reinterpret_cast<float *>(scr + SC::SCR_ROWS);
-    const uint8_t *lstart = reinterpret_cast<const uint8_t *>(scr + SC::SCR_LSTART);
-    const int nrows = (int)m1.x;
-    const uint32_t flags = m1.y, active = m1.w & 0xffffu;
-    const int cmax = (int)(flags >> 24), jmax = (int)((m1.w >> 16) & 15u);
-    const int cmax_w = __reduce_max_sync(wmask, cmax), jmax_w = __reduce_max_sync(wmask, jmax);
-    // velocities, joint rows, level starts, pair rows -> shared memory
-    {
-        constexpr int NB = SC::N + 6 * SC::J;       // the velocities and the joint rows are contiguous neither in memory nor here: two sources, one volley
-        constexpr int KB = (NB + GS - 1) / GS;
-        float4 v[KB];
-        uint32_t lw = 0u;
-        const float4 *src_v = reinterpret_cast<const float4 *>(stf + SC::ST_VEL), *src_j = reinterpret_cast<const float4 *>(scr + SC::SCR_JROW);
-#pragma unroll
-        for (int k = 0; k < KB; ++k) {
-            const int i = lane + k * GS;
-            v[k] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
-            if (i < SC::N) v[k] = __ldcg(src_v + i); else if (i < NB) v[k] = __ldcg(src_j + (i - SC::N));
-        }
-        static_assert(kLevCap / 4 <= 2 * GS, "level starts: at most two words per lane");
-        uint32_t lw2 = 0u;
-        if (lane < kLevCap / 4) lw = __ldcg(scr + SC::SCR_LSTART + lane);
-        if (lane + GS < kLevCap / 4) lw2 = __ldcg(scr + SC::SCR_LSTART + lane + GS);
-#pragma unroll
-        for (int k = 0; k < KB; ++k) {
-            const int i = lane + k * GS;
-            if (i < SC::N) sv[i] = v[k]; else if (i < NB) reinterpret_cast<float4 *>(sj)[i - SC::N] = v[k];
-        }
-        if (lane < kLevCap / 4) reinterpret_cast<uint32_t *>(sl)[lane] = lw;
-        if (lane + GS < kLevCap / 4) reinterpret_cast<uint32_t *>(sl)[lane + GS] = lw2;
-    }
-    stage_groups<6, GS>(reinterpret_cast<float4 *>(sr), reinterpret_cast<const float4 *>(rows), 7 * (nrows < kRowCap ? nrows : kRowCap), lane);
-    g.sync();
-    // this lane's joints and their levels (0: the joint takes no part)
-    int jlev[JPL > 0 ? JPL : 1];
-#pragma unroll
-    for (int q = 0; q < JPL; ++q) {
-        const int j = lane + q * GS;
-        jlev[q] = 0;
-        if (j < SC::J) {
-            const uint32_t jab = __float_as_uint(sj[j * kJointWords + JR_JAB]);
-            if ((jab >> 24) & 1u) jlev[q] = (int)((jab >> 25) & 7u);
-        }
-    }
-#define K2D_ROW(r) ((r) < kRowCap ? sr + (r) * kRowWords : rows + (r) * kRowWords)
-#define K2D_LSTART(L) ((L) < kLevCap ? (int)sl[L] : (int)lstart[L])
-    // One sweep over the pair rows / the joint rows, level by level; the rows of a level go to the lanes round robin.  All
-    // groups of the warp walk the same number of levels and meet after each, so that they execute the rows together.
-#define K2D_SWEEP_PAIRS(MODE)                                                                         \
-    _Pragma("unroll 1") for (int L = 1; L <= cmax_w; ++L) {                                           \
-        int r = 0, r1 = 0;                                                                            \
-        if (L <= cmax) { r = K2D_LSTART(L); r1 = K2D_LSTART(L + 1); }                                 \
-        const int rounds = (__reduce_max_sync(wmask, r1 - r) + GS - 1) / GS;                          \
-        r += lane;                                                                                    \
-        _Pragma("unroll 1") for (int q = 0; q < rounds; ++q, r += GS)                                 \
-            if (r < r1) solve_pair<MODE>(K2D_ROW(r), sv);                                             \
-        __syncwarp(wmask);                                                                            \
-    }
-#define K2D_SWEEP_JOINTS(MODE)                                                                        \
-    if (SC::J > 0) {                                                                                  \
-        _Pragma("unroll 1") for (int L = 1; L <= jmax_w; ++L) {                                       \
-            _Pragma("unroll") for (int q = 0; q < JPL; ++q)                                           \
-                if (jlev[q] == L) solve_joint<MODE>(sj + (lane + q * GS) * kJointWords, sv);          \
-            __syncwarp(wmask);                                                                        \
-        }                                                                                             \
-    }
-    // warm start: contacts, then joints (Algorithm 1); solver iterations: joints, then contacts
-    K2D_SWEEP_PAIRS(0)
-    K2D_SWEEP_JOINTS(0)
-#pragma unroll 1
-    for (int it = 0; it < prm.solver_iters; ++it) {
-        K2D_SWEEP_JOINTS(1)
-        K2D_SWEEP_PAIRS(1)
-    }
-    // Euler step with the solved velocities; the velocities go back to the state record and the array holds positions from here on
-    bool finite = true;
-    {
-        constexpr int KN = (SC::N + GS - 1) / GS;
-        float4 p[KN];
-#pragma unroll
-        for (int k = 0; k < KN; ++k) { const int i = lane + k * GS; p[k] = (i < SC::N) ? ld4(stf + SC::ST_POS + 4 * i) : make_float4(0.0f, 0.0f, 0.0f, 0.0f); }
-#pragma unroll
-        for (int k = 0; k < KN; ++k) {
-            const int i = lane + k * GS;
-            if (i < SC::N) {
-                const float4 v4 = sv[i];
-                float4 p4 = p[k];
-                if ((active >> i) & 1u) { p4.x = __fmaf_rn(prm.dt, v4.x, p4.x); p4.y = __fmaf_rn(prm.dt, v4.y, p4.y); p4.z = __fmaf_rn(prm.dt, v4.z, p4.z); }
-                finite = finite && finite_bits(v4.x) && finite_bits(v4.y) && finite_bits(v4.z);
-                st4(stf + SC::ST_VEL + 4 * i, v4.x, v4.y, v4.z);
-                sv[i] = p4;
-            }
-        }
-    }
-    __syncwarp(wmask);
-    // positional corrections: every active manifold moves its two bodies apart along the normal, then the joints close their gaps
-    K2D_SWEEP_PAIRS(2)
-    K2D_SWEEP_JOINTS(2)
-    for (int i = lane; i < SC::N; i += GS) {
-        const float4 p4 = sv[i];
-        finite = finite && finite_bits(p4.x) && finite_bits(p4.y) && finite_bits(p4.z);
-        st4(stf + SC::ST_POS + 4 * i, p4.x, p4.y, p4.z);
-    }
-    finite = !g.any(!finite);
-    // reward and termination (paper, "Reward"): green touches blue = +1, green touches red = -1, either ends the episode
-    const int step_count = (int)m0.x + 1;
-    const bool touch_gb = (flags & 1u) != 0u, touch_gr = (flags & 2u) != 0u;
-    const bool timeout = prm.max_episode_steps > 0 && step_count >= prm.max_episode_steps;
-    float reward = (float)((int)touch_gb - (int)touch_gr);
-    if (prm.dense_kappa != 0.0f && ((flags >> 2) & 1u)) {
-        const float4 pg = sv[(flags >> 8) & 255u], pb = sv[(flags >> 16) & 255u];
-        const float dx = pb.x - pg.x, dy = pb.y - pg.y;
-        reward = reward + prm.dense_kappa * (__uint_as_float(m1.z) - sqrtf(dot2(dx, dy, dx, dy)));
-    }
-    bool done = touch_gb || touch_gr || timeout;
-    uint32_t status = m0.w;
-    if (!finite) { reward = 0.0f; done = true; status |= 1u; }
-    if (lane == 0) {
-        prm.reward[e] = reward;
-        prm.done[e] = done ? 1 : 0;
-        if (!finite) atomicAdd(prm.counters + 0, 1ULL);
-    }
-    if (!(done && prm.auto_reset != 0)) {
-        // the accumulated impulses of this step's rows warm-start the next step
-        for (int r = lane; r < nrows; r += GS) {
-            const float *row = K2D_ROW(r);
-            const float4 acc = ld4(row + R_ACC);
-            uint32_t *wr = st + SC::ST_WARM + kWarmWords * r;
-            wr[0] = (__float_as_uint(row[R_AB]) >> 12) & 127u;
-            wr[1] = __float_as_uint(acc.x); wr[2] = __float_as_uint(acc.y); wr[3] = __float_as_uint(acc.z); wr[4] = __float_as_uint(acc.w);
-        }
-        for (int j = lane; j < SC::J; j += GS) {
-            const float *jr = sj + j * kJointWords;
-            st[SC::ST_JACC + 3 * j] = __float_as_uint(jr[JR_ACCX]);
-            st[SC::ST_JACC + 3 * j + 1] = __float_as_uint(jr[JR_ACCY]);
-            st[SC::ST_JACC + 3 * j + 2] = __float_as_uint(jr[JR_ACCR]);
-        }
-        if (lane == 0) {
-            st[SC::ST_META + META_STEP] = (uint32_t)step_count;
-            st[SC::ST_META + META_STATUS] = status;
-        }
-        return;
-    }
-#undef K2D_SWEEP_JOINTS
-#undef K2D_SWEEP_PAIRS
-#undef K2D_LSTART
-#undef K2D_ROW
-    // auto-reset of a finished env: next level (its own, or drawn from the pool by the hash of seed, global env index
-    // and episode), pose from the level, no accumulated impulses
-    const int episode = (int)m0.y + 1;
-    int level = (int)m0.z;
-    if (prm.auto_reset == 2) {
-        const unsigned long long h = mix64(prm.seed + ((unsigned long long)(prm.env_offset + e) + 1ULL) * 0x9E3779B97F4A7C15ULL +
-                                           (unsigned long long)episode * 0xD1B54A32D192ED03ULL);
-        level = (int)(h % (unsigned long long)prm.n_levels);
-    }
-    const float *lv = reinterpret_cast<const float *>(prm.levels + (size_t)level * SC::LV_WORDS);
-    for (int i = lane; i < SC::N; i += GS) {
-        st4(stf + SC::ST_POS + 4 * i, lv[SC::LV_X + i], lv[SC::LV_Y + i], lv[SC::LV_TH + i]);
-        st4(stf + SC::ST_VEL + 4 * i, lv[SC::LV_VX + i], lv[SC::LV_VY + i], lv[SC::LV_W + i]);
-    }
-    for (int j = lane; j < 3 * SC::J; j += GS) st[SC::ST_JACC + j] = 0u;
-    if (lane == 0) {
-        *reinterpret_cast<uint4 *>(st + SC::ST_META) = make_uint4(0u, (uint32_t)episode, (uint32_t)level, 0u);
-        st[SC::ST_META + META_NROWS] = 0u;
-        atomicAdd(prm.counters + 1, 1ULL);
-    }
-}
-
-// ---------------------------------------------------------------- reset kernel: one block per env
+// ---------------------------------------------------------------- reset kernel: one thread per (env, word)
 template <class SC>
 __global__ void k2d_reset_kernel(uint32_t *state, const uint32_t *levels, const int *level_ids, int n_envs, int n_levels) {
     const int e = blockIdx.x;
@@ -1389,10 +1574,8 @@ __global__ void k2d_reset_kernel(uint32_t *state, const uint32_t *levels, const 
     const uint32_t *lv = levels + (size_t)l * SC::LV_WORDS;
     for (int i = threadIdx.x; i < SC::ST_WARM; i += blockDim.x) {
         uint32_t v = 0u;
-        if (i < 8 * SC::N) {
-            const int half = i / (4 * SC::N), r = i - half * 4 * SC::N, body = r >> 2, f = r & 3;     // position or velocity group, body, component
-            if (f < 3) v = lv[SC::LV_X + (3 * half + f) * SC::N + body];
-        } else if (i == SC::ST_META + META_LEVEL) v = (uint32_t)l;
+        if (i < 6 * SC::N) v = lv[SC::LV_X + i];
+        else if (i == SC::ST_META + 2) v = (uint32_t)l;
         st[i] = v;
     }
 }
@@ -1414,13 +1597,13 @@ __global__ void __launch_bounds__(kObsThreads) k2d_obs_kernel(const uint32_t *st
     float *img = obs_smem + (size_t)w * ((width + 2 * SC::N + 3) / 4 * 4);
     float *cs = img + width;                 // cos, sin of every shape's angle
     const uint32_t *st = state + (size_t)e * SC::ST_WORDS;
-    const uint32_t *lv = levels + (size_t)st[SC::ST_META + META_LEVEL] * SC::LV_WORDS;
+    const uint32_t *lv = levels + (size_t)st[SC::ST_META + 2] * SC::LV_WORDS;
     const float *stf = reinterpret_cast<const float *>(st);
     const float *lvf = reinterpret_cast<const float *>(lv);
     for (int ci = lane; ci < n_shapes; ci += 32) {
         const int i = ci < n_polygons ? ci : SC::P + (ci - n_polygons);     // internal shape index
         float c, sn;
-        sincos_spec(stf[SC::ST_POS + 4 * i + 2], c, sn);
+        sincos_spec(stf[2 * SC::N + i], c, sn);
         cs[i] = c; cs[SC::N + i] = sn;
         float *o = img + ci * 29;
         const uint32_t fl = lv[SC::LV_FLAGS + i];
@@ -1431,9 +1614,9 @@ __global__ void __launch_bounds__(kObsThreads) k2d_obs_kernel(const uint32_t *st
         const int nv = flag_nverts(fl);
         const uint32_t role = flag_role(fl);
         const bool poly = i < SC::P;
-        o[0] = stf[SC::ST_POS + 4 * i]; o[1] = stf[SC::ST_POS + 4 * i + 1]; o[2] = stf[SC::ST_VEL + 4 * i]; o[3] = stf[SC::ST_VEL + 4 * i + 1];
+        o[0] = stf[i]; o[1] = stf[SC::N + i]; o[2] = stf[3 * SC::N + i]; o[3] = stf[4 * SC::N + i];
         o[4] = lvf[SC::LV_IM + i]; o[5] = lvf[SC::LV_II + i]; o[6] = lvf[SC::LV_DENS + i];
-        o[7] = tanh_spec(stf[SC::ST_VEL + 4 * i + 2] * 0.1f);
+        o[7] = tanh_spec(stf[5 * SC::N + i] * 0.1f);
 #pragma unroll
         for (int r = 0; r < 4; ++r) o[8 + r] = (role == (uint32_t)r) ? 1.0f : 0.0f;
         o[12] = sn; o[13] = c; o[14] = lvf[SC::LV_FR + i]; o[15] = lvf[SC::LV_RE + i];
@@ -1525,14 +1708,14 @@ __global__ void __launch_bounds__(kRenderThreads) k2d_render_kernel(const uint32
         const uint32_t fl = lv[SC::LV_FLAGS + i];
         int nv = -1;
         if (fl & F_ACTIVE) {
-            const float x = stf[SC::ST_POS + 4 * i], y = stf[SC::ST_POS + 4 * i + 1];
+            const float x = stf[i], y = stf[SC::N + i];
             const uint32_t role = flag_role(fl);
             uint32_t rgb = role == 1u ? (200u << 8) : role == 2u ? (220u << 16) : role == 3u ? 220u : ((fl & F_DYNAMIC) ? 0x808080u : 0x404040u);
             s_col[i] = rgb | 0xff000000u;
             if (i < SC::P) {
                 nv = (int)flag_nverts(fl);
                 float c, sn;
-                sincos_spec(stf[SC::ST_POS + 4 * i + 2], c, sn);
+                sincos_spec(stf[2 * SC::N + i], c, sn);
                 float nxs[4] = { 0.0f, 0.0f, 0.0f, 0.0f }, nys[4] = { 0.0f, 0.0f, 0.0f, 0.0f }, offs[4] = { 0.0f, 0.0f, 0.0f, 0.0f };
                 float x0 = 0.0f, y0 = 0.0f, x1 = 0.0f, y1 = 0.0f;
 #pragma unroll

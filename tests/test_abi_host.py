@@ -40,9 +40,9 @@ def test_sizes_and_defaults():
     assert lib.k2d_canonical_words(C.byref(cfg)) == 6 * 16 + 2 * 186 + 18 + 4
     sb = lib.k2d_state_bytes(C.byref(cfg))
     assert sb > 16384 * 6 * 16 * 4 and sb % 256 == 0
-    # without the scratch tail: still the env states, and smaller by the tail (per env 120 pair rows of 28 words, 6 joint rows of 24, 32 words of level starts, 120 staging entries of 12)
+    # without the overflow-scratch tail: still the env states, and smaller by the tail (8192 slots of 120 pairs x 29 words)
     ns = lib.k2d_state_bytes_no_scratch(C.byref(cfg))
-    assert 16384 * 6 * 16 * 4 < ns < sb and ns % 256 == 0 and sb - ns == 16384 * (120 * 28 + 6 * 24 + 32 + 120 * 12) * 4
+    assert 16384 * 6 * 16 * 4 < ns < sb and ns % 256 == 0 and sb - ns == 8192 * 120 * 29 * 4
     for dims, width in (((5, 2, 1, 1), 235), ((6, 3, 2, 2), 333)):
         lib.k2d_default_config(C.byref(cfg), 8, *dims)
         assert lib.k2d_obs_floats(C.byref(cfg)) == width

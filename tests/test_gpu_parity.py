@@ -423,6 +423,21 @@ def test_noop_rollout_outcomes_match_the_oracle():
     assert (got != 0).any()
 
 
+def test_status_reports_a_wait_that_ran_out_and_reset_clears_it():
+    # the kernel records a wait that ran out in a word of the control block; here the word is set from the host side
+    # (nothing hangs, nothing waits) to check that k2d_status reports it and k2d_reset clears it
+    import torch
+    lv = scenes.make_levels("S", 4, 3)
+    env = k2d.Env(lv, 4)
+    env.status()
+    env.state_buf[128:144].view(torch.int32)[2] = 1          # work-queue words follow the eight counters: ticket, left, error
+    torch.cuda.synchronize()
+    with pytest.raises(k2d.K2DError, match="waiting"):
+        env.status()
+    env.reset()
+    assert env.status().sum() == 0
+
+
 def test_frame_skip_matches_the_oracle():
     n_envs = 64
     lv = scenes.make_levels("L", n_envs, 97, static_prob=0.1)
