@@ -244,6 +244,12 @@ int k2d_level_info(const k2d_config *cfg, const k2d_level *host_level, float *ho
 int k2d_set_trace(k2d_state *s, float *dev_trace);
 int k2d_trace_slots(const k2d_state *s);
 
+/* Test aid.  With more envs than the device holds scene groups, k2d_step hands out runs of 8 steps of an env to whichever
+ * group is free; a group that gets a later run of an env before the earlier one is back in memory polls for it, about
+ * every 100 ns, at most `polls` times (default 2^24, a few seconds; values below 64 are raised to 64), then records
+ * K2D_ERR_WAIT for k2d_status and gives up.  A small limit lets a test make that wait run out. */
+int k2d_set_wait_limit(k2d_state *s, uint32_t polls);
+
 /* Evaluates the library's own sine/cosine and tanh routines on n device floats (the step
  * uses these instead of libm so that results are reproducible bit for bit). */
 int k2d_eval_sincos_tanh(const float *dev_x, int32_t n, float *dev_cos, float *dev_sin, float *dev_tanh, void *cuda_stream);

@@ -89,6 +89,7 @@ struct k2d_state {
     k2d_config cfg;
     ClassInfo ci;
     int G, grid, groups, slots;
+    unsigned wait_limit;
     size_t smem_bytes;
     cudaStream_t stream;
     unsigned char *dev_base;
@@ -304,7 +305,7 @@ static StepParams step_params(const k2d_state *s, const float *dev_actions, int 
     prm.counters = s->dev_counters; prm.queue = s->dev_queue; prm.chunks_done = s->dev_chunks; prm.scratch = scratch; prm.trace = s->dev_trace;
     prm.n_envs = c.n_envs; prm.n_steps = n_steps; prm.n_actions = c.n_actions; prm.n_levels = c.n_levels;
     prm.discrete = discrete; prm.dense_kappa = c.dense_kappa; prm.frame_skip = c.frame_skip;
-    prm.chunk_steps = n_steps; prm.n_chunks = 1;
+    prm.chunk_steps = n_steps; prm.n_chunks = 1; prm.wait_limit = s->wait_limit;
     if (c.n_envs > s->groups && n_steps > kChunkSteps) {
         const int n_chunks = (n_steps + kChunkSteps - 1) / kChunkSteps;
         if ((unsigned long long)c.n_envs * (unsigned long long)n_chunks + (unsigned long long)s->groups < 0xffffffffULL) {
@@ -385,6 +386,7 @@ int k2d_create(const k2d_config *cfg, void *dev_state_buf, void *dev_level_pool_
     s->cfg = *cfg; s->ci = ci;
     s->G = cfg->lanes_per_scene ? cfg->lanes_per_scene : 16;
     s->stream = (cudaStream_t)cfg->cuda_stream;
+    s->wait_limit = kWaitLimit;
     s->dev_trace = nullptr;
     // index maps between the caller's scene dimensions and the internal size class
     const int nP = cfg->n_polygons, nC = cfg->n_circles, nN = nP + nC;
@@ -606,6 +608,12 @@ int k2d_set_trace(k2d_state *s, float *dev_trace) {
 }
 
 int k2d_trace_slots(const k2d_state *s) { return s ? s->ci.NSLOTS : 0; }
+
+int k2d_set_wait_limit(k2d_state *s, uint32_t polls) {
+    if (!s) return K2D_ERR_NULL;
+    s->wait_limit = polls < 64u ? 64u : polls;
+    return K2D_OK;
+}
 
 int k2d_eval_sincos_tanh(const float *dev_x, int32_t n, float *dev_cos, float *dev_sin, float *dev_tanh, void *cuda_stream) {
     if (!dev_x) return K2D_ERR_NULL;

@@ -33,7 +33,7 @@ constexpr int kMinBlocks = K2D_MIN_BLOCKS;   // resident blocks per SM the step 
 constexpr int kObsThreads = 128;   // observation kernel: one warp per env, four envs per block
 constexpr int kMaxActions = 16;
 enum { Q_TICKET = 0, Q_LEFT = 1, Q_ERROR = 2 };
-constexpr unsigned kWaitLimit = 1u << 24;   // polls (about 100 ns apart) before a wait for another group's chunk gives up
+constexpr unsigned kWaitLimit = 1u << 24;   // default number of polls (about 100 ns apart) before a wait for another group's chunk gives up
 constexpr int kRecWords = 24;   // contact pair record
 constexpr int kWarmWords = 5;   // pair index + 4 accumulated impulses
 constexpr int kStageWords = 9;  // packed pair word, normal, two contact points with penetration
@@ -147,6 +147,7 @@ struct StepParams {
     float *trace;
     int n_envs, n_steps, n_actions, n_levels;
     int chunk_steps, n_chunks;   // a launch is cut into n_chunks pieces of chunk_steps steps; work items are (chunk, env)
+    unsigned wait_limit;         // polls before a wait for another group's chunk gives up
     int solver_iters, warm_start, auto_reset, max_episode_steps;
     int discrete;             // actions are int32 codes (multi-discrete action space) instead of floats
     int frame_skip;           // engine steps each action row is held for
@@ -1537,7 +1538,7 @@ __global__ void __launch_bounds__(kBlockThreads, kMinBlocks) k2d_step_kernel(con
                 const volatile unsigned int *err = prm.queue + Q_ERROR;
                 unsigned polls = 0u;
                 while (*flag != (unsigned)c) {
-                    if (*err != 0u || ++polls > kWaitLimit) { atomicExch(prm.queue + Q_ERROR, 1u); ok = false; break; }
+                    if (*err != 0u || ++polls > prm.wait_limit) { atomicExch(prm.queue + Q_ERROR, 1u); ok = false; break; }
                     __nanosleep(100);
                 }
             }

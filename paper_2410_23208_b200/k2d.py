@@ -20,7 +20,7 @@ EXPORTS = (
     "k2d_default_config", "k2d_state_bytes", "k2d_state_bytes_no_scratch", "k2d_level_pool_bytes", "k2d_create", "k2d_reset", "k2d_step",
     "k2d_step_discrete", "k2d_step_static_scratch", "k2d_obs", "k2d_render",
     "k2d_obs_floats", "k2d_canonical_words", "k2d_get_state", "k2d_set_state", "k2d_status", "k2d_level_info",
-    "k2d_set_trace", "k2d_trace_slots", "k2d_eval_sincos_tanh", "k2d_error_string", "k2d_destroy",
+    "k2d_set_trace", "k2d_trace_slots", "k2d_set_wait_limit", "k2d_eval_sincos_tanh", "k2d_error_string", "k2d_destroy",
 )
 
 
@@ -83,6 +83,7 @@ def load_library():
         lib.k2d_level_info.argtypes = [C.POINTER(Config), vp, vp, vp, vp]
         lib.k2d_set_trace.argtypes = [vp, vp]
         lib.k2d_trace_slots.argtypes = [vp]
+        lib.k2d_set_wait_limit.argtypes = [vp, C.c_uint32]
         lib.k2d_eval_sincos_tanh.argtypes = [vp, i32, vp, vp, vp, vp]
         lib.k2d_error_string.argtypes = [C.c_int]
         lib.k2d_error_string.restype = C.c_char_p
@@ -243,6 +244,10 @@ class Env:
         out = np.zeros(8, np.int64)
         _check(self.lib.k2d_status(self._h, out.ctypes.data), "k2d_status")
         return out
+
+    def set_wait_limit(self, polls: int):
+        """test aid: polls a scene group waits for another group's part of the same env before it gives up"""
+        _check(self.lib.k2d_set_wait_limit(self._h, int(polls)), "k2d_set_wait_limit")
 
     def enable_trace(self):
         torch = self.torch

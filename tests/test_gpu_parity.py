@@ -438,6 +438,35 @@ def test_status_reports_a_wait_that_ran_out_and_reset_clears_it():
     assert env.status().sum() == 0
 
 
+def test_a_wait_that_runs_out_ends_the_launch_and_is_reported():
+    # With more envs than resident scene groups a launch of 16 steps is two runs of 8 steps per env, handed out in the order
+    # (run, env) by a ticket counter.  Here the counter is moved past the first runs from the host, so only second runs are
+    # handed out; each waits for a first run that nobody does.  The wait is bounded (64 polls of about 100 ns here): the first
+    # group to run out records the error, every other wait ends at once, the kernel returns, k2d_status reports it and
+    # k2d_reset clears it.  Nothing hangs and nothing faults.
+    import torch
+    n_envs = 6144
+    lv = scenes.make_levels("L", 64, 5, static_prob=0.1)
+    env = k2d.Env(lv, n_envs, max_fused_steps=16, lanes_per_scene=16)
+    env.set_wait_limit(1)                                     # raised to the floor of 64 polls
+    act = torch.zeros((16, n_envs, env.n_actions), device="cuda")
+    before = env.get_state()
+    env.state_buf[128:144].view(torch.int32)[0] = n_envs      # work-queue words follow the eight counters: ticket, left, error
+    torch.cuda.synchronize()
+    env.step(act)
+    torch.cuda.synchronize()
+    with pytest.raises(k2d.K2DError, match="waiting"):
+        env.status()
+    after = env.get_state()
+    assert np.array_equal(before["pos"], after["pos"]) and np.all(after["step_count"] == 0)      # no run was stepped
+    env.reset()
+    assert env.status().sum() == 0
+    env.set_wait_limit(1 << 24)
+    r, d = env.step(act)                                       # the queue rewound itself: the next launch is an ordinary one
+    torch.cuda.synchronize()
+    assert np.all(env.get_state()["step_count"] == 16) and env.status()[3] == 16 * n_envs and d.shape == (16, n_envs)
+
+
 def test_frame_skip_matches_the_oracle():
     n_envs = 64
     lv = scenes.make_levels("L", n_envs, 97, static_prob=0.1)
