@@ -203,6 +203,13 @@ int k2d_step_static_scratch(k2d_state *s, const float *dev_actions, int32_t n_st
 int k2d_obs(k2d_state *s, float *dev_obs);
 int k2d_obs_floats(const k2d_config *cfg);
 
+/* k2d_step followed by k2d_obs of the state it leaves, as one kernel launch: the group of lanes that has stepped an env
+ * writes the env's observation rows from shared memory before it moves on, so the state is not read back from memory
+ * by a second kernel.  This is the call for a training loop that takes one engine step (or one frame-skip window) and
+ * one observation at a time (paper, "Kinetix": step, then the Symbolic-Entity observation).  Same arguments as k2d_step
+ * plus dev_obs as for k2d_obs; results identical to the two separate calls. */
+int k2d_step_obs(k2d_state *s, const float *dev_actions, int32_t n_steps, float *dev_reward, uint8_t *dev_done, float *dev_obs);
+
 /* Pixel observation (paper: the "Pixels" observation space, a 125 x 125 image; the paper gives
  * no more than the size).  dev_pixels is [n_envs][K2D_PIXELS][K2D_PIXELS][4] bytes, RGBA, row 0
  * at the top, 4-byte aligned.  The centre of pixel (row r, column c) is the world point

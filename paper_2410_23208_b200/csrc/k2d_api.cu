@@ -304,6 +304,7 @@ static StepParams step_params(const k2d_state *s, const float *dev_actions, int 
     prm.state = s->dev_env; prm.levels = s->dev_levels; prm.actions = dev_actions; prm.reward = dev_reward; prm.done = dev_done;
     prm.counters = s->dev_counters; prm.queue = s->dev_queue; prm.chunks_done = s->dev_chunks; prm.scratch = scratch; prm.trace = s->dev_trace;
     prm.n_envs = c.n_envs; prm.n_steps = n_steps; prm.n_actions = c.n_actions; prm.n_levels = c.n_levels;
+    prm.obs = nullptr; prm.n_polygons = c.n_polygons; prm.n_circles = c.n_circles; prm.n_joints = c.n_joints; prm.n_thrusters = c.n_thrusters;
     prm.discrete = discrete; prm.dense_kappa = c.dense_kappa; prm.frame_skip = c.frame_skip;
     prm.chunk_steps = n_steps; prm.n_chunks = 1; prm.wait_limit = s->wait_limit;
     if (c.n_envs > s->groups && n_steps > kChunkSteps) {
@@ -323,6 +324,12 @@ static StepParams step_params(const k2d_state *s, const float *dev_actions, int 
     ((s)->ci.id == 0 ? ((s)->G == 32 ? FN<ClassS, 32>(__VA_ARGS__) : (s)->G == 16 ? FN<ClassS, 16>(__VA_ARGS__) : FN<ClassS, 8>(__VA_ARGS__)) \
    : (s)->ci.id == 1 ? ((s)->G == 32 ? FN<ClassM, 32>(__VA_ARGS__) : (s)->G == 16 ? FN<ClassM, 16>(__VA_ARGS__) : FN<ClassM, 8>(__VA_ARGS__)) \
                      : ((s)->G == 32 ? FN<ClassL, 32>(__VA_ARGS__) : (s)->G == 16 ? FN<ClassL, 16>(__VA_ARGS__) : FN<ClassL, 8>(__VA_ARGS__)))
+
+// does the observation image of the handle's scenes fit into the part of a scene's shared-memory region the step kernel can spare for it?
+template <class SC, int G>
+static bool obs_fits(const k2d_state *s) {
+    return SC::WVX + k2d_obs_floats(&s->cfg) <= region_words<SC, G>();
+}
 
 }  // namespace k2d
 
@@ -452,6 +459,19 @@ int k2d_step(k2d_state *s, const float *dev_actions, int32_t n_steps, float *dev
     CUDA_OK(cudaSetDevice(s->cfg.device));
     const StepParams prm = step_params(s, dev_actions, n_steps, dev_reward, dev_done, s->dev_scratch);
     CUDA_OK(K2D_DISPATCH(launch_step, s, s, prm));
+    return K2D_OK;
+}
+
+int k2d_step_obs(k2d_state *s, const float *dev_actions, int32_t n_steps, float *dev_reward, uint8_t *dev_done, float *dev_obs) {
+    if (!s || !dev_actions || !dev_reward || !dev_done || !dev_obs) return K2D_ERR_NULL;
+    if (n_steps < 1 || n_steps > s->cfg.max_fused_steps) return K2D_ERR_STEPS;
+    if (((uintptr_t)dev_actions & 3) || ((uintptr_t)dev_reward & 3) || ((uintptr_t)dev_obs & 3)) return K2D_ERR_ALIGN;
+    CUDA_OK(cudaSetDevice(s->cfg.device));
+    StepParams prm = step_params(s, dev_actions, n_steps, dev_reward, dev_done, s->dev_scratch);
+    const bool fused = K2D_DISPATCH(obs_fits, s, s);
+    if (fused) prm.obs = dev_obs;
+    CUDA_OK(K2D_DISPATCH(launch_step, s, s, prm));
+    if (!fused) return k2d_obs(s, dev_obs);       // scenes whose observation is wider than the region's spare part: a second launch
     return K2D_OK;
 }
 

@@ -145,6 +145,8 @@ struct StepParams {
     unsigned int *chunks_done; // per env: chunks of this launch already stepped (0 again when the launch is over)
     uint32_t *scratch;
     float *trace;
+    float *obs;               // k2d_step_obs: the symbolic observation after the call's last step, [n_envs][obs_floats]; else null
+    int n_polygons, n_circles, n_joints, n_thrusters;      // the caller's scene dimensions (observation layout)
     int n_envs, n_steps, n_actions, n_levels;
     int chunk_steps, n_chunks;   // a launch is cut into n_chunks pieces of chunk_steps steps; work items are (chunk, env)
     unsigned wait_limit;         // polls before a wait for another group's chunk gives up
@@ -844,6 +846,104 @@ __device__ __noinline__ void trace_clear(float *trace) {
     g.sync();
 }
 
+// ---- symbolic per-entity observation of the scene as it stands (paper, tables "Information provided for shapes /
+// joints / thrusters"), written after the state record has gone back to memory: the image is built in the part of the
+// scene's shared-memory region that only holds per-step data (from the world-frame vertices up) and copied out with
+// 16-byte stores.  The same rows, value for value, as k2d_obs_kernel writes.
+struct ObsDims { int n_polygons, n_circles, n_joints, n_thrusters, n_actions; };
+template <class SC, int G>
+__device__ __noinline__ void write_obs(float *sm, const uint32_t *levels, float *obs, ObsDims dims, int e) {
+    const Group<G> g;
+    const int lane = g.lane;
+    const uint32_t *smu = reinterpret_cast<const uint32_t *>(sm);
+    const uint32_t *lv = levels + (size_t)smu[SC::META + META_LEVEL] * SC::LV_WORDS;
+    const float *lvf = reinterpret_cast<const float *>(lv);
+    const int n_shapes = dims.n_polygons + dims.n_circles;
+    const int jw = 11 + dims.n_actions;
+    const int width = n_shapes * 29 + 2 * dims.n_joints * jw + 6 * dims.n_thrusters;
+    float *img = sm + SC::WVX;
+    g.sync();
+    for (int i = lane; i < SC::N; i += G) {
+        float c, sn;
+        sincos_spec(sm[SC::BPOS + 4 * i + 2], c, sn);
+        sm[SC::BC + i] = c; sm[SC::BS + i] = sn;
+    }
+    g.sync();
+    for (int ci = lane; ci < n_shapes; ci += G) {
+        const int i = ci < dims.n_polygons ? ci : SC::P + (ci - dims.n_polygons);     // internal shape index
+        float *o = img + ci * 29;
+        const uint32_t fl = smu[SC::BFL + i];
+        if (!(fl & F_ACTIVE)) {
+            for (int f = 0; f < 29; ++f) o[f] = 0.0f;
+            continue;
+        }
+        const int nv = flag_nverts(fl);
+        const uint32_t role = flag_role(fl);
+        const bool poly = i < SC::P;
+        const float4 p4 = ld4(sm + SC::BPOS + 4 * i), v4 = ld4(sm + SC::BVEL + 4 * i);
+        o[0] = p4.x; o[1] = p4.y; o[2] = v4.x; o[3] = v4.y;
+        o[4] = sm[SC::BIM + i]; o[5] = sm[SC::BII + i]; o[6] = lvf[SC::LV_DENS + i];
+        o[7] = tanh_spec(v4.z * 0.1f);
+#pragma unroll
+        for (int r = 0; r < 4; ++r) o[8 + r] = (role == (uint32_t)r) ? 1.0f : 0.0f;
+        o[12] = sm[SC::BS + i]; o[13] = sm[SC::BC + i]; o[14] = sm[SC::BFR + i]; o[15] = sm[SC::BRE + i];
+        o[16] = poly ? 1.0f : 0.0f; o[17] = poly ? 0.0f : 1.0f;
+        o[18] = poly ? 0.0f : sm[SC::RAD + (poly ? 0 : i - SC::P)];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const bool on = poly && k < nv;
+            o[19 + 2 * k] = on ? lvf[SC::LV_PVX + 4 * (poly ? i : 0) + k] : 0.0f;
+            o[20 + 2 * k] = on ? lvf[SC::LV_PVY + 4 * (poly ? i : 0) + k] : 0.0f;
+        }
+        o[27] = (poly && nv == 3) ? 1.0f : 0.0f;
+        o[28] = (poly && nv != 3) ? 1.0f : 0.0f;
+    }
+    float *jrows = img + n_shapes * 29;
+    for (int row = lane; row < 2 * dims.n_joints; row += G) {
+        const int j = row >> 1, d = row & 1;
+        const uint32_t *jl = lv + SC::LV_JOINT + kJointLevelWords * j;
+        const uint32_t jw0 = jl[0];
+        float *o = jrows + row * jw;
+        for (int f = 0; f < jw; ++f) o[f] = 0.0f;
+        if ((jw0 >> 28) & 1u) {
+            const int a = jw0 & 255, b = (jw0 >> 8) & 255;
+            const int from = d ? b : a, to = d ? a : b;
+            o[0] = 1.0f; o[1] = (jl[10] & 1u) ? 1.0f : 0.0f;
+#pragma unroll
+            for (int f = 2; f < 6; ++f) { const int side = ((f - 2) >> 1) ^ d; o[f] = __uint_as_float(jl[1 + 2 * side + ((f - 2) & 1)]); }
+            o[6] = __uint_as_float(jl[6]); o[7] = __uint_as_float(jl[5]);
+            const int bind = (int)((jw0 >> 16) & 255);
+            if (bind < dims.n_actions) o[9 + bind] = 1.0f;
+            o[9 + dims.n_actions] = __fmaf_rn(sm[SC::BS + to], sm[SC::BC + from], -(sm[SC::BC + to] * sm[SC::BS + from]));
+            o[10 + dims.n_actions] = __fmaf_rn(sm[SC::BC + to], sm[SC::BC + from], sm[SC::BS + to] * sm[SC::BS + from]);
+        }
+    }
+    float *trows = jrows + 2 * dims.n_joints * jw;
+    for (int t = lane; t < dims.n_thrusters; t += G) {
+        const uint32_t *th = lv + SC::LV_THR + 8 * t;
+        const uint32_t tp = th[0];
+        float *o = trows + t * 6;
+        for (int f = 0; f < 6; ++f) o[f] = 0.0f;
+        if ((tp >> 20) & 1u) {
+            const int i = tp & 255;
+            float dx, dy;
+            rot2(sm[SC::BC + i], sm[SC::BS + i], __uint_as_float(th[3]), __uint_as_float(th[4]), dx, dy);
+            o[0] = 1.0f; o[1] = __uint_as_float(th[1]); o[2] = __uint_as_float(th[2]); o[3] = __uint_as_float(th[5]);
+            o[4] = dy; o[5] = dx;
+        }
+    }
+    g.sync();
+    float *out = obs + (size_t)e * width;
+    if (((width & 3) == 0) && ((reinterpret_cast<uintptr_t>(obs) & 15) == 0)) {
+        const float4 *src = reinterpret_cast<const float4 *>(img);
+        float4 *dst = reinterpret_cast<float4 *>(out);
+        for (int q = lane; q < width / 4; q += G) dst[q] = src[q];
+    } else {
+        for (int q = lane; q < width; q += G) out[q] = img[q];
+    }
+    g.sync();
+}
+
 // ---------------------------------------------------------------- scene processing
 template <class SC, int G>
 struct Scene {
@@ -1493,6 +1593,10 @@ struct Scene {
         if (nw > G + G / 2) warm_out<SC, G>(ovf, st + SC::ST_WARM, nw);
         flush();
         g.sync();
+        if (prm.obs && s1 == prm.n_steps) {
+            ObsDims od; od.n_polygons = prm.n_polygons; od.n_circles = prm.n_circles; od.n_joints = prm.n_joints; od.n_thrusters = prm.n_thrusters; od.n_actions = prm.n_actions;
+            write_obs<SC, G>(sm, prm.levels, prm.obs, od, e);
+        }
     }
 };
 

@@ -18,7 +18,7 @@ RESET_NONE, RESET_SAME_LEVEL, RESET_POOL = 0, 1, 2
 
 EXPORTS = (
     "k2d_default_config", "k2d_state_bytes", "k2d_state_bytes_no_scratch", "k2d_level_pool_bytes", "k2d_create", "k2d_reset", "k2d_step",
-    "k2d_step_discrete", "k2d_step_static_scratch", "k2d_obs", "k2d_render",
+    "k2d_step_discrete", "k2d_step_static_scratch", "k2d_step_obs", "k2d_obs", "k2d_render",
     "k2d_obs_floats", "k2d_canonical_words", "k2d_get_state", "k2d_set_state", "k2d_status", "k2d_level_info",
     "k2d_set_trace", "k2d_trace_slots", "k2d_set_wait_limit", "k2d_eval_sincos_tanh", "k2d_error_string", "k2d_destroy",
 )
@@ -73,6 +73,7 @@ def load_library():
         lib.k2d_step.argtypes = [vp, vp, i32, vp, vp]
         lib.k2d_step_static_scratch.argtypes = [vp, vp, i32, vp, vp]
         lib.k2d_step_discrete.argtypes = [vp, vp, i32, vp, vp]
+        lib.k2d_step_obs.argtypes = [vp, vp, i32, vp, vp, vp]
         lib.k2d_obs.argtypes = [vp, vp]
         lib.k2d_render.argtypes = [vp, vp]
         lib.k2d_obs_floats.argtypes = [C.POINTER(Config)]
@@ -193,6 +194,25 @@ class Env:
                     else (self.lib.k2d_step_discrete, "k2d_step_discrete") if discrete else (self.lib.k2d_step, "k2d_step"))
         _check(fn(self._h, actions.data_ptr(), n_steps, reward.data_ptr(), done.data_ptr()), name)
         return reward, done
+
+    def step_obs(self, actions, reward=None, done=None, obs=None, n_steps=None):
+        """k2d_step_obs: the steps of ``step`` and the observation of the state they leave, in one launch;
+        returns (reward, done, obs)"""
+        torch = self.torch
+        assert actions.is_cuda and actions.dtype == torch.float32 and actions.is_contiguous()
+        if actions.dim() == 2:
+            actions = actions.unsqueeze(0)
+        fs = max(1, int(self.cfg.frame_skip))
+        n_steps = actions.shape[0] * fs if n_steps is None else int(n_steps)
+        assert tuple(actions.shape) == (-(-n_steps // fs), self.n_envs, self.n_actions), tuple(actions.shape)
+        if reward is None:
+            reward = torch.empty((n_steps, self.n_envs), dtype=torch.float32, device=self.device)
+        if done is None:
+            done = torch.empty((n_steps, self.n_envs), dtype=torch.uint8, device=self.device)
+        if obs is None:
+            obs = torch.empty((self.n_envs, self.obs_floats), dtype=torch.float32, device=self.device)
+        _check(self.lib.k2d_step_obs(self._h, actions.data_ptr(), n_steps, reward.data_ptr(), done.data_ptr(), obs.data_ptr()), "k2d_step_obs")
+        return reward, done, obs
 
     def obs(self, out=None):
         torch = self.torch

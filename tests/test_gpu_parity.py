@@ -268,6 +268,26 @@ def test_observation_parity(size):
     assert np.array_equal(got.view(np.uint32), want.view(np.uint32))
 
 
+@pytest.mark.parametrize("size,n_envs,lanes,n_actions", [("S", 40, 0, 0), ("M", 40, 8, 0), ("L", 72, 16, 0), ("L", 24, 32, 16), ("L", 7000, 0, 0)])
+def test_step_with_observation_in_one_launch(size, n_envs, lanes, n_actions):
+    # k2d_step_obs = k2d_step then k2d_obs: one step at a time (the training loop's use), then launches of several steps,
+    # with resets in between; 7000 envs are more than the device holds at once, so those launches are cut into runs and
+    # the observation must come from the last run only
+    import torch
+    lv = scenes.make_levels(size, min(n_envs, 256), 15, static_prob=0.1, triangle_prob=0.2, fixed_prob=0.2)
+    kw = dict(n_actions=n_actions) if n_actions else {}
+    env, ref = parity.make_pair(lv, n_envs, auto_reset=2, max_episode_steps=7, seed=9, lanes_per_scene=lanes, max_fused_steps=20, **kw)
+    act = scenes.make_actions(3 + 20 + 11, n_envs, env.n_actions, 15)
+    for lo, hi in ((0, 1), (1, 2), (2, 3), (3, 23), (23, 34)):
+        r, d, o = env.step_obs(torch.from_numpy(act[lo:hi]).cuda())
+        rr, dr = ref.step(act[lo:hi], n_threads=8)
+        assert np.array_equal(r.cpu().numpy(), rr) and np.array_equal(d.cpu().numpy(), dr)
+        assert np.array_equal(o.cpu().numpy().view(np.uint32), ref.obs().view(np.uint32)), (lo, hi)
+        assert torch.equal(o, env.obs())
+    err, exact = parity.errors(env, ref)
+    assert exact, err
+
+
 def test_non_finite_state_is_flagged_not_propagated():
     lv = scenes.make_levels("S", 8, 81)
     env, ref = parity.make_pair(lv, 8)
