@@ -3,6 +3,10 @@
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--workload 3] [--impl reference]
 
+With --gpus N > 1 and no torchrun environment the script starts the N ranks itself (one process per GPU,
+rendezvous on 127.0.0.1); under torchrun it is one of the ranks.  Envs are sharded over the ranks with no
+exchange of data; NCCL carries only the barrier and the maximum of the ranks' times.
+
 One "step" of the benchmark is one pass of the whole hot path over one batch of synthetic input:
 one k2d_step launch that advances every env by FUSED (32) engine steps (actions in, reward and done
 out, auto-reset inside), followed by one k2d_obs launch (the symbolic per-entity observation).
@@ -38,8 +42,17 @@ UNIT = "env-steps/s"
 FLOPS = dict(body=37, circle_box=4, polygon=84, box_test=8, cc=16, pc=94, pp=190,
              pair_prestep=5, man_prestep=54, man_warm=28, man_iter=57, man_pos=10,
              joint_fixed=48 + 33 + 18 + 8, joint_iter=38, thruster=27)
-# DRAM bytes one ncu capture measured for one k2d_step launch of the benchmark workload, per env
-NCU_DRAM_BYTES_PER_ENV_LAUNCH = 2064.0   # profiles/k2d_step_kernel_L_16384envs_32steps.md: (33.369 MB + 0.448 MB) / 16384 envs; None once the kernel has changed since
+
+
+def ncu_dram_bytes_per_env_launch(size: str, fused: int, n_envs: int):
+    """DRAM bytes (read + write) per env that an ncu capture of one k2d_step launch measured for this size class, number of
+    fused steps and env count, from the tracked table of captures; None when no capture of the current kernel matches."""
+    path = os.path.join(ROOT, "profiles", "k2d_step_kernel_dram_traffic.json")
+    if not os.path.exists(path):
+        return None
+    with open(path) as f:
+        table = json.load(f)
+    return table.get("captures", {}).get(f"{size}/{fused}/{n_envs}")
 
 
 def fp32_peak_tflops(sm_count: int = 148, sm_mhz: float = 1965.0) -> float:
@@ -305,13 +318,57 @@ def run_gpu(args) -> dict:
     e1.record()
     barrier()
     e2e_ms = e0.elapsed_time(e1)
+
+    # ---- the same loop with the observation copied to the host as well (a learner on the host, or logging)
+    host_obs = torch.empty(obs.shape, dtype=obs.dtype).pin_memory()
+    K_OBS = min(K, 8)
+    barrier()
+    o0, o1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    o0.record()
+    for i in range(K_OBS):
+        stages[0].copy_(host_actions[i % len(host_actions)], non_blocking=True)
+        env.step(stages[0], rewards[0], dones[0])
+        env.obs(obs)
+        host_reward.copy_(rewards[0], non_blocking=True)
+        host_done.copy_(dones[0], non_blocking=True)
+        host_obs.copy_(obs, non_blocking=True)
+    o1.record()
+    barrier()
+    e2e_obs_ms = o0.elapsed_time(o1) * K / K_OBS
+
+    # ---- other ways to drive the same path (L2 not flushed; the state of 16384 envs stays in L2 between launches anyway):
+    # one engine step and one observation per call, as a training loop does, with two launches and with the fused launch
+    modes = {}
+    if not args.pixels:
+        one = [a[:1].contiguous() for a in dev_actions[:2]]
+        r1, d1 = reward[:1], done[:1]
+        n_it = 64
+        for name in ("one_step_then_obs", "one_step_obs_fused"):
+            for _ in range(4):
+                env.step_obs(one[0], r1, d1, obs)
+            barrier()
+            m0, m1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            m0.record()
+            for i in range(n_it):
+                if name == "one_step_then_obs":
+                    env.step(one[i & 1], r1, d1)
+                    env.obs(obs)
+                else:
+                    env.step_obs(one[i & 1], r1, d1, obs)
+            m1.record()
+            barrier()
+            modes[name] = m0.elapsed_time(m1) / n_it
     clocks.__exit__()
     clk = clocks.summary()   # sampled every 100 ms from the first warm-up step to the end of the end-to-end loop
 
+    mode_names = sorted(modes)
     if world > 1:
-        t = torch.tensor([total_ms, e2e_ms, float(np.mean(step_ms))], device=dev, dtype=torch.float64)
+        t = torch.tensor([total_ms, e2e_ms, float(np.mean(step_ms)), e2e_obs_ms] + [modes[k] for k in mode_names], device=dev, dtype=torch.float64)
         torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
-        total_ms, e2e_ms, mean_step_ms = (float(x) for x in t.tolist())
+        vals = [float(x) for x in t.tolist()]
+        total_ms, e2e_ms, mean_step_ms, e2e_obs_ms = vals[:4]
+        modes = dict(zip(mode_names, vals[4:]))
+        torch.distributed.destroy_process_group()
     else:
         mean_step_ms = float(np.mean(step_ms))
     if rank != 0:
@@ -327,6 +384,8 @@ def run_gpu(args) -> dict:
         bytes_["obs"] = 125 * 125 * 4 + 4 * 6 * dims.n_shapes      # the image out, the poses in
     achieved_tflops = flops_step * env_steps_per_launch / (mean_step_ms * 1e-3) / 1e12
     peak = fp32_peak_tflops()
+    peak_measured = k2d.measure_fp32_peak(local)
+    traffic_per_env = ncu_dram_bytes_per_env_launch(w["size"], FUSED, n_envs)
     hbm_peak, hbm_src = measured_hbm_gbs()
     hbm_gbs = bytes_["step"] * n_envs / (mean_step_ms * 1e-3) / 1e9
     obs_gbs = bytes_["obs"] * n_envs / (float(np.mean(obs_ms)) * 1e-3) / 1e9
@@ -341,11 +400,21 @@ def run_gpu(args) -> dict:
                    "l2": "flushed between timed iterations (256 MiB write, untimed); K distinct action buffers"},
         "clocks": clk,
         "e2e": {"value": e2e_value, "unit": UNIT,
-                "h2d_bytes_per_step": int(stage.numel() * 4), "d2h_bytes_per_step": int(host_reward.numel() * 4 + host_done.numel())},
+                "h2d_bytes_per_step": int(stage.numel() * 4), "d2h_bytes_per_step": int(host_reward.numel() * 4 + host_done.numel()),
+                "note": "actions up, reward and done down every bench step; the observation stays on the device, where a policy network reads it"},
+        "e2e_with_obs": {"value": world * env_steps_per_launch * K / (e2e_obs_ms * 1e-3), "unit": UNIT,
+                         "h2d_bytes_per_step": int(stage.numel() * 4),
+                         "d2h_bytes_per_step": int(host_reward.numel() * 4 + host_done.numel() + host_obs.numel() * host_obs.element_size()),
+                         "note": "as e2e, and the observation is copied to pinned host memory every bench step; no overlap of copies and launches"},
+        "modes": {k: {"ms_per_call": v, "value": world * n_envs / (v * 1e-3), "unit": UNIT,
+                      "what": ("k2d_step(1 step) + k2d_obs: two launches per call" if k == "one_step_then_obs"
+                               else "k2d_step_obs(1 step): one launch per call")} for k, v in modes.items()},
         "gpu_launches": 2 * K,
         "roofline": {"bound": "alu", "kernel": "k2d_step_kernel", "achieved": achieved_tflops, "peak": peak, "unit": "TFLOP/s",
-                     "frac": achieved_tflops / peak, "traffic": None if NCU_DRAM_BYTES_PER_ENV_LAUNCH is None else NCU_DRAM_BYTES_PER_ENV_LAUNCH * n_envs,
+                     "frac": achieved_tflops / peak, "traffic": None if traffic_per_env is None else traffic_per_env * n_envs,
                      "peak_source": "derived: 148 SMs x 128 lanes x 2 x 1965 MHz",
+                     "peak_measured": peak_measured, "frac_of_measured": achieved_tflops / peak_measured,
+                     "peak_measured_source": "chains of fused multiply-adds on every SM, timed in this run (k2d_measure_fp32_peak)",
                      "flops_per_env_step": flops_step, "launch_ms": mean_step_ms,
                      "hbm": {"achieved": hbm_gbs, "peak": hbm_peak, "unit": "GB/s", "frac": hbm_gbs / hbm_peak, "of": hbm_src,
                              "bytes_per_env_launch": bytes_["step"]},
@@ -357,6 +426,40 @@ def run_gpu(args) -> dict:
     if world == 1 and not args.no_cpu_baseline:
         out["cpu_baseline"] = cpu_baseline(args, w, dims, levels)
     return out
+
+
+def spawn_ranks(n: int) -> int:
+    """--gpus N without a torchrun environment: start the N ranks (this script again, one process per GPU)."""
+    import socket
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        port = sk.getsockname()[1]
+    procs = []
+    for r in range(n):
+        env = dict(os.environ, RANK=str(r), LOCAL_RANK=str(r), WORLD_SIZE=str(n), MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+        procs.append(subprocess.Popen([sys.executable, os.path.abspath(__file__)] + sys.argv[1:], env=env))
+    return max(p.wait() for p in procs)
+
+
+def run_plan(args) -> dict:
+    """--plan: no GPU work; every rank joins a gloo group and reports the env range it would step."""
+    import torch
+    import torch.distributed as dist
+    from paper_2410_23208_b200 import k2d
+    rank, world = int(os.environ.get("RANK", "0")), int(os.environ.get("WORLD_SIZE", "1"))
+    n_envs = args.envs or scenes.WORKLOADS[args.workload]["n_envs"]
+    mine = torch.tensor([rank, int(os.environ.get("LOCAL_RANK", "0")), rank * n_envs, n_envs], dtype=torch.int64)
+    rows = [mine]
+    if world > 1:
+        dist.init_process_group("gloo")
+        rows = [torch.zeros_like(mine) for _ in range(world)]
+        dist.all_gather(rows, mine)
+        dist.destroy_process_group()
+    if rank != 0:
+        return {}
+    return {"plan": [dict(rank=int(r[0]), local_rank=int(r[1]), env_offset=int(r[2]), n_envs=int(r[3])) for r in rows],
+            "n_gpus": world, "scaling": "weak", "total_envs": int(sum(int(r[3]) for r in rows)),
+            "shard_of_total": [list(k2d.shard_envs(world * n_envs, k, world)) for k in range(world)]}
 
 
 def main():
@@ -371,7 +474,15 @@ def main():
     ap.add_argument("--fused", type=int, default=FUSED, help="engine steps per k2d_step launch (1 = one launch and one observation per step)")
     ap.add_argument("--pixels", action="store_true", help="the observation of a bench step is the 125 x 125 pixel image (k2d_render) instead of the entity rows")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--plan", action="store_true", help="no GPU work: the ranks rendezvous over gloo and rank 0 prints which envs each would step")
     args = ap.parse_args()
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ and (args.impl == "k2d" or args.plan):
+        sys.exit(spawn_ranks(args.gpus))
+    if args.plan:
+        out = run_plan(args)
+        if out:
+            print(json.dumps(out), flush=True)
+        return
     args.warmup = max(args.warmup, 3) if args.impl == "k2d" else args.warmup
     if args.impl == "reference":
         if int(os.environ.get("RANK", "0")) != 0:

@@ -261,6 +261,12 @@ int k2d_set_wait_limit(k2d_state *s, uint32_t polls);
  * uses these instead of libm so that results are reproducible bit for bit). */
 int k2d_eval_sincos_tanh(const float *dev_x, int32_t n, float *dev_cos, float *dev_sin, float *dev_tanh, void *cuda_stream);
 
+/* Measurement aid, not part of the step: runs chains of dependent fused multiply-adds on every SM of the device (eight
+ * independent chains per thread, 2048 threads per SM) on the default stream and returns the FP32 rate they reach, in
+ * TFLOP/s (a multiply-add counts 2), in *host_tflops: the measured counterpart of SMs x 128 lanes x 2 x clock.
+ * dev_scratch: at least 2048 x the device's SM count floats of device memory (overwritten).  Synchronous. */
+int k2d_measure_fp32_peak(int32_t device, float *dev_scratch, size_t scratch_floats, float *host_tflops);
+
 const char *k2d_error_string(int code);
 void k2d_destroy(k2d_state *s);
 

@@ -687,6 +687,33 @@ int k2d_step_static_scratch(k2d_state *s, const float *dev_actions, int32_t n_st
     return K2D_OK;
 }
 
+int k2d_measure_fp32_peak(int32_t device, float *dev_scratch, size_t scratch_floats, float *host_tflops) {
+    if (!dev_scratch || !host_tflops) return K2D_ERR_NULL;
+    CUDA_OK(cudaSetDevice(device));
+    int num_sms = 0;
+    CUDA_OK(cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, device));
+    const int threads = 256, blocks = num_sms * 8;        // 2048 threads per SM: every scheduler has chains to pick from
+    if (scratch_floats < (size_t)threads * blocks) return K2D_ERR_ARG;
+    cudaEvent_t e0, e1;
+    CUDA_OK(cudaEventCreate(&e0));
+    CUDA_OK(cudaEventCreate(&e1));
+    float best_ms = 0.0f;
+    for (int rep = 0; rep < 5; ++rep) {       // the first launches warm up; the best of the rest counts
+        CUDA_OK(cudaEventRecord(e0, 0));
+        k2d_fma_chain_kernel<<<blocks, threads>>>(dev_scratch, 0.999f, 1e-3f);
+        CUDA_OK(cudaEventRecord(e1, 0));
+        CUDA_OK(cudaEventSynchronize(e1));
+        float ms = 0.0f;
+        CUDA_OK(cudaEventElapsedTime(&ms, e0, e1));
+        if (rep >= 2 && (best_ms == 0.0f || ms < best_ms)) best_ms = ms;
+    }
+    CUDA_OK(cudaEventDestroy(e0));
+    CUDA_OK(cudaEventDestroy(e1));
+    const double flops = 2.0 * kFmaChainSteps * kFmaChains * (double)threads * blocks;
+    *host_tflops = (float)(flops / (best_ms * 1e-3) / 1e12);
+    return K2D_OK;
+}
+
 const char *k2d_error_string(int code) {
     switch (code) {
         case K2D_OK: return "ok";

@@ -1900,4 +1900,25 @@ __global__ void k2d_eval_kernel(const float *x, int n, float *c, float *s, float
     if (t) t[i] = tanh_spec(x[i]);
 }
 
+// ---------------------------------------------------------------- FP32 throughput probe
+// Eight independent chains of fused multiply-adds per thread, kFmaChainSteps links each: what the FP32 pipes of the device
+// sustain when nothing else limits them.  The result is stored so that the chains are not removed.
+constexpr int kFmaChainSteps = 4096, kFmaChains = 8;
+__global__ void __launch_bounds__(256) k2d_fma_chain_kernel(float *out, float a, float b) {
+    float v[kFmaChains];
+#pragma unroll
+    for (int k = 0; k < kFmaChains; ++k) v[k] = (float)(threadIdx.x + k) * 1e-3f;
+#pragma unroll 1
+    for (int i = 0; i < kFmaChainSteps; i += 4) {
+#pragma unroll
+        for (int u = 0; u < 4; ++u)
+#pragma unroll
+            for (int k = 0; k < kFmaChains; ++k) v[k] = __fmaf_rn(v[k], a, b);
+    }
+    float sum = 0.0f;
+#pragma unroll
+    for (int k = 0; k < kFmaChains; ++k) sum += v[k];
+    out[blockIdx.x * blockDim.x + threadIdx.x] = sum;
+}
+
 }  // namespace k2d

@@ -20,7 +20,7 @@ EXPORTS = (
     "k2d_default_config", "k2d_state_bytes", "k2d_state_bytes_no_scratch", "k2d_level_pool_bytes", "k2d_create", "k2d_reset", "k2d_step",
     "k2d_step_discrete", "k2d_step_static_scratch", "k2d_step_obs", "k2d_obs", "k2d_render",
     "k2d_obs_floats", "k2d_canonical_words", "k2d_get_state", "k2d_set_state", "k2d_status", "k2d_level_info",
-    "k2d_set_trace", "k2d_trace_slots", "k2d_set_wait_limit", "k2d_eval_sincos_tanh", "k2d_error_string", "k2d_destroy",
+    "k2d_set_trace", "k2d_trace_slots", "k2d_set_wait_limit", "k2d_eval_sincos_tanh", "k2d_measure_fp32_peak", "k2d_error_string", "k2d_destroy",
 )
 
 
@@ -86,6 +86,7 @@ def load_library():
         lib.k2d_trace_slots.argtypes = [vp]
         lib.k2d_set_wait_limit.argtypes = [vp, C.c_uint32]
         lib.k2d_eval_sincos_tanh.argtypes = [vp, i32, vp, vp, vp, vp]
+        lib.k2d_measure_fp32_peak.argtypes = [i32, vp, C.c_size_t, vp]
         lib.k2d_error_string.argtypes = [C.c_int]
         lib.k2d_error_string.restype = C.c_char_p
         lib.k2d_destroy.argtypes = [vp]
@@ -297,6 +298,17 @@ def eval_sincos_tanh(x):
     _check(lib.k2d_eval_sincos_tanh(x.data_ptr(), x.numel(), c.data_ptr(), s.data_ptr(), t.data_ptr(),
                                     torch.cuda.current_stream(x.device).cuda_stream), "k2d_eval_sincos_tanh")
     return c, s, t
+
+
+def measure_fp32_peak(device: int = 0) -> float:
+    """TFLOP/s the device's FP32 pipes reach on chains of fused multiply-adds (k2d_measure_fp32_peak)"""
+    import torch
+    lib = load_library()
+    n = 2048 * torch.cuda.get_device_properties(device).multi_processor_count
+    buf = torch.empty(n, dtype=torch.float32, device=torch.device("cuda", device))
+    out = C.c_float()
+    _check(lib.k2d_measure_fp32_peak(device, buf.data_ptr(), n, C.byref(out)), "k2d_measure_fp32_peak")
+    return float(out.value)
 
 
 def first_outcomes(reward: np.ndarray, done: np.ndarray) -> np.ndarray:

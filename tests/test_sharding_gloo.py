@@ -58,3 +58,24 @@ def test_two_ranks_reproduce_one_process(tmp_path):
     assert np.array_equal(np.concatenate([p["r"] for p in parts], axis=1), r)
     assert np.array_equal(np.concatenate([p["d"] for p in parts], axis=1), d)
     assert d.sum() > N_ENVS            # resets happened, so the hash-based level draws were exercised
+
+
+def test_bench_starts_its_own_ranks_with_disjoint_env_ranges():
+    # `bench.py --gpus 2` outside torchrun starts two ranks itself; with --plan they do no GPU work, meet over gloo and rank 0
+    # prints who would step what: every rank its own RANK / LOCAL_RANK and a range of envs that no other rank has
+    import json
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "LOCAL_RANK", "WORLD_SIZE", "MASTER_ADDR", "MASTER_PORT")}
+    out = subprocess.run([sys.executable, os.path.join(root, "bench.py"), "--gpus", "2", "--plan", "--envs", "96"],
+                         capture_output=True, text=True, timeout=300, env=env)
+    assert out.returncode == 0, out.stderr[-2000:]
+    lines = [ln for ln in out.stdout.splitlines() if ln.startswith("{")]
+    assert len(lines) == 1                                   # rank 0 alone prints
+    plan = json.loads(lines[0])
+    assert plan["n_gpus"] == 2 and plan["total_envs"] == 192 and plan["scaling"] == "weak"
+    assert [(p["rank"], p["local_rank"]) for p in plan["plan"]] == [(0, 0), (1, 1)]
+    ranges = [range(p["env_offset"], p["env_offset"] + p["n_envs"]) for p in plan["plan"]]
+    assert set(ranges[0]).isdisjoint(ranges[1]) and len(set(ranges[0]) | set(ranges[1])) == 192
+    assert plan["shard_of_total"] == [[0, 96], [96, 96]]
