@@ -71,6 +71,13 @@ extern "C" {
  * gravity_y = -9.81, 8 solver iterations, contact_alpha = joint_alpha = 6 /s,
  * contact_beta = joint_beta = 0.1, joint_gamma = 6 /s, slop = 0.005 m,
  * restitution_threshold = 1 m/s, face_tol = 1e-3 m, motor_rho = 1, aabb_margin = 0.01 m, warm starting on. */
+/* solver_batch (paper, "Parallelised Computation and Batched Impulse Resolution"): the scene's manifold slots (two per
+ * polygon pair, one per other pair) are cut into ceil(n_slots / B) batches.  In every solver iteration, after the joints,
+ * the batches are solved one after the other; the rows of one batch are all solved against the velocities the batch
+ * starts with and applied together afterwards (in canonical order).  The active manifolds are spread over as many batches
+ * as possible: the i-th active manifold in canonical order goes to batch i mod n_batches.  While a scene has no more
+ * active manifolds than batches this is the sequential solve, bit for bit; the paper's default is B = 16.  The library
+ * runs this mode on its general, untuned path (constraint rows in the scratch tail); it is there for fidelity. */
 typedef struct k2d_config {
     int32_t n_envs;                /* >= 1                                                      */
     int32_t n_polygons;            /* 1 .. K2D_MAX_POLYGONS                                     */
@@ -100,6 +107,8 @@ typedef struct k2d_config {
     int64_t env_offset;            /* global index of env 0 (sharding over several GPUs)        */
     int32_t device;                /* CUDA device ordinal                                       */
     int32_t lanes_per_scene;       /* 0 = library default (32 for few envs, else 16); or 8, 16, 32 */
+    int32_t solver_batch;          /* 0 = contacts solved one after the other (default); B > 0 = the paper's batched solve, see below */
+    int32_t reserved;              /* 0 */
     void *cuda_stream;             /* cudaStream_t of the caller (NULL = default stream)        */
 } k2d_config;
 

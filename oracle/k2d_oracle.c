@@ -61,7 +61,7 @@ typedef struct { real x, y; } vec2;
 /* ---- configuration and raw level description (filled by the caller) ---- */
 typedef struct {
     int32_t n_polygons, n_circles, n_joints, n_thrusters, n_actions, n_levels, n_envs;
-    int32_t solver_iters, warm_start, auto_reset, max_episode_steps, broadphase, discrete_actions, frame_skip;
+    int32_t solver_iters, warm_start, auto_reset, max_episode_steps, broadphase, discrete_actions, frame_skip, solver_batch;
     real dt, gravity_y, contact_alpha, contact_beta, slop, restitution_threshold, face_tol;
     real joint_alpha, joint_beta, motor_rho, aabb_margin, joint_gamma, dense_kappa;
     uint64_t seed;
@@ -876,6 +876,46 @@ static void step_env(ref_sim *S, int e, const real *act, real *out_reward, uint8
                 angvel[q->a] = R_FMA(-lr, q->ia, angvel[q->a]);
                 angvel[q->b] = R_FMA(lr, q->ib, angvel[q->b]);
             }
+        }
+        /* Batched impulse resolution (paper, "Parallelised Computation and Batched Impulse Resolution"): the manifold
+         * slots are cut into batches of solver_batch; the rows of a batch are solved side by side, all against the
+         * velocities the batch starts with, and only then applied; batches follow one another.  The active manifolds
+         * are spread over as many batches as possible: the i-th active row (canonical order) goes to batch i mod
+         * n_batches.  With no more active rows than batches every batch holds one row and this is the sequential
+         * sweep below, operation for operation. */
+        if (cf->solver_batch > 0) {
+            const int n_batches = (S->n_slots + cf->solver_batch - 1) / cf->solver_batch;
+            real dn[256], dtan[256];
+            for (int b = 0; b < n_batches && b < n_rows; ++b) {
+                for (int i = b; i < n_rows; i += n_batches) {
+                    contact_row *r = &rows[i];
+                    /* private copies of the two bodies' velocities: the row's friction part sees its own normal impulse, nobody else's */
+                    real va[2] = { vel[2 * r->a], vel[2 * r->a + 1] }, vb[2] = { vel[2 * r->b], vel[2 * r->b + 1] };
+                    real wa = angvel[r->a], wb = angvel[r->b];
+                    real ma = inv_mass[r->a], mb = inv_mass[r->b];
+                    real vn = rel_vel(va, wa, vb, wb, r->n, r->rn_a, r->rn_b);
+                    real lam = (r->target - vn) * r->mass_n;
+                    real old = acc[2 * r->slot];
+                    real nw = rmax(old + lam, RC(0));
+                    acc[2 * r->slot] = nw;
+                    dn[i] = nw - old;
+                    apply_row(va, &wa, vb, &wb, ma, mb, dn[i], r->n, r->wn_a, r->wn_b);
+                    real vt = rel_vel(va, wa, vb, wb, r->t, r->rt_a, r->rt_b);
+                    real lamt = (-vt) * r->mass_t;
+                    real lim = r->mu * nw;
+                    real oldt = acc[2 * r->slot + 1];
+                    real nwt = rmax(rmin(oldt + lamt, lim), -lim);
+                    acc[2 * r->slot + 1] = nwt;
+                    dtan[i] = nwt - oldt;
+                }
+                for (int i = b; i < n_rows; i += n_batches) {
+                    contact_row *r = &rows[i];
+                    real ma = inv_mass[r->a], mb = inv_mass[r->b];
+                    apply_row(vel + 2 * r->a, &angvel[r->a], vel + 2 * r->b, &angvel[r->b], ma, mb, dn[i], r->n, r->wn_a, r->wn_b);
+                    apply_row(vel + 2 * r->a, &angvel[r->a], vel + 2 * r->b, &angvel[r->b], ma, mb, dtan[i], r->t, r->wt_a, r->wt_b);
+                }
+            }
+            continue;
         }
         for (int i = 0; i < n_rows; ++i) {
             contact_row *r = &rows[i];

@@ -16,7 +16,7 @@ _SRC = os.path.join(_HERE, "k2d_oracle.c")
 _LIBS = {}
 
 DEFAULTS = dict(
-    solver_iters=8, warm_start=1, auto_reset=0, max_episode_steps=0, broadphase=1, discrete_actions=0, frame_skip=1,
+    solver_iters=8, warm_start=1, auto_reset=0, max_episode_steps=0, broadphase=1, discrete_actions=0, frame_skip=1, solver_batch=0,
     dt=1.0 / 60.0, gravity_y=-9.81, contact_alpha=6.0, contact_beta=0.1, slop=0.005,
     restitution_threshold=1.0, face_tol=1e-3, joint_alpha=6.0, joint_beta=0.1, joint_gamma=6.0, dense_kappa=0.0, motor_rho=1.0,
     aabb_margin=0.01, seed=0, env_offset=0,
@@ -25,7 +25,7 @@ DEFAULTS = dict(
 _REAL_FIELDS = ("dt", "gravity_y", "contact_alpha", "contact_beta", "slop", "restitution_threshold", "face_tol",
                 "joint_alpha", "joint_beta", "motor_rho", "aabb_margin", "joint_gamma", "dense_kappa")
 _INT_FIELDS = ("n_polygons", "n_circles", "n_joints", "n_thrusters", "n_actions", "n_levels", "n_envs",
-               "solver_iters", "warm_start", "auto_reset", "max_episode_steps", "broadphase", "discrete_actions", "frame_skip")
+               "solver_iters", "warm_start", "auto_reset", "max_episode_steps", "broadphase", "discrete_actions", "frame_skip", "solver_batch")
 
 _LEVEL_REAL = ("poly_verts", "circle_radius", "pos", "angle", "vel", "angvel", "density", "friction", "restitution",
                "joint_anchor_a", "joint_anchor_b", "motor_speed", "motor_power", "joint_fixed_angle", "joint_min", "joint_max",

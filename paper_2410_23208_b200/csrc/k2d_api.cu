@@ -58,7 +58,7 @@ static int check_config(const k2d_config *c) {
         c->n_actions < 1 || c->n_actions > kMaxActions || c->n_levels < 1 || c->solver_iters < 0 || c->solver_iters > 1024 ||
         (c->warm_start != 0 && c->warm_start != 1) || c->auto_reset < 0 || c->auto_reset > 2 || c->max_episode_steps < 0 ||
         c->max_fused_steps < 1 || c->frame_skip < 1 || c->device < 0 ||
-        !(c->lanes_per_scene == 0 || c->lanes_per_scene == 8 || c->lanes_per_scene == 16 || c->lanes_per_scene == 32))
+        !(c->lanes_per_scene == 0 || c->lanes_per_scene == 8 || c->lanes_per_scene == 16 || c->lanes_per_scene == 32) || c->solver_batch < 0)
         return K2D_ERR_CONFIG;
     const float f[] = { c->dt, c->gravity_y, c->contact_alpha, c->contact_beta, c->slop, c->restitution_threshold, c->face_tol,
                         c->joint_alpha, c->joint_beta, c->motor_rho, c->aabb_margin, c->joint_gamma, c->dense_kappa };
@@ -307,6 +307,11 @@ static StepParams step_params(const k2d_state *s, const float *dev_actions, int 
     prm.obs = nullptr; prm.n_polygons = c.n_polygons; prm.n_circles = c.n_circles; prm.n_joints = c.n_joints; prm.n_thrusters = c.n_thrusters;
     prm.discrete = discrete; prm.dense_kappa = c.dense_kappa; prm.frame_skip = c.frame_skip;
     prm.chunk_steps = n_steps; prm.n_chunks = 1; prm.wait_limit = s->wait_limit;
+    {
+        const int n_slots = c.n_polygons * (c.n_polygons - 1) + c.n_polygons * c.n_circles + c.n_circles * (c.n_circles - 1) / 2;
+        prm.n_batches = c.solver_batch > 0 ? (n_slots + c.solver_batch - 1) / c.solver_batch : 0;
+        if (c.solver_batch > 0 && prm.n_batches < 1) prm.n_batches = 1;
+    }
     if (c.n_envs > s->groups && n_steps > kChunkSteps) {
         const int n_chunks = (n_steps + kChunkSteps - 1) / kChunkSteps;
         if ((unsigned long long)c.n_envs * (unsigned long long)n_chunks + (unsigned long long)s->groups < 0xffffffffULL) {

@@ -150,6 +150,7 @@ struct StepParams {
     int n_envs, n_steps, n_actions, n_levels;
     int chunk_steps, n_chunks;   // a launch is cut into n_chunks pieces of chunk_steps steps; work items are (chunk, env)
     unsigned wait_limit;         // polls before a wait for another group's chunk gives up
+    int n_batches;               // batched contact solve: number of batches the manifold slots are cut into (0: the sequential sweep)
     int solver_iters, warm_start, auto_reset, max_episode_steps;
     int discrete;             // actions are int32 codes (multi-discrete action space) instead of floats
     int frame_skip;           // engine steps each action row is held for
@@ -566,12 +567,88 @@ __device__ __forceinline__ void slow_sweep_pairs(float *sm, uint32_t *ovf, int n
     }
 }
 
+// ---- batched contact solve (paper, "Parallelised Computation and Batched Impulse Resolution"): the i-th active manifold
+// (canonical order) belongs to batch i mod n_batches; the rows of a batch are all solved against the velocities the batch
+// starts with, then applied; batches follow one another.  One iteration over the memory records in scratch; the warm
+// entries of the scratch, free between the pre-step and the end of the step, hold per record the rank of its first
+// manifold and the impulses to apply.
+__device__ __forceinline__ void apply_impulse(float d, float dx, float dy, float ma, float mb, float lev_a, float lev_b,
+                                              float &vax, float &vay, float &wa, float &vbx, float &vby, float &wb) {
+    const float px = d * dx, py = d * dy;
+    vax = __fmaf_rn(-ma, px, vax); vay = __fmaf_rn(-ma, py, vay); wa = __fmaf_rn(-lev_a, d, wa);
+    vbx = __fmaf_rn(mb, px, vbx); vby = __fmaf_rn(mb, py, vby); wb = __fmaf_rn(lev_b, d, wb);
+}
+template <class SC, int G>
+__device__ __noinline__ void slow_batched_iteration(float *sm, uint32_t *ovf, int nrec, int cmax, int nman, int n_batches) {
+    Group<G> g;
+    uint32_t *aux = ovf + SC::SCRATCH_WARM;
+    const int nb_used = nman < n_batches ? nman : n_batches;
+    for (int bt = 0; bt < nb_used; ++bt) {
+        // every row of the batch against the velocities as they stand: impulses and accumulated impulses, no velocity is written
+        for (int k = g.lane; k < nrec; k += G) {
+            uint32_t *r = ovf + (size_t)k * kRecWords;
+            RecM c;
+            recm_load(r, c);
+            const int a = c.ab & 31, b = (c.ab >> 5) & 31;
+            const unsigned amask = (c.ab >> 10) & 3u;
+            const int rank0 = (int)aux[kWarmWords * k];
+            const float ma = sm[SC::BIM + a], mb = sm[SC::BIM + b], ia = sm[SC::BII + a], ib = sm[SC::BII + b];
+            const float4 va4 = ld4(sm + SC::BVEL + 4 * a), vb4 = ld4(sm + SC::BVEL + 4 * b);
+#pragma unroll 1
+            for (int mi = 0; mi < 2; ++mi) {
+                if (!(amask & (1u << mi))) continue;
+                const int rank = rank0 + ((mi == 1 && (amask & 1u)) ? 1 : 0);
+                if (rank % n_batches != bt) continue;
+                float vax = va4.x, vay = va4.y, wa = va4.z, vbx = vb4.x, vby = vb4.y, wb = vb4.z;
+                const float old_n = c.accn[mi], old_t = c.acct[mi];
+                manifold_rows<1>(c.nx, c.ny, c.mu, ma, mb, ia, ib, c.rna[mi], c.rnb[mi], c.rta[mi], c.rtb[mi], c.massn[mi], c.masst[mi],
+                                 c.target[mi], c.accn[mi], c.acct[mi], vax, vay, wa, vbx, vby, wb);
+                r[R_M0 + mi * M_WORDS + M_ACCN] = __float_as_uint(c.accn[mi]);
+                r[R_M0 + mi * M_WORDS + M_ACCT] = __float_as_uint(c.acct[mi]);
+                aux[kWarmWords * k + 1 + 2 * mi] = __float_as_uint(c.accn[mi] - old_n);
+                aux[kWarmWords * k + 2 + 2 * mi] = __float_as_uint(c.acct[mi] - old_t);
+            }
+        }
+        g.sync();
+        // the batch's impulses, applied in canonical order per body: level by level
+        for (int lvl = 1; lvl <= cmax; ++lvl) {
+            for (int k = g.lane; k < nrec; k += G) {
+                const uint32_t *r = ovf + (size_t)k * kRecWords;
+                const uint32_t ab = r[R_AB];
+                if (((ab >> 19) & 127u) != (unsigned)lvl) continue;
+                const unsigned amask = (ab >> 10) & 3u;
+                const int rank0 = (int)aux[kWarmWords * k];
+                const bool in0 = (amask & 1u) && rank0 % n_batches == bt;
+                const bool in1 = (amask & 2u) && (rank0 + ((amask & 1u) ? 1 : 0)) % n_batches == bt;
+                if (!in0 && !in1) continue;
+                const int a = ab & 31, b = (ab >> 5) & 31;
+                const float nx = __uint_as_float(r[R_NX]), ny = __uint_as_float(r[R_NY]);
+                const float ma = sm[SC::BIM + a], mb = sm[SC::BIM + b], ia = sm[SC::BII + a], ib = sm[SC::BII + b];
+                const float4 va4 = ld4(sm + SC::BVEL + 4 * a), vb4 = ld4(sm + SC::BVEL + 4 * b);
+                float vax = va4.x, vay = va4.y, wa = va4.z, vbx = vb4.x, vby = vb4.y, wb = vb4.z;
+#pragma unroll 1
+                for (int mi = 0; mi < 2; ++mi) {
+                    if (!(mi ? in1 : in0)) continue;
+                    const uint32_t *m = r + R_M0 + mi * M_WORDS;
+                    const float rna = __uint_as_float(m[M_RNA]), rnb = __uint_as_float(m[M_RNB]), rta = __uint_as_float(m[M_RTA]), rtb = __uint_as_float(m[M_RTB]);
+                    const float dn = __uint_as_float(aux[kWarmWords * k + 1 + 2 * mi]), dt_ = __uint_as_float(aux[kWarmWords * k + 2 + 2 * mi]);
+                    apply_impulse(dn, nx, ny, ma, mb, ia * rna, ib * rnb, vax, vay, wa, vbx, vby, wb);
+                    apply_impulse(dt_, -ny, nx, ma, mb, ia * rta, ib * rtb, vax, vay, wa, vbx, vby, wb);
+                }
+                if ((ab >> 26) & 1u) st4(sm + SC::BVEL + 4 * a, vax, vay, wa);
+                if ((ab >> 27) & 1u) st4(sm + SC::BVEL + 4 * b, vbx, vby, wb);
+            }
+            g.sync();
+        }
+    }
+}
+
 // Records from the staged manifolds (the first G in shared memory, the rest already in scratch),
 // their levels, warm start and all solver iterations, joints included.  old_n / old_t: this lane's
 // first-manifold accumulated impulses of the previous step.  Returns the highest contact level.
 template <class SC, int G>
 __device__ __noinline__ int slow_solve(float *sm, uint32_t *ovf, int nrec, uint32_t jab, int jlevel, int jmax,
-                                       int solver_iters, int warm_start, float motor_rho, float old_n, float old_t, ContactConsts cc) {
+                                       int solver_iters, int warm_start, float motor_rho, float old_n, float old_t, ContactConsts cc, int n_batches) {
     Group<G> g;
     const int lane = g.lane;
     uint32_t *smu = reinterpret_cast<uint32_t *>(sm);
@@ -586,8 +663,8 @@ __device__ __noinline__ int slow_solve(float *sm, uint32_t *ovf, int nrec, uint3
         uint32_t *r = ovf + (size_t)lane * kRecWords, *r2 = ovf + (size_t)(G + lane) * kRecWords;
 #pragma unroll
         for (int f = 0; f < kStageWords; ++f) {
-            r[f] = smu[SC::STG + f * G + lane];
-            if (lane < G / 2) r2[f] = smu[SC::STG + LF_COUNT * G + ovs(f) * (G / 2) + lane];
+            if (lane < nrec) r[f] = smu[SC::STG + f * G + lane];
+            if (lane < G / 2 && G + lane < nrec) r2[f] = smu[SC::STG + LF_COUNT * G + ovs(f) * (G / 2) + lane];
         }
     }
     g.sync();
@@ -628,11 +705,24 @@ __device__ __noinline__ int slow_solve(float *sm, uint32_t *ovf, int nrec, uint3
         }
     }
     g.sync();
+    int nman = 0;
+    if (n_batches > 0) {
+        // rank of every record's first manifold among the active manifolds, in canonical order
+        if (lane == 0) {
+            for (int k = 0; k < nrec; ++k) {
+                ovf[SC::SCRATCH_WARM + kWarmWords * k] = (uint32_t)nman;
+                nman += __popc((ovf[(size_t)k * kRecWords + R_AB] >> 10) & 3u);
+            }
+        }
+        g.sync();
+        nman = g.shfl(nman, 0);
+    }
     slow_sweep_pairs<SC, G, 0>(sm, ovf, nrec, cmax);
     sweep_joints<SC, G, 0>(sm, jab, lane, jlevel, jmax, motor_rho);
     for (int it = 0; it < solver_iters; ++it) {
         sweep_joints<SC, G, 1>(sm, jab, lane, jlevel, jmax, motor_rho);
-        slow_sweep_pairs<SC, G, 1>(sm, ovf, nrec, cmax);
+        if (n_batches > 0) slow_batched_iteration<SC, G>(sm, ovf, nrec, cmax, nman, n_batches);
+        else slow_sweep_pairs<SC, G, 1>(sm, ovf, nrec, cmax);
     }
     return cmax;
 }
@@ -1366,11 +1456,12 @@ struct Scene {
         g.sync();
         c_rec += (unsigned)nrec << 16;
 
-        const bool overflow = nrec > G + G / 2;
+        // crowded scenes, and every scene with contacts when the batched contact solve is asked for, go through the memory records
+        const bool overflow = nrec > G + G / 2 || (prm.n_batches > 0 && nrec > 0);
         int cmax = 0, clevel = 0, clevel2 = 0;
         if (overflow) {
             cmax = slow_solve<SC, G>(sm, ovf, nrec, jab, jlevel, jmax, prm.solver_iters, prm.warm_start, prm.motor_rho,
-                                     rec.accn, rec.acct, contact_consts());
+                                     rec.accn, rec.acct, contact_consts(), prm.n_batches);
         } else {
             const ContactConsts cc = contact_consts();
             const bool two = nrec > G;      // some lanes get a second record
@@ -1492,10 +1583,14 @@ struct Scene {
             c_man += (unsigned)slow_finish<SC, G>(sm, ovf, nrec);
             // the first G + G / 2 pairs go back to their lanes
             const uint32_t *wr = ovf + SC::SCRATCH_WARM + (size_t)lane * kWarmWords, *wr2 = wr + (size_t)G * kWarmWords;
-            rec.ab = wr[0] << 12;
-            rec.accn = __uint_as_float(wr[1]); rec.acct = __uint_as_float(wr[2]);
-            lanef(LF_ACC2N) = __uint_as_float(wr[3]); lanef(LF_ACC2T) = __uint_as_float(wr[4]);
-            if (lane < G / 2) {
+            rec.ab = 0u; rec.accn = 0.0f; rec.acct = 0.0f;
+            lanef(LF_ACC2N) = 0.0f; lanef(LF_ACC2T) = 0.0f;
+            if (lane < nrec) {
+                rec.ab = wr[0] << 12;
+                rec.accn = __uint_as_float(wr[1]); rec.acct = __uint_as_float(wr[2]);
+                lanef(LF_ACC2N) = __uint_as_float(wr[3]); lanef(LF_ACC2T) = __uint_as_float(wr[4]);
+            }
+            if (lane < G / 2 && G + lane < nrec) {
                 ovl(R_AB) = __uint_as_float(wr2[0] << 12);
                 ovl(OV_ACC0N) = __uint_as_float(wr2[1]); ovl(OV_ACC0T) = __uint_as_float(wr2[2]);
                 ovl(OV_ACC1N) = __uint_as_float(wr2[3]); ovl(OV_ACC1T) = __uint_as_float(wr2[4]);

@@ -31,7 +31,7 @@ class Config(C.Structure):
         [(n, C.c_float) for n in ("dt", "gravity_y", "contact_alpha", "contact_beta", "slop", "restitution_threshold",
                                   "face_tol", "joint_alpha", "joint_beta", "motor_rho", "aabb_margin", "joint_gamma", "dense_kappa")] +
         [("seed", C.c_uint64), ("env_offset", C.c_int64), ("device", C.c_int32), ("lanes_per_scene", C.c_int32),
-         ("cuda_stream", C.c_void_p)])
+         ("solver_batch", C.c_int32), ("reserved", C.c_int32), ("cuda_stream", C.c_void_p)])
 
 
 LEVEL_DTYPE = np.dtype([

@@ -13,7 +13,7 @@ META_KEYS = ("step_count", "episode_count", "level_id", "status")
 
 ORACLE_CFG = ("solver_iters", "warm_start", "auto_reset", "max_episode_steps", "dt", "gravity_y", "contact_alpha",
               "contact_beta", "slop", "restitution_threshold", "face_tol", "joint_alpha", "joint_beta", "joint_gamma", "motor_rho",
-              "aabb_margin", "dense_kappa", "seed", "env_offset", "frame_skip", "n_actions")
+              "aabb_margin", "dense_kappa", "seed", "env_offset", "frame_skip", "n_actions", "solver_batch")
 
 
 def make_pair(levels, n_envs, broadphase=0, **cfg):

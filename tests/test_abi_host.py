@@ -24,7 +24,7 @@ def test_library_exports_every_declared_symbol():
 
 def test_struct_layouts_match_the_header():
     # sizes computed from the header's field lists
-    assert C.sizeof(k2d.Config) == 13 * 4 + 13 * 4 + 8 + 8 + 4 + 4 + 8
+    assert C.sizeof(k2d.Config) == 13 * 4 + 13 * 4 + 8 + 8 + 4 + 4 + 4 + 4 + 8
     n_float = 12 * 4 * 2 + 4 + 16 * 2 + 16 + 16 * 2 + 16 + 3 * 16 + 6 * 2 * 2 + 6 * 2 + 6 * 3 + 2 * 2 + 2 + 2
     n_int = 12 + 3 * 16 + 2 * 6 + 2 * 6 + 2 * 6 + 2 + 2 * 2
     assert k2d.LEVEL_DTYPE.itemsize == 4 * (n_float + n_int)

@@ -288,6 +288,31 @@ def test_step_with_observation_in_one_launch(size, n_envs, lanes, n_actions):
     assert exact, err
 
 
+@pytest.mark.parametrize("size,n_envs,lanes,batch", [("L", 72, 16, 16), ("L", 48, 32, 4), ("L", 24, 8, 1000), ("M", 48, 0, 16), ("S", 40, 0, 2), ("L", 40, 16, 1)])
+def test_batched_contact_solve_matches_the_oracle(size, n_envs, lanes, batch):
+    # the paper's batched impulse resolution (batches of `batch` manifold slots, rows of a batch solved side by side);
+    # a quarter of the scenes crowded, so that batches really hold several rows; batches of one slot are the sequential solve
+    lv = scenes.make_levels(size, n_envs, 16, static_prob=0.1, triangle_prob=0.2, fixed_prob=0.2)
+    lv["pos"][: n_envs // 4, 1:, 0] *= 0.15
+    env, ref = parity.make_pair(lv, n_envs, solver_batch=batch, lanes_per_scene=lanes, auto_reset=2, max_episode_steps=30, seed=8)
+    act = scenes.make_actions(50, n_envs, env.n_actions, 16)
+    (r, d), (rr, dr) = parity.step_both(env, ref, act[:1])
+    err, exact = parity.errors(env, ref)
+    _check_tolerances(err, 1)
+    assert exact, err
+    (r, d), (rr, dr) = parity.step_both(env, ref, act[1:], chunk=7)
+    err, exact = parity.errors(env, ref)
+    assert exact, err
+    assert np.array_equal(r, rr) and np.array_equal(d, dr)
+    assert parity.counters_match(env, ref)
+    seq = k2d_ref.RefSim(lv, n_envs, auto_reset=2, max_episode_steps=30, seed=8)
+    seq.step(act)
+    if batch == 1:
+        assert np.array_equal(seq.pos, ref.pos)          # batches of one slot: the sequential solve
+    if batch >= 16:
+        assert not np.array_equal(seq.pos, ref.pos)      # few batches: crowded scenes take another course
+
+
 def test_non_finite_state_is_flagged_not_propagated():
     lv = scenes.make_levels("S", 8, 81)
     env, ref = parity.make_pair(lv, 8)
