@@ -223,7 +223,7 @@ def run_gpu(args) -> dict:
     # weak scaling: every rank steps its own n_envs; env_offset makes level draws global
     env = k2d.Env(levels, n_envs, device=local, auto_reset=w["auto_reset"], max_episode_steps=w["max_episode_steps"],
                   seed=scenes.workload_seed(args.workload), env_offset=rank * n_envs, max_fused_steps=FUSED,
-                  lanes_per_scene=args.lanes)
+                  lanes_per_scene=args.lanes, solver_batch=args.solver_batch)
     K, W = args.steps, args.warmup
     n_bufs = max(K, 1)
     host_actions = [torch.from_numpy(scenes.make_actions(FUSED, n_envs, dims.n_actions, 100 + rank * 1000 + i)).pin_memory()
@@ -397,6 +397,7 @@ def run_gpu(args) -> dict:
                                f"(config {args.workload}: pool of {w['n_levels']} levels, horizon {w['max_episode_steps']})",
                    "lanes_per_scene": env.cfg.lanes_per_scene or (32 if n_envs < (48 if w["size"] == "L" else 24) * torch.cuda.get_device_properties(dev).multi_processor_count else 16), "fused_steps": FUSED,
                    "observation": "pixels 125x125 RGBA (k2d_render)" if args.pixels else "symbolic entity rows (k2d_obs)",
+                   "solver_batch": args.solver_batch,
                    "l2": "flushed between timed iterations (256 MiB write, untimed); K distinct action buffers"},
         "clocks": clk,
         "e2e": {"value": e2e_value, "unit": UNIT,
@@ -473,6 +474,7 @@ def main():
     ap.add_argument("--lanes", type=int, default=0, help="lanes per scene (0 = library default)")
     ap.add_argument("--fused", type=int, default=FUSED, help="engine steps per k2d_step launch (1 = one launch and one observation per step)")
     ap.add_argument("--pixels", action="store_true", help="the observation of a bench step is the 125 x 125 pixel image (k2d_render) instead of the entity rows")
+    ap.add_argument("--solver-batch", type=int, default=0, help="the paper's batched contact solve with batches of this many manifold slots (0 = sequential)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--plan", action="store_true", help="no GPU work: the ranks rendezvous over gloo and rank 0 prints which envs each would step")
     args = ap.parse_args()

@@ -48,6 +48,7 @@ extern "C" {
 #define K2D_ERR_ARG (-7)           /* another argument is invalid                        */
 #define K2D_ERR_LIMIT (-8)         /* a size is beyond a limit built into the library    */
 #define K2D_ERR_WAIT (-9)          /* k2d_status: a wait inside k2d_step ran out (see there) */
+#define K2D_ERR_CHECK (-10)        /* k2d_status of a checked build: an index was out of range    */
 
 #define K2D_MAX_POLYGONS 12
 #define K2D_MAX_CIRCLES 4
@@ -259,6 +260,12 @@ int k2d_level_info(const k2d_config *cfg, const k2d_level *host_level, float *ho
  * (slots indexed in the library's internal size class, see k2d_trace_slots). */
 int k2d_set_trace(k2d_state *s, float *dev_trace);
 int k2d_trace_slots(const k2d_state *s);
+
+/* 1 if the library was compiled with -DK2D_CHECKED, else 0.  The checked build compares every index its kernels unpack
+ * from packed words or read from tables (bodies, pairs, memory records, level ids, warm entries, solver levels, scratch
+ * slots, counts) with its limit; a violation is recorded (k2d_status then returns K2D_ERR_CHECK until the next
+ * k2d_reset) and the access is redirected to index 0; nothing traps.  It stands in for a memory checker. */
+int k2d_is_checked_build(void);
 
 /* Test aid.  With more envs than the device holds scene groups, k2d_step hands out runs of 8 steps of an env to whichever
  * group is free; a group that gets a later run of an env before the earlier one is back in memory polls for it, about

@@ -306,7 +306,7 @@ static StepParams step_params(const k2d_state *s, const float *dev_actions, int 
     prm.n_envs = c.n_envs; prm.n_steps = n_steps; prm.n_actions = c.n_actions; prm.n_levels = c.n_levels;
     prm.obs = nullptr; prm.n_polygons = c.n_polygons; prm.n_circles = c.n_circles; prm.n_joints = c.n_joints; prm.n_thrusters = c.n_thrusters;
     prm.discrete = discrete; prm.dense_kappa = c.dense_kappa; prm.frame_skip = c.frame_skip;
-    prm.chunk_steps = n_steps; prm.n_chunks = 1; prm.wait_limit = s->wait_limit;
+    prm.chunk_steps = n_steps; prm.n_chunks = 1; prm.wait_limit = s->wait_limit; prm.n_slots = scratch == s->dev_scratch ? s->slots : K2D_STATIC_SCRATCH_MAX_ENVS;
     {
         const int n_slots = c.n_polygons * (c.n_polygons - 1) + c.n_polygons * c.n_circles + c.n_circles * (c.n_circles - 1) / 2;
         prm.n_batches = c.solver_batch > 0 ? (n_slots + c.solver_batch - 1) / c.solver_batch : 0;
@@ -446,6 +446,9 @@ int k2d_reset(k2d_state *s, const int32_t *host_level_ids) {
         for (int e = 0; e < E; ++e) if (host_level_ids[e] < 0 || host_level_ids[e] >= s->cfg.n_levels) return K2D_ERR_ARG;
     CUDA_OK(cudaSetDevice(s->cfg.device));
     CUDA_OK(cudaMemsetAsync(s->dev_base, 0, kCtrlBytes, s->stream));
+#ifdef K2D_CHECKED
+    { const unsigned int zero = 0u; CUDA_OK(cudaMemcpyToSymbolAsync(k2d_check_bits, &zero, sizeof(zero), 0, cudaMemcpyHostToDevice, s->stream)); }
+#endif
     CUDA_OK(cudaMemsetAsync(s->dev_chunks, 0, (size_t)E * 4, s->stream));
     if (host_level_ids) CUDA_OK(cudaMemcpyAsync(s->dev_ids, host_level_ids, (size_t)E * 4, cudaMemcpyHostToDevice, s->stream));
     const int *ids = host_level_ids ? s->dev_ids : nullptr;
@@ -598,6 +601,11 @@ int k2d_status(k2d_state *s, int64_t *host_counts) {
     CUDA_OK(cudaMemcpy(host_counts, s->dev_counters, 8 * sizeof(int64_t), cudaMemcpyDeviceToHost));
     unsigned int queue[4] = { 0u, 0u, 0u, 0u };
     CUDA_OK(cudaMemcpy(queue, s->dev_queue, sizeof(queue), cudaMemcpyDeviceToHost));
+#ifdef K2D_CHECKED
+    unsigned int bits = 0u;
+    CUDA_OK(cudaMemcpyFromSymbol(&bits, k2d_check_bits, sizeof(bits)));
+    if (bits) { std::fprintf(stderr, "k2d_status: index checks failed, bits 0x%x\n", bits); return K2D_ERR_CHECK; }
+#endif
     return queue[Q_ERROR] ? K2D_ERR_WAIT : K2D_OK;
 }
 
@@ -633,6 +641,14 @@ int k2d_set_trace(k2d_state *s, float *dev_trace) {
 }
 
 int k2d_trace_slots(const k2d_state *s) { return s ? s->ci.NSLOTS : 0; }
+
+int k2d_is_checked_build(void) {
+#ifdef K2D_CHECKED
+    return 1;
+#else
+    return 0;
+#endif
+}
 
 int k2d_set_wait_limit(k2d_state *s, uint32_t polls) {
     if (!s) return K2D_ERR_NULL;
@@ -730,6 +746,7 @@ const char *k2d_error_string(int code) {
         case K2D_ERR_CUDA: return "CUDA runtime error";
         case K2D_ERR_ARG: return "invalid argument";
         case K2D_ERR_LIMIT: return "size beyond a built-in limit";
+        case K2D_ERR_CHECK: return "an index check of the checked build failed";
         case K2D_ERR_WAIT: return "a scene group gave up waiting for another; the last step is incomplete";
         default: return "unknown error";
     }

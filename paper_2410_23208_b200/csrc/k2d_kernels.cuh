@@ -150,6 +150,7 @@ struct StepParams {
     int n_envs, n_steps, n_actions, n_levels;
     int chunk_steps, n_chunks;   // a launch is cut into n_chunks pieces of chunk_steps steps; work items are (chunk, env)
     unsigned wait_limit;         // polls before a wait for another group's chunk gives up
+    int n_slots;                 // scratch slots the caller's buffer holds (one per resident scene group)
     int n_batches;               // batched contact solve: number of batches the manifold slots are cut into (0: the sequential sweep)
     int solver_iters, warm_start, auto_reset, max_episode_steps;
     int discrete;             // actions are int32 codes (multi-discrete action space) instead of floats
@@ -159,6 +160,24 @@ struct StepParams {
     unsigned long long seed;
     long long env_offset;
 };
+
+// ---------------------------------------------------------------- index checks of the checked build
+// With -DK2D_CHECKED every index that is unpacked from a packed word or read from a table (bodies, pairs, memory records,
+// level ids, warm entries, solver levels, scratch slots, counts) is compared with its limit before it is used; a violation
+// sets a bit in k2d_check_bits, which k2d_status reports, and the access goes to index 0 instead.  Nothing traps.  In the
+// ordinary build the checks compile to nothing.
+enum { CK_BODY = 0, CK_PAIR, CK_RECORD, CK_LEVEL_ID, CK_COUNT, CK_SLOT, CK_WARM, CK_SOLVER_LEVEL, CK_STAGE, CK_OBS };
+#ifdef K2D_CHECKED
+__device__ unsigned int k2d_check_bits;
+template <int CODE>
+__device__ __forceinline__ int ck_idx(int v, int limit) {
+    if ((unsigned)v >= (unsigned)limit) { atomicOr(&k2d_check_bits, 1u << CODE); return 0; }
+    return v;
+}
+#else
+template <int CODE>
+__device__ __forceinline__ int ck_idx(int v, int) { return v; }
+#endif
 
 // ---------------------------------------------------------------- exact helpers
 __device__ __forceinline__ float fmin_cmp(float a, float b) { return a < b ? a : b; }
@@ -390,11 +409,11 @@ __device__ __noinline__ float2 angular_row(float *jr, float ia, float ib, float 
 // 2: positional correction, 3: motor
 template <class SC, int MODE>
 __device__ __forceinline__ void visit_joint(float *sm, uint32_t jab, int j, float motor_rho, int discrete = 0) {
-    const int a = jab & 255, b = (jab >> 8) & 255;
+    const int a = ck_idx<CK_BODY>(jab & 255, SC::N), b = ck_idx<CK_BODY>((jab >> 8) & 255, SC::N);
     const bool dyn_a = (jab >> 29) & 1u, dyn_b = (jab >> 30) & 1u;
     float *jr = sm + SC::JROW + kJointWords * j;
     if (MODE == 3) {
-        const float av = sm[SC::ACT + ((jab >> 16) & 255)];
+        const float av = sm[SC::ACT + ck_idx<CK_COUNT>((jab >> 16) & 255, kMaxActions)];
         // paper, "Action Space": continuous in [-1, 1], or multi-discrete codes 0 off, 1 forwards, 2 backwards at full power
         const float A = discrete ? (__float_as_int(av) == 1 ? 1.0f : (__float_as_int(av) == 2 ? -1.0f : 0.0f))
                                  : fmax_cmp(fmin_cmp(av, 1.0f), -1.0f);
@@ -462,6 +481,7 @@ __device__ __forceinline__ void sweep_joints(float *sm, uint32_t jab, int lane, 
 template <class SC, int G>
 __device__ __forceinline__ void warm_lookup(const Group<G> &g, const float *sm, const uint32_t *ovf, int wi, float old_n, float old_t,
                                             int warm_start, float (&w)[4]) {
+    wi = (wi == 255) ? 255 : ck_idx<CK_WARM>(wi, SC::NPAIRS);
     const int src = (wi < G) ? wi : 0;
     const float *lf = sm + SC::STG;
     w[0] = g.shflf(old_n, src); w[1] = g.shflf(old_t, src);
@@ -490,15 +510,15 @@ __device__ __noinline__ int levels_by_one_lane(uint32_t *smu, uint32_t *ovf, int
     for (int i = 0; i < SC::N; ++i) bl[i] = 0;
     for (int k = 0; k < nrec; ++k) {
         uint32_t *w = (k < G) ? (smu + SC::STG + S_AB * G + k)
-                    : (k < G + G / 2) ? (smu + SC::STG + LF_COUNT * G + ovs(S_AB) * (G / 2) + (k - G)) : (ovf + (size_t)k * kRecWords + S_AB);
+                    : (k < G + G / 2) ? (smu + SC::STG + LF_COUNT * G + ovs(S_AB) * (G / 2) + (k - G)) : (ovf + (size_t)ck_idx<CK_RECORD>(k, SC::NPAIRS) * kRecWords + S_AB);
         const uint32_t ab = *w;
-        const int a = ab & 31, b = (ab >> 5) & 31;
+        const int a = ck_idx<CK_BODY>(ab & 31, SC::N), b = ck_idx<CK_BODY>((ab >> 5) & 31, SC::N);
         int lvl = 1;
         if ((ab >> 26) & 1u) lvl = max(lvl, bl[a] + 1);
         if ((ab >> 27) & 1u) lvl = max(lvl, bl[b] + 1);
         if ((ab >> 26) & 1u) bl[a] = (uint8_t)lvl;
         if ((ab >> 27) & 1u) bl[b] = (uint8_t)lvl;
-        *w = ab | ((uint32_t)lvl << 19);
+        *w = ab | ((uint32_t)ck_idx<CK_SOLVER_LEVEL>(lvl, 128) << 19);
         cmax = max(cmax, lvl);
     }
     return cmax;
@@ -537,11 +557,11 @@ __device__ __forceinline__ void slow_sweep_pairs(float *sm, uint32_t *ovf, int n
     Group<G> g;
     for (int lvl = 1; lvl <= cmax; ++lvl) {
         for (int k = g.lane; k < nrec; k += G) {
-            uint32_t *r = ovf + (size_t)k * kRecWords;
+            uint32_t *r = ovf + (size_t)ck_idx<CK_RECORD>(k, SC::NPAIRS) * kRecWords;
             if (((r[R_AB] >> 19) & 127u) != (unsigned)lvl) continue;
             RecM c;
             recm_load(r, c);
-            const int a = c.ab & 31, b = (c.ab >> 5) & 31;
+            const int a = ck_idx<CK_BODY>(c.ab & 31, SC::N), b = ck_idx<CK_BODY>((c.ab >> 5) & 31, SC::N);
             const unsigned amask = (c.ab >> 10) & 3u;
             const bool dyn_a = (c.ab >> 26) & 1u, dyn_b = (c.ab >> 27) & 1u;
             const float ma = sm[SC::BIM + a], mb = sm[SC::BIM + b];
@@ -586,10 +606,10 @@ __device__ __noinline__ void slow_batched_iteration(float *sm, uint32_t *ovf, in
     for (int bt = 0; bt < nb_used; ++bt) {
         // every row of the batch against the velocities as they stand: impulses and accumulated impulses, no velocity is written
         for (int k = g.lane; k < nrec; k += G) {
-            uint32_t *r = ovf + (size_t)k * kRecWords;
+            uint32_t *r = ovf + (size_t)ck_idx<CK_RECORD>(k, SC::NPAIRS) * kRecWords;
             RecM c;
             recm_load(r, c);
-            const int a = c.ab & 31, b = (c.ab >> 5) & 31;
+            const int a = ck_idx<CK_BODY>(c.ab & 31, SC::N), b = ck_idx<CK_BODY>((c.ab >> 5) & 31, SC::N);
             const unsigned amask = (c.ab >> 10) & 3u;
             const int rank0 = (int)aux[kWarmWords * k];
             const float ma = sm[SC::BIM + a], mb = sm[SC::BIM + b], ia = sm[SC::BII + a], ib = sm[SC::BII + b];
@@ -613,7 +633,7 @@ __device__ __noinline__ void slow_batched_iteration(float *sm, uint32_t *ovf, in
         // the batch's impulses, applied in canonical order per body: level by level
         for (int lvl = 1; lvl <= cmax; ++lvl) {
             for (int k = g.lane; k < nrec; k += G) {
-                const uint32_t *r = ovf + (size_t)k * kRecWords;
+                const uint32_t *r = ovf + (size_t)ck_idx<CK_RECORD>(k, SC::NPAIRS) * kRecWords;
                 const uint32_t ab = r[R_AB];
                 if (((ab >> 19) & 127u) != (unsigned)lvl) continue;
                 const unsigned amask = (ab >> 10) & 3u;
@@ -621,7 +641,7 @@ __device__ __noinline__ void slow_batched_iteration(float *sm, uint32_t *ovf, in
                 const bool in0 = (amask & 1u) && rank0 % n_batches == bt;
                 const bool in1 = (amask & 2u) && (rank0 + ((amask & 1u) ? 1 : 0)) % n_batches == bt;
                 if (!in0 && !in1) continue;
-                const int a = ab & 31, b = (ab >> 5) & 31;
+                const int a = ck_idx<CK_BODY>(ab & 31, SC::N), b = ck_idx<CK_BODY>((ab >> 5) & 31, SC::N);
                 const float nx = __uint_as_float(r[R_NX]), ny = __uint_as_float(r[R_NY]);
                 const float ma = sm[SC::BIM + a], mb = sm[SC::BIM + b], ia = sm[SC::BII + a], ib = sm[SC::BII + b];
                 const float4 va4 = ld4(sm + SC::BVEL + 4 * a), vb4 = ld4(sm + SC::BVEL + 4 * b);
@@ -677,7 +697,7 @@ __device__ __noinline__ int slow_solve(float *sm, uint32_t *ovf, int nrec, uint3
         uint32_t *r = ovf + (size_t)(valid ? k : 0) * kRecWords;
         uint32_t ab = 0u;
         int wi = 255;
-        if (valid) { ab = r[S_AB]; wi = widx[(ab >> 12) & 127]; }
+        if (valid) { ab = r[S_AB]; wi = widx[ck_idx<CK_PAIR>((ab >> 12) & 127, SC::NPAIRS)]; }
         float w[4];
         warm_lookup<SC, G>(g, sm, ovf, wi, old_n, old_t, warm_start, w);
         if (valid) {
@@ -685,7 +705,7 @@ __device__ __noinline__ int slow_solve(float *sm, uint32_t *ovf, int nrec, uint3
             c.ab = ab; c.nx = __uint_as_float(r[S_NX]); c.ny = __uint_as_float(r[S_NY]);
             const float pt[6] = { __uint_as_float(r[S_PX0]), __uint_as_float(r[S_PY0]), __uint_as_float(r[S_PEN0]),
                                   __uint_as_float(r[S_PX1]), __uint_as_float(r[S_PY1]), __uint_as_float(r[S_PEN1]) };
-            const int a = ab & 31, b = (ab >> 5) & 31;
+            const int a = ck_idx<CK_BODY>(ab & 31, SC::N), b = ck_idx<CK_BODY>((ab >> 5) & 31, SC::N);
             const float ma = sm[SC::BIM + a], mb = sm[SC::BIM + b], ia = sm[SC::BII + a], ib = sm[SC::BII + b];
             const float fra = sm[SC::BFR + a], frb = sm[SC::BFR + b];
             const float er = fmin_cmp(sm[SC::BRE + a], sm[SC::BRE + b]);
@@ -740,7 +760,7 @@ __device__ __noinline__ int slow_finish(float *sm, uint32_t *ovf, int nrec) {
     uint8_t *widx = reinterpret_cast<uint8_t *>(reinterpret_cast<uint32_t *>(sm) + SC::WIDX);
     int nman = 0;
     for (int k = g.lane; k < nrec; k += G) {
-        const uint32_t *r = ovf + (size_t)k * kRecWords;
+        const uint32_t *r = ovf + (size_t)ck_idx<CK_RECORD>(k, SC::NPAIRS) * kRecWords;
         uint32_t *wr = ovf + SC::SCRATCH_WARM + (size_t)k * kWarmWords;
         const uint32_t ab = r[R_AB];
         const int p = (ab >> 12) & 127;
@@ -750,7 +770,7 @@ __device__ __noinline__ int slow_finish(float *sm, uint32_t *ovf, int nrec) {
         wr[2] = (am & 1u) ? r[R_M0 + M_ACCT] : 0u;
         wr[3] = (am & 2u) ? r[R_M0 + M_WORDS + M_ACCN] : 0u;
         wr[4] = (am & 2u) ? r[R_M0 + M_WORDS + M_ACCT] : 0u;
-        widx[p] = (uint8_t)k;
+        widx[ck_idx<CK_PAIR>(p, SC::NPAIRS)] = (uint8_t)k;
         nman += __popc(am);
     }
     nman = g.sum_int(nman);
@@ -767,7 +787,7 @@ __device__ __noinline__ void warm_in(float *sm, uint32_t *ovf, const uint32_t *s
         uint32_t *wr = ovf + SC::SCRATCH_WARM + (size_t)k * kWarmWords;
 #pragma unroll
         for (int q = 0; q < kWarmWords; ++q) wr[q] = __ldcg(st_warm + kWarmWords * k + q);
-        widx[wr[0]] = (uint8_t)k;
+        widx[ck_idx<CK_PAIR>((int)wr[0], SC::NPAIRS)] = (uint8_t)k;
     }
 }
 template <class SC, int G>
@@ -787,7 +807,7 @@ __device__ __noinline__ void visit_second(float *sm) {
     float *ov = sm + SC::STG + LF_COUNT * G + Group<G>().lane;
     constexpr int H = G / 2;
     const uint32_t ab = __float_as_uint(ov[R_AB * H]);
-    const int a = ab & 31, b = (ab >> 5) & 31;
+    const int a = ck_idx<CK_BODY>(ab & 31, SC::N), b = ck_idx<CK_BODY>((ab >> 5) & 31, SC::N);
     const unsigned amask = (ab >> 10) & 3u;
     const bool dyn_a = (ab >> 26) & 1u, dyn_b = (ab >> 27) & 1u;
     const float nx = ov[R_NX * H], ny = ov[R_NY * H];
@@ -823,7 +843,7 @@ __device__ __noinline__ void second_lookup(float *sm, const uint32_t *ovf, int n
     const uint8_t *widx = reinterpret_cast<const uint8_t *>(reinterpret_cast<const uint32_t *>(sm) + SC::WIDX);
     const bool mine2 = g.lane < H && G + g.lane < nrec;
     int wi2 = 255;
-    if (mine2) wi2 = widx[(__float_as_uint(ov[ovs(S_AB) * H]) >> 12) & 127];
+    if (mine2) wi2 = widx[ck_idx<CK_PAIR>((__float_as_uint(ov[ovs(S_AB) * H]) >> 12) & 127, SC::NPAIRS)];
     float w2[4];
     warm_lookup<SC, G>(g, sm, ovf, wi2, old_n, old_t, warm_start, w2);
     if (mine2) {
@@ -840,7 +860,7 @@ __device__ __noinline__ unsigned second_build(float *sm, int nrec, ContactConsts
     if (!(lane < H && G + lane < nrec)) return 0u;
     float *ov = sm + SC::STG + LF_COUNT * G + lane;
     const uint32_t ab2 = __float_as_uint(ov[ovs(S_AB) * H]);
-    const int a2 = ab2 & 31, b2 = (ab2 >> 5) & 31;
+    const int a2 = ck_idx<CK_BODY>(ab2 & 31, SC::N), b2 = ck_idx<CK_BODY>((ab2 >> 5) & 31, SC::N);
     const float nx2 = ov[ovs(S_NX) * H], ny2 = ov[ovs(S_NY) * H];
     const float pt2[6] = { ov[ovs(S_PX0) * H], ov[ovs(S_PY0) * H], ov[ovs(S_PEN0) * H], ov[ovs(S_PX1) * H], ov[ovs(S_PY1) * H], ov[ovs(S_PEN1) * H] };
     float w2[4];
@@ -952,6 +972,7 @@ __device__ __noinline__ void write_obs(float *sm, const uint32_t *levels, float 
     const int jw = 11 + dims.n_actions;
     const int width = n_shapes * 29 + 2 * dims.n_joints * jw + 6 * dims.n_thrusters;
     float *img = sm + SC::WVX;
+    if (ck_idx<CK_OBS>(SC::WVX + width, region_words<SC, G>() + 1) == 0) return;      // cannot be 0 otherwise: the image starts beyond the body arrays
     g.sync();
     for (int i = lane; i < SC::N; i += G) {
         float c, sn;
@@ -1206,7 +1227,7 @@ struct Scene {
     template <int MODE>
     __device__ __forceinline__ void visit_pair() {
         const uint32_t ab = rec.ab;
-        const int a = ab & 31, b = (ab >> 5) & 31;
+        const int a = ck_idx<CK_BODY>(ab & 31, SC::N), b = ck_idx<CK_BODY>((ab >> 5) & 31, SC::N);
         const unsigned amask = (ab >> 10) & 3u;
         const bool dyn_a = (ab >> 26) & 1u, dyn_b = (ab >> 27) & 1u;
         if (MODE == 2) {
@@ -1246,7 +1267,7 @@ struct Scene {
             if (lane == 0) { prm.reward[(size_t)s * prm.n_envs + e] = 0.0f; prm.done[(size_t)s * prm.n_envs + e] = 1; }
             return;
         }
-        const uint32_t *lv = prm.levels + (size_t)smu[SC::META + META_LEVEL] * SC::LV_WORDS;
+        const uint32_t *lv = prm.levels + (size_t)ck_idx<CK_LEVEL_ID>((int)smu[SC::META + META_LEVEL], prm.n_levels) * SC::LV_WORDS;
         // dense reward: distance between the first green and the first blue shape before the step
         if (prm.dense_kappa != 0.0f && lane == 0) sm[SC::META + META_D0] = green_blue_distance();
         // actions of this step
@@ -1306,8 +1327,8 @@ struct Scene {
 #pragma unroll 1
             for (int lvl = 1; lvl <= tmax; ++lvl) {
                 if (tl == lvl) {
-                    const int i = tp & 255;
-                    const float tv = sm[SC::ACT + ((tp >> 8) & 255)];
+                    const int i = ck_idx<CK_BODY>(tp & 255, SC::N);
+                    const float tv = sm[SC::ACT + ck_idx<CK_COUNT>((tp >> 8) & 255, kMaxActions)];
                     // continuous in [0, 1], or multi-discrete: 0 off, anything else full power
                     const float A = prm.discrete ? (__float_as_int(tv) != 0 ? 1.0f : 0.0f) : fmax_cmp(fmin_cmp(tv, 1.0f), 0.0f);
                     const float c = sm[SC::BC + i], sn = sm[SC::BS + i];
@@ -1331,7 +1352,7 @@ struct Scene {
             int ang = 0;
             float kr = 0.0f, bias_r = 0.0f;
             if ((jab >> 24) & 1u) {
-                const int a = jab & 255, b = (jab >> 8) & 255;
+                const int a = ck_idx<CK_BODY>(jab & 255, SC::N), b = ck_idx<CK_BODY>((jab >> 8) & 255, SC::N);
                 const uint32_t *jl = smu + SC::LVC + (SC::LV_JOINT - SC::LV_ELEN) + kJointLevelWords * lane;
                 float rax, ray, rbx, rby;
                 rot2(sm[SC::BC + a], sm[SC::BS + a], __uint_as_float(jl[1]), __uint_as_float(jl[2]), rax, ray);
@@ -1383,7 +1404,7 @@ struct Scene {
                     keep = !(ba.z + mg < bb.x || bb.z + mg < ba.x || ba.w + mg < bb.y || bb.w + mg < ba.y);
                 }
                 const unsigned bal = g.ballot(keep);
-                if (keep) surv()[nsurv + __popc(bal & g.lanes_below())] = (uint8_t)p;
+                if (keep) surv()[ck_idx<CK_STAGE>(nsurv + __popc(bal & g.lanes_below()), SC::NPAIRS)] = (uint8_t)p;
                 nsurv += __popc(bal);
                 mine_pp += (keep && p < SC::NPP) ? 1 : 0;
                 mine_pc += (keep && p < SC::NPP + SC::NPC) ? 1 : 0;
@@ -1412,7 +1433,7 @@ struct Scene {
                 m[1].px = 0.0f; m[1].py = 0.0f; m[1].pen = 0.0f;
                 int p = 0, a = 0, b = 0;
                 if (idx < hi) {
-                    p = surv()[idx]; a = ptab[p] & 255; b = ptab[p] >> 8;
+                    p = ck_idx<CK_PAIR>(surv()[idx], SC::NPAIRS); a = ck_idx<CK_BODY>(ptab[p] & 255, SC::N); b = ck_idx<CK_BODY>(ptab[p] >> 8, SC::N);
                     if (kind == 0) act = manifold_pp(a, b, m);
                     else if (kind == 1) act = manifold_pc(a, b, m[0]);
                     else act = manifold_cc(a, b, m[0]);
@@ -1423,7 +1444,7 @@ struct Scene {
                 }
                 const unsigned bal = g.ballot(act != 0u);
                 if (act) {
-                    const int k = nrec + __popc(bal & g.lanes_below());
+                    const int k = ck_idx<CK_STAGE>(nrec + __popc(bal & g.lanes_below()), SC::NPAIRS);
                     const uint32_t fa = smu[SC::BFL + a], fb = smu[SC::BFL + b];
                     const uint32_t ra = flag_role(fa), rb = flag_role(fb);
                     t_gb |= (ra == 1u && rb == 2u) || (ra == 2u && rb == 1u);
@@ -1443,7 +1464,7 @@ struct Scene {
                         st[ovs(S_PX0) * H] = m[0].px; st[ovs(S_PY0) * H] = m[0].py; st[ovs(S_PEN0) * H] = m[0].pen;
                         st[ovs(S_PX1) * H] = m[1].px; st[ovs(S_PY1) * H] = m[1].py; st[ovs(S_PEN1) * H] = m[1].pen;
                     } else {
-                        uint32_t *st = ovf + (size_t)k * kRecWords;
+                        uint32_t *st = ovf + (size_t)ck_idx<CK_RECORD>(k, SC::NPAIRS) * kRecWords;
                         st[S_AB] = ab; st[S_NX] = __float_as_uint(nx); st[S_NY] = __float_as_uint(ny);
                         st[S_PX0] = __float_as_uint(m[0].px); st[S_PY0] = __float_as_uint(m[0].py); st[S_PEN0] = __float_as_uint(m[0].pen);
                         st[S_PX1] = __float_as_uint(m[1].px); st[S_PY1] = __float_as_uint(m[1].py); st[S_PEN1] = __float_as_uint(m[1].pen);
@@ -1478,7 +1499,7 @@ struct Scene {
             {
                 int wi = 255;
                 if (mine) {
-                    ab = __float_as_uint(lanef(S_AB)); wi = widx()[(ab >> 12) & 127];
+                    ab = __float_as_uint(lanef(S_AB)); wi = widx()[ck_idx<CK_PAIR>((ab >> 12) & 127, SC::NPAIRS)];
                     nx = lanef(S_NX); ny = lanef(S_NY);
                     pt[0] = lanef(S_PX0); pt[1] = lanef(S_PY0); pt[2] = lanef(S_PEN0); pt[3] = lanef(S_PX1); pt[4] = lanef(S_PY1); pt[5] = lanef(S_PEN1);
                 }
@@ -1487,7 +1508,7 @@ struct Scene {
                 if (two) second_lookup<SC, G>(sm, ovf, nrec, old_n, old_t, prm.warm_start);
             }
             g.sync();     // every lane has read the fields it needs from other lanes before they are rewritten
-            const int a = ab & 31, b = (ab >> 5) & 31;
+            const int a = ck_idx<CK_BODY>(ab & 31, SC::N), b = ck_idx<CK_BODY>((ab >> 5) & 31, SC::N);
             const unsigned amask = (ab >> 10) & 3u;
             rec.ab = ab; rec.nx = nx; rec.ny = ny;
             rec.ma = sm[SC::BIM + a]; rec.mb = sm[SC::BIM + b]; rec.ia = sm[SC::BII + a]; rec.ib = sm[SC::BII + b];
@@ -1596,8 +1617,8 @@ struct Scene {
                 ovl(OV_ACC1N) = __uint_as_float(wr2[3]); ovl(OV_ACC1T) = __uint_as_float(wr2[4]);
             }
         } else {
-            if (lane < nrec) widx()[(rec.ab >> 12) & 127] = (uint8_t)lane;
-            if (clevel2 != 0) widx()[(__float_as_uint(ovl(R_AB)) >> 12) & 127] = (uint8_t)(G + lane);
+            if (lane < nrec) widx()[ck_idx<CK_PAIR>((rec.ab >> 12) & 127, SC::NPAIRS)] = (uint8_t)lane;
+            if (clevel2 != 0) widx()[ck_idx<CK_PAIR>((__float_as_uint(ovl(R_AB)) >> 12) & 127, SC::NPAIRS)] = (uint8_t)(G + lane);
         }
 
         // reward, termination, counters, auto-reset
@@ -1633,8 +1654,8 @@ struct Scene {
             smu[SC::JROW + kJointWords * lane + JR_ACCR] = __ldcg(st + SC::ST_JACC + 3 * lane + 2);
         }
         for (int i = lane; i < (SC::NPAIRS + 3) / 4; i += G) smu[SC::WIDX + i] = 0xffffffffu;
-        const int level = (int)__ldcg(st + SC::ST_META + META_LEVEL);
-        const int nwarm = (int)__ldcg(st + SC::ST_META + META_NWARM);
+        const int level = ck_idx<CK_LEVEL_ID>((int)__ldcg(st + SC::ST_META + META_LEVEL), prm.n_levels);
+        const int nwarm = ck_idx<CK_COUNT>((int)__ldcg(st + SC::ST_META + META_NWARM), SC::NPAIRS + 1);
         jab = load_level_consts<SC, G>(smu, prm.levels + (size_t)level * SC::LV_WORDS);
         g.sync();
         // accumulated impulses of the previous launch: entry k goes to lane k
@@ -1646,7 +1667,7 @@ struct Scene {
             rec.ab = p << 12;
             rec.accn = __uint_as_float(__ldcg(wr + 1)); rec.acct = __uint_as_float(__ldcg(wr + 2));
             lanef(LF_ACC2N) = __uint_as_float(__ldcg(wr + 3)); lanef(LF_ACC2T) = __uint_as_float(__ldcg(wr + 4));
-            widx()[p] = (uint8_t)lane;
+            widx()[ck_idx<CK_PAIR>((int)p, SC::NPAIRS)] = (uint8_t)lane;
         }
         if (lane < G / 2 && G + lane < nwarm) {
             const uint32_t *wr = st + SC::ST_WARM + kWarmWords * (G + lane);
@@ -1654,7 +1675,7 @@ struct Scene {
             ovl(R_AB) = __uint_as_float(p << 12);
             ovl(OV_ACC0N) = __uint_as_float(__ldcg(wr + 1)); ovl(OV_ACC0T) = __uint_as_float(__ldcg(wr + 2));
             ovl(OV_ACC1N) = __uint_as_float(__ldcg(wr + 3)); ovl(OV_ACC1T) = __uint_as_float(__ldcg(wr + 4));
-            widx()[p] = (uint8_t)(G + lane);
+            widx()[ck_idx<CK_PAIR>((int)p, SC::NPAIRS)] = (uint8_t)(G + lane);
         }
         if (nwarm > G + G / 2) warm_in<SC, G>(sm, ovf, st + SC::ST_WARM, nwarm);
         g.sync();
@@ -1672,7 +1693,7 @@ struct Scene {
             st[SC::ST_JACC + 3 * lane + 2] = smu[SC::JROW + kJointWords * lane + JR_ACCR];
         }
         if (lane < 5) st[SC::ST_META + lane] = smu[SC::META + lane];
-        const int nw = (int)smu[SC::META + META_NWARM];
+        const int nw = ck_idx<CK_COUNT>((int)smu[SC::META + META_NWARM], SC::NPAIRS + 1);
         if (lane < nw) {
             uint32_t *wr = st + SC::ST_WARM + kWarmWords * lane;
             wr[0] = (rec.ab >> 12) & 127u;
@@ -1714,7 +1735,7 @@ __global__ void __launch_bounds__(kBlockThreads, kMinBlocks) k2d_step_kernel(con
     const int gib = threadIdx.x / G;
     const int slot = blockIdx.x * GPB + gib, nslots = gridDim.x * GPB;
     uint32_t *region = smem_raw + SC::PTAB_WORDS + gib * region_words<SC, G>();
-    uint32_t *scratch = prm.scratch + (size_t)slot * SC::SCRATCH_WORDS;
+    uint32_t *scratch = prm.scratch + (size_t)ck_idx<CK_SLOT>(slot, prm.n_slots) * SC::SCRATCH_WORDS;
     Scene<SC, G> scene(region, ptab, scratch, prm);
     // Work items are (chunk, env), handed out in that order by one ticket counter: a group that is done
     // takes the next item, so groups with cheap scenes take more of them.  Chunk c of an env may start

@@ -20,7 +20,7 @@ EXPORTS = (
     "k2d_default_config", "k2d_state_bytes", "k2d_state_bytes_no_scratch", "k2d_level_pool_bytes", "k2d_create", "k2d_reset", "k2d_step",
     "k2d_step_discrete", "k2d_step_static_scratch", "k2d_step_obs", "k2d_obs", "k2d_render",
     "k2d_obs_floats", "k2d_canonical_words", "k2d_get_state", "k2d_set_state", "k2d_status", "k2d_level_info",
-    "k2d_set_trace", "k2d_trace_slots", "k2d_set_wait_limit", "k2d_eval_sincos_tanh", "k2d_measure_fp32_peak", "k2d_error_string", "k2d_destroy",
+    "k2d_set_trace", "k2d_trace_slots", "k2d_is_checked_build", "k2d_set_wait_limit", "k2d_eval_sincos_tanh", "k2d_measure_fp32_peak", "k2d_error_string", "k2d_destroy",
 )
 
 
@@ -52,14 +52,13 @@ LEVEL_DTYPE = np.dtype([
     ("thr_binding", np.int32, (MAX_THRUSTERS,)), ("thr_active", np.int32, (MAX_THRUSTERS,)),
 ])
 
-_lib = None
+_libs = {}
 
 
-def load_library():
-    """Builds (if stale) and loads libk2d.so; raises if that is impossible."""
-    global _lib
-    if _lib is None:
-        lib = C.CDLL(_build.build())
+def load_library(checked: bool = False):
+    """Builds (if stale) and loads libk2d.so (checked=True: the build with index checks); raises if that is impossible."""
+    if checked not in _libs:
+        lib = C.CDLL(_build.build(checked=checked))
         vp, i32 = C.c_void_p, C.c_int32
         lib.k2d_default_config.argtypes = [C.POINTER(Config), i32, i32, i32, i32, i32]
         lib.k2d_state_bytes.argtypes = [C.POINTER(Config)]
@@ -90,8 +89,8 @@ def load_library():
         lib.k2d_error_string.argtypes = [C.c_int]
         lib.k2d_error_string.restype = C.c_char_p
         lib.k2d_destroy.argtypes = [vp]
-        _lib = lib
-    return _lib
+        _libs[checked] = lib
+    return _libs[checked]
 
 
 class K2DError(RuntimeError):
@@ -133,12 +132,12 @@ def make_config(levels: dict, n_envs: int, **kw) -> Config:
 class Env:
     """n_envs scenes on one CUDA device, stepped by the library."""
 
-    def __init__(self, levels: dict, n_envs: int, device: int = 0, stream=None, **cfg_kw):
+    def __init__(self, levels: dict, n_envs: int, device: int = 0, stream=None, checked: bool = False, **cfg_kw):
         import torch
         if not torch.cuda.is_available():
             raise K2DError("no CUDA device: the k2d library has no CPU fallback")
         self.torch = torch
-        self.lib = load_library()
+        self.lib = load_library(checked)
         self.device = torch.device("cuda", device)
         self.stream = stream if stream is not None else torch.cuda.current_stream(self.device)
         self.cfg = make_config(levels, n_envs, device=device, **cfg_kw)

@@ -21,7 +21,8 @@ def make_pair(levels, n_envs, broadphase=0, **cfg):
     may collide (``broadphase=0``): the library's bounding-box test in front of its narrowphase is thereby checked
     against a reference that has no such test.  ``broadphase=1`` gives the oracle the same test, which makes its
     counters of pairs past the test comparable too."""
-    env = k2d.Env(levels, n_envs, **cfg)
+    checked = cfg.pop("checked", False)
+    env = k2d.Env(levels, n_envs, checked=checked, **cfg)
     ocfg = {k: getattr(env.cfg, k) for k in ORACLE_CFG}
     ref = k2d_ref.RefSim(levels, n_envs, broadphase=broadphase, **ocfg)
     return env, ref
