@@ -295,6 +295,12 @@ static cudaError_t launch_obs(const k2d_state *s, float *dev_obs) {
     return cudaGetLastError();
 }
 
+template <class SC>
+static cudaError_t launch_render(const k2d_state *s, uint32_t *out) {
+    k2d_render_kernel<SC><<<s->cfg.n_envs, kRenderThreads, 0, s->stream>>>(s->dev_env, s->dev_levels, out, s->cfg.n_envs);
+    return cudaGetLastError();
+}
+
 // Kernel arguments of one k2d_step launch.  With more envs than resident scene groups the launch is cut
 // into chunks of kChunkSteps steps, so that the groups can balance the work between them.
 static StepParams step_params(const k2d_state *s, const float *dev_actions, int n_steps, float *dev_reward, uint8_t *dev_done,
@@ -497,10 +503,7 @@ int k2d_render(k2d_state *s, uint8_t *dev_pixels) {
     CUDA_OK(cudaSetDevice(s->cfg.device));
     const int E = s->cfg.n_envs;
     uint32_t *out = reinterpret_cast<uint32_t *>(dev_pixels);
-    if (s->ci.id == 0) k2d_render_kernel<ClassS><<<E, kRenderThreads, 0, s->stream>>>(s->dev_env, s->dev_levels, out, E);
-    else if (s->ci.id == 1) k2d_render_kernel<ClassM><<<E, kRenderThreads, 0, s->stream>>>(s->dev_env, s->dev_levels, out, E);
-    else k2d_render_kernel<ClassL><<<E, kRenderThreads, 0, s->stream>>>(s->dev_env, s->dev_levels, out, E);
-    CUDA_OK(cudaGetLastError());
+    CUDA_OK(s->ci.id == 0 ? launch_render<ClassS>(s, out) : s->ci.id == 1 ? launch_render<ClassM>(s, out) : launch_render<ClassL>(s, out));
     return K2D_OK;
 }
 

@@ -1919,6 +1919,8 @@ __global__ void __launch_bounds__(kRenderThreads) k2d_render_kernel(const uint32
     __shared__ float4 s_nx[SC::N], s_ny[SC::N], s_off[SC::N];   // polygon: face normals and offsets; circle: centre x, y, radius^2 in .x
     __shared__ uint32_t s_col[SC::N];
     __shared__ int s_nv[SC::N];              // vertices of a polygon, 0 for a circle, -1 for a shape that is not drawn
+    __shared__ uint2 s_span[kRenderThreads * SC::N];         // per row of the block: (first column | columns - 1 << 8, colour) of every shape the row cuts
+    __shared__ int s_nspan[kRenderThreads];
     const int e = blockIdx.x;
     if (e >= n_envs) return;
     const uint32_t *st = state + (size_t)e * SC::ST_WORDS;
@@ -1964,45 +1966,97 @@ __global__ void __launch_bounds__(kRenderThreads) k2d_render_kernel(const uint32
         s_nv[i] = nv;
     }
     __syncthreads();
+    // A warp paints 32 consecutive rows in two passes.  First every lane takes one row and goes over the shapes in index
+    // order: from the shape's faces (or its circle) it works out between which columns the row can cut the shape, and pins
+    // down the first and the last column that are inside with the exact inside test (the one that defines the image) on the
+    // few columns at either end of that span, where rounding could matter; the columns in between are inside (the shapes
+    // are convex).  That gives a short list of (first column, last column, shape) per row.  Then the warp writes the rows one
+    // after the other, lane l the columns l, l + 32, l + 64, l + 96: a pixel takes the colour of the last entry of its row's
+    // list that covers it, white if none does.
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    uint32_t *img = pixels + (size_t)e * kPix * kPix;
-    // a warp paints one row at a time in registers: lane l holds the pixels of columns l, l + 32, l + 64, l + 96;
-    // the shapes whose box reaches the row go over it in index order, each only over the 32-column blocks its box
-    // touches, so the highest index ends up on top
-    for (int r = warp; r < kPix; r += kRenderThreads / 32) {
+    uint2 *spans = s_span + (warp * 32 + lane) * SC::N;
+    const int r = 32 * warp + lane;
+    int n_span = 0;
+    if (r < kPix) {
         const float py = 5.75f - ((float)r + 0.5f) * 0.05f;
-        bool reach = false;
-        if (lane < SC::N && s_nv[lane] >= 0) reach = s_rng[lane].z <= r && r <= s_rng[lane].w;
-        unsigned m = __ballot_sync(0xffffffffu, reach);
-        uint32_t col[4] = { 0xffffffffu, 0xffffffffu, 0xffffffffu, 0xffffffffu };
-        while (m) {
-            const int i = __ffs(m) - 1;
-            m &= m - 1u;
-            const int4 rng = s_rng[i];
+#pragma unroll 1
+        for (int i = 0; i < SC::N; ++i) {
             const int nv = s_nv[i];
+            if (nv < 0) continue;
+            const int4 rng = s_rng[i];
+            if (r < rng.z || r > rng.w) continue;
             const float4 nx = s_nx[i], ny = s_ny[i], off = s_off[i];
-            const uint32_t shape_col = s_col[i];
-            // the row's share of every face's dot product (polygon) or of the squared distance (circle)
-            const float t0 = ny.x * py, t1 = ny.y * py, t2 = ny.z * py, t3 = ny.w * py;
-            const float dy = py - ny.x, dy2 = dy * dy;
+            float lo = -1.0e9f, hi = 1.0e9f;      // world x between which the row can be inside the shape
+            bool all_exact = false, none = false;
+            float t0 = 0.0f, t1 = 0.0f, t2 = 0.0f, t3 = 0.0f, dy2 = 0.0f;
+            if (nv > 0) {
+                t0 = ny.x * py; t1 = ny.y * py; t2 = ny.z * py; t3 = ny.w * py;
+                const float a[4] = { nx.x, nx.y, nx.z, nx.w }, c[4] = { t0 - off.x, t1 - off.y, t2 - off.z, t3 - off.w };
 #pragma unroll
-            for (int k = 0; k < 4; ++k) {
-                if (rng.y < 32 * k || rng.x > 32 * k + 31) continue;       // the same for the whole warp
-                const float px = -3.125f + ((float)(32 * k + lane) + 0.5f) * 0.05f;
-                bool inside;
-                if (nv > 0) {
-                    inside = !(__fmaf_rn(nx.x, px, t0) - off.x > 0.0f) && !(__fmaf_rn(nx.y, px, t1) - off.y > 0.0f) &&
-                             !(__fmaf_rn(nx.z, px, t2) - off.z > 0.0f) && (nv < 4 || !(__fmaf_rn(nx.w, px, t3) - off.w > 0.0f));
-                } else {
-                    const float dx = px - nx.x;
-                    inside = __fmaf_rn(dx, dx, dy2) <= off.x;
+                for (int k = 0; k < 4; ++k) {
+                    if (k < nv) {
+                        if (fabsf(a[k]) < 1.0e-3f) {          // a face nearly along the row: it is out, not binding, or too close to call
+                            if (c[k] > 1.0e-3f) none = true;
+                            else if (c[k] > -1.0e-3f) all_exact = true;
+                        } else {
+                            const float bound = __fdividef(-c[k], a[k]);      // an estimate is enough: the exact test decides the ends of the span
+                            if (a[k] > 0.0f) hi = fmin_cmp(hi, bound); else lo = fmax_cmp(lo, bound);
+                        }
+                    }
                 }
-                if (inside) col[k] = shape_col;
+            } else {
+                const float dy = py - ny.x;
+                dy2 = dy * dy;
+                const float h2 = off.x - dy2;
+                if (h2 < -1.0e-4f) none = true;
+                else { const float h = sqrtf(fmax_cmp(h2, 0.0f)); lo = nx.x - h; hi = nx.x + h; }
             }
+            if (none || hi < lo - 0.2f) continue;
+            // columns: pixel c has its centre at x = -3.125 + (c + 0.5) * 0.05
+            const float clo = fmax_cmp((lo + 3.125f) * 20.0f - 0.5f, -4.0f), chi = fmin_cmp((hi + 3.125f) * 20.0f - 0.5f, 130.0f);
+            const int c_first = max(max((int)floorf(clo) - 2, rng.x), 0), c_last = min(min((int)ceilf(chi) + 2, rng.y), kPix - 1);
+            // columns sure_first .. sure_last are inside without a test (none if a face is too close to call)
+            const int sure_first = all_exact ? c_last + 1 : max((int)ceilf(clo) + 2, c_first), sure_last = all_exact ? c_first - 1 : min((int)floorf(chi) - 2, c_last);
+            auto exact = [&](int c) -> bool {
+                const float px = -3.125f + ((float)c + 0.5f) * 0.05f;
+                if (nv > 0)
+                    return !(__fmaf_rn(nx.x, px, t0) - off.x > 0.0f) && !(__fmaf_rn(nx.y, px, t1) - off.y > 0.0f) &&
+                           !(__fmaf_rn(nx.z, px, t2) - off.z > 0.0f) && (nv < 4 || !(__fmaf_rn(nx.w, px, t3) - off.w > 0.0f));
+                const float dx = px - nx.x;
+                return __fmaf_rn(dx, dx, dy2) <= off.x;
+            };
+            const bool sure = sure_first <= sure_last;
+            int cf = sure ? sure_first : c_last + 1, cl = sure ? sure_last : c_first - 1;
+            // the first inside column: the lowest one below the sure span (or anywhere, if there is no sure span) that passes the test
+            const int left_end = sure ? sure_first - 1 : c_last;
+#pragma unroll 1
+            for (int c = c_first; c <= left_end; ++c) if (exact(c)) { cf = c; break; }
+            const int right_end = sure ? sure_last + 1 : max(cf, c_first);
+#pragma unroll 1
+            for (int c = c_last; c >= right_end; --c) if (exact(c)) { cl = c; break; }
+            if (!sure && cl < cf) cl = cf;      // a single column found from the left
+            if (cf <= cl && cf <= c_last) spans[n_span++] = make_uint2((uint32_t)cf | ((uint32_t)(cl - cf) << 8), s_col[i]);
+        }
+    }
+    s_nspan[warp * 32 + lane] = n_span;
+    __syncwarp();
+    const int n_rows = min(32, kPix - 32 * warp);
+    uint32_t *img = pixels + (size_t)e * kPix * kPix + (size_t)warp * 32 * kPix;
+#pragma unroll 1
+    for (int j = 0; j < n_rows; ++j) {
+        const int ns = s_nspan[warp * 32 + j];
+        const uint2 *sp = s_span + (warp * 32 + j) * SC::N;
+        uint32_t col[4] = { 0xffffffffu, 0xffffffffu, 0xffffffffu, 0xffffffffu };
+#pragma unroll 1
+        for (int k = 0; k < ns; ++k) {
+            const uint2 w = sp[k];
+            const unsigned cf = w.x & 255u, len = w.x >> 8;
+            const unsigned d = (unsigned)lane - cf;          // column - first column, for the lane's four columns d, d + 32, ...
+#pragma unroll
+            for (int q = 0; q < 4; ++q) if (d + 32u * q <= len) col[q] = w.y;
         }
 #pragma unroll
-        for (int k = 0; k < 4; ++k)
-            if (32 * k + lane < kPix) img[r * kPix + 32 * k + lane] = col[k];
+        for (int q = 0; q < 4; ++q) if (32 * q + lane < kPix) img[j * kPix + 32 * q + lane] = col[q];
     }
 }
 
