@@ -892,18 +892,36 @@ __device__ __noinline__ unsigned second_build(float *sm, int nrec, ContactConsts
 template <class SC, int G>
 __device__ __noinline__ uint32_t load_level_consts(uint32_t *smu, const uint32_t *lv) {
     const int lane = Group<G>().lane;
-    for (int i = lane; i < SC::N; i += G) {
-        smu[SC::BIM + i] = lv[SC::LV_IM + i];
-        smu[SC::BII + i] = lv[SC::LV_II + i];
-        smu[SC::BFR + i] = lv[SC::LV_FR + i];
-        smu[SC::BRE + i] = lv[SC::LV_RE + i];
-        smu[SC::BFL + i] = lv[SC::LV_FLAGS + i];
+    // all loads are asked for before the first of them is stored, so that the group waits for memory once
+    constexpr int KN = (SC::N + G - 1) / G, KL = (SC::LVC_WORDS + G - 1) / G, KC = (SC::C + G - 1) / G, KM = (SC::MASKW + G - 1) / G;
+    uint32_t cim[KN], cii[KN], cfr[KN], cre[KN], cfl[KN], lvc[KL], rad[KC], msk[KM];
+#pragma unroll
+    for (int k = 0; k < KN; ++k) {
+        const int i = lane + k * G; const bool in = i < SC::N;
+        cim[k] = in ? __ldg(lv + SC::LV_IM + i) : 0u; cii[k] = in ? __ldg(lv + SC::LV_II + i) : 0u; cfr[k] = in ? __ldg(lv + SC::LV_FR + i) : 0u;
+        cre[k] = in ? __ldg(lv + SC::LV_RE + i) : 0u; cfl[k] = in ? __ldg(lv + SC::LV_FLAGS + i) : 0u;
     }
-    for (int i = lane; i < SC::C; i += G) smu[SC::RAD + i] = lv[SC::LV_RAD + i];
-    for (int i = lane; i < SC::MASKW; i += G) smu[SC::MASK + i] = lv[SC::LV_MASK + i];
-    if (lane == 0) smu[SC::META + META_GB] = lv[SC::LV_GB];
-    for (int i = lane; i < SC::LVC_WORDS; i += G) smu[SC::LVC + i] = lv[SC::LV_ELEN + i];
-    return (SC::J > 0 && lane < SC::J) ? lv[SC::LV_JOINT + kJointLevelWords * lane] : 0u;
+#pragma unroll
+    for (int k = 0; k < KL; ++k) { const int i = lane + k * G; lvc[k] = (i < SC::LVC_WORDS) ? __ldg(lv + SC::LV_ELEN + i) : 0u; }
+#pragma unroll
+    for (int k = 0; k < KC; ++k) { const int i = lane + k * G; rad[k] = (i < SC::C) ? __ldg(lv + SC::LV_RAD + i) : 0u; }
+#pragma unroll
+    for (int k = 0; k < KM; ++k) { const int i = lane + k * G; msk[k] = (i < SC::MASKW) ? __ldg(lv + SC::LV_MASK + i) : 0u; }
+    const uint32_t gb = __ldg(lv + SC::LV_GB);
+    const uint32_t jab = (SC::J > 0 && lane < SC::J) ? __ldg(lv + SC::LV_JOINT + kJointLevelWords * lane) : 0u;
+#pragma unroll
+    for (int k = 0; k < KN; ++k) {
+        const int i = lane + k * G;
+        if (i < SC::N) { smu[SC::BIM + i] = cim[k]; smu[SC::BII + i] = cii[k]; smu[SC::BFR + i] = cfr[k]; smu[SC::BRE + i] = cre[k]; smu[SC::BFL + i] = cfl[k]; }
+    }
+#pragma unroll
+    for (int k = 0; k < KL; ++k) { const int i = lane + k * G; if (i < SC::LVC_WORDS) smu[SC::LVC + i] = lvc[k]; }
+#pragma unroll
+    for (int k = 0; k < KC; ++k) { const int i = lane + k * G; if (i < SC::C) smu[SC::RAD + i] = rad[k]; }
+#pragma unroll
+    for (int k = 0; k < KM; ++k) { const int i = lane + k * G; if (i < SC::MASKW) smu[SC::MASK + i] = msk[k]; }
+    if (lane == 0) smu[SC::META + META_GB] = gb;
+    return jab;
 }
 
 // Auto-reset of a finished env: next level (its own, or drawn from the pool by the hash of seed,
@@ -1274,6 +1292,15 @@ struct Scene {
         const float *act_row = prm.actions + ((size_t)(s / prm.frame_skip) * prm.n_envs + e) * prm.n_actions;
         if (lane < prm.n_actions) sm[SC::ACT + lane] = act_row[lane];
         if (G < kMaxActions && lane + G < prm.n_actions) sm[SC::ACT + lane + G] = act_row[lane + G];
+        // the body-frame vertices and normals this lane will turn are asked for now and used after the rotations are known
+        constexpr int KV = (SC::P4 + G - 1) / G;
+        float pvx[KV], pvy[KV], pnx[KV], pny[KV];
+#pragma unroll
+        for (int k = 0; k < KV; ++k) {
+            const int v = lane + k * G; const bool in = v < SC::P4;
+            pvx[k] = in ? __uint_as_float(__ldg(lv + SC::LV_PVX + v)) : 0.0f; pvy[k] = in ? __uint_as_float(__ldg(lv + SC::LV_PVY + v)) : 0.0f;
+            pnx[k] = in ? __uint_as_float(__ldg(lv + SC::LV_PNX + v)) : 0.0f; pny[k] = in ? __uint_as_float(__ldg(lv + SC::LV_PNY + v)) : 0.0f;
+        }
         // gravity, rotation, circle boxes
         for (int i = lane; i < SC::N; i += G) {
             const uint32_t fl = smu[SC::BFL + i];
@@ -1288,13 +1315,15 @@ struct Scene {
         }
         g.sync();
         // world-frame polygon vertices, normals, face offsets
-        for (int v = lane; v < SC::P4; v += G) {
+#pragma unroll
+        for (int kk = 0; kk < KV; ++kk) {
+            const int v = lane + kk * G;
             const int i = v >> 2, k = v & 3;
-            if (k < (int)flag_nverts(smu[SC::BFL + i])) {
+            if (v < SC::P4 && k < (int)flag_nverts(smu[SC::BFL + i])) {
                 const float c = sm[SC::BC + i], sn = sm[SC::BS + i];
                 float rx, ry, nx, ny;
-                rot2(c, sn, __uint_as_float(lv[SC::LV_PVX + v]), __uint_as_float(lv[SC::LV_PVY + v]), rx, ry);
-                rot2(c, sn, __uint_as_float(lv[SC::LV_PNX + v]), __uint_as_float(lv[SC::LV_PNY + v]), nx, ny);
+                rot2(c, sn, pvx[kk], pvy[kk], rx, ry);
+                rot2(c, sn, pnx[kk], pny[kk], nx, ny);
                 const float wx = rx + sm[SC::BPOS + 4 * i], wy = ry + sm[SC::BPOS + 4 * i + 1];
                 sm[SC::WVX + v] = wx; sm[SC::WVY + v] = wy; sm[SC::WNX + v] = nx; sm[SC::WNY + v] = ny;
                 sm[SC::WOFF + v] = dot2(nx, ny, wx, wy);
@@ -1646,27 +1675,40 @@ struct Scene {
     // launch, so it is read past the (non-coherent) L1.
     __device__ __forceinline__ void run(int e, int s0, int s1) {
         uint32_t *st = prm.state + (size_t)e * SC::ST_WORDS;
-        for (int i = lane; i < 6 * SC::N; i += G) smu[body_word<SC>(i)] = __ldcg(st + SC::ST_BODY + i);
-        if (lane < 5) smu[SC::META + lane] = __ldcg(st + SC::ST_META + lane);
+        // everything the state record holds for this lane is asked for in one go (the warm list entries are read a little
+        // past the count, inside the record, and dropped below), then the level's constants in a second go
+        constexpr int KB = (6 * SC::N + G - 1) / G;
+        uint32_t body[KB], meta = 0u, jacc[3] = { 0u, 0u, 0u }, wrm[kWarmWords];
+#pragma unroll
+        for (int k = 0; k < KB; ++k) { const int i = lane + k * G; body[k] = (i < 6 * SC::N) ? __ldcg(st + SC::ST_BODY + i) : 0u; }
+        if (lane < 5) meta = __ldcg(st + SC::ST_META + lane);
         if (SC::J > 0 && lane < SC::J) {
-            smu[SC::JROW + kJointWords * lane + JR_ACCX] = __ldcg(st + SC::ST_JACC + 3 * lane);
-            smu[SC::JROW + kJointWords * lane + JR_ACCY] = __ldcg(st + SC::ST_JACC + 3 * lane + 1);
-            smu[SC::JROW + kJointWords * lane + JR_ACCR] = __ldcg(st + SC::ST_JACC + 3 * lane + 2);
+#pragma unroll
+            for (int q = 0; q < 3; ++q) jacc[q] = __ldcg(st + SC::ST_JACC + 3 * lane + q);
         }
-        for (int i = lane; i < (SC::NPAIRS + 3) / 4; i += G) smu[SC::WIDX + i] = 0xffffffffu;
+#pragma unroll
+        for (int q = 0; q < kWarmWords; ++q) wrm[q] = (lane < SC::NPAIRS) ? __ldcg(st + SC::ST_WARM + kWarmWords * lane + q) : 0u;
         const int level = ck_idx<CK_LEVEL_ID>((int)__ldcg(st + SC::ST_META + META_LEVEL), prm.n_levels);
         const int nwarm = ck_idx<CK_COUNT>((int)__ldcg(st + SC::ST_META + META_NWARM), SC::NPAIRS + 1);
+#pragma unroll
+        for (int k = 0; k < KB; ++k) { const int i = lane + k * G; if (i < 6 * SC::N) smu[body_word<SC>(i)] = body[k]; }
+        if (lane < 5) smu[SC::META + lane] = meta;
+        if (SC::J > 0 && lane < SC::J) {
+            smu[SC::JROW + kJointWords * lane + JR_ACCX] = jacc[0];
+            smu[SC::JROW + kJointWords * lane + JR_ACCY] = jacc[1];
+            smu[SC::JROW + kJointWords * lane + JR_ACCR] = jacc[2];
+        }
+        for (int i = lane; i < (SC::NPAIRS + 3) / 4; i += G) smu[SC::WIDX + i] = 0xffffffffu;
         jab = load_level_consts<SC, G>(smu, prm.levels + (size_t)level * SC::LV_WORDS);
         g.sync();
         // accumulated impulses of the previous launch: entry k goes to lane k
         rec.ab = 0u; rec.accn = 0.0f; rec.acct = 0.0f;
         lanef(LF_ACC2N) = 0.0f; lanef(LF_ACC2T) = 0.0f;
         if (lane < nwarm) {
-            const uint32_t *wr = st + SC::ST_WARM + kWarmWords * lane;
-            const uint32_t p = __ldcg(wr);
+            const uint32_t p = wrm[0];
             rec.ab = p << 12;
-            rec.accn = __uint_as_float(__ldcg(wr + 1)); rec.acct = __uint_as_float(__ldcg(wr + 2));
-            lanef(LF_ACC2N) = __uint_as_float(__ldcg(wr + 3)); lanef(LF_ACC2T) = __uint_as_float(__ldcg(wr + 4));
+            rec.accn = __uint_as_float(wrm[1]); rec.acct = __uint_as_float(wrm[2]);
+            lanef(LF_ACC2N) = __uint_as_float(wrm[3]); lanef(LF_ACC2T) = __uint_as_float(wrm[4]);
             widx()[ck_idx<CK_PAIR>((int)p, SC::NPAIRS)] = (uint8_t)lane;
         }
         if (lane < G / 2 && G + lane < nwarm) {
