@@ -1844,8 +1844,10 @@ __global__ void k2d_reset_kernel(uint32_t *state, const uint32_t *levels, const 
 }
 
 // ---------------------------------------------------------------- observation kernel: one warp per env
-// Each lane writes whole entity rows (a shape, one side of a joint, a thruster) into the warp's
-// shared-memory image of the observation, then the warp copies the image out with coalesced stores.
+// Lanes 0..15 write one shape row each, lanes 16..27 one side of a joint each, lanes 28..29 a thruster row each, into the
+// warp's shared-memory image of the observation; then the warp copies the image out with coalesced stores.  Every lane asks
+// for all the words of the state record and of the level record its row needs before it uses the first of them.
+static_assert(K2D_MAX_SHAPES <= 16 && 2 * K2D_MAX_JOINTS <= 12 && K2D_MAX_THRUSTERS <= 2, "observation rows: one lane each");
 template <class SC>
 __global__ void __launch_bounds__(kObsThreads) k2d_obs_kernel(const uint32_t *state, const uint32_t *levels, float *obs,
                                                               int n_envs, int n_actions, int n_polygons, int n_circles,
@@ -1860,54 +1862,83 @@ __global__ void __launch_bounds__(kObsThreads) k2d_obs_kernel(const uint32_t *st
     float *img = obs_smem + (size_t)w * ((width + 2 * SC::N + 3) / 4 * 4);
     float *cs = img + width;                 // cos, sin of every shape's angle
     const uint32_t *st = state + (size_t)e * SC::ST_WORDS;
-    const uint32_t *lv = levels + (size_t)st[SC::ST_META + 2] * SC::LV_WORDS;
     const float *stf = reinterpret_cast<const float *>(st);
+    // the state words of this lane's shape do not wait for the level id
+    const bool shape_lane = lane < n_shapes;
+    const int i = shape_lane ? (lane < n_polygons ? lane : SC::P + (lane - n_polygons)) : 0;     // internal shape index
+    float sx = 0.0f, sy = 0.0f, sth = 0.0f, svx = 0.0f, svy = 0.0f, sw = 0.0f;
+    if (shape_lane) { sx = stf[i]; sy = stf[SC::N + i]; sth = stf[2 * SC::N + i]; svx = stf[3 * SC::N + i]; svy = stf[4 * SC::N + i]; sw = stf[5 * SC::N + i]; }
+    const uint32_t *lv = levels + (size_t)st[SC::ST_META + META_LEVEL] * SC::LV_WORDS;
     const float *lvf = reinterpret_cast<const float *>(lv);
-    for (int ci = lane; ci < n_shapes; ci += 32) {
-        const int i = ci < n_polygons ? ci : SC::P + (ci - n_polygons);     // internal shape index
+    const bool poly = i < SC::P;
+    uint32_t fl = 0u;
+    float c_im = 0.0f, c_ii = 0.0f, c_de = 0.0f, c_fr = 0.0f, c_re = 0.0f, c_rad = 0.0f, pv[8] = { 0.0f, 0.0f, 0.0f, 0.0f, 0.0f, 0.0f, 0.0f, 0.0f };
+    const int row = lane - 16, j = row >> 1, d = row & 1;                 // joint lanes
+    const bool joint_lane = row >= 0 && row < 2 * n_joints;
+    uint32_t jl[8] = { 0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u };                 // packed word, anchors, speed, power, kind
+    const int t = lane - 28;                                               // thruster lanes
+    const bool thr_lane = t >= 0 && t < n_thrusters;
+    uint32_t th[6] = { 0u, 0u, 0u, 0u, 0u, 0u };
+    if (shape_lane) {
+        fl = __ldg(lv + SC::LV_FLAGS + i);
+        c_im = __ldg(lvf + SC::LV_IM + i); c_ii = __ldg(lvf + SC::LV_II + i); c_de = __ldg(lvf + SC::LV_DENS + i);
+        c_fr = __ldg(lvf + SC::LV_FR + i); c_re = __ldg(lvf + SC::LV_RE + i);
+        if (poly) {
+#pragma unroll
+            for (int k = 0; k < 4; ++k) { pv[2 * k] = __ldg(lvf + SC::LV_PVX + 4 * i + k); pv[2 * k + 1] = __ldg(lvf + SC::LV_PVY + 4 * i + k); }
+        } else c_rad = __ldg(lvf + SC::LV_RAD + (i - SC::P));
+    }
+    if (joint_lane) {
+        const uint32_t *src = lv + SC::LV_JOINT + kJointLevelWords * j;
+#pragma unroll
+        for (int q = 0; q < 7; ++q) jl[q] = __ldg(src + q);
+        jl[7] = __ldg(src + 10);
+    }
+    if (thr_lane) {
+        const uint32_t *src = lv + SC::LV_THR + 8 * t;
+#pragma unroll
+        for (int q = 0; q < 6; ++q) th[q] = __ldg(src + q);
+    }
+    if (shape_lane) {
         float c, sn;
-        sincos_spec(stf[2 * SC::N + i], c, sn);
+        sincos_spec(sth, c, sn);
         cs[i] = c; cs[SC::N + i] = sn;
-        float *o = img + ci * 29;
-        const uint32_t fl = lv[SC::LV_FLAGS + i];
+        float *o = img + lane * 29;
         if (!(fl & F_ACTIVE)) {
             for (int f = 0; f < 29; ++f) o[f] = 0.0f;
-            continue;
-        }
-        const int nv = flag_nverts(fl);
-        const uint32_t role = flag_role(fl);
-        const bool poly = i < SC::P;
-        o[0] = stf[i]; o[1] = stf[SC::N + i]; o[2] = stf[3 * SC::N + i]; o[3] = stf[4 * SC::N + i];
-        o[4] = lvf[SC::LV_IM + i]; o[5] = lvf[SC::LV_II + i]; o[6] = lvf[SC::LV_DENS + i];
-        o[7] = tanh_spec(stf[5 * SC::N + i] * 0.1f);
+        } else {
+            const int nv = flag_nverts(fl);
+            const uint32_t role = flag_role(fl);
+            o[0] = sx; o[1] = sy; o[2] = svx; o[3] = svy;
+            o[4] = c_im; o[5] = c_ii; o[6] = c_de;
+            o[7] = tanh_spec(sw * 0.1f);
 #pragma unroll
-        for (int r = 0; r < 4; ++r) o[8 + r] = (role == (uint32_t)r) ? 1.0f : 0.0f;
-        o[12] = sn; o[13] = c; o[14] = lvf[SC::LV_FR + i]; o[15] = lvf[SC::LV_RE + i];
-        o[16] = poly ? 1.0f : 0.0f; o[17] = poly ? 0.0f : 1.0f;
-        o[18] = poly ? 0.0f : lvf[SC::LV_RAD + (poly ? 0 : i - SC::P)];
+            for (int r = 0; r < 4; ++r) o[8 + r] = (role == (uint32_t)r) ? 1.0f : 0.0f;
+            o[12] = sn; o[13] = c; o[14] = c_fr; o[15] = c_re;
+            o[16] = poly ? 1.0f : 0.0f; o[17] = poly ? 0.0f : 1.0f;
+            o[18] = poly ? 0.0f : c_rad;
 #pragma unroll
-        for (int k = 0; k < 4; ++k) {
-            const bool on = poly && k < nv;
-            o[19 + 2 * k] = on ? lvf[SC::LV_PVX + 4 * (poly ? i : 0) + k] : 0.0f;
-            o[20 + 2 * k] = on ? lvf[SC::LV_PVY + 4 * (poly ? i : 0) + k] : 0.0f;
+            for (int k = 0; k < 4; ++k) {
+                const bool on = poly && k < nv;
+                o[19 + 2 * k] = on ? pv[2 * k] : 0.0f;
+                o[20 + 2 * k] = on ? pv[2 * k + 1] : 0.0f;
+            }
+            o[27] = (poly && nv == 3) ? 1.0f : 0.0f;
+            o[28] = (poly && nv != 3) ? 1.0f : 0.0f;
         }
-        o[27] = (poly && nv == 3) ? 1.0f : 0.0f;
-        o[28] = (poly && nv != 3) ? 1.0f : 0.0f;
     }
     __syncwarp();
-    float *jrows = img + n_shapes * 29;
-    for (int row = lane; row < 2 * n_joints; row += 32) {
-        const int j = row >> 1, d = row & 1;
-        const uint32_t *jl = lv + SC::LV_JOINT + kJointLevelWords * j;
+    if (joint_lane) {
         const uint32_t jab = jl[0];
-        float *o = jrows + row * jw;
+        float *o = img + n_shapes * 29 + row * jw;
         for (int f = 0; f < jw; ++f) o[f] = 0.0f;
         if ((jab >> 28) & 1u) {
             const int a = jab & 255, b = (jab >> 8) & 255;
             const int from = d ? b : a, to = d ? a : b;
-            o[0] = 1.0f; o[1] = (jl[10] & 1u) ? 1.0f : 0.0f;
-#pragma unroll
-            for (int f = 2; f < 6; ++f) { const int side = ((f - 2) >> 1) ^ d; o[f] = __uint_as_float(jl[1 + 2 * side + ((f - 2) & 1)]); }
+            o[0] = 1.0f; o[1] = (jl[7] & 1u) ? 1.0f : 0.0f;
+            // anchor on the "from" shape, then on the "to" shape
+            o[2] = __uint_as_float(d ? jl[3] : jl[1]); o[3] = __uint_as_float(d ? jl[4] : jl[2]);
+            o[4] = __uint_as_float(d ? jl[1] : jl[3]); o[5] = __uint_as_float(d ? jl[2] : jl[4]);
             o[6] = __uint_as_float(jl[6]); o[7] = __uint_as_float(jl[5]);
             const int bind = (int)((jab >> 16) & 255);
             if (bind < n_actions) o[9 + bind] = 1.0f;
@@ -1915,16 +1946,14 @@ __global__ void __launch_bounds__(kObsThreads) k2d_obs_kernel(const uint32_t *st
             o[10 + n_actions] = __fmaf_rn(cs[to], cs[from], cs[SC::N + to] * cs[SC::N + from]);
         }
     }
-    float *trows = jrows + 2 * n_joints * jw;
-    for (int t = lane; t < n_thrusters; t += 32) {
-        const uint32_t *th = lv + SC::LV_THR + 8 * t;
+    if (thr_lane) {
         const uint32_t tp = th[0];
-        float *o = trows + t * 6;
+        float *o = img + n_shapes * 29 + 2 * n_joints * jw + t * 6;
         for (int f = 0; f < 6; ++f) o[f] = 0.0f;
         if ((tp >> 20) & 1u) {
-            const int i = tp & 255;
+            const int k = tp & 255;
             float dx, dy;
-            rot2(cs[i], cs[SC::N + i], __uint_as_float(th[3]), __uint_as_float(th[4]), dx, dy);
+            rot2(cs[k], cs[SC::N + k], __uint_as_float(th[3]), __uint_as_float(th[4]), dx, dy);
             o[0] = 1.0f; o[1] = __uint_as_float(th[1]); o[2] = __uint_as_float(th[2]); o[3] = __uint_as_float(th[5]);
             o[4] = dy; o[5] = dx;
         }
