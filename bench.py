@@ -44,14 +44,26 @@ FLOPS = dict(body=37, circle_box=4, polygon=84, box_test=8, cc=16, pc=94, pp=190
              joint_fixed=48 + 33 + 18 + 8, joint_iter=38, thruster=27)
 
 
+def kernel_source_sha256() -> str:
+    import hashlib
+    h = hashlib.sha256()
+    for name in ("k2d_kernels.cuh", "k2d_api.cu"):
+        with open(os.path.join(ROOT, "paper_2410_23208_b200", "csrc", name), "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()
+
+
 def ncu_dram_bytes_per_env_launch(size: str, fused: int, n_envs: int):
     """DRAM bytes (read + write) per env that an ncu capture of one k2d_step launch measured for this size class, number of
-    fused steps and env count, from the tracked table of captures; None when no capture of the current kernel matches."""
-    path = os.path.join(ROOT, "profiles", "k2d_step_kernel_dram_traffic.json")
+    fused steps and env count, from the tracked table of captures (JSON text).  None when no capture matches, and None
+    when the kernel sources have changed since the capture (the table carries their hash)."""
+    path = os.path.join(ROOT, "profiles", "k2d_step_kernel_dram_traffic.txt")
     if not os.path.exists(path):
         return None
     with open(path) as f:
         table = json.load(f)
+    if table.get("source_sha256") != kernel_source_sha256():
+        return None
     return table.get("captures", {}).get(f"{size}/{fused}/{n_envs}")
 
 
@@ -278,63 +290,70 @@ def run_gpu(args) -> dict:
     main_stream = torch.cuda.current_stream(dev)
     stages = [stage, torch.empty_like(stage)]
     rewards, dones = [reward, torch.empty_like(reward)], [done, torch.empty_like(done)]
-    ev_up = [torch.cuda.Event() for _ in range(K + 3)]
-    ev_done = [torch.cuda.Event() for _ in range(K + 3)]
-    ev_down = [torch.cuda.Event() for _ in range(K + 3)]
-
-    def upload(i):
-        with torch.cuda.stream(copy_stream):
-            if i >= 2:
-                copy_stream.wait_event(ev_done[i - 2])       # the launch that last read this staging buffer
-            stages[i % 2].copy_(host_actions[i % len(host_actions)], non_blocking=True)
-            ev_up[i].record(copy_stream)
-
-    def run(i):
-        main_stream.wait_event(ev_up[i])
-        if i >= 2:
-            main_stream.wait_event(ev_down[i - 2])           # its results have been read back
-        env.step(stages[i % 2], rewards[i % 2], dones[i % 2])
-        env.obs(obs)
-        ev_done[i].record(main_stream)
-
-    def download(i):
-        with torch.cuda.stream(copy_stream):
-            copy_stream.wait_event(ev_done[i])
-            host_reward.copy_(rewards[i % 2], non_blocking=True)
-            host_done.copy_(dones[i % 2], non_blocking=True)
-            ev_down[i].record(copy_stream)
-
-    barrier()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record()
-    copy_stream.wait_event(e0)
-    upload(0)
-    for i in range(K):
-        run(i)
-        if i + 1 < K:
-            upload(i + 1)
-        download(i)
-    main_stream.wait_event(ev_down[K - 1])
-    e1.record()
-    barrier()
-    e2e_ms = e0.elapsed_time(e1)
-
-    # ---- the same loop with the observation copied to the host as well (a learner on the host, or logging)
+    obses = [obs, torch.empty_like(obs)]
     host_obs = torch.empty(obs.shape, dtype=obs.dtype).pin_memory()
-    K_OBS = min(K, 8)
+
+    def e2e_loop(n, with_obs):
+        """n bench steps; with_obs: the observation of every step is copied to pinned host memory as well (two device
+        observation buffers, so that the copy of step i overlaps the launches of step i + 1)"""
+        ev_up = [torch.cuda.Event() for _ in range(n + 3)]
+        ev_done = [torch.cuda.Event() for _ in range(n + 3)]
+        ev_down = [torch.cuda.Event() for _ in range(n + 3)]
+
+        def upload(i):
+            with torch.cuda.stream(copy_stream):
+                if i >= 2:
+                    copy_stream.wait_event(ev_done[i - 2])       # the launch that last read this staging buffer
+                stages[i % 2].copy_(host_actions[i % len(host_actions)], non_blocking=True)
+                ev_up[i].record(copy_stream)
+
+        def run(i):
+            main_stream.wait_event(ev_up[i])
+            if i >= 2:
+                main_stream.wait_event(ev_down[i - 2])           # its results have been read back
+            env.step(stages[i % 2], rewards[i % 2], dones[i % 2])
+            env.obs(obses[i % 2 if with_obs else 0])
+            ev_done[i].record(main_stream)
+
+        def download(i):
+            with torch.cuda.stream(copy_stream):
+                copy_stream.wait_event(ev_done[i])
+                host_reward.copy_(rewards[i % 2], non_blocking=True)
+                host_done.copy_(dones[i % 2], non_blocking=True)
+                if with_obs:
+                    host_obs.copy_(obses[i % 2], non_blocking=True)
+                ev_down[i].record(copy_stream)
+
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        copy_stream.wait_event(e0)
+        upload(0)
+        for i in range(n):
+            run(i)
+            if i + 1 < n:
+                upload(i + 1)
+            download(i)
+        main_stream.wait_event(ev_down[n - 1])
+        e1.record()
+        barrier()
+        return e0.elapsed_time(e1)
+
+    e2e_ms = e2e_loop(K, False)
+    # ---- the same loop with the observation copied to the host as well (a learner on the host, or logging)
+    K_OBS = min(K, 16)
+    e2e_obs_ms = e2e_loop(K_OBS, True) * K / K_OBS
+
+    # ---- how fast this GPU takes a stream of plain stores: the 256 MiB flush buffer filled five times (a yardstick for the
+    # observation kernels, which write five to sixty times what they read; the copy figure in `peak` is half reads)
+    fill_ev = [torch.cuda.Event(enable_timing=True) for _ in range(6)]
+    flush.fill_(1)
+    for i in range(5):
+        fill_ev[i].record()
+        flush.fill_(i)
+    fill_ev[5].record()
     barrier()
-    o0, o1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    o0.record()
-    for i in range(K_OBS):
-        stages[0].copy_(host_actions[i % len(host_actions)], non_blocking=True)
-        env.step(stages[0], rewards[0], dones[0])
-        env.obs(obs)
-        host_reward.copy_(rewards[0], non_blocking=True)
-        host_done.copy_(dones[0], non_blocking=True)
-        host_obs.copy_(obs, non_blocking=True)
-    o1.record()
-    barrier()
-    e2e_obs_ms = o0.elapsed_time(o1) * K / K_OBS
+    write_only_gbs = flush.numel() / (min(fill_ev[i].elapsed_time(fill_ev[i + 1]) for i in range(5)) * 1e-3) / 1e9
 
     # ---- other ways to drive the same path (L2 not flushed; the state of 16384 envs stays in L2 between launches anyway):
     # one engine step and one observation per call, as a training loop does, with two launches and with the fused launch
@@ -406,7 +425,7 @@ def run_gpu(args) -> dict:
         "e2e_with_obs": {"value": world * env_steps_per_launch * K / (e2e_obs_ms * 1e-3), "unit": UNIT,
                          "h2d_bytes_per_step": int(stage.numel() * 4),
                          "d2h_bytes_per_step": int(host_reward.numel() * 4 + host_done.numel() + host_obs.numel() * host_obs.element_size()),
-                         "note": "as e2e, and the observation is copied to pinned host memory every bench step; no overlap of copies and launches"},
+                         "note": "as e2e, and the observation is copied to pinned host memory every bench step (two device observation buffers; the copy overlaps the next step's launches)"},
         "modes": {k: {"ms_per_call": v, "value": world * n_envs / (v * 1e-3), "unit": UNIT,
                       "what": ("k2d_step(1 step) + k2d_obs: two launches per call" if k == "one_step_then_obs"
                                else "k2d_step_obs(1 step): one launch per call")} for k, v in modes.items()},
@@ -420,7 +439,9 @@ def run_gpu(args) -> dict:
                      "hbm": {"achieved": hbm_gbs, "peak": hbm_peak, "unit": "GB/s", "frac": hbm_gbs / hbm_peak, "of": hbm_src,
                              "bytes_per_env_launch": bytes_["step"]},
                      "obs_kernel": {"achieved": obs_gbs, "peak": hbm_peak, "unit": "GB/s", "frac": obs_gbs / hbm_peak,
-                                    "launch_ms": float(np.mean(obs_ms)), "bytes_per_env_launch": bytes_["obs"]}},
+                                    "launch_ms": float(np.mean(obs_ms)), "bytes_per_env_launch": bytes_["obs"],
+                                    "write_only_gbs": write_only_gbs, "frac_of_write_only": obs_gbs / write_only_gbs,
+                                    "write_only_source": "a 256 MiB device buffer filled with torch's fill kernel, best of five, timed in this run"}},
         "work": {"manifolds_per_env_step": float(counts[2]) / max(1, int(counts[3])), "active_pairs_per_env_step": mean_pairs,
                  "resets": int(counts[1]), "nonfinite": int(counts[0]), "wall_s_timed_region": t_wall},
     }

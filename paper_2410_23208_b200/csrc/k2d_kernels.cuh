@@ -30,7 +30,7 @@ constexpr int kBlockThreads = K2D_BLOCK_THREADS;
 #define K2D_MIN_BLOCKS 5
 #endif
 constexpr int kMinBlocks = K2D_MIN_BLOCKS;   // resident blocks per SM the step kernel is compiled for (bounds its registers)
-constexpr int kObsThreads = 128;   // observation kernel: one warp per env, four envs per block
+constexpr int kObsThreads = 128;   // observation kernel: one half-warp per env, eight envs per block
 constexpr int kMaxActions = 16;
 enum { Q_TICKET = 0, Q_LEFT = 1, Q_ERROR = 2 };
 constexpr unsigned kWaitLimit = 1u << 24;   // default number of polls (about 100 ns apart) before a wait for another group's chunk gives up
@@ -1843,29 +1843,32 @@ __global__ void k2d_reset_kernel(uint32_t *state, const uint32_t *levels, const 
     }
 }
 
-// ---------------------------------------------------------------- observation kernel: one warp per env
-// Lanes 0..15 write one shape row each, lanes 16..27 one side of a joint each, lanes 28..29 a thruster row each, into the
-// warp's shared-memory image of the observation; then the warp copies the image out with coalesced stores.  Every lane asks
-// for all the words of the state record and of the level record its row needs before it uses the first of them.
-static_assert(K2D_MAX_SHAPES <= 16 && 2 * K2D_MAX_JOINTS <= 12 && K2D_MAX_THRUSTERS <= 2, "observation rows: one lane each");
+// ---------------------------------------------------------------- observation kernel: one half-warp per env
+// The 16 lanes of an env first ask for every word of the state record and of the level record that their rows need (lane l:
+// shape l, joint side l, thruster l - 12), clear the env's shared-memory image of the observation while the loads are in
+// flight, then write one shape row each, then one joint side or thruster row each, and copy the image out with coalesced
+// stores.  Two envs share every instruction of a warp.
+static_assert(K2D_MAX_SHAPES <= 16 && 2 * K2D_MAX_JOINTS <= 12 && K2D_MAX_THRUSTERS <= 4, "observation rows: one lane of sixteen each");
+constexpr int kObsEnvsPerBlock = 2 * (kObsThreads / 32);
 template <class SC>
 __global__ void __launch_bounds__(kObsThreads) k2d_obs_kernel(const uint32_t *state, const uint32_t *levels, float *obs,
                                                               int n_envs, int n_actions, int n_polygons, int n_circles,
                                                               int n_joints, int n_thrusters) {
     extern __shared__ __align__(16) float obs_smem[];
-    const int w = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int e = blockIdx.x * (kObsThreads / 32) + w;
-    if (e >= n_envs) return;
+    const int w = threadIdx.x >> 5, lane = threadIdx.x & 31, half = lane >> 4, hl = lane & 15;
+    const int e = blockIdx.x * kObsEnvsPerBlock + 2 * w + half;
+    if (blockIdx.x * kObsEnvsPerBlock + 2 * w >= n_envs) return;     // the whole warp is past the last env
+    const bool live = e < n_envs;
     const int n_shapes = n_polygons + n_circles;
     const int jw = 11 + n_actions;
     const int width = n_shapes * 29 + 2 * n_joints * jw + 6 * n_thrusters;
-    float *img = obs_smem + (size_t)w * ((width + 2 * SC::N + 3) / 4 * 4);
+    float *img = obs_smem + (size_t)(2 * w + half) * ((width + 2 * SC::N + 3) / 4 * 4);
     float *cs = img + width;                 // cos, sin of every shape's angle
-    const uint32_t *st = state + (size_t)e * SC::ST_WORDS;
+    const uint32_t *st = state + (size_t)(live ? e : 0) * SC::ST_WORDS;
     const float *stf = reinterpret_cast<const float *>(st);
     // the state words of this lane's shape do not wait for the level id
-    const bool shape_lane = lane < n_shapes;
-    const int i = shape_lane ? (lane < n_polygons ? lane : SC::P + (lane - n_polygons)) : 0;     // internal shape index
+    const bool shape_lane = live && hl < n_shapes;
+    const int i = shape_lane ? (hl < n_polygons ? hl : SC::P + (hl - n_polygons)) : 0;     // internal shape index
     float sx = 0.0f, sy = 0.0f, sth = 0.0f, svx = 0.0f, svy = 0.0f, sw = 0.0f;
     if (shape_lane) { sx = stf[i]; sy = stf[SC::N + i]; sth = stf[2 * SC::N + i]; svx = stf[3 * SC::N + i]; svy = stf[4 * SC::N + i]; sw = stf[5 * SC::N + i]; }
     const uint32_t *lv = levels + (size_t)st[SC::ST_META + META_LEVEL] * SC::LV_WORDS;
@@ -1873,12 +1876,11 @@ __global__ void __launch_bounds__(kObsThreads) k2d_obs_kernel(const uint32_t *st
     const bool poly = i < SC::P;
     uint32_t fl = 0u;
     float c_im = 0.0f, c_ii = 0.0f, c_de = 0.0f, c_fr = 0.0f, c_re = 0.0f, c_rad = 0.0f, pv[8] = { 0.0f, 0.0f, 0.0f, 0.0f, 0.0f, 0.0f, 0.0f, 0.0f };
-    const int row = lane - 16, j = row >> 1, d = row & 1;                 // joint lanes
-    const bool joint_lane = row >= 0 && row < 2 * n_joints;
-    uint32_t jl[8] = { 0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u };                 // packed word, anchors, speed, power, kind
-    const int t = lane - 28;                                               // thruster lanes
-    const bool thr_lane = t >= 0 && t < n_thrusters;
-    uint32_t th[6] = { 0u, 0u, 0u, 0u, 0u, 0u };
+    const int j = hl >> 1, d = hl & 1;                                     // joint side
+    const bool joint_lane = live && hl < 2 * n_joints;
+    const int t = hl - 12;                                                 // thruster
+    const bool thr_lane = live && t >= 0 && t < n_thrusters;
+    uint32_t rw[8] = { 0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u };                 // joint: packed word, anchors, speed, power, kind; thruster: its record
     if (shape_lane) {
         fl = __ldg(lv + SC::LV_FLAGS + i);
         c_im = __ldg(lvf + SC::LV_IM + i); c_ii = __ldg(lvf + SC::LV_II + i); c_de = __ldg(lvf + SC::LV_DENS + i);
@@ -1891,81 +1893,81 @@ __global__ void __launch_bounds__(kObsThreads) k2d_obs_kernel(const uint32_t *st
     if (joint_lane) {
         const uint32_t *src = lv + SC::LV_JOINT + kJointLevelWords * j;
 #pragma unroll
-        for (int q = 0; q < 7; ++q) jl[q] = __ldg(src + q);
-        jl[7] = __ldg(src + 10);
-    }
-    if (thr_lane) {
+        for (int q = 0; q < 7; ++q) rw[q] = __ldg(src + q);
+        rw[7] = __ldg(src + 10);
+    } else if (thr_lane) {
         const uint32_t *src = lv + SC::LV_THR + 8 * t;
 #pragma unroll
-        for (int q = 0; q < 6; ++q) th[q] = __ldg(src + q);
+        for (int q = 0; q < 6; ++q) rw[q] = __ldg(src + q);
     }
+    // absent entities and unset columns are zero
+    if (live) {
+        float4 *z = reinterpret_cast<float4 *>(img);
+        for (int q = hl; q < (width + 3) / 4; q += 16) z[q] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+    }
+    __syncwarp();
     if (shape_lane) {
         float c, sn;
         sincos_spec(sth, c, sn);
         cs[i] = c; cs[SC::N + i] = sn;
-        float *o = img + lane * 29;
-        if (!(fl & F_ACTIVE)) {
-            for (int f = 0; f < 29; ++f) o[f] = 0.0f;
-        } else {
+        if (fl & F_ACTIVE) {
+            float *o = img + hl * 29;
             const int nv = flag_nverts(fl);
             const uint32_t role = flag_role(fl);
             o[0] = sx; o[1] = sy; o[2] = svx; o[3] = svy;
             o[4] = c_im; o[5] = c_ii; o[6] = c_de;
             o[7] = tanh_spec(sw * 0.1f);
-#pragma unroll
-            for (int r = 0; r < 4; ++r) o[8 + r] = (role == (uint32_t)r) ? 1.0f : 0.0f;
+            o[8 + role] = 1.0f;
             o[12] = sn; o[13] = c; o[14] = c_fr; o[15] = c_re;
-            o[16] = poly ? 1.0f : 0.0f; o[17] = poly ? 0.0f : 1.0f;
-            o[18] = poly ? 0.0f : c_rad;
+            if (poly) {
+                o[16] = 1.0f;
 #pragma unroll
-            for (int k = 0; k < 4; ++k) {
-                const bool on = poly && k < nv;
-                o[19 + 2 * k] = on ? pv[2 * k] : 0.0f;
-                o[20 + 2 * k] = on ? pv[2 * k + 1] : 0.0f;
+                for (int k = 0; k < 4; ++k) {
+                    if (k < nv) { o[19 + 2 * k] = pv[2 * k]; o[20 + 2 * k] = pv[2 * k + 1]; }
+                }
+                o[nv == 3 ? 27 : 28] = 1.0f;
+            } else {
+                o[17] = 1.0f; o[18] = c_rad;
             }
-            o[27] = (poly && nv == 3) ? 1.0f : 0.0f;
-            o[28] = (poly && nv != 3) ? 1.0f : 0.0f;
         }
     }
     __syncwarp();
     if (joint_lane) {
-        const uint32_t jab = jl[0];
-        float *o = img + n_shapes * 29 + row * jw;
-        for (int f = 0; f < jw; ++f) o[f] = 0.0f;
+        const uint32_t jab = rw[0];
         if ((jab >> 28) & 1u) {
+            float *o = img + n_shapes * 29 + hl * jw;
             const int a = jab & 255, b = (jab >> 8) & 255;
             const int from = d ? b : a, to = d ? a : b;
-            o[0] = 1.0f; o[1] = (jl[7] & 1u) ? 1.0f : 0.0f;
+            o[0] = 1.0f; o[1] = (rw[7] & 1u) ? 1.0f : 0.0f;
             // anchor on the "from" shape, then on the "to" shape
-            o[2] = __uint_as_float(d ? jl[3] : jl[1]); o[3] = __uint_as_float(d ? jl[4] : jl[2]);
-            o[4] = __uint_as_float(d ? jl[1] : jl[3]); o[5] = __uint_as_float(d ? jl[2] : jl[4]);
-            o[6] = __uint_as_float(jl[6]); o[7] = __uint_as_float(jl[5]);
+            o[2] = __uint_as_float(d ? rw[3] : rw[1]); o[3] = __uint_as_float(d ? rw[4] : rw[2]);
+            o[4] = __uint_as_float(d ? rw[1] : rw[3]); o[5] = __uint_as_float(d ? rw[2] : rw[4]);
+            o[6] = __uint_as_float(rw[6]); o[7] = __uint_as_float(rw[5]);
             const int bind = (int)((jab >> 16) & 255);
             if (bind < n_actions) o[9 + bind] = 1.0f;
             o[9 + n_actions] = __fmaf_rn(cs[SC::N + to], cs[from], -(cs[to] * cs[SC::N + from]));
             o[10 + n_actions] = __fmaf_rn(cs[to], cs[from], cs[SC::N + to] * cs[SC::N + from]);
         }
-    }
-    if (thr_lane) {
-        const uint32_t tp = th[0];
-        float *o = img + n_shapes * 29 + 2 * n_joints * jw + t * 6;
-        for (int f = 0; f < 6; ++f) o[f] = 0.0f;
+    } else if (thr_lane) {
+        const uint32_t tp = rw[0];
         if ((tp >> 20) & 1u) {
+            float *o = img + n_shapes * 29 + 2 * n_joints * jw + t * 6;
             const int k = tp & 255;
             float dx, dy;
-            rot2(cs[k], cs[SC::N + k], __uint_as_float(th[3]), __uint_as_float(th[4]), dx, dy);
-            o[0] = 1.0f; o[1] = __uint_as_float(th[1]); o[2] = __uint_as_float(th[2]); o[3] = __uint_as_float(th[5]);
+            rot2(cs[k], cs[SC::N + k], __uint_as_float(rw[3]), __uint_as_float(rw[4]), dx, dy);
+            o[0] = 1.0f; o[1] = __uint_as_float(rw[1]); o[2] = __uint_as_float(rw[2]); o[3] = __uint_as_float(rw[5]);
             o[4] = dy; o[5] = dx;
         }
     }
     __syncwarp();
+    if (!live) return;
     float *out = obs + (size_t)e * width;
     if (((width & 3) == 0) && ((reinterpret_cast<uintptr_t>(obs) & 15) == 0)) {
         const float4 *src = reinterpret_cast<const float4 *>(img);
         float4 *dst = reinterpret_cast<float4 *>(out);
-        for (int q = lane; q < width / 4; q += 32) dst[q] = src[q];
+        for (int q = hl; q < width / 4; q += 16) dst[q] = src[q];
     } else {
-        for (int q = lane; q < width; q += 32) out[q] = img[q];
+        for (int q = hl; q < width; q += 16) out[q] = img[q];
     }
 }
 
