@@ -663,6 +663,76 @@ __device__ __noinline__ void slow_batched_iteration(float *sm, uint32_t *ovf, in
     }
 }
 
+// ---- all solver iterations of a scene in the batched order (paper, "Parallelised Computation and Batched Impulse Resolution"),
+// from the lanes' own records: the rank of a manifold among the scene's active manifolds (pair order, slot 0 then 1) gives
+// its batch, rank mod n_batches; per batch every row is solved against the velocities as they stand (its lane's private
+// copy), then the batch's impulses are applied level by level, which is the canonical order on every body.  For scenes
+// without second records.  Returns the accumulated impulses of the lane's first manifold.  Out of line: the default order
+// is the sequential one.
+template <class SC, int G>
+__device__ __noinline__ float2 batched_iterations(float *sm, Rec rec, uint32_t jab, int jlevel, int jmax, int cmax, int clevel,
+                                                  int solver_iters, float motor_rho, int n_batches) {
+    Group<G> g;
+    const int lane = g.lane;
+    const uint32_t ab = rec.ab;
+    const int a = ck_idx<CK_BODY>(ab & 31, SC::N), b = ck_idx<CK_BODY>((ab >> 5) & 31, SC::N);
+    const unsigned amask = (ab >> 10) & 3u;
+    float *lf = sm + SC::STG + lane;                 // this lane's fields: field f at lf[f * G]
+    const unsigned has0 = g.ballot(amask & 1u), has1 = g.ballot(amask & 2u);
+    const int rank0 = __popc(has0 & g.lanes_below()) + __popc(has1 & g.lanes_below());
+    const int b0 = (amask & 1u) ? rank0 % n_batches : -1;
+    const int b1 = (amask & 2u) ? (rank0 + (int)(amask & 1u)) % n_batches : -1;
+#pragma unroll 1
+    for (int it = 0; it < solver_iters; ++it) {
+        sweep_joints<SC, G, 1>(sm, jab, lane, jlevel, jmax, motor_rho);
+#pragma unroll 1
+        for (int bt = 0; bt < n_batches; ++bt) {
+            const bool in0 = b0 == bt, in1 = b1 == bt;
+            if (!g.any(in0 || in1)) break;      // batches are filled in order: the first empty one ends the sweep
+            float d0n = 0.0f, d0t = 0.0f, d1n = 0.0f, d1t = 0.0f;
+            if (in0 || in1) {
+                const float4 va4 = ld4(sm + SC::BVEL + 4 * a), vb4 = ld4(sm + SC::BVEL + 4 * b);
+                if (in0) {
+                    float vax = va4.x, vay = va4.y, wa = va4.z, vbx = vb4.x, vby = vb4.y, wb = vb4.z;
+                    const float old_n = rec.accn, old_t = rec.acct;
+                    manifold_rows<1>(rec.nx, rec.ny, rec.mu, rec.ma, rec.mb, rec.ia, rec.ib, rec.rna, rec.rnb, rec.rta, rec.rtb,
+                                     rec.massn, rec.masst, rec.target, rec.accn, rec.acct, vax, vay, wa, vbx, vby, wb);
+                    d0n = rec.accn - old_n; d0t = rec.acct - old_t;
+                }
+                if (in1) {
+                    float vax = va4.x, vay = va4.y, wa = va4.z, vbx = vb4.x, vby = vb4.y, wb = vb4.z;
+                    const float old_n = lf[LF_ACC2N * G], old_t = lf[LF_ACC2T * G];
+                    float accn = old_n, acct = old_t;
+                    manifold_rows<1>(rec.nx, rec.ny, rec.mu, rec.ma, rec.mb, rec.ia, rec.ib, lf[M2_RNA * G], lf[M2_RNB * G], lf[M2_RTA * G],
+                                     lf[M2_RTB * G], lf[M2_MASSN * G], lf[M2_MASST * G], lf[M2_TARGET * G], accn, acct, vax, vay, wa, vbx, vby, wb);
+                    lf[LF_ACC2N * G] = accn; lf[LF_ACC2T * G] = acct;
+                    d1n = accn - old_n; d1t = acct - old_t;
+                }
+            }
+            g.sync();
+#pragma unroll 1
+            for (int lvl = 1; lvl <= cmax; ++lvl) {
+                if (clevel == lvl && (in0 || in1)) {
+                    const float4 va4 = ld4(sm + SC::BVEL + 4 * a), vb4 = ld4(sm + SC::BVEL + 4 * b);
+                    float vax = va4.x, vay = va4.y, wa = va4.z, vbx = vb4.x, vby = vb4.y, wb = vb4.z;
+                    if (in0) {
+                        apply_impulse(d0n, rec.nx, rec.ny, rec.ma, rec.mb, rec.ia * rec.rna, rec.ib * rec.rnb, vax, vay, wa, vbx, vby, wb);
+                        apply_impulse(d0t, -rec.ny, rec.nx, rec.ma, rec.mb, rec.ia * rec.rta, rec.ib * rec.rtb, vax, vay, wa, vbx, vby, wb);
+                    }
+                    if (in1) {
+                        apply_impulse(d1n, rec.nx, rec.ny, rec.ma, rec.mb, rec.ia * lf[M2_RNA * G], rec.ib * lf[M2_RNB * G], vax, vay, wa, vbx, vby, wb);
+                        apply_impulse(d1t, -rec.ny, rec.nx, rec.ma, rec.mb, rec.ia * lf[M2_RTA * G], rec.ib * lf[M2_RTB * G], vax, vay, wa, vbx, vby, wb);
+                    }
+                    if ((ab >> 26) & 1u) st4(sm + SC::BVEL + 4 * a, vax, vay, wa);
+                    if ((ab >> 27) & 1u) st4(sm + SC::BVEL + 4 * b, vbx, vby, wb);
+                }
+                g.sync();
+            }
+        }
+    }
+    return make_float2(rec.accn, rec.acct);
+}
+
 // Records from the staged manifolds (the first G in shared memory, the rest already in scratch),
 // their levels, warm start and all solver iterations, joints included.  old_n / old_t: this lane's
 // first-manifold accumulated impulses of the previous step.  Returns the highest contact level.
@@ -741,7 +811,7 @@ __device__ __noinline__ int slow_solve(float *sm, uint32_t *ovf, int nrec, uint3
     sweep_joints<SC, G, 0>(sm, jab, lane, jlevel, jmax, motor_rho);
     for (int it = 0; it < solver_iters; ++it) {
         sweep_joints<SC, G, 1>(sm, jab, lane, jlevel, jmax, motor_rho);
-        if (n_batches > 0) slow_batched_iteration<SC, G>(sm, ovf, nrec, cmax, nman, n_batches);
+        if (nman > n_batches) slow_batched_iteration<SC, G>(sm, ovf, nrec, cmax, nman, n_batches);     // else one row per batch: the sequential sweep
         else slow_sweep_pairs<SC, G, 1>(sm, ovf, nrec, cmax);
     }
     return cmax;
@@ -1506,8 +1576,9 @@ struct Scene {
         g.sync();
         c_rec += (unsigned)nrec << 16;
 
-        // crowded scenes, and every scene with contacts when the batched contact solve is asked for, go through the memory records
-        const bool overflow = nrec > G + G / 2 || (prm.n_batches > 0 && nrec > 0);
+        // Crowded scenes go through the memory records; with the batched contact solve asked for, so does every scene with
+        // second records (more touching pairs than lanes).  The others run their batches from the lanes' records, below.
+        const bool overflow = nrec > G + G / 2 || (prm.n_batches > 0 && nrec > G);
         int cmax = 0, clevel = 0, clevel2 = 0;
         if (overflow) {
             cmax = slow_solve<SC, G>(sm, ovf, nrec, jab, jlevel, jmax, prm.solver_iters, prm.warm_start, prm.motor_rho,
@@ -1596,15 +1667,24 @@ struct Scene {
                 clevel = lvl;
                 cmax = g.max_int(lvl);
             }
-            c_man += (unsigned)(__popc(g.ballot(amask & 1u)) + __popc(g.ballot(amask & 2u)));
+            const int nman = __popc(g.ballot(amask & 1u)) + __popc(g.ballot(amask & 2u));
+            c_man += (unsigned)nman;
+            // The i-th active manifold goes to batch i mod n_batches: with no more active manifolds than batches every batch
+            // holds at most one row and the batched order is the sequential one, which the level schedule reproduces.
+            const bool batched = prm.n_batches > 0 && nman > prm.n_batches;
             // warm start: contacts, then joints
             sweep_pairs<0>(cmax, clevel, clevel2);
             sweep_joints<SC, G, 0>(sm, jab, lane, jlevel, jmax, prm.motor_rho);
             // solver iterations: joints, then contacts
+            if (batched) {
+                const float2 acc = batched_iterations<SC, G>(sm, rec, jab, jlevel, jmax, cmax, clevel, prm.solver_iters, prm.motor_rho, prm.n_batches);
+                rec.accn = acc.x; rec.acct = acc.y;
+            } else {
 #pragma unroll 1
-            for (int it = 0; it < prm.solver_iters; ++it) {
-                sweep_joints<SC, G, 1>(sm, jab, lane, jlevel, jmax, prm.motor_rho);
-                sweep_pairs<1>(cmax, clevel, clevel2);
+                for (int it = 0; it < prm.solver_iters; ++it) {
+                    sweep_joints<SC, G, 1>(sm, jab, lane, jlevel, jmax, prm.motor_rho);
+                    sweep_pairs<1>(cmax, clevel, clevel2);
+                }
             }
         }
         // Euler step with the solved velocities
