@@ -49,6 +49,7 @@ extern "C" {
 #define K2D_ERR_LIMIT (-8)         /* a size is beyond a limit built into the library    */
 #define K2D_ERR_WAIT (-9)          /* k2d_status: a wait inside k2d_step ran out (see there) */
 #define K2D_ERR_CHECK (-10)        /* k2d_status of a checked build: an index was out of range    */
+#define K2D_ERR_BUILD (-11)        /* the call needs a build of the library with another compile flag */
 
 #define K2D_MAX_POLYGONS 12
 #define K2D_MAX_CIRCLES 4
@@ -266,6 +267,15 @@ int k2d_trace_slots(const k2d_state *s);
  * slots, counts) with its limit; a violation is recorded (k2d_status then returns K2D_ERR_CHECK until the next
  * k2d_reset) and the access is redirected to index 0; nothing traps.  It stands in for a memory checker. */
 int k2d_is_checked_build(void);
+
+/* Measurement aid.  In a library compiled with -DK2D_PHASE_CLOCKS the step kernel adds up, per phase of an environment
+ * step (Algorithm 1's stages as this library cuts them), the SM cycles that every scene group spends in it.  The call waits
+ * for the handle's stream, copies the first n (<= K2D_PHASES) sums to host_cycles and clears them.  Order of the phases:
+ * world geometry and boxes; motors and thrusters; joint pre-step; box test; narrowphase; contact pre-step (records);
+ * solver levels; warm start; solver iterations; Euler step and positional corrections; reward / done / reset; the whole
+ * contact solve of scenes on the memory-record path; state load; state store.  In any other build: zeros and K2D_ERR_BUILD. */
+#define K2D_PHASES 14
+int k2d_phase_cycles(k2d_state *s, uint64_t *host_cycles, int32_t n);
 
 /* Test aid.  With more envs than the device holds scene groups, k2d_step hands out runs of 8 steps of an env to whichever
  * group is free; a group that gets a later run of an env before the earlier one is back in memory polls for it, about

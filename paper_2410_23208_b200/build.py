@@ -23,6 +23,7 @@ NVCC_FLAGS = [
 
 
 LIB_CHECKED = os.path.join(HERE, "libk2d_checked.so")
+LIB_PHASES = os.path.join(HERE, "libk2d_phases.so")
 
 
 def needs_build(lib: str = LIB) -> bool:
@@ -32,13 +33,17 @@ def needs_build(lib: str = LIB) -> bool:
     return any(os.path.getmtime(d) > t for d in DEPS)
 
 
-def build(force: bool = False, verbose: bool = False, checked: bool = False) -> str:
-    """The library, or (checked=True) the build with index checks in the kernels (-DK2D_CHECKED)."""
-    lib = LIB_CHECKED if checked else LIB
+def build(force: bool = False, verbose: bool = False, checked: bool = False, phase_clocks: bool = False) -> str:
+    """The library, or (checked=True) the build with index checks in the kernels (-DK2D_CHECKED), or (phase_clocks=True)
+    the build whose step kernel adds up the cycles spent per phase of a step (-DK2D_PHASE_CLOCKS)."""
+    if checked and phase_clocks:
+        raise ValueError("one variant at a time")
+    lib = LIB_CHECKED if checked else (LIB_PHASES if phase_clocks else LIB)
     if not force and not needs_build(lib):
         return lib
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
-    cmd = [nvcc, *NVCC_FLAGS, *(["-DK2D_CHECKED"] if checked else []), "-I", os.path.join(ROOT, "include"), "-o", lib, SRC]
+    defines = (["-DK2D_CHECKED"] if checked else []) + (["-DK2D_PHASE_CLOCKS"] if phase_clocks else [])
+    cmd = [nvcc, *NVCC_FLAGS, *defines, "-I", os.path.join(ROOT, "include"), "-o", lib, SRC]
     if verbose:
         cmd.insert(1, "-Xptxas")
         cmd.insert(2, "-v")
@@ -47,4 +52,4 @@ def build(force: bool = False, verbose: bool = False, checked: bool = False) -> 
 
 
 if __name__ == "__main__":
-    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv, checked="--checked" in sys.argv))
+    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv, checked="--checked" in sys.argv, phase_clocks="--phase-clocks" in sys.argv))

@@ -653,6 +653,25 @@ int k2d_is_checked_build(void) {
 #endif
 }
 
+int k2d_phase_cycles(k2d_state *s, uint64_t *host_cycles, int32_t n) {
+    if (!s || !host_cycles) return K2D_ERR_NULL;
+    if (n < 0 || n > K2D_PHASES) return K2D_ERR_ARG;
+    static_assert(K2D_PHASES == PH_COUNT, "the header's phase count is the kernels'");
+#ifdef K2D_PHASE_CLOCKS
+    CUDA_OK(cudaSetDevice(s->cfg.device));
+    CUDA_OK(cudaStreamSynchronize(s->stream));
+    unsigned long long sums[PH_COUNT];
+    CUDA_OK(cudaMemcpyFromSymbol(sums, k2d_phase_sums, sizeof(sums)));
+    for (int i = 0; i < n; ++i) host_cycles[i] = (uint64_t)sums[i];
+    std::memset(sums, 0, sizeof(sums));
+    CUDA_OK(cudaMemcpyToSymbol(k2d_phase_sums, sums, sizeof(sums)));
+    return K2D_OK;
+#else
+    for (int i = 0; i < n; ++i) host_cycles[i] = 0;
+    return K2D_ERR_BUILD;
+#endif
+}
+
 int k2d_set_wait_limit(k2d_state *s, uint32_t polls) {
     if (!s) return K2D_ERR_NULL;
     s->wait_limit = polls < 64u ? 64u : polls;
@@ -750,6 +769,7 @@ const char *k2d_error_string(int code) {
         case K2D_ERR_ARG: return "invalid argument";
         case K2D_ERR_LIMIT: return "size beyond a built-in limit";
         case K2D_ERR_CHECK: return "an index check of the checked build failed";
+        case K2D_ERR_BUILD: return "this build of the library does not have that feature compiled in";
         case K2D_ERR_WAIT: return "a scene group gave up waiting for another; the last step is incomplete";
         default: return "unknown error";
     }

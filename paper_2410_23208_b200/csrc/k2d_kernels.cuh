@@ -179,6 +179,21 @@ template <int CODE>
 __device__ __forceinline__ int ck_idx(int v, int) { return v; }
 #endif
 
+// With -DK2D_PHASE_CLOCKS the step kernel adds up, per phase of a step, the cycles that lane 0 of every scene group spends
+// in it (clock64 at the phase boundaries, one atomic add per boundary): k2d_phase_cycles reads the sums.  The phases:
+enum { PH_GEOMETRY, PH_ACTUATORS, PH_JOINT_PRESTEP, PH_BOX_TEST, PH_NARROWPHASE, PH_RECORDS, PH_LEVELS, PH_WARM_START, PH_ITERATIONS,
+       PH_INTEGRATE_CORRECT, PH_EPILOGUE, PH_MEMORY_RECORD_SOLVE, PH_LOAD, PH_STORE, PH_COUNT };
+#ifdef K2D_PHASE_CLOCKS
+__device__ unsigned long long k2d_phase_sums[PH_COUNT];
+#define K2D_PHASE_BEGIN() long long ph_t = clock64()
+#define K2D_PHASE_RESTART() ph_t = clock64()
+#define K2D_PHASE(i) do { const long long ph_n = clock64(); if (lane == 0) atomicAdd(&k2d_phase_sums[i], (unsigned long long)(ph_n - ph_t)); ph_t = ph_n; } while (0)
+#else
+#define K2D_PHASE_BEGIN() do { } while (0)
+#define K2D_PHASE_RESTART() do { } while (0)
+#define K2D_PHASE(i) do { } while (0)
+#endif
+
 // ---------------------------------------------------------------- exact helpers
 __device__ __forceinline__ float fmin_cmp(float a, float b) { return a < b ? a : b; }
 __device__ __forceinline__ float fmax_cmp(float a, float b) { return a > b ? a : b; }
@@ -1355,6 +1370,7 @@ struct Scene {
             if (lane == 0) { prm.reward[(size_t)s * prm.n_envs + e] = 0.0f; prm.done[(size_t)s * prm.n_envs + e] = 1; }
             return;
         }
+        K2D_PHASE_BEGIN();
         const uint32_t *lv = prm.levels + (size_t)ck_idx<CK_LEVEL_ID>((int)smu[SC::META + META_LEVEL], prm.n_levels) * SC::LV_WORDS;
         // dense reward: distance between the first green and the first blue shape before the step
         if (prm.dense_kappa != 0.0f && lane == 0) sm[SC::META + META_D0] = green_blue_distance();
@@ -1416,6 +1432,7 @@ struct Scene {
             }
             box4(i) = make_float4(x0, y0, x1, y1);
         }
+        K2D_PHASE(PH_GEOMETRY);
         // motors (joint order), thrusters (thruster order)
         sweep_joints<SC, G, 3>(sm, jab, lane, jlevel, jmax, prm.motor_rho, prm.discrete);
         if (SC::T > 0) {
@@ -1444,6 +1461,7 @@ struct Scene {
                 g.sync();
             }
         }
+        K2D_PHASE(PH_ACTUATORS);
         // joint pre-step (poses only; velocities are not read): the row goes to shared memory
         if (SC::J > 0 && lane < SC::J) {
             float *jr = sm + SC::JROW + kJointWords * lane;
@@ -1488,6 +1506,7 @@ struct Scene {
         }
         g.sync();
 
+        K2D_PHASE(PH_JOINT_PRESTEP);
         // bounding-box test over all pairs -> compact list of surviving pairs, in pair order
         int nsurv = 0, ns_pp, ns_pc;
         {
@@ -1515,6 +1534,7 @@ struct Scene {
         c_surv += (unsigned)ns_pp | ((unsigned)(ns_pc - ns_pp) << 16);
         c_rec += (unsigned)(nsurv - ns_pc);
 
+        K2D_PHASE(PH_BOX_TEST);
         // narrowphase: survivors of one kind at a time; active pairs are staged in pair order
         int nrec = 0;
         bool t_gb = false, t_gr = false;
@@ -1576,6 +1596,7 @@ struct Scene {
         g.sync();
         c_rec += (unsigned)nrec << 16;
 
+        K2D_PHASE(PH_NARROWPHASE);
         // Crowded scenes go through the memory records; with the batched contact solve asked for, so does every scene with
         // second records (more touching pairs than lanes).  The others run their batches from the lanes' records, below.
         const bool overflow = nrec > G + G / 2 || (prm.n_batches > 0 && nrec > G);
@@ -1583,6 +1604,7 @@ struct Scene {
         if (overflow) {
             cmax = slow_solve<SC, G>(sm, ovf, nrec, jab, jlevel, jmax, prm.solver_iters, prm.warm_start, prm.motor_rho,
                                      rec.accn, rec.acct, contact_consts(), prm.n_batches);
+            K2D_PHASE(PH_MEMORY_RECORD_SOLVE);
         } else {
             const ContactConsts cc = contact_consts();
             const bool two = nrec > G;      // some lanes get a second record
@@ -1636,6 +1658,7 @@ struct Scene {
             }
             lanef(LF_ACC2N) = acc2n; lanef(LF_ACC2T) = acc2t;
             sm[SC::WVX + lane] = corr0; sm[SC::WVX + G + lane] = corr1;
+            K2D_PHASE(PH_RECORDS);
             if (two) {
                 const unsigned r2 = second_build<SC, G>(sm, nrec, cc);     // level | active manifolds << 8
                 clevel2 = (int)(r2 & 127u);
@@ -1667,6 +1690,7 @@ struct Scene {
                 clevel = lvl;
                 cmax = g.max_int(lvl);
             }
+            K2D_PHASE(PH_LEVELS);
             const int nman = __popc(g.ballot(amask & 1u)) + __popc(g.ballot(amask & 2u));
             c_man += (unsigned)nman;
             // The i-th active manifold goes to batch i mod n_batches: with no more active manifolds than batches every batch
@@ -1675,6 +1699,7 @@ struct Scene {
             // warm start: contacts, then joints
             sweep_pairs<0>(cmax, clevel, clevel2);
             sweep_joints<SC, G, 0>(sm, jab, lane, jlevel, jmax, prm.motor_rho);
+            K2D_PHASE(PH_WARM_START);
             // solver iterations: joints, then contacts
             if (batched) {
                 const float2 acc = batched_iterations<SC, G>(sm, rec, jab, jlevel, jmax, cmax, clevel, prm.solver_iters, prm.motor_rho, prm.n_batches);
@@ -1687,6 +1712,7 @@ struct Scene {
                 }
             }
         }
+        if (!overflow) K2D_PHASE(PH_ITERATIONS);
         // Euler step with the solved velocities
         for (int i = lane; i < SC::N; i += G) {
             if (smu[SC::BFL + i] & F_ACTIVE) {
@@ -1705,6 +1731,7 @@ struct Scene {
         }
         finite = !g.any(!finite);
 
+        K2D_PHASE(PH_INTEGRATE_CORRECT);
         // where the pairs of this step keep their accumulated impulses for the next one
         for (int i = lane; i < (SC::NPAIRS + 3) / 4; i += G) smu[SC::WIDX + i] = 0xffffffffu;
         const int step_count = (int)smu[SC::META + META_STEP] + 1;
@@ -1748,6 +1775,7 @@ struct Scene {
         g.sync();
         if (done && prm.auto_reset != 0)
             jab = reset_env<SC, G>(smu, prm.levels, prm.n_levels, prm.auto_reset, prm.seed, prm.env_offset + e, prm.counters, jab);
+        K2D_PHASE(PH_EPILOGUE);
     }
 
     // ---- whole launch for one scene
@@ -1755,6 +1783,7 @@ struct Scene {
     // launch, so it is read past the (non-coherent) L1.
     __device__ __forceinline__ void run(int e, int s0, int s1) {
         uint32_t *st = prm.state + (size_t)e * SC::ST_WORDS;
+        K2D_PHASE_BEGIN();
         // everything the state record holds for this lane is asked for in one go (the warm list entries are read a little
         // past the count, inside the record, and dropped below), then the level's constants in a second go
         constexpr int KB = (6 * SC::N + G - 1) / G;
@@ -1801,12 +1830,14 @@ struct Scene {
         }
         if (nwarm > G + G / 2) warm_in<SC, G>(sm, ovf, st + SC::ST_WARM, nwarm);
         g.sync();
+        K2D_PHASE(PH_LOAD);
 #pragma unroll 1
         for (int s = s0; s < s1; ++s) {
             step(e, s);
             g.sync();
             if (((s - s0) & 255) == 255) flush();
         }
+        K2D_PHASE_RESTART();
         // write back
         for (int i = lane; i < 6 * SC::N; i += G) st[SC::ST_BODY + i] = smu[body_word<SC>(i)];
         if (SC::J > 0 && lane < SC::J) {
@@ -1831,6 +1862,7 @@ struct Scene {
         if (nw > G + G / 2) warm_out<SC, G>(ovf, st + SC::ST_WARM, nw);
         flush();
         g.sync();
+        K2D_PHASE(PH_STORE);
         if (prm.obs && s1 == prm.n_steps) {
             ObsDims od; od.n_polygons = prm.n_polygons; od.n_circles = prm.n_circles; od.n_joints = prm.n_joints; od.n_thrusters = prm.n_thrusters; od.n_actions = prm.n_actions;
             write_obs<SC, G>(sm, prm.levels, prm.obs, od, e);

@@ -20,7 +20,7 @@ EXPORTS = (
     "k2d_default_config", "k2d_state_bytes", "k2d_state_bytes_no_scratch", "k2d_level_pool_bytes", "k2d_create", "k2d_reset", "k2d_step",
     "k2d_step_discrete", "k2d_step_static_scratch", "k2d_step_obs", "k2d_obs", "k2d_render",
     "k2d_obs_floats", "k2d_canonical_words", "k2d_get_state", "k2d_set_state", "k2d_status", "k2d_level_info",
-    "k2d_set_trace", "k2d_trace_slots", "k2d_is_checked_build", "k2d_set_wait_limit", "k2d_eval_sincos_tanh", "k2d_measure_fp32_peak", "k2d_error_string", "k2d_destroy",
+    "k2d_set_trace", "k2d_trace_slots", "k2d_is_checked_build", "k2d_phase_cycles", "k2d_set_wait_limit", "k2d_eval_sincos_tanh", "k2d_measure_fp32_peak", "k2d_error_string", "k2d_destroy",
 )
 
 
@@ -55,10 +55,16 @@ LEVEL_DTYPE = np.dtype([
 _libs = {}
 
 
-def load_library(checked: bool = False):
-    """Builds (if stale) and loads libk2d.so (checked=True: the build with index checks); raises if that is impossible."""
-    if checked not in _libs:
-        lib = C.CDLL(_build.build(checked=checked))
+PHASES = ("geometry", "actuators", "joint_prestep", "box_test", "narrowphase", "records", "levels", "warm_start", "iterations",
+          "integrate_correct", "epilogue", "memory_record_solve", "load", "store")
+
+
+def load_library(checked: bool = False, phase_clocks: bool = False):
+    """Builds (if stale) and loads libk2d.so (checked=True: the build with index checks; phase_clocks=True: the build that
+    counts cycles per phase of a step); raises if that is impossible."""
+    key = "checked" if checked else ("phases" if phase_clocks else "")
+    if key not in _libs:
+        lib = C.CDLL(_build.build(checked=checked, phase_clocks=phase_clocks))
         vp, i32 = C.c_void_p, C.c_int32
         lib.k2d_default_config.argtypes = [C.POINTER(Config), i32, i32, i32, i32, i32]
         lib.k2d_state_bytes.argtypes = [C.POINTER(Config)]
@@ -84,13 +90,14 @@ def load_library(checked: bool = False):
         lib.k2d_set_trace.argtypes = [vp, vp]
         lib.k2d_trace_slots.argtypes = [vp]
         lib.k2d_set_wait_limit.argtypes = [vp, C.c_uint32]
+        lib.k2d_phase_cycles.argtypes = [vp, vp, i32]
         lib.k2d_eval_sincos_tanh.argtypes = [vp, i32, vp, vp, vp, vp]
         lib.k2d_measure_fp32_peak.argtypes = [i32, vp, C.c_size_t, vp]
         lib.k2d_error_string.argtypes = [C.c_int]
         lib.k2d_error_string.restype = C.c_char_p
         lib.k2d_destroy.argtypes = [vp]
-        _libs[checked] = lib
-    return _libs[checked]
+        _libs[key] = lib
+    return _libs[key]
 
 
 class K2DError(RuntimeError):
@@ -132,12 +139,12 @@ def make_config(levels: dict, n_envs: int, **kw) -> Config:
 class Env:
     """n_envs scenes on one CUDA device, stepped by the library."""
 
-    def __init__(self, levels: dict, n_envs: int, device: int = 0, stream=None, checked: bool = False, **cfg_kw):
+    def __init__(self, levels: dict, n_envs: int, device: int = 0, stream=None, checked: bool = False, phase_clocks: bool = False, **cfg_kw):
         import torch
         if not torch.cuda.is_available():
             raise K2DError("no CUDA device: the k2d library has no CPU fallback")
         self.torch = torch
-        self.lib = load_library(checked)
+        self.lib = load_library(checked, phase_clocks)
         self.device = torch.device("cuda", device)
         self.stream = stream if stream is not None else torch.cuda.current_stream(self.device)
         self.cfg = make_config(levels, n_envs, device=device, **cfg_kw)
@@ -268,6 +275,13 @@ class Env:
     def set_wait_limit(self, polls: int):
         """test aid: polls a scene group waits for another group's part of the same env before it gives up"""
         _check(self.lib.k2d_set_wait_limit(self._h, int(polls)), "k2d_set_wait_limit")
+
+    def phase_cycles(self) -> dict:
+        """measurement aid (phase_clocks=True builds): SM cycles the scene groups spent in each phase of a step since the last
+        call, by phase name; clears the sums"""
+        out = (C.c_uint64 * len(PHASES))()
+        _check(self.lib.k2d_phase_cycles(self._h, out, len(PHASES)), "k2d_phase_cycles")
+        return {name: int(out[i]) for i, name in enumerate(PHASES)}
 
     def enable_trace(self):
         torch = self.torch

@@ -22,7 +22,8 @@ def make_pair(levels, n_envs, broadphase=0, **cfg):
     against a reference that has no such test.  ``broadphase=1`` gives the oracle the same test, which makes its
     counters of pairs past the test comparable too."""
     checked = cfg.pop("checked", False)
-    env = k2d.Env(levels, n_envs, checked=checked, **cfg)
+    phase_clocks = cfg.pop("phase_clocks", False)
+    env = k2d.Env(levels, n_envs, checked=checked, phase_clocks=phase_clocks, **cfg)
     ocfg = {k: getattr(env.cfg, k) for k in ORACLE_CFG}
     ref = k2d_ref.RefSim(levels, n_envs, broadphase=broadphase, **ocfg)
     return env, ref

@@ -92,3 +92,34 @@ def test_a_bad_count_in_the_state_record_is_caught_and_redirected():
     env.reset()
     env.step(act)
     assert env.status()[3] == 4 * n_envs
+
+
+# ---------------------------------------------------------------- the build that counts cycles per phase of a step
+def test_phase_clock_library_builds_and_the_plain_library_refuses_the_call():
+    from paper_2410_23208_b200 import build
+    lib = k2d.load_library(phase_clocks=True)
+    assert build.LIB_PHASES.endswith("libk2d_phases.so") and lib.k2d_is_checked_build() == 0
+    assert len(k2d.PHASES) == 14
+
+
+@pytest.mark.gpu
+def test_phase_clocks_count_every_phase_and_change_no_result():
+    n_envs = 96
+    lv = scenes.make_levels("L", 48, 77, static_prob=0.1)
+    lv["pos"][:8, 1:, 0] *= 0.2                          # some crowded scenes: the memory-record path is timed too
+    env, ref = parity.make_pair(lv, n_envs, phase_clocks=True, lanes_per_scene=16, auto_reset=2, max_episode_steps=12, seed=5)
+    act = scenes.make_actions(24, n_envs, env.n_actions, 77)
+    (r, d), (rr, dr) = parity.step_both(env, ref, act, chunk=24)
+    assert np.array_equal(r.view(np.uint32), rr.view(np.uint32)) and np.array_equal(d, dr)
+    err, exact = parity.errors(env, ref)
+    assert exact, err
+    cycles = env.phase_cycles()
+    assert set(cycles) == set(k2d.PHASES)
+    for name in ("geometry", "box_test", "narrowphase", "records", "iterations", "integrate_correct", "epilogue", "load", "store"):
+        assert cycles[name] > 0, name
+    assert cycles["iterations"] > cycles["joint_prestep"]
+    assert sum(env.phase_cycles().values()) == 0             # reading clears the sums
+    # the library proper has no counters
+    plain = k2d.Env(lv, 8)
+    with pytest.raises(k2d.K2DError, match="build"):
+        plain.phase_cycles()
