@@ -1860,7 +1860,6 @@ struct Scene {
             wr[3] = __float_as_uint(ovl(OV_ACC1N)); wr[4] = __float_as_uint(ovl(OV_ACC1T));
         }
         if (nw > G + G / 2) warm_out<SC, G>(ovf, st + SC::ST_WARM, nw);
-        flush();
         g.sync();
         K2D_PHASE(PH_STORE);
         if (prm.obs && s1 == prm.n_steps) {
@@ -1922,6 +1921,9 @@ __global__ void __launch_bounds__(kBlockThreads, kMinBlocks) k2d_step_kernel(con
         if (ok) {
             const int s0 = c * prm.chunk_steps;
             scene.run(e, s0, min(prm.n_steps, s0 + prm.chunk_steps));
+            // the group's work counters go to the global ones every 64 steps or more (16-bit fields; a step adds at most
+            // one manifold per slot, 186, and a run flushes every 256 steps by itself: (63 + 256) x 186 < 65536)
+            if ((scene.c_man >> 16) >= 64u) scene.flush();
         }
         if (prm.n_chunks > 1) {
             __threadfence();      // this lane's part of the state record is visible before the count moves
@@ -1929,6 +1931,7 @@ __global__ void __launch_bounds__(kBlockThreads, kMinBlocks) k2d_step_kernel(con
             if (g.lane == 0) atomicExch(prm.chunks_done + e, (c + 1 == prm.n_chunks) ? 0u : (unsigned)(c + 1));
         }
     }
+    scene.flush();
     // the last group to leave rewinds the queue for the next launch
     if (g.lane == 0) {
         __threadfence();
