@@ -1896,12 +1896,16 @@ __global__ void __launch_bounds__(kBlockThreads, kMinBlocks) k2d_step_kernel(con
     // it); with items handed out chunk by chunk that is almost always long past, else the group waits for
     // the group that holds it, which is running.
     const Group<G> &g = scene.g;
+    // A group's first item is its own number, so that a launch does not start with every group drawing a ticket from the
+    // same word; the counter hands out the items after those.
     const unsigned items = (unsigned)prm.n_envs * (unsigned)prm.n_chunks;
+    unsigned t = (unsigned)slot;
 #pragma unroll 1
-    for (;;) {
-        unsigned t = 0u;
-        if (g.lane == 0) t = atomicAdd(prm.queue + Q_TICKET, 1u);
-        t = g.shflu(t, 0);
+    for (bool first = true;; first = false) {
+        if (!first) {
+            if (g.lane == 0) t = (unsigned)nslots + atomicAdd(prm.queue + Q_TICKET, 1u);
+            t = g.shflu(t, 0);
+        }
         if (t >= items) break;
         const int c = (int)(t / (unsigned)prm.n_envs), e = (int)(t - (unsigned)c * (unsigned)prm.n_envs);
         bool ok = true;
