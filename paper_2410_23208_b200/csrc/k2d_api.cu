@@ -289,7 +289,7 @@ static cudaError_t launch_obs(const k2d_state *s, float *dev_obs) {
     const k2d_config &c = s->cfg;
     const int epb = kObsEnvsPerBlock, grid = (c.n_envs + epb - 1) / epb;
     const int width = (c.n_polygons + c.n_circles) * 29 + c.n_joints * 2 * (11 + c.n_actions) + c.n_thrusters * 6;
-    const size_t smem = sizeof(float) * epb * ((width + 2 * SC::N + 3) / 4 * 4);
+    const size_t smem = sizeof(float) * epb * obs_image_stride(width, SC::N);
     k2d_obs_kernel<SC><<<grid, kObsThreads, smem, s->stream>>>(s->dev_env, s->dev_levels, dev_obs, c.n_envs, c.n_actions, c.n_polygons,
                                                               c.n_circles, c.n_joints, c.n_thrusters);
     return cudaGetLastError();

@@ -1969,6 +1969,12 @@ __global__ void k2d_reset_kernel(uint32_t *state, const uint32_t *levels, const 
 // stores.  Two envs share every instruction of a warp.
 static_assert(K2D_MAX_SHAPES <= 16 && 2 * K2D_MAX_JOINTS <= 12 && K2D_MAX_THRUSTERS <= 4, "observation rows: one lane of sixteen each");
 constexpr int kObsEnvsPerBlock = 2 * (kObsThreads / 32);
+// words between the images of two envs: room for the rows and the cos / sin table, a multiple of 4, and 16 past a multiple of
+// 32 so that the row stores of a warp's two envs (rows 29 or an odd number of words apart) fall into different banks
+__host__ __device__ inline int obs_image_stride(int width, int n_bodies) {
+    const int s = (width + 2 * n_bodies + 3) / 4 * 4;
+    return s + (48 - s % 32) % 32;
+}
 template <class SC>
 __global__ void __launch_bounds__(kObsThreads) k2d_obs_kernel(const uint32_t *state, const uint32_t *levels, float *obs,
                                                               int n_envs, int n_actions, int n_polygons, int n_circles,
@@ -1981,7 +1987,7 @@ __global__ void __launch_bounds__(kObsThreads) k2d_obs_kernel(const uint32_t *st
     const int n_shapes = n_polygons + n_circles;
     const int jw = 11 + n_actions;
     const int width = n_shapes * 29 + 2 * n_joints * jw + 6 * n_thrusters;
-    float *img = obs_smem + (size_t)(2 * w + half) * ((width + 2 * SC::N + 3) / 4 * 4);
+    float *img = obs_smem + (size_t)(2 * w + half) * obs_image_stride(width, SC::N);
     float *cs = img + width;                 // cos, sin of every shape's angle
     const uint32_t *st = state + (size_t)(live ? e : 0) * SC::ST_WORDS;
     const float *stf = reinterpret_cast<const float *>(st);
