@@ -2164,76 +2164,114 @@ __global__ void __launch_bounds__(kRenderThreads) k2d_render_kernel(const uint32
         s_nv[i] = nv;
     }
     __syncthreads();
-    // A warp paints 32 consecutive rows in two passes.  First every lane takes one row and goes over the shapes in index
-    // order: from the shape's faces (or its circle) it works out between which columns the row can cut the shape, and pins
-    // down the first and the last column that are inside with the exact inside test (the one that defines the image) on the
-    // few columns at either end of that span, where rounding could matter; the columns in between are inside (the shapes
-    // are convex).  That gives a short list of (first column, last column, shape) per row.  Then the warp writes the rows one
-    // after the other, lane l the columns l, l + 32, l + 64, l + 96: a pixel takes the colour of the last entry of its row's
-    // list that covers it, white if none does.
+    // A warp paints 32 consecutive rows in three passes.  First the (shape, row) pairs whose row the shape's box reaches are
+    // numbered (shape-major) and dealt out to the lanes, 32 at a time: from the shape's faces (or its circle) a lane works out
+    // between which columns the row can cut the shape, and pins down the first and the last column that are inside with the
+    // exact inside test (the one that defines the image) on the few columns at either end of that span, where rounding could
+    // matter; the columns in between are inside (the shapes are convex).  The result goes to the slot of (row, shape).  Then
+    // every lane takes one row and packs its slots into a short list of (first column, last column, colour) in shape order.
+    // Then the warp writes the rows one after the other, lane l the columns l, l + 32, l + 64, l + 96: a pixel takes the
+    // colour of the last entry of its row's list that covers it, white if none does.
+    static_assert(SC::N <= 16, "one lane of sixteen per shape");
+    constexpr uint32_t kNoSpan = 0xffffffffu;
+    __shared__ int s_first[kRenderThreads / 32][SC::N + 1];      // per warp: number of the first pair of every shape, and the total
+    __shared__ int s_row0[kRenderThreads / 32][SC::N];          // per warp: first of the warp's rows that the shape's box reaches
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    uint2 *spans = s_span + (warp * 32 + lane) * SC::N;
-    const int r = 32 * warp + lane;
-    int n_span = 0;
-    if (r < kPix) {
-        const float py = 5.75f - ((float)r + 0.5f) * 0.05f;
-#pragma unroll 1
-        for (int i = 0; i < SC::N; ++i) {
-            const int nv = s_nv[i];
-            if (nv < 0) continue;
-            const int4 rng = s_rng[i];
-            if (r < rng.z || r > rng.w) continue;
-            const float4 nx = s_nx[i], ny = s_ny[i], off = s_off[i];
-            float lo = -1.0e9f, hi = 1.0e9f;      // world x between which the row can be inside the shape
-            bool all_exact = false, none = false;
-            float t0 = 0.0f, t1 = 0.0f, t2 = 0.0f, t3 = 0.0f, dy2 = 0.0f;
-            if (nv > 0) {
-                t0 = ny.x * py; t1 = ny.y * py; t2 = ny.z * py; t3 = ny.w * py;
-                const float a[4] = { nx.x, nx.y, nx.z, nx.w }, c[4] = { t0 - off.x, t1 - off.y, t2 - off.z, t3 - off.w };
+    const int R0 = 32 * warp, R1 = min(R0 + 31, kPix - 1);
+    {
+        int cnt = 0, row0 = 0;
+        if (lane < SC::N && s_nv[lane] >= 0) {
+            const int4 rng = s_rng[lane];
+            row0 = max(rng.z, R0);
+            cnt = max(min(rng.w, R1) - row0 + 1, 0);
+        }
+        int incl = cnt;
 #pragma unroll
-                for (int k = 0; k < 4; ++k) {
-                    if (k < nv) {
-                        if (fabsf(a[k]) < 1.0e-3f) {          // a face nearly along the row: it is out, not binding, or too close to call
-                            if (c[k] > 1.0e-3f) none = true;
-                            else if (c[k] > -1.0e-3f) all_exact = true;
-                        } else {
-                            const float bound = __fdividef(-c[k], a[k]);      // an estimate is enough: the exact test decides the ends of the span
-                            if (a[k] > 0.0f) hi = fmin_cmp(hi, bound); else lo = fmax_cmp(lo, bound);
-                        }
+        for (int d = 1; d < 16; d <<= 1) { const int v = __shfl_up_sync(0xffffffffu, incl, d); if (lane >= d) incl += v; }
+        if (lane < SC::N) { s_first[warp][lane] = incl - cnt; s_row0[warp][lane] = row0; }
+        if (lane == SC::N - 1) s_first[warp][SC::N] = incl;
+    }
+    __syncwarp();
+    const int n_pairs = s_first[warp][SC::N];
+#pragma unroll 1
+    for (int base = 0; base < n_pairs; base += 32) {
+        const int item = base + lane;
+        if (item >= n_pairs) continue;
+        // the shape of the pair: the last one whose first pair is not after this one (shapes without pairs share their successor's number)
+        int i = 0;
+#pragma unroll
+        for (int step = 8; step >= 1; step >>= 1) if (i + step < SC::N && s_first[warp][i + step] <= item) i += step;
+        const int r = s_row0[warp][i] + (item - s_first[warp][i]);
+        uint2 *slot = s_span + (size_t)(r * SC::N + i);
+        const int nv = s_nv[i];
+        const int4 rng = s_rng[i];
+        const float py = 5.75f - ((float)r + 0.5f) * 0.05f;
+        const float4 nx = s_nx[i], ny = s_ny[i], off = s_off[i];
+        float lo = -1.0e9f, hi = 1.0e9f;      // world x between which the row can be inside the shape
+        bool all_exact = false, none = false;
+        float t0 = 0.0f, t1 = 0.0f, t2 = 0.0f, t3 = 0.0f, dy2 = 0.0f;
+        if (nv > 0) {
+            t0 = ny.x * py; t1 = ny.y * py; t2 = ny.z * py; t3 = ny.w * py;
+            const float a[4] = { nx.x, nx.y, nx.z, nx.w }, c[4] = { t0 - off.x, t1 - off.y, t2 - off.z, t3 - off.w };
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                if (k < nv) {
+                    if (fabsf(a[k]) < 1.0e-3f) {          // a face nearly along the row: it is out, not binding, or too close to call
+                        if (c[k] > 1.0e-3f) none = true;
+                        else if (c[k] > -1.0e-3f) all_exact = true;
+                    } else {
+                        const float bound = __fdividef(-c[k], a[k]);      // an estimate is enough: the exact test decides the ends of the span
+                        if (a[k] > 0.0f) hi = fmin_cmp(hi, bound); else lo = fmax_cmp(lo, bound);
                     }
                 }
-            } else {
-                const float dy = py - ny.x;
-                dy2 = dy * dy;
-                const float h2 = off.x - dy2;
-                if (h2 < -1.0e-4f) none = true;
-                else { const float h = sqrtf(fmax_cmp(h2, 0.0f)); lo = nx.x - h; hi = nx.x + h; }
             }
-            if (none || hi < lo - 0.2f) continue;
-            // columns: pixel c has its centre at x = -3.125 + (c + 0.5) * 0.05
-            const float clo = fmax_cmp((lo + 3.125f) * 20.0f - 0.5f, -4.0f), chi = fmin_cmp((hi + 3.125f) * 20.0f - 0.5f, 130.0f);
-            const int c_first = max(max((int)floorf(clo) - 2, rng.x), 0), c_last = min(min((int)ceilf(chi) + 2, rng.y), kPix - 1);
-            // columns sure_first .. sure_last are inside without a test (none if a face is too close to call)
-            const int sure_first = all_exact ? c_last + 1 : max((int)ceilf(clo) + 2, c_first), sure_last = all_exact ? c_first - 1 : min((int)floorf(chi) - 2, c_last);
-            auto exact = [&](int c) -> bool {
-                const float px = -3.125f + ((float)c + 0.5f) * 0.05f;
-                if (nv > 0)
-                    return !(__fmaf_rn(nx.x, px, t0) - off.x > 0.0f) && !(__fmaf_rn(nx.y, px, t1) - off.y > 0.0f) &&
-                           !(__fmaf_rn(nx.z, px, t2) - off.z > 0.0f) && (nv < 4 || !(__fmaf_rn(nx.w, px, t3) - off.w > 0.0f));
-                const float dx = px - nx.x;
-                return __fmaf_rn(dx, dx, dy2) <= off.x;
-            };
-            const bool sure = sure_first <= sure_last;
-            int cf = sure ? sure_first : c_last + 1, cl = sure ? sure_last : c_first - 1;
-            // the first inside column: the lowest one below the sure span (or anywhere, if there is no sure span) that passes the test
-            const int left_end = sure ? sure_first - 1 : c_last;
+        } else {
+            const float dy = py - ny.x;
+            dy2 = dy * dy;
+            const float h2 = off.x - dy2;
+            if (h2 < -1.0e-4f) none = true;
+            else { const float h = sqrtf(fmax_cmp(h2, 0.0f)); lo = nx.x - h; hi = nx.x + h; }
+        }
+        if (none || hi < lo - 0.2f) { slot->x = kNoSpan; continue; }
+        // columns: pixel c has its centre at x = -3.125 + (c + 0.5) * 0.05
+        const float clo = fmax_cmp((lo + 3.125f) * 20.0f - 0.5f, -4.0f), chi = fmin_cmp((hi + 3.125f) * 20.0f - 0.5f, 130.0f);
+        const int c_first = max(max((int)floorf(clo) - 2, rng.x), 0), c_last = min(min((int)ceilf(chi) + 2, rng.y), kPix - 1);
+        // columns sure_first .. sure_last are inside without a test (none if a face is too close to call)
+        const int sure_first = all_exact ? c_last + 1 : max((int)ceilf(clo) + 2, c_first), sure_last = all_exact ? c_first - 1 : min((int)floorf(chi) - 2, c_last);
+        auto exact = [&](int c) -> bool {
+            const float px = -3.125f + ((float)c + 0.5f) * 0.05f;
+            if (nv > 0)
+                return !(__fmaf_rn(nx.x, px, t0) - off.x > 0.0f) && !(__fmaf_rn(nx.y, px, t1) - off.y > 0.0f) &&
+                       !(__fmaf_rn(nx.z, px, t2) - off.z > 0.0f) && (nv < 4 || !(__fmaf_rn(nx.w, px, t3) - off.w > 0.0f));
+            const float dx = px - nx.x;
+            return __fmaf_rn(dx, dx, dy2) <= off.x;
+        };
+        const bool sure = sure_first <= sure_last;
+        int cf = sure ? sure_first : c_last + 1, cl = sure ? sure_last : c_first - 1;
+        // the first inside column: the lowest one below the sure span (or anywhere, if there is no sure span) that passes the test
+        const int left_end = sure ? sure_first - 1 : c_last;
 #pragma unroll 1
-            for (int c = c_first; c <= left_end; ++c) if (exact(c)) { cf = c; break; }
-            const int right_end = sure ? sure_last + 1 : max(cf, c_first);
+        for (int c = c_first; c <= left_end; ++c) if (exact(c)) { cf = c; break; }
+        const int right_end = sure ? sure_last + 1 : max(cf, c_first);
 #pragma unroll 1
-            for (int c = c_last; c >= right_end; --c) if (exact(c)) { cl = c; break; }
-            if (!sure && cl < cf) cl = cf;      // a single column found from the left
-            if (cf <= cl && cf <= c_last) spans[n_span++] = make_uint2((uint32_t)cf | ((uint32_t)(cl - cf) << 8), s_col[i]);
+        for (int c = c_last; c >= right_end; --c) if (exact(c)) { cl = c; break; }
+        if (!sure && cl < cf) cl = cf;      // a single column found from the left
+        if (cf <= cl && cf <= c_last) *slot = make_uint2((uint32_t)cf | ((uint32_t)(cl - cf) << 8), s_col[i]);
+        else slot->x = kNoSpan;
+    }
+    __syncwarp();
+    // the slots of a row, packed in place (the list is never ahead of the slot being read)
+    uint2 *spans = s_span + (warp * 32 + lane) * SC::N;
+    const int r = R0 + lane;
+    int n_span = 0;
+    if (r < kPix) {
+#pragma unroll 1
+        for (int i = 0; i < SC::N; ++i) {
+            if (s_nv[i] < 0) continue;
+            const int4 rng = s_rng[i];
+            if (r < rng.z || r > rng.w) continue;
+            const uint2 w = spans[i];
+            if (w.x != kNoSpan) spans[n_span++] = w;
         }
     }
     s_nspan[warp * 32 + lane] = n_span;
