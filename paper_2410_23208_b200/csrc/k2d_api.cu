@@ -17,7 +17,9 @@ using ClassM = SizeClass<6, 3, 2, 2>;
 using ClassL = SizeClass<12, 4, 6, 2>;
 
 constexpr int kMaxSlots = 8192;      // resident scene groups a launch may use (bounds the overflow scratch)
-constexpr size_t kCtrlBytes = 256;   // control block at the start of the state buffer: 8 x uint64 counters, then the work queue words
+constexpr size_t kCtrlBytes = 4096;  // control block at the start of the state buffer: 8 x uint64 counters, the work queue words at
+                                     // kQueueOffset, the counting sort's words (2 x 256 + 1) at kSortOffset
+constexpr size_t kSortOffset = 1024;
 constexpr size_t kQueueOffset = 128;
 #ifndef K2D_CHUNK_STEPS
 #define K2D_CHUNK_STEPS 8
@@ -94,7 +96,7 @@ struct k2d_state {
     cudaStream_t stream;
     unsigned char *dev_base;
     unsigned long long *dev_counters;
-    unsigned int *dev_queue, *dev_chunks;
+    unsigned int *dev_queue, *dev_chunks, *dev_sort;
     int *dev_ids;
     uint32_t *dev_env, *dev_scratch, *dev_levels;
     float *dev_trace;
@@ -202,6 +204,7 @@ static int pack_level(const k2d_config *cfg, const ClassInfo &ci, const k2d_leve
     // joint sharing a movable shape (so lanes can run a level's joints at once and keep the joint order)
     std::vector<int> body_level(ci.N, 0);
     std::vector<std::pair<int, int>> joined;
+    int joint_levels = 0;
     for (int j = 0; j < nJ; ++j) {
         uint32_t *jw = w + ci.LV_JOINT + kJointLevelWords * j;
         if (!L->joint_active[j]) continue;
@@ -221,6 +224,7 @@ static int pack_level(const k2d_config *cfg, const ClassInfo &ci, const k2d_leve
             if (!is_static[b]) lvl = std::max(lvl, body_level[b] + 1);
             if (!is_static[a]) body_level[a] = lvl;
             if (!is_static[b]) body_level[b] = lvl;
+            joint_levels = std::max(joint_levels, lvl);
         }
         jw[0] = (uint32_t)a | ((uint32_t)b << 8) | ((uint32_t)L->motor_binding[j] << 16) | ((on ? 1u : 0u) << 24) | ((uint32_t)lvl << 25) | (1u << 28) |
                 ((is_static[a] ? 0u : 1u) << 29) | ((is_static[b] ? 0u : 1u) << 30) |
@@ -229,6 +233,7 @@ static int pack_level(const k2d_config *cfg, const ClassInfo &ci, const k2d_leve
         jw[10] = L->joint_fixed[j] ? 1u : (L->joint_limited[j] ? 2u : 0u);
         joined.emplace_back(a, b);
     }
+    w[ci.LV_GB] |= (uint32_t)std::min(joint_levels, 7) << 24;      // what the launch's env order sorts by (with the touching pairs)
     std::fill(body_level.begin(), body_level.end(), 0);
     for (int t = 0; t < nT; ++t) {
         uint32_t *tw = w + ci.LV_THR + 8 * t;
@@ -312,6 +317,7 @@ static StepParams step_params(const k2d_state *s, const float *dev_actions, int 
     prm.n_envs = c.n_envs; prm.n_steps = n_steps; prm.n_actions = c.n_actions; prm.n_levels = c.n_levels;
     prm.obs = nullptr; prm.n_polygons = c.n_polygons; prm.n_circles = c.n_circles; prm.n_joints = c.n_joints; prm.n_thrusters = c.n_thrusters;
     prm.discrete = discrete; prm.dense_kappa = c.dense_kappa; prm.frame_skip = c.frame_skip;
+    prm.order = nullptr;
     prm.chunk_steps = n_steps; prm.n_chunks = 1; prm.wait_limit = s->wait_limit; prm.n_slots = scratch == s->dev_scratch ? s->slots : K2D_STATIC_SCRATCH_MAX_ENVS;
     {
         const int n_slots = c.n_polygons * (c.n_polygons - 1) + c.n_polygons * c.n_circles + c.n_circles * (c.n_circles - 1) / 2;
@@ -329,6 +335,23 @@ static StepParams step_params(const k2d_state *s, const float *dev_actions, int 
     prm.rest_thr = c.restitution_threshold; prm.face_tol = c.face_tol; prm.joint_alpha = c.joint_alpha; prm.joint_beta = c.joint_beta; prm.joint_gamma = c.joint_gamma;
     prm.motor_rho = c.motor_rho; prm.aabb_margin = c.aabb_margin; prm.seed = c.seed; prm.env_offset = c.env_offset;
     return prm;
+}
+
+// Launches of at least kOrderMinSteps steps with two or more scenes per warp and more envs than the device holds scene groups
+// first sort the envs by what their steps cost (see k2d_order_count_kernel); the order lives in the words that k2d_reset uses
+// for the level ids, free between resets.
+constexpr int kOrderMinSteps = 8;
+template <class SC>
+static cudaError_t launch_order(const k2d_state *s) {
+    const int n = s->cfg.n_envs, grid = (n + kOrderThreads - 1) / kOrderThreads;
+    k2d_order_count_kernel<SC><<<grid, kOrderThreads, 0, s->stream>>>(s->dev_env, s->dev_levels, s->dev_sort, n, s->cfg.n_levels);
+    k2d_order_place_kernel<SC><<<grid, kOrderThreads, 0, s->stream>>>(s->dev_env, s->dev_levels, s->dev_sort, s->dev_ids, n, s->cfg.n_levels);
+    return cudaGetLastError();
+}
+static cudaError_t order_envs(const k2d_state *s, StepParams &prm) {
+    if (s->G >= 32 || prm.n_steps < kOrderMinSteps || s->cfg.n_envs <= s->groups) return cudaSuccess;
+    prm.order = s->dev_ids;
+    return s->ci.id == 0 ? launch_order<ClassS>(s) : s->ci.id == 1 ? launch_order<ClassM>(s) : launch_order<ClassL>(s);
 }
 
 #define K2D_DISPATCH(FN, s, ...)                                                                      \
@@ -424,6 +447,7 @@ int k2d_create(const k2d_config *cfg, void *dev_state_buf, void *dev_level_pool_
     s->dev_base = (unsigned char *)dev_state_buf;
     s->dev_counters = (unsigned long long *)s->dev_base;
     s->dev_queue = (unsigned int *)(s->dev_base + kQueueOffset);
+    s->dev_sort = (unsigned int *)(s->dev_base + kSortOffset);
     s->dev_chunks = (unsigned int *)(s->dev_base + bl.chunks_off);
     s->dev_ids = (int *)(s->dev_base + bl.ids_off);
     s->dev_env = (uint32_t *)(s->dev_base + bl.env_off);
@@ -471,7 +495,8 @@ int k2d_step(k2d_state *s, const float *dev_actions, int32_t n_steps, float *dev
     if (n_steps < 1 || n_steps > s->cfg.max_fused_steps) return K2D_ERR_STEPS;
     if (((uintptr_t)dev_actions & 3) || ((uintptr_t)dev_reward & 3)) return K2D_ERR_ALIGN;
     CUDA_OK(cudaSetDevice(s->cfg.device));
-    const StepParams prm = step_params(s, dev_actions, n_steps, dev_reward, dev_done, s->dev_scratch);
+    StepParams prm = step_params(s, dev_actions, n_steps, dev_reward, dev_done, s->dev_scratch);
+    CUDA_OK(order_envs(s, prm));
     CUDA_OK(K2D_DISPATCH(launch_step, s, s, prm));
     return K2D_OK;
 }
@@ -484,6 +509,7 @@ int k2d_step_obs(k2d_state *s, const float *dev_actions, int32_t n_steps, float 
     StepParams prm = step_params(s, dev_actions, n_steps, dev_reward, dev_done, s->dev_scratch);
     const bool fused = K2D_DISPATCH(obs_fits, s, s);
     if (fused) prm.obs = dev_obs;
+    CUDA_OK(order_envs(s, prm));
     CUDA_OK(K2D_DISPATCH(launch_step, s, s, prm));
     if (!fused) return k2d_obs(s, dev_obs);       // scenes whose observation is wider than the region's spare part: a second launch
     return K2D_OK;
@@ -697,7 +723,8 @@ int k2d_step_discrete(k2d_state *s, const int32_t *dev_actions, int32_t n_steps,
     if (n_steps < 1 || n_steps > s->cfg.max_fused_steps) return K2D_ERR_STEPS;
     if (((uintptr_t)dev_actions & 3) || ((uintptr_t)dev_reward & 3)) return K2D_ERR_ALIGN;
     CUDA_OK(cudaSetDevice(s->cfg.device));
-    const StepParams prm = step_params(s, reinterpret_cast<const float *>(dev_actions), n_steps, dev_reward, dev_done, s->dev_scratch, 1);
+    StepParams prm = step_params(s, reinterpret_cast<const float *>(dev_actions), n_steps, dev_reward, dev_done, s->dev_scratch, 1);
+    CUDA_OK(order_envs(s, prm));
     CUDA_OK(K2D_DISPATCH(launch_step, s, s, prm));
     return K2D_OK;
 }

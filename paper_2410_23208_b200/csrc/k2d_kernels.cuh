@@ -143,6 +143,7 @@ struct StepParams {
     unsigned long long *counters;
     unsigned int *queue;       // work queue words: next ticket, groups that have left, error flag
     unsigned int *chunks_done; // per env: chunks of this launch already stepped (0 again when the launch is over)
+    const int *order;          // the envs in the order the launch hands them out (null: by index)
     uint32_t *scratch;
     float *trace;
     float *obs;               // k2d_step_obs: the symbolic observation after the call's last step, [n_envs][obs_floats]; else null
@@ -1869,6 +1870,62 @@ struct Scene {
     }
 };
 
+// ---------------------------------------------------------------- the order in which a launch hands out the envs
+// The two scenes of a warp run in lockstep, so each pays for the longer of the two in every phase.  Handing out the envs
+// sorted by what their steps cost puts like next to like: the key is the number of joint levels of the env's level and the
+// number of pairs that were touching after its last step.  A counting sort in two launches: the first counts the keys and
+// its last block turns the counts into first positions; the second writes every env to a position of its key.  The order
+// inside a key is whatever the atomics give; no result depends on it.  sort[0 .. 255] counts (zero between launches),
+// sort[256 .. 511] positions, sort[512] blocks that have counted.
+constexpr int kOrderThreads = 256, kOrderKeys = 256;
+template <class SC>
+__device__ __forceinline__ int order_key(const uint32_t *state, const uint32_t *levels, int e, int n_levels) {
+    const uint32_t *st = state + (size_t)e * SC::ST_WORDS;
+    const unsigned level = min(__ldcg(st + SC::ST_META + META_LEVEL), (unsigned)(n_levels - 1));
+    const unsigned touching = min(__ldcg(st + SC::ST_META + META_NWARM), 31u);
+    const unsigned joint_levels = (__ldg(levels + (size_t)level * SC::LV_WORDS + SC::LV_GB) >> 24) & 7u;
+    return kOrderKeys - 1 - (int)(joint_levels * 32u + touching);     // costly envs first: the cheap ones fill the end of the launch
+}
+template <class SC>
+__global__ void __launch_bounds__(kOrderThreads) k2d_order_count_kernel(const uint32_t *state, const uint32_t *levels, unsigned int *sort,
+                                                                        int n_envs, int n_levels) {
+    __shared__ unsigned int s_cnt[kOrderKeys];
+    __shared__ bool s_last;
+    s_cnt[threadIdx.x] = 0u;
+    __syncthreads();
+    const int e = blockIdx.x * kOrderThreads + threadIdx.x;
+    if (e < n_envs) atomicAdd(&s_cnt[order_key<SC>(state, levels, e, n_levels)], 1u);
+    __syncthreads();
+    if (s_cnt[threadIdx.x]) atomicAdd(sort + threadIdx.x, s_cnt[threadIdx.x]);
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) s_last = atomicAdd(sort + 2 * kOrderKeys, 1u) == gridDim.x - 1u;
+    __syncthreads();
+    if (!s_last) return;
+    // the last block to arrive: counts -> first positions (exclusive sums), counts back to zero for the next launch
+    __threadfence();
+    const unsigned int mine = __ldcg(sort + threadIdx.x);
+    s_cnt[threadIdx.x] = mine;
+    __syncthreads();
+    for (int d = 1; d < kOrderKeys; d <<= 1) {
+        const unsigned int v = threadIdx.x >= d ? s_cnt[threadIdx.x - d] : 0u;
+        __syncthreads();
+        s_cnt[threadIdx.x] += v;
+        __syncthreads();
+    }
+    sort[kOrderKeys + threadIdx.x] = s_cnt[threadIdx.x] - mine;
+    sort[threadIdx.x] = 0u;
+    if (threadIdx.x == 0) sort[2 * kOrderKeys] = 0u;
+}
+template <class SC>
+__global__ void __launch_bounds__(kOrderThreads) k2d_order_place_kernel(const uint32_t *state, const uint32_t *levels, unsigned int *sort,
+                                                                        int *order, int n_envs, int n_levels) {
+    const int e = blockIdx.x * kOrderThreads + threadIdx.x;
+    if (e >= n_envs) return;
+    const unsigned int pos = atomicAdd(sort + kOrderKeys + order_key<SC>(state, levels, e, n_levels), 1u);
+    if (pos < (unsigned)n_envs) order[pos] = e;
+}
+
 template <class SC>
 __device__ __forceinline__ uint16_t pair_code(int p) {
     int a, b;
@@ -1898,8 +1955,11 @@ __global__ void __launch_bounds__(kBlockThreads, kMinBlocks) k2d_step_kernel(con
     const Group<G> &g = scene.g;
     // A group's first item is its own number, so that a launch does not start with every group drawing a ticket from the
     // same word; the counter hands out the items after those.
+    // First items go round the blocks warp by warp (the scenes of a warp next to one another in the launch's order, the
+    // warps of a block far apart), so that every SM starts with a mix of cheap and costly envs.
     const unsigned items = (unsigned)prm.n_envs * (unsigned)prm.n_chunks;
-    unsigned t = (unsigned)slot;
+    constexpr int GPW = 32 / G;
+    unsigned t = (unsigned)(GPW * ((gib / GPW) * (int)gridDim.x + (int)blockIdx.x) + gib % GPW);
 #pragma unroll 1
     for (bool first = true;; first = false) {
         if (!first) {
@@ -1907,7 +1967,8 @@ __global__ void __launch_bounds__(kBlockThreads, kMinBlocks) k2d_step_kernel(con
             t = g.shflu(t, 0);
         }
         if (t >= items) break;
-        const int c = (int)(t / (unsigned)prm.n_envs), e = (int)(t - (unsigned)c * (unsigned)prm.n_envs);
+        const int c = (int)(t / (unsigned)prm.n_envs), idx = (int)(t - (unsigned)c * (unsigned)prm.n_envs);
+        const int e = prm.order ? ck_idx<CK_COUNT>(__ldg(prm.order + idx), prm.n_envs) : idx;
         bool ok = true;
         if (c > 0) {
             if (g.lane == 0) {

@@ -79,9 +79,9 @@ def test_a_bad_count_in_the_state_record_is_caught_and_redirected():
     act = torch.zeros((4, n_envs, env.n_actions), device="cuda")
     env.step(act)
     env.status()
-    # state buffer: 256-byte control block, then level ids and chunk counters (4 bytes per env each, 256-byte aligned), then
+    # state buffer: 4096-byte control block, then level ids and chunk counters (4 bytes per env each, 256-byte aligned), then
     # the env records; an S record has its meta words after 6 x 7 body words and 3 joint words, the count is meta word 4
-    offset = 768 + 4 * (6 * 7 + 3 + 4)
+    offset = 4096 + 512 + 4 * (6 * 7 + 3 + 4)
     assert int(env.state_buf[offset:offset + 4].view(torch.int32)[0]) <= 21
     env.state_buf[offset:offset + 4].view(torch.int32)[0] = 1000
     torch.cuda.synchronize()

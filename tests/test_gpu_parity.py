@@ -504,8 +504,10 @@ def test_a_wait_that_runs_out_ends_the_launch_and_is_reported():
     with pytest.raises(k2d.K2DError, match="waiting"):
         env.status()
     after = env.get_state()
-    # the last envs (beyond the device's scene groups: 5920 on 148 SMs) were never stepped, the first ones by 8 steps only
-    assert np.array_equal(before["pos"][-200:], after["pos"][-200:]) and np.all(after["step_count"][-200:] == 0)
+    # the envs beyond the device's scene groups (5920 on 148 SMs; which envs those are is the launch's business) were never
+    # stepped, the others by 8 steps only
+    idle = after["step_count"] == 0
+    assert idle.sum() >= 200 and np.array_equal(before["pos"][idle], after["pos"][idle])
     assert after["step_count"].max() <= 8
     env.reset()
     assert env.status().sum() == 0
