@@ -97,6 +97,7 @@ struct k2d_state {
     unsigned char *dev_base;
     unsigned long long *dev_counters;
     unsigned int *dev_queue, *dev_chunks, *dev_sort;
+    int order_age;       // launches since the envs were last sorted for the work queue (0: the order is not valid)
     int *dev_ids;
     uint32_t *dev_env, *dev_scratch, *dev_levels;
     float *dev_trace;
@@ -340,7 +341,7 @@ static StepParams step_params(const k2d_state *s, const float *dev_actions, int 
 // Launches of at least kOrderMinSteps steps with two or more scenes per warp and more envs than the device holds scene groups
 // first sort the envs by what their steps cost (see k2d_order_count_kernel); the order lives in the words that k2d_reset uses
 // for the level ids, free between resets.
-constexpr int kOrderMinSteps = 8;
+constexpr int kOrderMinSteps = 8, kOrderShortLaunches = 16;
 template <class SC>
 static cudaError_t launch_order(const k2d_state *s) {
     const int n = s->cfg.n_envs, grid = (n + kOrderThreads - 1) / kOrderThreads;
@@ -348,9 +349,13 @@ static cudaError_t launch_order(const k2d_state *s) {
     k2d_order_place_kernel<SC><<<grid, kOrderThreads, 0, s->stream>>>(s->dev_env, s->dev_levels, s->dev_sort, s->dev_ids, n, s->cfg.n_levels);
     return cudaGetLastError();
 }
-static cudaError_t order_envs(const k2d_state *s, StepParams &prm) {
-    if (s->G >= 32 || prm.n_steps < kOrderMinSteps || s->cfg.n_envs <= s->groups) return cudaSuccess;
+static cudaError_t order_envs(k2d_state *s, StepParams &prm) {
+    if (s->G >= 32 || s->cfg.n_envs <= s->groups) return cudaSuccess;
     prm.order = s->dev_ids;
+    // a short launch reuses the order of an earlier one (what an env's step costs changes slowly) and sorts again every
+    // kOrderShortLaunches launches; k2d_reset, which uses the same words, makes the next launch sort
+    if (prm.n_steps < kOrderMinSteps && s->order_age > 0 && s->order_age < kOrderShortLaunches) { ++s->order_age; return cudaSuccess; }
+    s->order_age = 1;
     return s->ci.id == 0 ? launch_order<ClassS>(s) : s->ci.id == 1 ? launch_order<ClassM>(s) : launch_order<ClassL>(s);
 }
 
@@ -476,6 +481,7 @@ int k2d_reset(k2d_state *s, const int32_t *host_level_ids) {
         for (int e = 0; e < E; ++e) if (host_level_ids[e] < 0 || host_level_ids[e] >= s->cfg.n_levels) return K2D_ERR_ARG;
     CUDA_OK(cudaSetDevice(s->cfg.device));
     CUDA_OK(cudaMemsetAsync(s->dev_base, 0, kCtrlBytes, s->stream));
+    s->order_age = 0;
 #ifdef K2D_CHECKED
     { const unsigned int zero = 0u; CUDA_OK(cudaMemcpyToSymbolAsync(k2d_check_bits, &zero, sizeof(zero), 0, cudaMemcpyHostToDevice, s->stream)); }
 #endif

@@ -136,3 +136,23 @@ def test_workload_4_large_scenes_131072_envs_fused_steps_and_observation():
     assert np.array_equal(got.view(np.uint32), want.view(np.uint32))
     # the horizon of 256 is not reached in 32 steps; resets here come from touches
     assert ref.counters[1] > 0
+
+
+def test_short_launches_through_the_work_queue_reuse_and_renew_the_order_of_the_envs():
+    # more envs than the device holds scene groups, one or two steps per launch: the launch hands the envs out in an order
+    # sorted by cost that it keeps for 16 launches; a reset with level ids (which uses the same words) makes the next launch
+    # sort again.  Whatever the order, every env is stepped once per step.
+    n_envs = 6400
+    lv = scenes.make_levels("L", 128, 91, static_prob=0.1)
+    env, ref = parity.make_pair(lv, n_envs, auto_reset=2, max_episode_steps=12, seed=91, max_fused_steps=8, lanes_per_scene=16)
+    act = scenes.make_actions(40, n_envs, env.n_actions, 91)
+    n_threads = os.cpu_count() or 1
+    (r, d), (rr, dr) = parity.step_both(env, ref, act[:20], chunk=1, n_threads=n_threads)      # 20 launches of one step
+    assert np.array_equal(r, rr) and np.array_equal(d, dr)
+    ids = (np.arange(n_envs)[::-1] % 128).astype(np.int32)
+    env.reset(ids); ref.reset(ids)
+    (r, d), (rr, dr) = parity.step_both(env, ref, act[20:], chunk=2, n_threads=n_threads)      # 10 launches of two steps
+    assert np.array_equal(r, rr) and np.array_equal(d, dr) and d.sum() > 0
+    err, exact = parity.errors(env, ref)
+    assert exact, err
+    assert env.status()[3] == 20 * n_envs and parity.counters_match(env, ref)      # both count from the reset
