@@ -265,6 +265,7 @@ def run_gpu(args) -> dict:
     barrier()
     counts0 = env.status().copy()
 
+    launches_per_step = env.step_launches(FUSED) + 1      # the step kernel (with the two launches that sort the envs for its work queue, when it has one) and the observation kernel
     # ---- device-resident timing: events around each step (k2d_step, then k2d_obs); L2 flushed in between, untimed
     ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(K)]
     barrier()
@@ -414,7 +415,7 @@ def run_gpu(args) -> dict:
         "dtype": "f32", "data": "synthetic",
         "config": {"workload": f"{w['size']} scenes, {n_envs} envs per GPU, {FUSED} fused engine steps + 1 observation per bench step "
                                f"(config {args.workload}: pool of {w['n_levels']} levels, horizon {w['max_episode_steps']})",
-                   "lanes_per_scene": env.cfg.lanes_per_scene or (32 if n_envs < (48 if w["size"] == "L" else 24) * torch.cuda.get_device_properties(dev).multi_processor_count else 16), "fused_steps": FUSED,
+                   "lanes_per_scene": env.lanes_per_scene, "resident_scene_groups": env.resident_groups, "kernel_launches_per_bench_step": launches_per_step, "fused_steps": FUSED,
                    "observation": "pixels 125x125 RGBA (k2d_render)" if args.pixels else "symbolic entity rows (k2d_obs)",
                    "solver_batch": args.solver_batch,
                    "l2": "flushed between timed iterations (256 MiB write, untimed); K distinct action buffers"},
@@ -429,7 +430,7 @@ def run_gpu(args) -> dict:
         "modes": {k: {"ms_per_call": v, "value": world * n_envs / (v * 1e-3), "unit": UNIT,
                       "what": ("k2d_step(1 step) + k2d_obs: two launches per call" if k == "one_step_then_obs"
                                else "k2d_step_obs(1 step): one launch per call")} for k, v in modes.items()},
-        "gpu_launches": 2 * K,
+        "gpu_launches": launches_per_step * K,
         "roofline": {"bound": "alu", "kernel": "k2d_step_kernel", "achieved": achieved_tflops, "peak": peak, "unit": "TFLOP/s",
                      "frac": achieved_tflops / peak, "traffic": None if traffic_per_env is None else traffic_per_env * n_envs,
                      "peak_source": "derived: 148 SMs x 128 lanes x 2 x 1965 MHz",

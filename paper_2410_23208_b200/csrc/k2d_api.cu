@@ -349,12 +349,16 @@ static cudaError_t launch_order(const k2d_state *s) {
     k2d_order_place_kernel<SC><<<grid, kOrderThreads, 0, s->stream>>>(s->dev_env, s->dev_levels, s->dev_sort, s->dev_ids, n, s->cfg.n_levels);
     return cudaGetLastError();
 }
+static bool uses_order(const k2d_state *s) { return s->G < 32 && s->cfg.n_envs > s->groups; }
+// a short launch reuses the order of an earlier one (what an env's step costs changes slowly) and sorts again every
+// kOrderShortLaunches launches; k2d_reset, which uses the same words, makes the next launch sort
+static bool reuses_order(const k2d_state *s, int n_steps) {
+    return n_steps < kOrderMinSteps && s->order_age > 0 && s->order_age < kOrderShortLaunches;
+}
 static cudaError_t order_envs(k2d_state *s, StepParams &prm) {
-    if (s->G >= 32 || s->cfg.n_envs <= s->groups) return cudaSuccess;
+    if (!uses_order(s)) return cudaSuccess;
     prm.order = s->dev_ids;
-    // a short launch reuses the order of an earlier one (what an env's step costs changes slowly) and sorts again every
-    // kOrderShortLaunches launches; k2d_reset, which uses the same words, makes the next launch sort
-    if (prm.n_steps < kOrderMinSteps && s->order_age > 0 && s->order_age < kOrderShortLaunches) { ++s->order_age; return cudaSuccess; }
+    if (reuses_order(s, prm.n_steps)) { ++s->order_age; return cudaSuccess; }
     s->order_age = 1;
     return s->ci.id == 0 ? launch_order<ClassS>(s) : s->ci.id == 1 ? launch_order<ClassM>(s) : launch_order<ClassL>(s);
 }
@@ -683,6 +687,13 @@ int k2d_is_checked_build(void) {
 #else
     return 0;
 #endif
+}
+
+int k2d_resident_groups(const k2d_state *s) { return s ? s->groups : 0; }
+int k2d_lanes_per_scene(const k2d_state *s) { return s ? s->G : 0; }
+int k2d_step_launches(const k2d_state *s, int32_t n_steps) {
+    if (!s) return 0;
+    return (uses_order(s) && !reuses_order(s, n_steps)) ? 3 : 1;
 }
 
 int k2d_phase_cycles(k2d_state *s, uint64_t *host_cycles, int32_t n) {

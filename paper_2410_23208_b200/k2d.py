@@ -20,7 +20,7 @@ EXPORTS = (
     "k2d_default_config", "k2d_state_bytes", "k2d_state_bytes_no_scratch", "k2d_level_pool_bytes", "k2d_create", "k2d_reset", "k2d_step",
     "k2d_step_discrete", "k2d_step_static_scratch", "k2d_step_obs", "k2d_obs", "k2d_render",
     "k2d_obs_floats", "k2d_canonical_words", "k2d_get_state", "k2d_set_state", "k2d_status", "k2d_level_info",
-    "k2d_set_trace", "k2d_trace_slots", "k2d_is_checked_build", "k2d_phase_cycles", "k2d_set_wait_limit", "k2d_eval_sincos_tanh", "k2d_measure_fp32_peak", "k2d_error_string", "k2d_destroy",
+    "k2d_set_trace", "k2d_trace_slots", "k2d_is_checked_build", "k2d_phase_cycles", "k2d_resident_groups", "k2d_lanes_per_scene", "k2d_step_launches", "k2d_set_wait_limit", "k2d_eval_sincos_tanh", "k2d_measure_fp32_peak", "k2d_error_string", "k2d_destroy",
 )
 
 
@@ -91,6 +91,9 @@ def load_library(checked: bool = False, phase_clocks: bool = False):
         lib.k2d_trace_slots.argtypes = [vp]
         lib.k2d_set_wait_limit.argtypes = [vp, C.c_uint32]
         lib.k2d_phase_cycles.argtypes = [vp, vp, i32]
+        lib.k2d_resident_groups.argtypes = [vp]
+        lib.k2d_lanes_per_scene.argtypes = [vp]
+        lib.k2d_step_launches.argtypes = [vp, i32]
         lib.k2d_eval_sincos_tanh.argtypes = [vp, i32, vp, vp, vp, vp]
         lib.k2d_measure_fp32_peak.argtypes = [i32, vp, C.c_size_t, vp]
         lib.k2d_error_string.argtypes = [C.c_int]
@@ -275,6 +278,19 @@ class Env:
     def set_wait_limit(self, polls: int):
         """test aid: polls a scene group waits for another group's part of the same env before it gives up"""
         _check(self.lib.k2d_set_wait_limit(self._h, int(polls)), "k2d_set_wait_limit")
+
+    @property
+    def resident_groups(self) -> int:
+        """scenes the device steps at once for this handle"""
+        return int(self.lib.k2d_resident_groups(self._h))
+
+    @property
+    def lanes_per_scene(self) -> int:
+        return int(self.lib.k2d_lanes_per_scene(self._h))
+
+    def step_launches(self, n_steps: int) -> int:
+        """kernel launches the next step call of n_steps steps makes (the step kernel, and the two that sort the envs when it does)"""
+        return int(self.lib.k2d_step_launches(self._h, int(n_steps)))
 
     def phase_cycles(self) -> dict:
         """measurement aid (phase_clocks=True builds): SM cycles the scene groups spent in each phase of a step since the last
