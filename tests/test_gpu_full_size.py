@@ -156,3 +156,30 @@ def test_short_launches_through_the_work_queue_reuse_and_renew_the_order_of_the_
     err, exact = parity.errors(env, ref)
     assert exact, err
     assert env.status()[3] == 20 * n_envs and parity.counters_match(env, ref)      # both count from the reset
+
+
+def test_discrete_actions_and_the_fused_observation_through_the_sorted_work_queue():
+    # the two other launching entry points with more envs than scene groups and launches long enough to sort the envs:
+    # k2d_step_discrete (multi-discrete codes) and k2d_step_obs (observation written by the stepping groups)
+    import torch
+    from oracle import k2d_ref
+    from paper_2410_23208_b200 import k2d
+    n_envs = 6400
+    lv = scenes.make_levels("L", 128, 93, static_prob=0.1)
+    env = k2d.Env(lv, n_envs, auto_reset=2, max_episode_steps=11, seed=93, max_fused_steps=16, lanes_per_scene=16)
+    ref = k2d_ref.RefSim(lv, n_envs, auto_reset=2, max_episode_steps=11, seed=93, broadphase=0, discrete_actions=1)
+    codes = np.random.default_rng(93).integers(0, 3, (32, n_envs, env.n_actions)).astype(np.int32)
+    (r, d), (rr, dr) = parity.step_both(env, ref, codes, chunk=16, n_threads=os.cpu_count() or 1)
+    assert np.array_equal(r, rr) and np.array_equal(d, dr) and d.sum() > 0
+    err, exact = parity.errors(env, ref)
+    assert exact, err
+
+    env, ref = parity.make_pair(lv, n_envs, auto_reset=2, max_episode_steps=11, seed=94, max_fused_steps=16, lanes_per_scene=16)
+    act = scenes.make_actions(32, n_envs, env.n_actions, 94)
+    for lo in (0, 16):
+        r, d, o = env.step_obs(torch.from_numpy(act[lo:lo + 16]).cuda())
+        rr, dr = ref.step(act[lo:lo + 16], n_threads=os.cpu_count() or 1)
+        assert np.array_equal(r.cpu().numpy(), rr) and np.array_equal(d.cpu().numpy(), dr)
+        assert np.array_equal(o.cpu().numpy().view(np.uint32), ref.obs().view(np.uint32))
+    err, exact = parity.errors(env, ref)
+    assert exact, err
