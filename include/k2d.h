@@ -276,6 +276,9 @@ int k2d_is_checked_build(void);
 int k2d_resident_groups(const k2d_state *s);
 int k2d_lanes_per_scene(const k2d_state *s);
 int k2d_step_launches(const k2d_state *s, int32_t n_steps);
+/* Test aid: the work items ((run of 8 steps, env) pairs) that one ticket of a launch's work queue stands for: the scene
+ * groups of the warps that step in lockstep (10 for L scenes on a full device). */
+int k2d_items_per_ticket(const k2d_state *s);
 
 /* Measurement aid.  In a library compiled with -DK2D_PHASE_CLOCKS the step kernel adds up, per phase of an environment
  * step (Algorithm 1's stages as this library cuts them), the SM cycles that every scene group spends in it.  The call waits

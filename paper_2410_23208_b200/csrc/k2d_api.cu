@@ -97,6 +97,8 @@ struct k2d_state {
     unsigned char *dev_base;
     unsigned long long *dev_counters;
     unsigned int *dev_queue, *dev_chunks, *dev_sort;
+    int block_threads;   // threads per block of the step kernel for this handle
+    bool large_block;    // one block per SM, warps in lockstep per scheduler (enough envs to fill the device)
     int order_age;       // launches since the envs were last sorted for the work queue (0: the order is not valid)
     int *dev_ids;
     uint32_t *dev_env, *dev_scratch, *dev_levels;
@@ -267,17 +269,31 @@ static int pack_level(const k2d_config *cfg, const ClassInfo &ci, const k2d_leve
 
 template <class SC, int G>
 static cudaError_t launch_step(const k2d_state *s, const StepParams &prm) {
-    k2d_step_kernel<SC, G><<<s->grid, kBlockThreads, s->smem_bytes, s->stream>>>(prm);
+    constexpr int LARGE = step_block_threads<SC, G>();
+    if (s->large_block) k2d_step_kernel<SC, G, LARGE><<<s->grid, LARGE, s->smem_bytes, s->stream>>>(prm);
+    else k2d_step_kernel<SC, G, kSmallBlock><<<s->grid, kSmallBlock, s->smem_bytes, s->stream>>>(prm);
     return cudaGetLastError();
 }
+// Launch shape of the step kernel for this handle.  With enough envs to give every scene group of the device one, the kernel
+// runs as one block per SM whose warps step in lockstep per scheduler; with fewer, as small blocks spread over all SMs.
 template <class SC, int G>
 static cudaError_t setup_step(k2d_state *s, int num_sms) {
-    constexpr int GPB = kBlockThreads / G;
-    s->smem_bytes = sizeof(uint32_t) * (SC::PTAB_WORDS + GPB * region_words<SC, G>());
-    cudaError_t err = cudaFuncSetAttribute(k2d_step_kernel<SC, G>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)s->smem_bytes);
-    if (err != cudaSuccess) return err;
+    constexpr int LARGE = step_block_threads<SC, G>();
+    s->large_block = LARGE > kSmallBlock && s->cfg.n_envs >= num_sms * (LARGE / G) && s->slots >= num_sms * (LARGE / G);
+    const int threads = s->large_block ? LARGE : kSmallBlock, GPB = threads / G;
+    s->block_threads = threads;
+    s->smem_bytes = step_block_smem<SC, G>(threads);
+    cudaError_t err;
     int per_sm = 0;
-    err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k2d_step_kernel<SC, G>, kBlockThreads, s->smem_bytes);
+    if (s->large_block) {
+        err = cudaFuncSetAttribute(k2d_step_kernel<SC, G, LARGE>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)s->smem_bytes);
+        if (err != cudaSuccess) return err;
+        err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k2d_step_kernel<SC, G, LARGE>, threads, s->smem_bytes);
+    } else {
+        err = cudaFuncSetAttribute(k2d_step_kernel<SC, G, kSmallBlock>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)s->smem_bytes);
+        if (err != cudaSuccess) return err;
+        err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k2d_step_kernel<SC, G, kSmallBlock>, threads, s->smem_bytes);
+    }
     if (err != cudaSuccess) return err;
     if (per_sm < 1) per_sm = 1;
     int grid = num_sms * per_sm;
@@ -349,7 +365,8 @@ static cudaError_t launch_order(const k2d_state *s) {
     k2d_order_place_kernel<SC><<<grid, kOrderThreads, 0, s->stream>>>(s->dev_env, s->dev_levels, s->dev_sort, s->dev_ids, n, s->cfg.n_levels);
     return cudaGetLastError();
 }
-static bool uses_order(const k2d_state *s) { return s->G < 32 && s->cfg.n_envs > s->groups; }
+// with one scene per warp and small blocks nothing runs in lockstep, and with no more envs than groups every group gets one env anyway
+static bool uses_order(const k2d_state *s) { return (s->G < 32 || s->large_block) && s->cfg.n_envs > s->groups; }
 // a short launch reuses the order of an earlier one (what an env's step costs changes slowly) and sorts again every
 // kOrderShortLaunches launches; k2d_reset, which uses the same words, makes the next launch sort
 static bool reuses_order(const k2d_state *s, int n_steps) {
@@ -691,6 +708,7 @@ int k2d_is_checked_build(void) {
 
 int k2d_resident_groups(const k2d_state *s) { return s ? s->groups : 0; }
 int k2d_lanes_per_scene(const k2d_state *s) { return s ? s->G : 0; }
+int k2d_items_per_ticket(const k2d_state *s) { return s ? (s->block_threads / 128) * (32 / s->G) : 0; }
 int k2d_step_launches(const k2d_state *s, int32_t n_steps) {
     if (!s) return 0;
     return (uses_order(s) && !reuses_order(s, n_steps)) ? 3 : 1;

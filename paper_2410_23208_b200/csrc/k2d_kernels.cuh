@@ -22,14 +22,11 @@
 
 namespace k2d {
 
-#ifndef K2D_BLOCK_THREADS
-#define K2D_BLOCK_THREADS 128
-#endif
-constexpr int kBlockThreads = K2D_BLOCK_THREADS;
-#ifndef K2D_MIN_BLOCKS
-#define K2D_MIN_BLOCKS 5
-#endif
-constexpr int kMinBlocks = K2D_MIN_BLOCKS;   // resident blocks per SM the step kernel is compiled for (bounds its registers)
+// The step kernel runs in blocks of kSmallBlock threads (several blocks per SM, for launches that do not fill the device) or in
+// one block per SM of up to kLargeBlock threads (see step_block_threads), in which the warps that share a scheduler step in
+// lockstep.  kStepRegisters bounds the kernel's registers: 65536 / 96 = 682 threads per SM.
+constexpr int kSmallBlock = 128, kSmallBlocksPerSM = 5, kLargeBlock = 640;
+constexpr size_t kMaxBlockSmem = 227 * 1024;
 constexpr int kObsThreads = 128;   // observation kernel: one half-warp per env, eight envs per block
 constexpr int kMaxActions = 16;
 enum { Q_TICKET = 0, Q_LEFT = 1, Q_ERROR = 2 };
@@ -124,6 +121,19 @@ template <class SC, int G>
 __host__ __device__ constexpr int region_words() {
     constexpr int raw = SC::STG + SC::LANE_FIELDS * G + kRecWords * (G / 2);
     return G < 32 ? (raw - G + 31) / 32 * 32 + G : (raw + 3) / 4 * 4;
+}
+
+// shared memory of a step-kernel block of `threads` threads, and the threads of the one-block-per-SM form: the largest
+// multiple of 128 up to kLargeBlock whose scenes fit into an SM's shared memory
+template <class SC, int G>
+__host__ __device__ constexpr size_t step_block_smem(int threads) {
+    return sizeof(uint32_t) * (size_t)(SC::PTAB_WORDS + (threads / G) * region_words<SC, G>());
+}
+template <class SC, int G>
+__host__ __device__ constexpr int step_block_threads() {
+    int t = kLargeBlock;
+    while (t > kSmallBlock && step_block_smem<SC, G>(t) + 1024 > kMaxBlockSmem) t -= 128;
+    return t;
 }
 
 // body flag word
@@ -1782,9 +1792,16 @@ struct Scene {
     // ---- whole launch for one scene
     // steps s0 .. s1-1 of env e.  The state record may have been written by another SM earlier in this
     // launch, so it is read past the (non-coherent) L1.
-    __device__ __forceinline__ void run(int e, int s0, int s1) {
+    // e_in < 0: this group has no env in the current batch.  n_sync: the steps every group of the batch goes through; after
+    // each of them the warps that share a scheduler meet at the named barrier `bar` (BAR_THREADS threads; none when a warp is
+    // alone on its barrier), so that they run the same phase of a step at about the same time and share its instructions.
+    template <int BAR_THREADS>
+    __device__ __forceinline__ void run(int e_in, int s0, int s1, int n_sync, int bar) {
+        const bool has = e_in >= 0;
+        const int e = has ? e_in : 0;
         uint32_t *st = prm.state + (size_t)e * SC::ST_WORDS;
         K2D_PHASE_BEGIN();
+        if (has) {
         // everything the state record holds for this lane is asked for in one go (the warm list entries are read a little
         // past the count, inside the record, and dropped below), then the level's constants in a second go
         constexpr int KB = (6 * SC::N + G - 1) / G;
@@ -1830,14 +1847,23 @@ struct Scene {
             widx()[ck_idx<CK_PAIR>((int)p, SC::NPAIRS)] = (uint8_t)(G + lane);
         }
         if (nwarm > G + G / 2) warm_in<SC, G>(sm, ovf, st + SC::ST_WARM, nwarm);
+        }
         g.sync();
         K2D_PHASE(PH_LOAD);
 #pragma unroll 1
-        for (int s = s0; s < s1; ++s) {
-            step(e, s);
+        for (int k = 0; k < n_sync; ++k) {
+            const int s = s0 + k;
+            if (has && s < s1) {
+                step(e, s);
+                if ((k & 255) == 255) flush();
+            }
             g.sync();
-            if (((s - s0) & 255) == 255) flush();
+            if (BAR_THREADS > 32) {
+                __syncwarp();
+                asm volatile("barrier.sync %0, %1;" :: "r"(bar), "r"(BAR_THREADS) : "memory");
+            }
         }
+        if (!has) return;
         K2D_PHASE_RESTART();
         // write back
         for (int i = lane; i < 6 * SC::N; i += G) st[SC::ST_BODY + i] = smu[body_word<SC>(i)];
@@ -1935,42 +1961,50 @@ __device__ __forceinline__ uint16_t pair_code(int p) {
     return (uint16_t)(a | (b << 8));
 }
 
-template <class SC, int G>
-__global__ void __launch_bounds__(kBlockThreads, kMinBlocks) k2d_step_kernel(const StepParams prm) {
+// THREADS: kSmallBlock (several blocks per SM) or step_block_threads<SC, G>() (one block per SM).
+template <class SC, int G, int THREADS>
+__global__ void __launch_bounds__(THREADS, THREADS == kSmallBlock ? kSmallBlocksPerSM : 1) k2d_step_kernel(const StepParams prm) {
     extern __shared__ __align__(16) uint32_t smem_raw[];
-    constexpr int GPB = kBlockThreads / G;
+    constexpr int GPB = THREADS / G;
     uint16_t *ptab = reinterpret_cast<uint16_t *>(smem_raw);
-    for (int p = threadIdx.x; p < SC::NPAIRS; p += kBlockThreads) ptab[p] = pair_code<SC>(p);
+    for (int p = threadIdx.x; p < SC::NPAIRS; p += THREADS) ptab[p] = pair_code<SC>(p);
     __syncthreads();
     const int gib = threadIdx.x / G;
     const int slot = blockIdx.x * GPB + gib, nslots = gridDim.x * GPB;
     uint32_t *region = smem_raw + SC::PTAB_WORDS + gib * region_words<SC, G>();
     uint32_t *scratch = prm.scratch + (size_t)ck_idx<CK_SLOT>(slot, prm.n_slots) * SC::SCRATCH_WORDS;
     Scene<SC, G> scene(region, ptab, scratch, prm);
-    // Work items are (chunk, env), handed out in that order by one ticket counter: a group that is done
-    // takes the next item, so groups with cheap scenes take more of them.  Chunk c of an env may start
-    // only when its chunk c - 1 is stepped and its state is back in memory (another group may have done
-    // it); with items handed out chunk by chunk that is almost always long past, else the group waits for
-    // the group that holds it, which is running.
     const Group<G> &g = scene.g;
-    // A group's first item is its own number, so that a launch does not start with every group drawing a ticket from the
-    // same word; the counter hands out the items after those.
-    // First items go round the blocks warp by warp (the scenes of a warp next to one another in the launch's order, the
-    // warps of a block far apart), so that every SM starts with a mix of cheap and costly envs.
+    // Work items are (chunk, env), numbered in that order and dealt out in batches of kBatch consecutive ones to the warps of
+    // the block that share a scheduler (warp number mod 4: WPS warps, kBatch scene groups), which step their scenes in
+    // lockstep, a named barrier after every step: the warps of a scheduler then run the same phase of a step at about the
+    // same time and fetch its instructions once.  With the envs sorted by cost the scenes of a batch are alike, so the
+    // barriers wait little.  First batches go round the SMs (no ticket, and every SM starts with a mix of cheap and costly
+    // envs); after that a leader draws the next batch number for its scheduler group from one ticket counter, so groups with
+    // cheap scenes take more batches.  Chunk c of an env may start only when its chunk c - 1 is stepped and its state is
+    // back in memory (another scheduler group may have done it); with batches handed out in order that is almost always
+    // long past, else the group waits, with a limit, for the group that holds it, which is running.  Every thread of a
+    // scheduler group goes through the same number of barriers: the batch number is the same for all of them, a batch takes
+    // chunk_steps steps whether a group has an env in it or not, and a wait that runs out only turns the group's env off.
+    constexpr int GPW = 32 / G, WPS = THREADS / 128, kBatch = WPS * GPW, BAR_THREADS = 32 * WPS;
+    __shared__ unsigned int s_batch[4];
+    const int warp = threadIdx.x >> 5, sub = warp & 3, bar = 1 + sub;
+    const int member = (warp >> 2) * GPW + gib % GPW;
     const unsigned items = (unsigned)prm.n_envs * (unsigned)prm.n_chunks;
-    constexpr int GPW = 32 / G;
-    unsigned t = (unsigned)(GPW * ((gib / GPW) * (int)gridDim.x + (int)blockIdx.x) + gib % GPW);
+    const unsigned n_item_batches = (items + kBatch - 1) / kBatch, n_sched = gridDim.x * 4u;
+    unsigned batch = (unsigned)sub * gridDim.x + blockIdx.x;
 #pragma unroll 1
-    for (bool first = true;; first = false) {
-        if (!first) {
-            if (g.lane == 0) t = (unsigned)nslots + atomicAdd(prm.queue + Q_TICKET, 1u);
-            t = g.shflu(t, 0);
+    for (;;) {
+        if (batch >= n_item_batches) break;
+        const unsigned t = batch * kBatch + member;
+        int e = -1, c = 0;
+        if (t < items) {
+            c = (int)(t / (unsigned)prm.n_envs);
+            const int idx = (int)(t - (unsigned)c * (unsigned)prm.n_envs);
+            e = prm.order ? ck_idx<CK_COUNT>(__ldg(prm.order + idx), prm.n_envs) : idx;
         }
-        if (t >= items) break;
-        const int c = (int)(t / (unsigned)prm.n_envs), idx = (int)(t - (unsigned)c * (unsigned)prm.n_envs);
-        const int e = prm.order ? ck_idx<CK_COUNT>(__ldg(prm.order + idx), prm.n_envs) : idx;
         bool ok = true;
-        if (c > 0) {
+        if (e >= 0 && c > 0) {
             if (g.lane == 0) {
                 const volatile unsigned int *flag = prm.chunks_done + e;
                 const volatile unsigned int *err = prm.queue + Q_ERROR;
@@ -1983,18 +2017,23 @@ __global__ void __launch_bounds__(kBlockThreads, kMinBlocks) k2d_step_kernel(con
             ok = g.shfl(ok ? 1 : 0, 0) != 0;
             __threadfence();
         }
-        if (ok) {
-            const int s0 = c * prm.chunk_steps;
-            scene.run(e, s0, min(prm.n_steps, s0 + prm.chunk_steps));
-            // the group's work counters go to the global ones every 64 steps or more (16-bit fields; a step adds at most
-            // one manifold per slot, 186, and a run flushes every 256 steps by itself: (63 + 256) x 186 < 65536)
-            if ((scene.c_man >> 16) >= 64u) scene.flush();
-        }
-        if (prm.n_chunks > 1) {
+        const int s0 = c * prm.chunk_steps;
+        scene.template run<BAR_THREADS>(ok ? e : -1, s0, min(prm.n_steps, s0 + prm.chunk_steps), prm.chunk_steps, bar);
+        // the group's work counters go to the global ones every 64 steps or more (16-bit fields; a step adds at most
+        // one manifold per slot, 186, and a run flushes every 256 steps by itself: (63 + 256) x 186 < 65536)
+        if ((scene.c_man >> 16) >= 64u) scene.flush();
+        if (e >= 0 && prm.n_chunks > 1) {
             __threadfence();      // this lane's part of the state record is visible before the count moves
             g.sync();
             if (g.lane == 0) atomicExch(prm.chunks_done + e, (c + 1 == prm.n_chunks) ? 0u : (unsigned)(c + 1));
         }
+        // the next batch of this scheduler group
+        if (warp < 4 && (threadIdx.x & 31) == 0) s_batch[sub] = n_sched + atomicAdd(prm.queue + Q_TICKET, 1u);
+        if (BAR_THREADS > 32) { __syncwarp(); asm volatile("barrier.sync %0, %1;" :: "r"(bar), "r"(BAR_THREADS) : "memory"); }
+        else __syncwarp();
+        batch = s_batch[sub];
+        if (BAR_THREADS > 32) { __syncwarp(); asm volatile("barrier.sync %0, %1;" :: "r"(bar), "r"(BAR_THREADS) : "memory"); }
+        else __syncwarp();
     }
     scene.flush();
     // the last group to leave rewinds the queue for the next launch

@@ -20,7 +20,7 @@ EXPORTS = (
     "k2d_default_config", "k2d_state_bytes", "k2d_state_bytes_no_scratch", "k2d_level_pool_bytes", "k2d_create", "k2d_reset", "k2d_step",
     "k2d_step_discrete", "k2d_step_static_scratch", "k2d_step_obs", "k2d_obs", "k2d_render",
     "k2d_obs_floats", "k2d_canonical_words", "k2d_get_state", "k2d_set_state", "k2d_status", "k2d_level_info",
-    "k2d_set_trace", "k2d_trace_slots", "k2d_is_checked_build", "k2d_phase_cycles", "k2d_resident_groups", "k2d_lanes_per_scene", "k2d_step_launches", "k2d_set_wait_limit", "k2d_eval_sincos_tanh", "k2d_measure_fp32_peak", "k2d_error_string", "k2d_destroy",
+    "k2d_set_trace", "k2d_trace_slots", "k2d_is_checked_build", "k2d_phase_cycles", "k2d_resident_groups", "k2d_lanes_per_scene", "k2d_step_launches", "k2d_items_per_ticket", "k2d_set_wait_limit", "k2d_eval_sincos_tanh", "k2d_measure_fp32_peak", "k2d_error_string", "k2d_destroy",
 )
 
 
@@ -94,6 +94,7 @@ def load_library(checked: bool = False, phase_clocks: bool = False):
         lib.k2d_resident_groups.argtypes = [vp]
         lib.k2d_lanes_per_scene.argtypes = [vp]
         lib.k2d_step_launches.argtypes = [vp, i32]
+        lib.k2d_items_per_ticket.argtypes = [vp]
         lib.k2d_eval_sincos_tanh.argtypes = [vp, i32, vp, vp, vp, vp]
         lib.k2d_measure_fp32_peak.argtypes = [i32, vp, C.c_size_t, vp]
         lib.k2d_error_string.argtypes = [C.c_int]
@@ -287,6 +288,11 @@ class Env:
     @property
     def lanes_per_scene(self) -> int:
         return int(self.lib.k2d_lanes_per_scene(self._h))
+
+    @property
+    def items_per_ticket(self) -> int:
+        """test aid: work items one ticket of the launch's work queue stands for"""
+        return int(self.lib.k2d_items_per_ticket(self._h))
 
     def step_launches(self, n_steps: int) -> int:
         """kernel launches the next step call of n_steps steps makes (the step kernel, and the two that sort the envs when it does)"""

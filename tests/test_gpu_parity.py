@@ -484,10 +484,10 @@ def test_status_reports_a_wait_that_ran_out_and_reset_clears_it():
 
 
 def test_a_wait_that_runs_out_ends_the_launch_and_is_reported():
-    # With more envs than resident scene groups a launch of 16 steps is two runs of 8 steps per env, handed out in the order
-    # (run, env): every group starts with the item of its own number, a ticket counter hands out the rest.  Here the counter
-    # is moved on by n_envs from the host, so the first runs of the last envs are skipped and only their second runs are
-    # handed out; each waits for a first run that nobody does.  The wait is bounded (64 polls of about 100 ns here): the first
+    # With more envs than resident scene groups a launch of 16 steps is two runs of 8 steps per env, numbered in the order
+    # (run, env) and handed out in batches: every scheduler group of warps starts with the batch of its own number, a ticket
+    # counter hands out the rest.  Here the counter is moved on by one run's worth of batches from the host, so the first
+    # runs of the last envs are skipped and only their second runs are handed out; each waits for a first run that nobody does.  The wait is bounded (64 polls of about 100 ns here): the first
     # group to run out records the error, every other wait ends at once, the kernel returns, k2d_status reports it and
     # k2d_reset clears it.  Nothing hangs and nothing faults.
     import torch
@@ -497,7 +497,8 @@ def test_a_wait_that_runs_out_ends_the_launch_and_is_reported():
     env.set_wait_limit(1)                                     # raised to the floor of 64 polls
     act = torch.zeros((16, n_envs, env.n_actions), device="cuda")
     before = env.get_state()
-    env.state_buf[128:144].view(torch.int32)[0] = n_envs      # work-queue words follow the eight counters: ticket, left, error
+    # work-queue words follow the eight counters: ticket, left, error
+    env.state_buf[128:144].view(torch.int32)[0] = -(-n_envs // env.items_per_ticket)
     torch.cuda.synchronize()
     env.step(act)
     torch.cuda.synchronize()
