@@ -484,7 +484,10 @@ int k2d_create(const k2d_config *cfg, void *dev_state_buf, void *dev_level_pool_
     if (err == cudaSuccess) err = cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, cfg->device);
     // default lanes per scene: a warp per scene while the device has warps to spare (measured on B200: faster below
     // about 48 envs per SM for the largest size class, 24 for the smaller ones), two scenes per warp beyond
-    if (err == cudaSuccess && !cfg->lanes_per_scene) s->G = (cfg->n_envs < (ci.id == 2 ? 48 : 24) * num_sms) ? 32 : 16;
+    // default lanes per scene: two scenes per warp once they fill the device's one-block-per-SM form (40 scenes per SM) with
+    // some to spare, one scene per warp below that (measured, env-steps/s with 16 against 32 lanes: L x 8192 132.8 M / 107.2 M,
+    // L x 6144 99.1 M / 103.3 M, L x 4096 70.3 M / 97.9 M, M x 4096 112.8 M / 143.3 M, S x 4096 147.7 M / 164.9 M)
+    if (err == cudaSuccess && !cfg->lanes_per_scene) s->G = (cfg->n_envs < (kLargeBlock / 16) * num_sms * 9 / 8) ? 32 : 16;
     if (err == cudaSuccess) err = K2D_DISPATCH(setup_step, s, s, num_sms);
     if (err == cudaSuccess) err = cudaMemcpyAsync(s->dev_levels, s->host_levels.data(), s->host_levels.size() * 4, cudaMemcpyHostToDevice, s->stream);
     if (err == cudaSuccess) err = cudaStreamSynchronize(s->stream);
