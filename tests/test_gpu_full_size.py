@@ -183,3 +183,15 @@ def test_discrete_actions_and_the_fused_observation_through_the_sorted_work_queu
         assert np.array_equal(o.cpu().numpy().view(np.uint32), ref.obs().view(np.uint32))
     err, exact = parity.errors(env, ref)
     assert exact, err
+
+
+@pytest.mark.parametrize("size,n_envs,lanes", [("L", 7200, 8), ("L", 3200, 32), ("M", 7200, 8), ("M", 3200, 32)])
+def test_one_block_per_sm_form_with_8_and_32_lanes_per_scene(size, n_envs, lanes):
+    # enough envs to fill every scene group of the device at these lane counts, so the step kernel runs as one block per SM
+    # whose warps step in lockstep per scheduler (three warps per scheduler for L scenes at 8 lanes, five otherwise)
+    index = 3 if size == "L" else 2
+    env, ref, seed = _workload_pair(index, n_envs, 24, lanes_per_scene=lanes, auto_reset=2, max_episode_steps=10)
+    assert env.resident_groups <= n_envs and env.items_per_ticket > 32 // lanes      # several warps per ticket: the one-block form
+    act = scenes.make_actions(40, n_envs, env.n_actions, seed)
+    d = _run_and_compare(env, ref, act, 20)               # work items of 8, 8 and 4 steps
+    assert d.sum() >= 2 * n_envs
