@@ -269,8 +269,8 @@ int k2d_trace_slots(const k2d_state *s);
 int k2d_is_checked_build(void);
 
 /* Host-side facts about a handle's launches.  k2d_resident_groups: scenes the device steps at once for this handle (with
- * more envs than that a launch goes through a work queue and first sorts the envs by what their steps cost, in two small
- * launches of its own; launches of fewer than 8 steps reuse that order 16 times).  k2d_lanes_per_scene: 8, 16 or 32.
+ * more envs than that a launch goes through a work queue, and from one and a half times as many on it first sorts the envs
+ * by what their steps cost, in two small launches of its own; launches of fewer than 8 steps reuse that order 16 times).  k2d_lanes_per_scene: 8, 16 or 32.
  * k2d_step_launches: kernel launches that the next k2d_step, k2d_step_discrete or k2d_step_obs call with n_steps steps
  * makes (1 or 3; k2d_step_obs one more for scenes whose observation does not fit beside the scene in shared memory). */
 int k2d_resident_groups(const k2d_state *s);

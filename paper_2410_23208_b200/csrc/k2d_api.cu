@@ -366,7 +366,12 @@ static cudaError_t launch_order(const k2d_state *s) {
     return cudaGetLastError();
 }
 // with one scene per warp and small blocks nothing runs in lockstep, and with no more envs than groups every group gets one env anyway
-static bool uses_order(const k2d_state *s) { return (s->G < 32 || s->large_block) && s->cfg.n_envs > s->groups; }
+static bool uses_order(const k2d_state *s) {
+    // one block per SM: from one and a half waves of envs on (measured on L scenes, sorted against unsorted env-steps/s:
+    // 7400 envs 114.6 M / 123.6 M, 8192 132.1 M / 135.8 M, 9000 140.3 M / 137.6 M, 12000 152.9 M / 141.9 M, 16384 158.3 M / 146.8 M)
+    if (s->large_block) return 2 * (long long)s->cfg.n_envs > 3 * (long long)s->groups;
+    return s->G < 32 && s->cfg.n_envs > s->groups;
+}
 // a short launch reuses the order of an earlier one (what an env's step costs changes slowly) and sorts again every
 // kOrderShortLaunches launches; k2d_reset, which uses the same words, makes the next launch sort
 static bool reuses_order(const k2d_state *s, int n_steps) {

@@ -139,10 +139,10 @@ def test_workload_4_large_scenes_131072_envs_fused_steps_and_observation():
 
 
 def test_short_launches_through_the_work_queue_reuse_and_renew_the_order_of_the_envs():
-    # more envs than the device holds scene groups, one or two steps per launch: the launch hands the envs out in an order
+    # one and a half times as many envs as the device holds scene groups (so that launches sort them), one or two steps per launch: the launch hands the envs out in an order
     # sorted by cost that it keeps for 16 launches; a reset with level ids (which uses the same words) makes the next launch
     # sort again.  Whatever the order, every env is stepped once per step.
-    n_envs = 6400
+    n_envs = 9000
     lv = scenes.make_levels("L", 128, 91, static_prob=0.1)
     env, ref = parity.make_pair(lv, n_envs, auto_reset=2, max_episode_steps=12, seed=91, max_fused_steps=8, lanes_per_scene=16)
     act = scenes.make_actions(40, n_envs, env.n_actions, 91)
@@ -164,7 +164,7 @@ def test_discrete_actions_and_the_fused_observation_through_the_sorted_work_queu
     import torch
     from oracle import k2d_ref
     from paper_2410_23208_b200 import k2d
-    n_envs = 6400
+    n_envs = 9000
     lv = scenes.make_levels("L", 128, 93, static_prob=0.1)
     env = k2d.Env(lv, n_envs, auto_reset=2, max_episode_steps=11, seed=93, max_fused_steps=16, lanes_per_scene=16)
     ref = k2d_ref.RefSim(lv, n_envs, auto_reset=2, max_episode_steps=11, seed=93, broadphase=0, discrete_actions=1)
